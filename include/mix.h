@@ -1,0 +1,218 @@
+/*
+ * mix.h -- C ABI of the per-layer MI hook for NVIDIA B200 (sm_100a).
+ *
+ * One call, mix_apply(), applies every registered MI function to the hidden states
+ * bf16[T, d] of a continuously batched, ragged set of requests at one hook.  A device-side
+ * token->slot map routes each token row to its request's function:
+ *
+ *   MIX_PROBE  read primitive  (paper, Section 3 "Read"; Section 4.2 "Executable units"):
+ *              z_c = b_c + sum_i W[c,i] h[t,i];  score = sigmoid(z) | softmax(z) | z,
+ *              written to the caller's score buffer (Section 4.2 "State and dataflow");
+ *              the hidden row is not modified.
+ *   MIX_STEER  write primitive (Section 3 "Write": add or subtract a vector):
+ *              h[t,:] <- bf16( h[t,:] + alpha * v ), in place.
+ *   MIX_SAE    sparse-autoencoder function (the paper names feature dictionaries only;
+ *              the arithmetic is the standard one): z = W_enc h + b_enc, activation
+ *              ReLU | JumpReLU (z > theta) | TopK (k largest pre-activations, then ReLU),
+ *              per-feature edits (clamp: f_j = c; ablate: f_j = 0), decode from W_dec,
+ *              optionally with the reconstruction error of the UNEDITED features added
+ *              back:  h' = xhat(f') + (h - xhat(f)).
+ *   slot -1    no app: the row is neither read nor written (Section 4.2 "Toggling
+ *              semantics": an inactive app costs a request nothing).
+ *
+ * Rows are independent.  Activation of an app for a request is data (the slot map and the
+ * small device tables), never launch structure: mix_apply() only enqueues kernels with a
+ * launch geometry fixed at mix_create(), performs no allocation, no host<->device
+ * synchronisation and no host read of device state, so it may be captured once in a CUDA
+ * graph at T_max rows and replayed while apps are toggled by the stream-ordered
+ * mix_set_* / mix_register_* / mix_update_* calls (Section 4.2 "CUDA-graph-safe kernel
+ * design", "Graph-level toggling and continuous batching").
+ *
+ * Conventions
+ *   - every function returns MIX_OK (0) or a negative mix_status; nothing throws, aborts
+ *     or prints.  mix_last_error() gives a message for the last failure on that context.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - "device" pointers are CUDA device pointers on the context's GPU; "host" pointers are
+ *     ordinary host memory.  bf16 tensors are row-major, densely packed.
+ *   - weights are BORROWED: the caller keeps them alive and unchanged until the app /
+ *     weight set is unregistered (or the context destroyed) and work already enqueued has
+ *     finished.  Everything else (tables, edit lists, slot map) is copied.
+ *   - one host thread per context at a time.
+ */
+#ifndef MIX_H_
+#define MIX_H_
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mix_ctx mix_ctx;
+
+typedef enum {
+  MIX_OK = 0,
+  MIX_ERR_INVALID_ARG = -1,   /* NULL pointer, bad enum, misaligned pointer */
+  MIX_ERR_OUT_OF_RANGE = -2,  /* an index or size exceeds what mix_create() was told */
+  MIX_ERR_UNSUPPORTED = -3,   /* shape not supported by the kernels (see mix_create) */
+  MIX_ERR_NO_MEMORY = -4,     /* device allocation failed in mix_create() */
+  MIX_ERR_CUDA = -5           /* a CUDA call failed; see mix_last_error() */
+} mix_status;
+
+enum { MIX_PROBE = 1, MIX_STEER = 2, MIX_SAE = 3 };                    /* app kinds */
+enum { MIX_ACT_SIGMOID = 0, MIX_ACT_SOFTMAX = 1, MIX_ACT_NONE = 2 };   /* probe activations */
+enum { MIX_SAE_RELU = 0, MIX_SAE_JUMPRELU = 1, MIX_SAE_TOPK = 2 };     /* SAE activations */
+enum { MIX_EDIT_CLAMP = 0, MIX_EDIT_ABLATE = 1 };                      /* per-feature edits */
+
+/* bits of the device status word (mix_get_status) */
+enum {
+  MIX_STATUS_BAD_SLOT = 1u << 0,      /* a live row named a slot id < -1, >= n_slots_max or unregistered; treated as -1 */
+  MIX_STATUS_BAD_GROUP = 1u << 1,     /* an SAE app names a weight set that is not registered; rows pass through */
+  MIX_STATUS_WAIT_TIMEOUT = 1u << 2,  /* a bounded wait inside the encode kernel expired; results of that call are invalid */
+  MIX_STATUS_TOPK_GENERAL = 1u << 3   /* informational: a row's TopK needed the general (many-ties) selection path */
+};
+
+/* flags for mix_config.flags */
+enum {
+  MIX_FLAG_ENCODE_SIMT = 1u << 0      /* run the SAE encode on the plain CUDA-core kernel instead of tcgen05 (cross-check) */
+};
+
+typedef struct {
+  int d_model;          /* hidden width d; multiple of 64 (16-byte vectors, 128-byte TMA rows) */
+  int T_max;            /* rows of every `hidden` passed to mix_apply (the capture size) */
+  int n_slots_max;      /* app slots 0 .. n_slots_max-1 */
+  int n_groups_max;     /* SAE weight sets 0 .. n_groups_max-1; 0 = no SAE kernels are ever launched */
+  int C_max;            /* row stride of scores_out and largest n_classes (<= 64) */
+  int k_max;            /* largest TopK k (<= 1024); also the row stride of the feature outputs */
+  int r_max;            /* largest edit list per SAE app (<= 64) */
+  long long d_sae_max;  /* largest SAE width; multiple of 256 */
+  unsigned flags;       /* MIX_FLAG_* */
+} mix_config;
+
+/* Read primitive.  W: device bf16 [n_classes, d].  b: device fp32 [n_classes] or NULL (= 0).
+   act = MIX_ACT_SIGMOID requires n_classes == 1. */
+typedef struct {
+  int n_classes;
+  int act;
+  const void* W;
+  const float* b;
+} mix_probe;
+
+/* Write primitive.  v: device bf16 [d]; used as given (not normalised); alpha any sign. */
+typedef struct {
+  const void* v;
+  float alpha;
+} mix_steer;
+
+/* One SAE weight set, shared by any number of app slots.  All pointers device.
+   W_enc bf16 [d_sae, d]: row j = encoder direction j.  b_enc fp32 [d_sae].
+   theta fp32 [d_sae] (JumpReLU only, else NULL).  W_dec bf16 [d_sae, d]: row j = decoder
+   direction j.  b_dec fp32 [d] or NULL.  center_input != 0 subtracts b_dec from the input
+   before the encoder (folded into an effective bias at registration; needs b_dec).
+   k: TopK only, 1 <= k <= min(k_max, d_sae). */
+typedef struct {
+  long long d_sae;
+  int act;
+  int k;
+  const void* W_enc;
+  const float* b_enc;
+  const float* theta;
+  const void* W_dec;
+  const float* b_dec;
+  int center_input;
+} mix_sae_weights;
+
+/* One SAE app slot = (weight set, edit list, error-term flag).  idx/val/mode are HOST arrays
+   of n_edit entries, copied; if an index occurs twice the later entry wins.  add_error != 0:
+   h' = xhat(f') + (h - xhat(f)) (a row with no effective edit is left untouched, bit for
+   bit); add_error == 0: h' = xhat(f'). */
+typedef struct {
+  int group;
+  int n_edit;
+  const int* idx;
+  const float* val;
+  const unsigned char* mode;
+  int add_error;
+} mix_sae_app;
+
+/* Create a context on the CURRENT CUDA device and allocate every table and workspace the
+   hook will ever need (the only allocating call besides registration of a centred SAE).
+   Workspace: a bf16 panel of (T_max + 128*n_groups_max) x d and an fp32 pre-activation
+   scratch of the same rows x d_sae_max, when n_groups_max > 0.
+   Errors: INVALID_ARG (NULL, non-positive sizes), UNSUPPORTED (d_model % 64, d_sae_max % 256,
+   C_max > 64, k_max > 1024, r_max > 64), NO_MEMORY, CUDA. */
+int mix_create(mix_ctx** out, const mix_config* cfg);
+
+/* Free everything the context owns.  Synchronises the device.  NULL is a no-op. */
+int mix_destroy(mix_ctx* ctx);
+
+/* Message for the last error on this context (static storage, valid until the next call). */
+const char* mix_last_error(const mix_ctx* ctx);
+
+/* Register / replace SAE weight set `group` (stream-ordered table write).  Not captured.
+   Errors: OUT_OF_RANGE (group, d_sae > d_sae_max, k), UNSUPPORTED (d_sae % 256), INVALID_ARG
+   (NULL or pointers not 16-byte aligned, JumpReLU without theta, centring without b_dec). */
+int mix_register_sae_weights(mix_ctx* ctx, int group, const mix_sae_weights* w, void* stream);
+int mix_unregister_sae_weights(mix_ctx* ctx, int group, void* stream);
+
+/* Attach an MI function to `slot` (paper, Section 4.2: functions are attached ahead of time
+   with their parameters).  `desc` points to a mix_probe, mix_steer or mix_sae_app according
+   to `kind`.  Stream-ordered; an entry becomes visible atomically (its valid flag is
+   written last).  Errors: OUT_OF_RANGE (slot, n_classes > C_max, n_edit > r_max, edit
+   index >= d_sae of the group, group), INVALID_ARG. */
+int mix_register_app(mix_ctx* ctx, int slot, int kind, const void* desc, void* stream);
+
+/* Make `slot` pass-through again.  Rows still naming it are left untouched and raise
+   MIX_STATUS_BAD_SLOT. */
+int mix_unregister_app(mix_ctx* ctx, int slot, void* stream);
+
+/* Cheap toggles that never touch launch structure (Section 4.2 "Toggling semantics"). */
+int mix_update_steer_alpha(mix_ctx* ctx, int slot, float alpha, void* stream);
+int mix_update_sae_edits(mix_ctx* ctx, int slot, int n_edit, const int* idx, const float* val,
+                         const unsigned char* mode, void* stream);
+
+/* Install the token->slot map for the next mix_apply calls: token_slot int32[T_live]
+   (host if src_is_device == 0, else device), -1 = no app.  Rows >= T_live are pass-through.
+   One async copy + a 4-byte store into fixed device buffers; never captured in a graph.
+   A host source must stay valid until the stream reaches the copy (use pinned memory for a
+   truly asynchronous copy).  Errors: OUT_OF_RANGE (T_live < 0 or > T_max). */
+int mix_set_slot_map(mix_ctx* ctx, const int* token_slot, int T_live, int src_is_device, void* stream);
+
+/* Two-level form: slot of token t = req_slot[token_req[t]] (token_req < 0 or >= n_req -> -1),
+   composed on the device.  Both arrays host or both device. */
+int mix_set_request_map(mix_ctx* ctx, const int* token_req, int T_live, const int* req_slot, int n_req,
+                        int src_is_device, void* stream);
+
+/* Optional feature read-out (device buffers, NULL = off): topk_idx int32 [T_max, k_max] and
+   topk_val fp32 [T_max, k_max] receive, for every TopK-SAE row, the selected feature ids
+   in order of decreasing pre-activation (ties: lower id first) and those pre-activations
+   (before ReLU and before edits); entries k..k_max-1 and other rows are not written.
+   n_active int32 [T_max] receives, for every SAE row, the number of features with f_j > 0
+   before edits.  Takes effect for later mix_apply calls; a captured graph keeps the
+   pointers it was captured with. */
+int mix_set_feature_out(mix_ctx* ctx, int* topk_idx, float* topk_val, int* n_active);
+
+/* Apply the hook.  hidden: device bf16 [T_max, d], modified in place.  T: number of rows of
+   `hidden` that may be live (<= T_max; rows >= min(T, T_live) are pass-through).  scores_out:
+   device fp32 [T_max, C_max] or NULL; only the first n_classes entries of probe rows are
+   written.  Enqueues kernels on `stream` and returns; safe to capture.  Device-side
+   problems (bad slot ids, ...) are reported through the status word, never by faulting.
+   Errors: INVALID_ARG (NULL hidden, misaligned), OUT_OF_RANGE (T), CUDA (launch failure). */
+int mix_apply(mix_ctx* ctx, void* hidden, int T, float* scores_out, void* stream);
+
+/* Copy the device status word (bits MIX_STATUS_*) to *bits and clear it on the device.
+   Synchronises `stream`. */
+int mix_get_status(mix_ctx* ctx, unsigned* bits, void* stream);
+
+/* Number of kernels one mix_apply() call launches on this context (fixed at mix_create). */
+int mix_launches_per_apply(const mix_ctx* ctx);
+
+/* Test / profiling taps into the SAE workspace after a mix_apply (device pointers owned by
+   the context; valid until mix_destroy):  panel_rows int32 [n_panel_rows] gives the token
+   index of each packed panel row (-1 = padding), z the fp32 pre-activations
+   [n_panel_rows, ld_z].  Any out pointer may be NULL. */
+int mix_debug_workspace(mix_ctx* ctx, const int** panel_rows, const float** z, long long* ld_z,
+                        int* n_panel_rows);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MIX_H_ */

@@ -1,0 +1,237 @@
+"""Thin ctypes binding of libmix.so: argument marshalling only.
+
+Every step of the hook runs in the CUDA kernels behind the C ABI (include/mix.h); this
+module turns torch tensors into device pointers and checks return codes.  There is no CPU
+fallback: if the library is missing or cannot be loaded, importing callers fail loudly.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+from . import _build
+
+MIX_PROBE, MIX_STEER, MIX_SAE = 1, 2, 3
+MIX_ACT_SIGMOID, MIX_ACT_SOFTMAX, MIX_ACT_NONE = 0, 1, 2
+MIX_SAE_RELU, MIX_SAE_JUMPRELU, MIX_SAE_TOPK = 0, 1, 2
+MIX_EDIT_CLAMP, MIX_EDIT_ABLATE = 0, 1
+MIX_STATUS_BAD_SLOT, MIX_STATUS_BAD_GROUP, MIX_STATUS_WAIT_TIMEOUT, MIX_STATUS_TOPK_GENERAL = 1, 2, 4, 8
+MIX_FLAG_ENCODE_SIMT = 1
+
+EXPORTS = [
+    "mix_create", "mix_destroy", "mix_last_error", "mix_register_sae_weights", "mix_unregister_sae_weights",
+    "mix_register_app", "mix_unregister_app", "mix_update_steer_alpha", "mix_update_sae_edits",
+    "mix_set_slot_map", "mix_set_request_map", "mix_set_feature_out", "mix_apply", "mix_get_status",
+    "mix_launches_per_apply", "mix_debug_workspace",
+]
+
+
+class MixConfig(C.Structure):
+    _fields_ = [("d_model", C.c_int), ("T_max", C.c_int), ("n_slots_max", C.c_int), ("n_groups_max", C.c_int),
+                ("C_max", C.c_int), ("k_max", C.c_int), ("r_max", C.c_int), ("d_sae_max", C.c_longlong),
+                ("flags", C.c_uint)]
+
+
+class MixProbe(C.Structure):
+    _fields_ = [("n_classes", C.c_int), ("act", C.c_int), ("W", C.c_void_p), ("b", C.c_void_p)]
+
+
+class MixSteer(C.Structure):
+    _fields_ = [("v", C.c_void_p), ("alpha", C.c_float)]
+
+
+class MixSaeWeights(C.Structure):
+    _fields_ = [("d_sae", C.c_longlong), ("act", C.c_int), ("k", C.c_int), ("W_enc", C.c_void_p),
+                ("b_enc", C.c_void_p), ("theta", C.c_void_p), ("W_dec", C.c_void_p), ("b_dec", C.c_void_p),
+                ("center_input", C.c_int)]
+
+
+class MixSaeApp(C.Structure):
+    _fields_ = [("group", C.c_int), ("n_edit", C.c_int), ("idx", C.c_void_p), ("val", C.c_void_p),
+                ("mode", C.c_void_p), ("add_error", C.c_int)]
+
+
+class MixError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__("mix error %d: %s" % (code, msg))
+        self.code = code
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None) -> C.CDLL:
+    """Load libmix.so (built in-tree).  Raises if it is absent: there is no other path."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    path = path or _build.LIB_PATH
+    if not os.path.exists(path):
+        raise RuntimeError("libmix.so not found at %s; run __graft_entry__.build() first" % path)
+    lib = C.CDLL(path)
+    vp, ci = C.c_void_p, C.c_int
+    lib.mix_create.argtypes = [C.POINTER(vp), C.POINTER(MixConfig)]
+    lib.mix_destroy.argtypes = [vp]
+    lib.mix_last_error.argtypes = [vp]
+    lib.mix_last_error.restype = C.c_char_p
+    lib.mix_register_sae_weights.argtypes = [vp, ci, C.POINTER(MixSaeWeights), vp]
+    lib.mix_unregister_sae_weights.argtypes = [vp, ci, vp]
+    lib.mix_register_app.argtypes = [vp, ci, ci, vp, vp]
+    lib.mix_unregister_app.argtypes = [vp, ci, vp]
+    lib.mix_update_steer_alpha.argtypes = [vp, ci, C.c_float, vp]
+    lib.mix_update_sae_edits.argtypes = [vp, ci, ci, vp, vp, vp, vp]
+    lib.mix_set_slot_map.argtypes = [vp, vp, ci, ci, vp]
+    lib.mix_set_request_map.argtypes = [vp, vp, ci, vp, ci, ci, vp]
+    lib.mix_set_feature_out.argtypes = [vp, vp, vp, vp]
+    lib.mix_apply.argtypes = [vp, vp, ci, vp, vp]
+    lib.mix_get_status.argtypes = [vp, C.POINTER(C.c_uint), vp]
+    lib.mix_launches_per_apply.argtypes = [vp]
+    lib.mix_debug_workspace.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(C.c_longlong), C.POINTER(ci)]
+    for name in EXPORTS:
+        if name != "mix_last_error":
+            getattr(lib, name).restype = ci
+    if path == _build.LIB_PATH:
+        _lib = lib
+    return lib
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    h = stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+    return h or None
+
+
+class Mix:
+    """One hook context on the current CUDA device (same names as the C ABI)."""
+
+    def __init__(self, d_model, T_max, n_slots_max, n_groups_max=0, C_max=1, k_max=0, r_max=0, d_sae_max=0,
+                 flags=0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("mix needs a CUDA device (sm_100a); there is no CPU path")
+        self.lib = load_library()
+        self.cfg = MixConfig(d_model, T_max, n_slots_max, n_groups_max, C_max, k_max, r_max, d_sae_max, flags)
+        self.ctx = C.c_void_p()
+        rc = self.lib.mix_create(C.byref(self.ctx), C.byref(self.cfg))
+        if rc != 0:
+            raise MixError(rc, "mix_create failed")
+        self._keep = {}          # borrowed weights must outlive their registration
+
+    def _check(self, rc):
+        if rc != 0:
+            raise MixError(rc, self.lib.mix_last_error(self.ctx).decode())
+
+    def destroy(self):
+        if self.ctx:
+            self.lib.mix_destroy(self.ctx)
+            self.ctx = C.c_void_p()
+            self._keep.clear()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def register_sae_weights(self, group, d_sae, act, k, W_enc, b_enc, W_dec, theta=None, b_dec=None,
+                             center_input=False, stream=None):
+        w = MixSaeWeights(int(d_sae), int(act), int(k), _ptr(W_enc), _ptr(b_enc), _ptr(theta), _ptr(W_dec),
+                          _ptr(b_dec), int(bool(center_input)))
+        self._check(self.lib.mix_register_sae_weights(self.ctx, group, C.byref(w), _stream(stream)))
+        self._keep[("g", group)] = (W_enc, b_enc, W_dec, theta, b_dec)
+
+    def unregister_sae_weights(self, group, stream=None):
+        self._check(self.lib.mix_unregister_sae_weights(self.ctx, group, _stream(stream)))
+
+    def register_probe(self, slot, W, b, act, stream=None):
+        d = MixProbe(int(W.shape[0]), int(act), _ptr(W), _ptr(b))
+        self._check(self.lib.mix_register_app(self.ctx, slot, MIX_PROBE, C.byref(d), _stream(stream)))
+        self._keep[("a", slot)] = (W, b)
+
+    def register_steer(self, slot, v, alpha, stream=None):
+        d = MixSteer(_ptr(v), float(alpha))
+        self._check(self.lib.mix_register_app(self.ctx, slot, MIX_STEER, C.byref(d), _stream(stream)))
+        self._keep[("a", slot)] = (v,)
+
+    @staticmethod
+    def _edit_arrays(idx, val, mode):
+        idx = np.ascontiguousarray(idx, dtype=np.int32)
+        val = np.ascontiguousarray(val, dtype=np.float32)
+        mode = np.ascontiguousarray(mode, dtype=np.uint8)
+        assert len(idx) == len(val) == len(mode)
+        return idx, val, mode
+
+    def register_sae_app(self, slot, group, idx, val, mode, add_error, stream=None):
+        idx, val, mode = self._edit_arrays(idx, val, mode)
+        d = MixSaeApp(int(group), len(idx), idx.ctypes.data, val.ctypes.data, mode.ctypes.data, int(bool(add_error)))
+        self._check(self.lib.mix_register_app(self.ctx, slot, MIX_SAE, C.byref(d), _stream(stream)))
+
+    def unregister_app(self, slot, stream=None):
+        self._check(self.lib.mix_unregister_app(self.ctx, slot, _stream(stream)))
+        self._keep.pop(("a", slot), None)
+
+    def update_steer_alpha(self, slot, alpha, stream=None):
+        self._check(self.lib.mix_update_steer_alpha(self.ctx, slot, float(alpha), _stream(stream)))
+
+    def update_sae_edits(self, slot, idx, val, mode, stream=None):
+        idx, val, mode = self._edit_arrays(idx, val, mode)
+        self._check(self.lib.mix_update_sae_edits(self.ctx, slot, len(idx), idx.ctypes.data, val.ctypes.data,
+                                                  mode.ctypes.data, _stream(stream)))
+
+    def set_slot_map(self, token_slot, T_live=None, stream=None):
+        """token_slot: int32 torch tensor (CUDA, or CPU -- pinned for an async copy) or numpy array."""
+        if isinstance(token_slot, np.ndarray):
+            token_slot = np.ascontiguousarray(token_slot, dtype=np.int32)
+            n = len(token_slot) if T_live is None else T_live
+            self._check(self.lib.mix_set_slot_map(self.ctx, token_slot.ctypes.data, n, 0, _stream(stream)))
+            return
+        assert token_slot.dtype == torch.int32 and token_slot.is_contiguous()
+        n = token_slot.numel() if T_live is None else T_live
+        self._check(self.lib.mix_set_slot_map(self.ctx, token_slot.data_ptr(), n, int(token_slot.is_cuda),
+                                              _stream(stream)))
+
+    def set_request_map(self, token_req, req_slot, T_live=None, stream=None):
+        if isinstance(token_req, np.ndarray):
+            token_req = np.ascontiguousarray(token_req, dtype=np.int32)
+            req_slot = np.ascontiguousarray(req_slot, dtype=np.int32)
+            n = len(token_req) if T_live is None else T_live
+            self._check(self.lib.mix_set_request_map(self.ctx, token_req.ctypes.data, n, req_slot.ctypes.data,
+                                                     len(req_slot), 0, _stream(stream)))
+            return
+        n = token_req.numel() if T_live is None else T_live
+        self._check(self.lib.mix_set_request_map(self.ctx, token_req.data_ptr(), n, req_slot.data_ptr(),
+                                                 req_slot.numel(), int(token_req.is_cuda), _stream(stream)))
+
+    def set_feature_out(self, topk_idx=None, topk_val=None, n_active=None):
+        self._check(self.lib.mix_set_feature_out(self.ctx, _ptr(topk_idx), _ptr(topk_val), _ptr(n_active)))
+        self._keep["fo"] = (topk_idx, topk_val, n_active)
+
+    def apply(self, hidden, scores_out=None, T=None, stream=None):
+        assert hidden.dtype == torch.bfloat16 and hidden.is_cuda and hidden.is_contiguous()
+        T = hidden.shape[0] if T is None else T
+        self._check(self.lib.mix_apply(self.ctx, hidden.data_ptr(), int(T), _ptr(scores_out), _stream(stream)))
+
+    def get_status(self, stream=None) -> int:
+        bits = C.c_uint(0)
+        self._check(self.lib.mix_get_status(self.ctx, C.byref(bits), _stream(stream)))
+        return int(bits.value)
+
+    def launches_per_apply(self) -> int:
+        return int(self.lib.mix_launches_per_apply(self.ctx))
+
+    def debug_workspace(self):
+        pr, z, ld, n = C.c_void_p(), C.c_void_p(), C.c_longlong(), C.c_int()
+        self._check(self.lib.mix_debug_workspace(self.ctx, C.byref(pr), C.byref(z), C.byref(ld), C.byref(n)))
+        return pr.value, z.value, ld.value, n.value

@@ -1,0 +1,419 @@
+// Host side of the C ABI declared in mix.h: context, device tables, registration, and the
+// fixed launch sequence of mix_apply().
+#include <cudaTypedefs.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include "mix_internal.h"
+
+using namespace mix;
+
+struct mix_ctx : public Ctx {};
+
+namespace {
+
+#define MIX_FAIL(ctx, code, ...)                          \
+  do {                                                    \
+    snprintf((ctx)->err, sizeof((ctx)->err), __VA_ARGS__); \
+    return (code);                                        \
+  } while (0)
+
+#define MIX_CUDA(ctx, expr)                                                                  \
+  do {                                                                                       \
+    cudaError_t e_ = (expr);                                                                 \
+    if (e_ != cudaSuccess) MIX_FAIL(ctx, MIX_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e_)); \
+  } while (0)
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
+
+int load_encode_fn() {
+  if (g_encode) return MIX_OK;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+      qres != cudaDriverEntryPointSuccess)
+    return MIX_ERR_CUDA;
+  g_encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+  return MIX_OK;
+}
+
+// bf16 [rows, d] row-major; box = kTileK columns x box_rows rows; 128-byte swizzle.
+int make_tmap(CUtensorMap* out, const void* base, unsigned long long rows, int d, int box_rows) {
+  cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)d * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = g_encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? MIX_OK : MIX_ERR_CUDA;
+}
+
+template <typename T>
+cudaError_t dev_alloc(T** p, size_t n) {
+  *p = nullptr;
+  if (n == 0) return cudaSuccess;
+  return cudaMalloc(reinterpret_cast<void**>(p), n * sizeof(T));
+}
+
+void free_all(mix_ctx* c) {
+  cudaFree(c->d_token_slot); cudaFree(c->d_n_live); cudaFree(c->d_apps); cudaFree(c->d_groups);
+  cudaFree(c->d_edit_idx); cudaFree(c->d_edit_val); cudaFree(c->d_edit_mode); cudaFree(c->d_status);
+  cudaFree(c->d_tmp_req); cudaFree(c->d_tmp_req_slot); cudaFree(c->d_panel); cudaFree(c->d_panel_row);
+  cudaFree(c->d_mtile_group); cudaFree(c->d_route); cudaFree(c->d_z); cudaFree(c->d_topk_idx);
+  cudaFree(c->d_topk_val); cudaFree(c->d_tmap_w);
+  if (c->owned_b_eff)
+    for (int g = 0; g < c->cfg.n_groups_max; ++g) cudaFree(c->owned_b_eff[g]);
+  free(c->owned_b_eff); free(c->h_apps); free(c->h_groups);
+}
+
+int check_slot(mix_ctx* c, int slot) {
+  if (slot < 0 || slot >= c->cfg.n_slots_max) MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "slot %d outside [0, %d)", slot, c->cfg.n_slots_max);
+  return MIX_OK;
+}
+
+// Publish an app entry: body first with valid = 0, then the valid word.
+int publish_app(mix_ctx* c, int slot, cudaStream_t s) {
+  AppEntry tmp = c->h_apps[slot];
+  const int valid = tmp.valid;
+  tmp.valid = 0;
+  MIX_CUDA(c, cudaMemcpyAsync(c->d_apps + slot, &tmp, sizeof(AppEntry), cudaMemcpyHostToDevice, s));
+  if (valid) MIX_CUDA(c, cudaMemcpyAsync(&c->d_apps[slot].valid, &valid, sizeof(int), cudaMemcpyHostToDevice, s));
+  return MIX_OK;
+}
+
+int upload_edits(mix_ctx* c, int slot, int group, int n_edit, const int* idx, const float* val,
+                 const unsigned char* mode, cudaStream_t s) {
+  if (n_edit < 0 || n_edit > c->cfg.r_max) MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "n_edit %d outside [0, r_max=%d]", n_edit, c->cfg.r_max);
+  if (n_edit > 0 && (!idx || !val || !mode)) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "edit arrays are NULL");
+  const long long S = c->h_groups[group].d_sae;
+  for (int e = 0; e < n_edit; ++e) {
+    if (idx[e] < 0 || idx[e] >= S) MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "edit %d: feature %d outside [0, %lld)", e, idx[e], S);
+    if (mode[e] != MIX_EDIT_CLAMP && mode[e] != MIX_EDIT_ABLATE) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "edit %d: bad mode %d", e, mode[e]);
+  }
+  if (n_edit > 0) {
+    const size_t off = (size_t)slot * c->cfg.r_max;
+    MIX_CUDA(c, cudaMemcpyAsync(c->d_edit_idx + off, idx, n_edit * sizeof(int), cudaMemcpyHostToDevice, s));
+    MIX_CUDA(c, cudaMemcpyAsync(c->d_edit_val + off, val, n_edit * sizeof(float), cudaMemcpyHostToDevice, s));
+    MIX_CUDA(c, cudaMemcpyAsync(c->d_edit_mode + off, mode, n_edit, cudaMemcpyHostToDevice, s));
+  }
+  return MIX_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int mix_create(mix_ctx** out, const mix_config* cfg) {
+  if (!out || !cfg) return MIX_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (cfg->d_model <= 0 || cfg->T_max <= 0 || cfg->n_slots_max <= 0 || cfg->n_groups_max < 0 || cfg->C_max <= 0 ||
+      cfg->k_max < 0 || cfg->r_max < 0 || cfg->d_sae_max < 0)
+    return MIX_ERR_INVALID_ARG;
+  if (cfg->d_model % 64 || cfg->d_model > 8192 || cfg->C_max > kMaxClasses || cfg->k_max > kMaxK ||
+      cfg->r_max > kMaxEdits || cfg->n_groups_max > kMaxGroups || cfg->d_sae_max % kTileN ||
+      cfg->d_sae_max > 0x7fffffffll || (cfg->n_groups_max > 0 && cfg->d_sae_max == 0))
+    return MIX_ERR_UNSUPPORTED;
+  {  // the routing kernel keeps (T_max / 32) x n_groups counters in static-size shared memory
+    const long long chunks = (cfg->T_max + 1023) / 1024;
+    if (chunks * 32 * cfg->n_groups_max * 4 > 40 * 1024) return MIX_ERR_UNSUPPORTED;
+  }
+  mix_ctx* c = static_cast<mix_ctx*>(calloc(1, sizeof(mix_ctx)));
+  if (!c) return MIX_ERR_NO_MEMORY;
+  c->cfg = *cfg;
+  if (c->cfg.r_max == 0) c->cfg.r_max = 1;      // keeps table strides non-zero
+  if (c->cfg.k_max == 0) c->cfg.k_max = 1;
+  cudaError_t e = cudaGetDevice(&c->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, c->device);
+  if (e != cudaSuccess) { free(c); return MIX_ERR_CUDA; }
+  const int G = cfg->n_groups_max, NS = cfg->n_slots_max, T = cfg->T_max;
+  c->h_apps = static_cast<AppEntry*>(calloc(NS, sizeof(AppEntry)));
+  c->h_groups = static_cast<GroupEntry*>(calloc(G > 0 ? G : 1, sizeof(GroupEntry)));
+  c->owned_b_eff = static_cast<float**>(calloc(G > 0 ? G : 1, sizeof(float*)));
+  if (!c->h_apps || !c->h_groups || !c->owned_b_eff) { free_all(c); free(c); return MIX_ERR_NO_MEMORY; }
+  bool ok = true;
+  ok = ok && dev_alloc(&c->d_token_slot, T) == cudaSuccess;
+  ok = ok && dev_alloc(&c->d_n_live, 1) == cudaSuccess;
+  ok = ok && dev_alloc(&c->d_apps, NS) == cudaSuccess;
+  ok = ok && dev_alloc(&c->d_groups, G > 0 ? G : 1) == cudaSuccess;
+  ok = ok && dev_alloc(&c->d_edit_idx, (size_t)NS * c->cfg.r_max) == cudaSuccess;
+  ok = ok && dev_alloc(&c->d_edit_val, (size_t)NS * c->cfg.r_max) == cudaSuccess;
+  ok = ok && dev_alloc(&c->d_edit_mode, (size_t)NS * c->cfg.r_max) == cudaSuccess;
+  ok = ok && dev_alloc(&c->d_status, 1) == cudaSuccess;
+  ok = ok && dev_alloc(&c->d_tmp_req, T) == cudaSuccess;
+  ok = ok && dev_alloc(&c->d_tmp_req_slot, T) == cudaSuccess;
+  if (ok && G > 0) {
+    c->panel_rows_cap = ((T + kTileM - 1) / kTileM + G) * kTileM;
+    const size_t P = c->panel_rows_cap;
+    ok = ok && dev_alloc(&c->d_panel, P * cfg->d_model) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_panel_row, P) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_mtile_group, P / kTileM) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_route, 1) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_z, P * (size_t)cfg->d_sae_max) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_topk_idx, P * (size_t)c->cfg.k_max) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_topk_val, P * (size_t)c->cfg.k_max) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_tmap_w, G) == cudaSuccess;
+  }
+  if (!ok) { cudaGetLastError(); free_all(c); free(c); return MIX_ERR_NO_MEMORY; }
+  e = cudaMemset(c->d_token_slot, 0xff, T * sizeof(int));
+  if (e == cudaSuccess) e = cudaMemset(c->d_n_live, 0, sizeof(int));
+  if (e == cudaSuccess) e = cudaMemset(c->d_apps, 0, NS * sizeof(AppEntry));
+  if (e == cudaSuccess) e = cudaMemset(c->d_groups, 0, (G > 0 ? G : 1) * sizeof(GroupEntry));
+  if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, sizeof(unsigned));
+  if (e == cudaSuccess && G > 0) {
+    e = cudaMemset(c->d_panel, 0, (size_t)c->panel_rows_cap * cfg->d_model * sizeof(__nv_bfloat16));
+    if (e == cudaSuccess) e = cudaMemset(c->d_route, 0, sizeof(RouteState));
+    if (e == cudaSuccess) e = cudaMemset(c->d_panel_row, 0xff, c->panel_rows_cap * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(c->d_mtile_group, 0xff, c->panel_rows_cap / kTileM * sizeof(int));
+    if (e == cudaSuccess && !(cfg->flags & MIX_FLAG_ENCODE_SIMT)) {
+      if (load_encode_fn() != MIX_OK ||
+          make_tmap(&c->tmap_panel, c->d_panel, c->panel_rows_cap, cfg->d_model, kTileM) != MIX_OK)
+        e = cudaErrorUnknown;
+      if (e == cudaSuccess) e = encode_tc_prepare();
+    }
+  }
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) { free_all(c); free(c); return MIX_ERR_CUDA; }
+  c->err[0] = 0;
+  *out = c;
+  return MIX_OK;
+}
+
+int mix_destroy(mix_ctx* c) {
+  if (!c) return MIX_OK;
+  cudaDeviceSynchronize();
+  free_all(c);
+  free(c);
+  return MIX_OK;
+}
+
+const char* mix_last_error(const mix_ctx* c) { return c ? c->err : "null context"; }
+
+int mix_register_sae_weights(mix_ctx* c, int group, const mix_sae_weights* w, void* stream) {
+  if (!c) return MIX_ERR_INVALID_ARG;
+  if (!w) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "weights are NULL");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (group < 0 || group >= c->cfg.n_groups_max) MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "group %d outside [0, %d)", group, c->cfg.n_groups_max);
+  if (w->d_sae <= 0 || w->d_sae > c->cfg.d_sae_max) MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "d_sae %lld outside (0, %lld]", w->d_sae, c->cfg.d_sae_max);
+  if (w->d_sae % kTileN) MIX_FAIL(c, MIX_ERR_UNSUPPORTED, "d_sae %lld is not a multiple of %d", w->d_sae, kTileN);
+  if (w->act != MIX_SAE_RELU && w->act != MIX_SAE_JUMPRELU && w->act != MIX_SAE_TOPK) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "bad SAE activation %d", w->act);
+  if (!w->W_enc || !w->b_enc || !w->W_dec) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "W_enc, b_enc and W_dec are required");
+  if (!aligned16(w->W_enc) || !aligned16(w->W_dec) || !aligned16(w->b_enc) || (w->b_dec && !aligned16(w->b_dec)))
+    MIX_FAIL(c, MIX_ERR_INVALID_ARG, "weight pointers must be 16-byte aligned");
+  if (w->act == MIX_SAE_JUMPRELU && !w->theta) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "JumpReLU needs theta");
+  if (w->act == MIX_SAE_TOPK && (w->k < 1 || w->k > c->cfg.k_max || w->k > w->d_sae))
+    MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "k %d outside [1, min(k_max=%d, d_sae)]", w->k, c->cfg.k_max);
+  if (w->center_input && !w->b_dec) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "center_input needs b_dec");
+
+  GroupEntry ge;
+  memset(&ge, 0, sizeof(ge));
+  ge.valid = 1;
+  ge.act = w->act;
+  ge.k = w->act == MIX_SAE_TOPK ? w->k : 0;
+  ge.d_sae = w->d_sae;
+  ge.W_enc = static_cast<const __nv_bfloat16*>(w->W_enc);
+  ge.b_eff = w->b_enc;
+  ge.theta = w->theta;
+  ge.W_dec = static_cast<const __nv_bfloat16*>(w->W_dec);
+  ge.b_dec = w->b_dec;
+  if (w->center_input) {
+    // z = W_enc (h - b_dec) + b_enc = W_enc h + (b_enc - W_enc b_dec): fold once, here
+    if (c->owned_b_eff[group]) { cudaStreamSynchronize(s); cudaFree(c->owned_b_eff[group]); c->owned_b_eff[group] = nullptr; }
+    if (cudaMalloc(reinterpret_cast<void**>(&c->owned_b_eff[group]), w->d_sae * sizeof(float)) != cudaSuccess) {
+      cudaGetLastError();
+      MIX_FAIL(c, MIX_ERR_NO_MEMORY, "cannot allocate the folded bias");
+    }
+    MIX_CUDA(c, launch_fold_bias(ge.W_enc, w->b_enc, w->b_dec, c->owned_b_eff[group], w->d_sae, c->cfg.d_model, s));
+    ge.b_eff = c->owned_b_eff[group];
+  }
+  if (!(c->cfg.flags & MIX_FLAG_ENCODE_SIMT)) {
+    CUtensorMap tm;
+    if (make_tmap(&tm, w->W_enc, (unsigned long long)w->d_sae, c->cfg.d_model, kTileN) != MIX_OK)
+      MIX_FAIL(c, MIX_ERR_CUDA, "cuTensorMapEncodeTiled failed for W_enc");
+    MIX_CUDA(c, cudaMemcpyAsync(c->d_tmap_w + group, &tm, sizeof(tm), cudaMemcpyHostToDevice, s));
+  }
+  c->h_groups[group] = ge;
+  GroupEntry tmp = ge;
+  tmp.valid = 0;
+  MIX_CUDA(c, cudaMemcpyAsync(c->d_groups + group, &tmp, sizeof(tmp), cudaMemcpyHostToDevice, s));
+  const int one = 1;
+  MIX_CUDA(c, cudaMemcpyAsync(&c->d_groups[group].valid, &one, sizeof(int), cudaMemcpyHostToDevice, s));
+  return MIX_OK;
+}
+
+int mix_unregister_sae_weights(mix_ctx* c, int group, void* stream) {
+  if (!c) return MIX_ERR_INVALID_ARG;
+  if (group < 0 || group >= c->cfg.n_groups_max) MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "group %d outside [0, %d)", group, c->cfg.n_groups_max);
+  c->h_groups[group].valid = 0;
+  const int zero = 0;
+  MIX_CUDA(c, cudaMemcpyAsync(&c->d_groups[group].valid, &zero, sizeof(int), cudaMemcpyHostToDevice,
+                              static_cast<cudaStream_t>(stream)));
+  return MIX_OK;
+}
+
+int mix_register_app(mix_ctx* c, int slot, int kind, const void* desc, void* stream) {
+  if (!c) return MIX_ERR_INVALID_ARG;
+  if (!desc) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "descriptor is NULL");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc = check_slot(c, slot);
+  if (rc != MIX_OK) return rc;
+  AppEntry e;
+  memset(&e, 0, sizeof(e));
+  e.valid = 1;
+  e.kind = kind;
+  if (kind == MIX_PROBE) {
+    const mix_probe* p = static_cast<const mix_probe*>(desc);
+    if (p->n_classes < 1 || p->n_classes > c->cfg.C_max) MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "n_classes %d outside [1, C_max=%d]", p->n_classes, c->cfg.C_max);
+    if (p->act != MIX_ACT_SIGMOID && p->act != MIX_ACT_SOFTMAX && p->act != MIX_ACT_NONE) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "bad probe activation %d", p->act);
+    if (p->act == MIX_ACT_SIGMOID && p->n_classes != 1) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "sigmoid probes have one class");
+    if (!p->W || !aligned16(p->W)) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "probe W is NULL or not 16-byte aligned");
+    e.n_classes = p->n_classes;
+    e.act = p->act;
+    e.W = p->W;
+    e.b = p->b;
+  } else if (kind == MIX_STEER) {
+    const mix_steer* p = static_cast<const mix_steer*>(desc);
+    if (!p->v || !aligned16(p->v)) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "steering vector is NULL or not 16-byte aligned");
+    e.W = p->v;
+    e.alpha = p->alpha;
+  } else if (kind == MIX_SAE) {
+    const mix_sae_app* p = static_cast<const mix_sae_app*>(desc);
+    if (p->group < 0 || p->group >= c->cfg.n_groups_max || !c->h_groups[p->group].valid)
+      MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "SAE weight set %d is not registered", p->group);
+    rc = upload_edits(c, slot, p->group, p->n_edit, p->idx, p->val, p->mode, s);
+    if (rc != MIX_OK) return rc;
+    e.group = p->group;
+    e.n_edit = p->n_edit;
+    e.add_error = p->add_error ? 1 : 0;
+  } else {
+    MIX_FAIL(c, MIX_ERR_INVALID_ARG, "bad app kind %d", kind);
+  }
+  c->h_apps[slot] = e;
+  return publish_app(c, slot, s);
+}
+
+int mix_unregister_app(mix_ctx* c, int slot, void* stream) {
+  if (!c) return MIX_ERR_INVALID_ARG;
+  int rc = check_slot(c, slot);
+  if (rc != MIX_OK) return rc;
+  memset(&c->h_apps[slot], 0, sizeof(AppEntry));
+  const int zero = 0;
+  MIX_CUDA(c, cudaMemcpyAsync(&c->d_apps[slot].valid, &zero, sizeof(int), cudaMemcpyHostToDevice,
+                              static_cast<cudaStream_t>(stream)));
+  return MIX_OK;
+}
+
+int mix_update_steer_alpha(mix_ctx* c, int slot, float alpha, void* stream) {
+  if (!c) return MIX_ERR_INVALID_ARG;
+  int rc = check_slot(c, slot);
+  if (rc != MIX_OK) return rc;
+  if (!c->h_apps[slot].valid || c->h_apps[slot].kind != MIX_STEER) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "slot %d is not a steering app", slot);
+  c->h_apps[slot].alpha = alpha;
+  MIX_CUDA(c, cudaMemcpyAsync(&c->d_apps[slot].alpha, &alpha, sizeof(float), cudaMemcpyHostToDevice,
+                              static_cast<cudaStream_t>(stream)));
+  return MIX_OK;
+}
+
+int mix_update_sae_edits(mix_ctx* c, int slot, int n_edit, const int* idx, const float* val,
+                         const unsigned char* mode, void* stream) {
+  if (!c) return MIX_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc = check_slot(c, slot);
+  if (rc != MIX_OK) return rc;
+  if (!c->h_apps[slot].valid || c->h_apps[slot].kind != MIX_SAE) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "slot %d is not an SAE app", slot);
+  // shrink first, grow last, so a concurrent reader never sees a count beyond valid entries
+  const int old_n = c->h_apps[slot].n_edit;
+  if (n_edit < old_n && n_edit >= 0)
+    MIX_CUDA(c, cudaMemcpyAsync(&c->d_apps[slot].n_edit, &n_edit, sizeof(int), cudaMemcpyHostToDevice, s));
+  rc = upload_edits(c, slot, c->h_apps[slot].group, n_edit, idx, val, mode, s);
+  if (rc != MIX_OK) return rc;
+  c->h_apps[slot].n_edit = n_edit;
+  MIX_CUDA(c, cudaMemcpyAsync(&c->d_apps[slot].n_edit, &n_edit, sizeof(int), cudaMemcpyHostToDevice, s));
+  return MIX_OK;
+}
+
+int mix_set_slot_map(mix_ctx* c, const int* token_slot, int T_live, int src_is_device, void* stream) {
+  if (!c) return MIX_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (T_live < 0 || T_live > c->cfg.T_max) MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "T_live %d outside [0, T_max=%d]", T_live, c->cfg.T_max);
+  if (T_live > 0 && !token_slot) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "token_slot is NULL");
+  if (T_live > 0)
+    MIX_CUDA(c, cudaMemcpyAsync(c->d_token_slot, token_slot, (size_t)T_live * sizeof(int),
+                                src_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, s));
+  MIX_CUDA(c, cudaMemcpyAsync(c->d_n_live, &T_live, sizeof(int), cudaMemcpyHostToDevice, s));
+  return MIX_OK;
+}
+
+int mix_set_request_map(mix_ctx* c, const int* token_req, int T_live, const int* req_slot, int n_req,
+                        int src_is_device, void* stream) {
+  if (!c) return MIX_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (T_live < 0 || T_live > c->cfg.T_max) MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "T_live %d outside [0, T_max=%d]", T_live, c->cfg.T_max);
+  if (n_req < 0 || n_req > c->cfg.T_max) MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "n_req %d outside [0, T_max=%d]", n_req, c->cfg.T_max);
+  if (T_live > 0 && (!token_req || (n_req > 0 && !req_slot))) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "map arrays are NULL");
+  const cudaMemcpyKind kind = src_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+  if (T_live > 0) {
+    MIX_CUDA(c, cudaMemcpyAsync(c->d_tmp_req, token_req, (size_t)T_live * sizeof(int), kind, s));
+    if (n_req > 0) MIX_CUDA(c, cudaMemcpyAsync(c->d_tmp_req_slot, req_slot, (size_t)n_req * sizeof(int), kind, s));
+    MIX_CUDA(c, launch_compose_map(c, T_live, n_req, s));
+  }
+  MIX_CUDA(c, cudaMemcpyAsync(c->d_n_live, &T_live, sizeof(int), cudaMemcpyHostToDevice, s));
+  return MIX_OK;
+}
+
+int mix_set_feature_out(mix_ctx* c, int* topk_idx, float* topk_val, int* n_active) {
+  if (!c) return MIX_ERR_INVALID_ARG;
+  c->out_topk_idx = topk_idx;
+  c->out_topk_val = topk_val;
+  c->out_n_active = n_active;
+  return MIX_OK;
+}
+
+int mix_apply(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream) {
+  if (!c) return MIX_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (!hidden || !aligned16(hidden)) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "hidden is NULL or not 16-byte aligned");
+  if (T < 0 || T > c->cfg.T_max) MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "T %d outside [0, T_max=%d]", T, c->cfg.T_max);
+  __nv_bfloat16* h = static_cast<__nv_bfloat16*>(hidden);
+  MIX_CUDA(c, launch_probe_steer(c, h, T, scores_out, s));
+  if (c->cfg.n_groups_max > 0) {
+    MIX_CUDA(c, launch_route(c, T, s));
+    MIX_CUDA(c, launch_pack(c, h, s));
+    if (c->cfg.flags & MIX_FLAG_ENCODE_SIMT)
+      MIX_CUDA(c, launch_encode_simt(c, s));
+    else
+      MIX_CUDA(c, launch_encode_tc(c, s));
+    MIX_CUDA(c, launch_select(c, s));
+    MIX_CUDA(c, launch_decode(c, h, s));
+  }
+  return MIX_OK;
+}
+
+int mix_launches_per_apply(const mix_ctx* c) {
+  if (!c) return 0;
+  return c->cfg.n_groups_max > 0 ? 6 : 1;
+}
+
+int mix_get_status(mix_ctx* c, unsigned* bits, void* stream) {
+  if (!c) return MIX_ERR_INVALID_ARG;
+  if (!bits) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "bits is NULL");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  MIX_CUDA(c, cudaMemcpyAsync(bits, c->d_status, sizeof(unsigned), cudaMemcpyDeviceToHost, s));
+  MIX_CUDA(c, cudaMemsetAsync(c->d_status, 0, sizeof(unsigned), s));
+  MIX_CUDA(c, cudaStreamSynchronize(s));
+  return MIX_OK;
+}
+
+int mix_debug_workspace(mix_ctx* c, const int** panel_rows, const float** z, long long* ld_z, int* n_panel_rows) {
+  if (!c) return MIX_ERR_INVALID_ARG;
+  if (panel_rows) *panel_rows = c->d_panel_row;
+  if (z) *z = c->d_z;
+  if (ld_z) *ld_z = c->cfg.d_sae_max;
+  if (n_panel_rows) *n_panel_rows = c->panel_rows_cap;
+  return MIX_OK;
+}
+
+}  // extern "C"

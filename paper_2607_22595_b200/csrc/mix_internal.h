@@ -1,0 +1,115 @@
+// Internal declarations shared by the translation units of libmix.so.
+// Device tables live at fixed addresses owned by the context; kernels read every piece of
+// dynamic state (slot map, live count, app table, edit lists, route results) from them, so
+// a captured graph never needs its kernel parameters changed.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mix.h"
+
+namespace mix {
+
+constexpr int kTileM = 128;        // token rows per encode tile (UMMA M)
+constexpr int kTileN = 256;        // SAE features per encode tile (UMMA N)
+constexpr int kTileK = 64;         // bf16 elements per 128-byte swizzled smem row
+constexpr int kMaxGroups = 32;
+constexpr int kMaxClasses = 64;
+constexpr int kMaxK = 1024;
+constexpr int kMaxEdits = 64;
+
+struct __align__(16) AppEntry {
+  int valid;          // written last by registration; 0 = slot is pass-through
+  int kind;           // MIX_PROBE | MIX_STEER | MIX_SAE
+  int n_classes;      // probe
+  int act;            // probe
+  float alpha;        // steer
+  int group;          // sae
+  int n_edit;         // sae
+  int add_error;      // sae
+  const void* W;      // probe: bf16 [C, d]; steer: bf16 [d]
+  const float* b;     // probe: fp32 [C] or null
+};
+
+struct __align__(16) GroupEntry {
+  int valid;
+  int act;
+  int k;
+  int pad_;
+  long long d_sae;
+  const __nv_bfloat16* W_enc;
+  const float* b_eff;   // b_enc, or b_enc - W_enc b_dec when the input is centred
+  const float* theta;
+  const __nv_bfloat16* W_dec;
+  const float* b_dec;
+};
+
+// Result of the routing step for the SAE path (one instance in device memory).
+struct RouteState {
+  int n_panel_rows;                 // rows of the packed panel in use (multiple of kTileM)
+  int n_sae_rows;                   // SAE rows routed this call
+  int n_mtiles;                     // = n_panel_rows / kTileM
+  int total_tiles;                  // encode tiles over all groups
+  int group_count[kMaxGroups];      // M_g
+  int group_mtile0[kMaxGroups + 1]; // first m-tile of group g in the panel
+  int group_tile0[kMaxGroups + 1];  // first linear encode tile of group g
+};
+
+struct Ctx {
+  mix_config cfg;
+  int device;
+  int n_sms;
+  char err[256];
+
+  // tables
+  int* d_token_slot;        // [T_max]
+  int* d_n_live;            // [1]
+  AppEntry* d_apps;         // [n_slots_max]
+  GroupEntry* d_groups;     // [n_groups_max]
+  int* d_edit_idx;          // [n_slots_max * r_max]
+  float* d_edit_val;
+  unsigned char* d_edit_mode;
+  unsigned* d_status;
+  int* d_tmp_req;           // [T_max] staging for the two-level map
+  int* d_tmp_req_slot;      // [T_max]
+
+  // host mirrors (validation only)
+  AppEntry* h_apps;
+  GroupEntry* h_groups;
+  float** owned_b_eff;      // per group: library-owned folded bias or null
+
+  // SAE workspace
+  int panel_rows_cap;       // P
+  __nv_bfloat16* d_panel;   // [P, d]
+  int* d_panel_row;         // [P] token index or -1
+  int* d_mtile_group;       // [P / kTileM] group of each m-tile or -1
+  RouteState* d_route;
+  float* d_z;               // [P, d_sae_max]
+  int* d_topk_idx;          // [P, k_max]
+  float* d_topk_val;        // [P, k_max]
+  CUtensorMap* d_tmap_w;    // [n_groups_max] W_enc maps (box kTileK x kTileN, 128B swizzle)
+  CUtensorMap tmap_panel;   // panel map (box kTileK x kTileM, 128B swizzle)
+
+  // optional outputs
+  int* out_topk_idx;
+  float* out_topk_val;
+  int* out_n_active;
+};
+
+// kernel launchers (each returns the CUDA error of the launch)
+cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s);
+cudaError_t launch_route(const Ctx* c, int T, cudaStream_t s);
+cudaError_t launch_pack(const Ctx* c, const __nv_bfloat16* hidden, cudaStream_t s);
+cudaError_t launch_encode_simt(const Ctx* c, cudaStream_t s);
+cudaError_t launch_encode_tc(const Ctx* c, cudaStream_t s);
+cudaError_t launch_select(const Ctx* c, cudaStream_t s);
+cudaError_t launch_decode(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s);
+cudaError_t launch_compose_map(const Ctx* c, int T_live, int n_req, cudaStream_t s);
+cudaError_t launch_fold_bias(const __nv_bfloat16* W_enc, const float* b_enc, const float* b_dec, float* b_eff,
+                             long long d_sae, int d, cudaStream_t s);
+cudaError_t encode_tc_prepare();   // opt in to the large dynamic shared memory size
+
+}  // namespace mix

@@ -1,0 +1,298 @@
+// SAE encode on the 5th-generation tensor cores (sm_100a only).
+//
+//   Z[p, j] = sum_i panel[p, i] * W_enc[j, i] + b_eff[j]        bf16 x bf16 -> fp32
+//
+// One persistent CTA per SM walks a device-built tile schedule (group, feature tile, row tile).
+// Warp roles:  warp 0 = TMA producer (panel tile 128x64 and W_enc tile 256x64 per k-block into
+// a 4-stage ring of 128-byte-swizzled shared memory), warp 1 = MMA issuer (tcgen05.mma
+// 128x256x16, fp32 accumulators in tensor memory, double buffered so the epilogue of one tile
+// overlaps the main loop of the next), warps 2..5 = epilogue (tcgen05.ld, + bias, fp32 store).
+// No TMA multicast and no clusters.  Every wait is bounded: on expiry the CTA raises
+// MIX_STATUS_WAIT_TIMEOUT, lets its copies land, frees its tensor memory and returns.
+#include "mix_internal.h"
+
+namespace mix {
+
+namespace {
+
+constexpr int kStages = 4;
+constexpr int kABytes = kTileM * kTileK * 2;   // 16 KiB
+constexpr int kBBytes = kTileN * kTileK * 2;   // 32 KiB
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kTcThreads = 192;
+constexpr int kTmemCols = 512;                 // two 128 x 256 fp32 accumulators
+constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz
+
+struct __align__(8) TcShared {
+  unsigned long long full[kStages];
+  unsigned long long empty[kStages];
+  unsigned long long tmem_full[2];
+  unsigned long long tmem_empty[2];
+  unsigned tmem_base;
+  volatile int abort_flag;
+  RouteState rs;
+};
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + (int)sizeof(TcShared);
+
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded wait.  Returns false if the wait expired or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, TcShared* sh, unsigned* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  unsigned spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 255u) == 0u) {
+      if (sh->abort_flag) return false;
+      if (clock64() - t0 > kWaitCycles) {
+        sh->abort_flag = 1;
+        atomicOr(status, MIX_STATUS_WAIT_TIMEOUT);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(unsigned dst, const CUtensorMap* map, int x, int y, unsigned bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+
+// K-major operand tile, 128-byte swizzle: rows of 64 bf16 (128 B), 8-row groups 1024 B apart.
+__device__ __forceinline__ unsigned long long umma_desc(unsigned smem_addr) {
+  unsigned long long d = 0;
+  d |= (unsigned long long)((smem_addr & 0x3FFFFu) >> 4);   // start address, 16-byte units
+  d |= (unsigned long long)1 << 16;                         // leading byte offset (unused when swizzled)
+  d |= (unsigned long long)(1024 >> 4) << 32;               // stride byte offset between 8-row groups
+  d |= (unsigned long long)1 << 46;                         // descriptor version (sm_100)
+  d |= (unsigned long long)2 << 61;                         // 128-byte swizzle
+  return d;
+}
+
+// kind::f16 instruction descriptor: D fp32, A and B bf16, both K-major, N = 256, M = 128.
+constexpr unsigned kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(kTileN >> 3) << 17) |
+                            ((unsigned)(kTileM >> 4) << 24);
+
+__device__ __forceinline__ void umma(unsigned d_tmem, unsigned long long a, unsigned long long b, unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a), "l"(b), "r"(kIdesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(unsigned bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(unsigned taddr, float* v) {
+  unsigned* r = reinterpret_cast<unsigned*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+struct Tile {
+  int group, n_tile, m_tile_global, rows_valid;
+};
+
+__device__ __forceinline__ Tile decode_tile(const RouteState& rs, const GroupEntry* groups, int n_groups, int tile) {
+  int g = 0;
+  while (g + 1 < n_groups && tile >= rs.group_tile0[g + 1]) ++g;
+  const int local = tile - rs.group_tile0[g];
+  const int count = rs.group_count[g];
+  const int mt = (count + kTileM - 1) / kTileM;
+  Tile t;
+  t.group = g;
+  t.n_tile = local / mt;
+  const int m_local = local - t.n_tile * mt;
+  t.m_tile_global = rs.group_mtile0[g] + m_local;
+  t.rows_valid = min(kTileM, count - m_local * kTileM);
+  return t;
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorMap* __restrict__ tmap_w,
+                 const RouteState* __restrict__ rs_g, const GroupEntry* __restrict__ groups, int n_groups,
+                 float* __restrict__ Z, long long ldz, int d, unsigned* __restrict__ status) {
+  extern __shared__ unsigned char smem_raw[];
+  // 1024-byte alignment: required by the 128-byte swizzle atoms
+  unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  TcShared* sh = reinterpret_cast<TcShared*>(tiles + kStages * kStageBytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  for (int i = threadIdx.x; i < (int)(sizeof(RouteState) / sizeof(int)); i += kTcThreads)
+    reinterpret_cast<int*>(&sh->rs)[i] = reinterpret_cast<const int*>(rs_g)[i];
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(smem_u32(&sh->full[s]), 1);
+      mbar_init(smem_u32(&sh->empty[s]), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(smem_u32(&sh->tmem_full[a]), 1);
+      mbar_init(smem_u32(&sh->tmem_empty[a]), 4);
+    }
+    sh->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  const int total_tiles = sh->rs.total_tiles;
+  if (total_tiles == 0) return;            // nothing routed to any SAE: no tensor memory is taken
+
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const unsigned tmem_base = sh->tmem_base;
+  const int num_kb = d / kTileK;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      unsigned phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const Tile t = decode_tile(sh->rs, groups, n_groups, tile);
+        const CUtensorMap* tw = tmap_w + t.group;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(smem_u32(&sh->empty[stage]), phase ^ 1u, sh, status)) { ok = false; break; }
+          const unsigned bar = smem_u32(&sh->full[stage]);
+          mbar_expect_tx(bar, kStageBytes);
+          const unsigned sa = smem_u32(tiles + stage * kStageBytes);
+          tma_load_2d(sa, &tmap_panel, kb * kTileK, t.m_tile_global * kTileM, bar);
+          tma_load_2d(sa + kABytes, tw, kb * kTileK, t.n_tile * kTileN, bar);
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      int stage = 0;
+      unsigned phase = 0, acc = 0, acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        if (!mbar_wait(smem_u32(&sh->tmem_empty[acc]), acc_phase ^ 1u, sh, status)) break;
+        tc_fence_after();
+        const unsigned d_tmem = tmem_base + acc * kTileN;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(smem_u32(&sh->full[stage]), phase, sh, status)) { ok = false; break; }
+          tc_fence_after();
+          const unsigned sa = smem_u32(tiles + stage * kStageBytes);
+          const unsigned long long da = umma_desc(sa), db = umma_desc(sa + kABytes);
+#pragma unroll
+          for (int k = 0; k < kTileK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per step
+            umma(d_tmem, da + 2ull * k, db + 2ull * k, (unsigned)((kb | k) != 0));
+          umma_commit(smem_u32(&sh->empty[stage]));
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit(smem_u32(&sh->tmem_full[acc]));
+        acc ^= 1u;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else {
+    const int q = warp & 3;                  // tensor-memory lane quarter this warp may read
+    unsigned acc = 0, acc_phase = 0;
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+      const Tile t = decode_tile(sh->rs, groups, n_groups, tile);
+      // warp-uniform decision: tcgen05.ld below needs the whole warp
+      if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&sh->tmem_full[acc]), acc_phase, sh, status))) break;
+      tc_fence_after();
+      const int row_local = q * 32 + lane;
+      const bool valid = row_local < t.rows_valid;
+      const size_t p = (size_t)t.m_tile_global * kTileM + row_local;
+      const float* bias = groups[t.group].b_eff + (size_t)t.n_tile * kTileN;
+      float* out = Z + p * (size_t)ldz + (size_t)t.n_tile * kTileN;
+#pragma unroll 1
+      for (int c = 0; c < kTileN; c += 32) {
+        float v[32];
+        tmem_ld32(tmem_base + ((unsigned)(q * 32) << 16) + acc * kTileN + c, v);
+        if (valid) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 4) {
+            const float4 b4 = __ldg(reinterpret_cast<const float4*>(bias + c + i));
+            float4 o;
+            o.x = v[i] + b4.x;
+            o.y = v[i + 1] + b4.y;
+            o.z = v[i + 2] + b4.z;
+            o.w = v[i + 3] + b4.w;
+            *reinterpret_cast<float4*>(out + c + i) = o;
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[acc]));
+      acc ^= 1u;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (sh->abort_flag) {
+    // give copies that are still in flight time to land before shared memory is released
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000ll) __nanosleep(1000);
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+}  // namespace
+
+cudaError_t encode_tc_prepare() {
+  return cudaFuncSetAttribute(encode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+}
+
+cudaError_t launch_encode_tc(const Ctx* c, cudaStream_t s) {
+  encode_tc_kernel<<<c->n_sms, kTcThreads, kSmemBytes, s>>>(c->tmap_panel, c->d_tmap_w, c->d_route, c->d_groups,
+                                                             c->cfg.n_groups_max, c->d_z, c->cfg.d_sae_max,
+                                                             c->cfg.d_model, c->d_status);
+  return cudaGetLastError();
+}
+
+}  // namespace mix

@@ -1,0 +1,166 @@
+"""Shared helpers of the GPU parity tests: run the CUDA path through the C ABI, run the
+float64 oracle on the same bits, compare row by row with the stated tolerances."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import workloads as W
+from oracle import mi_hook as O
+
+# Tolerances (from the benchmark spec):
+#   routing, pass-through rows, un-probed score rows : bit-exact
+#   probe scores                                      : |gpu - ref| <= 1e-3 * |ref|
+#   modified hidden (steer, SAE)                      : |gpu - ref| <= 1e-2 * max|h_in|
+#   TopK index sets                                   : equal, except members whose pre-activation is within
+#                                                       1e-3 of the oracle's k-th value may be swapped
+SCORE_RTOL = 1e-3
+HIDDEN_TOL_FRAC = 1e-2
+TOPK_TIE_TOL = 1e-3
+CANARY_F32 = np.uint32(0x7FC0DEAD)          # a NaN payload nobody computes
+CANARY_I32 = np.int32(-559038737)
+
+
+def run_gpu(w, flags=0, graph=False, feature_out=True, hidden=None, mix=None, replays=1):
+    """Apply the hook to workload `w` (tensors on cuda).  Returns numpy outputs."""
+    import os
+    import paper_2607_22595_b200 as mixlib
+    if os.environ.get("MIX_TEST_FORCE_SIMT"):      # debugging aid: route every encode to the cross-check kernel
+        flags |= mixlib.MIX_FLAG_ENCODE_SIMT
+    m = mix or W.make_context(mixlib.Mix, w, flags=flags)
+    T, C = w.T_max, max(w.C_max, 1)
+    h = (w.hidden if hidden is None else hidden).clone()
+    scores = torch.from_numpy(np.full((T, C), CANARY_F32, dtype=np.uint32).view(np.float32)).cuda()
+    k_max = max(w.k_max, 1)
+    tk_idx = torch.full((T, k_max), int(CANARY_I32), dtype=torch.int32, device="cuda")
+    tk_val = torch.from_numpy(np.full((T, k_max), CANARY_F32, dtype=np.uint32).view(np.float32)).cuda()
+    n_act = torch.full((T,), int(CANARY_I32), dtype=torch.int32, device="cuda")
+    if feature_out and w.n_groups_max > 0:
+        m.set_feature_out(tk_idx, tk_val, n_act)
+    if graph:
+        h_static = h.clone()
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s):
+            m.apply(h_static, scores, stream=s)            # warm-up outside capture
+            h_static.copy_(h)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                m.apply(h_static, scores, stream=s)
+        torch.cuda.current_stream().wait_stream(s)
+        for _ in range(replays):
+            h_static.copy_(h)
+            g.replay()
+        torch.cuda.synchronize()
+        h = h_static
+    else:
+        m.apply(h, scores)
+        torch.cuda.synchronize()
+    out = dict(hidden=W.bits(h), scores=scores.cpu().numpy(), topk_idx=tk_idx.cpu().numpy(),
+               topk_val=tk_val.cpu().numpy(), n_active=n_act.cpu().numpy(), status=m.get_status(), mix=m)
+    return out
+
+
+def bf16_ulp(x):
+    a = np.maximum(np.abs(x), 2.0 ** -126)
+    return 2.0 ** (np.floor(np.log2(a)) - 7)
+
+
+def check_parity(wh, out, rows=None, expect_status=0, check_features=True):
+    """wh: host workload (numpy); out: run_gpu result.  Asserts parity on `rows` (default all)."""
+    T = wh.T_max
+    rows = list(range(T)) if rows is None else sorted(set(int(r) for r in rows))
+    ref = O.apply_hook(wh, rows, keep_z=True)
+    hmax = float(np.abs(O.bf16_to_f64(wh.hidden)).max())
+    hid = out["hidden"]
+    scores_bits = out["scores"].view(np.uint32)
+    stats = dict(max_score_rel=0.0, max_hidden_err=0.0, max_hidden_ulp=0.0, topk_swaps=0, rows=len(rows))
+    redo = {}
+    for t in rows:
+        kind = ref.kind[t]
+        if kind == 0 or kind == O.KIND_PROBE:
+            assert np.array_equal(hid[t], wh.hidden[t]), "row %d (kind %d) must be bit-identical" % (t, kind)
+        if kind != O.KIND_PROBE:
+            assert (scores_bits[t] == CANARY_F32).all(), "scores of non-probe row %d were written" % t
+        if kind == O.KIND_PROBE:
+            s_ref = ref.scores[t]
+            C = len(s_ref)
+            s_gpu = out["scores"][t, :C].astype(np.float64)
+            rel = np.abs(s_gpu - s_ref) / np.abs(s_ref)
+            assert (rel <= SCORE_RTOL).all(), "row %d probe scores off: rel %g" % (t, rel.max())
+            assert (scores_bits[t, C:] == CANARY_F32).all()
+            stats["max_score_rel"] = max(stats["max_score_rel"], float(rel.max()))
+        if kind == O.KIND_SAE and t in ref.topk and check_features:
+            K_ref = ref.topk[t]
+            k = len(K_ref)
+            K_gpu = out["topk_idx"][t, :k].astype(np.int64)
+            z = ref.z[t]
+            assert len(set(K_gpu.tolist())) == k and K_gpu.min() >= 0 and K_gpu.max() < len(z), "row %d bad TopK ids" % t
+            kth = z[K_ref[-1]]
+            diff = set(K_gpu.tolist()) ^ set(K_ref.tolist())
+            for j in diff:
+                assert abs(z[j] - kth) <= TOPK_TIE_TOL, "row %d: TopK member %d differs and is not a near-tie" % (t, j)
+            # what the GPU kept must dominate what it dropped, within the tie tolerance
+            assert np.delete(z, K_gpu).max() - z[K_gpu].min() <= TOPK_TIE_TOL
+            assert np.abs(out["topk_val"][t, :k] - z[K_gpu]).max() <= 1e-3 * max(1.0, np.abs(z[K_gpu]).max())
+            assert (np.diff(out["topk_val"][t, :k]) <= 0).all(), "row %d TopK values not descending" % t
+            assert (out["topk_idx"][t, k:] == CANARY_I32).all()
+            if diff:
+                stats["topk_swaps"] += 1
+                redo[t] = K_gpu
+    if redo:       # re-evaluate those rows with the GPU's (valid) choice among near-ties
+        ref2 = O.apply_hook(wh, list(redo), topk_override=redo)
+        for t in redo:
+            ref.y[t] = ref2.y[t]
+            ref.n_active[t] = ref2.n_active[t]
+    for t in rows:
+        kind = ref.kind[t]
+        if kind in (O.KIND_STEER, O.KIND_SAE):
+            g = O.bf16_to_f64(hid[t])
+            err = np.abs(g - ref.y[t])
+            assert err.max() <= HIDDEN_TOL_FRAC * hmax, "row %d (kind %d) hidden off by %g (bound %g)" % (
+                t, kind, err.max(), HIDDEN_TOL_FRAC * hmax)
+            stats["max_hidden_err"] = max(stats["max_hidden_err"], float(err.max()))
+            stats["max_hidden_ulp"] = max(stats["max_hidden_ulp"], float((err / bf16_ulp(ref.y[t])).max()))
+        if kind == O.KIND_SAE and check_features:
+            na = int(out["n_active"][t])
+            if t in ref.topk:
+                assert na == ref.n_active[t], "row %d n_active %d != %d" % (t, na, ref.n_active[t])
+            else:   # ReLU / JumpReLU: entries within 1e-4 of their threshold may fall either way
+                sae = wh.groups[wh.apps[int(wh.token_slot[t])].group]
+                thr = np.zeros_like(ref.z[t]) if sae.theta is None else np.maximum(sae.theta.astype(np.float64), 0)
+                slack = int((np.abs(ref.z[t] - thr) <= 1e-4).sum())
+                assert abs(na - ref.n_active[t]) <= slack, "row %d n_active %d vs %d" % (t, na, ref.n_active[t])
+        elif check_features:
+            assert int(out["n_active"][t]) == int(CANARY_I32)
+    if expect_status is not None:
+        assert out["status"] == expect_status, "status word %#x, expected %#x" % (out["status"], expect_status)
+    return stats
+
+
+def sample_rows(wh, per_kind=24, seed=0):
+    """A seeded sample of rows covering every kind, every SAE group's first and last row and
+    every request's last token."""
+    rng = np.random.default_rng(seed)
+    T = wh.T_max
+    kinds = {}
+    for t in range(T):
+        s = int(wh.token_slot[t]) if t < wh.T_live else -1
+        a = wh.apps.get(s)
+        key = (0,) if a is None else ((a.kind, a.group) if a.kind == O.KIND_SAE else (a.kind,))
+        kinds.setdefault(key, []).append(t)
+    rows = []
+    for key, ts in kinds.items():
+        ts = np.asarray(ts)
+        pick = set(rng.choice(ts, size=min(per_kind, len(ts)), replace=False).tolist())
+        pick |= {int(ts[0]), int(ts[-1])}
+        rows += sorted(pick)
+    return sorted(set(rows))
+
+
+def oracle_edit_hint(gi, sae, h_row):
+    """Edit hint for the generators: the oracle's active features on one row."""
+    x = O.bf16_to_f64(W.bits(h_row))
+    z = O.sae_preact(x, W.bits(sae.W_enc), W.bits(sae.b_enc))[0]
+    f, K = O.sae_activate(z, sae.act, sae.k, None if sae.theta is None else W.bits(sae.theta))
+    return np.nonzero(f > 0)[0]

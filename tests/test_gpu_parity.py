@@ -1,0 +1,348 @@
+"""GPU parity: the CUDA path (through the C ABI) against the float64 oracle, row by row."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as W
+from oracle import mi_hook as O
+
+from parity import CANARY_F32, check_parity, oracle_edit_hint, run_gpu, sample_rows
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _mixlib():
+    import paper_2607_22595_b200 as mixlib
+    return mixlib
+
+
+# ------------------------------------------------------------------ config 0
+@pytest.mark.parametrize("graph", [False, True])
+@pytest.mark.parametrize("simt", [False, True])
+def test_tiny_full(graph, simt):
+    w = W.make_tiny(DEV)
+    out = run_gpu(w, flags=_mixlib().MIX_FLAG_ENCODE_SIMT if simt else 0, graph=graph)
+    st = check_parity(W.host(w), out)
+    assert st["rows"] == 64
+
+
+def test_tiny_graph_replay_is_repeatable():
+    w = W.make_tiny(DEV)
+    a = run_gpu(w, graph=True, replays=1)
+    b = run_gpu(w, graph=True, replays=5)
+    assert np.array_equal(a["hidden"], b["hidden"]) and np.array_equal(a["topk_idx"], b["topk_idx"])
+
+
+# ------------------------------------------------------------------ config 1
+@pytest.mark.parametrize("graph", [False, True])
+def test_decode_full(graph):
+    w = W.make_decode(DEV)
+    out = run_gpu(w, graph=graph)
+    st = check_parity(W.host(w), out, check_features=False)
+    assert st["max_hidden_ulp"] <= 1.0 + 1e-9          # steering is one rounding away from the exact value
+
+
+# ------------------------------------------------------------------ shrunk configs 2-4 (several tiles, ragged tails)
+@pytest.mark.parametrize("simt", [False, True])
+def test_sae_heavy_small(simt):
+    w = W.make_sae_heavy(DEV, d=256, d_sae=2048, k=16, T=700, R=12, G=3, n_edit=8, edit_hint=oracle_edit_hint)
+    out = run_gpu(w, flags=_mixlib().MIX_FLAG_ENCODE_SIMT if simt else 0)
+    check_parity(W.host(w), out)
+
+
+def test_mixed_small():
+    w = W.make_mixed(DEV, d=320, T=1500, R=40, d_sae=1024, cap=200, mu=3.5, edit_hint=oracle_edit_hint)
+    out = run_gpu(w, graph=True)
+    st = check_parity(W.host(w), out)
+    assert st["rows"] == 1500
+
+
+def test_replay_small_fresh_maps_one_capture():
+    mixlib = _mixlib()
+    w = W.make_replay(DEV, d=256, T_max=512, d_sae=4096, k=16, G=3, n_probe=6, n_steer=4, n_sae_slots=9, n_edit=6)
+    m = W.make_context(mixlib.Mix, w)
+    T, k_max = w.T_max, w.k_max
+    h_static = w.hidden.clone()
+    scores = torch.empty((T, 1), dtype=torch.float32, device=DEV)
+    tk_idx = torch.empty((T, k_max), dtype=torch.int32, device=DEV)
+    tk_val = torch.empty((T, k_max), dtype=torch.float32, device=DEV)
+    n_act = torch.empty((T,), dtype=torch.int32, device=DEV)
+    m.set_feature_out(tk_idx, tk_val, n_act)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        m.apply(h_static, scores, stream=s)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            m.apply(h_static, scores, stream=s)
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    for r in range(8):
+        token_slot, n_live = W.replay_map(w, r)
+        m.set_slot_map(token_slot, n_live)
+        h_static.copy_(w.hidden)
+        scores.copy_(torch.from_numpy(np.full((T, 1), CANARY_F32, dtype=np.uint32).view(np.float32)))
+        tk_idx.fill_(-559038737); n_act.fill_(-559038737)
+        g.replay()
+        torch.cuda.synchronize()
+        w.token_slot, w.T_live = token_slot, n_live
+        out = dict(hidden=W.bits(h_static), scores=scores.cpu().numpy(), topk_idx=tk_idx.cpu().numpy(),
+                   topk_val=tk_val.cpu().numpy(), n_active=n_act.cpu().numpy(), status=m.get_status())
+        check_parity(W.host(w), out)
+
+
+# ------------------------------------------------------------------ edge cases
+def test_all_unhooked_zero_live_and_single_row():
+    w = W.make_tiny(DEV)
+    base = w.token_slot.copy()
+    w.token_slot = np.full_like(base, -1)
+    out = run_gpu(w)
+    assert np.array_equal(out["hidden"], W.bits(w.hidden)) and (out["scores"].view(np.uint32) == CANARY_F32).all()
+    w.token_slot = base
+    w.T_live = 0
+    out = run_gpu(w)
+    assert np.array_equal(out["hidden"], W.bits(w.hidden)) and out["status"] == 0
+    w.T_live = 1
+    check_parity(W.host(w), run_gpu(w))
+    for s in (0, 1, 2, 3):                 # every row on one slot
+        w.T_live = w.T_max
+        w.token_slot = np.full_like(base, s)
+        check_parity(W.host(w), run_gpu(w))
+
+
+def test_bad_slots_raise_status_and_pass_through():
+    mixlib = _mixlib()
+    w = W.make_tiny(DEV)
+    w.token_slot[0] = 1000
+    w.token_slot[1] = -7
+    w.token_slot[2] = 6                     # in range, never registered
+    out = run_gpu(w)
+    check_parity(W.host(w), out, expect_status=mixlib.MIX_STATUS_BAD_SLOT)
+
+
+def test_alpha_zero_and_opposite_alphas():
+    w = W.make_decode(DEV, d=512, T=64, n_probe=2, n_steer=2)
+    steer_slots = [s for s, a in w.apps.items() if a.kind == W.KIND_STEER]
+    for s in steer_slots:
+        w.apps[s].alpha = 0.0
+    # negative zeros in the input must survive alpha = 0
+    hb = W.bits(w.hidden).copy(); hb[:, 3] = 0x8000
+    w.hidden = W.from_bits(hb, DEV)
+    out = run_gpu(w)
+    assert np.array_equal(out["hidden"], hb)
+    w.apps[steer_slots[0]].alpha = 3.0
+    out = run_gpu(w)
+    check_parity(W.host(w), out, check_features=False)
+    # +alpha then -alpha returns within one bf16 ulp
+    h1 = W.from_bits(out["hidden"], DEV)
+    w.apps[steer_slots[0]].alpha = -3.0
+    out2 = run_gpu(w, hidden=h1)
+    a, b = O.bf16_to_f64(out2["hidden"]), O.bf16_to_f64(hb)
+    from parity import bf16_ulp
+    assert (np.abs(a - b) <= bf16_ulp(np.maximum(np.abs(b), np.abs(O.bf16_to_f64(out["hidden"]))))).all()
+
+
+def _one_sae_workload(d, S, act, k, T, add_error, edits, b_dec=False, center=False, seed=5, W_enc=None,
+                      b_enc=None, b_enc_mean=-0.1):
+    g = torch.Generator(device=DEV); g.manual_seed(seed)
+    sae = W.make_sae_weights(g, DEV, d, S, act, k=k, theta_range=(0.05, 0.3), b_enc_mean=b_enc_mean)
+    if W_enc is not None:
+        sae.W_enc = W_enc
+    if b_enc is not None:
+        sae.b_enc = b_enc
+    if b_dec:
+        sae.b_dec = torch.randn(d, generator=g, device=DEV, dtype=torch.float32)
+        sae.center_input = center
+    hidden = torch.randn((T, d), generator=g, device=DEV, dtype=torch.float32).to(torch.bfloat16)
+    idx, val, mode = edits
+    app = W.SaeApp(0, np.asarray(idx, np.int32), np.asarray(val, np.float32), np.asarray(mode, np.uint8), add_error)
+    return W.Workload("one_sae", d, T, T, hidden, np.zeros(T, dtype=np.int32), {0: app}, {0: sae}, n_slots_max=2,
+                      n_groups_max=1, C_max=1, k_max=max(k, 1), r_max=max(len(idx), 1), d_sae_max=S)
+
+
+@pytest.mark.parametrize("act", [W.SAE_RELU, W.SAE_JUMPRELU, W.SAE_TOPK])
+@pytest.mark.parametrize("add_error", [True, False])
+def test_sae_modes_with_b_dec_and_centering(act, add_error):
+    # replace mode on ReLU / JumpReLU sums every active feature: keep them sparse with a low bias
+    w = _one_sae_workload(192, 1024, act, 24, 150, add_error, ([5, 900, 17, 5], [3.0, 0.0, 6.5, 4.0], [0, 1, 0, 0]),
+                          b_dec=True, center=True, b_enc_mean=-0.1 if add_error else -2.0)
+    out = run_gpu(w)
+    check_parity(W.host(w), out)
+
+
+def test_no_edit_with_error_leaves_rows_bit_exact():
+    w = _one_sae_workload(128, 512, W.SAE_TOPK, 8, 40, True, ([], [], []))
+    out = run_gpu(w)
+    assert np.array_equal(out["hidden"], W.bits(w.hidden))
+    check_parity(W.host(w), out)
+
+
+def test_topk_exact_ties_pick_lower_index():
+    # duplicate encoder rows give exactly equal pre-activations; the lower feature id must win
+    d, S, k = 128, 512, 8
+    g = torch.Generator(device=DEV); g.manual_seed(3)
+    We = (torch.randn((S, d), generator=g, device=DEV) * d ** -0.5).to(torch.bfloat16)
+    We[256:] = We[:256]
+    be = torch.full((S,), -0.1, dtype=torch.float32, device=DEV)
+    w = _one_sae_workload(d, S, W.SAE_TOPK, k, 33, True, ([1], [2.0], [0]), W_enc=We, b_enc=be)
+    out = run_gpu(w)
+    check_parity(W.host(w), out)
+    ref = O.apply_hook(W.host(w), keep_z=False)
+    for t in range(33):
+        assert out["topk_idx"][t, :k].tolist() == ref.topk[t].tolist()      # exact, order included
+
+
+def test_topk_massive_ties_use_general_path():
+    # W_enc = 0: every pre-activation equals the bias -> more ties than the candidate buffer holds
+    mixlib = _mixlib()
+    d, S, k = 128, 8192, 16
+    We = torch.zeros((S, d), dtype=torch.bfloat16, device=DEV)
+    be = torch.full((S,), 0.25, dtype=torch.float32, device=DEV)
+    be[5000] = 1.0; be[77] = 0.5
+    w = _one_sae_workload(d, S, W.SAE_TOPK, k, 5, False, ([77], [0.0], [1]), W_enc=We, b_enc=be)
+    out = run_gpu(w)
+    check_parity(W.host(w), out, expect_status=mixlib.MIX_STATUS_TOPK_GENERAL)
+    assert out["topk_idx"][0, :k].tolist() == [5000, 77] + list(range(14))
+
+
+def test_identity_encoder_topk_of_own_coordinates():
+    d, S, k = 128, 512, 8
+    I = torch.zeros((S, d), dtype=torch.bfloat16, device=DEV); I[:d] = torch.eye(d, dtype=torch.bfloat16, device=DEV)
+    w = _one_sae_workload(d, S, W.SAE_TOPK, k, 20, False, ([], [], []), W_enc=I,
+                          b_enc=torch.zeros(S, dtype=torch.float32, device=DEV))
+    w.groups[0].W_dec = I.clone()
+    out = run_gpu(w)
+    check_parity(W.host(w), out)
+    h = O.bf16_to_f64(W.bits(w.hidden))
+    for t in range(20):                      # output = ReLU of the row's own k largest coordinates
+        K = out["topk_idx"][t, :k]
+        want = np.zeros(d); want[K] = np.maximum(h[t, K], 0)
+        assert np.array_equal(O.bf16_to_f64(out["hidden"][t]), want)
+
+
+# ------------------------------------------------------------------ toggling under one captured graph
+def test_toggle_without_recapture():
+    mixlib = _mixlib()
+    w = W.make_tiny(DEV)
+    m = W.make_context(mixlib.Mix, w)
+    T = w.T_max
+    h_static = w.hidden.clone()
+    scores = torch.zeros((T, 1), dtype=torch.float32, device=DEV)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        m.apply(h_static, scores, stream=s)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            m.apply(h_static, scores, stream=s)
+    torch.cuda.current_stream().wait_stream(s)
+
+    def replay_and_check(expect_status=0):
+        h_static.copy_(w.hidden)
+        scores.copy_(torch.from_numpy(np.full((T, 1), CANARY_F32, dtype=np.uint32).view(np.float32)))
+        g.replay()
+        torch.cuda.synchronize()
+        out = dict(hidden=W.bits(h_static), scores=scores.cpu().numpy(), status=m.get_status())
+        check_parity(W.host(w), out, check_features=False, expect_status=expect_status)
+
+    replay_and_check()
+    w.apps[1].alpha = -2.5; m.update_steer_alpha(1, -2.5)                 # change a parameter
+    replay_and_check()
+    idx, val, mode = np.array([7, 9], np.int32), np.array([1.5, 0], np.float32), np.array([0, 1], np.uint8)
+    w.apps[2].edit_idx, w.apps[2].edit_val, w.apps[2].edit_mode = idx, val, mode
+    m.update_sae_edits(2, idx, val, mode)                                 # change an edit list
+    replay_and_check()
+    rng = np.random.default_rng(1)
+    w.token_slot = rng.permutation(w.token_slot).astype(np.int32); m.set_slot_map(w.token_slot)
+    replay_and_check()
+    del w.apps[0]; m.unregister_app(0)                                    # rows still naming slot 0 pass through
+    replay_and_check(expect_status=mixlib.MIX_STATUS_BAD_SLOT)
+    g2 = torch.Generator(device=DEV); g2.manual_seed(9)
+    w.apps[5] = W.Steer(v=torch.randn(w.d_model, generator=g2, device=DEV).to(torch.bfloat16), alpha=0.75)
+    m.register_steer(5, w.apps[5].v, 0.75)
+    w.token_slot = np.where(w.token_slot == 0, 5, w.token_slot).astype(np.int32); m.set_slot_map(w.token_slot)
+    replay_and_check()
+
+
+def test_request_map_two_level_matches_flat_map():
+    mixlib = _mixlib()
+    w = W.make_tiny(DEV)
+    m = W.make_context(mixlib.Mix, w)
+    token_req = w.meta["token_req"].astype(np.int32)
+    m.set_request_map(token_req, w.meta["req_slot"].astype(np.int32))
+    out = run_gpu(w, mix=m)
+    check_parity(W.host(w), out)
+    m.set_request_map(torch.from_numpy(token_req).cuda(), torch.from_numpy(w.meta["req_slot"].astype(np.int32)).cuda())
+    check_parity(W.host(w), run_gpu(w, mix=m))
+
+
+def test_permutation_equivariance_on_gpu():
+    w = W.make_tiny(DEV)
+    a = run_gpu(w)
+    perm = np.random.default_rng(0).permutation(w.T_max)
+    w2 = W.make_tiny(DEV)
+    w2.hidden = w.hidden[torch.from_numpy(perm).cuda()].contiguous()
+    w2.token_slot = w.token_slot[perm].copy()
+    b = run_gpu(w2)
+    assert np.array_equal(b["hidden"], a["hidden"][perm])
+    assert np.array_equal(b["scores"].view(np.uint32), a["scores"].view(np.uint32)[perm])
+
+
+def test_api_error_codes():
+    mixlib = _mixlib()
+    with pytest.raises(mixlib.MixError) as e:
+        mixlib.Mix(d_model=100, T_max=8, n_slots_max=2)                    # d % 64
+    assert e.value.code == -3
+    m = mixlib.Mix(d_model=128, T_max=8, n_slots_max=2, n_groups_max=1, C_max=2, k_max=4, r_max=2, d_sae_max=256)
+    v = torch.zeros(128, dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(mixlib.MixError) as e:
+        m.register_steer(5, v, 1.0)
+    assert e.value.code == -2 and "slot" in str(e.value)
+    Wp = torch.zeros((3, 128), dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(mixlib.MixError) as e:
+        m.register_probe(0, Wp, None, mixlib.MIX_ACT_SOFTMAX)              # C > C_max
+    assert e.value.code == -2
+    with pytest.raises(mixlib.MixError) as e:
+        m.register_sae_app(0, 0, [1], [1.0], [0], True)                   # group not registered
+    assert e.value.code == -2
+    We = torch.zeros((256, 128), dtype=torch.bfloat16, device=DEV); be = torch.zeros(256, device=DEV)
+    with pytest.raises(mixlib.MixError) as e:
+        m.register_sae_weights(0, 256, mixlib.MIX_SAE_TOPK, 9, We, be, We)  # k > k_max
+    assert e.value.code == -2
+    with pytest.raises(mixlib.MixError) as e:
+        m.register_sae_weights(0, 256, mixlib.MIX_SAE_JUMPRELU, 0, We, be, We)  # no theta
+    assert e.value.code == -1
+    m.register_sae_weights(0, 256, mixlib.MIX_SAE_TOPK, 4, We, be, We)
+    with pytest.raises(mixlib.MixError) as e:
+        m.register_sae_app(0, 0, [256], [1.0], [0], True)                 # feature id out of range
+    assert e.value.code == -2
+    with pytest.raises(mixlib.MixError) as e:
+        m.register_sae_app(0, 0, [1, 2, 3], [1.0, 1, 1], [0, 0, 0], True)  # n_edit > r_max
+    assert e.value.code == -2
+    with pytest.raises(mixlib.MixError) as e:
+        m.set_slot_map(np.zeros(9, dtype=np.int32))                       # T_live > T_max
+    assert e.value.code == -2
+    assert m.launches_per_apply() == 6
+    m.destroy()
+
+
+# ------------------------------------------------------------------ full-size configs, sampled rows
+def test_sae_heavy_full_size_sampled_rows():
+    w = W.make_sae_heavy(DEV, edit_hint=oracle_edit_hint)
+    out = run_gpu(w, graph=True)
+    wh = W.host(w)
+    rows = sample_rows(wh, per_kind=6, seed=2)
+    st = check_parity(wh, out, rows=rows)
+    assert st["rows"] >= 24
+
+
+def test_mixed_full_size_sampled_rows():
+    w = W.make_mixed(DEV, edit_hint=oracle_edit_hint)
+    out = run_gpu(w, graph=True)
+    wh = W.host(w)
+    # every unhooked row is bit-identical, at full size
+    unh = np.nonzero(wh.token_slot < 0)[0]
+    assert np.array_equal(out["hidden"][unh], wh.hidden[unh])
+    rows = sample_rows(wh, per_kind=16, seed=3)
+    check_parity(wh, out, rows=rows)
