@@ -1,0 +1,426 @@
+#!/usr/bin/env python
+"""Benchmark of the MI hook on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl mix|reference] [--no-extras]
+
+A step is one mix_apply() over one synthetic decode batch (d = 4096, 256 one-token requests,
+64 probes + 32 steering vectors, 25 % of rows unhooked).  The timed region replays CUDA graphs
+whose nodes are consecutive steps on ROTATING hidden-state buffers (512 MiB in total, four
+times the L2), so every step finds its activations cold in L2; inputs are resident in HBM.
+One JSON line goes to stdout (rank 0).  With N > 1 every rank runs its own replica on its own
+batch (rows are independent: no collective on the data path), time = max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads as W  # noqa: E402
+
+METRIC = "mi_hook_token_rows_per_s"
+UNIT = "token-rows/s"
+WORKLOAD = "decode: d=4096, T=256 (256 requests x 1 token), 64 probes + 32 steering vectors, 25% unhooked"
+ROTATE_BYTES = 512 << 20
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return dict(hbm_gbs=float(j["hbm_gbs"]), bf16_tflops=float(j["bf16_tflops"]),
+                    bf16_tflops_sustained=float(j.get("bf16_tflops_sustained", j["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.samples = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(device_index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL,
+                text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 7:
+                self.samples.append((time.time(), parts))
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()           # the exact child started above
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                pass
+
+    def summary(self, t0, t1):
+        inside = [p for (ts, p) in self.samples if t0 <= ts <= t1]
+        pool = inside or [p for (_, p) in self.samples[-3:]]
+        if not pool:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        def num(x):
+            try:
+                return float(x)
+            except ValueError:
+                return None
+        sm = [num(p[0]) for p in pool if num(p[0]) is not None]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({n for p in pool for n, v in zip(names, p[3:7]) if v.lower().startswith("active")})
+        pw = [num(p[2]) for p in pool if num(p[2]) is not None]
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": num(pool[0][1]), "reasons": reasons,
+                "power_w_max": max(pw) if pw else None, "samples": len(inside)}
+
+
+# ------------------------------------------------------------------------------ helpers
+def decode_bytes(w):
+    """Algorithmic bytes of one decode-config launch: hidden rows read (probe + steer), steer rows
+    written back, each distinct weight vector once, the slot map, the scores."""
+    d = w.d_model
+    rows_p = rows_s = 0
+    used = set()
+    for t in range(w.T_live):
+        a = w.apps.get(int(w.token_slot[t]))
+        if a is None:
+            continue
+        used.add(int(w.token_slot[t]))
+        if a.kind == W.KIND_PROBE:
+            rows_p += 1
+        elif a.kind == W.KIND_STEER:
+            rows_s += 1
+    wbytes = sum((w.apps[s].n_classes if w.apps[s].kind == W.KIND_PROBE else 1) * d * 2 for s in used)
+    return (rows_p + 2 * rows_s) * d * 2 + wbytes + 4 * w.T_max + 4 * rows_p, rows_p, rows_s
+
+
+def capture_steps(m, hiddens, scores, idxs, stream):
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=stream):
+        for i in idxs:
+            m.apply(hiddens[i], scores[i], stream=stream)
+    return g
+
+
+def dist_max(x: float, world: int) -> float:
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device="cuda" if torch.cuda.is_available() else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def dist_sum(x: float, world: int) -> float:
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device="cuda" if torch.cuda.is_available() else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+# ------------------------------------------------------------------------------ oracle legs
+def oracle_leg(seconds_target=10.0, max_batches=10000):
+    """Time the float64 oracle, as it stands, on whole decode batches for about `seconds_target` s."""
+    from oracle import mi_hook as O
+    wh = W.host(W.make_decode("cpu"))
+    O.apply_hook(wh)                                   # warm-up (page in numpy / BLAS)
+    n, t0 = 0, time.perf_counter()
+    while True:
+        O.apply_hook(wh)
+        n += 1
+        dt = time.perf_counter() - t0
+        if dt >= seconds_target or n >= max_batches:
+            break
+    return dict(rows_per_s=n * wh.T_max / dt, batches=n, seconds=dt, rows=n * wh.T_max)
+
+
+def run_reference(args, rank, world):
+    """--impl reference: the oracle on the host cores, same metric and config."""
+    if rank != 0:
+        return
+    steps, warm = args.steps or 20, args.warmup if args.warmup is not None else 3
+    from oracle import mi_hook as O
+    wh = W.host(W.make_decode("cpu"))
+    for _ in range(max(warm, 1)):
+        O.apply_hook(wh)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        O.apply_hook(wh)
+    dt = time.perf_counter() - t0
+    val = steps * wh.T_max / dt
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+            "warmup": warm, "ms_per_step": 1e3 * dt / steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "note": "float64 CPU oracle, one whole batch per step"},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle",
+                             "sample": "%d whole decode batches (256 rows each)" % steps},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------ extras
+def time_stages(m, fn, reps=5):
+    """Per-kernel milliseconds of one apply via the library's stage-event taps (best of reps)."""
+    n = m.launches_per_apply()
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+    m.set_stage_events(evs)
+    best = None
+    for _ in range(reps):
+        fn()
+        torch.cuda.synchronize()
+        ms = [evs[i].elapsed_time(evs[i + 1]) for i in range(n)]
+        best = ms if best is None else [min(a, b) for a, b in zip(best, ms)]
+    m.set_stage_events(None)
+    return dict(zip(m.STAGES[:n], best))
+
+
+def extras_sae(name, w, peaks, mixlib):
+    """SAE-carrying config: per-kernel times, encode flop rate and weight-stream bandwidth."""
+    m = W.make_context(mixlib.Mix, w)
+    h = w.hidden.clone()
+    scores = torch.zeros((w.T_max, max(w.C_max, 1)), dtype=torch.float32, device="cuda")
+    def fn():
+        h.copy_(w.hidden)
+        m.apply(h, scores)
+    for _ in range(2):
+        fn()
+    torch.cuda.synchronize()
+    st = time_stages(m, fn)
+    # whole call under graph replay
+    s = torch.cuda.Stream(); s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        m.apply(h, scores, stream=s)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            m.apply(h, scores, stream=s)
+    torch.cuda.current_stream().wait_stream(s)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    times = []
+    for _ in range(5):
+        h.copy_(w.hidden)
+        e0.record(); g.replay(); e1.record(); torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    counts = {}
+    for t in range(w.T_live):
+        a = w.apps.get(int(w.token_slot[t]))
+        if a is not None and a.kind == W.KIND_SAE:
+            counts[a.group] = counts.get(a.group, 0) + 1
+    flops = sum(2.0 * n * w.d_model * w.groups[g].d_sae for g, n in counts.items())
+    wbytes = sum(2.0 * w.d_model * w.groups[g].d_sae for g in counts)
+    enc_s = st["encode"] * 1e-3
+    status = m.get_status()
+    m.destroy()
+    return {"workload": name, "t_call_ms_graph": min(times), "stage_ms": st, "sae_rows_per_group": counts,
+            "encode_tflops": flops / enc_s / 1e12, "encode_frac_bf16_peak": flops / enc_s / 1e12 / peaks["bf16_tflops"],
+            "encode_weight_stream_gbs": wbytes / enc_s / 1e9,
+            "encode_frac_hbm_peak": wbytes / enc_s / 1e9 / peaks["hbm_gbs"],
+            "token_rows_per_s": w.T_live / (min(times) * 1e-3), "status": status}
+
+
+def extras_sweep(peaks, mixlib):
+    """Bandwidth kernels alone at a size that cannot hide in L2: d = 8192, T = 65536, every row hooked."""
+    d, T = 8192, 65536
+    g = torch.Generator(device="cuda"); g.manual_seed(1)
+    hidden = torch.randn((T, d), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    v = torch.randn((d,), generator=g, device="cuda").to(torch.bfloat16)
+    Wp = (torch.randn((1, d), generator=g, device="cuda") * d ** -0.5).to(torch.bfloat16)
+    m = mixlib.Mix(d_model=d, T_max=T, n_slots_max=2)
+    m.register_steer(0, v, 2.0)
+    m.register_probe(1, Wp, None, mixlib.MIX_ACT_SIGMOID)
+    scores = torch.zeros((T, 1), dtype=torch.float32, device="cuda")
+    out = {}
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for name, slot, nbytes in (("steer", 0, 2.0 * T * d * 2), ("probe", 1, 1.0 * T * d * 2)):
+        m.set_slot_map(torch.full((T,), slot, dtype=torch.int32, device="cuda"))
+        best = 1e9
+        for _ in range(6):
+            e0.record(); m.apply(hidden, scores); e1.record(); torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        out[name] = {"ms": best, "gbs": nbytes / best / 1e6, "frac_hbm_peak": nbytes / best / 1e6 / peaks["hbm_gbs"]}
+    m.destroy()
+    return out
+
+
+# ------------------------------------------------------------------------------ main arm
+def run_mix(args, rank, world, local_rank):
+    import paper_2607_22595_b200 as mixlib
+    from paper_2607_22595_b200 import _build
+    _build.build()
+    torch.cuda.set_device(local_rank)
+    peaks = measured_peaks()
+    w = W.make_decode("cuda", seed=W.BASE_SEED + 1000 + rank)
+    m = W.make_context(mixlib.Mix, w)
+    T, d = w.T_max, w.d_model
+    R = max(2, -(-ROTATE_BYTES // (T * d * 2)))
+    hiddens = [w.hidden.clone() for _ in range(R)]
+    scores = [torch.zeros((T, 1), dtype=torch.float32, device="cuda") for _ in range(R)]
+    K = args.steps or 400 * R
+    Wm = args.warmup if args.warmup is not None else 3 * R
+    Wm = max(Wm, 3)
+
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(stream):
+        for i in range(min(Wm, R)):
+            m.apply(hiddens[i], scores[i], stream=stream)            # untimed warm-up, eager
+        g_full = capture_steps(m, hiddens, scores, range(R), stream) if K >= R else None
+        rem = K % R
+        g_rem = capture_steps(m, hiddens, scores, range(rem), stream) if rem else None
+        for _ in range(max(0, (Wm - R) // R)):
+            if g_full is not None:
+                g_full.replay()
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    time.sleep(0.3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(world); torch.cuda.synchronize()
+    t0 = time.time()
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for _ in range(K // R):
+            g_full.replay()
+        if g_rem is not None:
+            g_rem.replay()
+        e1.record(stream)
+    torch.cuda.synchronize(); barrier(world)
+    t1 = time.time()
+    ms_local = e0.elapsed_time(e1)
+    ms = dist_max(ms_local, world)
+    rows_total = dist_sum(float(K) * w.T_live, world)
+    clocks = sampler.summary(t0, t1)
+
+    # warm-L2 variant (one buffer), for context
+    with torch.cuda.stream(stream):
+        g_warm = capture_steps(m, hiddens, scores, [0] * min(R, 256), stream)
+        g_warm.replay()
+        e0.record(stream)
+        for _ in range(4):
+            g_warm.replay()
+        e1.record(stream)
+    torch.cuda.synchronize()
+    warm_us = e0.elapsed_time(e1) * 1e3 / (4 * min(R, 256))
+
+    # end to end through the public API with host buffers
+    K_e2e = min(K, 2000)
+    h_in = torch.empty((T, d), dtype=torch.bfloat16).pin_memory(); h_in.copy_(w.hidden.cpu())
+    h_out = torch.empty((T, d), dtype=torch.bfloat16).pin_memory()
+    s_out = torch.empty((T, 1), dtype=torch.float32).pin_memory()
+    slot_pin = torch.from_numpy(w.token_slot.copy()).pin_memory()
+    hd, sd = hiddens[0], scores[0]
+    def e2e_step():
+        hd.copy_(h_in, non_blocking=True)
+        m.set_slot_map(slot_pin, w.T_live)
+        m.apply(hd, sd)
+        h_out.copy_(hd, non_blocking=True)
+        s_out.copy_(sd, non_blocking=True)
+    for _ in range(3):
+        e2e_step()
+    torch.cuda.synchronize(); barrier(world)
+    te = time.perf_counter()
+    for _ in range(K_e2e):
+        e2e_step()
+    torch.cuda.synchronize()
+    e2e_s = dist_max(time.perf_counter() - te, world)
+    sampler.stop()
+    e2e_rows = dist_sum(float(K_e2e) * w.T_live, world)
+    status = m.get_status()
+
+    if rank != 0:
+        return
+    nbytes, rows_p, rows_s = decode_bytes(w)
+    ms_per_step = ms / K
+    achieved = nbytes / (ms_per_step * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": rows_total / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "l2": "inputs rotate over %d hidden buffers (%d MiB > 4x L2); weights (0.75 MiB) stay warm" % (R, R * T * d * 2 >> 20),
+                   "graph": "CUDA-graph replay, %d steps per graph" % R, "probe_rows": rows_p, "steer_rows": rows_s,
+                   "us_added_per_decode_step": ms_per_step * 1e3, "us_added_per_decode_step_warm_l2": warm_us,
+                   "status_word": status},
+        "clocks": clocks,
+        "e2e": {"value": e2e_rows / e2e_s, "unit": UNIT, "h2d_bytes_per_step": T * d * 2 + 4 * T,
+                "d2h_bytes_per_step": T * d * 2 + 4 * T, "steps": K_e2e},
+        "gpu_launches": K * m.launches_per_apply(),
+        "roofline": {"bound": "hbm", "kernel": "probe_steer_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                     "algorithmic_bytes_per_launch": nbytes,
+                     "note": "2.9 MB per launch: launch-latency-bound, not bandwidth-bound; see extras.sweep for the same kernel on 2 GiB"},
+    }
+    if world == 1:
+        cb = oracle_leg(args.cpu_seconds)
+        line["cpu_baseline"] = {"value": cb["rows_per_s"], "unit": UNIT, "cores": 1, "kind": "oracle",
+                                "sample": "%d whole decode batches (%d rows) in %.1f s" % (cb["batches"], cb["rows"], cb["seconds"])}
+        if not args.no_extras:
+            ex = {}
+            try:
+                ex["sweep"] = extras_sweep(peaks, mixlib)
+                ex["sae_heavy"] = extras_sae("sae_heavy (config 2)", W.make_sae_heavy("cuda"), peaks, mixlib)
+                torch.cuda.empty_cache()
+                ex["mixed"] = extras_sae("mixed (config 3)", W.make_mixed("cuda"), peaks, mixlib)
+            except Exception as e:                       # extras never break the contract line
+                ex["error"] = repr(e)
+            line["extras"] = ex
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="mix", choices=["mix", "reference"])
+    ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=10.0)
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    try:
+        run_mix(args, rank, world, local_rank)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -205,6 +205,13 @@ int mix_get_status(mix_ctx* ctx, unsigned* bits, void* stream);
 /* Number of kernels one mix_apply() call launches on this context (fixed at mix_create). */
 int mix_launches_per_apply(const mix_ctx* ctx);
 
+/* Per-kernel timing taps (profiling only; do not use while capturing a graph).  events: HOST
+   array of mix_launches_per_apply() + 1 cudaEvent_t handles created by the caller with timing
+   enabled, or NULL to switch the taps off.  Every later mix_apply() records events[0] before
+   its first kernel and events[i] after its i-th kernel, on the call's stream; the array is
+   copied.  Kernel order: probe_steer, route, pack, encode, select, decode. */
+int mix_set_stage_events(mix_ctx* ctx, void* const* events);
+
 /* Test / profiling taps into the SAE workspace after a mix_apply (device pointers owned by
    the context; valid until mix_destroy):  panel_rows int32 [n_panel_rows] gives the token
    index of each packed panel row (-1 = padding), z the fp32 pre-activations

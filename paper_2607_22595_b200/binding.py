@@ -26,7 +26,7 @@ EXPORTS = [
     "mix_create", "mix_destroy", "mix_last_error", "mix_register_sae_weights", "mix_unregister_sae_weights",
     "mix_register_app", "mix_unregister_app", "mix_update_steer_alpha", "mix_update_sae_edits",
     "mix_set_slot_map", "mix_set_request_map", "mix_set_feature_out", "mix_apply", "mix_get_status",
-    "mix_launches_per_apply", "mix_debug_workspace",
+    "mix_launches_per_apply", "mix_set_stage_events", "mix_debug_workspace",
 ]
 
 
@@ -90,6 +90,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.mix_apply.argtypes = [vp, vp, ci, vp, vp]
     lib.mix_get_status.argtypes = [vp, C.POINTER(C.c_uint), vp]
     lib.mix_launches_per_apply.argtypes = [vp]
+    lib.mix_set_stage_events.argtypes = [vp, C.POINTER(vp)]
     lib.mix_debug_workspace.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(C.c_longlong), C.POINTER(ci)]
     for name in EXPORTS:
         if name != "mix_last_error":
@@ -230,6 +231,20 @@ class Mix:
 
     def launches_per_apply(self) -> int:
         return int(self.lib.mix_launches_per_apply(self.ctx))
+
+    STAGES = ["probe_steer", "route", "pack", "encode", "select", "decode"]
+
+    def set_stage_events(self, events=None):
+        """events: list of launches_per_apply() + 1 torch.cuda.Event(enable_timing=True), or None."""
+        if events is None:
+            self._check(self.lib.mix_set_stage_events(self.ctx, None))
+            self._keep.pop("ev", None)
+            return
+        for e in events:
+            e.record()                       # torch creates the CUDA event lazily, on first record
+        arr = (C.c_void_p * len(events))(*[e.cuda_event for e in events])
+        self._check(self.lib.mix_set_stage_events(self.ctx, arr))
+        self._keep["ev"] = events
 
     def debug_workspace(self):
         pr, z, ld, n = C.c_void_p(), C.c_void_p(), C.c_longlong(), C.c_int()

@@ -378,16 +378,27 @@ int mix_apply(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream) 
   if (!hidden || !aligned16(hidden)) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "hidden is NULL or not 16-byte aligned");
   if (T < 0 || T > c->cfg.T_max) MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "T %d outside [0, T_max=%d]", T, c->cfg.T_max);
   __nv_bfloat16* h = static_cast<__nv_bfloat16*>(hidden);
+  int stage = 0;
+  auto tap = [&]() -> cudaError_t {
+    return c->stage_events_on ? cudaEventRecord(c->stage_events[stage++], s) : cudaSuccess;
+  };
+  MIX_CUDA(c, tap());
   MIX_CUDA(c, launch_probe_steer(c, h, T, scores_out, s));
+  MIX_CUDA(c, tap());
   if (c->cfg.n_groups_max > 0) {
     MIX_CUDA(c, launch_route(c, T, s));
+    MIX_CUDA(c, tap());
     MIX_CUDA(c, launch_pack(c, h, s));
+    MIX_CUDA(c, tap());
     if (c->cfg.flags & MIX_FLAG_ENCODE_SIMT)
       MIX_CUDA(c, launch_encode_simt(c, s));
     else
       MIX_CUDA(c, launch_encode_tc(c, s));
+    MIX_CUDA(c, tap());
     MIX_CUDA(c, launch_select(c, s));
+    MIX_CUDA(c, tap());
     MIX_CUDA(c, launch_decode(c, h, s));
+    MIX_CUDA(c, tap());
   }
   return MIX_OK;
 }
@@ -404,6 +415,20 @@ int mix_get_status(mix_ctx* c, unsigned* bits, void* stream) {
   MIX_CUDA(c, cudaMemcpyAsync(bits, c->d_status, sizeof(unsigned), cudaMemcpyDeviceToHost, s));
   MIX_CUDA(c, cudaMemsetAsync(c->d_status, 0, sizeof(unsigned), s));
   MIX_CUDA(c, cudaStreamSynchronize(s));
+  return MIX_OK;
+}
+
+int mix_set_stage_events(mix_ctx* c, void* const* events) {
+  if (!c) return MIX_ERR_INVALID_ARG;
+  c->stage_events_on = 0;
+  if (events) {
+    const int n = mix_launches_per_apply(c) + 1;
+    for (int i = 0; i < n; ++i) {
+      if (!events[i]) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "stage event %d is NULL", i);
+      c->stage_events[i] = static_cast<cudaEvent_t>(events[i]);
+    }
+    c->stage_events_on = 1;
+  }
   return MIX_OK;
 }
 

@@ -93,6 +93,10 @@ struct Ctx {
   CUtensorMap* d_tmap_w;    // [n_groups_max] W_enc maps (box kTileK x kTileN, 128B swizzle)
   CUtensorMap tmap_panel;   // panel map (box kTileK x kTileM, 128B swizzle)
 
+  // profiling taps
+  int stage_events_on;
+  cudaEvent_t stage_events[8];
+
   // optional outputs
   int* out_topk_idx;
   float* out_topk_val;
