@@ -219,6 +219,46 @@ int mix_set_stage_events(mix_ctx* ctx, void* const* events);
 int mix_debug_workspace(mix_ctx* ctx, const int** panel_rows, const float** z, long long* ld_z,
                         int* n_panel_rows);
 
+/* ---------------------------------------------------------------------------------------
+ * SAE function for callers that cannot allocate device memory.  (The paper has no counterpart
+ * to this call; it exists for integration reasons only.)
+ *
+ * Who needs it: code that runs inside a serving engine which has already handed the whole
+ * HBM budget to its own pools (weights, KV cache) and forbids plugins to call cudaMalloc;
+ * code on a latency-critical path, where cudaMalloc / cudaFree would stall the device with
+ * their implicit synchronisation; and tools that must leave the process's allocator state
+ * untouched.  Such callers cannot use mix_create(), which allocates the hook's tables and
+ * workspace.  This single call needs no context: all of its scratch (tables, routing state,
+ * the packed bf16 row panel, the fp32 pre-activations, TopK lists) sits in one fixed array
+ * inside the library image, about 5.2 MiB, which every GPU that loads the library keeps
+ * until the process exits.  The call allocates nothing and frees nothing.
+ *
+ * What it computes: the MIX_SAE function of mix_apply() for ONE app on EVERY one of the
+ * n_rows rows of `hidden` (device bf16 [n_rows, d_model], modified in place): encode,
+ * ReLU / JumpReLU / TopK, the app's edits, decode, error term as `app->add_error` says.
+ * `w` and `app` are host structs as for registration (w's pointers device, app's edit
+ * arrays host, app->group ignored).  topk_idx int32 / topk_val fp32 [n_rows, w->k]: optional
+ * device outputs for TopK SAEs (NULL = off), as in mix_set_feature_out with k_max = w->k.
+ * The encode runs on the CUDA-core kernel (the one MIX_FLAG_ENCODE_SIMT selects).
+ *
+ * Limits (the array has a fixed size): n_rows <= MIX_STATIC_MAX_ROWS, d_model <=
+ * MIX_STATIC_MAX_D_MODEL (multiple of 64), w->d_sae <= MIX_STATIC_MAX_D_SAE (multiple of 256),
+ * w->k <= MIX_STATIC_MAX_K, app->n_edit <= 64, no input centring.  Anything beyond returns
+ * MIX_ERR_OUT_OF_RANGE / MIX_ERR_UNSUPPORTED with a message in errbuf (optional, host).
+ *
+ * Sharing: every call on a device uses the same array, and the array keeps the previous
+ * call's contents; each call rewrites what it reads, so consecutive calls on one stream are
+ * independent, but two calls that overlap on the GPU (different streams, or different host
+ * threads) race on it -- serialise them.  The first call on each device looks up the
+ * array's device address (no allocation); make that first call before any stream capture
+ * begins.  Enqueues on `stream` and returns; results are ready when the stream reaches them. */
+#define MIX_STATIC_MAX_ROWS 128
+#define MIX_STATIC_MAX_D_MODEL 4096
+#define MIX_STATIC_MAX_D_SAE 8192
+#define MIX_STATIC_MAX_K 128
+int mix_sae_apply_static(void* hidden, int n_rows, int d_model, const mix_sae_weights* w, const mix_sae_app* app,
+                         int* topk_idx, float* topk_val, void* stream, char* errbuf, int errbuf_len);
+
 #ifdef __cplusplus
 }
 #endif

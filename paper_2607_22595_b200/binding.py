@@ -26,7 +26,7 @@ EXPORTS = [
     "mix_create", "mix_destroy", "mix_last_error", "mix_register_sae_weights", "mix_unregister_sae_weights",
     "mix_register_app", "mix_unregister_app", "mix_update_steer_alpha", "mix_update_sae_edits",
     "mix_set_slot_map", "mix_set_request_map", "mix_set_feature_out", "mix_apply", "mix_get_status",
-    "mix_launches_per_apply", "mix_set_stage_events", "mix_debug_workspace",
+    "mix_launches_per_apply", "mix_set_stage_events", "mix_debug_workspace", "mix_sae_apply_static",
 ]
 
 
@@ -91,6 +91,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.mix_get_status.argtypes = [vp, C.POINTER(C.c_uint), vp]
     lib.mix_launches_per_apply.argtypes = [vp]
     lib.mix_set_stage_events.argtypes = [vp, C.POINTER(vp)]
+    lib.mix_sae_apply_static.argtypes = [vp, ci, ci, C.POINTER(MixSaeWeights), C.POINTER(MixSaeApp), vp, vp, vp,
+                                         C.c_char_p, ci]
     lib.mix_debug_workspace.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(C.c_longlong), C.POINTER(ci)]
     for name in EXPORTS:
         if name != "mix_last_error":
@@ -250,3 +252,24 @@ class Mix:
         pr, z, ld, n = C.c_void_p(), C.c_void_p(), C.c_longlong(), C.c_int()
         self._check(self.lib.mix_debug_workspace(self.ctx, C.byref(pr), C.byref(z), C.byref(ld), C.byref(n)))
         return pr.value, z.value, ld.value, n.value
+
+
+STATIC_MAX_ROWS, STATIC_MAX_D_MODEL, STATIC_MAX_D_SAE, STATIC_MAX_K = 128, 4096, 8192, 128
+
+
+def sae_apply_static(hidden, d_sae, act, k, W_enc, b_enc, W_dec, idx, val, mode, add_error, theta=None, b_dec=None,
+                     topk_idx=None, topk_val=None, stream=None):
+    """The SAE function on every row of `hidden` (CUDA bf16 [n_rows, d], in place) without any
+    device allocation: for callers that may not call cudaMalloc (see mix_sae_apply_static in
+    mix.h for who they are, the size limits, and why overlapping calls race).  Needs no Mix
+    context.  Raises MixError with the library's message when a size exceeds the fixed limits."""
+    lib = load_library()
+    assert hidden.dtype == torch.bfloat16 and hidden.is_cuda and hidden.is_contiguous()
+    idx, val, mode = Mix._edit_arrays(idx, val, mode)
+    w = MixSaeWeights(int(d_sae), int(act), int(k), _ptr(W_enc), _ptr(b_enc), _ptr(theta), _ptr(W_dec), _ptr(b_dec), 0)
+    a = MixSaeApp(0, len(idx), idx.ctypes.data, val.ctypes.data, mode.ctypes.data, int(bool(add_error)))
+    err = C.create_string_buffer(256)
+    rc = lib.mix_sae_apply_static(hidden.data_ptr(), int(hidden.shape[0]), int(hidden.shape[1]), C.byref(w),
+                                  C.byref(a), _ptr(topk_idx), _ptr(topk_val), _stream(stream), err, 256)
+    if rc != 0:
+        raise MixError(rc, err.value.decode())
