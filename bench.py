@@ -247,6 +247,86 @@ def extras_sae(name, w, peaks, mixlib):
             "token_rows_per_s": w.T_live / (min(times) * 1e-3), "status": status}
 
 
+def run_replay(peaks, mixlib, n_replays):
+    """Config 4: one captured graph at T_max = 2048, a fresh slot map and live count per replay."""
+    w = W.make_replay("cuda")
+    m = W.make_context(mixlib.Mix, w)
+    T = w.T_max
+    h = w.hidden.clone()
+    scores = torch.zeros((T, 1), dtype=torch.float32, device="cuda")
+    s = torch.cuda.Stream(); s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        m.apply(h, scores, stream=s)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            m.apply(h, scores, stream=s)
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    slot_pin = torch.empty(T, dtype=torch.int32).pin_memory()
+    rec, bad_status = [], 0
+    for r in range(n_replays):
+        token_slot, n_live = W.replay_map(w, r)
+        slot_pin.copy_(torch.from_numpy(token_slot))
+        m.set_slot_map(slot_pin, n_live)
+        if r % 50 == 0:
+            h.copy_(w.hidden)
+        e0.record(); g.replay(); e1.record(); torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        counts = {}
+        for t in range(n_live):
+            a = w.apps.get(int(token_slot[t]))
+            if a is not None and a.kind == W.KIND_SAE:
+                counts[a.group] = counts.get(a.group, 0) + 1
+        wbytes = sum(2.0 * w.d_model * w.groups[gi].d_sae for gi in counts)
+        flops = sum(2.0 * n * w.d_model * w.groups[gi].d_sae for gi, n in counts.items())
+        bound_ms = max(wbytes / (peaks["hbm_gbs"] * 1e9), flops / (peaks["bf16_tflops"] * 1e12)) * 1e3
+        rec.append((n_live, sum(counts.values()), len(counts), ms, bound_ms))
+        if r % 50 == 49 or r == n_replays - 1:
+            bad_status |= m.get_status()
+    m.destroy()
+    a = np.array(rec)
+    live = a[a[:, 2] > 0]
+    ratio = live[:, 4] / live[:, 3] if len(live) else np.array([0.0])
+    return {"workload": "replay (config 4)", "replays": n_replays, "status_or": bad_status,
+            "t_call_ms": {"min": float(a[:, 3].min()), "p50": float(np.median(a[:, 3])), "p90": float(np.quantile(a[:, 3], 0.9)),
+                          "max": float(a[:, 3].max())},
+            "empty_replay_ms": float(a[a[:, 0] == 0][:, 3].min()) if (a[:, 0] == 0).any() else None,
+            "bound_over_time": {"p10": float(np.quantile(ratio, 0.1)), "p50": float(np.median(ratio)),
+                                "p90": float(np.quantile(ratio, 0.9))},
+            "token_rows_per_s_mean": float(a[:, 0].sum() / (a[:, 3].sum() * 1e-3)),
+            "worst": {"n_live": int(a[a[:, 3].argmax(), 0]), "sae_rows": int(a[a[:, 3].argmax(), 1]),
+                      "groups_live": int(a[a[:, 3].argmax(), 2]), "ms": float(a[:, 3].max()),
+                      "bound_ms": float(a[a[:, 3].argmax(), 4])}}
+
+
+def run_workload(args):
+    """--workload X: one of the other configurations alone (not the contract line)."""
+    import paper_2607_22595_b200 as mixlib
+    from paper_2607_22595_b200 import _build
+    _build.build()
+    torch.cuda.set_device(0)
+    peaks = measured_peaks()
+    name = args.workload
+    if name == "sweep":
+        out = extras_sweep(peaks, mixlib)
+    elif name == "sae_heavy":
+        out = extras_sae("sae_heavy (config 2)", W.make_sae_heavy("cuda"), peaks, mixlib)
+    elif name == "sae_small":     # profiling case: weights (256 MiB) exceed L2, < 1 GiB on the device
+        out = extras_sae("sae_small (d=4096, d_sae=16384, 2 sets, T=256)",
+                         W.make_sae_heavy("cuda", d_sae=16384, T=256, R=16, G=2), peaks, mixlib)
+    elif name == "mixed":
+        out = extras_sae("mixed (config 3)", W.make_mixed("cuda"), peaks, mixlib)
+    elif name == "mixed_small":   # profiling case for the tensor-bound regime
+        out = extras_sae("mixed_small (d=5120, d_sae=8192, T=4096)",
+                         W.make_mixed("cuda", T=4096, d_sae=8192, R=32), peaks, mixlib)
+    elif name == "replay":
+        out = run_replay(peaks, mixlib, args.steps or 200)
+    else:
+        raise SystemExit("unknown workload %r" % name)
+    print(json.dumps(out), flush=True)
+
+
 def extras_sweep(peaks, mixlib):
     """Bandwidth kernels alone at a size that cannot hide in L2: d = 8192, T = 65536, every row hooked."""
     d, T = 8192, 65536
@@ -402,6 +482,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="mix", choices=["mix", "reference"])
     ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--workload", default="decode",
+                    help="decode (the contract line) | sweep | sae_heavy | sae_small | mixed | mixed_small | replay")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -409,6 +491,10 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank, world)
+        return
+    if args.workload != "decode":
+        if rank == 0:
+            run_workload(args)
         return
     if world > 1:
         import torch.distributed as dist

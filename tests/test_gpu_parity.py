@@ -346,3 +346,33 @@ def test_mixed_full_size_sampled_rows():
     assert np.array_equal(out["hidden"][unh], wh.hidden[unh])
     rows = sample_rows(wh, per_kind=16, seed=3)
     check_parity(wh, out, rows=rows)
+
+
+def test_replay_full_size_sampled_rows():
+    """Config 4 at full size (8 SAEs of 131072 x 8192, 32 GiB of weights), replay 1 (all 2048 rows
+    live) under the captured graph; the oracle checks every probe / steer / unhooked row of a sample
+    and SAE rows of two weight sets (their weights alone are copied to the host)."""
+    mixlib = _mixlib()
+    w = W.make_replay(DEV)
+    w.token_slot, w.T_live = W.replay_map(w, 1)
+    out = run_gpu(w, graph=True)
+    assert out["status"] == 0
+    keep = [0, 5]
+    wh = W.host(w, only_groups=keep)
+    rows, per_group = [], {}
+    for t in range(w.T_max):
+        a = w.apps.get(int(w.token_slot[t]))
+        if a is None or a.kind != W.KIND_SAE:
+            if t % 16 == 0:
+                rows.append(t)
+        elif a.group in keep and per_group.get(a.group, 0) < 3:
+            per_group[a.group] = per_group.get(a.group, 0) + 1
+            rows.append(t)
+    assert len(per_group) == 2
+    st = check_parity(wh, out, rows=rows, expect_status=None)
+    assert st["rows"] == len(rows)
+    # unhooked rows: all of them, bit for bit
+    unh = np.nonzero(w.token_slot < 0)[0]
+    assert np.array_equal(out["hidden"][unh], W.bits(w.hidden)[unh])
+    out["mix"].destroy()
+    torch.cuda.empty_cache()

@@ -105,8 +105,10 @@ def from_bits(a: np.ndarray, device="cpu"):
     return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).view(torch.bfloat16).to(device)
 
 
-def host(w: Workload) -> Workload:
-    """Copy of the workload with every tensor as a numpy array (bf16 -> uint16 bits)."""
+def host(w: Workload, only_groups=None) -> Workload:
+    """Copy of the workload with every tensor as a numpy array (bf16 -> uint16 bits).
+    `only_groups` keeps just those SAE weight sets (large configs: copying 32 GiB of weights to
+    the host to check a few rows is pointless); apps of the other sets then count as unhooked."""
     apps = {}
     for s, a in w.apps.items():
         if a.kind == KIND_PROBE:
@@ -118,7 +120,7 @@ def host(w: Workload) -> Workload:
     groups = {
         g: SaeWeights(sw.d_sae, sw.act, sw.k, bits(sw.W_enc), bits(sw.b_enc), bits(sw.W_dec),
                       bits(sw.theta), bits(sw.b_dec), sw.center_input)
-        for g, sw in w.groups.items()
+        for g, sw in w.groups.items() if only_groups is None or g in only_groups
     }
     return Workload(w.name, w.d_model, w.T_max, w.T_live, bits(w.hidden), w.token_slot.copy(),
                     apps, groups, w.n_slots_max, w.n_groups_max, w.C_max, w.k_max, w.r_max,
