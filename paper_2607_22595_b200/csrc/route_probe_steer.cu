@@ -32,17 +32,18 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
-// h + alpha v for one row; nvec = d / 8 16-byte vectors.
+// h + alpha v for one row; nvec = d / 8 16-byte vectors.  The `stride` threads that share the
+// row start at `first` (a warp: lane, 32; a CTA team: threadIdx.x, blockDim.x).
 __device__ __forceinline__ void steer_row(uint4* __restrict__ h, const uint4* __restrict__ v, float alpha,
-                                          int nvec, int lane) {
+                                          int nvec, int first, int stride) {
   constexpr int U = 4;
-  int i = lane;
-  for (; i + (U - 1) * 32 < nvec; i += U * 32) {
+  int i = first;
+  for (; i + (U - 1) * stride < nvec; i += U * stride) {
     uint4 hq[U], vq[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      hq[u] = __ldcs(h + i + u * 32);
-      vq[u] = __ldg(v + i + u * 32);
+      hq[u] = __ldcs(h + i + u * stride);
+      vq[u] = __ldg(v + i + u * stride);
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
@@ -51,10 +52,10 @@ __device__ __forceinline__ void steer_row(uint4* __restrict__ h, const uint4* __
       unpack8(vq[u], b);
 #pragma unroll
       for (int e = 0; e < 8; ++e) a[e] = fmaf(alpha, b[e], a[e]);
-      __stcs(h + i + u * 32, pack8(a));
+      __stcs(h + i + u * stride, pack8(a));
     }
   }
-  for (; i < nvec; i += 32) {
+  for (; i < nvec; i += stride) {
     float a[8], b[8];
     unpack8(__ldcs(h + i), a);
     unpack8(__ldg(v + i), b);
@@ -64,119 +65,73 @@ __device__ __forceinline__ void steer_row(uint4* __restrict__ h, const uint4* __
   }
 }
 
-// NC logits of one row against NC consecutive probe rows; every lane returns the full sums.
-template <int NC>
-__device__ __forceinline__ void probe_dots(const uint4* __restrict__ h, const uint4* __restrict__ W, int nvec,
-                                           int nc, int lane, float* out) {
-  float acc[NC];
+// Partial logits of RB rows against NC consecutive probe rows over this thread's share of the
+// columns; warp-reduced, so every lane of a warp returns the warp's sums.
+template <int RB, int NC>
+__device__ __forceinline__ void probe_dots(const uint4* const* __restrict__ h, const uint4* __restrict__ W, int nvec,
+                                           int nc, int first, int stride, float (*out)[NC]) {
+  float acc[RB][NC];
 #pragma unroll
-  for (int c = 0; c < NC; ++c) acc[c] = 0.f;
-  constexpr int U = (NC == 1) ? 4 : 1;
-  int i = lane;
-  for (; i + (U - 1) * 32 < nvec; i += U * 32) {
-    uint4 hq[U];
+  for (int r = 0; r < RB; ++r)
 #pragma unroll
-    for (int u = 0; u < U; ++u) hq[u] = __ldg(h + i + u * 32);
+    for (int c = 0; c < NC; ++c) acc[r][c] = 0.f;
+  constexpr int U = (NC == 1 && RB == 1) ? 4 : 1;
+  int i = first;
+  for (; i + (U - 1) * stride < nvec; i += U * stride) {
+    uint4 hq[U][RB];
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+#pragma unroll
+      for (int r = 0; r < RB; ++r) hq[u][r] = __ldg(h[r] + i + u * stride);
     uint4 wq[U][NC];
 #pragma unroll
     for (int u = 0; u < U; ++u)
 #pragma unroll
       for (int c = 0; c < NC; ++c)
-        if (c < nc) wq[u][c] = __ldg(W + (size_t)c * nvec + i + u * 32);
+        if (c < nc) wq[u][c] = __ldg(W + (size_t)c * nvec + i + u * stride);
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      float a[8];
-      unpack8(hq[u], a);
 #pragma unroll
       for (int c = 0; c < NC; ++c)
         if (c < nc) {
           float b[8];
           unpack8(wq[u][c], b);
 #pragma unroll
-          for (int e = 0; e < 8; ++e) acc[c] = fmaf(a[e], b[e], acc[c]);
+          for (int r = 0; r < RB; ++r) {
+            float a[8];
+            unpack8(hq[u][r], a);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[r][c] = fmaf(a[e], b[e], acc[r][c]);
+          }
         }
     }
   }
   if (U > 1) {
-    for (; i < nvec; i += 32) {
+    for (; i < nvec; i += stride) {
       float a[8], b[8];
-      unpack8(__ldg(h + i), a);
+      unpack8(__ldg(h[0] + i), a);
       unpack8(__ldg(W + i), b);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) acc[0] = fmaf(a[e], b[e], acc[0]);
+      for (int e = 0; e < 8; ++e) acc[0][0] = fmaf(a[e], b[e], acc[0][0]);
     }
   }
 #pragma unroll
-  for (int c = 0; c < NC; ++c) out[c] = warp_sum(acc[c]);
+  for (int r = 0; r < RB; ++r)
+#pragma unroll
+    for (int c = 0; c < NC; ++c) out[r][c] = warp_sum(acc[r][c]);
 }
 
-constexpr int kWarpsPerBlock = 8;
-
-__global__ void __launch_bounds__(kWarpsPerBlock * 32)
-probe_steer_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
-                   const AppEntry* __restrict__ apps, int n_slots, __nv_bfloat16* __restrict__ hidden, int d,
-                   float* __restrict__ scores, int C_max, unsigned* __restrict__ status) {
-  __shared__ float s_logit[kWarpsPerBlock][kMaxClasses];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int t = blockIdx.x * kWarpsPerBlock + warp;
-  const int n_live = min(T, __ldg(n_live_p));
-  if (t >= n_live) return;
-  const int s = __ldg(token_slot + t);
-  if (s == -1) return;
-  if (s < -1 || s >= n_slots) {
-    if (lane == 0) atomicOr(status, MIX_STATUS_BAD_SLOT);
-    return;
-  }
-  const AppEntry* e = apps + s;
-  const int4 head = __ldg(reinterpret_cast<const int4*>(e));   // valid, kind, n_classes, act
-  if (!head.x) {
-    if (lane == 0) atomicOr(status, MIX_STATUS_BAD_SLOT);
-    return;
-  }
-  const int nvec = d >> 3;
-  uint4* hrow = reinterpret_cast<uint4*>(hidden + (size_t)t * d);
-  if (head.y == MIX_STEER) {
-    const float alpha = __ldg(&e->alpha);
-    if (alpha == 0.f) return;                 // identity, and keeps the row bit-exact (-0.0 stays -0.0)
-    steer_row(hrow, reinterpret_cast<const uint4*>(__ldg(reinterpret_cast<const unsigned long long*>(&e->W))),
-              alpha, nvec, lane);
-    return;
-  }
-  if (head.y != MIX_PROBE || scores == nullptr) return;
-  const int C = head.z, act = head.w;
-  const uint4* W = reinterpret_cast<const uint4*>(__ldg(reinterpret_cast<const unsigned long long*>(&e->W)));
-  const float* b = reinterpret_cast<const float*>(__ldg(reinterpret_cast<const unsigned long long*>(&e->b)));
-  float* out = scores + (size_t)t * C_max;
-  if (C == 1) {
-    float z;
-    probe_dots<1>(hrow, W, nvec, 1, lane, &z);
-    if (lane == 0) {
-      if (b) z += __ldg(b);
-      out[0] = (act == MIX_ACT_NONE) ? z : 1.f / (1.f + expf(-z));
-    }
-    return;
-  }
-  for (int c0 = 0; c0 < C; c0 += 8) {
-    float z[8];
-    const int nc = min(8, C - c0);
-    probe_dots<8>(hrow, W + (size_t)c0 * nvec, nvec, nc, lane, z);
-    if (lane == 0) {
-#pragma unroll
-      for (int c = 0; c < 8; ++c)
-        if (c < nc) s_logit[warp][c0 + c] = z[c] + (b ? __ldg(b + c0 + c) : 0.f);
-    }
-  }
-  __syncwarp();
-  // C <= 64: lane handles classes lane and lane + 32
-  float z0 = lane < C ? s_logit[warp][lane] : -INFINITY;
-  float z1 = lane + 32 < C ? s_logit[warp][lane + 32] : -INFINITY;
+// Logits (bias included) of one row in `logit` -> scores.  One warp; C <= 64.
+__device__ __forceinline__ void finish_probe(const float* logit, int C, int act, float* __restrict__ out, int lane) {
+  float z0 = lane < C ? logit[lane] : -INFINITY;
+  float z1 = lane + 32 < C ? logit[lane + 32] : -INFINITY;
   if (act == MIX_ACT_SOFTMAX) {
     float m = fmaxf(z0, z1);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    float e0 = lane < C ? expf(z0 - m) : 0.f;
-    float e1 = lane + 32 < C ? expf(z1 - m) : 0.f;
-    float sum = warp_sum(e0 + e1);
+    const float e0 = lane < C ? expf(z0 - m) : 0.f;
+    const float e1 = lane + 32 < C ? expf(z1 - m) : 0.f;
+    const float sum = warp_sum(e0 + e1);
     z0 = e0 / sum;
     z1 = e1 / sum;
   } else if (act == MIX_ACT_SIGMOID) {
@@ -185,6 +140,173 @@ probe_steer_kernel(const int* __restrict__ token_slot, const int* __restrict__ n
   }
   if (lane < C) out[lane] = z0;
   if (lane + 32 < C) out[lane + 32] = z1;
+}
+
+struct RowApp {
+  int kind, C, act;     // kind 0: nothing to do
+  float alpha;
+  const uint4* W;
+  const float* b;
+};
+
+// Slot -> app for one row; flags bad slot ids.  `leader` is the one thread that may raise status.
+__device__ __forceinline__ RowApp lookup(int s, const AppEntry* __restrict__ apps, int n_slots,
+                                         unsigned* __restrict__ status, bool leader) {
+  RowApp r;
+  r.kind = 0;
+  if (s == -1) return r;
+  if (s < -1 || s >= n_slots) {
+    if (leader) atomicOr(status, MIX_STATUS_BAD_SLOT);
+    return r;
+  }
+  const AppEntry* e = apps + s;
+  const int4 head = __ldg(reinterpret_cast<const int4*>(e));   // valid, kind, n_classes, act
+  if (!head.x) {
+    if (leader) atomicOr(status, MIX_STATUS_BAD_SLOT);
+    return r;
+  }
+  r.kind = head.y;
+  r.C = head.z;
+  r.act = head.w;
+  r.alpha = __ldg(&e->alpha);
+  r.W = reinterpret_cast<const uint4*>(__ldg(reinterpret_cast<const unsigned long long*>(&e->W)));
+  r.b = reinterpret_cast<const float*>(__ldg(reinterpret_cast<const unsigned long long*>(&e->b)));
+  return r;
+}
+
+constexpr int kWarpsPerBlock = 8;
+constexpr int kRowsPerWarp = 4;
+
+// Large batches: a warp owns kRowsPerWarp consecutive rows.  Consecutive rows usually belong to
+// one request; when they share a multi-class probe the warp streams the probe matrix once for
+// all of them instead of once per row.
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+probe_steer_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
+                   const AppEntry* __restrict__ apps, int n_slots, __nv_bfloat16* __restrict__ hidden, int d,
+                   float* __restrict__ scores, int C_max, unsigned* __restrict__ status) {
+  __shared__ float s_logit[kWarpsPerBlock][kRowsPerWarp][kMaxClasses];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t0 = (blockIdx.x * kWarpsPerBlock + warp) * kRowsPerWarp;
+  const int n_live = min(T, __ldg(n_live_p));
+  if (t0 >= n_live) return;
+  const int nvec = d >> 3;
+  int my_slot = -1;
+  if (lane < kRowsPerWarp && t0 + lane < n_live) my_slot = __ldg(token_slot + t0 + lane);
+  int slot[kRowsPerWarp];
+#pragma unroll
+  for (int r = 0; r < kRowsPerWarp; ++r) slot[r] = __shfl_sync(0xffffffffu, my_slot, r);
+  bool same = t0 + kRowsPerWarp <= n_live;
+#pragma unroll
+  for (int r = 1; r < kRowsPerWarp; ++r) same = same && slot[r] == slot[0];
+  if (same && slot[0] >= 0 && scores != nullptr) {
+    const RowApp a = lookup(slot[0], apps, n_slots, status, lane == 0);
+    if (a.kind == MIX_PROBE && a.C > 1) {
+      const uint4* h[kRowsPerWarp];
+#pragma unroll
+      for (int r = 0; r < kRowsPerWarp; ++r) h[r] = reinterpret_cast<const uint4*>(hidden + (size_t)(t0 + r) * d);
+      for (int c0 = 0; c0 < a.C; c0 += 8) {
+        float z[kRowsPerWarp][8];
+        const int nc = min(8, a.C - c0);
+        probe_dots<kRowsPerWarp, 8>(h, a.W + (size_t)c0 * nvec, nvec, nc, lane, 32, z);
+        if (lane == 0) {
+#pragma unroll
+          for (int r = 0; r < kRowsPerWarp; ++r)
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+              if (c < nc) s_logit[warp][r][c0 + c] = z[r][c] + (a.b ? __ldg(a.b + c0 + c) : 0.f);
+        }
+      }
+      __syncwarp();
+#pragma unroll
+      for (int r = 0; r < kRowsPerWarp; ++r)
+        finish_probe(s_logit[warp][r], a.C, a.act, scores + (size_t)(t0 + r) * C_max, lane);
+      return;
+    }
+  }
+#pragma unroll 1
+  for (int r = 0; r < kRowsPerWarp; ++r) {
+    const int t = t0 + r;
+    if (t >= n_live) break;
+    const RowApp a = lookup(slot[r], apps, n_slots, status, lane == 0);
+    uint4* hrow = reinterpret_cast<uint4*>(hidden + (size_t)t * d);
+    if (a.kind == MIX_STEER) {
+      if (a.alpha != 0.f) steer_row(hrow, a.W, a.alpha, nvec, lane, 32);   // alpha = 0: row stays bit-exact
+    } else if (a.kind == MIX_PROBE && scores != nullptr) {
+      const uint4* h1[1] = {hrow};
+      float* out = scores + (size_t)t * C_max;
+      if (a.C == 1) {
+        float z[1][1];
+        probe_dots<1, 1>(h1, a.W, nvec, 1, lane, 32, z);
+        if (lane == 0) {
+          const float zz = z[0][0] + (a.b ? __ldg(a.b) : 0.f);
+          out[0] = (a.act == MIX_ACT_NONE) ? zz : 1.f / (1.f + expf(-zz));
+        }
+      } else {
+        for (int c0 = 0; c0 < a.C; c0 += 8) {
+          float z[1][8];
+          const int nc = min(8, a.C - c0);
+          probe_dots<1, 8>(h1, a.W + (size_t)c0 * nvec, nvec, nc, lane, 32, z);
+          if (lane == 0) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+              if (c < nc) s_logit[warp][0][c0 + c] = z[0][c] + (a.b ? __ldg(a.b + c0 + c) : 0.f);
+          }
+        }
+        __syncwarp();
+        finish_probe(s_logit[warp][0], a.C, a.act, out, lane);
+        __syncwarp();
+      }
+    }
+  }
+}
+
+// Small batches (decode): one CTA of NW warps per row, so a row's loads are all in flight at
+// once and the batch still fills the machine.  Control flow is uniform across the CTA.
+template <int NW>
+__global__ void __launch_bounds__(NW * 32)
+probe_steer_team_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
+                        const AppEntry* __restrict__ apps, int n_slots, __nv_bfloat16* __restrict__ hidden, int d,
+                        float* __restrict__ scores, int C_max, unsigned* __restrict__ status) {
+  __shared__ float s_part[NW][kMaxClasses];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t = blockIdx.x;
+  if (t >= min(T, __ldg(n_live_p))) return;
+  const RowApp a = lookup(__ldg(token_slot + t), apps, n_slots, status, threadIdx.x == 0);
+  const int nvec = d >> 3;
+  uint4* hrow = reinterpret_cast<uint4*>(hidden + (size_t)t * d);
+  if (a.kind == MIX_STEER) {
+    if (a.alpha != 0.f) steer_row(hrow, a.W, a.alpha, nvec, threadIdx.x, NW * 32);
+    return;
+  }
+  if (a.kind != MIX_PROBE || scores == nullptr) return;
+  const uint4* h1[1] = {hrow};
+  if (a.C == 1) {
+    float z[1][1];
+    probe_dots<1, 1>(h1, a.W, nvec, 1, threadIdx.x, NW * 32, z);
+    if (lane == 0) s_part[warp][0] = z[0][0];
+  } else {
+    for (int c0 = 0; c0 < a.C; c0 += 8) {
+      float z[1][8];
+      const int nc = min(8, a.C - c0);
+      probe_dots<1, 8>(h1, a.W + (size_t)c0 * nvec, nvec, nc, threadIdx.x, NW * 32, z);
+      if (lane == 0) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          if (c < nc) s_part[warp][c0 + c] = z[0][c];
+      }
+    }
+  }
+  __syncthreads();
+  if (warp == 0) {
+    for (int c = lane; c < a.C; c += 32) {
+      float z = a.b ? __ldg(a.b + c) : 0.f;
+#pragma unroll
+      for (int w = 0; w < NW; ++w) z += s_part[w][c];
+      s_part[0][c] = z;            // only this lane reads or writes column c from here on
+    }
+    __syncwarp();
+    finish_probe(s_part[0], a.C, a.act, scores + (size_t)t * C_max, lane);
+  }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -329,11 +451,20 @@ __global__ void fold_bias_kernel(const __nv_bfloat16* __restrict__ W_enc, const 
 
 }  // namespace
 
+constexpr int kTeamMaxRows = 2048;   // up to here one CTA per row keeps the whole GPU busy
+
 cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s) {
-  const int blocks = (c->cfg.T_max + kWarpsPerBlock - 1) / kWarpsPerBlock;
-  probe_steer_kernel<<<blocks, kWarpsPerBlock * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps,
-                                                            c->cfg.n_slots_max, hidden, c->cfg.d_model, scores,
-                                                            c->cfg.C_max, c->d_status);
+  if (c->cfg.T_max <= kTeamMaxRows) {
+    probe_steer_team_kernel<8><<<c->cfg.T_max, 8 * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps,
+                                                              c->cfg.n_slots_max, hidden, c->cfg.d_model, scores,
+                                                              c->cfg.C_max, c->d_status);
+  } else {
+    const int rows_per_block = kWarpsPerBlock * kRowsPerWarp;
+    const int blocks = (c->cfg.T_max + rows_per_block - 1) / rows_per_block;
+    probe_steer_kernel<<<blocks, kWarpsPerBlock * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps,
+                                                              c->cfg.n_slots_max, hidden, c->cfg.d_model, scores,
+                                                              c->cfg.C_max, c->d_status);
+  }
   return cudaGetLastError();
 }
 
