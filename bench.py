@@ -411,6 +411,18 @@ def run_mix(args, rank, world, local_rank):
     torch.cuda.synchronize()
     warm_us = e0.elapsed_time(e1) * 1e3 / (4 * min(R, 256))
 
+    # launch floor: the same graph with zero live rows (every CTA exits after one 4-byte load)
+    m.set_slot_map(torch.from_numpy(w.token_slot.copy()).cuda(), 0)
+    with torch.cuda.stream(stream):
+        g_warm.replay()
+        e0.record(stream)
+        for _ in range(4):
+            g_warm.replay()
+        e1.record(stream)
+    torch.cuda.synchronize()
+    floor_us = e0.elapsed_time(e1) * 1e3 / (4 * min(R, 256))
+    m.set_slot_map(torch.from_numpy(w.token_slot.copy()).cuda(), w.T_live)
+
     # end to end through the public API with host buffers
     K_e2e = min(K, 2000)
     h_in = torch.empty((T, d), dtype=torch.bfloat16).pin_memory(); h_in.copy_(w.hidden.cpu())
@@ -448,6 +460,7 @@ def run_mix(args, rank, world, local_rank):
         "config": {"workload": WORKLOAD, "l2": "inputs rotate over %d hidden buffers (%d MiB > 4x L2); weights (0.75 MiB) stay warm" % (R, R * T * d * 2 >> 20),
                    "graph": "CUDA-graph replay, %d steps per graph" % R, "probe_rows": rows_p, "steer_rows": rows_s,
                    "us_added_per_decode_step": ms_per_step * 1e3, "us_added_per_decode_step_warm_l2": warm_us,
+                   "us_per_step_zero_live_rows": floor_us,
                    "status_word": status},
         "clocks": clocks,
         "e2e": {"value": e2e_rows / e2e_s, "unit": UNIT, "h2d_bytes_per_step": T * d * 2 + 4 * T,

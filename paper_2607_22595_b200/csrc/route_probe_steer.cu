@@ -159,141 +159,199 @@ __device__ __forceinline__ RowApp lookup(int s, const AppEntry* __restrict__ app
     if (leader) atomicOr(status, MIX_STATUS_BAD_SLOT);
     return r;
   }
-  const AppEntry* e = apps + s;
-  const int4 head = __ldg(reinterpret_cast<const int4*>(e));   // valid, kind, n_classes, act
-  if (!head.x) {
+  // the whole 48-byte entry in three independent 16-byte loads (one round trip)
+  const int4* e = reinterpret_cast<const int4*>(apps + s);
+  const int4 q0 = __ldg(e), q1 = __ldg(e + 1), q2 = __ldg(e + 2);
+  if (!q0.x) {                                   // valid
     if (leader) atomicOr(status, MIX_STATUS_BAD_SLOT);
     return r;
   }
-  r.kind = head.y;
-  r.C = head.z;
-  r.act = head.w;
-  r.alpha = __ldg(&e->alpha);
-  r.W = reinterpret_cast<const uint4*>(__ldg(reinterpret_cast<const unsigned long long*>(&e->W)));
-  r.b = reinterpret_cast<const float*>(__ldg(reinterpret_cast<const unsigned long long*>(&e->b)));
+  r.kind = q0.y;
+  r.C = q0.z;
+  r.act = q0.w;
+  r.alpha = __int_as_float(q1.x);
+  r.W = reinterpret_cast<const uint4*>(((unsigned long long)(unsigned)q2.y << 32) | (unsigned)q2.x);
+  r.b = reinterpret_cast<const float*>(((unsigned long long)(unsigned)q2.w << 32) | (unsigned)q2.z);
   return r;
 }
 
-constexpr int kWarpsPerBlock = 8;
-constexpr int kRowsPerWarp = 4;
+constexpr int kWarpsPerBlock = 8;      // = rows per CTA of the large-batch kernel
+constexpr int kRowGroup = 4;           // rows that share one pass over a probe matrix
 
-// Large batches: a warp owns kRowsPerWarp consecutive rows.  Consecutive rows usually belong to
-// one request; when they share a multi-class probe the warp streams the probe matrix once for
-// all of them instead of once per row.
-__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+// One row, one warp: steer, single-class probe, or multi-class probe.
+__device__ __forceinline__ void warp_row(const RowApp& a, __nv_bfloat16* __restrict__ hidden, int t, int d,
+                                         float* __restrict__ scores, int C_max, float* s_logit, int lane) {
+  const int nvec = d >> 3;
+  uint4* hrow = reinterpret_cast<uint4*>(hidden + (size_t)t * d);
+  if (a.kind == MIX_STEER) {
+    if (a.alpha != 0.f) steer_row(hrow, a.W, a.alpha, nvec, lane, 32);   // alpha = 0: row stays bit-exact
+    return;
+  }
+  if (a.kind != MIX_PROBE || scores == nullptr) return;
+  const uint4* h1[1] = {hrow};
+  float* out = scores + (size_t)t * C_max;
+  if (a.C == 1) {
+    float z[1][1];
+    probe_dots<1, 1>(h1, a.W, nvec, 1, lane, 32, z);
+    if (lane == 0) {
+      const float zz = z[0][0] + (a.b ? __ldg(a.b) : 0.f);
+      out[0] = (a.act == MIX_ACT_NONE) ? zz : 1.f / (1.f + expf(-zz));
+    }
+    return;
+  }
+  for (int c0 = 0; c0 < a.C; c0 += 8) {
+    float z[1][8];
+    const int nc = min(8, a.C - c0);
+    probe_dots<1, 8>(h1, a.W + (size_t)c0 * nvec, nvec, nc, lane, 32, z);
+    if (lane == 0) {
+#pragma unroll
+      for (int c = 0; c < 8; ++c)
+        if (c < nc) s_logit[c0 + c] = z[0][c] + (a.b ? __ldg(a.b + c0 + c) : 0.f);
+    }
+  }
+  __syncwarp();
+  finish_probe(s_logit, a.C, a.act, out, lane);
+}
+
+// Large batches: a CTA owns 8 consecutive rows, one warp per row.  Consecutive rows usually
+// belong to one request; when all 8 share a multi-class probe the CTA switches to a
+// cooperative pass (columns split over the warps, kRowGroup rows x 4 classes per pass) that
+// streams the probe matrix from L2 twice per 8 rows instead of eight times.
+__global__ void __launch_bounds__(kWarpsPerBlock * 32, 3)
 probe_steer_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
                    const AppEntry* __restrict__ apps, int n_slots, __nv_bfloat16* __restrict__ hidden, int d,
                    float* __restrict__ scores, int C_max, unsigned* __restrict__ status) {
-  __shared__ float s_logit[kWarpsPerBlock][kRowsPerWarp][kMaxClasses];
+  __shared__ float s_part[kWarpsPerBlock][kWarpsPerBlock][kMaxClasses];   // [warp][row][class]
+  __shared__ int s_slot[kWarpsPerBlock];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int t0 = (blockIdx.x * kWarpsPerBlock + warp) * kRowsPerWarp;
+  const int t0 = blockIdx.x * kWarpsPerBlock;
   const int n_live = min(T, __ldg(n_live_p));
   if (t0 >= n_live) return;
+  const int t = t0 + warp;
+  const int my_slot = t < n_live ? __ldg(token_slot + t) : -1;
+  if (lane == 0) s_slot[warp] = my_slot;
+  __syncthreads();
+  bool same = t0 + kWarpsPerBlock <= n_live && s_slot[0] >= 0 && scores != nullptr;
+#pragma unroll
+  for (int r = 1; r < kWarpsPerBlock; ++r) same = same && s_slot[r] == s_slot[0];
+  const RowApp a = lookup(my_slot, apps, n_slots, status, lane == 0);
+  if (!(same && a.kind == MIX_PROBE && a.C > 1)) {       // CTA-uniform: every warp sees the same slots
+    if (t < n_live) warp_row(a, hidden, t, d, scores, C_max, s_part[warp][0], lane);
+    return;
+  }
   const int nvec = d >> 3;
-  int my_slot = -1;
-  if (lane < kRowsPerWarp && t0 + lane < n_live) my_slot = __ldg(token_slot + t0 + lane);
-  int slot[kRowsPerWarp];
+  for (int rg = 0; rg < kWarpsPerBlock; rg += kRowGroup) {
+    const uint4* h[kRowGroup];
 #pragma unroll
-  for (int r = 0; r < kRowsPerWarp; ++r) slot[r] = __shfl_sync(0xffffffffu, my_slot, r);
-  bool same = t0 + kRowsPerWarp <= n_live;
+    for (int r = 0; r < kRowGroup; ++r) h[r] = reinterpret_cast<const uint4*>(hidden + (size_t)(t0 + rg + r) * d);
+    for (int c0 = 0; c0 < a.C; c0 += 4) {
+      float z[kRowGroup][4];
+      const int nc = min(4, a.C - c0);
+      probe_dots<kRowGroup, 4>(h, a.W + (size_t)c0 * nvec, nvec, nc, threadIdx.x, kWarpsPerBlock * 32, z);
+      if (lane == 0) {
 #pragma unroll
-  for (int r = 1; r < kRowsPerWarp; ++r) same = same && slot[r] == slot[0];
-  if (same && slot[0] >= 0 && scores != nullptr) {
-    const RowApp a = lookup(slot[0], apps, n_slots, status, lane == 0);
-    if (a.kind == MIX_PROBE && a.C > 1) {
-      const uint4* h[kRowsPerWarp];
+        for (int r = 0; r < kRowGroup; ++r)
 #pragma unroll
-      for (int r = 0; r < kRowsPerWarp; ++r) h[r] = reinterpret_cast<const uint4*>(hidden + (size_t)(t0 + r) * d);
-      for (int c0 = 0; c0 < a.C; c0 += 8) {
-        float z[kRowsPerWarp][8];
-        const int nc = min(8, a.C - c0);
-        probe_dots<kRowsPerWarp, 8>(h, a.W + (size_t)c0 * nvec, nvec, nc, lane, 32, z);
-        if (lane == 0) {
-#pragma unroll
-          for (int r = 0; r < kRowsPerWarp; ++r)
-#pragma unroll
-            for (int c = 0; c < 8; ++c)
-              if (c < nc) s_logit[warp][r][c0 + c] = z[r][c] + (a.b ? __ldg(a.b + c0 + c) : 0.f);
-        }
-      }
-      __syncwarp();
-#pragma unroll
-      for (int r = 0; r < kRowsPerWarp; ++r)
-        finish_probe(s_logit[warp][r], a.C, a.act, scores + (size_t)(t0 + r) * C_max, lane);
-      return;
-    }
-  }
-#pragma unroll 1
-  for (int r = 0; r < kRowsPerWarp; ++r) {
-    const int t = t0 + r;
-    if (t >= n_live) break;
-    const RowApp a = lookup(slot[r], apps, n_slots, status, lane == 0);
-    uint4* hrow = reinterpret_cast<uint4*>(hidden + (size_t)t * d);
-    if (a.kind == MIX_STEER) {
-      if (a.alpha != 0.f) steer_row(hrow, a.W, a.alpha, nvec, lane, 32);   // alpha = 0: row stays bit-exact
-    } else if (a.kind == MIX_PROBE && scores != nullptr) {
-      const uint4* h1[1] = {hrow};
-      float* out = scores + (size_t)t * C_max;
-      if (a.C == 1) {
-        float z[1][1];
-        probe_dots<1, 1>(h1, a.W, nvec, 1, lane, 32, z);
-        if (lane == 0) {
-          const float zz = z[0][0] + (a.b ? __ldg(a.b) : 0.f);
-          out[0] = (a.act == MIX_ACT_NONE) ? zz : 1.f / (1.f + expf(-zz));
-        }
-      } else {
-        for (int c0 = 0; c0 < a.C; c0 += 8) {
-          float z[1][8];
-          const int nc = min(8, a.C - c0);
-          probe_dots<1, 8>(h1, a.W + (size_t)c0 * nvec, nvec, nc, lane, 32, z);
-          if (lane == 0) {
-#pragma unroll
-            for (int c = 0; c < 8; ++c)
-              if (c < nc) s_logit[warp][0][c0 + c] = z[0][c] + (a.b ? __ldg(a.b + c0 + c) : 0.f);
-          }
-        }
-        __syncwarp();
-        finish_probe(s_logit[warp][0], a.C, a.act, out, lane);
-        __syncwarp();
+          for (int c = 0; c < 4; ++c)
+            if (c < nc) s_part[warp][rg + r][c0 + c] = z[r][c];
       }
     }
   }
+  __syncthreads();
+  // warp r finishes row r: sum the 8 column shares, add the bias, activate
+  for (int c = lane; c < a.C; c += 32) {
+    float z = a.b ? __ldg(a.b + c) : 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarpsPerBlock; ++w) z += s_part[w][warp][c];
+    s_part[0][warp][c] = z;     // s_part[*][warp][*] is read and written by this warp only
+  }
+  __syncwarp();
+  finish_probe(s_part[0][warp], a.C, a.act, scores + (size_t)t * C_max, lane);
 }
 
-// Small batches (decode): one CTA of NW warps per row, so a row's loads are all in flight at
-// once and the batch still fills the machine.  Control flow is uniform across the CTA.
+// Small batches (decode): one CTA of NW warps per row, the row held in registers (up to kTeamVec
+// 16-byte vectors per thread).  The row's loads are issued as soon as the slot id is known to be
+// >= 0, in parallel with the app-table lookup, so a cold row costs two dependent round trips
+// (slot, then entry + data) instead of three.  Control flow is uniform across the CTA.
+constexpr int kTeamVec = 4;     // NW * 32 * kTeamVec * 8 >= d_model: 8192 columns at NW = 8
+
 template <int NW>
 __global__ void __launch_bounds__(NW * 32)
 probe_steer_team_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
                         const AppEntry* __restrict__ apps, int n_slots, __nv_bfloat16* __restrict__ hidden, int d,
                         float* __restrict__ scores, int C_max, unsigned* __restrict__ status) {
   __shared__ float s_part[NW][kMaxClasses];
+  constexpr int NT = NW * 32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t = blockIdx.x;
   if (t >= min(T, __ldg(n_live_p))) return;
-  const RowApp a = lookup(__ldg(token_slot + t), apps, n_slots, status, threadIdx.x == 0);
+  const int slot = __ldg(token_slot + t);
+  if (slot == -1) return;
   const int nvec = d >> 3;
   uint4* hrow = reinterpret_cast<uint4*>(hidden + (size_t)t * d);
+  uint4 hq[kTeamVec];
+  if (slot >= 0 && slot < n_slots) {
+#pragma unroll
+    for (int u = 0; u < kTeamVec; ++u) {
+      const int v = threadIdx.x + u * NT;
+      if (v < nvec) hq[u] = __ldcs(hrow + v);
+    }
+  }
+  const RowApp a = lookup(slot, apps, n_slots, status, threadIdx.x == 0);
   if (a.kind == MIX_STEER) {
-    if (a.alpha != 0.f) steer_row(hrow, a.W, a.alpha, nvec, threadIdx.x, NW * 32);
+    if (a.alpha == 0.f) return;                  // identity; the row stays bit-exact
+    uint4 vq[kTeamVec];
+#pragma unroll
+    for (int u = 0; u < kTeamVec; ++u) {
+      const int v = threadIdx.x + u * NT;
+      if (v < nvec) vq[u] = __ldg(a.W + v);
+    }
+#pragma unroll
+    for (int u = 0; u < kTeamVec; ++u) {
+      const int v = threadIdx.x + u * NT;
+      if (v < nvec) {
+        float x[8], y[8];
+        unpack8(hq[u], x);
+        unpack8(vq[u], y);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) x[e] = fmaf(a.alpha, y[e], x[e]);
+        __stcs(hrow + v, pack8(x));
+      }
+    }
     return;
   }
   if (a.kind != MIX_PROBE || scores == nullptr) return;
-  const uint4* h1[1] = {hrow};
-  if (a.C == 1) {
-    float z[1][1];
-    probe_dots<1, 1>(h1, a.W, nvec, 1, threadIdx.x, NW * 32, z);
-    if (lane == 0) s_part[warp][0] = z[0][0];
-  } else {
-    for (int c0 = 0; c0 < a.C; c0 += 8) {
-      float z[1][8];
-      const int nc = min(8, a.C - c0);
-      probe_dots<1, 8>(h1, a.W + (size_t)c0 * nvec, nvec, nc, threadIdx.x, NW * 32, z);
-      if (lane == 0) {
+  for (int c0 = 0; c0 < a.C; c0 += 4) {
+    const int nc = min(4, a.C - c0);
+    uint4 wq[4][kTeamVec];
 #pragma unroll
-        for (int c = 0; c < 8; ++c)
-          if (c < nc) s_part[warp][c0 + c] = z[0][c];
+    for (int c = 0; c < 4; ++c)
+#pragma unroll
+      for (int u = 0; u < kTeamVec; ++u) {
+        const int v = threadIdx.x + u * NT;
+        if (c < nc && v < nvec) wq[c][u] = __ldg(a.W + (size_t)(c0 + c) * nvec + v);
       }
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int u = 0; u < kTeamVec; ++u) {
+      const int v = threadIdx.x + u * NT;
+      if (v < nvec) {
+        float x[8];
+        unpack8(hq[u], x);
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          if (c < nc) {
+            float y[8];
+            unpack8(wq[c][u], y);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[c] = fmaf(x[e], y[e], acc[c]);
+          }
+      }
+    }
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const float z = warp_sum(acc[c]);
+      if (lane == 0 && c < nc) s_part[warp][c0 + c] = z;
     }
   }
   __syncthreads();
@@ -459,8 +517,7 @@ cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float
                                                               c->cfg.n_slots_max, hidden, c->cfg.d_model, scores,
                                                               c->cfg.C_max, c->d_status);
   } else {
-    const int rows_per_block = kWarpsPerBlock * kRowsPerWarp;
-    const int blocks = (c->cfg.T_max + rows_per_block - 1) / rows_per_block;
+    const int blocks = (c->cfg.T_max + kWarpsPerBlock - 1) / kWarpsPerBlock;
     probe_steer_kernel<<<blocks, kWarpsPerBlock * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps,
                                                               c->cfg.n_slots_max, hidden, c->cfg.d_model, scores,
                                                               c->cfg.C_max, c->d_status);

@@ -58,6 +58,17 @@ def test_mixed_small():
     assert st["rows"] == 1500
 
 
+@pytest.mark.parametrize("t_live", [2601, 1999])
+def test_mixed_large_batch_kernel(t_live):
+    # T_max > 2048 selects the warp-per-row kernel and its cooperative multi-class probe pass;
+    # 2601 rows leave a ragged last CTA, and a live count below T_max cuts a request in two
+    w = W.make_mixed(DEV, d=320, T=2601, R=48, d_sae=1024, cap=300, mu=4.0, edit_hint=oracle_edit_hint)
+    w.T_live = t_live
+    out = run_gpu(w)
+    st = check_parity(W.host(w), out)
+    assert st["rows"] == 2601
+
+
 def test_replay_small_fresh_maps_one_capture():
     mixlib = _mixlib()
     w = W.make_replay(DEV, d=256, T_max=512, d_sae=4096, k=16, G=3, n_probe=6, n_steer=4, n_sae_slots=9, n_edit=6)
