@@ -61,6 +61,7 @@ enum { MIX_PROBE = 1, MIX_STEER = 2, MIX_SAE = 3 };                    /* app ki
 enum { MIX_ACT_SIGMOID = 0, MIX_ACT_SOFTMAX = 1, MIX_ACT_NONE = 2 };   /* probe activations */
 enum { MIX_SAE_RELU = 0, MIX_SAE_JUMPRELU = 1, MIX_SAE_TOPK = 2 };     /* SAE activations */
 enum { MIX_EDIT_CLAMP = 0, MIX_EDIT_ABLATE = 1 };                      /* per-feature edits */
+enum { MIX_GATE_GE = 0, MIX_GATE_LT = 1 };                             /* gate comparisons */
 
 /* bits of the device status word (mix_get_status) */
 enum {
@@ -169,6 +170,24 @@ int mix_update_steer_alpha(mix_ctx* ctx, int slot, float alpha, void* stream);
 int mix_update_sae_edits(mix_ctx* ctx, int slot, int n_edit, const int* idx, const float* val,
                          const unsigned char* mode, void* stream);
 
+/* Conditional write driven by an earlier read (paper, Section 3 "Conditional Write": the
+   condition can depend on activations at another layer; Section 4.1, the example
+   gate="probe(layer=18) >= 0"; Section 4.2 "State and dataflow" / "Activation and control
+   semantics": a buffer written at one hook decides, on the device, whether a function at a
+   later hook runs).  After this call the app in `slot` applies to token row t only if
+       scores[t * row_stride + column]  >=  threshold      (MIX_GATE_GE)
+       scores[t * row_stride + column]  <   threshold      (MIX_GATE_LT)
+   and the row passes through untouched otherwise (a NaN score fails either comparison).
+   `scores` is a device fp32 buffer indexed by token row, typically the scores_out of a
+   mix_apply() at an earlier layer of the same forward pass (use MIX_ACT_NONE probes to gate on
+   the raw logit); it is read when the later mix_apply() runs, so both calls can sit in one
+   captured graph.  scores == NULL removes the gate.  Registering the slot again also removes
+   it.  Stream-ordered, not captured.  Works for every app kind (a gated probe writes no score
+   for rows whose gate is closed).  Errors: OUT_OF_RANGE (slot), INVALID_ARG (slot not
+   registered, bad cmp, row_stride < 1, column outside [0, row_stride)). */
+int mix_set_gate(mix_ctx* ctx, int slot, const float* scores, int row_stride, int column, int cmp, float threshold,
+                 void* stream);
+
 /* Install the token->slot map for the next mix_apply calls: token_slot int32[T_live]
    (host if src_is_device == 0, else device), -1 = no app.  Rows >= T_live are pass-through.
    One async copy + a 4-byte store into fixed device buffers; never captured in a graph.
@@ -202,14 +221,16 @@ int mix_apply(mix_ctx* ctx, void* hidden, int T, float* scores_out, void* stream
    Synchronises `stream`. */
 int mix_get_status(mix_ctx* ctx, unsigned* bits, void* stream);
 
-/* Number of kernels one mix_apply() call launches on this context (fixed at mix_create). */
+/* Number of kernels one mix_apply() call launches on this context (fixed at mix_create):
+   1 without SAE weight sets, else 8 (6 with MIX_FLAG_ENCODE_SIMT). */
 int mix_launches_per_apply(const mix_ctx* ctx);
 
 /* Per-kernel timing taps (profiling only; do not use while capturing a graph).  events: HOST
    array of mix_launches_per_apply() + 1 cudaEvent_t handles created by the caller with timing
    enabled, or NULL to switch the taps off.  Every later mix_apply() records events[0] before
    its first kernel and events[i] after its i-th kernel, on the call's stream; the array is
-   copied.  Kernel order: probe_steer, route, pack, encode, select, decode. */
+   copied.  Kernel order: probe_steer, route, pack, encode, merge, encode (flagged row tiles),
+   select, decode; with MIX_FLAG_ENCODE_SIMT: probe_steer, route, pack, encode, select, decode. */
 int mix_set_stage_events(mix_ctx* ctx, void* const* events);
 
 /* Test / profiling taps into the SAE workspace after a mix_apply (device pointers owned by

@@ -36,6 +36,7 @@ KIND_PROBE, KIND_STEER, KIND_SAE = 1, 2, 3
 ACT_SIGMOID, ACT_SOFTMAX, ACT_NONE = 0, 1, 2
 SAE_RELU, SAE_JUMPRELU, SAE_TOPK = 0, 1, 2
 EDIT_CLAMP, EDIT_ABLATE = 0, 1
+GATE_GE, GATE_LT = 0, 1
 
 _CHUNK = 4096   # weight rows converted to float64 at a time
 
@@ -96,6 +97,22 @@ def probe_scores(h: np.ndarray, W: np.ndarray, b: Optional[np.ndarray], act: int
 def steer(h: np.ndarray, v: np.ndarray, alpha: float) -> np.ndarray:
     """h' = h + alpha * v   (alpha is an fp32 parameter, used at its exact value)."""
     return h + float(np.float32(alpha)) * v
+
+
+# ---------------------------------------------------------------------------
+# conditional write, activation-driven  (Section 3, "Conditional Write"; Section 4.1, the
+# gate="probe(layer=18) >= 0" example; Section 4.2, "Activation and control semantics")
+# ---------------------------------------------------------------------------
+def gate_open(gate, t: int) -> bool:
+    """The app applies to row t iff cmp(scores[t, column], threshold).  scores and threshold are
+    fp32 values compared exactly; a NaN score fails either comparison."""
+    v = float(np.float32(np.asarray(gate.scores)[t, gate.column]))
+    thr = float(np.float32(gate.threshold))
+    if gate.cmp == GATE_GE:
+        return v >= thr
+    if gate.cmp == GATE_LT:
+        return v < thr
+    raise ValueError("unknown gate comparison %r" % gate.cmp)
 
 
 # ---------------------------------------------------------------------------
@@ -213,7 +230,8 @@ def apply_hook(w, rows: Optional[Iterable[int]] = None, keep_z: bool = False,
     """Evaluate the hook on a host workload (numpy arrays; bf16 as uint16 bits).
 
     for each row t:  s = token_slot[t] if t < T_live else -1
-      s < 0, out of range or unregistered  -> pass-through (bits unchanged, no score)
+      s < 0, out of range, unregistered, or the slot's gate closed for row t
+                                           -> pass-through (bits unchanged, no score)
       probe  -> scores[t, :C]; hidden unchanged
       steer  -> h + alpha v
       SAE    -> encode, activate, edit, decode (+ error term)
@@ -231,6 +249,8 @@ def apply_hook(w, rows: Optional[Iterable[int]] = None, keep_z: bool = False,
         app = w.apps.get(s) if 0 <= s < w.n_slots_max else None
         if app is not None and app.kind == KIND_SAE and app.group not in w.groups:
             app = None
+        if app is not None and getattr(app, "gate", None) is not None and not gate_open(app.gate, t):
+            app = None                       # gate closed: the row passes through
         if app is None:
             res.kind[t] = 0
             res.modified[t] = False

@@ -19,12 +19,13 @@ MIX_PROBE, MIX_STEER, MIX_SAE = 1, 2, 3
 MIX_ACT_SIGMOID, MIX_ACT_SOFTMAX, MIX_ACT_NONE = 0, 1, 2
 MIX_SAE_RELU, MIX_SAE_JUMPRELU, MIX_SAE_TOPK = 0, 1, 2
 MIX_EDIT_CLAMP, MIX_EDIT_ABLATE = 0, 1
+MIX_GATE_GE, MIX_GATE_LT = 0, 1
 MIX_STATUS_BAD_SLOT, MIX_STATUS_BAD_GROUP, MIX_STATUS_WAIT_TIMEOUT, MIX_STATUS_TOPK_GENERAL = 1, 2, 4, 8
 MIX_FLAG_ENCODE_SIMT = 1
 
 EXPORTS = [
     "mix_create", "mix_destroy", "mix_last_error", "mix_register_sae_weights", "mix_unregister_sae_weights",
-    "mix_register_app", "mix_unregister_app", "mix_update_steer_alpha", "mix_update_sae_edits",
+    "mix_register_app", "mix_unregister_app", "mix_set_gate", "mix_update_steer_alpha", "mix_update_sae_edits",
     "mix_set_slot_map", "mix_set_request_map", "mix_set_feature_out", "mix_apply", "mix_get_status",
     "mix_launches_per_apply", "mix_set_stage_events", "mix_debug_workspace", "mix_sae_apply_static",
 ]
@@ -82,6 +83,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.mix_unregister_sae_weights.argtypes = [vp, ci, vp]
     lib.mix_register_app.argtypes = [vp, ci, ci, vp, vp]
     lib.mix_unregister_app.argtypes = [vp, ci, vp]
+    lib.mix_set_gate.argtypes = [vp, ci, vp, ci, ci, ci, C.c_float, vp]
     lib.mix_update_steer_alpha.argtypes = [vp, ci, C.c_float, vp]
     lib.mix_update_sae_edits.argtypes = [vp, ci, ci, vp, vp, vp, vp]
     lib.mix_set_slot_map.argtypes = [vp, vp, ci, ci, vp]
@@ -185,6 +187,17 @@ class Mix:
         self._check(self.lib.mix_unregister_app(self.ctx, slot, _stream(stream)))
         self._keep.pop(("a", slot), None)
 
+    def set_gate(self, slot, scores, column=0, cmp=MIX_GATE_GE, threshold=0.0, stream=None):
+        """Gate the app in `slot` on scores[t, column] (CUDA fp32 [T_max, stride]); scores=None removes it."""
+        if scores is None:
+            self._check(self.lib.mix_set_gate(self.ctx, slot, None, 1, 0, 0, 0.0, _stream(stream)))
+            self._keep.pop(("gate", slot), None)
+            return
+        assert scores.dtype == torch.float32 and scores.dim() == 2
+        self._check(self.lib.mix_set_gate(self.ctx, slot, _ptr(scores), int(scores.shape[1]), int(column), int(cmp),
+                                          float(threshold), _stream(stream)))
+        self._keep[("gate", slot)] = scores
+
     def update_steer_alpha(self, slot, alpha, stream=None):
         self._check(self.lib.mix_update_steer_alpha(self.ctx, slot, float(alpha), _stream(stream)))
 
@@ -234,7 +247,13 @@ class Mix:
     def launches_per_apply(self) -> int:
         return int(self.lib.mix_launches_per_apply(self.ctx))
 
-    STAGES = ["probe_steer", "route", "pack", "encode", "select", "decode"]
+    @property
+    def STAGES(self):
+        if self.cfg.n_groups_max == 0:
+            return ["probe_steer"]
+        if self.cfg.flags & MIX_FLAG_ENCODE_SIMT:
+            return ["probe_steer", "route", "pack", "encode", "select", "decode"]
+        return ["probe_steer", "route", "pack", "encode", "merge", "encode_flagged", "select", "decode"]
 
     def set_stage_events(self, events=None):
         """events: list of launches_per_apply() + 1 torch.cuda.Event(enable_timing=True), or None."""

@@ -60,11 +60,12 @@ cudaError_t dev_alloc(T** p, size_t n) {
 }
 
 void free_all(mix_ctx* c) {
-  cudaFree(c->d_token_slot); cudaFree(c->d_n_live); cudaFree(c->d_apps); cudaFree(c->d_groups);
+  cudaFree(c->d_token_slot); cudaFree(c->d_n_live); cudaFree(c->d_apps); cudaFree(c->d_groups); cudaFree(c->d_gates);
   cudaFree(c->d_edit_idx); cudaFree(c->d_edit_val); cudaFree(c->d_edit_mode); cudaFree(c->d_status);
   cudaFree(c->d_tmp_req); cudaFree(c->d_tmp_req_slot); cudaFree(c->d_panel); cudaFree(c->d_panel_row);
   cudaFree(c->d_mtile_group); cudaFree(c->d_route); cudaFree(c->d_z); cudaFree(c->d_topk_idx);
-  cudaFree(c->d_topk_val); cudaFree(c->d_tmap_w);
+  cudaFree(c->d_topk_val); cudaFree(c->d_tmap_w); cudaFree(c->d_cand_val); cudaFree(c->d_cand_idx);
+  cudaFree(c->d_cand_ninth); cudaFree(c->d_row_flag); cudaFree(c->d_mtile_flag); cudaFree(c->d_n_flagged);
   if (c->owned_b_eff)
     for (int g = 0; g < c->cfg.n_groups_max; ++g) cudaFree(c->owned_b_eff[g]);
   free(c->owned_b_eff); free(c->h_apps); free(c->h_groups);
@@ -139,6 +140,7 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
   ok = ok && dev_alloc(&c->d_n_live, 1) == cudaSuccess;
   ok = ok && dev_alloc(&c->d_apps, NS) == cudaSuccess;
   ok = ok && dev_alloc(&c->d_groups, G > 0 ? G : 1) == cudaSuccess;
+  ok = ok && dev_alloc(&c->d_gates, NS) == cudaSuccess;
   ok = ok && dev_alloc(&c->d_edit_idx, (size_t)NS * c->cfg.r_max) == cudaSuccess;
   ok = ok && dev_alloc(&c->d_edit_val, (size_t)NS * c->cfg.r_max) == cudaSuccess;
   ok = ok && dev_alloc(&c->d_edit_mode, (size_t)NS * c->cfg.r_max) == cudaSuccess;
@@ -156,12 +158,23 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
     ok = ok && dev_alloc(&c->d_topk_idx, P * (size_t)c->cfg.k_max) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_topk_val, P * (size_t)c->cfg.k_max) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_tmap_w, G) == cudaSuccess;
+    if (!(cfg->flags & MIX_FLAG_ENCODE_SIMT)) {
+      c->cand_tiles = (int)(cfg->d_sae_max / kTileN);
+      const size_t nc = P * (size_t)c->cand_tiles;
+      ok = ok && dev_alloc(&c->d_cand_val, nc * kCandPerTile) == cudaSuccess;
+      ok = ok && dev_alloc(&c->d_cand_idx, nc * kCandPerTile) == cudaSuccess;
+      ok = ok && dev_alloc(&c->d_cand_ninth, nc) == cudaSuccess;
+      ok = ok && dev_alloc(&c->d_row_flag, P) == cudaSuccess;
+      ok = ok && dev_alloc(&c->d_mtile_flag, P / kTileM) == cudaSuccess;
+      ok = ok && dev_alloc(&c->d_n_flagged, 1) == cudaSuccess;
+    }
   }
   if (!ok) { cudaGetLastError(); free_all(c); free(c); return MIX_ERR_NO_MEMORY; }
   e = cudaMemset(c->d_token_slot, 0xff, T * sizeof(int));
   if (e == cudaSuccess) e = cudaMemset(c->d_n_live, 0, sizeof(int));
   if (e == cudaSuccess) e = cudaMemset(c->d_apps, 0, NS * sizeof(AppEntry));
   if (e == cudaSuccess) e = cudaMemset(c->d_groups, 0, (G > 0 ? G : 1) * sizeof(GroupEntry));
+  if (e == cudaSuccess) e = cudaMemset(c->d_gates, 0, NS * sizeof(GateEntry));
   if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, sizeof(unsigned));
   if (e == cudaSuccess && G > 0) {
     e = cudaMemset(c->d_panel, 0, (size_t)c->panel_rows_cap * cfg->d_model * sizeof(__nv_bfloat16));
@@ -306,11 +319,44 @@ int mix_unregister_app(mix_ctx* c, int slot, void* stream) {
   return MIX_OK;
 }
 
+int mix_set_gate(mix_ctx* c, int slot, const float* scores, int row_stride, int column, int cmp, float threshold,
+                 void* stream) {
+  if (!c) return MIX_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc = check_slot(c, slot);
+  if (rc != MIX_OK) return rc;
+  if (!c->h_apps[slot].valid) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "slot %d has no app to gate", slot);
+  int kind = c->h_apps[slot].kind & kKindMask;
+  if (!scores) {                      // remove: drop the flag first, the entry may then go stale
+    c->h_apps[slot].kind = kind;
+    MIX_CUDA(c, cudaMemcpyAsync(&c->d_apps[slot].kind, &kind, sizeof(int), cudaMemcpyHostToDevice, s));
+    return MIX_OK;
+  }
+  if (cmp != MIX_GATE_GE && cmp != MIX_GATE_LT) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "bad gate comparison %d", cmp);
+  if (row_stride < 1 || column < 0 || column >= row_stride)
+    MIX_FAIL(c, MIX_ERR_INVALID_ARG, "gate column %d outside [0, row_stride=%d)", column, row_stride);
+  GateEntry g;
+  memset(&g, 0, sizeof(g));
+  g.scores = scores;
+  g.stride = row_stride;
+  g.col = column;
+  g.cmp = cmp;
+  g.thr = threshold;
+  // replacing a live gate: close the flag, rewrite the entry, raise the flag again
+  if (c->h_apps[slot].kind & kKindGated)
+    MIX_CUDA(c, cudaMemcpyAsync(&c->d_apps[slot].kind, &kind, sizeof(int), cudaMemcpyHostToDevice, s));
+  MIX_CUDA(c, cudaMemcpyAsync(c->d_gates + slot, &g, sizeof(g), cudaMemcpyHostToDevice, s));
+  kind |= kKindGated;
+  c->h_apps[slot].kind = kind;
+  MIX_CUDA(c, cudaMemcpyAsync(&c->d_apps[slot].kind, &kind, sizeof(int), cudaMemcpyHostToDevice, s));
+  return MIX_OK;
+}
+
 int mix_update_steer_alpha(mix_ctx* c, int slot, float alpha, void* stream) {
   if (!c) return MIX_ERR_INVALID_ARG;
   int rc = check_slot(c, slot);
   if (rc != MIX_OK) return rc;
-  if (!c->h_apps[slot].valid || c->h_apps[slot].kind != MIX_STEER) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "slot %d is not a steering app", slot);
+  if (!c->h_apps[slot].valid || (c->h_apps[slot].kind & kKindMask) != MIX_STEER) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "slot %d is not a steering app", slot);
   c->h_apps[slot].alpha = alpha;
   MIX_CUDA(c, cudaMemcpyAsync(&c->d_apps[slot].alpha, &alpha, sizeof(float), cudaMemcpyHostToDevice,
                               static_cast<cudaStream_t>(stream)));
@@ -323,7 +369,7 @@ int mix_update_sae_edits(mix_ctx* c, int slot, int n_edit, const int* idx, const
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int rc = check_slot(c, slot);
   if (rc != MIX_OK) return rc;
-  if (!c->h_apps[slot].valid || c->h_apps[slot].kind != MIX_SAE) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "slot %d is not an SAE app", slot);
+  if (!c->h_apps[slot].valid || (c->h_apps[slot].kind & kKindMask) != MIX_SAE) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "slot %d is not an SAE app", slot);
   // shrink first, grow last, so a concurrent reader never sees a count beyond valid entries
   const int old_n = c->h_apps[slot].n_edit;
   if (n_edit < old_n && n_edit >= 0)
@@ -390,13 +436,21 @@ int mix_apply(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream) 
     MIX_CUDA(c, tap());
     MIX_CUDA(c, launch_pack(c, h, s));
     MIX_CUDA(c, tap());
-    if (c->cfg.flags & MIX_FLAG_ENCODE_SIMT)
+    if (c->cfg.flags & MIX_FLAG_ENCODE_SIMT) {
       MIX_CUDA(c, launch_encode_simt(c, s));
-    else
-      MIX_CUDA(c, launch_encode_tc(c, s));
-    MIX_CUDA(c, tap());
-    MIX_CUDA(c, launch_select(c, s));
-    MIX_CUDA(c, tap());
+      MIX_CUDA(c, tap());
+      MIX_CUDA(c, launch_select(c, false, s));
+      MIX_CUDA(c, tap());
+    } else {
+      MIX_CUDA(c, launch_encode_tc(c, 0, s));      // TopK sets -> candidates, other sets -> Z
+      MIX_CUDA(c, tap());
+      MIX_CUDA(c, launch_merge(c, s));             // exact TopK from candidates, or a flag
+      MIX_CUDA(c, tap());
+      MIX_CUDA(c, launch_encode_tc(c, 1, s));      // flagged row tiles -> Z (returns at once if none)
+      MIX_CUDA(c, tap());
+      MIX_CUDA(c, launch_select(c, true, s));      // flagged TopK rows; active counts of the other sets
+      MIX_CUDA(c, tap());
+    }
     MIX_CUDA(c, launch_decode(c, h, s));
     MIX_CUDA(c, tap());
   }
@@ -405,7 +459,8 @@ int mix_apply(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream) 
 
 int mix_launches_per_apply(const mix_ctx* c) {
   if (!c) return 0;
-  return c->cfg.n_groups_max > 0 ? 6 : 1;
+  if (c->cfg.n_groups_max == 0) return 1;
+  return (c->cfg.flags & MIX_FLAG_ENCODE_SIMT) ? 6 : 8;
 }
 
 int mix_get_status(mix_ctx* c, unsigned* bits, void* stream) {

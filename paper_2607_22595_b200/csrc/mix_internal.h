@@ -20,10 +20,12 @@ constexpr int kMaxGroups = 32;
 constexpr int kMaxClasses = 64;
 constexpr int kMaxK = 1024;
 constexpr int kMaxEdits = 64;
+constexpr int kCandPerTile = 8;     // TopK candidates the encode epilogue keeps per (row, feature tile)
+constexpr int kCandMax = 4096;      // candidates per row the merge step can sort in shared memory
 
 struct __align__(16) AppEntry {
   int valid;          // written last by registration; 0 = slot is pass-through
-  int kind;           // MIX_PROBE | MIX_STEER | MIX_SAE
+  int kind;           // MIX_PROBE | MIX_STEER | MIX_SAE, | kKindGated
   int n_classes;      // probe
   int act;            // probe
   float alpha;        // steer
@@ -32,6 +34,19 @@ struct __align__(16) AppEntry {
   int add_error;      // sae
   const void* W;      // probe: bf16 [C, d]; steer: bf16 [d]
   const float* b;     // probe: fp32 [C] or null
+};
+
+constexpr int kKindMask = 0xff;     // AppEntry.kind: low byte = MIX_* kind
+constexpr int kKindGated = 0x100;   //                bit 8    = the slot has a gate (see GateEntry)
+
+// Gate of a slot: the app applies to row t iff cmp(scores[t * stride + col], thr).
+struct __align__(16) GateEntry {
+  const float* scores;
+  int stride;
+  int col;
+  int cmp;            // MIX_GATE_GE | MIX_GATE_LT
+  float thr;
+  int pad_[2];
 };
 
 struct __align__(16) GroupEntry {
@@ -53,6 +68,8 @@ struct RouteState {
   int n_sae_rows;                   // SAE rows routed this call
   int n_mtiles;                     // = n_panel_rows / kTileM
   int total_tiles;                  // encode tiles over all groups
+  int n_topk_rows;                  // SAE rows whose weight set is TopK
+  int pad_[3];
   int group_count[kMaxGroups];      // M_g
   int group_mtile0[kMaxGroups + 1]; // first m-tile of group g in the panel
   int group_tile0[kMaxGroups + 1];  // first linear encode tile of group g
@@ -69,6 +86,7 @@ struct Ctx {
   int* d_n_live;            // [1]
   AppEntry* d_apps;         // [n_slots_max]
   GroupEntry* d_groups;     // [n_groups_max]
+  GateEntry* d_gates;       // [n_slots_max]
   int* d_edit_idx;          // [n_slots_max * r_max]
   float* d_edit_val;
   unsigned char* d_edit_mode;
@@ -90,12 +108,19 @@ struct Ctx {
   float* d_z;               // [P, d_sae_max]
   int* d_topk_idx;          // [P, k_max]
   float* d_topk_val;        // [P, k_max]
+  float* d_cand_val;        // [P, cand_tiles, kCandPerTile] per-tile TopK candidates (fused epilogue)
+  int* d_cand_idx;          // same shape: feature ids
+  float* d_cand_ninth;      // [P, cand_tiles] the (kCandPerTile+1)-th largest value of each tile
+  int cand_tiles;           // d_sae_max / kTileN
+  int* d_row_flag;          // [P] row needs the exact fallback selection
+  int* d_mtile_flag;        // [P / kTileM] some row of the tile is flagged
+  int* d_n_flagged;         // [1]
   CUtensorMap* d_tmap_w;    // [n_groups_max] W_enc maps (box kTileK x kTileN, 128B swizzle)
   CUtensorMap tmap_panel;   // panel map (box kTileK x kTileM, 128B swizzle)
 
   // profiling taps
   int stage_events_on;
-  cudaEvent_t stage_events[8];
+  cudaEvent_t stage_events[12];
 
   // optional outputs
   int* out_topk_idx;
@@ -108,8 +133,9 @@ cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float
 cudaError_t launch_route(const Ctx* c, int T, cudaStream_t s);
 cudaError_t launch_pack(const Ctx* c, const __nv_bfloat16* hidden, cudaStream_t s);
 cudaError_t launch_encode_simt(const Ctx* c, cudaStream_t s);
-cudaError_t launch_encode_tc(const Ctx* c, cudaStream_t s);
-cudaError_t launch_select(const Ctx* c, cudaStream_t s);
+cudaError_t launch_encode_tc(const Ctx* c, int mode, cudaStream_t s);   // 0: all tiles; 1: flagged row tiles -> Z
+cudaError_t launch_merge(const Ctx* c, cudaStream_t s);
+cudaError_t launch_select(const Ctx* c, bool flagged_only, cudaStream_t s);
 cudaError_t launch_decode(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s);
 cudaError_t launch_compose_map(const Ctx* c, int T_live, int n_req, cudaStream_t s);
 cudaError_t launch_fold_bias(const __nv_bfloat16* W_enc, const float* b_enc, const float* b_dec, float* b_eff,

@@ -143,17 +143,31 @@ __device__ __forceinline__ void finish_probe(const float* logit, int C, int act,
 }
 
 struct RowApp {
+  bool gated;           // the slot has a gate (whether or not it let this row through)
   int kind, C, act;     // kind 0: nothing to do
   float alpha;
   const uint4* W;
   const float* b;
 };
 
-// Slot -> app for one row; flags bad slot ids.  `leader` is the one thread that may raise status.
-__device__ __forceinline__ RowApp lookup(int s, const AppEntry* __restrict__ apps, int n_slots,
+// Does row t pass the gate of its slot?  (NaN fails both comparisons.)
+__device__ __forceinline__ bool gate_open(const GateEntry* __restrict__ gates, int s, int t) {
+  const int4 g0 = __ldg(reinterpret_cast<const int4*>(gates + s));        // scores ptr, stride, col
+  const int4 g1 = __ldg(reinterpret_cast<const int4*>(gates + s) + 1);    // cmp, thr
+  const float* sc = reinterpret_cast<const float*>(((unsigned long long)(unsigned)g0.y << 32) | (unsigned)g0.x);
+  const float v = __ldg(sc + (size_t)t * g0.z + g0.w);
+  const float thr = __int_as_float(g1.y);
+  return g1.x == MIX_GATE_GE ? v >= thr : v < thr;
+}
+
+// Slot -> app for row t; flags bad slot ids; applies the slot's gate.  `leader` is the one
+// thread that may raise status.
+__device__ __forceinline__ RowApp lookup(int s, int t, const AppEntry* __restrict__ apps,
+                                         const GateEntry* __restrict__ gates, int n_slots,
                                          unsigned* __restrict__ status, bool leader) {
   RowApp r;
   r.kind = 0;
+  r.gated = false;
   if (s == -1) return r;
   if (s < -1 || s >= n_slots) {
     if (leader) atomicOr(status, MIX_STATUS_BAD_SLOT);
@@ -166,7 +180,9 @@ __device__ __forceinline__ RowApp lookup(int s, const AppEntry* __restrict__ app
     if (leader) atomicOr(status, MIX_STATUS_BAD_SLOT);
     return r;
   }
-  r.kind = q0.y;
+  r.gated = (q0.y & kKindGated) != 0;
+  if (r.gated && !gate_open(gates, s, t)) return r;               // gate closed: the row passes through
+  r.kind = q0.y & kKindMask;
   r.C = q0.z;
   r.act = q0.w;
   r.alpha = __int_as_float(q1.x);
@@ -219,7 +235,8 @@ __device__ __forceinline__ void warp_row(const RowApp& a, __nv_bfloat16* __restr
 // streams the probe matrix from L2 twice per 8 rows instead of eight times.
 __global__ void __launch_bounds__(kWarpsPerBlock * 32, 3)
 probe_steer_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
-                   const AppEntry* __restrict__ apps, int n_slots, __nv_bfloat16* __restrict__ hidden, int d,
+                   const AppEntry* __restrict__ apps, const GateEntry* __restrict__ gates, int n_slots,
+                   __nv_bfloat16* __restrict__ hidden, int d,
                    float* __restrict__ scores, int C_max, unsigned* __restrict__ status) {
   __shared__ float s_part[kWarpsPerBlock][kWarpsPerBlock][kMaxClasses];   // [warp][row][class]
   __shared__ int s_slot[kWarpsPerBlock];
@@ -234,8 +251,9 @@ probe_steer_kernel(const int* __restrict__ token_slot, const int* __restrict__ n
   bool same = t0 + kWarpsPerBlock <= n_live && s_slot[0] >= 0 && scores != nullptr;
 #pragma unroll
   for (int r = 1; r < kWarpsPerBlock; ++r) same = same && s_slot[r] == s_slot[0];
-  const RowApp a = lookup(my_slot, apps, n_slots, status, lane == 0);
-  if (!(same && a.kind == MIX_PROBE && a.C > 1)) {       // CTA-uniform: every warp sees the same slots
+  const RowApp a = lookup(my_slot, t, apps, gates, n_slots, status, lane == 0);
+  // one decision for the whole CTA (a gate can open for some rows of a request and not others)
+  if (!__syncthreads_and(same && a.kind == MIX_PROBE && a.C > 1 && !a.gated)) {
     if (t < n_live) warp_row(a, hidden, t, d, scores, C_max, s_part[warp][0], lane);
     return;
   }
@@ -278,7 +296,8 @@ constexpr int kTeamVec = 4;     // NW * 32 * kTeamVec * 8 >= d_model: 8192 colum
 template <int NW>
 __global__ void __launch_bounds__(NW * 32)
 probe_steer_team_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
-                        const AppEntry* __restrict__ apps, int n_slots, __nv_bfloat16* __restrict__ hidden, int d,
+                        const AppEntry* __restrict__ apps, const GateEntry* __restrict__ gates, int n_slots,
+                   __nv_bfloat16* __restrict__ hidden, int d,
                         float* __restrict__ scores, int C_max, unsigned* __restrict__ status) {
   __shared__ float s_part[NW][kMaxClasses];
   constexpr int NT = NW * 32;
@@ -297,7 +316,7 @@ probe_steer_team_kernel(const int* __restrict__ token_slot, const int* __restric
       if (v < nvec) hq[u] = __ldcs(hrow + v);
     }
   }
-  const RowApp a = lookup(slot, apps, n_slots, status, threadIdx.x == 0);
+  const RowApp a = lookup(slot, t, apps, gates, n_slots, status, threadIdx.x == 0);
   if (a.kind == MIX_STEER) {
     if (a.alpha == 0.f) return;                  // identity; the row stays bit-exact
     uint4 vq[kTeamVec];
@@ -376,9 +395,11 @@ constexpr int kRouteWarps = kRouteThreads / 32;
 
 __global__ void __launch_bounds__(kRouteThreads)
 route_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
-             const AppEntry* __restrict__ apps, int n_slots, const GroupEntry* __restrict__ groups, int n_groups,
+             const AppEntry* __restrict__ apps, const GateEntry* __restrict__ gates, int n_slots,
+             const GroupEntry* __restrict__ groups, int n_groups,
              int* __restrict__ panel_row, int panel_cap, int* __restrict__ mtile_group, RouteState* __restrict__ rs,
-             unsigned* __restrict__ status) {
+             unsigned* __restrict__ status, int* __restrict__ row_flag, int* __restrict__ mtile_flag,
+             int* __restrict__ n_flagged) {
   extern __shared__ int s_cnt[];                      // [n_chunks * kRouteWarps][n_groups]
   __shared__ int s_total[kMaxGroups], s_base[kMaxGroups + 1];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -387,13 +408,19 @@ route_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_
 
   for (int p = tid; p < panel_cap; p += kRouteThreads) panel_row[p] = -1;
   for (int m = tid; m < panel_cap / kTileM; m += kRouteThreads) mtile_group[m] = -1;
+  if (row_flag) {             // fallback-selection flags of the fused TopK path start clear every call
+    for (int p = tid; p < panel_cap; p += kRouteThreads) row_flag[p] = 0;
+    for (int m = tid; m < panel_cap / kTileM; m += kRouteThreads) mtile_flag[m] = 0;
+    if (tid == 0) *n_flagged = 0;
+  }
 
   auto group_of = [&](int t) -> int {
     if (t >= n_live) return -1;
     const int s = token_slot[t];
     if (s < 0 || s >= n_slots) return -1;
     const AppEntry* e = apps + s;
-    if (!e->valid || e->kind != MIX_SAE) return -1;
+    if (!e->valid || (e->kind & kKindMask) != MIX_SAE) return -1;
+    if ((e->kind & kKindGated) && !gate_open(gates, s, t)) return -1;
     const int g = e->group;
     if (g < 0 || g >= n_groups || !groups[g].valid) {
       atomicOr(status, MIX_STATUS_BAD_GROUP);
@@ -431,7 +458,7 @@ route_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_
   }
   __syncthreads();
   if (tid == 0) {
-    int mt = 0, tiles = 0, rows = 0;
+    int mt = 0, tiles = 0, rows = 0, topk_rows = 0;
     for (int q = 0; q < n_groups; ++q) {
       s_base[q] = mt * kTileM;
       rs->group_count[q] = s_total[q];
@@ -441,6 +468,7 @@ route_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_
       for (int m = 0; m < m_tiles; ++m) mtile_group[mt + m] = q;
       mt += m_tiles;
       rows += s_total[q];
+      if (s_total[q] > 0 && groups[q].act == MIX_SAE_TOPK) topk_rows += s_total[q];
       tiles += s_total[q] > 0 ? m_tiles * (int)(groups[q].d_sae / kTileN) : 0;
     }
     s_base[n_groups] = mt * kTileM;
@@ -453,6 +481,7 @@ route_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_
     rs->n_mtiles = mt;
     rs->n_sae_rows = rows;
     rs->total_tiles = tiles;
+    rs->n_topk_rows = topk_rows;
   }
   __syncthreads();
   // phase C: stable scatter
@@ -513,12 +542,12 @@ constexpr int kTeamMaxRows = 2048;   // up to here one CTA per row keeps the who
 
 cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s) {
   if (c->cfg.T_max <= kTeamMaxRows) {
-    probe_steer_team_kernel<8><<<c->cfg.T_max, 8 * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps,
+    probe_steer_team_kernel<8><<<c->cfg.T_max, 8 * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates,
                                                               c->cfg.n_slots_max, hidden, c->cfg.d_model, scores,
                                                               c->cfg.C_max, c->d_status);
   } else {
     const int blocks = (c->cfg.T_max + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    probe_steer_kernel<<<blocks, kWarpsPerBlock * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps,
+    probe_steer_kernel<<<blocks, kWarpsPerBlock * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates,
                                                               c->cfg.n_slots_max, hidden, c->cfg.d_model, scores,
                                                               c->cfg.C_max, c->d_status);
   }
@@ -528,9 +557,10 @@ cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float
 cudaError_t launch_route(const Ctx* c, int T, cudaStream_t s) {
   const int n_chunks = (c->cfg.T_max + kRouteThreads - 1) / kRouteThreads;
   const size_t smem = (size_t)n_chunks * kRouteWarps * c->cfg.n_groups_max * sizeof(int);
-  route_kernel<<<1, kRouteThreads, smem, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->cfg.n_slots_max,
+  route_kernel<<<1, kRouteThreads, smem, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates, c->cfg.n_slots_max,
                                               c->d_groups, c->cfg.n_groups_max, c->d_panel_row, c->panel_rows_cap,
-                                              c->d_mtile_group, c->d_route, c->d_status);
+                                              c->d_mtile_group, c->d_route, c->d_status, c->d_row_flag,
+                                              c->d_mtile_flag, c->d_n_flagged);
   return cudaGetLastError();
 }
 

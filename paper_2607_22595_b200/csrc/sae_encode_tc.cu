@@ -6,7 +6,9 @@
 // Warp roles:  warp 0 = TMA producer (panel tile 128x64 and W_enc tile 256x64 per k-block into
 // a 4-stage ring of 128-byte-swizzled shared memory), warp 1 = MMA issuer (tcgen05.mma
 // 128x256x16, fp32 accumulators in tensor memory, double buffered so the epilogue of one tile
-// overlaps the main loop of the next), warps 2..5 = epilogue (tcgen05.ld, + bias, fp32 store).
+// overlaps the main loop of the next), warps 2..5 = epilogue (tcgen05.ld, + bias, then either
+// the fp32 pre-activations to the Z scratch, or -- for TopK weight sets -- only the tile's 8
+// largest values per row plus its 9th, which the merge step turns into the exact TopK).
 // No TMA multicast and no clusters.  Every wait is bounded: on expiry the CTA raises
 // MIX_STATUS_WAIT_TIMEOUT, lets its copies land, frees its tensor memory and returns.
 #include "mix_internal.h"
@@ -145,10 +147,42 @@ __device__ __forceinline__ Tile decode_tile(const RouteState& rs, const GroupEnt
   return t;
 }
 
+// mode 0: every tile; TopK weight sets emit candidates, the others write Z.
+// mode 1: only row tiles flagged by the merge step (TopK sets), written to Z for the exact
+//         fallback selection; returns at once when nothing is flagged.
+__device__ __forceinline__ bool tile_wanted(const Tile& t, const GroupEntry* __restrict__ groups, int mode,
+                                            const int* __restrict__ mtile_flag) {
+  if (mode == 0) return true;
+  return groups[t.group].act == MIX_SAE_TOPK && mtile_flag[t.m_tile_global] != 0;
+}
+
+// Insert (x, c) into the descending list tv[0..8] if it beats the 9th entry.  Equal values keep
+// the earlier (lower) column in front, which is the tie rule of the selection.
+__device__ __forceinline__ void top9_insert(float (&tv)[kCandPerTile + 1], int (&ti)[kCandPerTile + 1], float x, int c) {
+  if (!(x > tv[kCandPerTile])) return;
+  bool placed = false;
+#pragma unroll
+  for (int s = kCandPerTile; s >= 1; --s) {
+    const bool gt = x > tv[s - 1];
+    const float nv = gt ? tv[s - 1] : (placed ? tv[s] : x);
+    const int ni = gt ? ti[s - 1] : (placed ? ti[s] : c);
+    placed = placed || !gt;
+    tv[s] = nv;
+    ti[s] = ni;
+  }
+  if (!placed) {
+    tv[0] = x;
+    ti[0] = c;
+  }
+}
+
 __global__ void __launch_bounds__(kTcThreads, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorMap* __restrict__ tmap_w,
                  const RouteState* __restrict__ rs_g, const GroupEntry* __restrict__ groups, int n_groups,
-                 float* __restrict__ Z, long long ldz, int d, unsigned* __restrict__ status) {
+                 float* __restrict__ Z, long long ldz, int d, unsigned* __restrict__ status, int mode,
+                 const int* __restrict__ mtile_flag, const int* __restrict__ n_flagged, float* __restrict__ cand_val,
+                 int* __restrict__ cand_idx, float* __restrict__ cand_ninth, int cand_tiles) {
+  if (mode == 1 && *n_flagged == 0) return;
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment: required by the 128-byte swizzle atoms
   unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -193,6 +227,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
         const Tile t = decode_tile(sh->rs, groups, n_groups, tile);
+        if (!tile_wanted(t, groups, mode, mtile_flag)) continue;
         const CUtensorMap* tw = tmap_w + t.group;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(smem_u32(&sh->empty[stage]), phase ^ 1u, sh, status)) { ok = false; break; }
@@ -211,6 +246,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
       unsigned phase = 0, acc = 0, acc_phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        if (mode != 0 && !tile_wanted(decode_tile(sh->rs, groups, n_groups, tile), groups, mode, mtile_flag)) continue;
         if (!mbar_wait(smem_u32(&sh->tmem_empty[acc]), acc_phase ^ 1u, sh, status)) break;
         tc_fence_after();
         const unsigned d_tmem = tmem_base + acc * kTileN;
@@ -236,6 +272,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
     unsigned acc = 0, acc_phase = 0;
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
       const Tile t = decode_tile(sh->rs, groups, n_groups, tile);
+      if (!tile_wanted(t, groups, mode, mtile_flag)) continue;
       // warp-uniform decision: tcgen05.ld below needs the whole warp
       if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&sh->tmem_full[acc]), acc_phase, sh, status))) break;
       tc_fence_after();
@@ -243,21 +280,56 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
       const bool valid = row_local < t.rows_valid;
       const size_t p = (size_t)t.m_tile_global * kTileM + row_local;
       const float* bias = groups[t.group].b_eff + (size_t)t.n_tile * kTileN;
-      float* out = Z + p * (size_t)ldz + (size_t)t.n_tile * kTileN;
+      const unsigned taddr = tmem_base + ((unsigned)(q * 32) << 16) + acc * kTileN;
+      if (mode == 0 && groups[t.group].act == MIX_SAE_TOPK) {
+        float tv[kCandPerTile + 1];
+        int ti[kCandPerTile + 1];
+#pragma unroll
+        for (int s = 0; s <= kCandPerTile; ++s) {
+          tv[s] = -INFINITY;
+          ti[s] = 0;
+        }
 #pragma unroll 1
-      for (int c = 0; c < kTileN; c += 32) {
-        float v[32];
-        tmem_ld32(tmem_base + ((unsigned)(q * 32) << 16) + acc * kTileN + c, v);
-        if (valid) {
+        for (int c = 0; c < kTileN; c += 32) {
+          float v[32];
+          tmem_ld32(taddr + c, v);
 #pragma unroll
           for (int i = 0; i < 32; i += 4) {
             const float4 b4 = __ldg(reinterpret_cast<const float4*>(bias + c + i));
-            float4 o;
-            o.x = v[i] + b4.x;
-            o.y = v[i + 1] + b4.y;
-            o.z = v[i + 2] + b4.z;
-            o.w = v[i + 3] + b4.w;
-            *reinterpret_cast<float4*>(out + c + i) = o;
+            top9_insert(tv, ti, v[i] + b4.x, c + i);
+            top9_insert(tv, ti, v[i + 1] + b4.y, c + i + 1);
+            top9_insert(tv, ti, v[i + 2] + b4.z, c + i + 2);
+            top9_insert(tv, ti, v[i + 3] + b4.w, c + i + 3);
+          }
+        }
+        if (valid) {
+          const size_t slot = p * (size_t)cand_tiles + (size_t)t.n_tile;
+          float4* cv = reinterpret_cast<float4*>(cand_val + slot * kCandPerTile);
+          int4* ci = reinterpret_cast<int4*>(cand_idx + slot * kCandPerTile);
+          const int j0 = t.n_tile * kTileN;
+          cv[0] = make_float4(tv[0], tv[1], tv[2], tv[3]);
+          cv[1] = make_float4(tv[4], tv[5], tv[6], tv[7]);
+          ci[0] = make_int4(j0 + ti[0], j0 + ti[1], j0 + ti[2], j0 + ti[3]);
+          ci[1] = make_int4(j0 + ti[4], j0 + ti[5], j0 + ti[6], j0 + ti[7]);
+          cand_ninth[slot] = tv[kCandPerTile];
+        }
+      } else {
+        float* out = Z + p * (size_t)ldz + (size_t)t.n_tile * kTileN;
+#pragma unroll 1
+        for (int c = 0; c < kTileN; c += 32) {
+          float v[32];
+          tmem_ld32(taddr + c, v);
+          if (valid) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+              const float4 b4 = __ldg(reinterpret_cast<const float4*>(bias + c + i));
+              float4 o;
+              o.x = v[i] + b4.x;
+              o.y = v[i + 1] + b4.y;
+              o.z = v[i + 2] + b4.z;
+              o.w = v[i + 3] + b4.w;
+              *reinterpret_cast<float4*>(out + c + i) = o;
+            }
           }
         }
       }
@@ -288,10 +360,12 @@ cudaError_t encode_tc_prepare() {
   return cudaFuncSetAttribute(encode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
 }
 
-cudaError_t launch_encode_tc(const Ctx* c, cudaStream_t s) {
+cudaError_t launch_encode_tc(const Ctx* c, int mode, cudaStream_t s) {
   encode_tc_kernel<<<c->n_sms, kTcThreads, kSmemBytes, s>>>(c->tmap_panel, c->d_tmap_w, c->d_route, c->d_groups,
                                                              c->cfg.n_groups_max, c->d_z, c->cfg.d_sae_max,
-                                                             c->cfg.d_model, c->d_status);
+                                                             c->cfg.d_model, c->d_status, mode, c->d_mtile_flag,
+                                                             c->d_n_flagged, c->d_cand_val, c->d_cand_idx,
+                                                             c->d_cand_ninth, c->cand_tiles);
   return cudaGetLastError();
 }
 

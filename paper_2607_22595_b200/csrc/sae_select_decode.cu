@@ -74,8 +74,9 @@ encode_simt_kernel(const __nv_bfloat16* __restrict__ panel, const int* __restric
 // selection
 // ---------------------------------------------------------------------------------------
 constexpr int kSelThreads = 512;
-constexpr int kCand = 4096;
+constexpr int kCand = 1024;        // composites sorted in shared memory (>= k_max)
 constexpr int kBins = 2048;
+static_assert(kCand >= kMaxK, "the sort buffer must hold a full TopK list");
 
 __device__ __forceinline__ unsigned f2key(float f) {
   const unsigned b = __float_as_uint(f + 0.f);          // -0.0 -> +0.0: equal values, equal keys
@@ -83,6 +84,57 @@ __device__ __forceinline__ unsigned f2key(float f) {
 }
 __device__ __forceinline__ float key2f(unsigned k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+// In-place bitonic sort of the first n entries of `a` (shared memory), descending.  Entries up
+// to the next power of two are overwritten with 0 (the smallest composite key).
+__device__ void bitonic_sort_desc(unsigned long long* a, int n) {
+  const int tid = threadIdx.x;
+  int n2 = 1;
+  while (n2 < n) n2 <<= 1;
+  for (int i = n + tid; i < n2; i += kSelThreads) a[i] = 0ull;
+  __syncthreads();
+  for (int size = 2; size <= n2; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int i = tid; i < n2 / 2; i += kSelThreads) {
+        const int lo = 2 * i - (i & (stride - 1));
+        const int hi = lo + stride;
+        const bool desc = ((lo & size) == 0);
+        const unsigned long long x = a[lo], y = a[hi];
+        if ((x < y) == desc) {
+          a[lo] = y;
+          a[hi] = x;
+        }
+      }
+      __syncthreads();
+    }
+  }
+}
+
+// Write the first k sorted composites (key << 32 | ~id) as the row's TopK lists.
+__device__ void emit_topk(const unsigned long long* a, int k, int k_max, int p, int t, int* __restrict__ ws_idx,
+                          float* __restrict__ ws_val, int* __restrict__ out_idx, float* __restrict__ out_val,
+                          int* __restrict__ out_n_active, int* s_count) {
+  const int tid = threadIdx.x;
+  int pos_cnt = 0;
+  for (int i = tid; i < k; i += kSelThreads) {
+    const unsigned long long c = a[i];
+    const int j = (int)(0xffffffffu - (unsigned)(c & 0xffffffffull));
+    const float v = key2f((unsigned)(c >> 32));
+    ws_idx[(size_t)p * k_max + i] = j;
+    ws_val[(size_t)p * k_max + i] = v;
+    if (out_idx) out_idx[(size_t)t * k_max + i] = j;
+    if (out_val) out_val[(size_t)t * k_max + i] = v;
+    pos_cnt += v > 0.f;
+  }
+  if (out_n_active) {
+    if (tid == 0) *s_count = 0;
+    __syncthreads();
+    pos_cnt = __reduce_add_sync(0xffffffffu, pos_cnt);
+    if ((tid & 31) == 0) atomicAdd(s_count, pos_cnt);
+    __syncthreads();
+    if (tid == 0) out_n_active[t] = *s_count;
+  }
 }
 
 // Largest digit D with count(digit >= D) >= need, and the count of digits > D.  One warp.
@@ -113,64 +165,57 @@ __device__ void find_digit(const int* hist, int n_bins, int need, int* s_out) {
   }
 }
 
-__global__ void __launch_bounds__(kSelThreads)
-select_kernel(const float* __restrict__ Z, long long ldz, const int* __restrict__ panel_row,
-              const int* __restrict__ mtile_group, const RouteState* __restrict__ rs,
-              const GroupEntry* __restrict__ groups, int k_max, int* __restrict__ ws_idx, float* __restrict__ ws_val,
-              int* __restrict__ out_idx, float* __restrict__ out_val, int* __restrict__ out_n_active,
-              unsigned* __restrict__ status) {
-  __shared__ int s_hist[kBins];
-  __shared__ unsigned long long s_cand[kCand];
-  __shared__ int s_n, s_res[2], s_count;
-  const int p = blockIdx.x;
-  if (p >= rs->n_panel_rows) return;
-  const int t = panel_row[p];
-  if (t < 0) return;
-  const GroupEntry ge = groups[mtile_group[p / kTileM]];
-  const int S = (int)ge.d_sae;
-  const float* z = Z + (size_t)p * ldz;
-  const int tid = threadIdx.x;
+// The two places a row's values can come from.
+struct ZRow {            // all pre-activations of the row; position = feature id
+  const float* z;
+  int n;
+  __device__ __forceinline__ unsigned key(int i) const { return f2key(z[i]); }
+  __device__ __forceinline__ unsigned id(int i) const { return (unsigned)i; }
+};
+struct CandRow {         // per-tile candidates of the fused encode epilogue
+  const float* v;
+  const int* j;
+  int n;
+  __device__ __forceinline__ unsigned key(int i) const { return f2key(v[i]); }
+  __device__ __forceinline__ unsigned id(int i) const { return (unsigned)j[i]; }
+};
 
-  if (ge.act != MIX_SAE_TOPK) {
-    if (out_n_active == nullptr) return;
-    int cnt = 0;
-    for (int j = tid; j < S; j += kSelThreads) {
-      const float v = z[j];
-      const bool on = ge.act == MIX_SAE_RELU ? v > 0.f : (v > ge.theta[j] && v > 0.f);
-      cnt += on;
-    }
-    if (tid == 0) s_count = 0;
-    __syncthreads();
-    cnt = __reduce_add_sync(0xffffffffu, cnt);
-    if ((tid & 31) == 0) atomicAdd(&s_count, cnt);
-    __syncthreads();
-    if (tid == 0) out_n_active[t] = s_count;
-    return;
-  }
+struct SelShared {
+  int hist[kBins];
+  unsigned long long cand[kCand];
+  int n, res[2], count;
+};
 
-  const int k = ge.k;
-  // radix refinement: 11 + 11 + 10 bits from the top
+// Collect into sh.cand (unsorted composites key << 32 | ~id) a set that contains the k largest
+// entries of `src` under the order (value descending, id ascending): radix refinement on the
+// order-preserving keys, 11 + 11 + 10 bits from the top, until what is still undecided fits the
+// buffer.  If more than the buffer's worth of entries tie EXACTLY with the k-th value:
+//   ORDERED sources (position order = id order) finish with an index-ordered pass and return 2;
+//   other sources return 0 (the caller falls back).
+// Returns 1 in the ordinary case.  Every thread of the CTA must call this.
+template <bool ORDERED, class Src>
+__device__ int radix_collect(const Src& src, int k, SelShared& sh) {
+  const int tid = threadIdx.x, n = src.n;
   const int shifts[3] = {21, 10, 0};
   const int widths[3] = {11, 11, 10};
   unsigned prefix = 0;          // digits fixed so far (value of key >> (shift + width))
   int need = k;                 // winners still to be found inside the prefix set
   bool done = false;
-  int pass = 0;
-  unsigned thr_hi = 0;          // elements with (key >> thr_shift) >= thr_hi are candidates
+  unsigned thr_hi = 0;          // entries with (key >> thr_shift) >= thr_hi are collected
   int thr_shift = 0;
-  for (; pass < 3 && !done; ++pass) {
+  for (int pass = 0; pass < 3 && !done; ++pass) {
     const int shift = shifts[pass], nb = 1 << widths[pass];
-    for (int b = tid; b < nb; b += kSelThreads) s_hist[b] = 0;
+    for (int b = tid; b < nb; b += kSelThreads) sh.hist[b] = 0;
     __syncthreads();
-    for (int j = tid; j < S; j += kSelThreads) {
-      const unsigned key = f2key(z[j]);
-      if (pass == 0 || (key >> (shift + widths[pass])) == prefix) atomicAdd(&s_hist[(key >> shift) & (nb - 1)], 1);
+    for (int i = tid; i < n; i += kSelThreads) {
+      const unsigned key = src.key(i);
+      if (pass == 0 || (key >> (shift + widths[pass])) == prefix) atomicAdd(&sh.hist[(key >> shift) & (nb - 1)], 1);
     }
     __syncthreads();
-    if (tid < 32) find_digit(s_hist, nb, need, s_res);
+    if (tid < 32) find_digit(sh.hist, nb, need, sh.res);
     __syncthreads();
-    const int D = s_res[0], above = s_res[1];
-    const int in_bin = s_hist[D];
+    const int D = sh.res[0], above = sh.res[1];
+    const int in_bin = sh.hist[D];
     need -= above;
     prefix = (prefix << widths[pass]) | (unsigned)D;
     thr_hi = prefix;
@@ -178,91 +223,149 @@ select_kernel(const float* __restrict__ Z, long long ldz, const int* __restrict_
     if ((k - need) + in_bin <= kCand) done = true;
     __syncthreads();
   }
-
-  if (tid == 0) s_n = 0;
+  if (tid == 0) sh.n = 0;
   __syncthreads();
   if (done) {
-    for (int j = tid; j < S; j += kSelThreads) {
-      const unsigned key = f2key(z[j]);
+    for (int i = tid; i < n; i += kSelThreads) {
+      const unsigned key = src.key(i);
       if ((key >> thr_shift) >= thr_hi) {
-        const int pos = atomicAdd(&s_n, 1);
-        s_cand[pos] = ((unsigned long long)key << 32) | (unsigned)(0xffffffffu - (unsigned)j);
+        const int pos = atomicAdd(&sh.n, 1);
+        sh.cand[pos] = ((unsigned long long)key << 32) | (0xffffffffu - src.id(i));
       }
     }
+    __syncthreads();
+    return 1;
+  }
+  if constexpr (!ORDERED) {
+    return 0;
   } else {
-    // more than kCand exact ties at the k-th value: take every larger key, then the `need`
-    // lowest feature ids among the tied ones, in index order.
-    if (tid == 0) atomicOr(status, MIX_STATUS_TOPK_GENERAL);
-    for (int j = tid; j < S; j += kSelThreads) {
-      const unsigned key = f2key(z[j]);
-      if (key > prefix) {
-        const int pos = atomicAdd(&s_n, 1);
-        s_cand[pos] = ((unsigned long long)key << 32) | (unsigned)(0xffffffffu - (unsigned)j);
-      }
-    }
-    __syncthreads();
-    int taken = 0;               // uniform across the block
-    for (int j0 = 0; j0 < S && taken < need; j0 += kSelThreads) {
-      const int j = j0 + tid;
-      const bool eq = j < S && f2key(z[j]) == prefix;
-      const unsigned m = __ballot_sync(0xffffffffu, eq);
-      if ((tid & 31) == 0) s_hist[tid >> 5] = __popc(m);
-      __syncthreads();
-      int before = 0, total = 0;
-      for (int w = 0; w < kSelThreads / 32; ++w) {
-        const int c = s_hist[w];
-        if (w < (tid >> 5)) before += c;
-        total += c;
-      }
-      const int rank = taken + before + __popc(m & ((1u << (tid & 31)) - 1u));
-      if (eq && rank < need) {
-        const int pos = atomicAdd(&s_n, 1);
-        s_cand[pos] = ((unsigned long long)prefix << 32) | (unsigned)(0xffffffffu - (unsigned)j);
-      }
-      taken += total;
-      __syncthreads();
+  // every larger key, then the `need` lowest ids among the exact ties, in index order
+  for (int i = tid; i < n; i += kSelThreads) {
+    const unsigned key = src.key(i);
+    if (key > prefix) {
+      const int pos = atomicAdd(&sh.n, 1);
+      sh.cand[pos] = ((unsigned long long)key << 32) | (0xffffffffu - src.id(i));
     }
   }
   __syncthreads();
-  const int n = s_n;
-  int n2 = 1;
-  while (n2 < n) n2 <<= 1;
-  for (int i = n + tid; i < n2; i += kSelThreads) s_cand[i] = 0ull;
-  __syncthreads();
-  // bitonic sort, descending
-  for (int size = 2; size <= n2; size <<= 1) {
-    for (int stride = size >> 1; stride > 0; stride >>= 1) {
-      for (int i = tid; i < n2 / 2; i += kSelThreads) {
-        const int lo = 2 * i - (i & (stride - 1));
-        const int hi = lo + stride;
-        const bool desc = ((lo & size) == 0);
-        const unsigned long long a = s_cand[lo], b = s_cand[hi];
-        if ((a < b) == desc) {
-          s_cand[lo] = b;
-          s_cand[hi] = a;
-        }
-      }
-      __syncthreads();
+  int taken = 0;               // uniform across the block
+  for (int i0 = 0; i0 < n && taken < need; i0 += kSelThreads) {
+    const int i = i0 + tid;
+    const bool eq = i < n && src.key(i) == prefix;
+    const unsigned m = __ballot_sync(0xffffffffu, eq);
+    if ((tid & 31) == 0) sh.hist[tid >> 5] = __popc(m);
+    __syncthreads();
+    int before = 0, total = 0;
+    for (int w = 0; w < kSelThreads / 32; ++w) {
+      const int c = sh.hist[w];
+      if (w < (tid >> 5)) before += c;
+      total += c;
     }
-  }
-  int pos_cnt = 0;
-  for (int i = tid; i < k; i += kSelThreads) {
-    const unsigned long long c = s_cand[i];
-    const int j = (int)(0xffffffffu - (unsigned)(c & 0xffffffffull));
-    const float v = key2f((unsigned)(c >> 32));
-    ws_idx[(size_t)p * k_max + i] = j;
-    ws_val[(size_t)p * k_max + i] = v;
-    if (out_idx) out_idx[(size_t)t * k_max + i] = j;
-    if (out_val) out_val[(size_t)t * k_max + i] = v;
-    pos_cnt += v > 0.f;
-  }
-  if (out_n_active) {
-    if (tid == 0) s_count = 0;
+    const int rank = taken + before + __popc(m & ((1u << (tid & 31)) - 1u));
+    if (eq && rank < need) {
+      const int pos = atomicAdd(&sh.n, 1);
+      sh.cand[pos] = ((unsigned long long)prefix << 32) | (0xffffffffu - src.id(i));
+    }
+    taken += total;
     __syncthreads();
-    pos_cnt = __reduce_add_sync(0xffffffffu, pos_cnt);
-    if ((tid & 31) == 0) atomicAdd(&s_count, pos_cnt);
+  }
+  __syncthreads();
+  return 2;
+  }
+}
+
+// select_kernel: exact TopK of a row from the Z scratch (all rows, or only rows the merge step
+// flagged), and the active count of ReLU / JumpReLU rows.
+__global__ void __launch_bounds__(kSelThreads)
+select_kernel(const float* __restrict__ Z, long long ldz, const int* __restrict__ panel_row,
+              const int* __restrict__ mtile_group, const RouteState* __restrict__ rs,
+              const GroupEntry* __restrict__ groups, int k_max, int* __restrict__ ws_idx, float* __restrict__ ws_val,
+              int* __restrict__ out_idx, float* __restrict__ out_val, int* __restrict__ out_n_active,
+              unsigned* __restrict__ status, const int* __restrict__ row_flag, const int* __restrict__ n_flagged) {
+  __shared__ SelShared sh;
+  // nothing to do: no flagged TopK row, and nobody asked for the other sets' active counts
+  if (row_flag != nullptr && *n_flagged == 0 && (out_n_active == nullptr || rs->n_topk_rows == rs->n_sae_rows)) return;
+  const int n_rows = rs->n_panel_rows;
+  for (int p = blockIdx.x; p < n_rows; p += gridDim.x) {
+    const int t = panel_row[p];
+    if (t < 0) continue;
+    const GroupEntry ge = groups[mtile_group[p / kTileM]];
+    const int S = (int)ge.d_sae;
+    const float* z = Z + (size_t)p * ldz;
+    const int tid = threadIdx.x;
+    if (ge.act != MIX_SAE_TOPK) {
+      if (out_n_active == nullptr) continue;
+      int cnt = 0;
+      for (int j = tid; j < S; j += kSelThreads) {
+        const float v = z[j];
+        const bool on = ge.act == MIX_SAE_RELU ? v > 0.f : (v > ge.theta[j] && v > 0.f);
+        cnt += on;
+      }
+      if (tid == 0) sh.count = 0;
+      __syncthreads();
+      cnt = __reduce_add_sync(0xffffffffu, cnt);
+      if ((tid & 31) == 0) atomicAdd(&sh.count, cnt);
+      __syncthreads();
+      if (tid == 0) out_n_active[t] = sh.count;
+      __syncthreads();
+      continue;
+    }
+    if (row_flag != nullptr && !row_flag[p]) continue;   // the merge step already settled this row
+    ZRow src{z, S};
+    const int how = radix_collect<true>(src, ge.k, sh);
+    if (how == 2 && tid == 0) atomicOr(status, MIX_STATUS_TOPK_GENERAL);
+    bitonic_sort_desc(sh.cand, sh.n);
+    emit_topk(sh.cand, ge.k, k_max, p, t, ws_idx, ws_val, out_idx, out_val, out_n_active, &sh.count);
     __syncthreads();
-    if (tid == 0) out_n_active[t] = s_count;
+  }
+}
+
+// merge_kernel: exact TopK from the per-tile candidates of the fused encode epilogue.
+// Every (row, feature tile) contributed its 8 largest pre-activations and its 9th.  The k
+// largest candidates are the row's TopK unless some tile's 9th value reaches the k-th
+// candidate, i.e. that tile may hide a winner (or an exact tie whose order matters).  Such rows
+// are flagged; their row tiles are re-encoded to Z and selected exactly by select_kernel.
+__global__ void __launch_bounds__(kSelThreads)
+merge_kernel(const float* __restrict__ cand_val, const int* __restrict__ cand_idx, const float* __restrict__ cand_ninth,
+             int cand_tiles, const int* __restrict__ panel_row, const int* __restrict__ mtile_group,
+             const RouteState* __restrict__ rs, const GroupEntry* __restrict__ groups, int k_max,
+             int* __restrict__ ws_idx, float* __restrict__ ws_val, int* __restrict__ out_idx, float* __restrict__ out_val,
+             int* __restrict__ out_n_active, int* __restrict__ row_flag, int* __restrict__ mtile_flag,
+             int* __restrict__ n_flagged) {
+  __shared__ SelShared sh;
+  if (rs->n_topk_rows == 0) return;                  // no TopK row routed this call
+  const int n_rows = rs->n_panel_rows;
+  for (int p = blockIdx.x; p < n_rows; p += gridDim.x) {
+    const int t = panel_row[p];
+    if (t < 0) continue;
+    const GroupEntry ge = groups[mtile_group[p / kTileM]];
+    if (ge.act != MIX_SAE_TOPK) continue;
+    const int tid = threadIdx.x;
+    const int n_tiles = (int)(ge.d_sae / kTileN);
+    const int n = n_tiles * kCandPerTile, k = ge.k;
+    bool flag = n < k;                               // uniform
+    if (!flag) {
+      CandRow src{cand_val + (size_t)p * cand_tiles * kCandPerTile, cand_idx + (size_t)p * cand_tiles * kCandPerTile, n};
+      flag = radix_collect<false>(src, k, sh) == 0;
+    }
+    if (!flag) {
+      bitonic_sort_desc(sh.cand, sh.n);
+      const unsigned kth = (unsigned)(sh.cand[k - 1] >> 32);
+      const float* ninth = cand_ninth + (size_t)p * cand_tiles;
+      int over = 0;
+      for (int i = tid; i < n_tiles; i += kSelThreads) over |= f2key(ninth[i]) >= kth;
+      flag = __syncthreads_or(over) != 0;
+    }
+    if (flag) {
+      if (tid == 0) {
+        row_flag[p] = 1;
+        mtile_flag[p / kTileM] = 1;
+        atomicAdd(n_flagged, 1);
+      }
+    } else {
+      emit_topk(sh.cand, k, k_max, p, t, ws_idx, ws_val, out_idx, out_val, out_n_active, &sh.count);
+    }
+    __syncthreads();
   }
 }
 
@@ -334,16 +437,23 @@ decode_kernel(__nv_bfloat16* __restrict__ hidden, int d, const float* __restrict
     const int j = s_eidx[tid];
     bool alive = true;
     for (int e2 = tid + 1; e2 < n_edit; ++e2) alive = alive && (s_eidx[e2] != j);
-    const float zj = z[j];
     float f;
     if (ge.act == MIX_SAE_RELU) {
-      f = fmaxf(zj, 0.f);
+      f = fmaxf(z[j], 0.f);
     } else if (ge.act == MIX_SAE_JUMPRELU) {
+      const float zj = z[j];
       f = zj > ge.theta[j] ? zj : 0.f;
     } else {
+      // TopK: the pre-activation of a selected feature comes from the row's TopK list (the Z
+      // scratch is not written for TopK sets unless the row took the fallback selection)
+      float zk = 0.f;
       bool in = false;
-      for (int i = 0; i < ge.k; ++i) in = in || (K[i] == j);
-      f = in ? fmaxf(zj, 0.f) : 0.f;
+      for (int i = 0; i < ge.k; ++i)
+        if (K[i] == j) {
+          in = true;
+          zk = Kv[i];
+        }
+      f = in ? fmaxf(zk, 0.f) : 0.f;
     }
     const float fnew = edit_mode[slot * r_max + tid] == MIX_EDIT_CLAMP ? edit_val[slot * r_max + tid] : 0.f;
     s_alive[tid] = alive;
@@ -441,6 +551,12 @@ decode_kernel(__nv_bfloat16* __restrict__ hidden, int d, const float* __restrict
 
 }  // namespace
 
+// one CTA per packed row, but never more than a few waves: rows are walked grid-stride
+static int row_grid(const Ctx* c) {
+  const int cap = (c->n_sms > 0 ? c->n_sms : 148) * 8;
+  return c->panel_rows_cap < cap ? c->panel_rows_cap : cap;
+}
+
 cudaError_t launch_encode_simt(const Ctx* c, cudaStream_t s) {
   dim3 grid((unsigned)(c->cfg.d_sae_max / 64), (unsigned)(c->panel_rows_cap / 64));
   encode_simt_kernel<<<grid, 256, 0, s>>>(c->d_panel, c->d_mtile_group, c->d_route, c->d_groups, c->d_z,
@@ -448,11 +564,21 @@ cudaError_t launch_encode_simt(const Ctx* c, cudaStream_t s) {
   return cudaGetLastError();
 }
 
-cudaError_t launch_select(const Ctx* c, cudaStream_t s) {
-  select_kernel<<<c->panel_rows_cap, kSelThreads, 0, s>>>(c->d_z, c->cfg.d_sae_max, c->d_panel_row,
+cudaError_t launch_merge(const Ctx* c, cudaStream_t s) {
+  merge_kernel<<<row_grid(c), kSelThreads, 0, s>>>(c->d_cand_val, c->d_cand_idx, c->d_cand_ninth, c->cand_tiles,
+                                                         c->d_panel_row, c->d_mtile_group, c->d_route, c->d_groups,
+                                                         c->cfg.k_max, c->d_topk_idx, c->d_topk_val, c->out_topk_idx,
+                                                         c->out_topk_val, c->out_n_active, c->d_row_flag,
+                                                         c->d_mtile_flag, c->d_n_flagged);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_select(const Ctx* c, bool flagged_only, cudaStream_t s) {
+  select_kernel<<<row_grid(c), kSelThreads, 0, s>>>(c->d_z, c->cfg.d_sae_max, c->d_panel_row,
                                                           c->d_mtile_group, c->d_route, c->d_groups, c->cfg.k_max,
                                                           c->d_topk_idx, c->d_topk_val, c->out_topk_idx,
-                                                          c->out_topk_val, c->out_n_active, c->d_status);
+                                                          c->out_topk_val, c->out_n_active, c->d_status,
+                                                          flagged_only ? c->d_row_flag : nullptr, c->d_n_flagged);
   return cudaGetLastError();
 }
 

@@ -28,7 +28,8 @@ constexpr size_t kOffTokenSlot = 0;
 constexpr size_t kOffNLive = kOffTokenSlot + align256(kStaticRows * sizeof(int));
 constexpr size_t kOffStatus = kOffNLive + 256;
 constexpr size_t kOffApp = kOffStatus + 256;
-constexpr size_t kOffGroup = kOffApp + align256(sizeof(AppEntry));
+constexpr size_t kOffGate = kOffApp + align256(sizeof(AppEntry));
+constexpr size_t kOffGroup = kOffGate + align256(sizeof(GateEntry));
 constexpr size_t kOffEditIdx = kOffGroup + align256(sizeof(GroupEntry));
 constexpr size_t kOffEditVal = kOffEditIdx + align256(kMaxEdits * sizeof(int));
 constexpr size_t kOffEditMode = kOffEditVal + align256(kMaxEdits * sizeof(float));
@@ -121,6 +122,7 @@ extern "C" int mix_sae_apply_static(void* hidden, int n_rows, int d_model, const
   c.d_n_live = reinterpret_cast<int*>(base + kOffNLive);
   c.d_status = reinterpret_cast<unsigned*>(base + kOffStatus);
   c.d_apps = reinterpret_cast<AppEntry*>(base + kOffApp);
+  c.d_gates = reinterpret_cast<GateEntry*>(base + kOffGate);     // never read: the app entry carries no gate flag
   c.d_groups = reinterpret_cast<GroupEntry*>(base + kOffGroup);
   c.d_edit_idx = reinterpret_cast<int*>(base + kOffEditIdx);
   c.d_edit_val = reinterpret_cast<float*>(base + kOffEditVal);
@@ -172,7 +174,7 @@ extern "C" int mix_sae_apply_static(void* hidden, int n_rows, int d_model, const
   if (e == cudaSuccess) e = launch_route(&c, n_rows, s);
   if (e == cudaSuccess) e = launch_pack(&c, h, s);
   if (e == cudaSuccess) e = launch_encode_simt(&c, s);
-  if (e == cudaSuccess) e = launch_select(&c, s);
+  if (e == cudaSuccess) e = launch_select(&c, false, s);
   if (e == cudaSuccess) e = launch_decode(&c, h, s);
   if (e != cudaSuccess) return fail(errbuf, errbuf_len, MIX_ERR_CUDA, "CUDA error %lld while enqueuing the static SAE call", (long long)e);
   return MIX_OK;

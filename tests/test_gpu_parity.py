@@ -334,7 +334,7 @@ def test_api_error_codes():
     with pytest.raises(mixlib.MixError) as e:
         m.set_slot_map(np.zeros(9, dtype=np.int32))                       # T_live > T_max
     assert e.value.code == -2
-    assert m.launches_per_apply() == 6
+    assert m.launches_per_apply() == 8
     m.destroy()
 
 

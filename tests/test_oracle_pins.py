@@ -326,3 +326,37 @@ def test_hook_all_unhooked_is_identity_and_topk_override():
     K2 = K.copy(); K2[-1] = other
     r_over = O.apply_hook(w, rows=[t], topk_override={t: K2})
     assert r_over.topk[t].tolist() == K2.tolist()
+
+
+# ------------------------------------------------------------------ activation-driven gates
+def test_gate_closed_form_cases():
+    sc = np.array([[0.0, -1.0], [0.5, 2.0], [np.nan, 0.5], [0.5, 0.5]], dtype=np.float32)
+    G = lambda col, cmp, thr: W.Gate(sc, col, cmp, thr)
+    assert [O.gate_open(G(0, O.GATE_GE, 0.5), t) for t in range(4)] == [False, True, False, True]
+    assert [O.gate_open(G(0, O.GATE_LT, 0.5), t) for t in range(4)] == [True, False, False, False]   # NaN fails both
+    assert [O.gate_open(G(1, O.GATE_GE, 0.5), t) for t in range(4)] == [False, True, True, True]     # == threshold: GE open
+    assert all(O.gate_open(G(1, O.GATE_GE, -np.inf), t) for t in range(4))
+    assert not any(O.gate_open(G(1, O.GATE_GE, np.inf), t) for t in range(4))
+
+
+def test_gated_hook_limits_and_complement():
+    w = W.host(W.make_tiny(d=64, T=48, d_sae=256, k=8, seed=14))
+    base = O.apply_hook(w)
+    rng = np.random.default_rng(3)
+    sc = rng.standard_normal((48, 2)).astype(np.float32)
+
+    def run(cmp, thr):
+        wg = W.host(W.make_tiny(d=64, T=48, d_sae=256, k=8, seed=14))
+        for a in wg.apps.values():
+            a.gate = W.Gate(sc, 1, cmp, thr)
+        return O.apply_hook(wg)
+
+    always, never = run(O.GATE_GE, -np.inf), run(O.GATE_GE, np.inf)
+    ge, lt = run(O.GATE_GE, 0.1), run(O.GATE_LT, 0.1)
+    for t in range(48):
+        assert np.array_equal(always.out_bits[t], base.out_bits[t]) and (t in always.scores) == (t in base.scores)
+        assert never.kind[t] == 0 and np.array_equal(never.out_bits[t], w.hidden[t]) and t not in never.scores
+        # the two comparisons split the hooked rows between them
+        assert (ge.kind[t] != 0) + (lt.kind[t] != 0) == (base.kind[t] != 0)
+        src = ge if sc[t, 1] >= np.float32(0.1) else lt
+        assert np.array_equal(src.out_bits[t], base.out_bits[t])

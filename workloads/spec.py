@@ -28,12 +28,25 @@ SAE_RELU, SAE_JUMPRELU, SAE_TOPK = 0, 1, 2
 EDIT_CLAMP, EDIT_ABLATE = 0, 1
 
 
+GATE_GE, GATE_LT = 0, 1
+
+
+@dataclass
+class Gate:
+    """Activation-driven condition: the app applies to row t iff cmp(scores[t, column], threshold)."""
+    scores: object            # fp32 [T_max, stride]
+    column: int
+    cmp: int                  # GATE_GE | GATE_LT
+    threshold: float
+
+
 @dataclass
 class Probe:
     W: object                 # bf16 [C, d] (torch) or uint16 bits (numpy)
     b: object                 # fp32 [C]
     act: int
     kind: int = KIND_PROBE
+    gate: Optional[Gate] = None
 
     @property
     def n_classes(self) -> int:
@@ -45,6 +58,7 @@ class Steer:
     v: object                 # bf16 [d]
     alpha: float
     kind: int = KIND_STEER
+    gate: Optional[Gate] = None
 
 
 @dataclass
@@ -68,6 +82,7 @@ class SaeApp:
     edit_mode: np.ndarray     # uint8 [r]  EDIT_CLAMP | EDIT_ABLATE
     add_error: bool
     kind: int = KIND_SAE
+    gate: Optional[Gate] = None
 
 
 @dataclass
@@ -111,12 +126,13 @@ def host(w: Workload, only_groups=None) -> Workload:
     the host to check a few rows is pointless); apps of the other sets then count as unhooked."""
     apps = {}
     for s, a in w.apps.items():
+        g = None if a.gate is None else Gate(bits(a.gate.scores), a.gate.column, a.gate.cmp, a.gate.threshold)
         if a.kind == KIND_PROBE:
-            apps[s] = Probe(bits(a.W), bits(a.b), a.act)
+            apps[s] = Probe(bits(a.W), bits(a.b), a.act, gate=g)
         elif a.kind == KIND_STEER:
-            apps[s] = Steer(bits(a.v), float(a.alpha))
+            apps[s] = Steer(bits(a.v), float(a.alpha), gate=g)
         else:
-            apps[s] = a
+            apps[s] = SaeApp(a.group, a.edit_idx, a.edit_val, a.edit_mode, a.add_error, gate=g)
     groups = {
         g: SaeWeights(sw.d_sae, sw.act, sw.k, bits(sw.W_enc), bits(sw.b_enc), bits(sw.W_dec),
                       bits(sw.theta), bits(sw.b_dec), sw.center_input)
