@@ -222,15 +222,17 @@ int mix_apply(mix_ctx* ctx, void* hidden, int T, float* scores_out, void* stream
 int mix_get_status(mix_ctx* ctx, unsigned* bits, void* stream);
 
 /* Number of kernels one mix_apply() call launches on this context (fixed at mix_create):
-   1 without SAE weight sets, else 8 (6 with MIX_FLAG_ENCODE_SIMT). */
+   1 without SAE weight sets, else 8 (6 with MIX_FLAG_ENCODE_SIMT); one more when T_max > 2048
+   and C_max > 1 (multi-class probes of large batches run in a kernel of their own). */
 int mix_launches_per_apply(const mix_ctx* ctx);
 
 /* Per-kernel timing taps (profiling only; do not use while capturing a graph).  events: HOST
    array of mix_launches_per_apply() + 1 cudaEvent_t handles created by the caller with timing
    enabled, or NULL to switch the taps off.  Every later mix_apply() records events[0] before
    its first kernel and events[i] after its i-th kernel, on the call's stream; the array is
-   copied.  Kernel order: probe_steer, route, pack, encode, merge, encode (flagged row tiles),
-   select, decode; with MIX_FLAG_ENCODE_SIMT: probe_steer, route, pack, encode, select, decode. */
+   copied.  Kernel order: probe_steer, [probe_multiclass: only if T_max > 2048 and C_max > 1,]
+   route, pack, encode, merge, encode (flagged row tiles), select, decode; with
+   MIX_FLAG_ENCODE_SIMT the SAE part is route, pack, encode, select, decode. */
 int mix_set_stage_events(mix_ctx* ctx, void* const* events);
 
 /* Test / profiling taps into the SAE workspace after a mix_apply (device pointers owned by

@@ -34,6 +34,9 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
            "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
            "-o", LIB_PATH] + [os.path.join(CSRC, s) for s in SOURCES] + ["-lcudart"]
+    extra = os.environ.get("MIX_NVCC_EXTRA")      # e.g. "-DMIX_SOMETHING" for one-off experiments
+    if extra:
+        cmd[1:1] = extra.split()
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

@@ -249,11 +249,14 @@ class Mix:
 
     @property
     def STAGES(self):
+        front = ["probe_steer"]
+        if self.cfg.T_max > 2048 and self.cfg.C_max > 1:
+            front.append("probe_multiclass")
         if self.cfg.n_groups_max == 0:
-            return ["probe_steer"]
+            return front
         if self.cfg.flags & MIX_FLAG_ENCODE_SIMT:
-            return ["probe_steer", "route", "pack", "encode", "select", "decode"]
-        return ["probe_steer", "route", "pack", "encode", "merge", "encode_flagged", "select", "decode"]
+            return front + ["route", "pack", "encode", "select", "decode"]
+        return front + ["route", "pack", "encode", "merge", "encode_flagged", "select", "decode"]
 
     def set_stage_events(self, events=None):
         """events: list of launches_per_apply() + 1 torch.cuda.Event(enable_timing=True), or None."""

@@ -431,6 +431,10 @@ int mix_apply(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream) 
   MIX_CUDA(c, tap());
   MIX_CUDA(c, launch_probe_steer(c, h, T, scores_out, s));
   MIX_CUDA(c, tap());
+  if (has_multiclass_stage(c)) {
+    MIX_CUDA(c, launch_probe_multiclass(c, h, T, scores_out, s));
+    MIX_CUDA(c, tap());
+  }
   if (c->cfg.n_groups_max > 0) {
     MIX_CUDA(c, launch_route(c, T, s));
     MIX_CUDA(c, tap());
@@ -459,8 +463,9 @@ int mix_apply(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream) 
 
 int mix_launches_per_apply(const mix_ctx* c) {
   if (!c) return 0;
-  if (c->cfg.n_groups_max == 0) return 1;
-  return (c->cfg.flags & MIX_FLAG_ENCODE_SIMT) ? 6 : 8;
+  const int front = has_multiclass_stage(c) ? 2 : 1;
+  if (c->cfg.n_groups_max == 0) return front;
+  return front + ((c->cfg.flags & MIX_FLAG_ENCODE_SIMT) ? 5 : 7);
 }
 
 int mix_get_status(mix_ctx* c, unsigned* bits, void* stream) {

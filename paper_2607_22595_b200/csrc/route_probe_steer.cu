@@ -164,7 +164,7 @@ __device__ __forceinline__ bool gate_open(const GateEntry* __restrict__ gates, i
 // thread that may raise status.
 __device__ __forceinline__ RowApp lookup(int s, int t, const AppEntry* __restrict__ apps,
                                          const GateEntry* __restrict__ gates, int n_slots,
-                                         unsigned* __restrict__ status, bool leader) {
+                                         unsigned* __restrict__ status, bool leader, bool eval_gate = true) {
   RowApp r;
   r.kind = 0;
   r.gated = false;
@@ -181,7 +181,7 @@ __device__ __forceinline__ RowApp lookup(int s, int t, const AppEntry* __restric
     return r;
   }
   r.gated = (q0.y & kKindGated) != 0;
-  if (r.gated && !gate_open(gates, s, t)) return r;               // gate closed: the row passes through
+  if (eval_gate && r.gated && !gate_open(gates, s, t)) return r;  // gate closed: the row passes through
   r.kind = q0.y & kKindMask;
   r.C = q0.z;
   r.act = q0.w;
@@ -192,7 +192,7 @@ __device__ __forceinline__ RowApp lookup(int s, int t, const AppEntry* __restric
 }
 
 constexpr int kWarpsPerBlock = 8;      // = rows per CTA of the large-batch kernel
-constexpr int kRowGroup = 4;           // rows that share one pass over a probe matrix
+constexpr int kCoopMaxClasses = 32;    // widest probe the cooperative tensor-core pass takes
 
 // One row, one warp: steer, single-class probe, or multi-class probe.
 __device__ __forceinline__ void warp_row(const RowApp& a, __nv_bfloat16* __restrict__ hidden, int t, int d,
@@ -215,13 +215,13 @@ __device__ __forceinline__ void warp_row(const RowApp& a, __nv_bfloat16* __restr
     }
     return;
   }
-  for (int c0 = 0; c0 < a.C; c0 += 8) {
-    float z[1][8];
-    const int nc = min(8, a.C - c0);
-    probe_dots<1, 8>(h1, a.W + (size_t)c0 * nvec, nvec, nc, lane, 32, z);
+  for (int c0 = 0; c0 < a.C; c0 += 4) {
+    float z[1][4];
+    const int nc = min(4, a.C - c0);
+    probe_dots<1, 4>(h1, a.W + (size_t)c0 * nvec, nvec, nc, lane, 32, z);
     if (lane == 0) {
 #pragma unroll
-      for (int c = 0; c < 8; ++c)
+      for (int c = 0; c < 4; ++c)
         if (c < nc) s_logit[c0 + c] = z[0][c] + (a.b ? __ldg(a.b + c0 + c) : 0.f);
     }
   }
@@ -229,62 +229,170 @@ __device__ __forceinline__ void warp_row(const RowApp& a, __nv_bfloat16* __restr
   finish_probe(s_logit, a.C, a.act, out, lane);
 }
 
-// Large batches: a CTA owns 8 consecutive rows, one warp per row.  Consecutive rows usually
-// belong to one request; when all 8 share a multi-class probe the CTA switches to a
-// cooperative pass (columns split over the warps, kRowGroup rows x 4 classes per pass) that
-// streams the probe matrix from L2 twice per 8 rows instead of eight times.
+// Large batches: a CTA owns 8 consecutive rows, one warp per row: streaming work (steering,
+// single-class probes).  Multi-class probes up to kCoopMaxClasses classes are left to
+// probe_multiclass_kernel when `multiclass_elsewhere` is set.
 __global__ void __launch_bounds__(kWarpsPerBlock * 32, 3)
 probe_steer_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
                    const AppEntry* __restrict__ apps, const GateEntry* __restrict__ gates, int n_slots,
                    __nv_bfloat16* __restrict__ hidden, int d,
-                   float* __restrict__ scores, int C_max, unsigned* __restrict__ status) {
-  __shared__ float s_part[kWarpsPerBlock][kWarpsPerBlock][kMaxClasses];   // [warp][row][class]
-  __shared__ int s_slot[kWarpsPerBlock];
+                   float* __restrict__ scores, int C_max, unsigned* __restrict__ status, int multiclass_elsewhere) {
+  __shared__ float s_logit[kWarpsPerBlock][kMaxClasses];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int t0 = blockIdx.x * kWarpsPerBlock;
-  const int n_live = min(T, __ldg(n_live_p));
-  if (t0 >= n_live) return;
-  const int t = t0 + warp;
-  const int my_slot = t < n_live ? __ldg(token_slot + t) : -1;
-  if (lane == 0) s_slot[warp] = my_slot;
-  __syncthreads();
-  bool same = t0 + kWarpsPerBlock <= n_live && s_slot[0] >= 0 && scores != nullptr;
+  const int t = blockIdx.x * kWarpsPerBlock + warp;
+  if (t >= min(T, __ldg(n_live_p))) return;
+  const RowApp a = lookup(__ldg(token_slot + t), t, apps, gates, n_slots, status, lane == 0);
+  if (a.kind == 0) return;
+  if (multiclass_elsewhere && a.kind == MIX_PROBE && a.C > 1 && a.C <= kCoopMaxClasses) return;
+  warp_row(a, hidden, t, d, scores, C_max, s_logit[warp], lane);
+}
+
+// 16-byte read-only load that the compiler may not sink below later volatile statements: keeps
+// all loads of a batch in flight before the first MMA that consumes them.
+__device__ __forceinline__ uint4 ldg128_early(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+constexpr int kMcRows = 16;            // rows per CTA of probe_multiclass_kernel (one m16 MMA tile)
+constexpr int kMcWarps = 8;            // warps per CTA: they split d between them
+
+// One warp's share of the contraction of 16 rows against one probe matrix on the warp-level
+// tensor-core MMA (m16n8k16, bf16 -> fp32): every kMcWarps-th 32-column chunk of d, UB chunks in flight,
+// KCT 8-class tiles.  Fragments come straight from global memory, 16 contiguous bytes per lane:
+// lane (g, q) takes columns 8q..8q+7 of the chunk for rows g and g + 8 and for class g of each
+// 8-class tile.  Which columns a fragment slot holds is immaterial as long as A and B agree,
+// because the sum runs over all of them.  Partial logits go to part[row][class].
+template <int KCT, int UB>
+__device__ __forceinline__ void mc_contract(const uint4* __restrict__ h_lo, const uint4* __restrict__ h_hi,
+                                            const uint4* __restrict__ W, int C, int n_chunks, int row_vecs,
+                                            float (*part)[kCoopMaxClasses]) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, q = lane & 3;
+  float acc[KCT][4];
 #pragma unroll
-  for (int r = 1; r < kWarpsPerBlock; ++r) same = same && s_slot[r] == s_slot[0];
-  const RowApp a = lookup(my_slot, t, apps, gates, n_slots, status, lane == 0);
-  // one decision for the whole CTA (a gate can open for some rows of a request and not others)
-  if (!__syncthreads_and(same && a.kind == MIX_PROBE && a.C > 1 && !a.gated)) {
-    if (t < n_live) warp_row(a, hidden, t, d, scores, C_max, s_part[warp][0], lane);
-    return;
-  }
-  const int nvec = d >> 3;
-  for (int rg = 0; rg < kWarpsPerBlock; rg += kRowGroup) {
-    const uint4* h[kRowGroup];
+  for (int ct = 0; ct < KCT; ++ct) acc[ct][0] = acc[ct][1] = acc[ct][2] = acc[ct][3] = 0.f;
+  for (int ch0 = warp; ch0 < n_chunks; ch0 += kMcWarps * UB) {
+    uint4 lo[UB], hi[UB], wq[UB][KCT];
 #pragma unroll
-    for (int r = 0; r < kRowGroup; ++r) h[r] = reinterpret_cast<const uint4*>(hidden + (size_t)(t0 + rg + r) * d);
-    for (int c0 = 0; c0 < a.C; c0 += 4) {
-      float z[kRowGroup][4];
-      const int nc = min(4, a.C - c0);
-      probe_dots<kRowGroup, 4>(h, a.W + (size_t)c0 * nvec, nvec, nc, threadIdx.x, kWarpsPerBlock * 32, z);
-      if (lane == 0) {
+    for (int u = 0; u < UB; ++u) {
+      const int ch = ch0 + u * kMcWarps;
+      const bool in = ch < n_chunks;
+      lo[u] = in ? ldg128_early(h_lo + ch * 4 + q) : make_uint4(0u, 0u, 0u, 0u);
+      hi[u] = in ? ldg128_early(h_hi + ch * 4 + q) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-        for (int r = 0; r < kRowGroup; ++r)
+      for (int ct = 0; ct < KCT; ++ct) {
+        const int cls = ct * 8 + g;
+        wq[u][ct] = (in && cls < C) ? ldg128_early(W + (size_t)cls * row_vecs + ch * 4 + q) : make_uint4(0u, 0u, 0u, 0u);
+      }
+    }
 #pragma unroll
-          for (int c = 0; c < 4; ++c)
-            if (c < nc) s_part[warp][rg + r][c0 + c] = z[r][c];
+    for (int u = 0; u < UB; ++u) {
+#pragma unroll
+      for (int ct = 0; ct < KCT; ++ct) {
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+            "{%0, %1, %2, %3};"
+            : "+f"(acc[ct][0]), "+f"(acc[ct][1]), "+f"(acc[ct][2]), "+f"(acc[ct][3])
+            : "r"(lo[u].x), "r"(hi[u].x), "r"(lo[u].y), "r"(hi[u].y), "r"(wq[u][ct].x), "r"(wq[u][ct].y));
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+            "{%0, %1, %2, %3};"
+            : "+f"(acc[ct][0]), "+f"(acc[ct][1]), "+f"(acc[ct][2]), "+f"(acc[ct][3])
+            : "r"(lo[u].z), "r"(hi[u].z), "r"(lo[u].w), "r"(hi[u].w), "r"(wq[u][ct].z), "r"(wq[u][ct].w));
       }
     }
   }
-  __syncthreads();
-  // warp r finishes row r: sum the 8 column shares, add the bias, activate
-  for (int c = lane; c < a.C; c += 32) {
-    float z = a.b ? __ldg(a.b + c) : 0.f;
+  // lane (g, q): rows g (acc 0, 1) and g + 8 (acc 2, 3), classes 8 ct + 2q and + 1
 #pragma unroll
-    for (int w = 0; w < kWarpsPerBlock; ++w) z += s_part[w][warp][c];
-    s_part[0][warp][c] = z;     // s_part[*][warp][*] is read and written by this warp only
+  for (int ct = 0; ct < KCT; ++ct) {
+    if (ct * 8 < C) {
+      part[g][ct * 8 + 2 * q] = acc[ct][0];
+      part[g][ct * 8 + 2 * q + 1] = acc[ct][1];
+      part[g + 8][ct * 8 + 2 * q] = acc[ct][2];
+      part[g + 8][ct * 8 + 2 * q + 1] = acc[ct][3];
+    }
   }
-  __syncwarp();
-  finish_probe(s_part[0][warp], a.C, a.act, scores + (size_t)t * C_max, lane);
+}
+
+// What the CTA knows about each of its rows.
+struct McRow {
+  const uint4* W;
+  const float* b;
+  int C, act;
+  int slot;      // slot id if the row is a multi-class probe this kernel takes and its gate is open, else -1
+};
+
+// Multi-class probes of large batches.  16 rows x C classes x d is a skinny dense contraction;
+// consecutive rows usually belong to one request and share the probe.  For every distinct
+// multi-class probe among the CTA's 16 rows, the warps split d between them and contract ALL
+// 16 rows against that probe's matrix, which is therefore streamed from L2 once per 16 rows;
+// only the rows that belong to the probe keep their result.
+__global__ void __launch_bounds__(kMcWarps * 32, 2)
+probe_multiclass_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
+                        const AppEntry* __restrict__ apps, const GateEntry* __restrict__ gates, int n_slots,
+                        const __nv_bfloat16* __restrict__ hidden, int d, float* __restrict__ scores, int C_max) {
+  __shared__ float s_part[kMcWarps][kMcRows][kCoopMaxClasses];   // [warp][row][class]
+  __shared__ float s_logit[kMcWarps][kCoopMaxClasses];
+  __shared__ McRow s_row[kMcRows];
+  __shared__ int s_any;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t0 = blockIdx.x * kMcRows;
+  const int n_live = min(T, __ldg(n_live_p));
+  if (t0 >= n_live || scores == nullptr) return;
+  if (threadIdx.x == 0) s_any = 0;
+  __syncthreads();
+  if (threadIdx.x < kMcRows) {           // one thread per row: slot -> entry -> gate
+    const int t = t0 + threadIdx.x;
+    McRow r;
+    r.slot = -1;
+    if (t < n_live) {
+      const int s = __ldg(token_slot + t);
+      const RowApp a = lookup(s, t, apps, gates, n_slots, nullptr, false);   // bad slots are flagged by probe_steer_kernel
+      if (a.kind == MIX_PROBE && a.C > 1 && a.C <= kCoopMaxClasses) {
+        r.W = a.W;
+        r.b = a.b;
+        r.C = a.C;
+        r.act = a.act;
+        r.slot = s;
+        s_any = 1;
+      }
+    }
+    s_row[threadIdx.x] = r;
+  }
+  __syncthreads();
+  if (!s_any) return;                    // CTA-uniform
+  const int g = lane >> 2;
+  const uint4* h_lo = reinterpret_cast<const uint4*>(hidden + (size_t)min(t0 + g, n_live - 1) * d);
+  const uint4* h_hi = reinterpret_cast<const uint4*>(hidden + (size_t)min(t0 + g + 8, n_live - 1) * d);
+  const int n_chunks = d >> 5, row_vecs = d >> 3;
+  for (int r = 0; r < kMcRows; ++r) {
+    const McRow ci = s_row[r];
+    if (ci.slot < 0) continue;
+    bool first = true;
+    for (int r2 = 0; r2 < r; ++r2) first = first && s_row[r2].slot != ci.slot;
+    if (!first) continue;
+    if (ci.C <= 16)
+      mc_contract<2, 4>(h_lo, h_hi, ci.W, ci.C, n_chunks, row_vecs, s_part[warp]);
+    else
+      mc_contract<kCoopMaxClasses / 8, 2>(h_lo, h_hi, ci.W, ci.C, n_chunks, row_vecs, s_part[warp]);
+    __syncthreads();
+#pragma unroll 1
+    for (int rr = warp; rr < kMcRows; rr += kMcWarps) {     // warp w finishes row w
+      if (s_row[rr].slot != ci.slot) continue;
+      for (int c = lane; c < ci.C; c += 32) {
+        float z = ci.b ? __ldg(ci.b + c) : 0.f;
+#pragma unroll
+        for (int w = 0; w < kMcWarps; ++w) z += s_part[w][rr][c];
+        s_logit[warp][c] = z;
+      }
+      __syncwarp();
+      finish_probe(s_logit[warp], ci.C, ci.act, scores + (size_t)(t0 + rr) * C_max, lane);
+      __syncwarp();
+    }
+    __syncthreads();                     // s_part is reused by the next probe
+  }
 }
 
 // Small batches (decode): one CTA of NW warps per row, the row held in registers (up to kTeamVec
@@ -540,6 +648,8 @@ __global__ void fold_bias_kernel(const __nv_bfloat16* __restrict__ W_enc, const 
 
 constexpr int kTeamMaxRows = 2048;   // up to here one CTA per row keeps the whole GPU busy
 
+bool has_multiclass_stage(const Ctx* c) { return c->cfg.T_max > kTeamMaxRows && c->cfg.C_max > 1; }
+
 cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s) {
   if (c->cfg.T_max <= kTeamMaxRows) {
     probe_steer_team_kernel<8><<<c->cfg.T_max, 8 * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates,
@@ -549,8 +659,16 @@ cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float
     const int blocks = (c->cfg.T_max + kWarpsPerBlock - 1) / kWarpsPerBlock;
     probe_steer_kernel<<<blocks, kWarpsPerBlock * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates,
                                                               c->cfg.n_slots_max, hidden, c->cfg.d_model, scores,
-                                                              c->cfg.C_max, c->d_status);
+                                                              c->cfg.C_max, c->d_status, has_multiclass_stage(c) ? 1 : 0);
   }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_probe_multiclass(const Ctx* c, const __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s) {
+  const int blocks = (c->cfg.T_max + kMcRows - 1) / kMcRows;
+  probe_multiclass_kernel<<<blocks, kMcWarps * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates,
+                                                                 c->cfg.n_slots_max, hidden, c->cfg.d_model, scores,
+                                                                 c->cfg.C_max);
   return cudaGetLastError();
 }
 
