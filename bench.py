@@ -423,25 +423,36 @@ def run_mix(args, rank, world, local_rank):
     floor_us = e0.elapsed_time(e1) * 1e3 / (4 * min(R, 256))
     m.set_slot_map(torch.from_numpy(w.token_slot.copy()).cuda(), w.T_live)
 
-    # end to end through the public API with host buffers
+    # end to end through the public API with host buffers: every step copies its hidden states
+    # and slot map from pinned host memory, applies the hook, and copies hidden + scores back.
+    # Steps are independent batches, so they are pipelined over a few contexts (one stream and
+    # one device buffer each): the H2D of one step overlaps the D2H of another, as a serving
+    # engine with several batches in flight would do.
     K_e2e = min(K, 2000)
-    h_in = torch.empty((T, d), dtype=torch.bfloat16).pin_memory(); h_in.copy_(w.hidden.cpu())
-    h_out = torch.empty((T, d), dtype=torch.bfloat16).pin_memory()
-    s_out = torch.empty((T, 1), dtype=torch.float32).pin_memory()
-    slot_pin = torch.from_numpy(w.token_slot.copy()).pin_memory()
-    hd, sd = hiddens[0], scores[0]
-    def e2e_step():
-        hd.copy_(h_in, non_blocking=True)
-        m.set_slot_map(slot_pin, w.T_live)
-        m.apply(hd, sd)
-        h_out.copy_(hd, non_blocking=True)
-        s_out.copy_(sd, non_blocking=True)
-    for _ in range(3):
-        e2e_step()
+    n_pipe = 3
+    pipes = []
+    for i in range(n_pipe):
+        mi = m if i == 0 else W.make_context(mixlib.Mix, w)
+        h_in = torch.empty((T, d), dtype=torch.bfloat16).pin_memory(); h_in.copy_(w.hidden.cpu())
+        pipes.append(dict(m=mi, st=torch.cuda.Stream(), h_in=h_in,
+                          h_out=torch.empty((T, d), dtype=torch.bfloat16).pin_memory(),
+                          s_out=torch.empty((T, 1), dtype=torch.float32).pin_memory(),
+                          slot=torch.from_numpy(w.token_slot.copy()).pin_memory(), hd=hiddens[i], sd=scores[i]))
+    def e2e_step(i):
+        p = pipes[i % n_pipe]
+        with torch.cuda.stream(p["st"]):
+            p["hd"].copy_(p["h_in"], non_blocking=True)
+            p["m"].set_slot_map(p["slot"], w.T_live, stream=p["st"])
+            p["m"].apply(p["hd"], p["sd"], stream=p["st"])
+            p["h_out"].copy_(p["hd"], non_blocking=True)
+            p["s_out"].copy_(p["sd"], non_blocking=True)
+    torch.cuda.synchronize()
+    for i in range(2 * n_pipe):
+        e2e_step(i)
     torch.cuda.synchronize(); barrier(world)
     te = time.perf_counter()
-    for _ in range(K_e2e):
-        e2e_step()
+    for i in range(K_e2e):
+        e2e_step(i)
     torch.cuda.synchronize()
     e2e_s = dist_max(time.perf_counter() - te, world)
     sampler.stop()
@@ -464,7 +475,7 @@ def run_mix(args, rank, world, local_rank):
                    "status_word": status},
         "clocks": clocks,
         "e2e": {"value": e2e_rows / e2e_s, "unit": UNIT, "h2d_bytes_per_step": T * d * 2 + 4 * T,
-                "d2h_bytes_per_step": T * d * 2 + 4 * T, "steps": K_e2e},
+                "d2h_bytes_per_step": T * d * 2 + 4 * T, "steps": K_e2e, "pipeline_depth": n_pipe},
         "gpu_launches": K * m.launches_per_apply(),
         "roofline": {"bound": "hbm", "kernel": "probe_steer_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],

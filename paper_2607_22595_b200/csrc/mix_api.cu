@@ -63,7 +63,7 @@ void free_all(mix_ctx* c) {
   cudaFree(c->d_token_slot); cudaFree(c->d_n_live); cudaFree(c->d_apps); cudaFree(c->d_groups); cudaFree(c->d_gates);
   cudaFree(c->d_edit_idx); cudaFree(c->d_edit_val); cudaFree(c->d_edit_mode); cudaFree(c->d_status);
   cudaFree(c->d_tmp_req); cudaFree(c->d_tmp_req_slot); cudaFree(c->d_panel); cudaFree(c->d_panel_row);
-  cudaFree(c->d_mtile_group); cudaFree(c->d_route); cudaFree(c->d_z); cudaFree(c->d_topk_idx);
+  cudaFree(c->d_mtile_group); cudaFree(c->d_row_group); cudaFree(c->d_route); cudaFree(c->d_z); cudaFree(c->d_topk_idx);
   cudaFree(c->d_topk_val); cudaFree(c->d_tmap_w); cudaFree(c->d_cand_val); cudaFree(c->d_cand_idx);
   cudaFree(c->d_cand_ninth); cudaFree(c->d_row_flag); cudaFree(c->d_mtile_flag); cudaFree(c->d_n_flagged);
   if (c->owned_b_eff)
@@ -153,6 +153,7 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
     ok = ok && dev_alloc(&c->d_panel, P * cfg->d_model) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_panel_row, P) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_mtile_group, P / kTileM) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_row_group, T) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_route, 1) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_z, P * (size_t)cfg->d_sae_max) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_topk_idx, P * (size_t)c->cfg.k_max) == cudaSuccess;

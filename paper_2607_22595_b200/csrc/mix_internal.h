@@ -104,6 +104,7 @@ struct Ctx {
   __nv_bfloat16* d_panel;   // [P, d]
   int* d_panel_row;         // [P] token index or -1
   int* d_mtile_group;       // [P / kTileM] group of each m-tile or -1
+  int* d_row_group;         // [T_max] routing scratch: weight set of each token row or -1
   RouteState* d_route;
   float* d_z;               // [P, d_sae_max]
   int* d_topk_idx;          // [P, k_max]

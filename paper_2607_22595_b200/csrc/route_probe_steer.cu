@@ -500,6 +500,7 @@ probe_steer_team_kernel(const int* __restrict__ token_slot, const int* __restric
 // ---------------------------------------------------------------------------------------
 constexpr int kRouteThreads = 1024;
 constexpr int kRouteWarps = kRouteThreads / 32;
+constexpr int kRouteBatch = 8;          // chunks of 1024 rows whose lookups are in flight together
 
 __global__ void __launch_bounds__(kRouteThreads)
 route_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
@@ -507,7 +508,7 @@ route_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_
              const GroupEntry* __restrict__ groups, int n_groups,
              int* __restrict__ panel_row, int panel_cap, int* __restrict__ mtile_group, RouteState* __restrict__ rs,
              unsigned* __restrict__ status, int* __restrict__ row_flag, int* __restrict__ mtile_flag,
-             int* __restrict__ n_flagged) {
+             int* __restrict__ n_flagged, int* __restrict__ row_group) {
   extern __shared__ int s_cnt[];                      // [n_chunks * kRouteWarps][n_groups]
   __shared__ int s_total[kMaxGroups], s_base[kMaxGroups + 1];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -522,27 +523,51 @@ route_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_
     if (tid == 0) *n_flagged = 0;
   }
 
-  auto group_of = [&](int t) -> int {
-    if (t >= n_live) return -1;
-    const int s = token_slot[t];
-    if (s < 0 || s >= n_slots) return -1;
-    const AppEntry* e = apps + s;
-    if (!e->valid || (e->kind & kKindMask) != MIX_SAE) return -1;
-    if ((e->kind & kKindGated) && !gate_open(gates, s, t)) return -1;
-    const int g = e->group;
-    if (g < 0 || g >= n_groups || !groups[g].valid) {
-      atomicOr(status, MIX_STATUS_BAD_GROUP);
-      return -1;
+  // phase A: the group of every row this thread owns (row c * 1024 + tid of chunk c), resolved
+  // stage by stage for kRouteBatch chunks at a time so that their loads are in flight together
+  // (slot ids, then app entries, then weight-set entries: three round trips per batch instead
+  // of three per chunk); then per (chunk, warp) counts per group.
+  for (int c0 = 0; c0 < n_chunks; c0 += kRouteBatch) {
+    int slot[kRouteBatch], grp[kRouteBatch];
+#pragma unroll
+    for (int c = 0; c < kRouteBatch; ++c) {
+      const int t = (c0 + c) * kRouteThreads + tid;
+      slot[c] = (c0 + c < n_chunks && t < n_live) ? __ldg(token_slot + t) : -1;
+      if (slot[c] >= n_slots) slot[c] = -1;
     }
-    return g;
-  };
-
-  // phase A: per (chunk, warp) counts per group
-  for (int c = 0; c < n_chunks; ++c) {
-    const int g = group_of(c * kRouteThreads + tid);
-    for (int q = 0; q < n_groups; ++q) {
-      const unsigned m = __ballot_sync(0xffffffffu, g == q);
-      if (lane == 0) s_cnt[(c * kRouteWarps + warp) * n_groups + q] = __popc(m);
+    int2 head[kRouteBatch];
+    int group_id[kRouteBatch];
+#pragma unroll
+    for (int c = 0; c < kRouteBatch; ++c) {
+      head[c] = make_int2(0, 0);
+      group_id[c] = -1;
+      if (slot[c] >= 0) {
+        head[c] = __ldg(reinterpret_cast<const int2*>(apps + slot[c]));          // valid, kind
+        group_id[c] = __ldg(&apps[slot[c]].group);
+      }
+    }
+#pragma unroll
+    for (int c = 0; c < kRouteBatch; ++c) {
+      grp[c] = -1;
+      if (head[c].x && (head[c].y & kKindMask) == MIX_SAE) {
+        const int g = group_id[c];
+        if (g < 0 || g >= n_groups || !__ldg(&groups[g].valid)) {
+          atomicOr(status, MIX_STATUS_BAD_GROUP);
+        } else if (!(head[c].y & kKindGated) || gate_open(gates, slot[c], (c0 + c) * kRouteThreads + tid)) {
+          grp[c] = g;
+        }
+      }
+    }
+#pragma unroll
+    for (int c = 0; c < kRouteBatch; ++c) {
+      if (c0 + c < n_chunks) {                       // uniform across the CTA
+        const int t = (c0 + c) * kRouteThreads + tid;
+        if (t < n_live) row_group[t] = grp[c];       // read back by this same thread in phase C
+        for (int q = 0; q < n_groups; ++q) {
+          const unsigned m = __ballot_sync(0xffffffffu, grp[c] == q);
+          if (lane == 0) s_cnt[((c0 + c) * kRouteWarps + warp) * n_groups + q] = __popc(m);
+        }
+      }
     }
   }
   __syncthreads();
@@ -593,14 +618,24 @@ route_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_
   }
   __syncthreads();
   // phase C: stable scatter
-  for (int c = 0; c < n_chunks; ++c) {
-    const int t = c * kRouteThreads + tid;
-    const int g = group_of(t);
-    for (int q = 0; q < n_groups; ++q) {
-      const unsigned m = __ballot_sync(0xffffffffu, g == q);
-      if (g == q) {
-        const int pos = s_base[q] + s_cnt[(c * kRouteWarps + warp) * n_groups + q] + __popc(m & ((1u << lane) - 1u));
-        panel_row[pos] = t;
+  for (int c0 = 0; c0 < n_chunks; c0 += kRouteBatch) {
+    int grp[kRouteBatch];
+#pragma unroll
+    for (int c = 0; c < kRouteBatch; ++c) {
+      const int t = (c0 + c) * kRouteThreads + tid;
+      grp[c] = t < n_live ? row_group[t] : -1;
+    }
+#pragma unroll
+    for (int c = 0; c < kRouteBatch; ++c) {
+      if (c0 + c < n_chunks) {
+        for (int q = 0; q < n_groups; ++q) {
+          const unsigned m = __ballot_sync(0xffffffffu, grp[c] == q);
+          if (grp[c] == q) {
+            const int pos = s_base[q] + s_cnt[((c0 + c) * kRouteWarps + warp) * n_groups + q] +
+                            __popc(m & ((1u << lane) - 1u));
+            panel_row[pos] = (c0 + c) * kRouteThreads + tid;
+          }
+        }
       }
     }
   }
@@ -678,7 +713,7 @@ cudaError_t launch_route(const Ctx* c, int T, cudaStream_t s) {
   route_kernel<<<1, kRouteThreads, smem, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates, c->cfg.n_slots_max,
                                               c->d_groups, c->cfg.n_groups_max, c->d_panel_row, c->panel_rows_cap,
                                               c->d_mtile_group, c->d_route, c->d_status, c->d_row_flag,
-                                              c->d_mtile_flag, c->d_n_flagged);
+                                              c->d_mtile_flag, c->d_n_flagged, c->d_row_group);
   return cudaGetLastError();
 }
 

@@ -36,7 +36,8 @@ constexpr size_t kOffEditMode = kOffEditVal + align256(kMaxEdits * sizeof(float)
 constexpr size_t kOffRoute = kOffEditMode + align256(kMaxEdits);
 constexpr size_t kOffPanelRow = kOffRoute + align256(sizeof(RouteState));
 constexpr size_t kOffMtileGroup = kOffPanelRow + align256(kStaticRows * sizeof(int));
-constexpr size_t kOffTopkIdx = kOffMtileGroup + 256;
+constexpr size_t kOffRowGroup = kOffMtileGroup + 256;
+constexpr size_t kOffTopkIdx = kOffRowGroup + align256(kStaticRows * sizeof(int));
 constexpr size_t kOffTopkVal = kOffTopkIdx + align256((size_t)kStaticRows * kStaticK * sizeof(int));
 constexpr size_t kOffPanel = kOffTopkVal + align256((size_t)kStaticRows * kStaticK * sizeof(float));
 constexpr size_t kOffZ = kOffPanel + align256((size_t)kStaticRows * kStaticD * sizeof(__nv_bfloat16));
@@ -130,6 +131,7 @@ extern "C" int mix_sae_apply_static(void* hidden, int n_rows, int d_model, const
   c.d_route = reinterpret_cast<RouteState*>(base + kOffRoute);
   c.d_panel_row = reinterpret_cast<int*>(base + kOffPanelRow);
   c.d_mtile_group = reinterpret_cast<int*>(base + kOffMtileGroup);
+  c.d_row_group = reinterpret_cast<int*>(base + kOffRowGroup);
   c.d_topk_idx = reinterpret_cast<int*>(base + kOffTopkIdx);
   c.d_topk_val = reinterpret_cast<float*>(base + kOffTopkVal);
   c.d_panel = reinterpret_cast<__nv_bfloat16*>(base + kOffPanel);
