@@ -33,6 +33,10 @@ METRIC = "mi_hook_token_rows_per_s"
 UNIT = "token-rows/s"
 WORKLOAD = "decode: d=4096, T=256 (256 requests x 1 token), 64 probes + 32 steering vectors, 25% unhooked"
 ROTATE_BYTES = 512 << 20
+# dram__bytes_read.sum + dram__bytes_write.sum of one probe_steer_team_kernel launch on this workload,
+# from the ncu capture summarised in profiles/probe_steer_kernel_decode.md (reads 2.40 MB, writes 0:
+# the steered rows are still dirty in L2 when the kernel ends).
+DECODE_DRAM_BYTES_PER_LAUNCH = 2399232
 
 
 def measured_peaks():
@@ -477,8 +481,9 @@ def run_mix(args, rank, world, local_rank):
         "e2e": {"value": e2e_rows / e2e_s, "unit": UNIT, "h2d_bytes_per_step": T * d * 2 + 4 * T,
                 "d2h_bytes_per_step": T * d * 2 + 4 * T, "steps": K_e2e, "pipeline_depth": n_pipe},
         "gpu_launches": K * m.launches_per_apply(),
-        "roofline": {"bound": "hbm", "kernel": "probe_steer_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
-                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+        "roofline": {"bound": "hbm", "kernel": "probe_steer_team_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": DECODE_DRAM_BYTES_PER_LAUNCH,
+                     "peak_source": peaks["source"],
                      "algorithmic_bytes_per_launch": nbytes,
                      "note": "2.9 MB per launch: launch-latency-bound, not bandwidth-bound; see extras.sweep for the same kernel on 2 GiB"},
     }
