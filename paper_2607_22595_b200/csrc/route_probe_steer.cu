@@ -211,7 +211,8 @@ __device__ __forceinline__ void warp_row(const RowApp& a, __nv_bfloat16* __restr
     probe_dots<1, 1>(h1, a.W, nvec, 1, lane, 32, z);
     if (lane == 0) {
       const float zz = z[0][0] + (a.b ? __ldg(a.b) : 0.f);
-      out[0] = (a.act == MIX_ACT_NONE) ? zz : 1.f / (1.f + expf(-zz));
+      // one class: raw logit, sigmoid, or a softmax over a single entry (= 1)
+      out[0] = a.act == MIX_ACT_NONE ? zz : (a.act == MIX_ACT_SOFTMAX ? 1.f : 1.f / (1.f + expf(-zz)));
     }
     return;
   }

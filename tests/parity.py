@@ -66,8 +66,11 @@ def bf16_ulp(x):
     return 2.0 ** (np.floor(np.log2(a)) - 7)
 
 
-def check_parity(wh, out, rows=None, expect_status=0, check_features=True):
-    """wh: host workload (numpy); out: run_gpu result.  Asserts parity on `rows` (default all)."""
+def check_parity(wh, out, rows=None, expect_status=0, check_features=True, scale_with_output=False):
+    """wh: host workload (numpy); out: run_gpu result.  Asserts parity on `rows` (default all).
+    scale_with_output: take the hidden-state bound as 1e-2 * max(|h_in|, |y_ref|) -- for inputs where
+    an app's output dwarfs the hidden state (a huge steering vector on a tiny h), so that the bf16
+    rounding of the output alone would exceed 1e-2 * max|h_in|."""
     T = wh.T_max
     rows = list(range(T)) if rows is None else sorted(set(int(r) for r in rows))
     ref = O.apply_hook(wh, rows, keep_z=True)
@@ -108,6 +111,8 @@ def check_parity(wh, out, rows=None, expect_status=0, check_features=True):
             if diff:
                 stats["topk_swaps"] += 1
                 redo[t] = K_gpu
+    if scale_with_output:
+        hmax = max([hmax] + [float(np.abs(ref.y[t]).max()) for t in rows if ref.kind[t] in (O.KIND_STEER, O.KIND_SAE)])
     if redo:       # re-evaluate those rows with the GPU's (valid) choice among near-ties
         ref2 = O.apply_hook(wh, list(redo), topk_override=redo)
         for t in redo:

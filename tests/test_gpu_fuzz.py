@@ -1,0 +1,86 @@
+"""Seeded random small workloads (shapes, app mixes, live counts, gates, edit lists) through the
+C ABI against the oracle.  Every case is tiny; together they sweep the corners the fixed
+configurations do not: widths that are not powers of two, one-row batches, weight sets with no
+rows, slots shared by many requests, edits that repeat a feature, T_live in the middle of a
+request, both encode paths."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as W
+
+from parity import check_parity, run_gpu
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def random_workload(seed):
+    rng = np.random.default_rng(seed)
+    g = torch.Generator(device=DEV); g.manual_seed(int(seed))
+    d = int(rng.choice([64, 128, 192, 320, 512]))
+    T = int(rng.choice([1, 7, 33, 128, 129, 300, 2100]))       # 2100 > 2048: the large-batch kernels
+    n_groups = int(rng.integers(0, 4))
+    hidden = (torch.randn((T, d), generator=g, device=DEV) * float(rng.choice([0.1, 1.0, 8.0]))).to(torch.bfloat16)
+    apps, groups = {}, {}
+    slot = 0
+    C_max = int(rng.choice([1, 3, 16, 40]))
+    for _ in range(int(rng.integers(1, 4))):                    # probes
+        C = 1 if C_max == 1 or rng.random() < 0.4 else int(rng.integers(2, C_max + 1))
+        act = W.ACT_SIGMOID if C == 1 and rng.random() < 0.7 else (W.ACT_NONE if rng.random() < 0.3 else W.ACT_SOFTMAX)
+        Wp = (torch.randn((C, d), generator=g, device=DEV) * d ** -0.5).to(torch.bfloat16)
+        b = torch.randn(C, generator=g, device=DEV) * 0.3 if rng.random() < 0.5 else None
+        apps[slot] = W.Probe(Wp, b, act); slot += 1
+    for _ in range(int(rng.integers(1, 4))):                    # steering vectors
+        v = torch.randn(d, generator=g, device=DEV).to(torch.bfloat16)
+        apps[slot] = W.Steer(v, float(np.float32(rng.uniform(-6, 6)))); slot += 1
+    k_max = r_max = 1
+    d_sae_max = 0
+    for gi in range(n_groups):
+        S = int(rng.choice([256, 512, 1280, 2048]))
+        act = int(rng.choice([W.SAE_RELU, W.SAE_JUMPRELU, W.SAE_TOPK]))
+        k = int(rng.integers(1, min(48, S // 8))) if act == W.SAE_TOPK else 0
+        sae = W.make_sae_weights(g, DEV, d, S, act, k=k, theta_range=(0.05, 0.3),
+                                 b_enc_mean=float(rng.choice([-0.1, -1.5])))
+        if rng.random() < 0.5:
+            sae.b_dec = torch.randn(d, generator=g, device=DEV) * 0.2
+            sae.center_input = bool(rng.random() < 0.5)
+        groups[gi] = sae
+        k_max, d_sae_max = max(k_max, k), max(d_sae_max, S)
+        for _ in range(int(rng.integers(0, 3))):                # app slots on this weight set (maybe none)
+            n_edit = int(rng.integers(0, 7))
+            idx = rng.integers(0, S, size=n_edit).astype(np.int32)
+            if n_edit >= 2 and rng.random() < 0.5:
+                idx[-1] = idx[0]                                # a repeated feature: the later entry wins
+            mode = rng.integers(0, 2, size=n_edit).astype(np.uint8)
+            val = np.where(mode == W.EDIT_CLAMP, rng.uniform(-2, 6, size=n_edit), 0).astype(np.float32)
+            # replace mode on dense activations is legal but slow: keep it to sparse sets
+            add_error = bool(rng.random() < 0.6) or (act != W.SAE_TOPK and float(sae.b_enc.mean()) > -1.0)
+            apps[slot] = W.SaeApp(gi, idx, val, mode, add_error); slot += 1
+            r_max = max(r_max, n_edit)
+    n_slots = slot + int(rng.integers(0, 3))                    # some never-registered slots at the end
+    slots = np.array(sorted(apps), dtype=np.int32)
+    token_slot = np.full(T, -1, dtype=np.int32)
+    t = 0
+    while t < T:                                                # requests of random length
+        seg = int(min(T - t, rng.choice([1, 2, 9, 40, 200])))
+        token_slot[t:t + seg] = -1 if rng.random() < 0.25 else int(rng.choice(slots))
+        t += seg
+    T_live = T if rng.random() < 0.6 else int(rng.integers(0, T + 1))
+    if rng.random() < 0.4:                                      # gate a few apps on a given buffer
+        sc = torch.randn((T, 2), generator=g, device=DEV)
+        for s in rng.choice(slots, size=min(2, len(slots)), replace=False):
+            apps[int(s)].gate = W.Gate(sc, int(rng.integers(0, 2)), int(rng.integers(0, 2)), float(rng.normal()))
+    return W.Workload("fuzz%d" % seed, d, T, T_live, hidden, token_slot, apps, groups, n_slots_max=n_slots,
+                      n_groups_max=n_groups, C_max=C_max, k_max=k_max, r_max=r_max, d_sae_max=d_sae_max)
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_random_small_workload(seed):
+    import paper_2607_22595_b200 as mixlib
+    w = random_workload(1000 + seed)
+    flags = mixlib.MIX_FLAG_ENCODE_SIMT if seed % 4 == 3 else 0
+    out = run_gpu(w, flags=flags, graph=bool(seed % 2))
+    st = check_parity(W.host(w), out, expect_status=None, scale_with_output=True)
+    assert out["status"] & ~mixlib.MIX_STATUS_TOPK_GENERAL == 0       # no bad slots, groups or timeouts
+    assert st["rows"] == w.T_max

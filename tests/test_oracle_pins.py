@@ -76,6 +76,7 @@ def test_probe_closed_forms():
     h = rng.standard_normal(64)
     assert O.probe_scores(h, np.zeros((1, 64)), None, O.ACT_SIGMOID)[0] == 0.5
     assert np.allclose(O.probe_scores(h, np.zeros((7, 64)), np.zeros(7), O.ACT_SOFTMAX), 1 / 7, atol=1e-16)
+    assert O.probe_scores(h, rng.standard_normal((1, 64)), None, O.ACT_SOFTMAX).tolist() == [1.0]   # softmax of one class
     e = np.zeros((1, 64)); e[0, 5] = 1.0
     assert O.probe_scores(h, e, None, O.ACT_SIGMOID)[0] == pytest.approx(1 / (1 + math.exp(-h[5])), rel=1e-15)
     Wm = rng.standard_normal((5, 64)); b = rng.standard_normal(5)
