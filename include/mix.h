@@ -17,6 +17,9 @@
  *              per-feature edits (clamp: f_j = c; ablate: f_j = 0), decode from W_dec,
  *              optionally with the reconstruction error of the UNEDITED features added
  *              back:  h' = xhat(f') + (h - xhat(f)).
+ *   MIX_PROJECT directional ablation, the usual statement of "subtract a vector" for a refusal-style
+ *              direction (Section 3 "Write"; Table 1, row 1): h[t,:] <- bf16( h - beta (h . r) r ),
+ *              in place; r is used as given (pass a unit vector for an orthogonal projection).
  *   slot -1    no app: the row is neither read nor written (Section 4.2 "Toggling
  *              semantics": an inactive app costs a request nothing).
  *
@@ -57,7 +60,7 @@ typedef enum {
   MIX_ERR_CUDA = -5           /* a CUDA call failed; see mix_last_error() */
 } mix_status;
 
-enum { MIX_PROBE = 1, MIX_STEER = 2, MIX_SAE = 3 };                    /* app kinds */
+enum { MIX_PROBE = 1, MIX_STEER = 2, MIX_SAE = 3, MIX_PROJECT = 4 };   /* app kinds */
 enum { MIX_ACT_SIGMOID = 0, MIX_ACT_SOFTMAX = 1, MIX_ACT_NONE = 2 };   /* probe activations */
 enum { MIX_SAE_RELU = 0, MIX_SAE_JUMPRELU = 1, MIX_SAE_TOPK = 2 };     /* SAE activations */
 enum { MIX_EDIT_CLAMP = 0, MIX_EDIT_ABLATE = 1 };                      /* per-feature edits */
@@ -102,6 +105,13 @@ typedef struct {
   const void* v;
   float alpha;
 } mix_steer;
+
+/* Directional ablation.  r: device bf16 [d], used as given; beta = 1 removes the component along
+   r (for unit r), 0 < beta < 1 shrinks it, beta = 0 leaves the row untouched bit for bit. */
+typedef struct {
+  const void* r;
+  float beta;
+} mix_project;
 
 /* One SAE weight set, shared by any number of app slots.  All pointers device.
    W_enc bf16 [d_sae, d]: row j = encoder direction j.  b_enc fp32 [d_sae].
@@ -155,8 +165,8 @@ int mix_register_sae_weights(mix_ctx* ctx, int group, const mix_sae_weights* w, 
 int mix_unregister_sae_weights(mix_ctx* ctx, int group, void* stream);
 
 /* Attach an MI function to `slot` (paper, Section 4.2: functions are attached ahead of time
-   with their parameters).  `desc` points to a mix_probe, mix_steer or mix_sae_app according
-   to `kind`.  Stream-ordered; an entry becomes visible atomically (its valid flag is
+   with their parameters).  `desc` points to a mix_probe, mix_steer, mix_sae_app or mix_project
+   according to `kind`.  Stream-ordered; an entry becomes visible atomically (its valid flag is
    written last).  Errors: OUT_OF_RANGE (slot, n_classes > C_max, n_edit > r_max, edit
    index >= d_sae of the group, group), INVALID_ARG. */
 int mix_register_app(mix_ctx* ctx, int slot, int kind, const void* desc, void* stream);
@@ -165,7 +175,8 @@ int mix_register_app(mix_ctx* ctx, int slot, int kind, const void* desc, void* s
    MIX_STATUS_BAD_SLOT. */
 int mix_unregister_app(mix_ctx* ctx, int slot, void* stream);
 
-/* Cheap toggles that never touch launch structure (Section 4.2 "Toggling semantics"). */
+/* Cheap toggles that never touch launch structure (Section 4.2 "Toggling semantics").
+   mix_update_steer_alpha also sets beta of a MIX_PROJECT app. */
 int mix_update_steer_alpha(mix_ctx* ctx, int slot, float alpha, void* stream);
 int mix_update_sae_edits(mix_ctx* ctx, int slot, int n_edit, const int* idx, const float* val,
                          const unsigned char* mode, void* stream);

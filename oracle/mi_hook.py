@@ -2,8 +2,8 @@
 
 This module is the slow, plain definition of what one hook call computes on a
 ragged batch: every token row is dispatched by its slot id to a read primitive
-(linear probe -> score), a write primitive (additive steering vector) or an
-SAE function (encode, activation, per-feature edits, decode, optional
+(linear probe -> score), a write primitive (additive steering vector, or
+ablation of a direction) or an SAE function (encode, activation, per-feature edits, decode, optional
 reconstruction-error term); rows without an app are copied bit for bit.  It
 follows the paper's description of the three primitives (Section 3,
 "Read" / "Write" / "Conditional Write"), of the function contract (Section
@@ -32,7 +32,7 @@ from typing import Dict, Iterable, Optional
 import numpy as np
 
 # kinds / enums restated here on purpose (the oracle depends on nothing else)
-KIND_PROBE, KIND_STEER, KIND_SAE = 1, 2, 3
+KIND_PROBE, KIND_STEER, KIND_SAE, KIND_PROJECT = 1, 2, 3, 4
 ACT_SIGMOID, ACT_SOFTMAX, ACT_NONE = 0, 1, 2
 SAE_RELU, SAE_JUMPRELU, SAE_TOPK = 0, 1, 2
 EDIT_CLAMP, EDIT_ABLATE = 0, 1
@@ -97,6 +97,12 @@ def probe_scores(h: np.ndarray, W: np.ndarray, b: Optional[np.ndarray], act: int
 def steer(h: np.ndarray, v: np.ndarray, alpha: float) -> np.ndarray:
     """h' = h + alpha * v   (alpha is an fp32 parameter, used at its exact value)."""
     return h + float(np.float32(alpha)) * v
+
+
+def project(h: np.ndarray, r: np.ndarray, beta: float) -> np.ndarray:
+    """Directional ablation, the usual statement of "subtract a vector" along a direction
+    (Section 3, "Write"; Table 1, row 1):  h' = h - beta (h . r) r, with r used as given."""
+    return h - float(np.float32(beta)) * float(h @ r) * r
 
 
 # ---------------------------------------------------------------------------
@@ -266,6 +272,11 @@ def apply_hook(w, rows: Optional[Iterable[int]] = None, keep_z: bool = False,
             res.y[t] = h
         elif app.kind == KIND_STEER:
             y = steer(h, bf16_to_f64(app.v), app.alpha)
+            res.modified[t] = True
+            res.y[t] = y
+            res.out_bits[t] = f64_to_bf16_bits(y)
+        elif app.kind == KIND_PROJECT:
+            y = project(h, bf16_to_f64(app.r), app.beta)
             res.modified[t] = True
             res.y[t] = y
             res.out_bits[t] = f64_to_bf16_bits(y)

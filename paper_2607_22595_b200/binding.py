@@ -15,7 +15,7 @@ import torch
 
 from . import _build
 
-MIX_PROBE, MIX_STEER, MIX_SAE = 1, 2, 3
+MIX_PROBE, MIX_STEER, MIX_SAE, MIX_PROJECT = 1, 2, 3, 4
 MIX_ACT_SIGMOID, MIX_ACT_SOFTMAX, MIX_ACT_NONE = 0, 1, 2
 MIX_SAE_RELU, MIX_SAE_JUMPRELU, MIX_SAE_TOPK = 0, 1, 2
 MIX_EDIT_CLAMP, MIX_EDIT_ABLATE = 0, 1
@@ -169,6 +169,11 @@ class Mix:
         d = MixSteer(_ptr(v), float(alpha))
         self._check(self.lib.mix_register_app(self.ctx, slot, MIX_STEER, C.byref(d), _stream(stream)))
         self._keep[("a", slot)] = (v,)
+
+    def register_project(self, slot, r, beta, stream=None):
+        d = MixSteer(_ptr(r), float(beta))          # mix_project has the layout of mix_steer: (pointer, float)
+        self._check(self.lib.mix_register_app(self.ctx, slot, MIX_PROJECT, C.byref(d), _stream(stream)))
+        self._keep[("a", slot)] = (r,)
 
     @staticmethod
     def _edit_arrays(idx, val, mode):

@@ -293,6 +293,11 @@ int mix_register_app(mix_ctx* c, int slot, int kind, const void* desc, void* str
     if (!p->v || !aligned16(p->v)) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "steering vector is NULL or not 16-byte aligned");
     e.W = p->v;
     e.alpha = p->alpha;
+  } else if (kind == MIX_PROJECT) {
+    const mix_project* p = static_cast<const mix_project*>(desc);
+    if (!p->r || !aligned16(p->r)) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "projection vector is NULL or not 16-byte aligned");
+    e.W = p->r;
+    e.alpha = p->beta;
   } else if (kind == MIX_SAE) {
     const mix_sae_app* p = static_cast<const mix_sae_app*>(desc);
     if (p->group < 0 || p->group >= c->cfg.n_groups_max || !c->h_groups[p->group].valid)
@@ -357,7 +362,9 @@ int mix_update_steer_alpha(mix_ctx* c, int slot, float alpha, void* stream) {
   if (!c) return MIX_ERR_INVALID_ARG;
   int rc = check_slot(c, slot);
   if (rc != MIX_OK) return rc;
-  if (!c->h_apps[slot].valid || (c->h_apps[slot].kind & kKindMask) != MIX_STEER) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "slot %d is not a steering app", slot);
+  const int kind_ = c->h_apps[slot].kind & kKindMask;
+  if (!c->h_apps[slot].valid || (kind_ != MIX_STEER && kind_ != MIX_PROJECT))
+    MIX_FAIL(c, MIX_ERR_INVALID_ARG, "slot %d is not a steering or projection app", slot);
   c->h_apps[slot].alpha = alpha;
   MIX_CUDA(c, cudaMemcpyAsync(&c->d_apps[slot].alpha, &alpha, sizeof(float), cudaMemcpyHostToDevice,
                               static_cast<cudaStream_t>(stream)));

@@ -203,8 +203,15 @@ __device__ __forceinline__ void warp_row(const RowApp& a, __nv_bfloat16* __restr
     if (a.alpha != 0.f) steer_row(hrow, a.W, a.alpha, nvec, lane, 32);   // alpha = 0: row stays bit-exact
     return;
   }
-  if (a.kind != MIX_PROBE || scores == nullptr) return;
   const uint4* h1[1] = {hrow};
+  if (a.kind == MIX_PROJECT) {                 // h - beta (h . r) r: one pass for the dot, one for the update
+    if (a.alpha == 0.f) return;
+    float z[1][1];
+    probe_dots<1, 1>(h1, a.W, nvec, 1, lane, 32, z);
+    steer_row(hrow, a.W, -a.alpha * z[0][0], nvec, lane, 32);
+    return;
+  }
+  if (a.kind != MIX_PROBE || scores == nullptr) return;
   float* out = scores + (size_t)t * C_max;
   if (a.C == 1) {
     float z[1][1];
@@ -443,6 +450,43 @@ probe_steer_team_kernel(const int* __restrict__ token_slot, const int* __restric
         unpack8(vq[u], y);
 #pragma unroll
         for (int e = 0; e < 8; ++e) x[e] = fmaf(a.alpha, y[e], x[e]);
+        __stcs(hrow + v, pack8(x));
+      }
+    }
+    return;
+  }
+  if (a.kind == MIX_PROJECT) {                 // h - beta (h . r) r
+    if (a.alpha == 0.f) return;
+    uint4 rq[kTeamVec];
+    float dot = 0.f;
+#pragma unroll
+    for (int u = 0; u < kTeamVec; ++u) {
+      const int v = threadIdx.x + u * NT;
+      if (v < nvec) {
+        rq[u] = __ldg(a.W + v);
+        float x[8], y[8];
+        unpack8(hq[u], x);
+        unpack8(rq[u], y);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) dot = fmaf(x[e], y[e], dot);
+      }
+    }
+    dot = warp_sum(dot);
+    if (lane == 0) s_part[warp][0] = dot;
+    __syncthreads();
+    float total = 0.f;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) total += s_part[w][0];
+    const float coef = -a.alpha * total;
+#pragma unroll
+    for (int u = 0; u < kTeamVec; ++u) {
+      const int v = threadIdx.x + u * NT;
+      if (v < nvec) {
+        float x[8], y[8];
+        unpack8(hq[u], x);
+        unpack8(rq[u], y);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) x[e] = fmaf(coef, y[e], x[e]);
         __stcs(hrow + v, pack8(x));
       }
     }

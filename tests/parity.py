@@ -112,7 +112,7 @@ def check_parity(wh, out, rows=None, expect_status=0, check_features=True, scale
                 stats["topk_swaps"] += 1
                 redo[t] = K_gpu
     if scale_with_output:
-        hmax = max([hmax] + [float(np.abs(ref.y[t]).max()) for t in rows if ref.kind[t] in (O.KIND_STEER, O.KIND_SAE)])
+        hmax = max([hmax] + [float(np.abs(ref.y[t]).max()) for t in rows if ref.kind[t] in (O.KIND_STEER, O.KIND_SAE, O.KIND_PROJECT)])
     if redo:       # re-evaluate those rows with the GPU's (valid) choice among near-ties
         ref2 = O.apply_hook(wh, list(redo), topk_override=redo)
         for t in redo:
@@ -120,7 +120,7 @@ def check_parity(wh, out, rows=None, expect_status=0, check_features=True, scale
             ref.n_active[t] = ref2.n_active[t]
     for t in rows:
         kind = ref.kind[t]
-        if kind in (O.KIND_STEER, O.KIND_SAE):
+        if kind in (O.KIND_STEER, O.KIND_SAE, O.KIND_PROJECT):
             g = O.bf16_to_f64(hid[t])
             err = np.abs(g - ref.y[t])
             assert err.max() <= HIDDEN_TOL_FRAC * hmax, "row %d (kind %d) hidden off by %g (bound %g)" % (

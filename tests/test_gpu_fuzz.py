@@ -34,6 +34,9 @@ def random_workload(seed):
     for _ in range(int(rng.integers(1, 4))):                    # steering vectors
         v = torch.randn(d, generator=g, device=DEV).to(torch.bfloat16)
         apps[slot] = W.Steer(v, float(np.float32(rng.uniform(-6, 6)))); slot += 1
+    for _ in range(int(rng.integers(0, 3))):                    # directions to ablate
+        r = torch.randn(d, generator=g, device=DEV); r = (r / r.norm()).to(torch.bfloat16)
+        apps[slot] = W.Project(r, float(np.float32(rng.choice([1.0, 0.5, 0.0, -1.0])))); slot += 1
     k_max = r_max = 1
     d_sae_max = 0
     for gi in range(n_groups):

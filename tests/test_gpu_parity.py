@@ -154,6 +154,26 @@ def test_alpha_zero_and_opposite_alphas():
     assert (np.abs(a - b) <= bf16_ulp(np.maximum(np.abs(b), np.abs(O.bf16_to_f64(out["hidden"]))))).all()
 
 
+def test_project_rows_small_and_large_batch_kernels():
+    for T in (96, 2304):                              # team kernel / warp-per-row kernel
+        w = W.make_decode(DEV, d=1024, T=T, n_probe=2, n_steer=2)
+        g = torch.Generator(device=DEV); g.manual_seed(77)
+        for s, a in list(w.apps.items()):
+            if a.kind == W.KIND_STEER:
+                r = torch.randn(1024, generator=g, device=DEV); r = (r / r.norm()).to(torch.bfloat16)
+                w.apps[s] = W.Project(r, 1.0 if s % 2 else 0.5)
+        out = run_gpu(w, graph=True)
+        st = check_parity(W.host(w), out, check_features=False)
+        # with beta = 1 nothing (beyond rounding) is left along r
+        wh = W.host(w)
+        for t in range(T):
+            a = wh.apps.get(int(wh.token_slot[t]))
+            if a is not None and a.kind == W.KIND_PROJECT and a.beta == 1.0:
+                y = O.bf16_to_f64(out["hidden"][t]); r = O.bf16_to_f64(a.r)
+                assert abs(y @ r) <= 2e-2 * np.abs(O.bf16_to_f64(wh.hidden[t])).max()
+        assert st["max_hidden_ulp"] <= 1.0 + 1e-6 or st["max_hidden_err"] < 1e-2
+
+
 def _one_sae_workload(d, S, act, k, T, add_error, edits, b_dec=False, center=False, seed=5, W_enc=None,
                       b_enc=None, b_enc_mean=-0.1):
     g = torch.Generator(device=DEV); g.manual_seed(seed)

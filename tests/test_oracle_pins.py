@@ -361,3 +361,29 @@ def test_gated_hook_limits_and_complement():
         assert (ge.kind[t] != 0) + (lt.kind[t] != 0) == (base.kind[t] != 0)
         src = ge if sc[t, 1] >= np.float32(0.1) else lt
         assert np.array_equal(src.out_bits[t], base.out_bits[t])
+
+
+# ------------------------------------------------------------------ directional ablation
+def test_project_hand_worked_and_invariants():
+    g = GOLD["project"]; h = np.array(GOLD["h"]); r = np.array(g["r"])
+    assert float(h @ r) == g["dot"]
+    assert O.project(h, r, g["beta"]).tolist() == g["out"]
+    assert O.project(h, r, 0.5).tolist() == g["beta_half_out"]
+    rng = np.random.default_rng(21)
+    h = rng.standard_normal(48); r = rng.standard_normal(48); r /= np.linalg.norm(r)
+    y = O.project(h, r, 1.0)
+    assert abs(y @ r) < 1e-14                                      # nothing left along r
+    assert np.allclose(O.project(y, r, 1.0), y, rtol=0, atol=1e-14)   # idempotent
+    assert np.array_equal(O.project(h, r, 0.0), h)
+    assert np.allclose(h - y, (h @ r) * r, rtol=0, atol=1e-15)     # what was removed is parallel to r
+    e = np.zeros(48); e[9] = 1.0
+    out = O.project(h, e, 0.25)
+    assert out[9] == h[9] * 0.75 and np.array_equal(np.delete(out, 9), np.delete(h, 9))
+    # through the hook
+    w = W.host(W.make_tiny(d=64, T=48, d_sae=256, k=8, seed=15))
+    rv = bf(rng.standard_normal(64) / 8.0)
+    w.apps[1] = W.Project(rv, 1.0)
+    res = O.apply_hook(w)
+    for t in np.nonzero(w.token_slot == 1)[0]:
+        hh = O.bf16_to_f64(w.hidden[t]); rr = O.bf16_to_f64(rv)
+        assert np.array_equal(res.y[int(t)], hh - (hh @ rr) * rr) and res.kind[int(t)] == O.KIND_PROJECT

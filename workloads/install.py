@@ -1,7 +1,7 @@
 """Register a workload's apps with a hook context (any object with the binding's method names)."""
 from __future__ import annotations
 
-from .spec import KIND_PROBE, KIND_SAE, KIND_STEER, Workload
+from .spec import KIND_PROBE, KIND_PROJECT, KIND_SAE, KIND_STEER, Workload
 
 
 def make_context(mix_cls, w: Workload, flags: int = 0, **over):
@@ -23,6 +23,8 @@ def install(m, w: Workload):
             m.register_probe(s, a.W, a.b, a.act)
         elif a.kind == KIND_STEER:
             m.register_steer(s, a.v, a.alpha)
+        elif a.kind == KIND_PROJECT:
+            m.register_project(s, a.r, a.beta)
         elif a.kind == KIND_SAE:
             m.register_sae_app(s, a.group, a.edit_idx, a.edit_val, a.edit_mode, a.add_error)
         if getattr(a, "gate", None) is not None:

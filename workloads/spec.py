@@ -19,7 +19,7 @@ import numpy as np
 import torch
 
 # app kinds
-KIND_PROBE, KIND_STEER, KIND_SAE = 1, 2, 3
+KIND_PROBE, KIND_STEER, KIND_SAE, KIND_PROJECT = 1, 2, 3, 4
 # probe activations
 ACT_SIGMOID, ACT_SOFTMAX, ACT_NONE = 0, 1, 2
 # SAE activations
@@ -58,6 +58,14 @@ class Steer:
     v: object                 # bf16 [d]
     alpha: float
     kind: int = KIND_STEER
+    gate: Optional[Gate] = None
+
+
+@dataclass
+class Project:
+    r: object                 # bf16 [d], used as given
+    beta: float
+    kind: int = KIND_PROJECT
     gate: Optional[Gate] = None
 
 
@@ -131,6 +139,8 @@ def host(w: Workload, only_groups=None) -> Workload:
             apps[s] = Probe(bits(a.W), bits(a.b), a.act, gate=g)
         elif a.kind == KIND_STEER:
             apps[s] = Steer(bits(a.v), float(a.alpha), gate=g)
+        elif a.kind == KIND_PROJECT:
+            apps[s] = Project(bits(a.r), float(a.beta), gate=g)
         else:
             apps[s] = SaeApp(a.group, a.edit_idx, a.edit_val, a.edit_mode, a.add_error, gate=g)
     groups = {
