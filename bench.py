@@ -331,6 +331,42 @@ def run_workload(args):
     print(json.dumps(out), flush=True)
 
 
+def extras_decode_variants(w, hiddens, scores, mixlib):
+    """The decode config with its apps gated / turned into projections: L2-cold µs per step."""
+    T = w.T_max
+    R = len(hiddens)
+    out = {}
+    g = torch.Generator(device="cuda"); g.manual_seed(7)
+    gate_scores = torch.randn((T, 1), generator=g, device="cuda")          # about half of the gates open
+
+    def measure(m):
+        stream = torch.cuda.Stream(); stream.wait_stream(torch.cuda.current_stream())
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            m.apply(hiddens[0], scores[0], stream=stream)
+            gr = capture_steps(m, hiddens, scores, range(R), stream)
+            gr.replay()
+            e0.record(stream)
+            for _ in range(8):
+                gr.replay()
+            e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / (8 * R)
+
+    m = W.make_context(mixlib.Mix, w)
+    for s in w.apps:
+        m.set_gate(s, gate_scores, 0, mixlib.MIX_GATE_GE, 0.0)
+    out["all_apps_gated_us_per_step"] = measure(m)
+    m.destroy()
+    m = W.make_context(mixlib.Mix, w)
+    for s, a in w.apps.items():
+        if a.kind == W.KIND_STEER:
+            m.register_project(s, a.v, 1.0)
+    out["steer_as_projection_us_per_step"] = measure(m)
+    m.destroy()
+    return out
+
+
 def extras_sweep(peaks, mixlib):
     """Bandwidth kernels alone at a size that cannot hide in L2: d = 8192, T = 65536, every row hooked."""
     d, T = 8192, 65536
@@ -494,6 +530,7 @@ def run_mix(args, rank, world, local_rank):
         if not args.no_extras:
             ex = {}
             try:
+                ex["decode_variants"] = extras_decode_variants(w, hiddens, scores, mixlib)
                 ex["sweep"] = extras_sweep(peaks, mixlib)
                 ex["sae_heavy"] = extras_sae("sae_heavy (config 2)", W.make_sae_heavy("cuda"), peaks, mixlib)
                 torch.cuda.empty_cache()
