@@ -69,6 +69,9 @@ void free_all(mix_ctx* c) {
   if (c->owned_b_eff)
     for (int g = 0; g < c->cfg.n_groups_max; ++g) cudaFree(c->owned_b_eff[g]);
   free(c->owned_b_eff); free(c->h_apps); free(c->h_groups);
+  if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+  if (c->ev_join) cudaEventDestroy(c->ev_join);
+  if (c->side_stream) cudaStreamDestroy(c->side_stream);
 }
 
 int check_slot(mix_ctx* c, int slot) {
@@ -188,6 +191,11 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
         e = cudaErrorUnknown;
       if (e == cudaSuccess) e = encode_tc_prepare();
     }
+  }
+  if (e == cudaSuccess && G > 0) {
+    e = cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming);
   }
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) { free_all(c); free(c); return MIX_ERR_CUDA; }
@@ -436,13 +444,25 @@ int mix_apply(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream) 
   auto tap = [&]() -> cudaError_t {
     return c->stage_events_on ? cudaEventRecord(c->stage_events[stage++], s) : cudaSuccess;
   };
+  // Probes and steering touch rows the SAE path never touches, so when both are present they
+  // run side by side: the probe/steer kernels on the context's side stream (forked from and
+  // joined back into the caller's stream with events, which stream capture turns into graph
+  // edges), the SAE chain on the caller's stream.  With the timing taps on, everything runs in
+  // order on the caller's stream so that the per-stage times mean something.
+  const bool fork = c->cfg.n_groups_max > 0 && !c->stage_events_on;
+  cudaStream_t ps = fork ? c->side_stream : s;
+  if (fork) {
+    MIX_CUDA(c, cudaEventRecord(c->ev_fork, s));
+    MIX_CUDA(c, cudaStreamWaitEvent(ps, c->ev_fork, 0));
+  }
   MIX_CUDA(c, tap());
-  MIX_CUDA(c, launch_probe_steer(c, h, T, scores_out, s));
+  MIX_CUDA(c, launch_probe_steer(c, h, T, scores_out, ps));
   MIX_CUDA(c, tap());
   if (has_multiclass_stage(c)) {
-    MIX_CUDA(c, launch_probe_multiclass(c, h, T, scores_out, s));
+    MIX_CUDA(c, launch_probe_multiclass(c, h, T, scores_out, ps));
     MIX_CUDA(c, tap());
   }
+  if (fork) MIX_CUDA(c, cudaEventRecord(c->ev_join, ps));
   if (c->cfg.n_groups_max > 0) {
     MIX_CUDA(c, launch_route(c, T, s));
     MIX_CUDA(c, tap());
@@ -466,6 +486,7 @@ int mix_apply(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream) 
     MIX_CUDA(c, launch_decode(c, h, s));
     MIX_CUDA(c, tap());
   }
+  if (fork) MIX_CUDA(c, cudaStreamWaitEvent(s, c->ev_join, 0));
   return MIX_OK;
 }
 

@@ -119,6 +119,10 @@ struct Ctx {
   CUtensorMap* d_tmap_w;    // [n_groups_max] W_enc maps (box kTileK x kTileN, 128B swizzle)
   CUtensorMap tmap_panel;   // panel map (box kTileK x kTileM, 128B swizzle)
 
+  // probe/steer kernels run beside the SAE chain on this stream (created with the context)
+  cudaStream_t side_stream;
+  cudaEvent_t ev_fork, ev_join;
+
   // profiling taps
   int stage_events_on;
   cudaEvent_t stage_events[12];
