@@ -33,6 +33,8 @@ METRIC = "mi_hook_token_rows_per_s"
 UNIT = "token-rows/s"
 WORKLOAD = "decode: d=4096, T=256 (256 requests x 1 token), 64 probes + 32 steering vectors, 25% unhooked"
 ROTATE_BYTES = 512 << 20
+SAE_FLAGS = 2            # mix_config.flags of the SAE contexts of the extras / --workload runs: MIX_FLAG_RETILE_W_ENC
+                         # (tile-contiguous copy of W_enc made at registration); --no-retile streams W_enc as given
 # dram__bytes_read.sum + dram__bytes_write.sum of one probe_steer_team_kernel launch on this workload,
 # from the ncu capture summarised in profiles/probe_steer_kernel_decode.md (reads 2.40 MB, writes 0:
 # the steered rows are still dirty in L2 when the kernel ends).
@@ -210,7 +212,7 @@ def time_stages(m, fn, reps=5):
 
 def extras_sae(name, w, peaks, mixlib):
     """SAE-carrying config: per-kernel times, encode flop rate and weight-stream bandwidth."""
-    m = W.make_context(mixlib.Mix, w)
+    m = W.make_context(mixlib.Mix, w, flags=SAE_FLAGS)
     h = w.hidden.clone()
     scores = torch.zeros((w.T_max, max(w.C_max, 1)), dtype=torch.float32, device="cuda")
     def fn():
@@ -244,7 +246,8 @@ def extras_sae(name, w, peaks, mixlib):
     enc_s = st["encode"] * 1e-3
     status = m.get_status()
     m.destroy()
-    return {"workload": name, "t_call_ms_graph": min(times), "stage_ms": st, "sae_rows_per_group": counts,
+    return {"workload": name, "w_enc_layout": "tile-contiguous copy" if SAE_FLAGS & 2 else "as registered",
+            "t_call_ms_graph": min(times), "stage_ms": st, "sae_rows_per_group": counts,
             "encode_tflops": flops / enc_s / 1e12, "encode_frac_bf16_peak": flops / enc_s / 1e12 / peaks["bf16_tflops"],
             "encode_weight_stream_gbs": wbytes / enc_s / 1e9,
             "encode_frac_hbm_peak": wbytes / enc_s / 1e9 / peaks["hbm_gbs"],
@@ -254,7 +257,7 @@ def extras_sae(name, w, peaks, mixlib):
 def run_replay(peaks, mixlib, n_replays):
     """Config 4: one captured graph at T_max = 2048, a fresh slot map and live count per replay."""
     w = W.make_replay("cuda")
-    m = W.make_context(mixlib.Mix, w)
+    m = W.make_context(mixlib.Mix, w, flags=SAE_FLAGS)
     T = w.T_max
     h = w.hidden.clone()
     scores = torch.zeros((T, 1), dtype=torch.float32, device="cuda")
@@ -548,10 +551,15 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="mix", choices=["mix", "reference"])
     ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--no-retile", action="store_true",
+                    help="SAE contexts stream W_enc as registered instead of a tile-contiguous copy (MIX_FLAG_RETILE_W_ENC)")
     ap.add_argument("--workload", default="decode",
                     help="decode (the contract line) | sweep | sae_heavy | sae_small | mixed | mixed_small | replay")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     args = ap.parse_args()
+    if args.no_retile:
+        global SAE_FLAGS
+        SAE_FLAGS = 0
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

@@ -76,7 +76,12 @@ enum {
 
 /* flags for mix_config.flags */
 enum {
-  MIX_FLAG_ENCODE_SIMT = 1u << 0      /* run the SAE encode on the plain CUDA-core kernel instead of tcgen05 (cross-check) */
+  MIX_FLAG_ENCODE_SIMT = 1u << 0,     /* run the SAE encode on the plain CUDA-core kernel instead of tcgen05 (cross-check) */
+  MIX_FLAG_RETILE_W_ENC = 1u << 1     /* keep a library-owned copy of every registered W_enc, re-laid out so that each
+                                         256-feature x 64-column encode tile is one contiguous 32 KiB block: the encode then
+                                         streams whole DRAM pages instead of 128-byte pieces of 256 different rows.  Costs
+                                         2 * d_sae * d bytes per weight set, allocated at registration (W_enc itself is no
+                                         longer read by mix_apply and need not stay alive) */
 };
 
 typedef struct {

@@ -68,6 +68,9 @@ void free_all(mix_ctx* c) {
   cudaFree(c->d_cand_ninth); cudaFree(c->d_row_flag); cudaFree(c->d_mtile_flag); cudaFree(c->d_n_flagged);
   if (c->owned_b_eff)
     for (int g = 0; g < c->cfg.n_groups_max; ++g) cudaFree(c->owned_b_eff[g]);
+  if (c->owned_w_tiled)
+    for (int g = 0; g < c->cfg.n_groups_max; ++g) cudaFree(c->owned_w_tiled[g]);
+  free(c->owned_w_tiled);
   free(c->owned_b_eff); free(c->h_apps); free(c->h_groups);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->ev_join) cudaEventDestroy(c->ev_join);
@@ -137,7 +140,8 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
   c->h_apps = static_cast<AppEntry*>(calloc(NS, sizeof(AppEntry)));
   c->h_groups = static_cast<GroupEntry*>(calloc(G > 0 ? G : 1, sizeof(GroupEntry)));
   c->owned_b_eff = static_cast<float**>(calloc(G > 0 ? G : 1, sizeof(float*)));
-  if (!c->h_apps || !c->h_groups || !c->owned_b_eff) { free_all(c); free(c); return MIX_ERR_NO_MEMORY; }
+  c->owned_w_tiled = static_cast<__nv_bfloat16**>(calloc(G > 0 ? G : 1, sizeof(__nv_bfloat16*)));
+  if (!c->h_apps || !c->h_groups || !c->owned_b_eff || !c->owned_w_tiled) { free_all(c); free(c); return MIX_ERR_NO_MEMORY; }
   bool ok = true;
   ok = ok && dev_alloc(&c->d_token_slot, T) == cudaSuccess;
   ok = ok && dev_alloc(&c->d_n_live, 1) == cudaSuccess;
@@ -253,8 +257,20 @@ int mix_register_sae_weights(mix_ctx* c, int group, const mix_sae_weights* w, vo
   }
   if (!(c->cfg.flags & MIX_FLAG_ENCODE_SIMT)) {
     CUtensorMap tm;
-    if (make_tmap(&tm, w->W_enc, (unsigned long long)w->d_sae, c->cfg.d_model, kTileN) != MIX_OK)
+    if (c->cfg.flags & MIX_FLAG_RETILE_W_ENC) {
+      // library-owned tile-contiguous copy: [S/256][d/64][256][64], seen by TMA as a 64-column matrix
+      if (c->owned_w_tiled[group]) { cudaStreamSynchronize(s); cudaFree(c->owned_w_tiled[group]); c->owned_w_tiled[group] = nullptr; }
+      const size_t n_el = (size_t)w->d_sae * c->cfg.d_model;
+      if (cudaMalloc(reinterpret_cast<void**>(&c->owned_w_tiled[group]), n_el * sizeof(__nv_bfloat16)) != cudaSuccess) {
+        cudaGetLastError();
+        MIX_FAIL(c, MIX_ERR_NO_MEMORY, "cannot allocate the re-tiled copy of W_enc");
+      }
+      MIX_CUDA(c, launch_retile(ge.W_enc, c->owned_w_tiled[group], w->d_sae, c->cfg.d_model, s));
+      if (make_tmap(&tm, c->owned_w_tiled[group], (unsigned long long)(n_el / kTileK), kTileK, kTileN) != MIX_OK)
+        MIX_FAIL(c, MIX_ERR_CUDA, "cuTensorMapEncodeTiled failed for the re-tiled W_enc");
+    } else if (make_tmap(&tm, w->W_enc, (unsigned long long)w->d_sae, c->cfg.d_model, kTileN) != MIX_OK) {
       MIX_FAIL(c, MIX_ERR_CUDA, "cuTensorMapEncodeTiled failed for W_enc");
+    }
     MIX_CUDA(c, cudaMemcpyAsync(c->d_tmap_w + group, &tm, sizeof(tm), cudaMemcpyHostToDevice, s));
   }
   c->h_groups[group] = ge;

@@ -98,6 +98,7 @@ struct Ctx {
   AppEntry* h_apps;
   GroupEntry* h_groups;
   float** owned_b_eff;      // per group: library-owned folded bias or null
+  __nv_bfloat16** owned_w_tiled;   // per group: library-owned tile-contiguous copy of W_enc or null
 
   // SAE workspace
   int panel_rows_cap;       // P
@@ -147,6 +148,7 @@ cudaError_t launch_decode(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s);
 cudaError_t launch_compose_map(const Ctx* c, int T_live, int n_req, cudaStream_t s);
 cudaError_t launch_fold_bias(const __nv_bfloat16* W_enc, const float* b_enc, const float* b_dec, float* b_eff,
                              long long d_sae, int d, cudaStream_t s);
+cudaError_t launch_retile(const __nv_bfloat16* W_enc, __nv_bfloat16* W_tiled, long long d_sae, int d, cudaStream_t s);
 cudaError_t encode_tc_prepare();   // opt in to the large dynamic shared memory size
 
 }  // namespace mix

@@ -181,7 +181,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
                  const RouteState* __restrict__ rs_g, const GroupEntry* __restrict__ groups, int n_groups,
                  float* __restrict__ Z, long long ldz, int d, unsigned* __restrict__ status, int mode,
                  const int* __restrict__ mtile_flag, const int* __restrict__ n_flagged, float* __restrict__ cand_val,
-                 int* __restrict__ cand_idx, float* __restrict__ cand_ninth, int cand_tiles) {
+                 int* __restrict__ cand_idx, float* __restrict__ cand_ninth, int cand_tiles, int w_tiled) {
   if (mode == 1 && *n_flagged == 0) return;
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment: required by the 128-byte swizzle atoms
@@ -235,7 +235,12 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
           mbar_expect_tx(bar, kStageBytes);
           const unsigned sa = smem_u32(tiles + stage * kStageBytes);
           tma_load_2d(sa, &tmap_panel, kb * kTileK, t.m_tile_global * kTileM, bar);
-          tma_load_2d(sa + kABytes, tw, kb * kTileK, t.n_tile * kTileN, bar);
+          // W_enc tile: rows n_tile*256.. of the row-major matrix, or -- when the weights were re-laid
+          // out at registration -- block (n_tile, kb) of the tile-contiguous copy [S/256][d/64][256][64]
+          if (w_tiled)
+            tma_load_2d(sa + kABytes, tw, 0, (t.n_tile * num_kb + kb) * kTileN, bar);
+          else
+            tma_load_2d(sa + kABytes, tw, kb * kTileK, t.n_tile * kTileN, bar);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -354,7 +359,29 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
   }
 }
 
+// Registration-time copy of W_enc [S, d] into [S/256][d/64][256][64]: one thread per 16 bytes.
+__global__ void retile_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, long long d_sae, int d) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;      // index of a 16-byte piece of dst
+  const int num_kb = d / kTileK;
+  const long long total = d_sae * (long long)d / 8;
+  if (i >= total) return;
+  const int piece = (int)(i & 7);                       // 8 pieces per 64-column row
+  const long long row_in_all = i >> 3;                  // row of the [.., 256, 64] blocks
+  const int r = (int)(row_in_all % kTileN);
+  const long long blk = row_in_all / kTileN;
+  const int kb = (int)(blk % num_kb);
+  const long long n_tile = blk / num_kb;
+  dst[i] = src[((n_tile * kTileN + r) * (long long)d + (long long)kb * kTileK) / 8 + piece];
+}
+
 }  // namespace
+
+cudaError_t launch_retile(const __nv_bfloat16* W_enc, __nv_bfloat16* W_tiled, long long d_sae, int d, cudaStream_t s) {
+  const long long total = d_sae * (long long)d / 8;
+  retile_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(reinterpret_cast<const uint4*>(W_enc),
+                                                                reinterpret_cast<uint4*>(W_tiled), d_sae, d);
+  return cudaGetLastError();
+}
 
 cudaError_t encode_tc_prepare() {
   return cudaFuncSetAttribute(encode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
@@ -365,7 +392,8 @@ cudaError_t launch_encode_tc(const Ctx* c, int mode, cudaStream_t s) {
                                                              c->cfg.n_groups_max, c->d_z, c->cfg.d_sae_max,
                                                              c->cfg.d_model, c->d_status, mode, c->d_mtile_flag,
                                                              c->d_n_flagged, c->d_cand_val, c->d_cand_idx,
-                                                             c->d_cand_ninth, c->cand_tiles);
+                                                             c->d_cand_ninth, c->cand_tiles,
+                                                             (c->cfg.flags & MIX_FLAG_RETILE_W_ENC) ? 1 : 0);
   return cudaGetLastError();
 }
 

@@ -51,6 +51,16 @@ def test_sae_heavy_small(simt):
     check_parity(W.host(w), out)
 
 
+def test_retiled_w_enc_matches_oracle():
+    # the tile-contiguous copy of W_enc (several feature tiles, several k-blocks, two row tiles)
+    mixlib = _mixlib()
+    w = W.make_sae_heavy(DEV, d=320, d_sae=1280, k=16, T=400, R=8, G=2, n_edit=8, edit_hint=oracle_edit_hint)
+    out = run_gpu(w, flags=mixlib.MIX_FLAG_RETILE_W_ENC, graph=True)
+    check_parity(W.host(w), out)
+    w = W.make_mixed(DEV, d=320, T=1500, R=40, d_sae=1024, cap=200, mu=3.5, edit_hint=oracle_edit_hint)
+    check_parity(W.host(w), run_gpu(w, flags=mixlib.MIX_FLAG_RETILE_W_ENC))
+
+
 def test_mixed_small():
     w = W.make_mixed(DEV, d=320, T=1500, R=40, d_sae=1024, cap=200, mu=3.5, edit_hint=oracle_edit_hint)
     out = run_gpu(w, graph=True)
