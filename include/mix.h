@@ -39,7 +39,10 @@
  *     ordinary host memory.  bf16 tensors are row-major, densely packed.
  *   - weights are BORROWED: the caller keeps them alive and unchanged until the app /
  *     weight set is unregistered (or the context destroyed) and work already enqueued has
- *     finished.  Everything else (tables, edit lists, slot map) is copied.
+ *     finished.  (The library may also keep its own copy of small weights -- contexts with
+ *     T_max <= 2048 copy steering / projection vectors and one-class probe weights at
+ *     registration -- so changing borrowed weights in place needs a new registration.)
+ *     Everything else (tables, edit lists, slot map) is copied.
  *   - one host thread per context at a time.
  */
 #ifndef MIX_H_

@@ -60,7 +60,7 @@ cudaError_t dev_alloc(T** p, size_t n) {
 }
 
 void free_all(mix_ctx* c) {
-  cudaFree(c->d_token_slot); cudaFree(c->d_n_live); cudaFree(c->d_apps); cudaFree(c->d_groups); cudaFree(c->d_gates);
+  cudaFree(c->d_token_slot); cudaFree(c->d_n_live); cudaFree(c->d_apps); cudaFree(c->d_groups); cudaFree(c->d_gates); cudaFree(c->d_vec_arena);
   cudaFree(c->d_edit_idx); cudaFree(c->d_edit_val); cudaFree(c->d_edit_mode); cudaFree(c->d_status);
   cudaFree(c->d_tmp_req); cudaFree(c->d_tmp_req_slot); cudaFree(c->d_panel); cudaFree(c->d_panel_row);
   cudaFree(c->d_mtile_group); cudaFree(c->d_row_group); cudaFree(c->d_route); cudaFree(c->d_z); cudaFree(c->d_topk_idx);
@@ -148,6 +148,7 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
   ok = ok && dev_alloc(&c->d_apps, NS) == cudaSuccess;
   ok = ok && dev_alloc(&c->d_groups, G > 0 ? G : 1) == cudaSuccess;
   ok = ok && dev_alloc(&c->d_gates, NS) == cudaSuccess;
+  if (T <= kTeamMaxRows) ok = ok && dev_alloc(&c->d_vec_arena, (size_t)NS * cfg->d_model) == cudaSuccess;
   ok = ok && dev_alloc(&c->d_edit_idx, (size_t)NS * c->cfg.r_max) == cudaSuccess;
   ok = ok && dev_alloc(&c->d_edit_val, (size_t)NS * c->cfg.r_max) == cudaSuccess;
   ok = ok && dev_alloc(&c->d_edit_mode, (size_t)NS * c->cfg.r_max) == cudaSuccess;
@@ -183,6 +184,7 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
   if (e == cudaSuccess) e = cudaMemset(c->d_apps, 0, NS * sizeof(AppEntry));
   if (e == cudaSuccess) e = cudaMemset(c->d_groups, 0, (G > 0 ? G : 1) * sizeof(GroupEntry));
   if (e == cudaSuccess) e = cudaMemset(c->d_gates, 0, NS * sizeof(GateEntry));
+  if (e == cudaSuccess && c->d_vec_arena) e = cudaMemset(c->d_vec_arena, 0, (size_t)NS * cfg->d_model * sizeof(__nv_bfloat16));
   if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, sizeof(unsigned));
   if (e == cudaSuccess && G > 0) {
     e = cudaMemset(c->d_panel, 0, (size_t)c->panel_rows_cap * cfg->d_model * sizeof(__nv_bfloat16));
@@ -333,6 +335,13 @@ int mix_register_app(mix_ctx* c, int slot, int kind, const void* desc, void* str
     e.add_error = p->add_error ? 1 : 0;
   } else {
     MIX_FAIL(c, MIX_ERR_INVALID_ARG, "bad app kind %d", kind);
+  }
+  // Single-vector weights are copied into the context's vector arena (row = slot), so that the
+  // one-CTA-per-row kernel can request them from the slot id alone, before it has the entry.
+  if (c->d_vec_arena && (kind == MIX_STEER || kind == MIX_PROJECT || (kind == MIX_PROBE && e.n_classes == 1))) {
+    __nv_bfloat16* dst = c->d_vec_arena + (size_t)slot * c->cfg.d_model;
+    MIX_CUDA(c, cudaMemcpyAsync(dst, e.W, (size_t)c->cfg.d_model * sizeof(__nv_bfloat16), cudaMemcpyDeviceToDevice, s));
+    e.W = dst;
   }
   c->h_apps[slot] = e;
   return publish_app(c, slot, s);

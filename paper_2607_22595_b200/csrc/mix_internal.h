@@ -17,6 +17,7 @@ constexpr int kTileM = 128;        // token rows per encode tile (UMMA M)
 constexpr int kTileN = 256;        // SAE features per encode tile (UMMA N)
 constexpr int kTileK = 64;         // bf16 elements per 128-byte swizzled smem row
 constexpr int kMaxGroups = 32;
+constexpr int kTeamMaxRows = 2048;  // contexts up to this T_max run probes / steering with one CTA per row
 constexpr int kMaxClasses = 64;
 constexpr int kMaxK = 1024;
 constexpr int kMaxEdits = 64;
@@ -87,6 +88,7 @@ struct Ctx {
   AppEntry* d_apps;         // [n_slots_max]
   GroupEntry* d_groups;     // [n_groups_max]
   GateEntry* d_gates;       // [n_slots_max]
+  __nv_bfloat16* d_vec_arena;   // [n_slots_max, d] copies of single-vector weights (T_max <= kTeamMaxRows), else null
   int* d_edit_idx;          // [n_slots_max * r_max]
   float* d_edit_val;
   unsigned char* d_edit_mode;

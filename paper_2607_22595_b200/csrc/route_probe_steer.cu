@@ -413,8 +413,8 @@ template <int NW>
 __global__ void __launch_bounds__(NW * 32)
 probe_steer_team_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
                         const AppEntry* __restrict__ apps, const GateEntry* __restrict__ gates, int n_slots,
-                   __nv_bfloat16* __restrict__ hidden, int d,
-                        float* __restrict__ scores, int C_max, unsigned* __restrict__ status) {
+                        __nv_bfloat16* __restrict__ hidden, int d, float* __restrict__ scores, int C_max,
+                        unsigned* __restrict__ status, const uint4* __restrict__ vec_arena) {
   __shared__ float s_part[NW][kMaxClasses];
   constexpr int NT = NW * 32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -424,23 +424,23 @@ probe_steer_team_kernel(const int* __restrict__ token_slot, const int* __restric
   if (slot == -1) return;
   const int nvec = d >> 3;
   uint4* hrow = reinterpret_cast<uint4*>(hidden + (size_t)t * d);
-  uint4 hq[kTeamVec];
+  // Single-vector weights (steering, projection, one-class probe) were copied at registration
+  // into row `slot` of the context's vector arena, so their address follows from the slot id
+  // alone: the row AND its vector are requested together, before the app entry is known.
+  uint4 hq[kTeamVec], vq[kTeamVec];
   if (slot >= 0 && slot < n_slots) {
 #pragma unroll
     for (int u = 0; u < kTeamVec; ++u) {
       const int v = threadIdx.x + u * NT;
-      if (v < nvec) hq[u] = __ldcs(hrow + v);
+      if (v < nvec) {
+        hq[u] = __ldcs(hrow + v);
+        vq[u] = __ldg(vec_arena + (size_t)slot * nvec + v);
+      }
     }
   }
   const RowApp a = lookup(slot, t, apps, gates, n_slots, status, threadIdx.x == 0);
   if (a.kind == MIX_STEER) {
     if (a.alpha == 0.f) return;                  // identity; the row stays bit-exact
-    uint4 vq[kTeamVec];
-#pragma unroll
-    for (int u = 0; u < kTeamVec; ++u) {
-      const int v = threadIdx.x + u * NT;
-      if (v < nvec) vq[u] = __ldg(a.W + v);
-    }
 #pragma unroll
     for (int u = 0; u < kTeamVec; ++u) {
       const int v = threadIdx.x + u * NT;
@@ -457,16 +457,14 @@ probe_steer_team_kernel(const int* __restrict__ token_slot, const int* __restric
   }
   if (a.kind == MIX_PROJECT) {                 // h - beta (h . r) r
     if (a.alpha == 0.f) return;
-    uint4 rq[kTeamVec];
     float dot = 0.f;
 #pragma unroll
     for (int u = 0; u < kTeamVec; ++u) {
       const int v = threadIdx.x + u * NT;
       if (v < nvec) {
-        rq[u] = __ldg(a.W + v);
         float x[8], y[8];
         unpack8(hq[u], x);
-        unpack8(rq[u], y);
+        unpack8(vq[u], y);
 #pragma unroll
         for (int e = 0; e < 8; ++e) dot = fmaf(x[e], y[e], dot);
       }
@@ -484,7 +482,7 @@ probe_steer_team_kernel(const int* __restrict__ token_slot, const int* __restric
       if (v < nvec) {
         float x[8], y[8];
         unpack8(hq[u], x);
-        unpack8(rq[u], y);
+        unpack8(vq[u], y);
 #pragma unroll
         for (int e = 0; e < 8; ++e) x[e] = fmaf(coef, y[e], x[e]);
         __stcs(hrow + v, pack8(x));
@@ -493,7 +491,23 @@ probe_steer_team_kernel(const int* __restrict__ token_slot, const int* __restric
     return;
   }
   if (a.kind != MIX_PROBE || scores == nullptr) return;
-  for (int c0 = 0; c0 < a.C; c0 += 4) {
+  if (a.C == 1) {                              // the probe vector is already here
+    float acc = 0.f;
+#pragma unroll
+    for (int u = 0; u < kTeamVec; ++u) {
+      const int v = threadIdx.x + u * NT;
+      if (v < nvec) {
+        float x[8], y[8];
+        unpack8(hq[u], x);
+        unpack8(vq[u], y);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc = fmaf(x[e], y[e], acc);
+      }
+    }
+    acc = warp_sum(acc);
+    if (lane == 0) s_part[warp][0] = acc;
+  }
+  for (int c0 = 0; c0 < (a.C == 1 ? 0 : a.C); c0 += 4) {
     const int nc = min(4, a.C - c0);
     uint4 wq[4][kTeamVec];
 #pragma unroll
@@ -726,7 +740,6 @@ __global__ void fold_bias_kernel(const __nv_bfloat16* __restrict__ W_enc, const 
 
 }  // namespace
 
-constexpr int kTeamMaxRows = 2048;   // up to here one CTA per row keeps the whole GPU busy
 
 bool has_multiclass_stage(const Ctx* c) { return c->cfg.T_max > kTeamMaxRows && c->cfg.C_max > 1; }
 
@@ -734,7 +747,8 @@ cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float
   if (c->cfg.T_max <= kTeamMaxRows) {
     probe_steer_team_kernel<8><<<c->cfg.T_max, 8 * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates,
                                                               c->cfg.n_slots_max, hidden, c->cfg.d_model, scores,
-                                                              c->cfg.C_max, c->d_status);
+                                                              c->cfg.C_max, c->d_status,
+                                                              reinterpret_cast<const uint4*>(c->d_vec_arena));
   } else {
     const int blocks = (c->cfg.T_max + kWarpsPerBlock - 1) / kWarpsPerBlock;
     probe_steer_kernel<<<blocks, kWarpsPerBlock * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates,
