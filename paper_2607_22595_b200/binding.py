@@ -23,6 +23,7 @@ MIX_GATE_GE, MIX_GATE_LT = 0, 1
 MIX_STATUS_BAD_SLOT, MIX_STATUS_BAD_GROUP, MIX_STATUS_WAIT_TIMEOUT, MIX_STATUS_TOPK_GENERAL = 1, 2, 4, 8
 MIX_FLAG_ENCODE_SIMT = 1
 MIX_FLAG_RETILE_W_ENC = 2
+MIX_FLAG_TEST_STALL_ENCODE = 4
 
 EXPORTS = [
     "mix_create", "mix_destroy", "mix_last_error", "mix_register_sae_weights", "mix_unregister_sae_weights",

@@ -24,6 +24,7 @@ constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kTcThreads = 192;
 constexpr int kTmemCols = 512;                 // two 128 x 256 fp32 accumulators
 constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz
+constexpr long long kWaitCyclesTest = 2000000ll;  // ~1 ms: the cap under MIX_FLAG_TEST_STALL_ENCODE
 
 struct __align__(8) TcShared {
   unsigned long long full[kStages];
@@ -32,6 +33,7 @@ struct __align__(8) TcShared {
   unsigned long long tmem_empty[2];
   unsigned tmem_base;
   volatile int abort_flag;
+  long long wait_cycles;      // cap of every bounded wait in this launch
   RouteState rs;
 };
 constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + (int)sizeof(TcShared);
@@ -67,7 +69,7 @@ __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, TcShare
   while (!mbar_try_wait(bar, parity)) {
     if ((++spins & 255u) == 0u) {
       if (sh->abort_flag) return false;
-      if (clock64() - t0 > kWaitCycles) {
+      if (clock64() - t0 > sh->wait_cycles) {
         sh->abort_flag = 1;
         atomicOr(status, MIX_STATUS_WAIT_TIMEOUT);
         return false;
@@ -181,7 +183,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
                  const RouteState* __restrict__ rs_g, const GroupEntry* __restrict__ groups, int n_groups,
                  float* __restrict__ Z, long long ldz, int d, unsigned* __restrict__ status, int mode,
                  const int* __restrict__ mtile_flag, const int* __restrict__ n_flagged, float* __restrict__ cand_val,
-                 int* __restrict__ cand_idx, float* __restrict__ cand_ninth, int cand_tiles, int w_tiled) {
+                 int* __restrict__ cand_idx, float* __restrict__ cand_ninth, int cand_tiles, int w_tiled, int test_stall) {
   if (mode == 1 && *n_flagged == 0) return;
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment: required by the 128-byte swizzle atoms
@@ -201,6 +203,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
       mbar_init(smem_u32(&sh->tmem_empty[a]), 4);
     }
     sh->abort_flag = 0;
+    sh->wait_cycles = test_stall ? kWaitCyclesTest : kWaitCycles;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -231,6 +234,9 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
         const CUtensorMap* tw = tmap_w + t.group;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(smem_u32(&sh->empty[stage]), phase ^ 1u, sh, status)) { ok = false; break; }
+          // Test hook (MIX_FLAG_TEST_STALL_ENCODE): the producer never fills a stage, so the consumer's
+          // bounded wait runs out and the whole CTA leaves through the time-out path.
+          if (test_stall) { ok = false; break; }
           const unsigned bar = smem_u32(&sh->full[stage]);
           mbar_expect_tx(bar, kStageBytes);
           const unsigned sa = smem_u32(tiles + stage * kStageBytes);
@@ -393,7 +399,8 @@ cudaError_t launch_encode_tc(const Ctx* c, int mode, cudaStream_t s) {
                                                              c->cfg.d_model, c->d_status, mode, c->d_mtile_flag,
                                                              c->d_n_flagged, c->d_cand_val, c->d_cand_idx,
                                                              c->d_cand_ninth, c->cand_tiles,
-                                                             (c->cfg.flags & MIX_FLAG_RETILE_W_ENC) ? 1 : 0);
+                                                             (c->cfg.flags & MIX_FLAG_RETILE_W_ENC) ? 1 : 0,
+                                                             (c->cfg.flags & MIX_FLAG_TEST_STALL_ENCODE) ? 1 : 0);
   return cudaGetLastError();
 }
 

@@ -506,8 +506,10 @@ decode_kernel(__nv_bfloat16* __restrict__ hidden, int d, const float* __restrict
         const int j = K[i];
         bool edited = false;
         for (int e = 0; e < n_edit; ++e) edited = edited || (s_eidx[e] == j);
-        s_coef[i] = edited ? 0.f : fmaxf(Kv[i], 0.f);
-        s_feat[i] = j;
+        // an id outside the SAE can only come from a call whose encode timed out: never address with it
+        const bool in_range = (unsigned)j < (unsigned)S;
+        s_coef[i] = (edited || !in_range) ? 0.f : fmaxf(Kv[i], 0.f);
+        s_feat[i] = in_range ? j : 0;
       }
       __syncthreads();
       accumulate_list(acc, s_coef, s_feat, ge.k, ge.W_dec, d, nvec);

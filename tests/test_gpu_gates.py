@@ -148,3 +148,53 @@ def test_gate_toggles_without_recapture_and_api_errors():
     with pytest.raises(mixlib.MixError) as e:
         m.set_gate(1, sc, cmp=7)
     assert e.value.code == -1
+
+
+def test_several_apps_on_the_same_rows_by_chaining_contexts_in_one_graph():
+    """Composition of apps on one model instance: a probe, a steering vector and an SAE edit all act
+    on the SAME token rows, as three hook contexts applied back to back inside one captured graph.
+    The oracle applies the three hooks in the same order."""
+    import paper_2607_22595_b200 as mixlib
+    base = W.make_tiny(DEV)
+    T, d = base.T_max, base.d_model
+    rows = np.where(np.arange(T) % 3 != 0, 0, -1).astype(np.int32)          # two thirds of the rows, slot 0
+    def ctx(app, groups=None):
+        w = W.Workload("c", d, T, T, base.hidden, rows, {0: app}, groups or {}, n_slots_max=1,
+                       n_groups_max=1 if groups else 0, C_max=1, k_max=base.k_max, r_max=base.r_max,
+                       d_sae_max=base.d_sae_max if groups else 0)
+        return w, W.make_context(mixlib.Mix, w)
+    wP, mP = ctx(base.apps[0])
+    wS, mS = ctx(base.apps[1])
+    wE, mE = ctx(base.apps[2], {0: base.groups[0]})
+    h = base.hidden.clone()
+    scores = torch.from_numpy(np.full((T, 1), CANARY_F32, dtype=np.uint32).view(np.float32)).to(DEV)
+    s = torch.cuda.Stream(); s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        for m in (mP, mS, mE):
+            m.apply(h, scores, stream=s)
+        h.copy_(base.hidden)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            mP.apply(h, scores, stream=s)       # read first: the probe sees the unmodified row
+            mS.apply(h, None, stream=s)
+            mE.apply(h, None, stream=s)
+    torch.cuda.current_stream().wait_stream(s)
+    g.replay(); torch.cuda.synchronize()
+    # oracle, hook after hook (each stage's bf16 output is the next stage's input)
+    whP = W.host(wP)
+    rP = O.apply_hook(whP)
+    whS = W.host(wS)
+    rS = O.apply_hook(whS)
+    whE = W.host(wE)
+    whE.hidden = np.stack([rS.out_bits[t] for t in range(T)])
+    rE = O.apply_hook(whE, keep_z=True)
+    got = W.bits(h)
+    hmax = float(np.abs(O.bf16_to_f64(whE.hidden)).max())
+    sc = scores.cpu().numpy()
+    for t in range(T):
+        if rows[t] < 0:
+            assert np.array_equal(got[t], whP.hidden[t]) and sc.view(np.uint32)[t, 0] == CANARY_F32
+            continue
+        assert abs(sc[t, 0] - rP.scores[t][0]) <= 1e-3 * abs(rP.scores[t][0])
+        assert np.abs(O.bf16_to_f64(got[t]) - rE.y[t]).max() <= 1e-2 * hmax
+    assert mP.get_status() == 0 and mS.get_status() == 0 and mE.get_status() == 0

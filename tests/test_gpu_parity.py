@@ -422,3 +422,27 @@ def test_replay_full_size_sampled_rows():
     assert np.array_equal(out["hidden"][unh], W.bits(w.hidden)[unh])
     out["mix"].destroy()
     torch.cuda.empty_cache()
+
+
+def test_encode_timeout_path_raises_status_and_leaves_the_context_usable():
+    """Failure detection without a GPU fault: with the test hook the encode kernel's producer never
+    delivers a tile, every CTA's bounded wait (capped at ~1 ms) runs out, the kernel returns with
+    MIX_STATUS_WAIT_TIMEOUT, and the next, ordinary call on the same device is correct."""
+    mixlib = _mixlib()
+    w = W.make_tiny(DEV)
+    m = W.make_context(mixlib.Mix, w, flags=mixlib.MIX_FLAG_TEST_STALL_ENCODE)
+    h = w.hidden.clone()
+    scores = torch.zeros((w.T_max, 1), dtype=torch.float32, device=DEV)
+    m.apply(h, scores)
+    torch.cuda.synchronize()                                   # returns: nothing hangs
+    st = m.get_status()
+    assert st & mixlib.MIX_STATUS_WAIT_TIMEOUT
+    assert m.get_status() == 0                                 # reading the word clears it
+    # rows without an SAE app are unaffected by the failed encode
+    wh = W.host(w)
+    ref = O.apply_hook(wh)
+    for t in range(w.T_max):
+        if ref.kind[t] in (0, O.KIND_PROBE):
+            assert np.array_equal(W.bits(h)[t], wh.hidden[t])
+    m.destroy()
+    check_parity(wh, run_gpu(w))                               # a fresh ordinary context works
