@@ -64,7 +64,8 @@ def f64_to_bf16_bits(x) -> np.ndarray:
     q = np.ldexp(1.0, qexp)
     r = np.rint(a / q) * q                   # rint = round half to even; a/q is exact
     r = np.where(np.isfinite(a), r, a)
-    r32 = r.astype(np.float32)               # exact: r has <= 8 significant bits
+    with np.errstate(over="ignore"):          # beyond the largest bf16 the next line sets infinity
+        r32 = r.astype(np.float32)           # exact: r has <= 8 significant bits
     r32 = np.where(r > 3.3895313892515355e38, np.float32(np.inf), r32)   # max bf16
     out = (r32.view(np.uint32) >> np.uint32(16)).astype(np.uint16)
     out = np.where(np.isnan(x), np.uint16(0x7FC0), out)
