@@ -210,9 +210,9 @@ def time_stages(m, fn, reps=5):
     return dict(zip(m.STAGES[:n], best))
 
 
-def extras_sae(name, w, peaks, mixlib):
+def extras_sae(name, w, peaks, mixlib, extra_flags=0):
     """SAE-carrying config: per-kernel times, encode flop rate and weight-stream bandwidth."""
-    m = W.make_context(mixlib.Mix, w, flags=SAE_FLAGS)
+    m = W.make_context(mixlib.Mix, w, flags=SAE_FLAGS | extra_flags)
     h = w.hidden.clone()
     scores = torch.zeros((w.T_max, max(w.C_max, 1)), dtype=torch.float32, device="cuda")
     def fn():
@@ -537,7 +537,14 @@ def run_mix(args, rank, world, local_rank):
                 ex["sweep"] = extras_sweep(peaks, mixlib)
                 ex["sae_heavy"] = extras_sae("sae_heavy (config 2)", W.make_sae_heavy("cuda"), peaks, mixlib)
                 torch.cuda.empty_cache()
-                ex["mixed"] = extras_sae("mixed (config 3)", W.make_mixed("cuda"), peaks, mixlib)
+                wm = W.make_mixed("cuda")
+                ex["mixed"] = extras_sae("mixed (config 3)", wm, peaks, mixlib)
+                eo = extras_sae("mixed (config 3), edit-only shortcut", wm, peaks, mixlib, extra_flags=8)
+                ex["mixed_edit_only_shortcut"] = {
+                    "note": "MIX_FLAG_SAE_EDIT_ONLY: JumpReLU rows with the error term skip the encode (16 dot products "
+                            "per row instead); an algorithmic shortcut, not counted toward any tensor-pipe fraction",
+                    "t_call_ms_graph": eo["t_call_ms_graph"], "stage_ms": eo["stage_ms"],
+                    "token_rows_per_s": eo["token_rows_per_s"], "status": eo["status"]}
             except Exception as e:                       # extras never break the contract line
                 ex["error"] = repr(e)
             line["extras"] = ex

@@ -88,7 +88,11 @@ enum {
   MIX_FLAG_TEST_STALL_ENCODE = 1u << 2 /* test hook for the time-out path: the encode kernel's producer never delivers a
                                          tile and every bounded wait is capped at ~1 ms, so each CTA gives up, raises
                                          MIX_STATUS_WAIT_TIMEOUT, frees its tensor memory and returns; the SAE rows of that
-                                         call are not meaningful.  Nothing hangs and the context stays usable */
+                                         call are not meaningful.  Nothing hangs and the context stays usable */,
+  MIX_FLAG_SAE_EDIT_ONLY = 1u << 3    /* algorithmic shortcut: rows of a ReLU / JumpReLU weight set whose app has the
+                                         error term on skip the encode; only the pre-activations of their edited
+                                         features are computed (|edits| dot products per row).  Same hidden output;
+                                         n_active is not produced for those rows.  TopK rows are unaffected */
 };
 
 typedef struct {
@@ -248,7 +252,8 @@ int mix_get_status(mix_ctx* ctx, unsigned* bits, void* stream);
 
 /* Number of kernels one mix_apply() call launches on this context (fixed at mix_create):
    1 without SAE weight sets, else 8 (6 with MIX_FLAG_ENCODE_SIMT); one more when T_max > 2048
-   and C_max > 1 (multi-class probes of large batches run in a kernel of their own). */
+   and C_max > 1 (multi-class probes of large batches run in a kernel of their own), and one more
+   with MIX_FLAG_SAE_EDIT_ONLY. */
 int mix_launches_per_apply(const mix_ctx* ctx);
 
 /* Per-kernel timing taps (profiling only; do not use while capturing a graph).  events: HOST
@@ -257,7 +262,8 @@ int mix_launches_per_apply(const mix_ctx* ctx);
    its first kernel and events[i] after its i-th kernel, on the call's stream; the array is
    copied.  Kernel order: probe_steer, [probe_multiclass: only if T_max > 2048 and C_max > 1,]
    route, pack, encode, merge, encode (flagged row tiles), select, decode; with
-   MIX_FLAG_ENCODE_SIMT the SAE part is route, pack, encode, select, decode. */
+   MIX_FLAG_ENCODE_SIMT the SAE part is route, pack, encode, select, decode; with
+   MIX_FLAG_SAE_EDIT_ONLY an edit_only kernel comes last. */
 int mix_set_stage_events(mix_ctx* ctx, void* const* events);
 
 /* Test / profiling taps into the SAE workspace after a mix_apply (device pointers owned by

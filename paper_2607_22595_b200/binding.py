@@ -24,6 +24,7 @@ MIX_STATUS_BAD_SLOT, MIX_STATUS_BAD_GROUP, MIX_STATUS_WAIT_TIMEOUT, MIX_STATUS_T
 MIX_FLAG_ENCODE_SIMT = 1
 MIX_FLAG_RETILE_W_ENC = 2
 MIX_FLAG_TEST_STALL_ENCODE = 4
+MIX_FLAG_SAE_EDIT_ONLY = 8
 
 EXPORTS = [
     "mix_create", "mix_destroy", "mix_last_error", "mix_register_sae_weights", "mix_unregister_sae_weights",
@@ -261,9 +262,10 @@ class Mix:
             front.append("probe_multiclass")
         if self.cfg.n_groups_max == 0:
             return front
+        tail = ["edit_only"] if self.cfg.flags & MIX_FLAG_SAE_EDIT_ONLY else []
         if self.cfg.flags & MIX_FLAG_ENCODE_SIMT:
-            return front + ["route", "pack", "encode", "select", "decode"]
-        return front + ["route", "pack", "encode", "merge", "encode_flagged", "select", "decode"]
+            return front + ["route", "pack", "encode", "select", "decode"] + tail
+        return front + ["route", "pack", "encode", "merge", "encode_flagged", "select", "decode"] + tail
 
     def set_stage_events(self, events=None):
         """events: list of launches_per_apply() + 1 torch.cuda.Event(enable_timing=True), or None."""

@@ -510,6 +510,10 @@ int mix_apply(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream) 
     }
     MIX_CUDA(c, launch_decode(c, h, s));
     MIX_CUDA(c, tap());
+    if (c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) {
+      MIX_CUDA(c, launch_edit_only(c, h, T, s));
+      MIX_CUDA(c, tap());
+    }
   }
   if (fork) MIX_CUDA(c, cudaStreamWaitEvent(s, c->ev_join, 0));
   return MIX_OK;
@@ -519,7 +523,7 @@ int mix_launches_per_apply(const mix_ctx* c) {
   if (!c) return 0;
   const int front = has_multiclass_stage(c) ? 2 : 1;
   if (c->cfg.n_groups_max == 0) return front;
-  return front + ((c->cfg.flags & MIX_FLAG_ENCODE_SIMT) ? 5 : 7);
+  return front + ((c->cfg.flags & MIX_FLAG_ENCODE_SIMT) ? 5 : 7) + ((c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) ? 1 : 0);
 }
 
 int mix_get_status(mix_ctx* c, unsigned* bits, void* stream) {

@@ -147,6 +147,7 @@ cudaError_t launch_encode_tc(const Ctx* c, int mode, cudaStream_t s);   // 0: al
 cudaError_t launch_merge(const Ctx* c, cudaStream_t s);
 cudaError_t launch_select(const Ctx* c, bool flagged_only, cudaStream_t s);
 cudaError_t launch_decode(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s);
+cudaError_t launch_edit_only(const Ctx* c, __nv_bfloat16* hidden, int T, cudaStream_t s);
 cudaError_t launch_compose_map(const Ctx* c, int T_live, int n_req, cudaStream_t s);
 cudaError_t launch_fold_bias(const __nv_bfloat16* W_enc, const float* b_enc, const float* b_dec, float* b_eff,
                              long long d_sae, int d, cudaStream_t s);

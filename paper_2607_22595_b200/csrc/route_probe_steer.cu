@@ -567,7 +567,7 @@ route_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_
              const GroupEntry* __restrict__ groups, int n_groups,
              int* __restrict__ panel_row, int panel_cap, int* __restrict__ mtile_group, RouteState* __restrict__ rs,
              unsigned* __restrict__ status, int* __restrict__ row_flag, int* __restrict__ mtile_flag,
-             int* __restrict__ n_flagged, int* __restrict__ row_group) {
+             int* __restrict__ n_flagged, int* __restrict__ row_group, int edit_only) {
   extern __shared__ int s_cnt[];                      // [n_chunks * kRouteWarps][n_groups]
   __shared__ int s_total[kMaxGroups], s_base[kMaxGroups + 1];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -612,6 +612,9 @@ route_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_
         const int g = group_id[c];
         if (g < 0 || g >= n_groups || !__ldg(&groups[g].valid)) {
           atomicOr(status, MIX_STATUS_BAD_GROUP);
+        } else if (edit_only && __ldg(&apps[slot[c]].add_error) && __ldg(&groups[g].act) != MIX_SAE_TOPK) {
+          // handled by sae_edit_only_kernel: with the error term on, a ReLU / JumpReLU row needs
+          // only the pre-activations of its edited features, not the whole encode
         } else if (!(head[c].y & kKindGated) || gate_open(gates, slot[c], (c0 + c) * kRouteThreads + tid)) {
           grp[c] = g;
         }
@@ -772,7 +775,8 @@ cudaError_t launch_route(const Ctx* c, int T, cudaStream_t s) {
   route_kernel<<<1, kRouteThreads, smem, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates, c->cfg.n_slots_max,
                                               c->d_groups, c->cfg.n_groups_max, c->d_panel_row, c->panel_rows_cap,
                                               c->d_mtile_group, c->d_route, c->d_status, c->d_row_flag,
-                                              c->d_mtile_flag, c->d_n_flagged, c->d_row_group);
+                                              c->d_mtile_flag, c->d_n_flagged, c->d_row_group,
+                                              (c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) ? 1 : 0);
   return cudaGetLastError();
 }
 

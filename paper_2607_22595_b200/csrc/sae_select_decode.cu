@@ -551,6 +551,103 @@ decode_kernel(__nv_bfloat16* __restrict__ hidden, int d, const float* __restrict
   }
 }
 
+// ---------------------------------------------------------------------------------------
+// edit-only shortcut (MIX_FLAG_SAE_EDIT_ONLY)
+// ---------------------------------------------------------------------------------------
+// With the error term on, h' = h + sum over edited j of (f'_j - f_j) W_dec[j]: for ReLU and JumpReLU
+// sets f_j depends on z_j alone, so a row needs just the |edits| pre-activations
+// z_j = W_enc[j] . h + b_eff[j] -- 16 dot products instead of the d_sae-wide encode.  (TopK rows
+// still need every pre-activation to know which features are kept.)  One CTA per token row,
+// straight from the slot map; rows of other kinds leave after one table lookup.
+__global__ void __launch_bounds__(kDecThreads)
+sae_edit_only_kernel(__nv_bfloat16* __restrict__ hidden, int d, const int* __restrict__ token_slot,
+                     const int* __restrict__ n_live_p, int T, const AppEntry* __restrict__ apps,
+                     const GateEntry* __restrict__ gates, int n_slots, const GroupEntry* __restrict__ groups,
+                     int n_groups, const int* __restrict__ edit_idx, const float* __restrict__ edit_val,
+                     const unsigned char* __restrict__ edit_mode, int r_max) {
+  __shared__ float s_coef[kMaxEdits];
+  __shared__ int s_feat[kMaxEdits];
+  __shared__ int s_any;
+  const int t = blockIdx.x;
+  if (t >= min(T, *n_live_p)) return;
+  const int slot = token_slot[t];
+  if (slot < 0 || slot >= n_slots) return;
+  const AppEntry app = apps[slot];
+  if (!app.valid || (app.kind & kKindMask) != MIX_SAE || !app.add_error) return;
+  if (app.group < 0 || app.group >= n_groups) return;
+  const GroupEntry ge = groups[app.group];
+  if (!ge.valid || ge.act == MIX_SAE_TOPK) return;
+  if (app.kind & kKindGated) {
+    const GateEntry gt = gates[slot];
+    const float v = gt.scores[(size_t)t * gt.stride + gt.col];
+    if (!(gt.cmp == MIX_GATE_GE ? v >= gt.thr : v < gt.thr)) return;
+  }
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n_edit = app.n_edit, nvec = d >> 3;
+  const uint4* hrow = reinterpret_cast<const uint4*>(hidden + (size_t)t * d);
+  if (tid == 0) s_any = 0;
+  if (tid < n_edit) s_feat[tid] = edit_idx[slot * r_max + tid];
+  __syncthreads();
+  for (int e = warp; e < n_edit; e += kDecThreads / 32) {      // one warp per edited feature
+    const int j = s_feat[e];
+    const uint4* wrow = reinterpret_cast<const uint4*>(ge.W_enc + (size_t)j * d);
+    float acc = 0.f;
+    for (int v = lane; v < nvec; v += 32) {
+      const uint4 a = hrow[v], b = __ldg(wrow + v);
+      const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
+      const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 x = __bfloat1622float2(pa[i]), y = __bfloat1622float2(pb[i]);
+        acc = fmaf(x.x, y.x, acc);
+        acc = fmaf(x.y, y.y, acc);
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) {
+      const float z = acc + ge.b_eff[j];
+      const float f = ge.act == MIX_SAE_RELU ? fmaxf(z, 0.f) : (z > ge.theta[j] ? z : 0.f);
+      bool alive = true;                                     // a later entry for the same feature wins
+      for (int e2 = e + 1; e2 < n_edit; ++e2) alive = alive && (s_feat[e2] != j);
+      const float fnew = edit_mode[slot * r_max + e] == MIX_EDIT_CLAMP ? edit_val[slot * r_max + e] : 0.f;
+      const float delta = alive ? fnew - f : 0.f;
+      s_coef[e] = delta;
+      if (delta != 0.f) s_any = 1;
+    }
+  }
+  __syncthreads();
+  if (!s_any) return;                                        // no effective edit: the row stays bit-exact
+  float acc[kDecU][8];
+#pragma unroll
+  for (int u = 0; u < kDecU; ++u) {
+    const int v = tid + u * kDecThreads;
+    if (v < nvec) {
+      const uint4 q = hrow[v];
+      const __nv_bfloat162* pp = reinterpret_cast<const __nv_bfloat162*>(&q);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 f2 = __bfloat1622float2(pp[i]);
+        acc[u][2 * i] = f2.x;
+        acc[u][2 * i + 1] = f2.y;
+      }
+    }
+  }
+  accumulate_list(acc, s_coef, s_feat, n_edit, ge.W_dec, d, nvec);
+  uint4* hout = reinterpret_cast<uint4*>(hidden + (size_t)t * d);
+#pragma unroll
+  for (int u = 0; u < kDecU; ++u) {
+    const int v = tid + u * kDecThreads;
+    if (v < nvec) {
+      uint4 q;
+      __nv_bfloat162* pp = reinterpret_cast<__nv_bfloat162*>(&q);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) pp[i] = __floats2bfloat162_rn(acc[u][2 * i], acc[u][2 * i + 1]);
+      hout[v] = q;
+    }
+  }
+}
+
 }  // namespace
 
 // one CTA per packed row, but never more than a few waves: rows are walked grid-stride
@@ -581,6 +678,14 @@ cudaError_t launch_select(const Ctx* c, bool flagged_only, cudaStream_t s) {
                                                           c->d_topk_idx, c->d_topk_val, c->out_topk_idx,
                                                           c->out_topk_val, c->out_n_active, c->d_status,
                                                           flagged_only ? c->d_row_flag : nullptr, c->d_n_flagged);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_edit_only(const Ctx* c, __nv_bfloat16* hidden, int T, cudaStream_t s) {
+  sae_edit_only_kernel<<<c->cfg.T_max, kDecThreads, 0, s>>>(hidden, c->cfg.d_model, c->d_token_slot, c->d_n_live, T,
+                                                            c->d_apps, c->d_gates, c->cfg.n_slots_max, c->d_groups,
+                                                            c->cfg.n_groups_max, c->d_edit_idx, c->d_edit_val,
+                                                            c->d_edit_mode, c->cfg.r_max);
   return cudaGetLastError();
 }
 

@@ -61,6 +61,27 @@ def test_retiled_w_enc_matches_oracle():
     check_parity(W.host(w), run_gpu(w, flags=mixlib.MIX_FLAG_RETILE_W_ENC))
 
 
+@pytest.mark.parametrize("simt", [False, True])
+def test_edit_only_shortcut_gives_the_same_hidden(simt):
+    # ReLU / JumpReLU rows with the error term skip the encode; TopK rows and replace-mode rows do not
+    mixlib = _mixlib()
+    flags = mixlib.MIX_FLAG_SAE_EDIT_ONLY | (mixlib.MIX_FLAG_ENCODE_SIMT if simt else 0)
+    w = W.make_mixed(DEV, d=320, T=1500, R=40, d_sae=1024, cap=200, mu=3.5, edit_hint=oracle_edit_hint)
+    g = torch.Generator(device=DEV); g.manual_seed(3)
+    sc = torch.randn((w.T_max, 1), generator=g, device=DEV)
+    sae_slots = [s for s, a in w.apps.items() if a.kind == W.KIND_SAE]
+    w.apps[sae_slots[0]].gate = W.Gate(sc, 0, W.GATE_GE, 0.0)          # a gated edit-only app
+    w.apps[sae_slots[1]].add_error = False                              # this one still needs the encode
+    w.groups[1].b_enc = w.groups[1].b_enc - 2.0                         # keep its replace-mode decode sparse
+    w.apps[sae_slots[1]].group = 1
+    out = run_gpu(w, flags=flags, graph=True)
+    check_parity(W.host(w), out, check_features=False)
+    for act in (W.SAE_RELU, W.SAE_TOPK):
+        w1 = _one_sae_workload(192, 1024, act, 24, 150, True, ([5, 900, 17, 5], [3.0, 0.0, 6.5, 4.0], [0, 1, 0, 0]),
+                               b_dec=True, center=True)
+        check_parity(W.host(w1), run_gpu(w1, flags=flags), check_features=False)
+
+
 def test_mixed_small():
     w = W.make_mixed(DEV, d=320, T=1500, R=40, d_sae=1024, cap=200, mu=3.5, edit_hint=oracle_edit_hint)
     out = run_gpu(w, graph=True)
