@@ -63,7 +63,7 @@ typedef enum {
   MIX_ERR_CUDA = -5           /* a CUDA call failed; see mix_last_error() */
 } mix_status;
 
-enum { MIX_PROBE = 1, MIX_STEER = 2, MIX_SAE = 3, MIX_PROJECT = 4 };   /* app kinds */
+enum { MIX_PROBE = 1, MIX_STEER = 2, MIX_SAE = 3, MIX_PROJECT = 4, MIX_ROUTER = 5 };   /* app kinds */
 enum { MIX_ACT_SIGMOID = 0, MIX_ACT_SOFTMAX = 1, MIX_ACT_NONE = 2 };   /* probe activations */
 enum { MIX_SAE_RELU = 0, MIX_SAE_JUMPRELU = 1, MIX_SAE_TOPK = 2 };     /* SAE activations */
 enum { MIX_EDIT_CLAMP = 0, MIX_EDIT_ABLATE = 1 };                      /* per-feature edits */
@@ -129,6 +129,15 @@ typedef struct {
   float beta;
 } mix_project;
 
+/* MoE router-logit steering (paper, Table 1 row 7: a conditional write whose target is the router
+   logits, used to switch experts on or off).  delta: device fp32 [n_experts], added to the router
+   logits of the app's rows by mix_apply_router(); +-INFINITY entries force an expert in or out of
+   the top-k that the model's router takes afterwards.  mix_apply() ignores apps of this kind. */
+typedef struct {
+  int n_experts;
+  const float* delta;
+} mix_router;
+
 /* One SAE weight set, shared by any number of app slots.  All pointers device.
    W_enc bf16 [d_sae, d]: row j = encoder direction j.  b_enc fp32 [d_sae].
    theta fp32 [d_sae] (JumpReLU only, else NULL).  W_dec bf16 [d_sae, d]: row j = decoder
@@ -181,8 +190,8 @@ int mix_register_sae_weights(mix_ctx* ctx, int group, const mix_sae_weights* w, 
 int mix_unregister_sae_weights(mix_ctx* ctx, int group, void* stream);
 
 /* Attach an MI function to `slot` (paper, Section 4.2: functions are attached ahead of time
-   with their parameters).  `desc` points to a mix_probe, mix_steer, mix_sae_app or mix_project
-   according to `kind`.  Stream-ordered; an entry becomes visible atomically (its valid flag is
+   with their parameters).  `desc` points to a mix_probe, mix_steer, mix_sae_app, mix_project or
+   mix_router according to `kind`.  Stream-ordered; an entry becomes visible atomically (its valid flag is
    written last).  Errors: OUT_OF_RANGE (slot, n_classes > C_max, n_edit > r_max, edit
    index >= d_sae of the group, group), INVALID_ARG. */
 int mix_register_app(mix_ctx* ctx, int slot, int kind, const void* desc, void* stream);
@@ -245,6 +254,13 @@ int mix_set_feature_out(mix_ctx* ctx, int* topk_idx, float* topk_val, int* n_act
    problems (bad slot ids, ...) are reported through the status word, never by faulting.
    Errors: INVALID_ARG (NULL hidden, misaligned), OUT_OF_RANGE (T), CUDA (launch failure). */
 int mix_apply(mix_ctx* ctx, void* hidden, int T, float* scores_out, void* stream);
+
+/* The hook on a different target tensor: router logits (device fp32 [T_max, n_experts], modified in
+   place).  Rows whose slot holds a MIX_ROUTER app with the same n_experts (and an open gate, if it
+   has one) get logits[t, :] += delta; every other row is neither read nor written.  Uses the same
+   slot map, live count and gates as mix_apply(); one kernel, capturable.
+   Errors: INVALID_ARG (NULL logits, n_experts < 1), OUT_OF_RANGE (T). */
+int mix_apply_router(mix_ctx* ctx, float* logits, int n_experts, int T, void* stream);
 
 /* Copy the device status word (bits MIX_STATUS_*) to *bits and clear it on the device.
    Synchronises `stream`. */

@@ -32,7 +32,7 @@ from typing import Dict, Iterable, Optional
 import numpy as np
 
 # kinds / enums restated here on purpose (the oracle depends on nothing else)
-KIND_PROBE, KIND_STEER, KIND_SAE, KIND_PROJECT = 1, 2, 3, 4
+KIND_PROBE, KIND_STEER, KIND_SAE, KIND_PROJECT, KIND_ROUTER = 1, 2, 3, 4, 5
 ACT_SIGMOID, ACT_SOFTMAX, ACT_NONE = 0, 1, 2
 SAE_RELU, SAE_JUMPRELU, SAE_TOPK = 0, 1, 2
 EDIT_CLAMP, EDIT_ABLATE = 0, 1
@@ -281,6 +281,11 @@ def apply_hook(w, rows: Optional[Iterable[int]] = None, keep_z: bool = False,
             res.modified[t] = True
             res.y[t] = y
             res.out_bits[t] = f64_to_bf16_bits(y)
+        elif app.kind == KIND_ROUTER:            # acts on the router logits, not on the hidden state
+            res.kind[t] = 0
+            res.modified[t] = False
+            res.out_bits[t] = hidden_bits[t].copy()
+            res.y[t] = h
         elif app.kind == KIND_SAE:
             sae_rows.setdefault(app.group, []).append(t)
         else:
@@ -302,3 +307,22 @@ def apply_hook(w, rows: Optional[Iterable[int]] = None, keep_z: bool = False,
             if keep_z:
                 res.z[t] = Z[n].copy()
     return res
+
+
+# ---------------------------------------------------------------------------
+# router-logit steering  (Table 1, row 7: a conditional write on the MoE router logits)
+# ---------------------------------------------------------------------------
+def apply_router_hook(w, logits: np.ndarray) -> np.ndarray:
+    """logits fp32 [T, E] -> float64 [T, E]: rows whose slot holds a router app with E experts (and
+    an open gate) get logits + delta; every other row is returned unchanged."""
+    out = np.asarray(logits, dtype=np.float64).copy()
+    E = out.shape[1]
+    for t in range(min(w.T_live, w.T_max)):
+        s = int(w.token_slot[t])
+        app = w.apps.get(s) if 0 <= s < w.n_slots_max else None
+        if app is None or app.kind != KIND_ROUTER or len(app.delta) != E:
+            continue
+        if getattr(app, "gate", None) is not None and not gate_open(app.gate, t):
+            continue
+        out[t] = out[t] + np.asarray(app.delta, dtype=np.float64)
+    return out

@@ -15,7 +15,7 @@ import torch
 
 from . import _build
 
-MIX_PROBE, MIX_STEER, MIX_SAE, MIX_PROJECT = 1, 2, 3, 4
+MIX_PROBE, MIX_STEER, MIX_SAE, MIX_PROJECT, MIX_ROUTER = 1, 2, 3, 4, 5
 MIX_ACT_SIGMOID, MIX_ACT_SOFTMAX, MIX_ACT_NONE = 0, 1, 2
 MIX_SAE_RELU, MIX_SAE_JUMPRELU, MIX_SAE_TOPK = 0, 1, 2
 MIX_EDIT_CLAMP, MIX_EDIT_ABLATE = 0, 1
@@ -29,7 +29,7 @@ MIX_FLAG_SAE_EDIT_ONLY = 8
 EXPORTS = [
     "mix_create", "mix_destroy", "mix_last_error", "mix_register_sae_weights", "mix_unregister_sae_weights",
     "mix_register_app", "mix_unregister_app", "mix_set_gate", "mix_update_steer_alpha", "mix_update_sae_edits",
-    "mix_set_slot_map", "mix_set_request_map", "mix_set_feature_out", "mix_apply", "mix_get_status",
+    "mix_set_slot_map", "mix_set_request_map", "mix_set_feature_out", "mix_apply", "mix_apply_router", "mix_get_status",
     "mix_launches_per_apply", "mix_set_stage_events", "mix_debug_workspace", "mix_sae_apply_static",
 ]
 
@@ -46,6 +46,10 @@ class MixProbe(C.Structure):
 
 class MixSteer(C.Structure):
     _fields_ = [("v", C.c_void_p), ("alpha", C.c_float)]
+
+
+class MixRouter(C.Structure):
+    _fields_ = [("n_experts", C.c_int), ("delta", C.c_void_p)]
 
 
 class MixSaeWeights(C.Structure):
@@ -93,6 +97,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.mix_set_request_map.argtypes = [vp, vp, ci, vp, ci, ci, vp]
     lib.mix_set_feature_out.argtypes = [vp, vp, vp, vp]
     lib.mix_apply.argtypes = [vp, vp, ci, vp, vp]
+    lib.mix_apply_router.argtypes = [vp, vp, ci, ci, vp]
     lib.mix_get_status.argtypes = [vp, C.POINTER(C.c_uint), vp]
     lib.mix_launches_per_apply.argtypes = [vp]
     lib.mix_set_stage_events.argtypes = [vp, C.POINTER(vp)]
@@ -177,6 +182,17 @@ class Mix:
         d = MixSteer(_ptr(r), float(beta))          # mix_project has the layout of mix_steer: (pointer, float)
         self._check(self.lib.mix_register_app(self.ctx, slot, MIX_PROJECT, C.byref(d), _stream(stream)))
         self._keep[("a", slot)] = (r,)
+
+    def register_router(self, slot, delta, stream=None):
+        assert delta.dtype == torch.float32 and delta.dim() == 1
+        d = MixRouter(int(delta.numel()), _ptr(delta))
+        self._check(self.lib.mix_register_app(self.ctx, slot, MIX_ROUTER, C.byref(d), _stream(stream)))
+        self._keep[("a", slot)] = (delta,)
+
+    def apply_router(self, logits, T=None, stream=None):
+        assert logits.dtype == torch.float32 and logits.is_cuda and logits.is_contiguous() and logits.dim() == 2
+        T = logits.shape[0] if T is None else T
+        self._check(self.lib.mix_apply_router(self.ctx, logits.data_ptr(), int(logits.shape[1]), int(T), _stream(stream)))
 
     @staticmethod
     def _edit_arrays(idx, val, mode):

@@ -324,6 +324,12 @@ int mix_register_app(mix_ctx* c, int slot, int kind, const void* desc, void* str
     if (!p->r || !aligned16(p->r)) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "projection vector is NULL or not 16-byte aligned");
     e.W = p->r;
     e.alpha = p->beta;
+  } else if (kind == MIX_ROUTER) {
+    const mix_router* p = static_cast<const mix_router*>(desc);
+    if (p->n_experts < 1) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "n_experts %d < 1", p->n_experts);
+    if (!p->delta) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "router delta is NULL");
+    e.n_classes = p->n_experts;
+    e.W = p->delta;
   } else if (kind == MIX_SAE) {
     const mix_sae_app* p = static_cast<const mix_sae_app*>(desc);
     if (p->group < 0 || p->group >= c->cfg.n_groups_max || !c->h_groups[p->group].valid)
@@ -516,6 +522,14 @@ int mix_apply(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream) 
     }
   }
   if (fork) MIX_CUDA(c, cudaStreamWaitEvent(s, c->ev_join, 0));
+  return MIX_OK;
+}
+
+int mix_apply_router(mix_ctx* c, float* logits, int n_experts, int T, void* stream) {
+  if (!c) return MIX_ERR_INVALID_ARG;
+  if (!logits || n_experts < 1) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "logits is NULL or n_experts < 1");
+  if (T < 0 || T > c->cfg.T_max) MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "T %d outside [0, T_max=%d]", T, c->cfg.T_max);
+  MIX_CUDA(c, launch_router(c, logits, n_experts, T, static_cast<cudaStream_t>(stream)));
   return MIX_OK;
 }
 

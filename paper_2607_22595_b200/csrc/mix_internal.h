@@ -140,6 +140,7 @@ struct Ctx {
 cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s);
 cudaError_t launch_probe_multiclass(const Ctx* c, const __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s);
 bool has_multiclass_stage(const Ctx* c);   // large batches with multi-class probes get a kernel of their own
+cudaError_t launch_router(const Ctx* c, float* logits, int n_experts, int T, cudaStream_t s);
 cudaError_t launch_route(const Ctx* c, int T, cudaStream_t s);
 cudaError_t launch_pack(const Ctx* c, const __nv_bfloat16* hidden, cudaStream_t s);
 cudaError_t launch_encode_simt(const Ctx* c, cudaStream_t s);

@@ -721,6 +721,19 @@ pack_kernel(const __nv_bfloat16* __restrict__ hidden, const int* __restrict__ pa
   for (int i = lane; i < nvec; i += 32) dst[i] = __ldg(src + i);
 }
 
+// Router-logit steering: one thread per (row, expert).
+__global__ void __launch_bounds__(256)
+router_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
+              const AppEntry* __restrict__ apps, const GateEntry* __restrict__ gates, int n_slots,
+              float* __restrict__ logits, int n_experts) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int t = (int)(i / n_experts), e = (int)(i - (long long)t * n_experts);
+  if (t >= min(T, __ldg(n_live_p))) return;
+  const RowApp a = lookup(__ldg(token_slot + t), t, apps, gates, n_slots, nullptr, false);
+  if (a.kind != MIX_ROUTER || a.C != n_experts) return;
+  logits[i] += __ldg(reinterpret_cast<const float*>(a.W) + e);
+}
+
 __global__ void compose_map_kernel(const int* __restrict__ token_req, const int* __restrict__ req_slot, int T_live,
                                    int n_req, int* __restrict__ token_slot) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
@@ -766,6 +779,13 @@ cudaError_t launch_probe_multiclass(const Ctx* c, const __nv_bfloat16* hidden, i
   probe_multiclass_kernel<<<blocks, kMcWarps * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates,
                                                                  c->cfg.n_slots_max, hidden, c->cfg.d_model, scores,
                                                                  c->cfg.C_max);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_router(const Ctx* c, float* logits, int n_experts, int T, cudaStream_t s) {
+  const long long n = (long long)c->cfg.T_max * n_experts;
+  router_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates,
+                                                            c->cfg.n_slots_max, logits, n_experts);
   return cudaGetLastError();
 }
 

@@ -198,3 +198,52 @@ def test_several_apps_on_the_same_rows_by_chaining_contexts_in_one_graph():
         assert abs(sc[t, 0] - rP.scores[t][0]) <= 1e-3 * abs(rP.scores[t][0])
         assert np.abs(O.bf16_to_f64(got[t]) - rE.y[t]).max() <= 1e-2 * hmax
     assert mP.get_status() == 0 and mS.get_status() == 0 and mE.get_status() == 0
+
+
+def test_router_logit_steering_matches_oracle_and_leaves_hidden_alone():
+    import paper_2607_22595_b200 as mixlib
+    rng = np.random.default_rng(51)
+    T, E, d = 300, 8, 128
+    g = torch.Generator(device=DEV); g.manual_seed(51)
+    hidden = torch.randn((T, d), generator=g, device=DEV).to(torch.bfloat16)
+    logits = torch.randn((T, E), generator=g, device=DEV)
+    d0 = torch.tensor([0, 1.5, float("-inf"), 0, 0, float("inf"), -2.0, 0.25], device=DEV)
+    d1 = torch.randn(E, generator=g, device=DEV)
+    v = torch.randn(d, generator=g, device=DEV).to(torch.bfloat16)
+    sc = torch.randn((T, 1), generator=g, device=DEV)
+    apps = {0: W.Router(d0), 1: W.Router(d1, gate=W.Gate(sc, 0, W.GATE_LT, 0.1)), 2: W.Steer(v, 2.0),
+            3: W.Router(torch.zeros(16, device=DEV))}                       # 16 experts: not this tensor's width
+    slots = rng.choice([-1, 0, 1, 2, 3, 7], size=T).astype(np.int32)
+    w = W.Workload("router", d, T, 280, hidden, slots, apps, {}, n_slots_max=8)
+    m = W.make_context(mixlib.Mix, w)
+    lg, h = logits.clone(), hidden.clone()
+    s = torch.cuda.Stream(); s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        m.apply_router(lg, stream=s); lg.copy_(logits)
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr, stream=s):
+            m.apply_router(lg, stream=s)
+            m.apply(h, None, stream=s)
+    torch.cuda.current_stream().wait_stream(s)
+    gr.replay(); torch.cuda.synchronize()
+    wh = W.host(w)
+    want = O.apply_router_hook(wh, logits.cpu().numpy())
+    got = lg.cpu().numpy().astype(np.float64)
+    touched = 0
+    for t in range(T):
+        if np.array_equal(want[t], logits[t].cpu().numpy().astype(np.float64)):
+            assert np.array_equal(lg[t].cpu().numpy().view(np.uint32), logits[t].cpu().numpy().view(np.uint32))   # bit-exact
+        else:
+            touched += 1
+            fin = np.isfinite(want[t])
+            assert np.array_equal(got[t][~fin], want[t][~fin])
+            assert np.abs(got[t][fin] - want[t][fin]).max() <= 1e-6 * np.maximum(1.0, np.abs(want[t][fin])).max()
+    assert touched > 40
+    # the hidden-state hook saw the same map: steering rows changed, router rows did not
+    out = dict(hidden=W.bits(h), scores=np.full((T, 1), 0, dtype=np.float32).view(np.uint32).view(np.float32),
+               status=m.get_status())
+    ref = O.apply_hook(wh)
+    for t in range(T):
+        if ref.kind[t] == 0:
+            assert np.array_equal(out["hidden"][t], wh.hidden[t])
+    assert out["status"] == mixlib.MIX_STATUS_BAD_SLOT              # slot 7 was never registered

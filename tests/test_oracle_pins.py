@@ -387,3 +387,28 @@ def test_project_hand_worked_and_invariants():
     for t in np.nonzero(w.token_slot == 1)[0]:
         hh = O.bf16_to_f64(w.hidden[t]); rr = O.bf16_to_f64(rv)
         assert np.array_equal(res.y[int(t)], hh - (hh @ rr) * rr) and res.kind[int(t)] == O.KIND_PROJECT
+
+
+# ------------------------------------------------------------------ router-logit steering
+def test_router_hook_adds_delta_only_where_the_app_is():
+    rng = np.random.default_rng(31)
+    T, E = 12, 8
+    logits = rng.standard_normal((T, E)).astype(np.float32)
+    delta = np.array([0, 1.5, -np.inf, 0, 0, np.inf, -2.0, 0], dtype=np.float32)
+    slots = np.array([0, -1, 1, 0, 2, 0, -1, 1, 0, 0, 5, 0], dtype=np.int32)
+    apps = {0: W.Router(delta), 1: W.Steer(bf(np.zeros(4)), 1.0), 2: W.Router(np.zeros(4, dtype=np.float32))}
+    w = W.Workload("r", 4, T, 10, bf(np.zeros((T, 4))), slots, apps, {}, n_slots_max=4)
+    out = O.apply_router_hook(w, logits)
+    for t in range(T):
+        hit = t < 10 and slots[t] == 0
+        want = logits[t].astype(np.float64) + (delta.astype(np.float64) if hit else 0.0)
+        assert np.array_equal(out[t], want), t            # other kinds, other widths, rows past T_live: untouched
+    assert out[0, 2] == -np.inf and out[0, 5] == np.inf    # forced out / forced in
+    # the hidden-state hook ignores router apps
+    r = O.apply_hook(w)
+    assert all(r.kind[t] == 0 for t in range(T) if slots[t] in (0, 2))
+    # gated
+    sc = np.where(np.arange(T) % 2 == 0, 1.0, -1.0).astype(np.float32)[:, None]
+    apps[0].gate = W.Gate(sc, 0, O.GATE_GE, 0.0)
+    out = O.apply_router_hook(w, logits)
+    assert np.array_equal(out[3], logits[3].astype(np.float64)) and out[8, 1] == np.float64(logits[8, 1]) + 1.5

@@ -1,7 +1,7 @@
 """Register a workload's apps with a hook context (any object with the binding's method names)."""
 from __future__ import annotations
 
-from .spec import KIND_PROBE, KIND_PROJECT, KIND_SAE, KIND_STEER, Workload
+from .spec import KIND_PROBE, KIND_PROJECT, KIND_ROUTER, KIND_SAE, KIND_STEER, Workload
 
 
 def make_context(mix_cls, w: Workload, flags: int = 0, **over):
@@ -25,6 +25,8 @@ def install(m, w: Workload):
             m.register_steer(s, a.v, a.alpha)
         elif a.kind == KIND_PROJECT:
             m.register_project(s, a.r, a.beta)
+        elif a.kind == KIND_ROUTER:
+            m.register_router(s, a.delta)
         elif a.kind == KIND_SAE:
             m.register_sae_app(s, a.group, a.edit_idx, a.edit_val, a.edit_mode, a.add_error)
         if getattr(a, "gate", None) is not None:

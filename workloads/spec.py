@@ -19,7 +19,7 @@ import numpy as np
 import torch
 
 # app kinds
-KIND_PROBE, KIND_STEER, KIND_SAE, KIND_PROJECT = 1, 2, 3, 4
+KIND_PROBE, KIND_STEER, KIND_SAE, KIND_PROJECT, KIND_ROUTER = 1, 2, 3, 4, 5
 # probe activations
 ACT_SIGMOID, ACT_SOFTMAX, ACT_NONE = 0, 1, 2
 # SAE activations
@@ -66,6 +66,13 @@ class Project:
     r: object                 # bf16 [d], used as given
     beta: float
     kind: int = KIND_PROJECT
+    gate: Optional[Gate] = None
+
+
+@dataclass
+class Router:
+    delta: object             # fp32 [n_experts], added to the router logits
+    kind: int = KIND_ROUTER
     gate: Optional[Gate] = None
 
 
@@ -141,6 +148,8 @@ def host(w: Workload, only_groups=None) -> Workload:
             apps[s] = Steer(bits(a.v), float(a.alpha), gate=g)
         elif a.kind == KIND_PROJECT:
             apps[s] = Project(bits(a.r), float(a.beta), gate=g)
+        elif a.kind == KIND_ROUTER:
+            apps[s] = Router(bits(a.delta), gate=g)
         else:
             apps[s] = SaeApp(a.group, a.edit_idx, a.edit_val, a.edit_mode, a.add_error, gate=g)
     groups = {
