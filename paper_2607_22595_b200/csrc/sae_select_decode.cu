@@ -137,30 +137,47 @@ __device__ void emit_topk(const unsigned long long* a, int k, int k_max, int p, 
   }
 }
 
-// Largest digit D with count(digit >= D) >= need, and the count of digits > D.  One warp.
+// Largest digit D with count(digit >= D) >= need, and the count of digits > D.  One warp, two
+// levels: each lane sums a run of n_bins / 32 bins (largest digits in lane 0) and a warp scan
+// finds the run where the running count reaches `need`; then the 32 lanes split that run.
 __device__ void find_digit(const int* hist, int n_bins, int need, int* s_out) {
   const int lane = threadIdx.x & 31;
-  const int per = n_bins / 32;
-  // lane L owns bins [n_bins - (L+1)*per, n_bins - L*per): lane 0 holds the largest digits
-  const int hi = n_bins - lane * per;
+  const int per = n_bins / 32;                  // 64 or 32: a multiple of 4
+  const int hi = n_bins - lane * per;           // this lane's run is [hi - per, hi)
   int sum = 0;
-  for (int b = hi - per; b < hi; ++b) sum += hist[b];
+  const int4* h4 = reinterpret_cast<const int4*>(hist + hi - per);
+  for (int i = 0; i < per / 4; ++i) {
+    const int4 v = h4[i];
+    sum += v.x + v.y + v.z + v.w;
+  }
   int incl = sum;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
     const int y = __shfl_up_sync(0xffffffffu, incl, o);
     if (lane >= o) incl += y;
   }
-  const int excl = incl - sum;                 // elements in bins above this lane's range
-  if (excl < need && incl >= need) {
-    int above = excl;
-    for (int b = hi - 1; b >= hi - per; --b) {
-      if (above + hist[b] >= need) {
-        s_out[0] = b;
-        s_out[1] = above;
-        break;
-      }
-      above += hist[b];
+  const int excl = incl - sum;                  // elements in bins above this lane's run
+  const unsigned hit = __ballot_sync(0xffffffffu, excl < need && incl >= need);
+  const int L = __ffs(hit) - 1;                 // exactly one lane (need <= total count)
+  const int run_hi = n_bins - L * per;
+  const int above_run = __shfl_sync(0xffffffffu, excl, L);
+  // level 2: lane l takes bins run_hi - 1 - l*w .. run_hi - (l+1)*w, w = per / 32 (2 or 1), descending
+  const int w = per / 32;
+  int c0 = hist[run_hi - 1 - lane * w], c1 = w == 2 ? hist[run_hi - 2 - lane * w] : 0;
+  int inc2 = c0 + c1;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, inc2, o);
+    if (lane >= o) inc2 += y;
+  }
+  const int before = above_run + inc2 - (c0 + c1);     // elements in bins above this lane's bins
+  if (before < need && before + c0 + c1 >= need) {
+    if (before + c0 >= need) {
+      s_out[0] = run_hi - 1 - lane * w;
+      s_out[1] = before;
+    } else {
+      s_out[0] = run_hi - 2 - lane * w;
+      s_out[1] = before + c0;
     }
   }
 }
