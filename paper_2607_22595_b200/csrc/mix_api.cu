@@ -65,6 +65,7 @@ void free_all(mix_ctx* c) {
   cudaFree(c->d_tmp_req); cudaFree(c->d_tmp_req_slot); cudaFree(c->d_panel); cudaFree(c->d_panel_row);
   cudaFree(c->d_mtile_group); cudaFree(c->d_row_group); cudaFree(c->d_route); cudaFree(c->d_z); cudaFree(c->d_topk_idx);
   cudaFree(c->d_topk_val); cudaFree(c->d_tmap_w); cudaFree(c->d_cand_val); cudaFree(c->d_cand_idx);
+  cudaFree(c->d_row_delta); cudaFree(c->d_edit_coef);
   cudaFree(c->d_cand_ninth); cudaFree(c->d_row_flag); cudaFree(c->d_mtile_flag); cudaFree(c->d_n_flagged);
   if (c->owned_b_eff)
     for (int g = 0; g < c->cfg.n_groups_max; ++g) cudaFree(c->owned_b_eff[g]);
@@ -167,6 +168,8 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
     ok = ok && dev_alloc(&c->d_topk_idx, P * (size_t)c->cfg.k_max) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_topk_val, P * (size_t)c->cfg.k_max) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_tmap_w, G) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_row_delta, P) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_edit_coef, P * (size_t)(cfg->r_max > 0 ? cfg->r_max : 1)) == cudaSuccess;
     if (!(cfg->flags & MIX_FLAG_ENCODE_SIMT)) {
       c->cand_tiles = (int)(cfg->d_sae_max / kTileN);
       const size_t nc = P * (size_t)c->cand_tiles;
@@ -514,7 +517,9 @@ int mix_apply(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream) 
       MIX_CUDA(c, launch_select(c, true, s));      // flagged TopK rows; active counts of the other sets
       MIX_CUDA(c, tap());
     }
-    MIX_CUDA(c, launch_decode(c, h, s));
+    MIX_CUDA(c, launch_decode(c, h, s));         // rows that replace the residual
+    MIX_CUDA(c, tap());
+    MIX_CUDA(c, launch_decode_delta(c, h, s));   // rows that keep the error term
     MIX_CUDA(c, tap());
     if (c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) {
       MIX_CUDA(c, launch_edit_only(c, h, T, s));
@@ -537,7 +542,7 @@ int mix_launches_per_apply(const mix_ctx* c) {
   if (!c) return 0;
   const int front = has_multiclass_stage(c) ? 2 : 1;
   if (c->cfg.n_groups_max == 0) return front;
-  return front + ((c->cfg.flags & MIX_FLAG_ENCODE_SIMT) ? 5 : 7) + ((c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) ? 1 : 0);
+  return front + ((c->cfg.flags & MIX_FLAG_ENCODE_SIMT) ? 6 : 8) + ((c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) ? 1 : 0);
 }
 
 int mix_get_status(mix_ctx* c, unsigned* bits, void* stream) {

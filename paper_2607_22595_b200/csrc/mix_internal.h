@@ -63,6 +63,13 @@ struct __align__(16) GroupEntry {
   const float* b_dec;
 };
 
+// What decode_kernel leaves for decode_delta_kernel about one packed row that keeps the error term.
+struct __align__(16) RowDelta {
+  int slot;                         // the row's slot, or -1: nothing to add (no effective edit, other kind of row)
+  int n_edit;
+  const __nv_bfloat16* W_dec;
+};
+
 // Result of the routing step for the SAE path (one instance in device memory).
 struct RouteState {
   int n_panel_rows;                 // rows of the packed panel in use (multiple of kTileM)
@@ -110,6 +117,8 @@ struct Ctx {
   int* d_row_group;         // [T_max] routing scratch: weight set of each token row or -1
   RouteState* d_route;
   float* d_z;               // [P, d_sae_max]
+  RowDelta* d_row_delta;    // [P]
+  float* d_edit_coef;       // [P, r_max] f'_j - f_j of each edit entry of the row's slot
   int* d_topk_idx;          // [P, k_max]
   float* d_topk_val;        // [P, k_max]
   float* d_cand_val;        // [P, cand_tiles, kCandPerTile] per-tile TopK candidates (fused epilogue)
@@ -147,7 +156,8 @@ cudaError_t launch_encode_simt(const Ctx* c, cudaStream_t s);
 cudaError_t launch_encode_tc(const Ctx* c, int mode, cudaStream_t s);   // 0: all tiles; 1: flagged row tiles -> Z
 cudaError_t launch_merge(const Ctx* c, cudaStream_t s);
 cudaError_t launch_select(const Ctx* c, bool flagged_only, cudaStream_t s);
-cudaError_t launch_decode(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s);
+cudaError_t launch_decode(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s);         // rows without the error term
+cudaError_t launch_decode_delta(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s);   // rows with it
 cudaError_t launch_edit_only(const Ctx* c, __nv_bfloat16* hidden, int T, cudaStream_t s);
 cudaError_t launch_compose_map(const Ctx* c, int T_live, int n_req, cudaStream_t s);
 cudaError_t launch_fold_bias(const __nv_bfloat16* W_enc, const float* b_enc, const float* b_dec, float* b_eff,

@@ -424,21 +424,26 @@ decode_kernel(__nv_bfloat16* __restrict__ hidden, int d, const float* __restrict
               const RouteState* __restrict__ rs, const AppEntry* __restrict__ apps,
               const GroupEntry* __restrict__ groups, const int* __restrict__ edit_idx,
               const float* __restrict__ edit_val, const unsigned char* __restrict__ edit_mode, int r_max, int k_max,
-              const int* __restrict__ ws_idx, const float* __restrict__ ws_val) {
+              const int* __restrict__ ws_idx, const float* __restrict__ ws_val,
+              RowDelta* __restrict__ row_delta, float* __restrict__ edit_coef) {
   __shared__ float s_coef[kDecList];
   __shared__ int s_feat[kDecList];
   __shared__ float s_fnew[kMaxEdits];
   __shared__ int s_eidx[kMaxEdits];
   __shared__ int s_alive[kMaxEdits];
+  __shared__ float s_fold[kMaxEdits];
   __shared__ int s_any, s_n;
   const int p = blockIdx.x;
+  const int tid = threadIdx.x;
   if (p >= rs->n_panel_rows) return;
   const int t = panel_row[p];
-  if (t < 0) return;
+  if (t < 0) {
+    if (tid == 0) row_delta[p].slot = -1;             // padding row of a tile
+    return;
+  }
   const int slot = token_slot[t];
   const AppEntry app = apps[slot];
   const GroupEntry ge = groups[app.group];
-  const int tid = threadIdx.x;
   const int n_edit = app.n_edit;
   const int S = (int)ge.d_sae;
   const float* z = Z + (size_t)p * ldz;
@@ -447,8 +452,22 @@ decode_kernel(__nv_bfloat16* __restrict__ hidden, int d, const float* __restrict
   const int nvec = d >> 3;
 
   if (tid == 0) { s_any = 0; s_n = 0; }
-  if (tid < n_edit) s_eidx[tid] = edit_idx[slot * r_max + tid];
+  if (tid < n_edit) {
+    s_eidx[tid] = edit_idx[slot * r_max + tid];
+    s_fold[tid] = 0.f;
+  }
   __syncthreads();
+  if (ge.act == MIX_SAE_TOPK) {
+    // TopK: the value of a selected feature comes from the row's TopK list (the Z scratch is not
+    // written for TopK sets unless the row took the fallback selection); an unselected one is 0.
+    // The list is scanned element-parallel against the edit list.
+    for (int i = tid; i < ge.k; i += kDecThreads) {
+      const int id = K[i];
+      for (int e = 0; e < n_edit; ++e)
+        if (s_eidx[e] == id) s_fold[e] = fmaxf(Kv[i], 0.f);
+    }
+    __syncthreads();
+  }
   // edits: f_j before and after; a later entry for the same feature overrides an earlier one
   if (tid < n_edit) {
     const int j = s_eidx[tid];
@@ -461,49 +480,35 @@ decode_kernel(__nv_bfloat16* __restrict__ hidden, int d, const float* __restrict
       const float zj = z[j];
       f = zj > ge.theta[j] ? zj : 0.f;
     } else {
-      // TopK: the pre-activation of a selected feature comes from the row's TopK list (the Z
-      // scratch is not written for TopK sets unless the row took the fallback selection)
-      float zk = 0.f;
-      bool in = false;
-      for (int i = 0; i < ge.k; ++i)
-        if (K[i] == j) {
-          in = true;
-          zk = Kv[i];
-        }
-      f = in ? fmaxf(zk, 0.f) : 0.f;
+      f = s_fold[tid];
     }
     const float fnew = edit_mode[slot * r_max + tid] == MIX_EDIT_CLAMP ? edit_val[slot * r_max + tid] : 0.f;
     s_alive[tid] = alive;
     s_fnew[tid] = fnew;
     if (app.add_error) {
       const float delta = alive ? fnew - f : 0.f;
-      s_coef[tid] = delta;
-      s_feat[tid] = j;
+      edit_coef[(size_t)p * r_max + tid] = delta;
       if (delta != 0.f) s_any = 1;
     }
   }
   __syncthreads();
 
+  if (app.add_error) {
+    // the row keeps the error term: decode_delta_kernel adds the deltas, eight rows at a time.
+    // No effective edit: the row is left alone and stays bit-exact.
+    if (tid == 0) {
+      RowDelta rd;
+      rd.slot = s_any ? slot : -1;
+      rd.n_edit = n_edit;
+      rd.W_dec = ge.W_dec;
+      row_delta[p] = rd;
+    }
+    return;
+  }
+  if (tid == 0) row_delta[p].slot = -1;
   float acc[kDecU][8];
   uint4* hrow = reinterpret_cast<uint4*>(hidden + (size_t)t * d);
-  if (app.add_error) {
-    if (!s_any) return;                       // no effective edit: the row stays bit-exact
-#pragma unroll
-    for (int u = 0; u < kDecU; ++u) {
-      const int v = tid + u * kDecThreads;
-      if (v < nvec) {
-        const uint4 q = hrow[v];
-        const __nv_bfloat162* pp = reinterpret_cast<const __nv_bfloat162*>(&q);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float2 f2 = __bfloat1622float2(pp[i]);
-          acc[u][2 * i] = f2.x;
-          acc[u][2 * i + 1] = f2.y;
-        }
-      }
-    }
-    accumulate_list(acc, s_coef, s_feat, n_edit, ge.W_dec, d, nvec);
-  } else {
+  {
 #pragma unroll
     for (int u = 0; u < kDecU; ++u) {
       const int v = tid + u * kDecThreads;
@@ -565,6 +570,131 @@ decode_kernel(__nv_bfloat16* __restrict__ hidden, int d, const float* __restrict
       for (int i = 0; i < 4; ++i) pp[i] = __floats2bfloat162_rn(acc[u][2 * i], acc[u][2 * i + 1]);
       hrow[v] = q;
     }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// decode of rows with the error term: h' = h + sum over edited j of (f'_j - f_j) W_dec[j]
+// ---------------------------------------------------------------------------------------
+// A CTA owns kDdRows consecutive packed rows and a slice of 1024 columns.  Consecutive packed rows
+// usually belong to one request, i.e. one slot and one edit list, so every edited W_dec row is
+// loaded once per CTA and applied to all of its rows with per-row coefficients (f_j differs by
+// row): the gather's L2 traffic drops by up to kDdRows.  Rows of different slots in one CTA are
+// handled by listing the edits of every distinct slot, with zero coefficients for foreign rows.
+constexpr int kDdRows = 8;
+constexpr int kDdThreads = 128;
+constexpr int kDdBatch = 8;
+constexpr int kDdEntries = kDdRows * kMaxEdits;
+
+__device__ __forceinline__ void decode_delta_fma(float (&acc)[kDdRows][8], const float* coef, const uint4& q) {
+  const float4 c0 = *reinterpret_cast<const float4*>(coef);
+  const float4 c1 = *reinterpret_cast<const float4*>(coef + 4);
+  axpy8(acc[0], c0.x, q);
+  axpy8(acc[1], c0.y, q);
+  axpy8(acc[2], c0.z, q);
+  axpy8(acc[3], c0.w, q);
+  axpy8(acc[4], c1.x, q);
+  axpy8(acc[5], c1.y, q);
+  axpy8(acc[6], c1.z, q);
+  axpy8(acc[7], c1.w, q);
+}
+
+// decode_kernel has already left, per packed row, the slot (or -1 when there is nothing to add), the
+// decoder matrix and one coefficient f'_j - f_j per edit entry, so the chain of dependent loads here
+// is short: row records -> (residual rows, edit lists, coefficients) -> decoder rows -> store.
+__global__ void __launch_bounds__(kDdThreads, 4)
+decode_delta_kernel(__nv_bfloat16* __restrict__ hidden, int d, const int* __restrict__ panel_row,
+                    const RouteState* __restrict__ rs, const RowDelta* __restrict__ row_delta,
+                    const float* __restrict__ edit_coef, const int* __restrict__ edit_idx, int r_max) {
+  __shared__ __align__(16) float s_coef[kDdEntries + kDdBatch][kDdRows];
+  __shared__ const uint4* s_wrow[kDdEntries + kDdBatch];
+  __shared__ int s_t[kDdRows], s_slot[kDdRows], s_nedit[kDdRows];
+  __shared__ const __nv_bfloat16* s_wdec[kDdRows];
+  const int p0 = blockIdx.x * kDdRows;
+  const int tid = threadIdx.x;
+  const int n_rows = rs->n_panel_rows;
+  if (tid < kDdRows) {
+    const int p = p0 + tid;                              // in bounds: the panel capacity is a multiple of 128
+    const int t = panel_row[p];
+    const RowDelta rd = row_delta[p];
+    const bool on = p < n_rows && t >= 0 && rd.slot >= 0;
+    s_t[tid] = on ? t : -1;
+    s_slot[tid] = on ? rd.slot : -1;
+    s_nedit[tid] = rd.n_edit;
+    s_wdec[tid] = rd.W_dec;
+  }
+  if (p0 >= n_rows) return;
+  __syncthreads();
+  bool any = false;
+#pragma unroll
+  for (int r = 0; r < kDdRows; ++r) any = any || s_slot[r] >= 0;
+  if (!any) return;
+  const int v = blockIdx.y * kDdThreads + tid;          // this thread's 16-byte column vector
+  const bool in_cols = v < (d >> 3);
+  uint4 hraw[kDdRows];
+#pragma unroll
+  for (int r = 0; r < kDdRows; ++r) {
+    const int t = s_t[r];
+    hraw[r] = make_uint4(0u, 0u, 0u, 0u);
+    if (t >= 0 && in_cols) hraw[r] = reinterpret_cast<const uint4*>(hidden + (size_t)t * d)[v];
+  }
+  // entries: the edit lists of the distinct slots, one after the other; thread e of a slot fills
+  // entry e for all rows (the coefficient of a row of another slot is zero)
+  int n_entries = 0;                                    // CTA-uniform
+  for (int r = 0; r < kDdRows; ++r) {
+    const int slot = s_slot[r];
+    bool first = slot >= 0;
+    for (int r2 = 0; r2 < r; ++r2) first = first && s_slot[r2] != slot;
+    if (!first) continue;
+    const int n_edit = s_nedit[r];
+    if (tid < n_edit) {
+      const int j = edit_idx[slot * r_max + tid];
+      float c[kDdRows];
+#pragma unroll
+      for (int r2 = 0; r2 < kDdRows; ++r2)
+        c[r2] = s_slot[r2] == slot ? edit_coef[(size_t)(p0 + r2) * r_max + tid] : 0.f;
+#pragma unroll
+      for (int r2 = 0; r2 < kDdRows; ++r2) s_coef[n_entries + tid][r2] = c[r2];
+      s_wrow[n_entries + tid] = reinterpret_cast<const uint4*>(s_wdec[r] + (size_t)j * d);
+    }
+    n_entries += n_edit;
+  }
+  __syncthreads();
+  // pad to a whole batch: repeats of the last decoder row with zero coefficients
+  if (tid < kDdBatch) {
+    s_wrow[n_entries + tid] = s_wrow[n_entries - 1];
+#pragma unroll
+    for (int r2 = 0; r2 < kDdRows; ++r2) s_coef[n_entries + tid][r2] = 0.f;
+  }
+  __syncthreads();
+  if (!in_cols) return;
+  float acc[kDdRows][8];
+#pragma unroll
+  for (int r = 0; r < kDdRows; ++r) {
+    const __nv_bfloat162* pp = reinterpret_cast<const __nv_bfloat162*>(&hraw[r]);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 f2 = __bfloat1622float2(pp[i]);
+      acc[r][2 * i] = f2.x;
+      acc[r][2 * i + 1] = f2.y;
+    }
+  }
+  // kDdBatch decoder rows in flight per thread: the loop is bound by load latency, not arithmetic
+  for (int e0 = 0; e0 < n_entries; e0 += kDdBatch) {
+    uint4 q[kDdBatch];
+#pragma unroll
+    for (int u = 0; u < kDdBatch; ++u) q[u] = __ldg(s_wrow[e0 + u] + v);
+#pragma unroll
+    for (int u = 0; u < kDdBatch; ++u) decode_delta_fma(acc, &s_coef[e0 + u][0], q[u]);
+  }
+#pragma unroll
+  for (int r = 0; r < kDdRows; ++r) {
+    if (s_slot[r] < 0) continue;
+    uint4 o;
+    __nv_bfloat162* pp = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) pp[i] = __floats2bfloat162_rn(acc[r][2 * i], acc[r][2 * i + 1]);
+    reinterpret_cast<uint4*>(hidden + (size_t)s_t[r] * d)[v] = o;
   }
 }
 
@@ -706,11 +836,23 @@ cudaError_t launch_edit_only(const Ctx* c, __nv_bfloat16* hidden, int T, cudaStr
   return cudaGetLastError();
 }
 
+// Two kernels: decode_kernel (one CTA per row) rebuilds the rows whose app replaces the residual and, for
+// the rows that keep the error term, only works out the coefficients of their edits; decode_delta_kernel
+// then adds those rows' deltas, eight rows per CTA.
 cudaError_t launch_decode(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s) {
   decode_kernel<<<c->panel_rows_cap, kDecThreads, 0, s>>>(hidden, c->cfg.d_model, c->d_z, c->cfg.d_sae_max,
                                                           c->d_panel_row, c->d_token_slot, c->d_route, c->d_apps,
                                                           c->d_groups, c->d_edit_idx, c->d_edit_val, c->d_edit_mode,
-                                                          c->cfg.r_max, c->cfg.k_max, c->d_topk_idx, c->d_topk_val);
+                                                          c->cfg.r_max, c->cfg.k_max, c->d_topk_idx, c->d_topk_val,
+                                                          c->d_row_delta, c->d_edit_coef);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_decode_delta(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s) {
+  dim3 grid((unsigned)((c->panel_rows_cap + kDdRows - 1) / kDdRows),
+            (unsigned)((c->cfg.d_model / 8 + kDdThreads - 1) / kDdThreads));
+  decode_delta_kernel<<<grid, kDdThreads, 0, s>>>(hidden, c->cfg.d_model, c->d_panel_row, c->d_route, c->d_row_delta,
+                                                  c->d_edit_coef, c->d_edit_idx, c->cfg.r_max);
   return cudaGetLastError();
 }
 

@@ -37,7 +37,9 @@ constexpr size_t kOffRoute = kOffEditMode + align256(kMaxEdits);
 constexpr size_t kOffPanelRow = kOffRoute + align256(sizeof(RouteState));
 constexpr size_t kOffMtileGroup = kOffPanelRow + align256(kStaticRows * sizeof(int));
 constexpr size_t kOffRowGroup = kOffMtileGroup + 256;
-constexpr size_t kOffTopkIdx = kOffRowGroup + align256(kStaticRows * sizeof(int));
+constexpr size_t kOffRowDelta = kOffRowGroup + align256(kStaticRows * sizeof(int));
+constexpr size_t kOffEditCoef = kOffRowDelta + align256(kStaticRows * sizeof(RowDelta));
+constexpr size_t kOffTopkIdx = kOffEditCoef + align256((size_t)kStaticRows * kMaxEdits * sizeof(float));
 constexpr size_t kOffTopkVal = kOffTopkIdx + align256((size_t)kStaticRows * kStaticK * sizeof(int));
 constexpr size_t kOffPanel = kOffTopkVal + align256((size_t)kStaticRows * kStaticK * sizeof(float));
 constexpr size_t kOffZ = kOffPanel + align256((size_t)kStaticRows * kStaticD * sizeof(__nv_bfloat16));
@@ -132,6 +134,8 @@ extern "C" int mix_sae_apply_static(void* hidden, int n_rows, int d_model, const
   c.d_panel_row = reinterpret_cast<int*>(base + kOffPanelRow);
   c.d_mtile_group = reinterpret_cast<int*>(base + kOffMtileGroup);
   c.d_row_group = reinterpret_cast<int*>(base + kOffRowGroup);
+  c.d_row_delta = reinterpret_cast<RowDelta*>(base + kOffRowDelta);
+  c.d_edit_coef = reinterpret_cast<float*>(base + kOffEditCoef);
   c.d_topk_idx = reinterpret_cast<int*>(base + kOffTopkIdx);
   c.d_topk_val = reinterpret_cast<float*>(base + kOffTopkVal);
   c.d_panel = reinterpret_cast<__nv_bfloat16*>(base + kOffPanel);
@@ -178,6 +182,7 @@ extern "C" int mix_sae_apply_static(void* hidden, int n_rows, int d_model, const
   if (e == cudaSuccess) e = launch_encode_simt(&c, s);
   if (e == cudaSuccess) e = launch_select(&c, false, s);
   if (e == cudaSuccess) e = launch_decode(&c, h, s);
+  if (e == cudaSuccess) e = launch_decode_delta(&c, h, s);
   if (e != cudaSuccess) return fail(errbuf, errbuf_len, MIX_ERR_CUDA, "CUDA error %lld while enqueuing the static SAE call", (long long)e);
   return MIX_OK;
 }

@@ -233,6 +233,34 @@ def test_sae_modes_with_b_dec_and_centering(act, add_error):
     check_parity(W.host(w), out)
 
 
+@pytest.mark.parametrize("act", [W.SAE_JUMPRELU, W.SAE_TOPK])
+def test_interleaved_slots_in_one_weight_set(act):
+    # consecutive packed rows alternate between five slots of ONE weight set: different edit lists
+    # (one with a repeated feature, one empty, one that clamps to the value it already has), rows that
+    # keep the error term next to rows that replace the residual, and unhooked rows in between
+    d, S, k, T = 320, 1024, 16, 203
+    g = torch.Generator(device=DEV); g.manual_seed(11)
+    sae = W.make_sae_weights(g, DEV, d, S, act, k=k, theta_range=(0.05, 0.3), b_enc_mean=-1.0)
+    hidden = torch.randn((T, d), generator=g, device=DEV, dtype=torch.float32).to(torch.bfloat16)
+    def app(idx, val, mode, err):
+        return W.SaeApp(0, np.asarray(idx, np.int32), np.asarray(val, np.float32), np.asarray(mode, np.uint8), err)
+    apps = {0: app([3, 700, 3], [2.0, 0.0, 5.0], [0, 1, 0], True),
+            1: app([], [], [], True),
+            2: app([9, 10, 11, 12, 1000], [1.0, 1.5, 0.0, 2.5, 4.0], [0, 0, 1, 0, 0], True),
+            3: app([44], [3.0], [0], False),
+            4: app([1023], [0.0], [1], True)}            # ablating a feature that is almost never active
+    slot = np.array([(t % 6) - 1 for t in range(T)], dtype=np.int32)   # -1 = unhooked
+    w = W.Workload("interleaved", d, T, T, hidden, slot, apps, {0: sae}, n_slots_max=5, n_groups_max=1, C_max=1,
+                   k_max=k, r_max=5, d_sae_max=S)
+    out = run_gpu(w, graph=True)
+    st = check_parity(W.host(w), out)
+    assert st["rows"] == T
+    h0 = W.bits(w.hidden)
+    for t in range(T):
+        if slot[t] in (-1, 1):
+            assert np.array_equal(out["hidden"][t], h0[t])            # unhooked / no edit: bit-exact
+
+
 def test_no_edit_with_error_leaves_rows_bit_exact():
     w = _one_sae_workload(128, 512, W.SAE_TOPK, 8, 40, True, ([], [], []))
     out = run_gpu(w)
@@ -385,7 +413,7 @@ def test_api_error_codes():
     with pytest.raises(mixlib.MixError) as e:
         m.set_slot_map(np.zeros(9, dtype=np.int32))                       # T_live > T_max
     assert e.value.code == -2
-    assert m.launches_per_apply() == 8
+    assert m.launches_per_apply() == 9
     m.destroy()
 
 
