@@ -307,6 +307,41 @@ def run_replay(peaks, mixlib, n_replays):
                       "bound_ms": float(a[a[:, 3].argmax(), 4])}}
 
 
+def extras_conditional(w, mixlib):
+    """mix_apply vs mix_apply_conditional on one SAE-carrying context, with and without SAE rows live:
+    graph replay, hidden state refreshed before every replay, best of 7."""
+    sae_slots = [s for s, a in w.apps.items() if a.kind == W.KIND_SAE]
+    full = np.asarray(w.token_slot, dtype=np.int32)
+    no_sae = np.where(np.isin(full, sae_slots), -1, full).astype(np.int32)
+    scores = torch.zeros((w.T_max, max(w.C_max, 1)), dtype=torch.float32, device="cuda")
+    out = {"workload": w.name, "unit": "ms per replayed call",
+           "rows_live": {"all_apps": int((full >= 0).sum()), "sae_rows_removed": int((no_sae >= 0).sum())}}
+    for label, cond in (("mix_apply", False), ("mix_apply_conditional", True)):
+        m = W.make_context(mixlib.Mix, w, flags=SAE_FLAGS)
+        h = w.hidden.clone()
+        s = torch.cuda.Stream(); s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s):
+            m.apply(h, scores, stream=s)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                (m.apply_conditional if cond else m.apply)(h, scores, stream=s)
+        torch.cuda.current_stream().wait_stream(s)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        res = {}
+        for name, slot_map in (("sae_rows_live", full), ("no_sae_row_live", no_sae)):
+            m.set_slot_map(slot_map)
+            best = 1e30
+            for _ in range(7):
+                h.copy_(w.hidden)
+                e0.record(); g.replay(); e1.record(); torch.cuda.synchronize()
+                best = min(best, e0.elapsed_time(e1))
+            res[name] = best
+        res["status"] = m.get_status()
+        out[label] = res
+        m.destroy()
+    return out
+
+
 def run_workload(args):
     """--workload X: one of the other configurations alone (not the contract line)."""
     import paper_2607_22595_b200 as mixlib
@@ -327,6 +362,10 @@ def run_workload(args):
     elif name == "mixed_small":   # profiling case for the tensor-bound regime
         out = extras_sae("mixed_small (d=5120, d_sae=8192, T=4096)",
                          W.make_mixed("cuda", T=4096, d_sae=8192, R=32), peaks, mixlib)
+    elif name == "conditional":   # the SAE chain as a graph IF node (config 3's context)
+        out = extras_conditional(W.make_mixed("cuda"), mixlib)
+    elif name == "conditional_small":
+        out = extras_conditional(W.make_mixed("cuda", T=4096, d_sae=8192, R=32), mixlib)
     elif name == "replay":
         out = run_replay(peaks, mixlib, args.steps or 200)
     else:
@@ -561,7 +600,7 @@ def main():
     ap.add_argument("--no-retile", action="store_true",
                     help="SAE contexts stream W_enc as registered instead of a tile-contiguous copy (MIX_FLAG_RETILE_W_ENC)")
     ap.add_argument("--workload", default="decode",
-                    help="decode (the contract line) | sweep | sae_heavy | sae_small | mixed | mixed_small | replay")
+                    help="decode (the contract line) | sweep | sae_heavy | sae_small | mixed | mixed_small | conditional | conditional_small | replay")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     args = ap.parse_args()
     if args.no_retile:

@@ -255,6 +255,20 @@ int mix_set_feature_out(mix_ctx* ctx, int* topk_idx, float* topk_val, int* n_act
    Errors: INVALID_ARG (NULL hidden, misaligned), OUT_OF_RANGE (T), CUDA (launch failure). */
 int mix_apply(mix_ctx* ctx, void* hidden, int T, float* scores_out, void* stream);
 
+/* mix_apply() with the SAE chain under a device-side predicate (implementation section of the
+   paper, paragraph "Graph-level toggling and continuous batching": for true data-dependent
+   control flow an upstream GPU computation decides whether a downstream intervention body
+   executes, as with CUDA conditional nodes, with no CPU in the loop).  `stream` MUST be capturing: the call adds to
+   the graph being captured the probe / steering kernels and the route kernel as mix_apply() does,
+   then one conditional IF node whose body holds the rest of the SAE chain (pack, encode,
+   selection, decode); the route kernel sets the node's condition to (SAE rows routed > 0).  A
+   replay with no SAE row live therefore launches none of the body's kernels, instead of eight
+   kernels that each find nothing to do.  Results are identical to mix_apply()'s.  The capture
+   continues after the node; work captured later on `stream` depends on it.  A context without
+   weight sets behaves exactly like mix_apply() (and then `stream` need not be capturing).
+   Errors: as mix_apply(), plus INVALID_ARG (`stream` is not capturing; stage events are on). */
+int mix_apply_conditional(mix_ctx* ctx, void* hidden, int T, float* scores_out, void* stream);
+
 /* The hook on a different target tensor: router logits (device fp32 [T_max, n_experts], modified in
    place).  Rows whose slot holds a MIX_ROUTER app with the same n_experts (and an open gate, if it
    has one) get logits[t, :] += delta; every other row is neither read nor written.  Uses the same

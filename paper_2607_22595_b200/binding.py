@@ -29,7 +29,7 @@ MIX_FLAG_SAE_EDIT_ONLY = 8
 EXPORTS = [
     "mix_create", "mix_destroy", "mix_last_error", "mix_register_sae_weights", "mix_unregister_sae_weights",
     "mix_register_app", "mix_unregister_app", "mix_set_gate", "mix_update_steer_alpha", "mix_update_sae_edits",
-    "mix_set_slot_map", "mix_set_request_map", "mix_set_feature_out", "mix_apply", "mix_apply_router", "mix_get_status",
+    "mix_set_slot_map", "mix_set_request_map", "mix_set_feature_out", "mix_apply", "mix_apply_conditional", "mix_apply_router", "mix_get_status",
     "mix_launches_per_apply", "mix_set_stage_events", "mix_debug_workspace", "mix_sae_apply_static",
 ]
 
@@ -97,6 +97,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.mix_set_request_map.argtypes = [vp, vp, ci, vp, ci, ci, vp]
     lib.mix_set_feature_out.argtypes = [vp, vp, vp, vp]
     lib.mix_apply.argtypes = [vp, vp, ci, vp, vp]
+    lib.mix_apply_conditional.argtypes = [vp, vp, ci, vp, vp]
     lib.mix_apply_router.argtypes = [vp, vp, ci, ci, vp]
     lib.mix_get_status.argtypes = [vp, C.POINTER(C.c_uint), vp]
     lib.mix_launches_per_apply.argtypes = [vp]
@@ -262,6 +263,13 @@ class Mix:
         assert hidden.dtype == torch.bfloat16 and hidden.is_cuda and hidden.is_contiguous()
         T = hidden.shape[0] if T is None else T
         self._check(self.lib.mix_apply(self.ctx, hidden.data_ptr(), int(T), _ptr(scores_out), _stream(stream)))
+
+    def apply_conditional(self, hidden, scores_out=None, T=None, stream=None):
+        """As apply(), inside a stream capture only: the SAE chain becomes the body of a graph IF node."""
+        assert hidden.dtype == torch.bfloat16 and hidden.is_cuda and hidden.is_contiguous()
+        T = hidden.shape[0] if T is None else T
+        self._check(self.lib.mix_apply_conditional(self.ctx, hidden.data_ptr(), int(T), _ptr(scores_out),
+                                                   _stream(stream)))
 
     def get_status(self, stream=None) -> int:
         bits = C.c_uint(0)

@@ -76,6 +76,7 @@ void free_all(mix_ctx* c) {
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->ev_join) cudaEventDestroy(c->ev_join);
   if (c->side_stream) cudaStreamDestroy(c->side_stream);
+  if (c->body_stream) cudaStreamDestroy(c->body_stream);
 }
 
 int check_slot(mix_ctx* c, int slot) {
@@ -203,6 +204,7 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
   }
   if (e == cudaSuccess && G > 0) {
     e = cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->body_stream, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming);
   }
@@ -468,12 +470,79 @@ int mix_set_feature_out(mix_ctx* c, int* topk_idx, float* topk_val, int* n_activ
   return MIX_OK;
 }
 
-int mix_apply(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream) {
+extern "C++" {
+namespace {
+
+// The SAE chain after routing: pack ... decode.  `tap` records a stage event after each launch.
+template <class Tap>
+int sae_chain(mix_ctx* c, __nv_bfloat16* h, cudaStream_t s, Tap&& tap) {
+  MIX_CUDA(c, launch_pack(c, h, s));
+  MIX_CUDA(c, tap());
+  if (c->cfg.flags & MIX_FLAG_ENCODE_SIMT) {
+    MIX_CUDA(c, launch_encode_simt(c, s));
+    MIX_CUDA(c, tap());
+    MIX_CUDA(c, launch_select(c, false, s));
+    MIX_CUDA(c, tap());
+  } else {
+    MIX_CUDA(c, launch_encode_tc(c, 0, s));      // TopK sets -> candidates, other sets -> Z
+    MIX_CUDA(c, tap());
+    MIX_CUDA(c, launch_merge(c, s));             // exact TopK from candidates, or a flag
+    MIX_CUDA(c, tap());
+    MIX_CUDA(c, launch_encode_tc(c, 1, s));      // flagged row tiles -> Z (returns at once if none)
+    MIX_CUDA(c, tap());
+    MIX_CUDA(c, launch_select(c, true, s));      // flagged TopK rows; active counts of the other sets
+    MIX_CUDA(c, tap());
+  }
+  MIX_CUDA(c, launch_decode(c, h, s));           // rows that replace the residual; edit coefficients
+  MIX_CUDA(c, tap());
+  MIX_CUDA(c, launch_decode_delta(c, h, s));     // rows that keep the error term
+  MIX_CUDA(c, tap());
+  return MIX_OK;
+}
+
+// Puts the SAE chain into the body of an IF node of the graph that `s` is capturing; the node
+// depends on whatever `s` has captured so far (the route kernel, which sets the condition), and
+// the capture continues after it.
+int sae_chain_conditional(mix_ctx* c, __nv_bfloat16* h, cudaStream_t s, cudaGraph_t graph,
+                          cudaGraphConditionalHandle handle) {
+  cudaStreamCaptureStatus st;
+  const cudaGraphNode_t* deps = nullptr;
+  size_t n_deps = 0;
+  MIX_CUDA(c, cudaStreamGetCaptureInfo_v2(s, &st, nullptr, nullptr, &deps, &n_deps));
+  cudaGraphNodeParams np = {cudaGraphNodeTypeConditional};   // zero-initialises the rest
+  np.conditional.handle = handle;
+  np.conditional.type = cudaGraphCondTypeIf;
+  np.conditional.size = 1;
+  cudaGraphNode_t node;
+  MIX_CUDA(c, cudaGraphAddNode(&node, graph, deps, n_deps, &np));
+  cudaGraph_t body = np.conditional.phGraph_out[0];
+  MIX_CUDA(c, cudaStreamBeginCaptureToGraph(c->body_stream, body, nullptr, nullptr, 0, cudaStreamCaptureModeRelaxed));
+  const int rc = sae_chain(c, h, c->body_stream, [] { return cudaSuccess; });
+  cudaGraph_t ended = nullptr;
+  const cudaError_t e_end = cudaStreamEndCapture(c->body_stream, &ended);
+  if (rc != MIX_OK) return rc;
+  MIX_CUDA(c, e_end);
+  MIX_CUDA(c, cudaStreamUpdateCaptureDependencies(s, &node, 1, cudaStreamSetCaptureDependencies));
+  return MIX_OK;
+}
+
+int apply_impl(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream, bool conditional) {
   if (!c) return MIX_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (!hidden || !aligned16(hidden)) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "hidden is NULL or not 16-byte aligned");
   if (T < 0 || T > c->cfg.T_max) MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "T %d outside [0, T_max=%d]", T, c->cfg.T_max);
   __nv_bfloat16* h = static_cast<__nv_bfloat16*>(hidden);
+  cudaGraph_t graph = nullptr;
+  cudaGraphConditionalHandle handle = 0;
+  conditional = conditional && c->cfg.n_groups_max > 0;     // without weight sets there is no SAE chain to skip
+  if (conditional) {
+    cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+    MIX_CUDA(c, cudaStreamGetCaptureInfo_v2(s, &st, nullptr, &graph, nullptr, nullptr));
+    if (st != cudaStreamCaptureStatusActive || !graph)
+      MIX_FAIL(c, MIX_ERR_INVALID_ARG, "mix_apply_conditional needs a stream that is being captured (status %d)", (int)st);
+    if (c->stage_events_on) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "stage events cannot be recorded inside a conditional body");
+    MIX_CUDA(c, cudaGraphConditionalHandleCreate(&handle, graph, 0, cudaGraphCondAssignDefault));
+  }
   int stage = 0;
   auto tap = [&]() -> cudaError_t {
     return c->stage_events_on ? cudaEventRecord(c->stage_events[stage++], s) : cudaSuccess;
@@ -498,29 +567,10 @@ int mix_apply(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream) 
   }
   if (fork) MIX_CUDA(c, cudaEventRecord(c->ev_join, ps));
   if (c->cfg.n_groups_max > 0) {
-    MIX_CUDA(c, launch_route(c, T, s));
+    MIX_CUDA(c, launch_route(c, T, s, handle, conditional ? 1 : 0));
     MIX_CUDA(c, tap());
-    MIX_CUDA(c, launch_pack(c, h, s));
-    MIX_CUDA(c, tap());
-    if (c->cfg.flags & MIX_FLAG_ENCODE_SIMT) {
-      MIX_CUDA(c, launch_encode_simt(c, s));
-      MIX_CUDA(c, tap());
-      MIX_CUDA(c, launch_select(c, false, s));
-      MIX_CUDA(c, tap());
-    } else {
-      MIX_CUDA(c, launch_encode_tc(c, 0, s));      // TopK sets -> candidates, other sets -> Z
-      MIX_CUDA(c, tap());
-      MIX_CUDA(c, launch_merge(c, s));             // exact TopK from candidates, or a flag
-      MIX_CUDA(c, tap());
-      MIX_CUDA(c, launch_encode_tc(c, 1, s));      // flagged row tiles -> Z (returns at once if none)
-      MIX_CUDA(c, tap());
-      MIX_CUDA(c, launch_select(c, true, s));      // flagged TopK rows; active counts of the other sets
-      MIX_CUDA(c, tap());
-    }
-    MIX_CUDA(c, launch_decode(c, h, s));         // rows that replace the residual
-    MIX_CUDA(c, tap());
-    MIX_CUDA(c, launch_decode_delta(c, h, s));   // rows that keep the error term
-    MIX_CUDA(c, tap());
+    const int rc = conditional ? sae_chain_conditional(c, h, s, graph, handle) : sae_chain(c, h, s, tap);
+    if (rc != MIX_OK) return rc;
     if (c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) {
       MIX_CUDA(c, launch_edit_only(c, h, T, s));
       MIX_CUDA(c, tap());
@@ -528,6 +578,17 @@ int mix_apply(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream) 
   }
   if (fork) MIX_CUDA(c, cudaStreamWaitEvent(s, c->ev_join, 0));
   return MIX_OK;
+}
+
+}  // namespace
+}  // extern "C++"
+
+int mix_apply(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream) {
+  return apply_impl(c, hidden, T, scores_out, stream, false);
+}
+
+int mix_apply_conditional(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream) {
+  return apply_impl(c, hidden, T, scores_out, stream, true);
 }
 
 int mix_apply_router(mix_ctx* c, float* logits, int n_experts, int T, void* stream) {

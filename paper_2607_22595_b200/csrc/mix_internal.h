@@ -133,6 +133,7 @@ struct Ctx {
 
   // probe/steer kernels run beside the SAE chain on this stream (created with the context)
   cudaStream_t side_stream;
+  cudaStream_t body_stream;   // used only to record the body of a conditional node (mix_apply_conditional)
   cudaEvent_t ev_fork, ev_join;
 
   // profiling taps
@@ -150,7 +151,8 @@ cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float
 cudaError_t launch_probe_multiclass(const Ctx* c, const __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s);
 bool has_multiclass_stage(const Ctx* c);   // large batches with multi-class probes get a kernel of their own
 cudaError_t launch_router(const Ctx* c, float* logits, int n_experts, int T, cudaStream_t s);
-cudaError_t launch_route(const Ctx* c, int T, cudaStream_t s);
+// cond/use_cond: graph-conditional handle the kernel sets to (SAE rows routed > 0); plain calls pass 0, 0
+cudaError_t launch_route(const Ctx* c, int T, cudaStream_t s, unsigned long long cond = 0, int use_cond = 0);
 cudaError_t launch_pack(const Ctx* c, const __nv_bfloat16* hidden, cudaStream_t s);
 cudaError_t launch_encode_simt(const Ctx* c, cudaStream_t s);
 cudaError_t launch_encode_tc(const Ctx* c, int mode, cudaStream_t s);   // 0: all tiles; 1: flagged row tiles -> Z

@@ -567,7 +567,8 @@ route_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_
              const GroupEntry* __restrict__ groups, int n_groups,
              int* __restrict__ panel_row, int panel_cap, int* __restrict__ mtile_group, RouteState* __restrict__ rs,
              unsigned* __restrict__ status, int* __restrict__ row_flag, int* __restrict__ mtile_flag,
-             int* __restrict__ n_flagged, int* __restrict__ row_group, int edit_only) {
+             int* __restrict__ n_flagged, int* __restrict__ row_group, int edit_only,
+             cudaGraphConditionalHandle cond, int use_cond) {
   extern __shared__ int s_cnt[];                      // [n_chunks * kRouteWarps][n_groups]
   __shared__ int s_total[kMaxGroups], s_base[kMaxGroups + 1];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -677,6 +678,8 @@ route_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_
     rs->n_sae_rows = rows;
     rs->total_tiles = tiles;
     rs->n_topk_rows = topk_rows;
+    // graph-conditional form: the SAE chain sits in the body of an IF node that runs only when a row needs it
+    if (use_cond) cudaGraphSetConditional(cond, rows > 0 ? 1u : 0u);
   }
   __syncthreads();
   // phase C: stable scatter
@@ -789,14 +792,15 @@ cudaError_t launch_router(const Ctx* c, float* logits, int n_experts, int T, cud
   return cudaGetLastError();
 }
 
-cudaError_t launch_route(const Ctx* c, int T, cudaStream_t s) {
+cudaError_t launch_route(const Ctx* c, int T, cudaStream_t s, unsigned long long cond, int use_cond) {
   const int n_chunks = (c->cfg.T_max + kRouteThreads - 1) / kRouteThreads;
   const size_t smem = (size_t)n_chunks * kRouteWarps * c->cfg.n_groups_max * sizeof(int);
   route_kernel<<<1, kRouteThreads, smem, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates, c->cfg.n_slots_max,
                                               c->d_groups, c->cfg.n_groups_max, c->d_panel_row, c->panel_rows_cap,
                                               c->d_mtile_group, c->d_route, c->d_status, c->d_row_flag,
                                               c->d_mtile_flag, c->d_n_flagged, c->d_row_group,
-                                              (c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) ? 1 : 0);
+                                              (c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) ? 1 : 0,
+                                              static_cast<cudaGraphConditionalHandle>(cond), use_cond);
   return cudaGetLastError();
 }
 

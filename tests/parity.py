@@ -21,7 +21,7 @@ CANARY_F32 = np.uint32(0x7FC0DEAD)          # a NaN payload nobody computes
 CANARY_I32 = np.int32(-559038737)
 
 
-def run_gpu(w, flags=0, graph=False, feature_out=True, hidden=None, mix=None, replays=1):
+def run_gpu(w, flags=0, graph=False, feature_out=True, hidden=None, mix=None, replays=1, conditional=False):
     """Apply the hook to workload `w` (tensors on cuda).  Returns numpy outputs."""
     import os
     import paper_2607_22595_b200 as mixlib
@@ -46,7 +46,7 @@ def run_gpu(w, flags=0, graph=False, feature_out=True, hidden=None, mix=None, re
             h_static.copy_(h)
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=s):
-                m.apply(h_static, scores, stream=s)
+                (m.apply_conditional if conditional else m.apply)(h_static, scores, stream=s)
         torch.cuda.current_stream().wait_stream(s)
         for _ in range(replays):
             h_static.copy_(h)
