@@ -27,7 +27,7 @@ routines, algebraic invariants).  Nothing is "parity unpinned".
 from __future__ import annotations
 
 from dataclasses import dataclass, field
-from typing import Dict, Iterable, Optional
+from typing import Dict, Iterable, List, Optional
 
 import numpy as np
 
@@ -306,6 +306,96 @@ def apply_hook(w, rows: Optional[Iterable[int]] = None, keep_z: bool = False,
                 res.topk[t] = K
             if keep_z:
                 res.z[t] = Z[n].copy()
+    return res
+
+
+# ---------------------------------------------------------------------------
+# several apps on one row  (composition model: every app contributes its own hook functions and
+# state and the runtime applies the active ones at the hook; "All Apps Combined" in the evaluation)
+# ---------------------------------------------------------------------------
+MAX_CHAIN = 4
+
+
+def chain_slots(w, s: int) -> List[int]:
+    """Slots applied, in order, to a row whose token slot is s: s, chains[s], chains[chains[s]], ...
+    (at most MAX_CHAIN of them; the walk stops at a slot without a link or without an app)."""
+    out: List[int] = []
+    chains = getattr(w, "chains", None) or {}
+    while 0 <= s < w.n_slots_max and s in w.apps and len(out) < MAX_CHAIN:
+        out.append(s)
+        if s not in chains:
+            break
+        s = int(chains[s])
+    return out
+
+
+@dataclass
+class ChainResult:
+    rows: np.ndarray
+    out_bits: Dict[int, np.ndarray] = field(default_factory=dict)   # bf16 bits of the row after the last app
+    y: Dict[int, np.ndarray] = field(default_factory=dict)          # float64 value the last write produced
+    modified: Dict[int, bool] = field(default_factory=dict)
+    scores: Dict[int, Dict[int, float]] = field(default_factory=dict)   # row -> {column: score}
+    topk: Dict[int, np.ndarray] = field(default_factory=dict)
+    n_active: Dict[int, int] = field(default_factory=dict)
+    applied: Dict[int, List[int]] = field(default_factory=dict)     # slots whose app ran on the row
+
+
+def apply_chain_hook(w, rows: Optional[Iterable[int]] = None,
+                     topk_override: Optional[Dict[int, np.ndarray]] = None) -> ChainResult:
+    """The hook with slot chains.  For row t the apps of chain_slots(w, token_slot[t]) are applied one
+    after the other; each sees the row as the previous one left it, rounded to bf16 (exactly what
+    separate hook calls on the bf16 residual stream would see).  Every app's gate is evaluated on its
+    own: a closed gate skips that app only.  The probes of a chain write side by side: a probe's
+    first column is the total class count of the chain's earlier probes (skipped ones included, so
+    the layout does not depend on the data).  Router apps do not act on the hidden state."""
+    T = w.T_max
+    rows = np.arange(T) if rows is None else np.unique(np.asarray(list(rows), dtype=np.int64))
+    res = ChainResult(rows=rows)
+    for t in rows:
+        t = int(t)
+        s = int(w.token_slot[t]) if t < w.T_live else -1
+        cur = w.hidden[t].copy()
+        res.modified[t] = False
+        res.scores[t] = {}
+        res.applied[t] = []
+        res.y[t] = bf16_to_f64(cur)
+        col = 0
+        for sl in chain_slots(w, s):
+            app = w.apps[sl]
+            n_cols = int(np.asarray(app.W).shape[0]) if app.kind == KIND_PROBE else 0
+            first_col, col = col, col + n_cols
+            if app.kind == KIND_SAE and app.group not in w.groups:
+                continue
+            if getattr(app, "gate", None) is not None and not gate_open(app.gate, t):
+                continue
+            h = bf16_to_f64(cur)
+            if app.kind == KIND_PROBE:
+                sc = probe_scores(h, bf16_to_f64(app.W), app.b, app.act)
+                for c in range(n_cols):
+                    res.scores[t][first_col + c] = float(sc[c])
+            elif app.kind == KIND_STEER:
+                y = steer(h, bf16_to_f64(app.v), app.alpha)
+            elif app.kind == KIND_PROJECT:
+                y = project(h, bf16_to_f64(app.r), app.beta)
+            elif app.kind == KIND_SAE:
+                sae = w.groups[app.group]
+                z = sae_preact(h[None, :], sae.W_enc, sae.b_enc, sae.b_dec, sae.center_input)[0]
+                Ko = None if topk_override is None else topk_override.get(t)
+                y, K, n_act, _ = sae_row(h, z, sae, app, Ko)
+                res.n_active[t] = n_act
+                if K is not None:
+                    res.topk[t] = K
+            elif app.kind == KIND_ROUTER:
+                continue
+            else:
+                raise ValueError("unknown app kind %r" % app.kind)
+            res.applied[t].append(sl)
+            if app.kind != KIND_PROBE:
+                res.modified[t] = True
+                res.y[t] = y
+                cur = f64_to_bf16_bits(y)
+        res.out_bits[t] = cur
     return res
 
 

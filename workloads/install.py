@@ -31,4 +31,6 @@ def install(m, w: Workload):
             m.register_sae_app(s, a.group, a.edit_idx, a.edit_val, a.edit_mode, a.add_error)
         if getattr(a, "gate", None) is not None:
             m.set_gate(s, a.gate.scores, a.gate.column, a.gate.cmp, a.gate.threshold)
+    for s, nxt in getattr(w, "chains", {}).items():
+        m.set_chain(s, nxt)
     m.set_slot_map(w.token_slot, w.T_live)

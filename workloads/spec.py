@@ -117,6 +117,7 @@ class Workload:
     r_max: int = 0
     d_sae_max: int = 0
     meta: dict = field(default_factory=dict)
+    chains: Dict[int, int] = field(default_factory=dict)   # slot -> next slot applied to the same row
 
 
 def bits(t):
@@ -159,4 +160,4 @@ def host(w: Workload, only_groups=None) -> Workload:
     }
     return Workload(w.name, w.d_model, w.T_max, w.T_live, bits(w.hidden), w.token_slot.copy(),
                     apps, groups, w.n_slots_max, w.n_groups_max, w.C_max, w.k_max, w.r_max,
-                    w.d_sae_max, dict(w.meta))
+                    w.d_sae_max, dict(w.meta), dict(w.chains))
