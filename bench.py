@@ -406,6 +406,29 @@ def extras_decode_variants(w, hiddens, scores, mixlib):
             m.register_project(s, a.v, 1.0)
     out["steer_as_projection_us_per_step"] = measure(m)
     m.destroy()
+    # several apps on one row: every hooked row gets a probe AND a steering vector, (a) as a slot
+    # chain in one call (the row is read once), (b) as two contexts applied one after the other
+    probes = [s for s, a in w.apps.items() if a.kind == W.KIND_PROBE]
+    steers = [s for s, a in w.apps.items() if a.kind == W.KIND_STEER]
+    slot = np.asarray(w.token_slot).copy()
+    hooked = slot >= 0
+    slot[hooked] = np.asarray(probes, dtype=np.int32)[np.arange(int(hooked.sum())) % len(probes)]
+    wc = W.Workload("decode, probe -> steer on every hooked row", w.d_model, T, T, w.hidden, slot, w.apps, {},
+                    n_slots_max=w.n_slots_max, C_max=1, chains={p: steers[i % len(steers)] for i, p in enumerate(probes)})
+    m = W.make_context(mixlib.Mix, wc, flags=mixlib.MIX_FLAG_SLOT_CHAINS)
+    out["probe_then_steer_chained_one_call_us_per_step"] = measure(m)
+    m.destroy()
+    link = {p: steers[i % len(steers)] for i, p in enumerate(probes)}
+    slot_b = np.where(hooked, np.asarray([link.get(int(x), -1) for x in slot], dtype=np.int32), -1).astype(np.int32)
+    ma = W.make_context(mixlib.Mix, W.Workload("a", w.d_model, T, T, w.hidden, slot, w.apps, {}, n_slots_max=w.n_slots_max))
+    mb = W.make_context(mixlib.Mix, W.Workload("b", w.d_model, T, T, w.hidden, slot_b, w.apps, {}, n_slots_max=w.n_slots_max))
+
+    class Two:
+        def apply(self, h, sc, stream=None):
+            ma.apply(h, sc, stream=stream)
+            mb.apply(h, sc, stream=stream)
+    out["probe_then_steer_two_calls_us_per_step"] = measure(Two())
+    ma.destroy(); mb.destroy()
     return out
 
 

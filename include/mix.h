@@ -92,7 +92,12 @@ enum {
   MIX_FLAG_SAE_EDIT_ONLY = 1u << 3    /* algorithmic shortcut: rows of a ReLU / JumpReLU weight set whose app has the
                                          error term on skip the encode; only the pre-activations of their edited
                                          features are computed (|edits| dot products per row).  Same hidden output;
-                                         n_active is not produced for those rows.  TopK rows are unaffected */
+                                         n_active is not produced for those rows.  TopK rows are unaffected */,
+  MIX_FLAG_SLOT_CHAINS = 1u << 4      /* allow mix_set_chain(): several apps applied, in order, to the same row in one
+                                         mix_apply.  Probes and steering then run in one kernel that keeps the row in
+                                         registers across the apps of its chain, and the SAE chain starts only after
+                                         that kernel (the two no longer overlap).  Not together with
+                                         MIX_FLAG_SAE_EDIT_ONLY */
 };
 
 typedef struct {
@@ -223,6 +228,23 @@ int mix_update_sae_edits(mix_ctx* ctx, int slot, int n_edit, const int* idx, con
    registered, bad cmp, row_stride < 1, column outside [0, row_stride)). */
 int mix_set_gate(mix_ctx* ctx, int slot, const float* scores, int row_stride, int column, int cmp, float threshold,
                  void* stream);
+
+/* Several apps on one row (the paper's composition model: every app contributes its own hook
+   functions and state, and the runtime applies the active ones at the hook; the evaluation's
+   "All Apps Combined" configuration).  After mix_set_chain(slot, next_slot) a row whose token
+   slot is `slot` gets the app of `slot` and then the app of `next_slot` (and so on along
+   next_slot's own link; at most 4 apps per row), each app seeing the row as the previous one left
+   it, rounded to bf16 -- bit for bit what separate mix_apply calls, one app each, would give.
+   Every app keeps its own gate: a closed gate skips that app only.  The probes of a chain write
+   their scores side by side: a probe's first column in scores_out[t, :] is the total n_classes of
+   the chain's earlier probes (whether their gates were open or not), so the sum over a chain
+   must not exceed C_max.  An SAE app can only be the last app of a chain; router apps cannot be
+   chained.  next_slot = -1 removes the link.  Registering `slot` again removes its link;
+   unregistering a slot removes the links that point to it.  The context must have been created
+   with MIX_FLAG_SLOT_CHAINS.  Stream-ordered, not captured.
+   Errors: INVALID_ARG (flag missing; a slot without an app; an app kind that cannot be chained
+   there; a cycle; a chain longer than 4; class columns beyond C_max), OUT_OF_RANGE (slot ids). */
+int mix_set_chain(mix_ctx* ctx, int slot, int next_slot, void* stream);
 
 /* Install the token->slot map for the next mix_apply calls: token_slot int32[T_live]
    (host if src_is_device == 0, else device), -1 = no app.  Rows >= T_live are pass-through.

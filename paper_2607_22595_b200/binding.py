@@ -25,10 +25,11 @@ MIX_FLAG_ENCODE_SIMT = 1
 MIX_FLAG_RETILE_W_ENC = 2
 MIX_FLAG_TEST_STALL_ENCODE = 4
 MIX_FLAG_SAE_EDIT_ONLY = 8
+MIX_FLAG_SLOT_CHAINS = 16
 
 EXPORTS = [
     "mix_create", "mix_destroy", "mix_last_error", "mix_register_sae_weights", "mix_unregister_sae_weights",
-    "mix_register_app", "mix_unregister_app", "mix_set_gate", "mix_update_steer_alpha", "mix_update_sae_edits",
+    "mix_register_app", "mix_unregister_app", "mix_set_gate", "mix_set_chain", "mix_update_steer_alpha", "mix_update_sae_edits",
     "mix_set_slot_map", "mix_set_request_map", "mix_set_feature_out", "mix_apply", "mix_apply_conditional", "mix_apply_router", "mix_get_status",
     "mix_launches_per_apply", "mix_set_stage_events", "mix_debug_workspace", "mix_sae_apply_static",
 ]
@@ -91,6 +92,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.mix_register_app.argtypes = [vp, ci, ci, vp, vp]
     lib.mix_unregister_app.argtypes = [vp, ci, vp]
     lib.mix_set_gate.argtypes = [vp, ci, vp, ci, ci, ci, C.c_float, vp]
+    lib.mix_set_chain.argtypes = [vp, ci, ci, vp]
     lib.mix_update_steer_alpha.argtypes = [vp, ci, C.c_float, vp]
     lib.mix_update_sae_edits.argtypes = [vp, ci, ci, vp, vp, vp, vp]
     lib.mix_set_slot_map.argtypes = [vp, vp, ci, ci, vp]
@@ -189,6 +191,10 @@ class Mix:
         d = MixRouter(int(delta.numel()), _ptr(delta))
         self._check(self.lib.mix_register_app(self.ctx, slot, MIX_ROUTER, C.byref(d), _stream(stream)))
         self._keep[("a", slot)] = (delta,)
+
+    def set_chain(self, slot, next_slot, stream=None):
+        """After the app of `slot`, apply the app of `next_slot` to the same row (-1 removes the link)."""
+        self._check(self.lib.mix_set_chain(self.ctx, int(slot), int(next_slot), _stream(stream)))
 
     def apply_router(self, logits, T=None, stream=None):
         assert logits.dtype == torch.float32 and logits.is_cuda and logits.is_contiguous() and logits.dim() == 2

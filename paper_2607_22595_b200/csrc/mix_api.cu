@@ -60,7 +60,7 @@ cudaError_t dev_alloc(T** p, size_t n) {
 }
 
 void free_all(mix_ctx* c) {
-  cudaFree(c->d_token_slot); cudaFree(c->d_n_live); cudaFree(c->d_apps); cudaFree(c->d_groups); cudaFree(c->d_gates); cudaFree(c->d_vec_arena);
+  cudaFree(c->d_token_slot); cudaFree(c->d_n_live); cudaFree(c->d_apps); cudaFree(c->d_groups); cudaFree(c->d_gates); cudaFree(c->d_vec_arena); cudaFree(c->d_chain_next); cudaFree(c->d_row_slot);
   cudaFree(c->d_edit_idx); cudaFree(c->d_edit_val); cudaFree(c->d_edit_mode); cudaFree(c->d_status);
   cudaFree(c->d_tmp_req); cudaFree(c->d_tmp_req_slot); cudaFree(c->d_panel); cudaFree(c->d_panel_row);
   cudaFree(c->d_mtile_group); cudaFree(c->d_row_group); cudaFree(c->d_route); cudaFree(c->d_z); cudaFree(c->d_topk_idx);
@@ -72,7 +72,7 @@ void free_all(mix_ctx* c) {
   if (c->owned_w_tiled)
     for (int g = 0; g < c->cfg.n_groups_max; ++g) cudaFree(c->owned_w_tiled[g]);
   free(c->owned_w_tiled);
-  free(c->owned_b_eff); free(c->h_apps); free(c->h_groups);
+  free(c->owned_b_eff); free(c->h_apps); free(c->h_groups); free(c->h_chain_next);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->ev_join) cudaEventDestroy(c->ev_join);
   if (c->side_stream) cudaStreamDestroy(c->side_stream);
@@ -112,6 +112,46 @@ int upload_edits(mix_ctx* c, int slot, int group, int n_edit, const int* idx, co
   return MIX_OK;
 }
 
+// Walks every chain of the host tables and checks what mix_set_chain() promises: at most kMaxChain
+// apps, only registered apps behind a link, an SAE app only at the end, no router app, and
+// the probes' class columns inside C_max.  (A cycle shows up as a chain that is too long.)
+int validate_chains(mix_ctx* c) {
+  const int NS = c->cfg.n_slots_max;
+  for (int s0 = 0; s0 < NS; ++s0) {
+    if (!c->h_apps[s0].valid || c->h_chain_next[s0] < 0) continue;
+    int len = 0, classes = 0;
+    for (int cur = s0; cur >= 0; cur = c->h_chain_next[cur]) {
+      if (len == kMaxChain) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "the chain through slot %d has a cycle or more than %d apps", s0, kMaxChain);
+      const AppEntry& a = c->h_apps[cur];
+      if (!a.valid) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "the chain from slot %d reaches slot %d, which has no app", s0, cur);
+      const int kind = a.kind & kKindMask;
+      if (kind == MIX_ROUTER) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "slot %d holds a router app: it cannot be part of a chain", cur);
+      if (kind == MIX_SAE && c->h_chain_next[cur] >= 0) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "slot %d holds an SAE app: it can only end a chain", cur);
+      if (kind == MIX_PROBE) classes += a.n_classes;
+      ++len;
+    }
+    if (classes > c->cfg.C_max) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "the probes of the chain from slot %d write %d columns, C_max is %d", s0, classes, c->cfg.C_max);
+  }
+  return MIX_OK;
+}
+
+// Sets or clears the link of `slot` on the device: link first, then the flag in the app entry
+// (when setting), the flag first (when clearing).
+int upload_chain(mix_ctx* c, int slot, cudaStream_t s) {
+  const int next = c->h_chain_next[slot];
+  int kind = c->h_apps[slot].kind & ~kKindChained;
+  if (next < 0) {
+    c->h_apps[slot].kind = kind;
+    if (c->h_apps[slot].valid) MIX_CUDA(c, cudaMemcpyAsync(&c->d_apps[slot].kind, &c->h_apps[slot].kind, sizeof(int), cudaMemcpyHostToDevice, s));
+    MIX_CUDA(c, cudaMemcpyAsync(c->d_chain_next + slot, c->h_chain_next + slot, sizeof(int), cudaMemcpyHostToDevice, s));
+  } else {
+    MIX_CUDA(c, cudaMemcpyAsync(c->d_chain_next + slot, c->h_chain_next + slot, sizeof(int), cudaMemcpyHostToDevice, s));
+    c->h_apps[slot].kind = kind | kKindChained;
+    MIX_CUDA(c, cudaMemcpyAsync(&c->d_apps[slot].kind, &c->h_apps[slot].kind, sizeof(int), cudaMemcpyHostToDevice, s));
+  }
+  return MIX_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -130,6 +170,7 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
     const long long chunks = (cfg->T_max + 1023) / 1024;
     if (chunks * 32 * cfg->n_groups_max * 4 > 40 * 1024) return MIX_ERR_UNSUPPORTED;
   }
+  if ((cfg->flags & MIX_FLAG_SLOT_CHAINS) && (cfg->flags & MIX_FLAG_SAE_EDIT_ONLY)) return MIX_ERR_INVALID_ARG;
   mix_ctx* c = static_cast<mix_ctx*>(calloc(1, sizeof(mix_ctx)));
   if (!c) return MIX_ERR_NO_MEMORY;
   c->cfg = *cfg;
@@ -141,15 +182,18 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
   const int G = cfg->n_groups_max, NS = cfg->n_slots_max, T = cfg->T_max;
   c->h_apps = static_cast<AppEntry*>(calloc(NS, sizeof(AppEntry)));
   c->h_groups = static_cast<GroupEntry*>(calloc(G > 0 ? G : 1, sizeof(GroupEntry)));
+  c->h_chain_next = static_cast<int*>(malloc(NS * sizeof(int)));
+  if (c->h_chain_next) memset(c->h_chain_next, 0xff, NS * sizeof(int));
   c->owned_b_eff = static_cast<float**>(calloc(G > 0 ? G : 1, sizeof(float*)));
   c->owned_w_tiled = static_cast<__nv_bfloat16**>(calloc(G > 0 ? G : 1, sizeof(__nv_bfloat16*)));
-  if (!c->h_apps || !c->h_groups || !c->owned_b_eff || !c->owned_w_tiled) { free_all(c); free(c); return MIX_ERR_NO_MEMORY; }
+  if (!c->h_apps || !c->h_groups || !c->h_chain_next || !c->owned_b_eff || !c->owned_w_tiled) { free_all(c); free(c); return MIX_ERR_NO_MEMORY; }
   bool ok = true;
   ok = ok && dev_alloc(&c->d_token_slot, T) == cudaSuccess;
   ok = ok && dev_alloc(&c->d_n_live, 1) == cudaSuccess;
   ok = ok && dev_alloc(&c->d_apps, NS) == cudaSuccess;
   ok = ok && dev_alloc(&c->d_groups, G > 0 ? G : 1) == cudaSuccess;
   ok = ok && dev_alloc(&c->d_gates, NS) == cudaSuccess;
+  ok = ok && dev_alloc(&c->d_chain_next, NS) == cudaSuccess;
   if (T <= kTeamMaxRows) ok = ok && dev_alloc(&c->d_vec_arena, (size_t)NS * cfg->d_model) == cudaSuccess;
   ok = ok && dev_alloc(&c->d_edit_idx, (size_t)NS * c->cfg.r_max) == cudaSuccess;
   ok = ok && dev_alloc(&c->d_edit_val, (size_t)NS * c->cfg.r_max) == cudaSuccess;
@@ -164,6 +208,7 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
     ok = ok && dev_alloc(&c->d_panel_row, P) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_mtile_group, P / kTileM) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_row_group, T) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_row_slot, T) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_route, 1) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_z, P * (size_t)cfg->d_sae_max) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_topk_idx, P * (size_t)c->cfg.k_max) == cudaSuccess;
@@ -188,6 +233,7 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
   if (e == cudaSuccess) e = cudaMemset(c->d_apps, 0, NS * sizeof(AppEntry));
   if (e == cudaSuccess) e = cudaMemset(c->d_groups, 0, (G > 0 ? G : 1) * sizeof(GroupEntry));
   if (e == cudaSuccess) e = cudaMemset(c->d_gates, 0, NS * sizeof(GateEntry));
+  if (e == cudaSuccess) e = cudaMemset(c->d_chain_next, 0xff, NS * sizeof(int));
   if (e == cudaSuccess && c->d_vec_arena) e = cudaMemset(c->d_vec_arena, 0, (size_t)NS * cfg->d_model * sizeof(__nv_bfloat16));
   if (e == cudaSuccess) e = cudaMemset(c->d_status, 0, sizeof(unsigned));
   if (e == cudaSuccess && G > 0) {
@@ -354,7 +400,19 @@ int mix_register_app(mix_ctx* c, int slot, int kind, const void* desc, void* str
     MIX_CUDA(c, cudaMemcpyAsync(dst, e.W, (size_t)c->cfg.d_model * sizeof(__nv_bfloat16), cudaMemcpyDeviceToDevice, s));
     e.W = dst;
   }
+  const AppEntry old = c->h_apps[slot];
+  const int old_next = c->h_chain_next[slot];
   c->h_apps[slot] = e;
+  c->h_chain_next[slot] = -1;                       // a new app starts without a successor
+  if (c->cfg.flags & MIX_FLAG_SLOT_CHAINS) {
+    rc = validate_chains(c);                        // chains that END in or pass through this slot must still fit
+    if (rc != MIX_OK) {
+      c->h_apps[slot] = old;
+      c->h_chain_next[slot] = old_next;
+      return rc;
+    }
+    if (old_next >= 0) MIX_CUDA(c, cudaMemcpyAsync(c->d_chain_next + slot, c->h_chain_next + slot, sizeof(int), cudaMemcpyHostToDevice, s));
+  }
   return publish_app(c, slot, s);
 }
 
@@ -366,7 +424,34 @@ int mix_unregister_app(mix_ctx* c, int slot, void* stream) {
   const int zero = 0;
   MIX_CUDA(c, cudaMemcpyAsync(&c->d_apps[slot].valid, &zero, sizeof(int), cudaMemcpyHostToDevice,
                               static_cast<cudaStream_t>(stream)));
+  if (c->cfg.flags & MIX_FLAG_SLOT_CHAINS) {        // links from and to the slot go with it
+    for (int p = 0; p < c->cfg.n_slots_max; ++p) {
+      if (p != slot && c->h_chain_next[p] != slot) continue;
+      if (c->h_chain_next[p] < 0) continue;
+      c->h_chain_next[p] = -1;
+      rc = upload_chain(c, p, static_cast<cudaStream_t>(stream));
+      if (rc != MIX_OK) return rc;
+    }
+  }
   return MIX_OK;
+}
+
+int mix_set_chain(mix_ctx* c, int slot, int next_slot, void* stream) {
+  if (!c) return MIX_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (!(c->cfg.flags & MIX_FLAG_SLOT_CHAINS)) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "the context was created without MIX_FLAG_SLOT_CHAINS");
+  int rc = check_slot(c, slot);
+  if (rc != MIX_OK) return rc;
+  if (next_slot < -1 || next_slot >= c->cfg.n_slots_max) MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "next_slot %d outside [-1, %d)", next_slot, c->cfg.n_slots_max);
+  if (!c->h_apps[slot].valid) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "slot %d has no app", slot);
+  const int old_next = c->h_chain_next[slot];
+  c->h_chain_next[slot] = next_slot;
+  rc = validate_chains(c);
+  if (rc != MIX_OK) {
+    c->h_chain_next[slot] = old_next;
+    return rc;
+  }
+  return upload_chain(c, slot, s);
 }
 
 int mix_set_gate(mix_ctx* c, int slot, const float* scores, int row_stride, int column, int cmp, float threshold,
@@ -376,7 +461,7 @@ int mix_set_gate(mix_ctx* c, int slot, const float* scores, int row_stride, int 
   int rc = check_slot(c, slot);
   if (rc != MIX_OK) return rc;
   if (!c->h_apps[slot].valid) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "slot %d has no app to gate", slot);
-  int kind = c->h_apps[slot].kind & kKindMask;
+  int kind = c->h_apps[slot].kind & ~kKindGated;
   if (!scores) {                      // remove: drop the flag first, the entry may then go stale
     c->h_apps[slot].kind = kind;
     MIX_CUDA(c, cudaMemcpyAsync(&c->d_apps[slot].kind, &kind, sizeof(int), cudaMemcpyHostToDevice, s));
@@ -569,6 +654,9 @@ int apply_impl(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream,
   if (c->cfg.n_groups_max > 0) {
     MIX_CUDA(c, launch_route(c, T, s, handle, conditional ? 1 : 0));
     MIX_CUDA(c, tap());
+    // with slot chains a steering app may precede an SAE app on the same row: the SAE chain reads
+    // the hidden state only after the probe / steering kernel is done
+    if (fork && (c->cfg.flags & MIX_FLAG_SLOT_CHAINS)) MIX_CUDA(c, cudaStreamWaitEvent(s, c->ev_join, 0));
     const int rc = conditional ? sae_chain_conditional(c, h, s, graph, handle) : sae_chain(c, h, s, tap);
     if (rc != MIX_OK) return rc;
     if (c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) {

@@ -39,6 +39,8 @@ struct __align__(16) AppEntry {
 
 constexpr int kKindMask = 0xff;     // AppEntry.kind: low byte = MIX_* kind
 constexpr int kKindGated = 0x100;   //                bit 8    = the slot has a gate (see GateEntry)
+constexpr int kKindChained = 0x200; //                bit 9    = another app follows on the same row (chain_next[slot])
+constexpr int kMaxChain = 4;        // apps applied to one row in one call
 
 // Gate of a slot: the app applies to row t iff cmp(scores[t * stride + col], thr).
 struct __align__(16) GateEntry {
@@ -95,6 +97,8 @@ struct Ctx {
   AppEntry* d_apps;         // [n_slots_max]
   GroupEntry* d_groups;     // [n_groups_max]
   GateEntry* d_gates;       // [n_slots_max]
+  int* d_chain_next;        // [n_slots_max] next slot applied to the same row, or -1 (MIX_FLAG_SLOT_CHAINS)
+  int* h_chain_next;        // host mirror
   __nv_bfloat16* d_vec_arena;   // [n_slots_max, d] copies of single-vector weights (T_max <= kTeamMaxRows), else null
   int* d_edit_idx;          // [n_slots_max * r_max]
   float* d_edit_val;
@@ -115,6 +119,7 @@ struct Ctx {
   int* d_panel_row;         // [P] token index or -1
   int* d_mtile_group;       // [P / kTileM] group of each m-tile or -1
   int* d_row_group;         // [T_max] routing scratch: weight set of each token row or -1
+  int* d_row_slot;          // [T_max] slot of the SAE app that acts on the row (the row's own slot, or the last of its chain), or -1
   RouteState* d_route;
   float* d_z;               // [P, d_sae_max]
   RowDelta* d_row_delta;    // [P]

@@ -144,6 +144,8 @@ __device__ __forceinline__ void finish_probe(const float* logit, int C, int act,
 
 struct RowApp {
   bool gated;           // the slot has a gate (whether or not it let this row through)
+  bool chained;         // another app follows on the same row (set even when the gate is closed)
+  int raw_kind;         // the slot's kind even when the gate is closed (0: no valid app)
   int kind, C, act;     // kind 0: nothing to do
   float alpha;
   const uint4* W;
@@ -167,7 +169,10 @@ __device__ __forceinline__ RowApp lookup(int s, int t, const AppEntry* __restric
                                          unsigned* __restrict__ status, bool leader, bool eval_gate = true) {
   RowApp r;
   r.kind = 0;
+  r.raw_kind = 0;
+  r.C = 0;
   r.gated = false;
+  r.chained = false;
   if (s == -1) return r;
   if (s < -1 || s >= n_slots) {
     if (leader) atomicOr(status, MIX_STATUS_BAD_SLOT);
@@ -181,9 +186,11 @@ __device__ __forceinline__ RowApp lookup(int s, int t, const AppEntry* __restric
     return r;
   }
   r.gated = (q0.y & kKindGated) != 0;
+  r.chained = (q0.y & kKindChained) != 0;
+  r.raw_kind = q0.y & kKindMask;
+  r.C = q0.z;
   if (eval_gate && r.gated && !gate_open(gates, s, t)) return r;  // gate closed: the row passes through
   r.kind = q0.y & kKindMask;
-  r.C = q0.z;
   r.act = q0.w;
   r.alpha = __int_as_float(q1.x);
   r.W = reinterpret_cast<const uint4*>(((unsigned long long)(unsigned)q2.y << 32) | (unsigned)q2.x);
@@ -553,6 +560,129 @@ probe_steer_team_kernel(const int* __restrict__ token_slot, const int* __restric
   }
 }
 
+// Contexts with slot chains: one CTA per row, the row held in registers while the apps of its chain
+// are applied one after the other (probe / steering / projection; an SAE app at the end of a chain
+// is left to the SAE kernels, which start after this one).  A write rounds the row to bf16 in
+// registers, exactly as a store and reload would; the row goes back to memory once, at the end,
+// if any app changed it.  The j-th probe of a chain writes its scores after those of the earlier
+// ones.  Control flow is uniform across the CTA.
+constexpr int kChainWarps = 8;
+
+__global__ void __launch_bounds__(kChainWarps * 32)
+probe_steer_chain_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
+                         const AppEntry* __restrict__ apps, const GateEntry* __restrict__ gates,
+                         const int* __restrict__ chain_next, int n_slots, __nv_bfloat16* __restrict__ hidden, int d,
+                         float* __restrict__ scores, int C_max, unsigned* __restrict__ status) {
+  __shared__ float s_part[kChainWarps][kMaxClasses];
+  constexpr int NT = kChainWarps * 32;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t = blockIdx.x;
+  if (t >= min(T, __ldg(n_live_p))) return;
+  int slot = __ldg(token_slot + t);
+  if (slot == -1) return;
+  const int nvec = d >> 3;
+  uint4* hrow = reinterpret_cast<uint4*>(hidden + (size_t)t * d);
+  uint4 hq[kTeamVec];
+#pragma unroll
+  for (int u = 0; u < kTeamVec; ++u) {
+    const int v = threadIdx.x + u * NT;
+    hq[u] = make_uint4(0u, 0u, 0u, 0u);
+    if (v < nvec && slot >= 0 && slot < n_slots) hq[u] = __ldcs(hrow + v);
+  }
+  bool dirty = false;
+  int col = 0;
+  for (int depth = 0; depth < kMaxChain; ++depth) {
+    const RowApp a = lookup(slot, t, apps, gates, n_slots, status, threadIdx.x == 0);
+    if ((a.kind == MIX_STEER || a.kind == MIX_PROJECT) && a.alpha != 0.f) {   // alpha = 0: identity, bit-exact
+      uint4 vq[kTeamVec];
+#pragma unroll
+      for (int u = 0; u < kTeamVec; ++u) {
+        const int v = threadIdx.x + u * NT;
+        vq[u] = make_uint4(0u, 0u, 0u, 0u);
+        if (v < nvec) vq[u] = __ldg(a.W + v);
+      }
+      float coef = a.alpha;
+      if (a.kind == MIX_PROJECT) {               // h - beta (h . r) r
+        float dot = 0.f;
+#pragma unroll
+        for (int u = 0; u < kTeamVec; ++u) {
+          float x[8], y[8];
+          unpack8(hq[u], x);
+          unpack8(vq[u], y);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) dot = fmaf(x[e], y[e], dot);
+        }
+        dot = warp_sum(dot);
+        if (lane == 0) s_part[warp][0] = dot;
+        __syncthreads();
+        float total = 0.f;
+#pragma unroll
+        for (int w = 0; w < kChainWarps; ++w) total += s_part[w][0];
+        coef = -a.alpha * total;
+      }
+#pragma unroll
+      for (int u = 0; u < kTeamVec; ++u) {
+        float x[8], y[8];
+        unpack8(hq[u], x);
+        unpack8(vq[u], y);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) x[e] = fmaf(coef, y[e], x[e]);
+        hq[u] = pack8(x);
+      }
+      dirty = true;
+    } else if (a.kind == MIX_PROBE && scores != nullptr) {
+      for (int c0 = 0; c0 < a.C; c0 += 4) {
+        const int nc = min(4, a.C - c0);
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int u = 0; u < kTeamVec; ++u) {
+          const int v = threadIdx.x + u * NT;
+          if (v < nvec) {
+            float x[8];
+            unpack8(hq[u], x);
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+              if (c < nc) {
+                float y[8];
+                unpack8(__ldg(a.W + (size_t)(c0 + c) * nvec + v), y);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[c] = fmaf(x[e], y[e], acc[c]);
+              }
+          }
+        }
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const float z = warp_sum(acc[c]);
+          if (lane == 0 && c < nc) s_part[warp][c0 + c] = z;
+        }
+      }
+      __syncthreads();
+      if (warp == 0) {
+        for (int c = lane; c < a.C; c += 32) {
+          float z = a.b ? __ldg(a.b + c) : 0.f;
+#pragma unroll
+          for (int w = 0; w < kChainWarps; ++w) z += s_part[w][c];
+          s_part[0][c] = z;            // only this lane reads or writes column c from here on
+        }
+        __syncwarp();
+        finish_probe(s_part[0], a.C, a.act, scores + (size_t)t * C_max + col, lane);
+      }
+    }
+    if (!a.chained) break;
+    if (a.raw_kind == MIX_PROBE) col += a.C;
+    slot = __ldg(chain_next + slot);             // slot was in range: lookup() found a valid entry
+    if (slot < 0) break;
+    __syncthreads();                             // s_part is reused by the next app
+  }
+  if (dirty) {
+#pragma unroll
+    for (int u = 0; u < kTeamVec; ++u) {
+      const int v = threadIdx.x + u * NT;
+      if (v < nvec) __stcs(hrow + v, hq[u]);
+    }
+  }
+}
+
 // ---------------------------------------------------------------------------------------
 // SAE routing: one CTA builds, in ascending row order, the packed-panel position of every
 // SAE row, the per-group counts and the encode tile schedule.  Integer work only.
@@ -568,7 +698,8 @@ route_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_
              int* __restrict__ panel_row, int panel_cap, int* __restrict__ mtile_group, RouteState* __restrict__ rs,
              unsigned* __restrict__ status, int* __restrict__ row_flag, int* __restrict__ mtile_flag,
              int* __restrict__ n_flagged, int* __restrict__ row_group, int edit_only,
-             cudaGraphConditionalHandle cond, int use_cond) {
+             cudaGraphConditionalHandle cond, int use_cond, const int* __restrict__ chain_next,
+             int* __restrict__ row_slot) {
   extern __shared__ int s_cnt[];                      // [n_chunks * kRouteWarps][n_groups]
   __shared__ int s_total[kMaxGroups], s_base[kMaxGroups + 1];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -606,6 +737,26 @@ route_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_
         group_id[c] = __ldg(&apps[slot[c]].group);
       }
     }
+    // a row whose slot starts a chain is an SAE row if the chain ends in an SAE app: follow the
+    // links (rare, so the dependent loads are not batched) and carry on with that app's slot
+#pragma unroll
+    for (int c = 0; c < kRouteBatch; ++c) {
+      if (head[c].x && (head[c].y & kKindChained) && (head[c].y & kKindMask) != MIX_SAE) {
+        int s2 = slot[c];
+        int2 h2 = head[c];
+        for (int depth = 1; depth < kMaxChain && s2 >= 0; ++depth) {
+          s2 = (h2.y & kKindChained) ? __ldg(chain_next + s2) : -1;
+          if (s2 < 0 || s2 >= n_slots) { s2 = -1; break; }
+          h2 = __ldg(reinterpret_cast<const int2*>(apps + s2));
+          if (!h2.x) { s2 = -1; break; }
+          if ((h2.y & kKindMask) == MIX_SAE) break;
+        }
+        if (s2 >= 0 && (h2.y & kKindMask) != MIX_SAE) s2 = -1;
+        slot[c] = s2;
+        head[c] = s2 >= 0 ? h2 : make_int2(0, 0);
+        group_id[c] = s2 >= 0 ? __ldg(&apps[s2].group) : -1;
+      }
+    }
 #pragma unroll
     for (int c = 0; c < kRouteBatch; ++c) {
       grp[c] = -1;
@@ -625,7 +776,10 @@ route_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_
     for (int c = 0; c < kRouteBatch; ++c) {
       if (c0 + c < n_chunks) {                       // uniform across the CTA
         const int t = (c0 + c) * kRouteThreads + tid;
-        if (t < n_live) row_group[t] = grp[c];       // read back by this same thread in phase C
+        if (t < n_live) {
+          row_group[t] = grp[c];                     // read back by this same thread in phase C
+          row_slot[t] = grp[c] >= 0 ? slot[c] : -1;  // the SAE app's slot, for the decode kernels
+        }
         for (int q = 0; q < n_groups; ++q) {
           const unsigned m = __ballot_sync(0xffffffffu, grp[c] == q);
           if (lane == 0) s_cnt[((c0 + c) * kRouteWarps + warp) * n_groups + q] = __popc(m);
@@ -760,10 +914,17 @@ __global__ void fold_bias_kernel(const __nv_bfloat16* __restrict__ W_enc, const 
 }  // namespace
 
 
-bool has_multiclass_stage(const Ctx* c) { return c->cfg.T_max > kTeamMaxRows && c->cfg.C_max > 1; }
+bool has_multiclass_stage(const Ctx* c) {
+  return c->cfg.T_max > kTeamMaxRows && c->cfg.C_max > 1 && !(c->cfg.flags & MIX_FLAG_SLOT_CHAINS);
+}
 
 cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s) {
-  if (c->cfg.T_max <= kTeamMaxRows) {
+  if (c->cfg.flags & MIX_FLAG_SLOT_CHAINS) {
+    probe_steer_chain_kernel<<<c->cfg.T_max, kChainWarps * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps,
+                                                                       c->d_gates, c->d_chain_next, c->cfg.n_slots_max,
+                                                                       hidden, c->cfg.d_model, scores, c->cfg.C_max,
+                                                                       c->d_status);
+  } else if (c->cfg.T_max <= kTeamMaxRows) {
     probe_steer_team_kernel<8><<<c->cfg.T_max, 8 * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates,
                                                               c->cfg.n_slots_max, hidden, c->cfg.d_model, scores,
                                                               c->cfg.C_max, c->d_status,
@@ -800,7 +961,8 @@ cudaError_t launch_route(const Ctx* c, int T, cudaStream_t s, unsigned long long
                                               c->d_mtile_group, c->d_route, c->d_status, c->d_row_flag,
                                               c->d_mtile_flag, c->d_n_flagged, c->d_row_group,
                                               (c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) ? 1 : 0,
-                                              static_cast<cudaGraphConditionalHandle>(cond), use_cond);
+                                              static_cast<cudaGraphConditionalHandle>(cond), use_cond, c->d_chain_next,
+                                              c->d_row_slot);
   return cudaGetLastError();
 }
 

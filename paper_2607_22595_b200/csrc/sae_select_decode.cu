@@ -420,7 +420,7 @@ __device__ __forceinline__ void accumulate_list(float (*acc)[8], const float* co
 
 __global__ void __launch_bounds__(kDecThreads)
 decode_kernel(__nv_bfloat16* __restrict__ hidden, int d, const float* __restrict__ Z, long long ldz,
-              const int* __restrict__ panel_row, const int* __restrict__ token_slot,
+              const int* __restrict__ panel_row, const int* __restrict__ row_slot,
               const RouteState* __restrict__ rs, const AppEntry* __restrict__ apps,
               const GroupEntry* __restrict__ groups, const int* __restrict__ edit_idx,
               const float* __restrict__ edit_val, const unsigned char* __restrict__ edit_mode, int r_max, int k_max,
@@ -441,7 +441,7 @@ decode_kernel(__nv_bfloat16* __restrict__ hidden, int d, const float* __restrict
     if (tid == 0) row_delta[p].slot = -1;             // padding row of a tile
     return;
   }
-  const int slot = token_slot[t];
+  const int slot = row_slot[t];                       // the SAE app's slot (the row's own, or the last of its chain)
   const AppEntry app = apps[slot];
   const GroupEntry ge = groups[app.group];
   const int n_edit = app.n_edit;
@@ -841,7 +841,7 @@ cudaError_t launch_edit_only(const Ctx* c, __nv_bfloat16* hidden, int T, cudaStr
 // then adds those rows' deltas, eight rows per CTA.
 cudaError_t launch_decode(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s) {
   decode_kernel<<<c->panel_rows_cap, kDecThreads, 0, s>>>(hidden, c->cfg.d_model, c->d_z, c->cfg.d_sae_max,
-                                                          c->d_panel_row, c->d_token_slot, c->d_route, c->d_apps,
+                                                          c->d_panel_row, c->d_row_slot, c->d_route, c->d_apps,
                                                           c->d_groups, c->d_edit_idx, c->d_edit_val, c->d_edit_mode,
                                                           c->cfg.r_max, c->cfg.k_max, c->d_topk_idx, c->d_topk_val,
                                                           c->d_row_delta, c->d_edit_coef);

@@ -37,7 +37,9 @@ constexpr size_t kOffRoute = kOffEditMode + align256(kMaxEdits);
 constexpr size_t kOffPanelRow = kOffRoute + align256(sizeof(RouteState));
 constexpr size_t kOffMtileGroup = kOffPanelRow + align256(kStaticRows * sizeof(int));
 constexpr size_t kOffRowGroup = kOffMtileGroup + 256;
-constexpr size_t kOffRowDelta = kOffRowGroup + align256(kStaticRows * sizeof(int));
+constexpr size_t kOffRowSlot = kOffRowGroup + align256(kStaticRows * sizeof(int));
+constexpr size_t kOffChainNext = kOffRowSlot + align256(kStaticRows * sizeof(int));
+constexpr size_t kOffRowDelta = kOffChainNext + 256;
 constexpr size_t kOffEditCoef = kOffRowDelta + align256(kStaticRows * sizeof(RowDelta));
 constexpr size_t kOffTopkIdx = kOffEditCoef + align256((size_t)kStaticRows * kMaxEdits * sizeof(float));
 constexpr size_t kOffTopkVal = kOffTopkIdx + align256((size_t)kStaticRows * kStaticK * sizeof(int));
@@ -134,6 +136,8 @@ extern "C" int mix_sae_apply_static(void* hidden, int n_rows, int d_model, const
   c.d_panel_row = reinterpret_cast<int*>(base + kOffPanelRow);
   c.d_mtile_group = reinterpret_cast<int*>(base + kOffMtileGroup);
   c.d_row_group = reinterpret_cast<int*>(base + kOffRowGroup);
+  c.d_row_slot = reinterpret_cast<int*>(base + kOffRowSlot);
+  c.d_chain_next = reinterpret_cast<int*>(base + kOffChainNext);   // never read: the app entry carries no chain flag
   c.d_row_delta = reinterpret_cast<RowDelta*>(base + kOffRowDelta);
   c.d_edit_coef = reinterpret_cast<float*>(base + kOffEditCoef);
   c.d_topk_idx = reinterpret_cast<int*>(base + kOffTopkIdx);

@@ -21,7 +21,7 @@ import numpy as np
 import torch
 
 from .spec import (ACT_SIGMOID, ACT_SOFTMAX, EDIT_ABLATE, EDIT_CLAMP, SAE_JUMPRELU, SAE_TOPK,
-                   Probe, SaeApp, SaeWeights, Steer, Workload)
+                   ACT_NONE, Probe, Project, SaeApp, SaeWeights, Steer, Workload)
 
 BASE_SEED = 20260722
 
@@ -172,6 +172,52 @@ def make_tiny(device="cpu", d=512, T=64, d_sae=4096, k=32, seed=None):
     return Workload("tiny", d, T, T, hidden, token_slot, apps, {0: sae}, n_slots_max=8,
                     n_groups_max=1, C_max=1, k_max=k, r_max=4, d_sae_max=d_sae,
                     meta={"lengths": lengths, "req_slot": req_slot, "token_req": token_req, "seed": seed})
+
+
+# --------------------------------------------------------------------------
+# several apps on one row ("all apps combined"): slot chains
+# --------------------------------------------------------------------------
+def make_chained(device="cpu", d=512, T=300, d_sae=2048, k=16, C=5, seed=None):
+    """Every hooked request carries a chain of apps on each of its tokens:
+         0 -> 1 -> 2 -> 3   sigmoid probe, steering, softmax probe (C classes), TopK SAE edit (error term on)
+         4 -> 5             projection, JumpReLU SAE edit (error term off)
+         6 -> 1 -> ...      a second head that joins the first chain at its steering app
+         7                  a steering app on its own; 8: a raw-logit probe on its own
+       plus requests that enter chain 0 in the middle (token slot 1, 2 or 3) and unhooked requests."""
+    seed = BASE_SEED + 5000 if seed is None else seed
+    g, rng = _gen(device, seed), np.random.default_rng(seed)
+    hidden = _hidden(g, device, T, d)
+    zero1 = torch.zeros(1, dtype=torch.float32, device=device)
+    sae_t = make_sae_weights(g, device, d, d_sae, SAE_TOPK, k=k)
+    sae_j = make_sae_weights(g, device, d, d_sae, SAE_JUMPRELU, k=0, theta_range=(0.05, 0.3), b_enc_mean=-2.0)
+    e_t = rng.choice(d_sae, size=4, replace=False).astype(np.int32)
+    e_j = rng.choice(d_sae, size=3, replace=False).astype(np.int32)
+    apps = {
+        0: Probe(W=_randn_bf16(g, device, 1, d, d ** -0.5), b=zero1.clone(), act=ACT_SIGMOID),
+        1: Steer(v=_unit_rows_bf16(g, device, 1, d)[0].contiguous(), alpha=4.0),
+        2: Probe(W=_randn_bf16(g, device, C, d, d ** -0.5),
+                 b=torch.randn(C, generator=g, device=device, dtype=torch.float32), act=ACT_SOFTMAX),
+        3: SaeApp(0, e_t, np.array([5.0, 0.0, 2.5, 0.0], np.float32),
+                  np.array([EDIT_CLAMP, EDIT_ABLATE, EDIT_CLAMP, EDIT_ABLATE], np.uint8), add_error=True),
+        4: Project(r=_unit_rows_bf16(g, device, 1, d)[0].contiguous(), beta=1.0),
+        5: SaeApp(1, e_j, np.array([3.0, 0.0, 1.0], np.float32),
+                  np.array([EDIT_CLAMP, EDIT_ABLATE, EDIT_CLAMP], np.uint8), add_error=False),
+        6: Probe(W=_randn_bf16(g, device, 1, d, d ** -0.5), b=None, act=ACT_SIGMOID),
+        7: Steer(v=_unit_rows_bf16(g, device, 1, d)[0].contiguous(), alpha=-2.0),
+        8: Probe(W=_randn_bf16(g, device, 1, d, d ** -0.5), b=zero1.clone(), act=ACT_NONE),
+    }
+    chains = {0: 1, 1: 2, 2: 3, 4: 5, 6: 1}
+    R = max(T // 12, 10)
+    lengths = ragged_lengths_uniform(rng, T, R)
+    req_slot = rng.choice(np.array([0, 0, 0, 4, 4, 6, 6, 7, 8, 1, 2, 3, 5, -1, -1], dtype=np.int32), size=R)
+    req_slot[:10] = np.array([0, 4, 6, 7, 8, 1, 2, 3, 5, -1], dtype=np.int32)     # every case at least once
+    rng.shuffle(req_slot)
+    order = rng.permutation(R)
+    token_slot, token_req, used = _token_slot_from_requests(lengths, req_slot, order, T)
+    return Workload("chained", d, T, used, hidden, token_slot, apps, {0: sae_t, 1: sae_j}, n_slots_max=9,
+                    n_groups_max=2, C_max=1 + C + 1, k_max=k, r_max=4, d_sae_max=d_sae,
+                    meta={"lengths": lengths, "req_slot": req_slot, "token_req": token_req, "seed": seed},
+                    chains=chains)
 
 
 # --------------------------------------------------------------------------
