@@ -22,7 +22,8 @@ memory (each pre-activation is still one full-length dot product).
 
 Parity pins: every function here is pinned by tests/test_oracle_pins.py
 (closed forms, hand-worked values under tests/golden/, brute force, library
-routines, algebraic invariants).  Nothing is "parity unpinned".
+routines, algebraic invariants), tests/test_oracle_chain.py (slot chains) and
+tests/test_oracle_fp8.py (8-bit encoder).  Nothing is "parity unpinned".
 """
 from __future__ import annotations
 
@@ -125,10 +126,28 @@ def gate_open(gate, t: int) -> bool:
 # ---------------------------------------------------------------------------
 # SAE function
 # ---------------------------------------------------------------------------
+def e4m3_to_f64(codes: np.ndarray) -> np.ndarray:
+    """Value of 8-bit E4M3 codes (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; no
+    infinities, S.1111.111 is NaN): +-2^(e-7) (1 + m/8) for e > 0, +-2^-6 (m/8) for e = 0."""
+    c = np.asarray(codes, dtype=np.uint8).astype(np.int64)
+    e, m = (c >> 3) & 0xF, c & 0x7
+    mag = np.where(e == 0, (m / 8.0) * 2.0 ** -6, (1.0 + m / 8.0) * np.exp2((e - 7).astype(np.float64)))
+    mag = np.where((e == 15) & (m == 7), np.nan, mag)
+    return np.where(c & 0x80, -mag, mag)
+
+
+def encoder_rows_f64(W_enc_bits: np.ndarray, w_scale: Optional[np.ndarray] = None) -> np.ndarray:
+    """Encoder rows as float64: bf16 bits, or (8-bit encoder) E4M3 codes times the row's fp32 scale."""
+    if w_scale is None:
+        return bf16_to_f64(W_enc_bits)
+    return e4m3_to_f64(W_enc_bits) * np.asarray(w_scale, dtype=np.float64)[:, None]
+
+
 def sae_preact(X: np.ndarray, W_enc_bits: np.ndarray, b_enc: np.ndarray,
-               b_dec: Optional[np.ndarray] = None, center_input: bool = False) -> np.ndarray:
+               b_dec: Optional[np.ndarray] = None, center_input: bool = False,
+               w_scale: Optional[np.ndarray] = None) -> np.ndarray:
     """Pre-activations z[n, j] = b_enc[j] + sum_i W_enc[j, i] * (X[n, i] - [center] b_dec[i]).
-    X [n, d] float64; W_enc given as bf16 bits [S, d]."""
+    X [n, d] float64; W_enc given as bf16 bits [S, d], or as E4M3 codes [S, d] with w_scale [S]."""
     X = np.atleast_2d(np.asarray(X, dtype=np.float64))
     if center_input and b_dec is not None:
         X = X - np.asarray(b_dec, dtype=np.float64)[None, :]
@@ -136,7 +155,7 @@ def sae_preact(X: np.ndarray, W_enc_bits: np.ndarray, b_enc: np.ndarray,
     Z = np.empty((X.shape[0], S), dtype=np.float64)
     for j0 in range(0, S, _CHUNK):
         j1 = min(S, j0 + _CHUNK)
-        Z[:, j0:j1] = X @ bf16_to_f64(W_enc_bits[j0:j1]).T
+        Z[:, j0:j1] = X @ encoder_rows_f64(W_enc_bits[j0:j1], None if w_scale is None else w_scale[j0:j1]).T
     return Z + np.asarray(b_enc, dtype=np.float64)[None, :]
 
 
@@ -293,7 +312,7 @@ def apply_hook(w, rows: Optional[Iterable[int]] = None, keep_z: bool = False,
     for g, ts in sae_rows.items():
         sae = w.groups[g]
         X = bf16_to_f64(hidden_bits[np.asarray(ts)])
-        Z = sae_preact(X, sae.W_enc, sae.b_enc, sae.b_dec, sae.center_input)
+        Z = sae_preact(X, sae.W_enc, sae.b_enc, sae.b_dec, sae.center_input, getattr(sae, "w_scale", None))
         for n, t in enumerate(ts):
             app = w.apps[int(w.token_slot[t])]
             Ko = None if topk_override is None else topk_override.get(t)
@@ -380,7 +399,8 @@ def apply_chain_hook(w, rows: Optional[Iterable[int]] = None,
                 y = project(h, bf16_to_f64(app.r), app.beta)
             elif app.kind == KIND_SAE:
                 sae = w.groups[app.group]
-                z = sae_preact(h[None, :], sae.W_enc, sae.b_enc, sae.b_dec, sae.center_input)[0]
+                z = sae_preact(h[None, :], sae.W_enc, sae.b_enc, sae.b_dec, sae.center_input,
+                               getattr(sae, "w_scale", None))[0]
                 Ko = None if topk_override is None else topk_override.get(t)
                 y, K, n_act, _ = sae_row(h, z, sae, app, Ko)
                 res.n_active[t] = n_act

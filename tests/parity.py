@@ -166,6 +166,6 @@ def sample_rows(wh, per_kind=24, seed=0):
 def oracle_edit_hint(gi, sae, h_row):
     """Edit hint for the generators: the oracle's active features on one row."""
     x = O.bf16_to_f64(W.bits(h_row))
-    z = O.sae_preact(x, W.bits(sae.W_enc), W.bits(sae.b_enc))[0]
+    z = O.sae_preact(x, W.bits(sae.W_enc), W.bits(sae.b_enc), w_scale=W.bits(sae.w_scale))[0]
     f, K = O.sae_activate(z, sae.act, sae.k, None if sae.theta is None else W.bits(sae.theta))
     return np.nonzero(f > 0)[0]

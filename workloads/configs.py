@@ -67,16 +67,24 @@ def _hidden(g, device, T, d, outlier_cols=None):
     return x.to(torch.bfloat16)
 
 
-def make_sae_weights(g, device, d, d_sae, act, k=0, theta_range=None, b_enc_mean=-0.1):
-    """W_enc ~ N(0, 1/d) (variance), W_dec rows unit-norm, b_enc ~ N(mean, std 0.02)."""
-    W_enc = _randn_bf16(g, device, d_sae, d, d ** -0.5)
+def make_sae_weights(g, device, d, d_sae, act, k=0, theta_range=None, b_enc_mean=-0.1, fp8=False):
+    """W_enc ~ N(0, 1/d) (variance), W_dec rows unit-norm, b_enc ~ N(mean, std 0.02).
+    fp8: the encoder is stored as E4M3 codes with one fp32 scale per feature (row absmax / 448),
+    rounded by torch's float8_e4m3fn conversion; the codes and scales ARE the weights."""
+    w_scale = None
+    if fp8:
+        Wf = torch.randn((d_sae, d), generator=g, device=device, dtype=torch.float32) * d ** -0.5
+        w_scale = (Wf.abs().amax(dim=1) / 448.0).clamp_min(1e-12)
+        W_enc = (Wf / w_scale[:, None]).to(torch.float8_e4m3fn).view(torch.uint8)
+    else:
+        W_enc = _randn_bf16(g, device, d_sae, d, d ** -0.5)
     W_dec = _unit_rows_bf16(g, device, d_sae, d)
     b_enc = (torch.randn((d_sae,), generator=g, device=device, dtype=torch.float32) * 0.02 + b_enc_mean)
     theta = None
     if act == SAE_JUMPRELU:
         lo, hi = theta_range
         theta = torch.rand((d_sae,), generator=g, device=device, dtype=torch.float32) * (hi - lo) + lo
-    return SaeWeights(d_sae=d_sae, act=act, k=k, W_enc=W_enc, b_enc=b_enc, W_dec=W_dec, theta=theta)
+    return SaeWeights(d_sae=d_sae, act=act, k=k, W_enc=W_enc, b_enc=b_enc, W_dec=W_dec, theta=theta, w_scale=w_scale)
 
 
 def ragged_lengths_uniform(rng, T, R):

@@ -81,12 +81,13 @@ class SaeWeights:
     d_sae: int
     act: int
     k: int                    # TopK only (0 otherwise)
-    W_enc: object             # bf16 [d_sae, d]; row j = encoder direction j
+    W_enc: object             # bf16 [d_sae, d]; row j = encoder direction j.  With w_scale set: uint8 [d_sae, d], E4M3 codes
     b_enc: object             # fp32 [d_sae]
     W_dec: object             # bf16 [d_sae, d]; row j = decoder direction j
     theta: Optional[object] = None   # fp32 [d_sae], JumpReLU only
     b_dec: Optional[object] = None   # fp32 [d]
     center_input: bool = False
+    w_scale: Optional[object] = None   # fp32 [d_sae]: 8-bit encoder, W_enc[j, i] = e4m3(code[j, i]) * w_scale[j]
 
 
 @dataclass
@@ -155,7 +156,7 @@ def host(w: Workload, only_groups=None) -> Workload:
             apps[s] = SaeApp(a.group, a.edit_idx, a.edit_val, a.edit_mode, a.add_error, gate=g)
     groups = {
         g: SaeWeights(sw.d_sae, sw.act, sw.k, bits(sw.W_enc), bits(sw.b_enc), bits(sw.W_dec),
-                      bits(sw.theta), bits(sw.b_dec), sw.center_input)
+                      bits(sw.theta), bits(sw.b_dec), sw.center_input, bits(sw.w_scale))
         for g, sw in w.groups.items() if only_groups is None or g in only_groups
     }
     return Workload(w.name, w.d_model, w.T_max, w.T_live, bits(w.hidden), w.token_slot.copy(),
