@@ -210,7 +210,7 @@ def time_stages(m, fn, reps=5):
     return dict(zip(m.STAGES[:n], best))
 
 
-def extras_sae(name, w, peaks, mixlib, extra_flags=0):
+def extras_sae(name, w, peaks, mixlib, extra_flags=0, w_enc_bytes_per_el=2.0):
     """SAE-carrying config: per-kernel times, encode flop rate and weight-stream bandwidth."""
     m = W.make_context(mixlib.Mix, w, flags=SAE_FLAGS | extra_flags)
     h = w.hidden.clone()
@@ -242,11 +242,13 @@ def extras_sae(name, w, peaks, mixlib, extra_flags=0):
         if a is not None and a.kind == W.KIND_SAE:
             counts[a.group] = counts.get(a.group, 0) + 1
     flops = sum(2.0 * n * w.d_model * w.groups[g].d_sae for g, n in counts.items())
-    wbytes = sum(2.0 * w.d_model * w.groups[g].d_sae for g in counts)
+    wbytes = sum(w_enc_bytes_per_el * w.d_model * w.groups[g].d_sae for g in counts)
     enc_s = st["encode"] * 1e-3
     status = m.get_status()
     m.destroy()
-    return {"workload": name, "w_enc_layout": "tile-contiguous copy" if SAE_FLAGS & 2 else "as registered",
+    layout = "8-bit E4M3 codes, tile-ordered copy" if extra_flags & 32 else (
+        "tile-contiguous copy" if SAE_FLAGS & 2 else "as registered")
+    return {"workload": name, "w_enc_layout": layout,
             "t_call_ms_graph": min(times), "stage_ms": st, "sae_rows_per_group": counts,
             "encode_tflops": flops / enc_s / 1e12, "encode_frac_bf16_peak": flops / enc_s / 1e12 / peaks["bf16_tflops"],
             "encode_weight_stream_gbs": wbytes / enc_s / 1e9,
@@ -354,6 +356,16 @@ def run_workload(args):
         out = extras_sweep(peaks, mixlib)
     elif name == "sae_heavy":
         out = extras_sae("sae_heavy (config 2)", W.make_sae_heavy("cuda"), peaks, mixlib)
+    elif name == "sae_heavy_fp8":   # config 2 with the encoder as 8-bit codes (MIX_FLAG_FP8_W_ENC)
+        out = extras_sae("sae_heavy (config 2), 8-bit encoder", W.make_sae_heavy("cuda", fp8=True), peaks, mixlib,
+                         extra_flags=32, w_enc_bytes_per_el=1.0)
+    elif name == "mixed_fp8":
+        out = extras_sae("mixed (config 3), 8-bit encoder", W.make_mixed("cuda", fp8=True), peaks, mixlib,
+                         extra_flags=32, w_enc_bytes_per_el=1.0)
+    elif name == "sae_small_fp8":   # profiling case for the 8-bit encoder
+        out = extras_sae("sae_small, 8-bit encoder (d=4096, d_sae=16384, 2 sets, T=256)",
+                         W.make_sae_heavy("cuda", d_sae=16384, T=256, R=16, G=2, fp8=True), peaks, mixlib,
+                         extra_flags=32, w_enc_bytes_per_el=1.0)
     elif name == "sae_small":     # profiling case: weights (256 MiB) exceed L2, < 1 GiB on the device
         out = extras_sae("sae_small (d=4096, d_sae=16384, 2 sets, T=256)",
                          W.make_sae_heavy("cuda", d_sae=16384, T=256, R=16, G=2), peaks, mixlib)
@@ -623,7 +635,7 @@ def main():
     ap.add_argument("--no-retile", action="store_true",
                     help="SAE contexts stream W_enc as registered instead of a tile-contiguous copy (MIX_FLAG_RETILE_W_ENC)")
     ap.add_argument("--workload", default="decode",
-                    help="decode (the contract line) | sweep | sae_heavy | sae_small | mixed | mixed_small | conditional | conditional_small | replay")
+                    help="decode (the contract line) | sweep | sae_heavy | sae_heavy_fp8 | sae_small | sae_small_fp8 | mixed | mixed_fp8 | mixed_small | conditional | conditional_small | replay")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     args = ap.parse_args()
     if args.no_retile:

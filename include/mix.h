@@ -97,7 +97,15 @@ enum {
                                          mix_apply.  Probes and steering then run in one kernel that keeps the row in
                                          registers across the apps of its chain, and the SAE chain starts only after
                                          that kernel (the two no longer overlap).  Not together with
-                                         MIX_FLAG_SAE_EDIT_ONLY */
+                                         MIX_FLAG_SAE_EDIT_ONLY */,
+  MIX_FLAG_FP8_W_ENC = 1u << 5        /* every weight set of the context gives its encoder as 8-bit E4M3 codes with one
+                                         fp32 scale per feature (mix_sae_weights.W_enc / W_enc_scale): the encoder takes
+                                         half the HBM and the encode streams half the bytes; the hidden state stays bf16
+                                         (the codes are widened to bf16 in shared memory, exactly, before the tensor-core
+                                         contraction) and the scale is applied to the fp32 accumulator.  A memory option:
+                                         the widening costs more time than the halved stream saves.  The paper has no
+                                         counterpart.  Not together with MIX_FLAG_ENCODE_SIMT, MIX_FLAG_SAE_EDIT_ONLY or
+                                         center_input */
 };
 
 typedef struct {
@@ -148,7 +156,13 @@ typedef struct {
    theta fp32 [d_sae] (JumpReLU only, else NULL).  W_dec bf16 [d_sae, d]: row j = decoder
    direction j.  b_dec fp32 [d] or NULL.  center_input != 0 subtracts b_dec from the input
    before the encoder (folded into an effective bias at registration; needs b_dec).
-   k: TopK only, 1 <= k <= min(k_max, d_sae). */
+   k: TopK only, 1 <= k <= min(k_max, d_sae).
+   In a context created with MIX_FLAG_FP8_W_ENC, W_enc is uint8 [d_sae, d] instead: E4M3 codes
+   (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; the NaN codes 0x7F / 0xFF must not
+   occur), and W_enc_scale fp32 [d_sae] is required: encoder entry (j, i) = e4m3(code[j, i]) *
+   W_enc_scale[j].  The library keeps its own tile-ordered copy of the codes (d_sae * d bytes);
+   W_enc need not stay alive after registration, W_enc_scale must.  Otherwise W_enc_scale is
+   ignored. */
 typedef struct {
   long long d_sae;
   int act;
@@ -159,6 +173,7 @@ typedef struct {
   const void* W_dec;
   const float* b_dec;
   int center_input;
+  const float* W_enc_scale;
 } mix_sae_weights;
 
 /* One SAE app slot = (weight set, edit list, error-term flag).  idx/val/mode are HOST arrays

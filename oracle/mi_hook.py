@@ -126,14 +126,21 @@ def gate_open(gate, t: int) -> bool:
 # ---------------------------------------------------------------------------
 # SAE function
 # ---------------------------------------------------------------------------
-def e4m3_to_f64(codes: np.ndarray) -> np.ndarray:
-    """Value of 8-bit E4M3 codes (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; no
-    infinities, S.1111.111 is NaN): +-2^(e-7) (1 + m/8) for e > 0, +-2^-6 (m/8) for e = 0."""
-    c = np.asarray(codes, dtype=np.uint8).astype(np.int64)
+def _e4m3_value(c: np.ndarray) -> np.ndarray:
+    c = np.asarray(c, dtype=np.int64)
     e, m = (c >> 3) & 0xF, c & 0x7
     mag = np.where(e == 0, (m / 8.0) * 2.0 ** -6, (1.0 + m / 8.0) * np.exp2((e - 7).astype(np.float64)))
     mag = np.where((e == 15) & (m == 7), np.nan, mag)
     return np.where(c & 0x80, -mag, mag)
+
+
+_E4M3_VALUES = _e4m3_value(np.arange(256))      # the definition, evaluated once for each of the 256 codes
+
+
+def e4m3_to_f64(codes: np.ndarray) -> np.ndarray:
+    """Value of 8-bit E4M3 codes (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; no
+    infinities, S.1111.111 is NaN): +-2^(e-7) (1 + m/8) for e > 0, +-2^-6 (m/8) for e = 0."""
+    return _E4M3_VALUES[np.asarray(codes, dtype=np.uint8)]
 
 
 def encoder_rows_f64(W_enc_bits: np.ndarray, w_scale: Optional[np.ndarray] = None) -> np.ndarray:

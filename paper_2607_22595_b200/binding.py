@@ -26,6 +26,7 @@ MIX_FLAG_RETILE_W_ENC = 2
 MIX_FLAG_TEST_STALL_ENCODE = 4
 MIX_FLAG_SAE_EDIT_ONLY = 8
 MIX_FLAG_SLOT_CHAINS = 16
+MIX_FLAG_FP8_W_ENC = 32
 
 EXPORTS = [
     "mix_create", "mix_destroy", "mix_last_error", "mix_register_sae_weights", "mix_unregister_sae_weights",
@@ -56,7 +57,7 @@ class MixRouter(C.Structure):
 class MixSaeWeights(C.Structure):
     _fields_ = [("d_sae", C.c_longlong), ("act", C.c_int), ("k", C.c_int), ("W_enc", C.c_void_p),
                 ("b_enc", C.c_void_p), ("theta", C.c_void_p), ("W_dec", C.c_void_p), ("b_dec", C.c_void_p),
-                ("center_input", C.c_int)]
+                ("center_input", C.c_int), ("W_enc_scale", C.c_void_p)]
 
 
 class MixSaeApp(C.Structure):
@@ -162,11 +163,12 @@ class Mix:
             pass
 
     def register_sae_weights(self, group, d_sae, act, k, W_enc, b_enc, W_dec, theta=None, b_dec=None,
-                             center_input=False, stream=None):
+                             center_input=False, w_scale=None, stream=None):
+        """W_enc: bf16 [d_sae, d]; in a MIX_FLAG_FP8_W_ENC context uint8 E4M3 codes with w_scale fp32 [d_sae]."""
         w = MixSaeWeights(int(d_sae), int(act), int(k), _ptr(W_enc), _ptr(b_enc), _ptr(theta), _ptr(W_dec),
-                          _ptr(b_dec), int(bool(center_input)))
+                          _ptr(b_dec), int(bool(center_input)), _ptr(w_scale))
         self._check(self.lib.mix_register_sae_weights(self.ctx, group, C.byref(w), _stream(stream)))
-        self._keep[("g", group)] = (W_enc, b_enc, W_dec, theta, b_dec)
+        self._keep[("g", group)] = (W_enc, b_enc, W_dec, theta, b_dec, w_scale)
 
     def unregister_sae_weights(self, group, stream=None):
         self._check(self.lib.mix_unregister_sae_weights(self.ctx, group, _stream(stream)))

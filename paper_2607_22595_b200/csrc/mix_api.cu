@@ -41,6 +41,18 @@ int load_encode_fn() {
 }
 
 // bf16 [rows, d] row-major; box = kTileK columns x box_rows rows; 128-byte swizzle.
+// 8-bit encoder tiles: rows of 64 bytes, plain (unswizzled) boxes of 256 rows
+int make_tmap_u8(CUtensorMap* out, const void* base, unsigned long long rows) {
+  cuuint64_t dims[2] = {(cuuint64_t)kTileK, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)kTileK};
+  cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)kTileN};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = g_encode(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? MIX_OK : MIX_ERR_CUDA;
+}
+
 int make_tmap(CUtensorMap* out, const void* base, unsigned long long rows, int d, int box_rows) {
   cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)d * 2};
@@ -171,6 +183,7 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
     if (chunks * 32 * cfg->n_groups_max * 4 > 40 * 1024) return MIX_ERR_UNSUPPORTED;
   }
   if ((cfg->flags & MIX_FLAG_SLOT_CHAINS) && (cfg->flags & MIX_FLAG_SAE_EDIT_ONLY)) return MIX_ERR_INVALID_ARG;
+  if ((cfg->flags & MIX_FLAG_FP8_W_ENC) && (cfg->flags & (MIX_FLAG_ENCODE_SIMT | MIX_FLAG_SAE_EDIT_ONLY))) return MIX_ERR_INVALID_ARG;
   mix_ctx* c = static_cast<mix_ctx*>(calloc(1, sizeof(mix_ctx)));
   if (!c) return MIX_ERR_NO_MEMORY;
   c->cfg = *cfg;
@@ -286,6 +299,9 @@ int mix_register_sae_weights(mix_ctx* c, int group, const mix_sae_weights* w, vo
   if (w->act == MIX_SAE_TOPK && (w->k < 1 || w->k > c->cfg.k_max || w->k > w->d_sae))
     MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "k %d outside [1, min(k_max=%d, d_sae)]", w->k, c->cfg.k_max);
   if (w->center_input && !w->b_dec) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "center_input needs b_dec");
+  const bool fp8 = (c->cfg.flags & MIX_FLAG_FP8_W_ENC) != 0;
+  if (fp8 && (!w->W_enc_scale || w->center_input))
+    MIX_FAIL(c, MIX_ERR_INVALID_ARG, "an 8-bit encoder needs W_enc_scale and does not take center_input");
 
   GroupEntry ge;
   memset(&ge, 0, sizeof(ge));
@@ -293,7 +309,8 @@ int mix_register_sae_weights(mix_ctx* c, int group, const mix_sae_weights* w, vo
   ge.act = w->act;
   ge.k = w->act == MIX_SAE_TOPK ? w->k : 0;
   ge.d_sae = w->d_sae;
-  ge.W_enc = static_cast<const __nv_bfloat16*>(w->W_enc);
+  ge.W_enc = fp8 ? nullptr : static_cast<const __nv_bfloat16*>(w->W_enc);
+  ge.w_scale = fp8 ? w->W_enc_scale : nullptr;
   ge.b_eff = w->b_enc;
   ge.theta = w->theta;
   ge.W_dec = static_cast<const __nv_bfloat16*>(w->W_dec);
@@ -310,7 +327,19 @@ int mix_register_sae_weights(mix_ctx* c, int group, const mix_sae_weights* w, vo
   }
   if (!(c->cfg.flags & MIX_FLAG_ENCODE_SIMT)) {
     CUtensorMap tm;
-    if (c->cfg.flags & MIX_FLAG_RETILE_W_ENC) {
+    if (fp8) {
+      // library-owned tile-ordered copy of the codes: [S/256][d/64][256][64] bytes, seen by TMA as a 64-byte-wide matrix
+      if (c->owned_w_tiled[group]) { cudaStreamSynchronize(s); cudaFree(c->owned_w_tiled[group]); c->owned_w_tiled[group] = nullptr; }
+      const size_t n_el = (size_t)w->d_sae * c->cfg.d_model;
+      if (cudaMalloc(reinterpret_cast<void**>(&c->owned_w_tiled[group]), n_el) != cudaSuccess) {
+        cudaGetLastError();
+        MIX_FAIL(c, MIX_ERR_NO_MEMORY, "cannot allocate the tile-ordered copy of the 8-bit W_enc");
+      }
+      unsigned char* tiled = reinterpret_cast<unsigned char*>(c->owned_w_tiled[group]);
+      MIX_CUDA(c, launch_retile_fp8(static_cast<const unsigned char*>(w->W_enc), tiled, w->d_sae, c->cfg.d_model, s));
+      if (make_tmap_u8(&tm, tiled, (unsigned long long)(n_el / kTileK)) != MIX_OK)
+        MIX_FAIL(c, MIX_ERR_CUDA, "cuTensorMapEncodeTiled failed for the 8-bit W_enc");
+    } else if (c->cfg.flags & MIX_FLAG_RETILE_W_ENC) {
       // library-owned tile-contiguous copy: [S/256][d/64][256][64], seen by TMA as a 64-column matrix
       if (c->owned_w_tiled[group]) { cudaStreamSynchronize(s); cudaFree(c->owned_w_tiled[group]); c->owned_w_tiled[group] = nullptr; }
       const size_t n_el = (size_t)w->d_sae * c->cfg.d_model;

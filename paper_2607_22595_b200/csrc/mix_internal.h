@@ -63,6 +63,8 @@ struct __align__(16) GroupEntry {
   const float* theta;
   const __nv_bfloat16* W_dec;
   const float* b_dec;
+  const float* w_scale; // 8-bit encoder: per-feature scale of the E4M3 codes, else null
+  const void* pad2_;
 };
 
 // What decode_kernel leaves for decode_delta_kernel about one packed row that keeps the error term.
@@ -170,6 +172,7 @@ cudaError_t launch_compose_map(const Ctx* c, int T_live, int n_req, cudaStream_t
 cudaError_t launch_fold_bias(const __nv_bfloat16* W_enc, const float* b_enc, const float* b_dec, float* b_eff,
                              long long d_sae, int d, cudaStream_t s);
 cudaError_t launch_retile(const __nv_bfloat16* W_enc, __nv_bfloat16* W_tiled, long long d_sae, int d, cudaStream_t s);
+cudaError_t launch_retile_fp8(const unsigned char* W_enc, unsigned char* W_tiled, long long d_sae, int d, cudaStream_t s);
 cudaError_t encode_tc_prepare();   // opt in to the large dynamic shared memory size
 
 }  // namespace mix

@@ -11,24 +11,46 @@
 // largest values per row plus its 9th, which the merge step turns into the exact TopK).
 // No TMA multicast and no clusters.  Every wait is bounded: on expiry the CTA raises
 // MIX_STATUS_WAIT_TIMEOUT, lets its copies land, frees its tensor memory and returns.
+//
+// 8-bit encoder (kFp8): the W_enc tile arrives as 256 x 64 E4M3 codes (16 KiB, half the bytes);
+// warps 6..13 (two teams on alternate k-blocks) widen it to bf16 -- exactly: every E4M3 value is
+// a bf16 value -- into the same 128-byte-swizzled layout TMA would have produced, and only then
+// is the k-block handed to the MMA warp; the per-feature scale is applied to the fp32
+// accumulator in the epilogue.  The copies land in a ring of 5 stages of 32 KiB (panel 16,
+// codes 16) and the widened tiles go through a separate ring of two 32 KiB slots.  This form
+// halves the encoder's footprint in HBM but is NOT faster than the bf16 form: the widening adds
+// 48 KiB of load/store traffic per k-block to a shared memory that the copies (32 KiB) and the
+// tensor core's operand reads (48 KiB) already keep busy, and the widening warps wait on it.
 #include "mix_internal.h"
 
 namespace mix {
 
 namespace {
 
-constexpr int kStages = 4;
+constexpr int kMaxStages = 5;
+constexpr int kBRing = 2;                      // 8-bit encoder: widened W_enc tiles in flight between the widening warps and the MMA
 constexpr int kABytes = kTileM * kTileK * 2;   // 16 KiB
 constexpr int kBBytes = kTileN * kTileK * 2;   // 32 KiB
-constexpr int kStageBytes = kABytes + kBBytes;
-constexpr int kTcThreads = 192;
+constexpr int kRawBytes = kTileN * kTileK;     // 16 KiB of E4M3 codes (8-bit encoder only)
+constexpr int kConvWarps = 4;                  // warps per widening team (8-bit encoder only)
+constexpr int kConvTeams = 2;                  // team g (warps 6 + 4g ..) widens every k-block with index = g mod 2, into slot g
+template <bool kFp8> struct TcCfg {
+  static constexpr int kStages = kFp8 ? 5 : 4;
+  static constexpr int kStageBytes = kABytes + (kFp8 ? kRawBytes : kBBytes);
+  static constexpr int kRingBytes = kStages * kStageBytes + (kFp8 ? kBRing * kBBytes : 0);
+  static constexpr int kThreads = 192 + (kFp8 ? kConvTeams * kConvWarps * 32 : 0);
+  static constexpr int kSmemBytes = kRingBytes + 1024 /* alignment slack */ + 1024 /* TcShared */;
+  static_assert(kSmemBytes <= 227 * 1024, "shared memory per CTA");
+};
 constexpr int kTmemCols = 512;                 // two 128 x 256 fp32 accumulators
 constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz
 constexpr long long kWaitCyclesTest = 2000000ll;  // ~1 ms: the cap under MIX_FLAG_TEST_STALL_ENCODE
 
 struct __align__(8) TcShared {
-  unsigned long long full[kStages];
-  unsigned long long empty[kStages];
+  unsigned long long full[kMaxStages];
+  unsigned long long empty[kMaxStages];
+  unsigned long long conv[kBRing];        // 8-bit encoder: slot holds a widened W_enc tile
+  unsigned long long b_empty[kBRing];     // 8-bit encoder: the MMAs that read the slot are done
   unsigned long long tmem_full[2];
   unsigned long long tmem_empty[2];
   unsigned tmem_base;
@@ -36,7 +58,7 @@ struct __align__(8) TcShared {
   long long wait_cycles;      // cap of every bounded wait in this launch
   RouteState rs;
 };
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + (int)sizeof(TcShared);
+static_assert(sizeof(TcShared) <= 1024, "TcShared must fit the space reserved for it");
 
 __device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
 
@@ -178,17 +200,40 @@ __device__ __forceinline__ void top9_insert(float (&tv)[kCandPerTile + 1], int (
   }
 }
 
-__global__ void __launch_bounds__(kTcThreads, 1)
+// Four packed E4M3 codes -> four bf16 values, exactly, without conversion instructions (those
+// run at a fraction of the ALU rate and would make the widening the bottleneck).  A code byte
+// s.eeee.mmm placed as s.0000eeee.mmm0000 IS the bf16 number 2^-120 times the code's value --
+// bf16 has 8 exponent bits, so the 4-bit exponent field and the 3 mantissa bits drop into place,
+// and the codes with e = 0 become bf16 subnormals with the right value -- and one bf16x2
+// multiplication by 2^120 (exact: a power of two, result in range) finishes the job.
+__device__ __forceinline__ void e4m3x4_to_bf16x4(unsigned w, unsigned& lo, unsigned& hi) {
+  const unsigned t0 = __byte_perm(w, 0u, 0x1404);        // (b1 << 24) | (b0 << 8)
+  const unsigned t1 = __byte_perm(w, 0u, 0x3424);        // (b3 << 24) | (b2 << 8)
+  const unsigned u0 = (t0 & 0x80008000u) | ((t0 >> 4) & 0x07f007f0u);
+  const unsigned u1 = (t1 & 0x80008000u) | ((t1 >> 4) & 0x07f007f0u);
+  const unsigned k2 = 0x7B807B80u;                        // bf16 2^120, twice
+  const __nv_bfloat162 r0 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&u0), *reinterpret_cast<const __nv_bfloat162*>(&k2));
+  const __nv_bfloat162 r1 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&u1), *reinterpret_cast<const __nv_bfloat162*>(&k2));
+  lo = *reinterpret_cast<const unsigned*>(&r0);
+  hi = *reinterpret_cast<const unsigned*>(&r1);
+}
+
+template <bool kFp8>
+__global__ void __launch_bounds__(TcCfg<kFp8>::kThreads, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorMap* __restrict__ tmap_w,
                  const RouteState* __restrict__ rs_g, const GroupEntry* __restrict__ groups, int n_groups,
                  float* __restrict__ Z, long long ldz, int d, unsigned* __restrict__ status, int mode,
                  const int* __restrict__ mtile_flag, const int* __restrict__ n_flagged, float* __restrict__ cand_val,
                  int* __restrict__ cand_idx, float* __restrict__ cand_ninth, int cand_tiles, int w_tiled, int test_stall) {
+  constexpr int kStages = TcCfg<kFp8>::kStages;
+  constexpr int kStageBytes = TcCfg<kFp8>::kStageBytes;
+  constexpr int kTcThreads = TcCfg<kFp8>::kThreads;
   if (mode == 1 && *n_flagged == 0) return;
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment: required by the 128-byte swizzle atoms
   unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  TcShared* sh = reinterpret_cast<TcShared*>(tiles + kStages * kStageBytes);
+  TcShared* sh = reinterpret_cast<TcShared*>(tiles + TcCfg<kFp8>::kRingBytes);
+  unsigned char* bring = tiles + kStages * kStageBytes;      // 8-bit encoder: the ring of widened tiles
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   for (int i = threadIdx.x; i < (int)(sizeof(RouteState) / sizeof(int)); i += kTcThreads)
@@ -197,6 +242,10 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&sh->full[s]), 1);
       mbar_init(smem_u32(&sh->empty[s]), 1);
+    }
+    for (int j = 0; j < kBRing; ++j) {
+      mbar_init(smem_u32(&sh->conv[j]), kConvWarps);
+      mbar_init(smem_u32(&sh->b_empty[j]), 1);
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&sh->tmem_full[a]), 1);
@@ -238,12 +287,14 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
           // bounded wait runs out and the whole CTA leaves through the time-out path.
           if (test_stall) { ok = false; break; }
           const unsigned bar = smem_u32(&sh->full[stage]);
-          mbar_expect_tx(bar, kStageBytes);
+          mbar_expect_tx(bar, kFp8 ? kABytes + kRawBytes : kABytes + kBBytes);
           const unsigned sa = smem_u32(tiles + stage * kStageBytes);
           tma_load_2d(sa, &tmap_panel, kb * kTileK, t.m_tile_global * kTileM, bar);
           // W_enc tile: rows n_tile*256.. of the row-major matrix, or -- when the weights were re-laid
           // out at registration -- block (n_tile, kb) of the tile-contiguous copy [S/256][d/64][256][64]
-          if (w_tiled)
+          if (kFp8)   // block (n_tile, kb) of the tile-ordered codes, into the stage's staging area
+            tma_load_2d(sa + kABytes, tw, 0, (t.n_tile * num_kb + kb) * kTileN, bar);
+          else if (w_tiled)
             tma_load_2d(sa + kABytes, tw, 0, (t.n_tile * num_kb + kb) * kTileN, bar);
           else
             tma_load_2d(sa + kABytes, tw, kb * kTileK, t.n_tile * kTileN, bar);
@@ -253,8 +304,8 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      int stage = 0;
-      unsigned phase = 0, acc = 0, acc_phase = 0;
+      int stage = 0, bs = 0;
+      unsigned phase = 0, bphase = 0, acc = 0, acc_phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
         if (mode != 0 && !tile_wanted(decode_tile(sh->rs, groups, n_groups, tile), groups, mode, mtile_flag)) continue;
@@ -262,20 +313,77 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
         tc_fence_after();
         const unsigned d_tmem = tmem_base + acc * kTileN;
         for (int kb = 0; kb < num_kb; ++kb) {
-          if (!mbar_wait(smem_u32(&sh->full[stage]), phase, sh, status)) { ok = false; break; }
+          // 8-bit encoder: the widening warps waited for the stage's copies and arrive on conv[] after
+          // their bf16 tile is visible to the tensor core's (async-proxy) reads
+          if (!mbar_wait(smem_u32(kFp8 ? &sh->conv[bs] : &sh->full[stage]), kFp8 ? bphase : phase, sh, status)) { ok = false; break; }
           tc_fence_after();
           const unsigned sa = smem_u32(tiles + stage * kStageBytes);
-          const unsigned long long da = umma_desc(sa), db = umma_desc(sa + kABytes);
+          const unsigned sb = kFp8 ? smem_u32(bring + bs * kBBytes) : sa + kABytes;
+          const unsigned long long da = umma_desc(sa), db = umma_desc(sb);
 #pragma unroll
           for (int k = 0; k < kTileK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per step
             umma(d_tmem, da + 2ull * k, db + 2ull * k, (unsigned)((kb | k) != 0));
           umma_commit(smem_u32(&sh->empty[stage]));
+          if (kFp8) {
+            umma_commit(smem_u32(&sh->b_empty[bs]));
+            bs ^= 1;
+            if (bs == 0) bphase ^= 1u;
+          }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
         umma_commit(smem_u32(&sh->tmem_full[acc]));
         acc ^= 1u;
         if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+  } else if (kFp8 && warp >= 6) {
+    // widen the stage's 256 x 64 codes to bf16.  Thread c of 128 takes the 16-byte pieces c, c + 128, ...
+    // (piece = row * 4 + quarter of the row): 16 codes in, two 16-byte chunks of the row's 128 bytes out,
+    // stored where the 128-byte swizzle puts them (chunk index XOR row mod 8).
+    // Two teams of four warps take alternate k-blocks (team = slot of the widened-tile ring), so one
+    // team's stores and proxy fence overlap the other team's arithmetic.
+    const int team = (warp - 6) / kConvWarps;
+    const int ct = threadIdx.x - (6 + team * kConvWarps) * 32;
+    int stage = 0, bs = 0;
+    unsigned phase = 0, bphase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      if (mode != 0 && !tile_wanted(decode_tile(sh->rs, groups, n_groups, tile), groups, mode, mtile_flag)) continue;
+      for (int kb = 0; kb < num_kb; ++kb) {
+        if (bs != team) {                      // the other team's k-block
+          bs ^= 1;
+          if (bs == 0) bphase ^= 1u;
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          continue;
+        }
+        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&sh->full[stage]), phase, sh, status))) { ok = false; break; }
+        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&sh->b_empty[bs]), bphase ^ 1u, sh, status))) { ok = false; break; }
+        const uint4* raw = reinterpret_cast<const uint4*>(tiles + stage * kStageBytes + kABytes);
+        unsigned char* bt = bring + bs * kBBytes;
+        constexpr int kPieces = kTileN * 4 / (kConvWarps * 32);    // 16-byte pieces of codes per thread: 8
+        uint4 in[kPieces];
+#pragma unroll
+        for (int it = 0; it < kPieces; ++it) in[it] = raw[it * (kConvWarps * 32) + ct];   // all loads first
+#pragma unroll
+        for (int it = 0; it < kPieces; ++it) {
+          const int piece = it * (kConvWarps * 32) + ct;
+          const int r = piece >> 2, qr = piece & 3;
+          uint4 lo, hi;
+          e4m3x4_to_bf16x4(in[it].x, lo.x, lo.y);
+          e4m3x4_to_bf16x4(in[it].y, lo.z, lo.w);
+          e4m3x4_to_bf16x4(in[it].z, hi.x, hi.y);
+          e4m3x4_to_bf16x4(in[it].w, hi.z, hi.w);
+          unsigned char* row = bt + r * 128;
+          *reinterpret_cast<uint4*>(row + (((2 * qr) ^ (r & 7)) << 4)) = lo;
+          *reinterpret_cast<uint4*>(row + (((2 * qr + 1) ^ (r & 7)) << 4)) = hi;
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> async-proxy reads
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&sh->conv[bs]));
+        bs ^= 1;
+        if (bs == 0) bphase ^= 1u;
+        if (++stage == kStages) { stage = 0; phase ^= 1u; }
       }
     }
   } else {
@@ -291,6 +399,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
       const bool valid = row_local < t.rows_valid;
       const size_t p = (size_t)t.m_tile_global * kTileM + row_local;
       const float* bias = groups[t.group].b_eff + (size_t)t.n_tile * kTileN;
+      const float* wsc = kFp8 ? groups[t.group].w_scale + (size_t)t.n_tile * kTileN : nullptr;
       const unsigned taddr = tmem_base + ((unsigned)(q * 32) << 16) + acc * kTileN;
       if (mode == 0 && groups[t.group].act == MIX_SAE_TOPK) {
         float tv[kCandPerTile + 1];
@@ -307,10 +416,12 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
 #pragma unroll
           for (int i = 0; i < 32; i += 4) {
             const float4 b4 = __ldg(reinterpret_cast<const float4*>(bias + c + i));
-            top9_insert(tv, ti, v[i] + b4.x, c + i);
-            top9_insert(tv, ti, v[i + 1] + b4.y, c + i + 1);
-            top9_insert(tv, ti, v[i + 2] + b4.z, c + i + 2);
-            top9_insert(tv, ti, v[i + 3] + b4.w, c + i + 3);
+            float4 s4 = make_float4(1.f, 1.f, 1.f, 1.f);
+            if (kFp8) s4 = __ldg(reinterpret_cast<const float4*>(wsc + c + i));
+            top9_insert(tv, ti, kFp8 ? fmaf(v[i], s4.x, b4.x) : v[i] + b4.x, c + i);
+            top9_insert(tv, ti, kFp8 ? fmaf(v[i + 1], s4.y, b4.y) : v[i + 1] + b4.y, c + i + 1);
+            top9_insert(tv, ti, kFp8 ? fmaf(v[i + 2], s4.z, b4.z) : v[i + 2] + b4.z, c + i + 2);
+            top9_insert(tv, ti, kFp8 ? fmaf(v[i + 3], s4.w, b4.w) : v[i + 3] + b4.w, c + i + 3);
           }
         }
         if (valid) {
@@ -334,11 +445,13 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
 #pragma unroll
             for (int i = 0; i < 32; i += 4) {
               const float4 b4 = __ldg(reinterpret_cast<const float4*>(bias + c + i));
+              float4 s4 = make_float4(1.f, 1.f, 1.f, 1.f);
+              if (kFp8) s4 = __ldg(reinterpret_cast<const float4*>(wsc + c + i));
               float4 o;
-              o.x = v[i] + b4.x;
-              o.y = v[i + 1] + b4.y;
-              o.z = v[i + 2] + b4.z;
-              o.w = v[i + 3] + b4.w;
+              o.x = kFp8 ? fmaf(v[i], s4.x, b4.x) : v[i] + b4.x;
+              o.y = kFp8 ? fmaf(v[i + 1], s4.y, b4.y) : v[i + 1] + b4.y;
+              o.z = kFp8 ? fmaf(v[i + 2], s4.z, b4.z) : v[i + 2] + b4.z;
+              o.w = kFp8 ? fmaf(v[i + 3], s4.w, b4.w) : v[i + 3] + b4.w;
               *reinterpret_cast<float4*>(out + c + i) = o;
             }
           }
@@ -380,7 +493,29 @@ __global__ void retile_kernel(const uint4* __restrict__ src, uint4* __restrict__
   dst[i] = src[((n_tile * kTileN + r) * (long long)d + (long long)kb * kTileK) / 8 + piece];
 }
 
+// The same for 8-bit codes: [S, d] bytes -> [S/256][d/64][256][64] bytes, one thread per 16 bytes.
+__global__ void retile_fp8_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, long long d_sae, int d) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int num_kb = d / kTileK;
+  const long long total = d_sae * (long long)d / 16;
+  if (i >= total) return;
+  const int piece = (int)(i & 3);                       // 4 pieces per 64-byte row
+  const long long row_in_all = i >> 2;
+  const int r = (int)(row_in_all % kTileN);
+  const long long blk = row_in_all / kTileN;
+  const int kb = (int)(blk % num_kb);
+  const long long n_tile = blk / num_kb;
+  dst[i] = src[((n_tile * kTileN + r) * (long long)d + (long long)kb * kTileK) / 16 + piece];
+}
+
 }  // namespace
+
+cudaError_t launch_retile_fp8(const unsigned char* W_enc, unsigned char* W_tiled, long long d_sae, int d, cudaStream_t s) {
+  const long long total = d_sae * (long long)d / 16;
+  retile_fp8_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(reinterpret_cast<const uint4*>(W_enc),
+                                                                    reinterpret_cast<uint4*>(W_tiled), d_sae, d);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_retile(const __nv_bfloat16* W_enc, __nv_bfloat16* W_tiled, long long d_sae, int d, cudaStream_t s) {
   const long long total = d_sae * (long long)d / 8;
@@ -390,17 +525,26 @@ cudaError_t launch_retile(const __nv_bfloat16* W_enc, __nv_bfloat16* W_tiled, lo
 }
 
 cudaError_t encode_tc_prepare() {
-  return cudaFuncSetAttribute(encode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(encode_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       TcCfg<false>::kSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(encode_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<true>::kSmemBytes);
+  return e;
 }
 
 cudaError_t launch_encode_tc(const Ctx* c, int mode, cudaStream_t s) {
-  encode_tc_kernel<<<c->n_sms, kTcThreads, kSmemBytes, s>>>(c->tmap_panel, c->d_tmap_w, c->d_route, c->d_groups,
-                                                             c->cfg.n_groups_max, c->d_z, c->cfg.d_sae_max,
-                                                             c->cfg.d_model, c->d_status, mode, c->d_mtile_flag,
-                                                             c->d_n_flagged, c->d_cand_val, c->d_cand_idx,
-                                                             c->d_cand_ninth, c->cand_tiles,
-                                                             (c->cfg.flags & MIX_FLAG_RETILE_W_ENC) ? 1 : 0,
-                                                             (c->cfg.flags & MIX_FLAG_TEST_STALL_ENCODE) ? 1 : 0);
+  const int w_tiled = (c->cfg.flags & MIX_FLAG_RETILE_W_ENC) ? 1 : 0;
+  const int stall = (c->cfg.flags & MIX_FLAG_TEST_STALL_ENCODE) ? 1 : 0;
+  if (c->cfg.flags & MIX_FLAG_FP8_W_ENC)
+    encode_tc_kernel<true><<<c->n_sms, TcCfg<true>::kThreads, TcCfg<true>::kSmemBytes, s>>>(
+        c->tmap_panel, c->d_tmap_w, c->d_route, c->d_groups, c->cfg.n_groups_max, c->d_z, c->cfg.d_sae_max, c->cfg.d_model,
+        c->d_status, mode, c->d_mtile_flag, c->d_n_flagged, c->d_cand_val, c->d_cand_idx, c->d_cand_ninth, c->cand_tiles,
+        w_tiled, stall);
+  else
+    encode_tc_kernel<false><<<c->n_sms, TcCfg<false>::kThreads, TcCfg<false>::kSmemBytes, s>>>(
+        c->tmap_panel, c->d_tmap_w, c->d_route, c->d_groups, c->cfg.n_groups_max, c->d_z, c->cfg.d_sae_max, c->cfg.d_model,
+        c->d_status, mode, c->d_mtile_flag, c->d_n_flagged, c->d_cand_val, c->d_cand_idx, c->d_cand_ninth, c->cand_tiles,
+        w_tiled, stall);
   return cudaGetLastError();
 }
 

@@ -261,12 +261,12 @@ def make_decode(device="cpu", d=4096, T=256, n_probe=64, n_steer=32, seed=None):
 # config 2: SAE-heavy
 # --------------------------------------------------------------------------
 def make_sae_heavy(device="cpu", d=4096, d_sae=65536, k=64, T=512, R=32, G=4, n_edit=16,
-                   edit_hint: Optional[EditHint] = None, seed=None):
+                   edit_hint: Optional[EditHint] = None, seed=None, fp8=False):
     seed = BASE_SEED + 2000 if seed is None else seed
     g, rng = _gen(device, seed), np.random.default_rng(seed)
     hidden = _hidden(g, device, T, d)
     lengths = ragged_lengths_uniform(rng, T, R)
-    groups = {gi: make_sae_weights(g, device, d, d_sae, SAE_TOPK, k=k) for gi in range(G)}
+    groups = {gi: make_sae_weights(g, device, d, d_sae, SAE_TOPK, k=k, fp8=fp8) for gi in range(G)}
     req_slot = np.arange(R, dtype=np.int32)          # one app slot per request
     req_group = np.arange(R) % G
     order = rng.permutation(R)
@@ -289,7 +289,7 @@ def make_sae_heavy(device="cpu", d=4096, d_sae=65536, k=64, T=512, R=32, G=4, n_
 # --------------------------------------------------------------------------
 def make_mixed(device="cpu", d=5120, T=8192, R=64, d_sae=32768, C=16, n_probe=8, n_steer=8, G=2,
                n_edit=16, cap=2048, mu=5.0, b_enc_mean=-0.1,
-               edit_hint: Optional[EditHint] = None, seed=None):
+               edit_hint: Optional[EditHint] = None, seed=None, fp8=False):
     seed = BASE_SEED + 3000 if seed is None else seed
     g, rng = _gen(device, seed), np.random.default_rng(seed)
     hidden = _hidden(g, device, T, d)
@@ -303,7 +303,7 @@ def make_mixed(device="cpu", d=5120, T=8192, R=64, d_sae=32768, C=16, n_probe=8,
     for i in range(n_steer):
         apps[n_probe + i] = Steer(v=Vs[i].contiguous(), alpha=float(np.float32(alphas[i])))
     groups = {gi: make_sae_weights(g, device, d, d_sae, SAE_JUMPRELU, theta_range=(0.05, 0.3),
-                                   b_enc_mean=b_enc_mean) for gi in range(G)}
+                                   b_enc_mean=b_enc_mean, fp8=fp8) for gi in range(G)}
     # deal requests (in a seeded order) unhooked until >= 30 % of rows, rest round-robin
     deal = rng.permutation(R)
     req_kind = np.zeros(R, dtype=np.int64)           # 0 none, 1 probe, 2 steer, 3 sae

@@ -17,7 +17,7 @@ def make_context(mix_cls, w: Workload, flags: int = 0, **over):
 def install(m, w: Workload):
     for g, sw in w.groups.items():
         m.register_sae_weights(g, sw.d_sae, sw.act, sw.k, sw.W_enc, sw.b_enc, sw.W_dec, theta=sw.theta,
-                               b_dec=sw.b_dec, center_input=sw.center_input)
+                               b_dec=sw.b_dec, center_input=sw.center_input, w_scale=getattr(sw, "w_scale", None))
     for s, a in w.apps.items():
         if a.kind == KIND_PROBE:
             m.register_probe(s, a.W, a.b, a.act)
