@@ -495,3 +495,41 @@ def test_encode_timeout_path_raises_status_and_leaves_the_context_usable():
             assert np.array_equal(W.bits(h)[t], wh.hidden[t])
     m.destroy()
     check_parity(wh, run_gpu(w))                               # a fresh ordinary context works
+
+
+# ------------------------------------------------------------------ the interface's maximum sizes
+@pytest.mark.parametrize("T", [48, 2100])
+def test_maximum_width_and_class_count(T):
+    """d = 8192 (widest hidden state), 64-class softmax probes (most classes), next to 33-class ones (one more
+    than the tensor-core probe kernel takes), in the small-batch and the large-batch kernels."""
+    d = 8192
+    g = torch.Generator(device=DEV); g.manual_seed(21)
+    hidden = torch.randn((T, d), generator=g, device=DEV, dtype=torch.float32).to(torch.bfloat16)
+    mk = lambda C, act: W.Probe((torch.randn((C, d), generator=g, device=DEV) * d ** -0.5).to(torch.bfloat16),
+                                torch.randn(C, generator=g, device=DEV), act)
+    v = torch.randn(d, generator=g, device=DEV); v = (v / v.norm()).to(torch.bfloat16)
+    apps = {0: mk(64, W.ACT_SOFTMAX), 1: mk(33, W.ACT_SOFTMAX), 2: mk(32, W.ACT_NONE), 3: W.Steer(v, 3.0), 4: W.Project(v, 1.0)}
+    slot = (np.arange(T) % 6 - 1).astype(np.int32)
+    w = W.Workload("max", d, T, T, hidden, slot, apps, {}, n_slots_max=5, C_max=64)
+    out = run_gpu(w, graph=True)
+    check_parity(W.host(w), out)
+
+
+@pytest.mark.parametrize("add_error", [True, False])
+def test_maximum_k_and_edit_list(add_error):
+    """TopK with k = 1024 (largest k) and 64 edits per app (longest list, with a repeated feature), on rows
+    that span two row tiles."""
+    d, S, k, T = 256, 4096, 1024, 150
+    g = torch.Generator(device=DEV); g.manual_seed(22)
+    sae = W.make_sae_weights(g, DEV, d, S, W.SAE_TOPK, k=k)
+    hidden = torch.randn((T, d), generator=g, device=DEV, dtype=torch.float32).to(torch.bfloat16)
+    rng = np.random.default_rng(22)
+    idx = rng.choice(S, size=64, replace=False).astype(np.int32); idx[63] = idx[0]
+    val = rng.uniform(0.5, 4.0, size=64).astype(np.float32)
+    mode = (np.arange(64) % 3 == 0).astype(np.uint8)
+    app = W.SaeApp(0, idx, val, mode, add_error)
+    w = W.Workload("maxk", d, T, T, hidden, np.zeros(T, dtype=np.int32), {0: app}, {0: sae}, n_slots_max=1,
+                   n_groups_max=1, C_max=1, k_max=k, r_max=64, d_sae_max=S)
+    out = run_gpu(w)
+    check_parity(W.host(w), out, expect_status=None)
+    assert out["status"] & ~_mixlib().MIX_STATUS_TOPK_GENERAL == 0
