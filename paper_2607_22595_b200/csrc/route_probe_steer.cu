@@ -255,8 +255,10 @@ probe_steer_kernel(const int* __restrict__ token_slot, const int* __restrict__ n
   __shared__ float s_logit[kWarpsPerBlock][kMaxClasses];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t = blockIdx.x * kWarpsPerBlock + warp;
-  if (t >= min(T, __ldg(n_live_p))) return;
-  const RowApp a = lookup(__ldg(token_slot + t), t, apps, gates, n_slots, status, lane == 0);
+  const int n_live = __ldg(n_live_p);            // issued together with the slot id: one round trip, not two
+  const int slot = t < T ? __ldg(token_slot + t) : -1;
+  if (t >= min(T, n_live)) return;
+  const RowApp a = lookup(slot, t, apps, gates, n_slots, status, lane == 0);
   if (a.kind == 0) return;
   if (multiclass_elsewhere && a.kind == MIX_PROBE && a.C > 1 && a.C <= kCoopMaxClasses) return;
   warp_row(a, hidden, t, d, scores, C_max, s_logit[warp], lane);
@@ -425,10 +427,10 @@ probe_steer_team_kernel(const int* __restrict__ token_slot, const int* __restric
   __shared__ float s_part[NW][kMaxClasses];
   constexpr int NT = NW * 32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int t = blockIdx.x;
-  if (t >= min(T, __ldg(n_live_p))) return;
+  const int t = blockIdx.x;                      // < T_max: the slot map has an entry for every row
+  const int n_live = __ldg(n_live_p);            // both loads issue together: one round trip, not two
   const int slot = __ldg(token_slot + t);
-  if (slot == -1) return;
+  if (t >= min(T, n_live) || slot == -1) return;
   const int nvec = d >> 3;
   uint4* hrow = reinterpret_cast<uint4*>(hidden + (size_t)t * d);
   // Single-vector weights (steering, projection, one-class probe) were copied at registration
@@ -576,10 +578,10 @@ probe_steer_chain_kernel(const int* __restrict__ token_slot, const int* __restri
   __shared__ float s_part[kChainWarps][kMaxClasses];
   constexpr int NT = kChainWarps * 32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int t = blockIdx.x;
-  if (t >= min(T, __ldg(n_live_p))) return;
+  const int t = blockIdx.x;                      // < T_max: the slot map has an entry for every row
+  const int n_live = __ldg(n_live_p);
   int slot = __ldg(token_slot + t);
-  if (slot == -1) return;
+  if (t >= min(T, n_live) || slot == -1) return;
   const int nvec = d >> 3;
   uint4* hrow = reinterpret_cast<uint4*>(hidden + (size_t)t * d);
   uint4 hq[kTeamVec];
