@@ -203,52 +203,90 @@ struct SelShared {
   int n, res[2], count;
 };
 
+// Append `c` to sh.cand for every thread whose `take` is set: one shared-memory atomic per warp
+// (the lanes of a warp are ranked by ballot), not one per element on a single hot counter.
+// Every thread of the warp must call this.
+__device__ __forceinline__ void push_cand(SelShared& sh, bool take, unsigned long long c) {
+  const unsigned m = __ballot_sync(0xffffffffu, take);
+  if (m == 0u) return;
+  const int lane = threadIdx.x & 31, leader = __ffs(m) - 1;
+  int base = 0;
+  if (lane == leader) base = atomicAdd(&sh.n, __popc(m));
+  base = __shfl_sync(0xffffffffu, base, leader);
+  if (take) {
+    const int pos = base + __popc(m & ((1u << lane) - 1u));
+    if (pos < kCand) sh.cand[pos] = c;
+  }
+}
+
 // Collect into sh.cand (unsorted composites key << 32 | ~id) a set that contains the k largest
 // entries of `src` under the order (value descending, id ascending): radix refinement on the
-// order-preserving keys, 11 + 11 + 10 bits from the top, until what is still undecided fits the
-// buffer.  If more than the buffer's worth of entries tie EXACTLY with the k-th value:
+// order-preserving keys, up to 11 bits at a time, until what is still undecided fits the buffer.
+// The first digit starts at the highest bit in which the keys differ at all (the candidates of a
+// row are its largest values: they share sign, exponent and often leading mantissa bits, and a
+// digit taken from those bits would put them all into a handful of bins -- thousands of atomic
+// increments on the same few counters).  If more than the buffer's worth of entries tie EXACTLY
+// with the k-th value:
 //   ORDERED sources (position order = id order) finish with an index-ordered pass and return 2;
 //   other sources return 0 (the caller falls back).
 // Returns 1 in the ordinary case.  Every thread of the CTA must call this.
 template <bool ORDERED, class Src>
 __device__ int radix_collect(const Src& src, int k, SelShared& sh) {
   const int tid = threadIdx.x, n = src.n;
-  const int shifts[3] = {21, 10, 0};
-  const int widths[3] = {11, 11, 10};
-  unsigned prefix = 0;          // digits fixed so far (value of key >> (shift + width))
+  // range of the keys
+  unsigned kmin = 0xffffffffu, kmax = 0u;
+  for (int i = tid; i < n; i += kSelThreads) {
+    const unsigned key = src.key(i);
+    kmin = min(kmin, key);
+    kmax = max(kmax, key);
+  }
+  kmin = __reduce_min_sync(0xffffffffu, kmin);
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+  if ((tid & 31) == 0) {
+    sh.hist[tid >> 5] = (int)kmin;
+    sh.hist[32 + (tid >> 5)] = (int)kmax;
+  }
+  __syncthreads();
+  for (int w = 0; w < kSelThreads / 32; ++w) {
+    kmin = min(kmin, (unsigned)sh.hist[w]);
+    kmax = max(kmax, (unsigned)sh.hist[32 + w]);
+  }
+  __syncthreads();
+  int hi_bit = (kmax ^ kmin) ? 32 - __clz(kmax ^ kmin) : 0;     // bits [0, hi_bit) vary; the rest is common
+  unsigned prefix = hi_bit >= 32 ? 0u : (kmax >> hi_bit);       // digits fixed so far (= key >> hi_bit of the k-th)
   int need = k;                 // winners still to be found inside the prefix set
+  // Refinement goes on while the undecided set is much larger than k, even if it would already fit
+  // the buffer: one more histogram pass costs far less than sorting a thousand composites.
+  const int enough = max(2 * k, 128);
   bool done = false;
-  unsigned thr_hi = 0;          // entries with (key >> thr_shift) >= thr_hi are collected
-  int thr_shift = 0;
-  for (int pass = 0; pass < 3 && !done; ++pass) {
-    const int shift = shifts[pass], nb = 1 << widths[pass];
-    for (int b = tid; b < nb; b += kSelThreads) sh.hist[b] = 0;
+  while (hi_bit > 0) {
+    const int width = min(11, hi_bit), shift = hi_bit - width, nb = 1 << width;
+    for (int b = tid; b < kBins; b += kSelThreads) sh.hist[b] = 0;     // digits >= nb do not occur: their bins stay 0
     __syncthreads();
     for (int i = tid; i < n; i += kSelThreads) {
       const unsigned key = src.key(i);
-      if (pass == 0 || (key >> (shift + widths[pass])) == prefix) atomicAdd(&sh.hist[(key >> shift) & (nb - 1)], 1);
+      if (hi_bit >= 32 || (key >> hi_bit) == prefix) atomicAdd(&sh.hist[(key >> shift) & (nb - 1)], 1);
     }
     __syncthreads();
-    if (tid < 32) find_digit(sh.hist, nb, need, sh.res);
+    if (tid < 32) find_digit(sh.hist, kBins, need, sh.res);
     __syncthreads();
     const int D = sh.res[0], above = sh.res[1];
     const int in_bin = sh.hist[D];
     need -= above;
-    prefix = (prefix << widths[pass]) | (unsigned)D;
-    thr_hi = prefix;
-    thr_shift = shift;
-    if ((k - need) + in_bin <= kCand) done = true;
+    prefix = (prefix << width) | (unsigned)D;
+    hi_bit = shift;
+    done = (k - need) + in_bin <= kCand;
     __syncthreads();
+    if (done && (k - need) + in_bin <= enough) break;
   }
   if (tid == 0) sh.n = 0;
   __syncthreads();
+  const int n_up = (n + kSelThreads - 1) / kSelThreads * kSelThreads;    // whole warps take part in every ballot
   if (done) {
-    for (int i = tid; i < n; i += kSelThreads) {
-      const unsigned key = src.key(i);
-      if ((key >> thr_shift) >= thr_hi) {
-        const int pos = atomicAdd(&sh.n, 1);
-        sh.cand[pos] = ((unsigned long long)key << 32) | (0xffffffffu - src.id(i));
-      }
+    for (int i = tid; i < n_up; i += kSelThreads) {
+      const unsigned key = i < n ? src.key(i) : 0u;
+      const bool take = i < n && (key >> hi_bit) >= prefix;
+      push_cand(sh, take, take ? (((unsigned long long)key << 32) | (0xffffffffu - src.id(i))) : 0ull);
     }
     __syncthreads();
     return 1;
@@ -257,12 +295,10 @@ __device__ int radix_collect(const Src& src, int k, SelShared& sh) {
     return 0;
   } else {
   // every larger key, then the `need` lowest ids among the exact ties, in index order
-  for (int i = tid; i < n; i += kSelThreads) {
-    const unsigned key = src.key(i);
-    if (key > prefix) {
-      const int pos = atomicAdd(&sh.n, 1);
-      sh.cand[pos] = ((unsigned long long)key << 32) | (0xffffffffu - src.id(i));
-    }
+  for (int i = tid; i < n_up; i += kSelThreads) {
+    const unsigned key = i < n ? src.key(i) : 0u;
+    const bool take = i < n && key > prefix;
+    push_cand(sh, take, take ? (((unsigned long long)key << 32) | (0xffffffffu - src.id(i))) : 0ull);
   }
   __syncthreads();
   int taken = 0;               // uniform across the block
