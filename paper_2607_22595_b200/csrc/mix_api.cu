@@ -166,6 +166,14 @@ int upload_chain(mix_ctx* c, int slot, cudaStream_t s) {
 
 }  // namespace
 
+namespace mix {
+int pdl_mask() {
+  // default: not the full encode pass -- measured, its early-resident CTAs cost config 3 about 7 us
+  static const int mask = getenv("MIX_PDL_MASK") ? atoi(getenv("MIX_PDL_MASK")) : (kPdlPack | kPdlTail);
+  return mask;
+}
+}  // namespace mix
+
 extern "C" {
 
 int mix_create(mix_ctx** out, const mix_config* cfg) {

@@ -153,6 +153,37 @@ struct Ctx {
   int* out_n_active;
 };
 
+// Programmatic dependent launch.  The kernels of the SAE chain are short and strictly ordered, so
+// what separates them is launch latency; launched this way, a kernel's CTAs may become resident
+// while its predecessor in the stream still runs.  Contract inside such a kernel: pdl_wait() is its
+// FIRST statement -- nothing the predecessor wrote is read before it, and no thread leaves without
+// it (a grid that ended without waiting would let ITS successor run ahead of the predecessor) --
+// followed by pdl_launch_dependents(), so that at most two kernels of the chain overlap.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Which launches use programmatic dependent launch: bit 0 pack, bit 1 the full encode pass, bit 2 everything after
+// it (merge ... decode_delta).  MIX_PDL_MASK in the environment overrides the default (A/B timing); read once.
+enum { kPdlPack = 1, kPdlEncode = 2, kPdlTail = 4 };
+int pdl_mask();
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(int which, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = (pdl_mask() & which) ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // kernel launchers (each returns the CUDA error of the launch)
 cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s);
 cudaError_t launch_probe_multiclass(const Ctx* c, const __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s);

@@ -866,6 +866,8 @@ route_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_
 __global__ void __launch_bounds__(256)
 pack_kernel(const __nv_bfloat16* __restrict__ hidden, const int* __restrict__ panel_row,
             const RouteState* __restrict__ rs, __nv_bfloat16* __restrict__ panel, int d) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int p = blockIdx.x * 8 + warp;
   if (p >= rs->n_panel_rows) return;
@@ -970,8 +972,7 @@ cudaError_t launch_route(const Ctx* c, int T, cudaStream_t s, unsigned long long
 
 cudaError_t launch_pack(const Ctx* c, const __nv_bfloat16* hidden, cudaStream_t s) {
   const int blocks = (c->panel_rows_cap + 7) / 8;
-  pack_kernel<<<blocks, 256, 0, s>>>(hidden, c->d_panel_row, c->d_route, c->d_panel, c->cfg.d_model);
-  return cudaGetLastError();
+  return launch_pdl(kPdlPack, pack_kernel, dim3(blocks), dim3(256), 0, s, hidden, c->d_panel_row, c->d_route, c->d_panel, c->cfg.d_model);
 }
 
 cudaError_t launch_compose_map(const Ctx* c, int T_live, int n_req, cudaStream_t s) {

@@ -228,6 +228,8 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
   constexpr int kStages = TcCfg<kFp8>::kStages;
   constexpr int kStageBytes = TcCfg<kFp8>::kStageBytes;
   constexpr int kTcThreads = TcCfg<kFp8>::kThreads;
+  pdl_wait();
+  pdl_launch_dependents();
   if (mode == 1 && *n_flagged == 0) return;
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment: required by the 128-byte swizzle atoms
@@ -536,16 +538,14 @@ cudaError_t launch_encode_tc(const Ctx* c, int mode, cudaStream_t s) {
   const int w_tiled = (c->cfg.flags & MIX_FLAG_RETILE_W_ENC) ? 1 : 0;
   const int stall = (c->cfg.flags & MIX_FLAG_TEST_STALL_ENCODE) ? 1 : 0;
   if (c->cfg.flags & MIX_FLAG_FP8_W_ENC)
-    encode_tc_kernel<true><<<c->n_sms, TcCfg<true>::kThreads, TcCfg<true>::kSmemBytes, s>>>(
-        c->tmap_panel, c->d_tmap_w, c->d_route, c->d_groups, c->cfg.n_groups_max, c->d_z, c->cfg.d_sae_max, c->cfg.d_model,
-        c->d_status, mode, c->d_mtile_flag, c->d_n_flagged, c->d_cand_val, c->d_cand_idx, c->d_cand_ninth, c->cand_tiles,
-        w_tiled, stall);
-  else
-    encode_tc_kernel<false><<<c->n_sms, TcCfg<false>::kThreads, TcCfg<false>::kSmemBytes, s>>>(
-        c->tmap_panel, c->d_tmap_w, c->d_route, c->d_groups, c->cfg.n_groups_max, c->d_z, c->cfg.d_sae_max, c->cfg.d_model,
-        c->d_status, mode, c->d_mtile_flag, c->d_n_flagged, c->d_cand_val, c->d_cand_idx, c->d_cand_ninth, c->cand_tiles,
-        w_tiled, stall);
-  return cudaGetLastError();
+    return launch_pdl(mode == 0 ? kPdlEncode : kPdlTail, encode_tc_kernel<true>, dim3(c->n_sms), dim3(TcCfg<true>::kThreads), TcCfg<true>::kSmemBytes, s,
+                      c->tmap_panel, c->d_tmap_w, c->d_route, c->d_groups, c->cfg.n_groups_max, c->d_z, c->cfg.d_sae_max,
+                      c->cfg.d_model, c->d_status, mode, c->d_mtile_flag, c->d_n_flagged, c->d_cand_val, c->d_cand_idx,
+                      c->d_cand_ninth, c->cand_tiles, w_tiled, stall);
+  return launch_pdl(mode == 0 ? kPdlEncode : kPdlTail, encode_tc_kernel<false>, dim3(c->n_sms), dim3(TcCfg<false>::kThreads), TcCfg<false>::kSmemBytes, s,
+                    c->tmap_panel, c->d_tmap_w, c->d_route, c->d_groups, c->cfg.n_groups_max, c->d_z, c->cfg.d_sae_max,
+                    c->cfg.d_model, c->d_status, mode, c->d_mtile_flag, c->d_n_flagged, c->d_cand_val, c->d_cand_idx,
+                    c->d_cand_ninth, c->cand_tiles, w_tiled, stall);
 }
 
 }  // namespace mix

@@ -20,6 +20,8 @@ __global__ void __launch_bounds__(256)
 encode_simt_kernel(const __nv_bfloat16* __restrict__ panel, const int* __restrict__ mtile_group,
                    const RouteState* __restrict__ rs, const GroupEntry* __restrict__ groups, float* __restrict__ Z,
                    long long ldz, int d) {
+  pdl_wait();
+  pdl_launch_dependents();
   constexpr int BM = 64, BN = 64, BK = 32;
   __shared__ float As[BK][BM + 1];
   __shared__ float Bs[BK][BN + 1];
@@ -335,6 +337,8 @@ select_kernel(const float* __restrict__ Z, long long ldz, const int* __restrict_
               const GroupEntry* __restrict__ groups, int k_max, int* __restrict__ ws_idx, float* __restrict__ ws_val,
               int* __restrict__ out_idx, float* __restrict__ out_val, int* __restrict__ out_n_active,
               unsigned* __restrict__ status, const int* __restrict__ row_flag, const int* __restrict__ n_flagged) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ SelShared sh;
   // nothing to do: no flagged TopK row, and nobody asked for the other sets' active counts
   if (row_flag != nullptr && *n_flagged == 0 && (out_n_active == nullptr || rs->n_topk_rows == rs->n_sae_rows)) return;
@@ -385,6 +389,8 @@ merge_kernel(const float* __restrict__ cand_val, const int* __restrict__ cand_id
              int* __restrict__ ws_idx, float* __restrict__ ws_val, int* __restrict__ out_idx, float* __restrict__ out_val,
              int* __restrict__ out_n_active, int* __restrict__ row_flag, int* __restrict__ mtile_flag,
              int* __restrict__ n_flagged) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ SelShared sh;
   if (rs->n_topk_rows == 0) return;                  // no TopK row routed this call
   const int n_rows = rs->n_panel_rows;
@@ -462,6 +468,8 @@ decode_kernel(__nv_bfloat16* __restrict__ hidden, int d, const float* __restrict
               const float* __restrict__ edit_val, const unsigned char* __restrict__ edit_mode, int r_max, int k_max,
               const int* __restrict__ ws_idx, const float* __restrict__ ws_val,
               RowDelta* __restrict__ row_delta, float* __restrict__ edit_coef) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ float s_coef[kDecList];
   __shared__ int s_feat[kDecList];
   __shared__ float s_fnew[kMaxEdits];
@@ -642,6 +650,8 @@ __global__ void __launch_bounds__(kDdThreads, 4)
 decode_delta_kernel(__nv_bfloat16* __restrict__ hidden, int d, const int* __restrict__ panel_row,
                     const RouteState* __restrict__ rs, const RowDelta* __restrict__ row_delta,
                     const float* __restrict__ edit_coef, const int* __restrict__ edit_idx, int r_max) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ __align__(16) float s_coef[kDdEntries + kDdBatch][kDdRows];
   __shared__ const uint4* s_wrow[kDdEntries + kDdBatch];
   __shared__ int s_t[kDdRows], s_slot[kDdRows], s_nedit[kDdRows];
@@ -748,6 +758,8 @@ sae_edit_only_kernel(__nv_bfloat16* __restrict__ hidden, int d, const int* __res
                      const GateEntry* __restrict__ gates, int n_slots, const GroupEntry* __restrict__ groups,
                      int n_groups, const int* __restrict__ edit_idx, const float* __restrict__ edit_val,
                      const unsigned char* __restrict__ edit_mode, int r_max) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ float s_coef[kMaxEdits];
   __shared__ int s_feat[kMaxEdits];
   __shared__ int s_any;
@@ -841,55 +853,49 @@ static int row_grid(const Ctx* c) {
 
 cudaError_t launch_encode_simt(const Ctx* c, cudaStream_t s) {
   dim3 grid((unsigned)(c->cfg.d_sae_max / 64), (unsigned)(c->panel_rows_cap / 64));
-  encode_simt_kernel<<<grid, 256, 0, s>>>(c->d_panel, c->d_mtile_group, c->d_route, c->d_groups, c->d_z,
+  return launch_pdl(kPdlEncode, encode_simt_kernel, dim3(grid), dim3(256), 0, s, c->d_panel, c->d_mtile_group, c->d_route, c->d_groups, c->d_z,
                                           c->cfg.d_sae_max, c->cfg.d_model);
-  return cudaGetLastError();
 }
 
 cudaError_t launch_merge(const Ctx* c, cudaStream_t s) {
-  merge_kernel<<<row_grid(c), kSelThreads, 0, s>>>(c->d_cand_val, c->d_cand_idx, c->d_cand_ninth, c->cand_tiles,
+  return launch_pdl(kPdlTail, merge_kernel, dim3(row_grid(c)), dim3(kSelThreads), 0, s, c->d_cand_val, c->d_cand_idx, c->d_cand_ninth, c->cand_tiles,
                                                          c->d_panel_row, c->d_mtile_group, c->d_route, c->d_groups,
                                                          c->cfg.k_max, c->d_topk_idx, c->d_topk_val, c->out_topk_idx,
                                                          c->out_topk_val, c->out_n_active, c->d_row_flag,
                                                          c->d_mtile_flag, c->d_n_flagged);
-  return cudaGetLastError();
 }
 
 cudaError_t launch_select(const Ctx* c, bool flagged_only, cudaStream_t s) {
-  select_kernel<<<row_grid(c), kSelThreads, 0, s>>>(c->d_z, c->cfg.d_sae_max, c->d_panel_row,
+  return launch_pdl(kPdlTail, select_kernel, dim3(row_grid(c)), dim3(kSelThreads), 0, s, c->d_z, c->cfg.d_sae_max, c->d_panel_row,
                                                           c->d_mtile_group, c->d_route, c->d_groups, c->cfg.k_max,
                                                           c->d_topk_idx, c->d_topk_val, c->out_topk_idx,
                                                           c->out_topk_val, c->out_n_active, c->d_status,
                                                           flagged_only ? c->d_row_flag : nullptr, c->d_n_flagged);
-  return cudaGetLastError();
 }
 
 cudaError_t launch_edit_only(const Ctx* c, __nv_bfloat16* hidden, int T, cudaStream_t s) {
-  sae_edit_only_kernel<<<c->cfg.T_max, kDecThreads, 0, s>>>(hidden, c->cfg.d_model, c->d_token_slot, c->d_n_live, T,
+  return launch_pdl(kPdlTail, sae_edit_only_kernel, dim3(c->cfg.T_max), dim3(kDecThreads), 0, s, hidden, c->cfg.d_model, c->d_token_slot, c->d_n_live, T,
                                                             c->d_apps, c->d_gates, c->cfg.n_slots_max, c->d_groups,
                                                             c->cfg.n_groups_max, c->d_edit_idx, c->d_edit_val,
                                                             c->d_edit_mode, c->cfg.r_max);
-  return cudaGetLastError();
 }
 
 // Two kernels: decode_kernel (one CTA per row) rebuilds the rows whose app replaces the residual and, for
 // the rows that keep the error term, only works out the coefficients of their edits; decode_delta_kernel
 // then adds those rows' deltas, eight rows per CTA.
 cudaError_t launch_decode(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s) {
-  decode_kernel<<<c->panel_rows_cap, kDecThreads, 0, s>>>(hidden, c->cfg.d_model, c->d_z, c->cfg.d_sae_max,
+  return launch_pdl(kPdlTail, decode_kernel, dim3(c->panel_rows_cap), dim3(kDecThreads), 0, s, hidden, c->cfg.d_model, c->d_z, c->cfg.d_sae_max,
                                                           c->d_panel_row, c->d_row_slot, c->d_route, c->d_apps,
                                                           c->d_groups, c->d_edit_idx, c->d_edit_val, c->d_edit_mode,
                                                           c->cfg.r_max, c->cfg.k_max, c->d_topk_idx, c->d_topk_val,
                                                           c->d_row_delta, c->d_edit_coef);
-  return cudaGetLastError();
 }
 
 cudaError_t launch_decode_delta(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s) {
   dim3 grid((unsigned)((c->panel_rows_cap + kDdRows - 1) / kDdRows),
             (unsigned)((c->cfg.d_model / 8 + kDdThreads - 1) / kDdThreads));
-  decode_delta_kernel<<<grid, kDdThreads, 0, s>>>(hidden, c->cfg.d_model, c->d_panel_row, c->d_route, c->d_row_delta,
+  return launch_pdl(kPdlTail, decode_delta_kernel, dim3(grid), dim3(kDdThreads), 0, s, hidden, c->cfg.d_model, c->d_panel_row, c->d_route, c->d_row_delta,
                                                   c->d_edit_coef, c->d_edit_idx, c->cfg.r_max);
-  return cudaGetLastError();
 }
 
 }  // namespace mix
