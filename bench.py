@@ -352,6 +352,42 @@ def extras_conditional(w, mixlib):
     return out
 
 
+def extras_multiclass(peaks, mixlib, small=False):
+    """Multi-class probes alone on a large batch (every row hooked, requests of 256 consecutive rows dealt
+    round-robin over the probes): the tensor-core probe kernel plus the pass of the streaming kernel that
+    skips these rows.  Bytes counted: the hidden state once."""
+    out = {}
+    shapes = [(5120, 16384, 16, 8)] if small else [(4096, 65536, 2, 4), (4096, 65536, 16, 8), (4096, 65536, 32, 4),
+                                                   (8192, 32768, 8, 4), (5120, 16384, 16, 8)]
+    for d, T, C, n_probe in shapes:
+        g = torch.Generator(device="cuda"); g.manual_seed(1)
+        hidden = torch.randn((T, d), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        m = mixlib.Mix(d_model=d, T_max=T, n_slots_max=n_probe, C_max=C)
+        keep = []
+        for s_ in range(n_probe):
+            Wp = (torch.randn((C, d), generator=g, device="cuda") * d ** -0.5).to(torch.bfloat16); keep.append(Wp)
+            m.register_probe(s_, Wp, None, mixlib.MIX_ACT_SOFTMAX)
+        m.set_slot_map(torch.from_numpy(((np.arange(T) // 256) % n_probe).astype(np.int32)).cuda())
+        scores = torch.zeros((T, C), dtype=torch.float32, device="cuda")
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        best = 1e9
+        for _ in range(6):
+            e0.record(); m.apply(hidden, scores); e1.record(); torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        nbytes = T * d * 2
+        st = time_stages(m, lambda: m.apply(hidden, scores))
+        tc_ms = st["probe_tc"]
+        out["d=%d T=%d C=%d probes=%d" % (d, T, C, n_probe)] = {
+            "ms": best, "gbs": nbytes / best / 1e6, "frac_hbm_peak": nbytes / best / 1e6 / peaks["hbm_gbs"],
+            "frac_hbm_nominal": nbytes / best / 1e6 / NOMINAL_HBM_GBS, "stage_ms": st,
+            "probe_tc_kernel_alone": {"gbs": nbytes / tc_ms / 1e6, "frac_hbm_peak": nbytes / tc_ms / 1e6 / peaks["hbm_gbs"]},
+            "status": m.get_status()}
+        m.destroy()
+        del hidden
+        torch.cuda.empty_cache()
+    return out
+
+
 def run_workload(args):
     """--workload X: one of the other configurations alone (not the contract line)."""
     import paper_2607_22595_b200 as mixlib
@@ -386,6 +422,10 @@ def run_workload(args):
         out = extras_conditional(W.make_mixed("cuda"), mixlib)
     elif name == "conditional_small":
         out = extras_conditional(W.make_mixed("cuda", T=4096, d_sae=8192, R=32), mixlib)
+    elif name == "multiclass":
+        out = extras_multiclass(peaks, mixlib)
+    elif name == "multiclass_small":   # profiling case: 168 MB of hidden state
+        out = extras_multiclass(peaks, mixlib, small=True)
     elif name == "replay":
         out = run_replay(peaks, mixlib, args.steps or 200)
     else:
@@ -672,7 +712,7 @@ def main():
     ap.add_argument("--no-retile", action="store_true",
                     help="SAE contexts stream W_enc as registered instead of a tile-contiguous copy (MIX_FLAG_RETILE_W_ENC)")
     ap.add_argument("--workload", default="decode",
-                    help="decode (the contract line) | sweep | sae_heavy | sae_heavy_fp8 | sae_small | sae_small_fp8 | mixed | mixed_fp8 | mixed_small | conditional | conditional_small | replay")
+                    help="decode (the contract line) | sweep | sae_heavy | sae_heavy_fp8 | sae_small | sae_small_fp8 | mixed | mixed_fp8 | mixed_small | conditional | conditional_small | multiclass | multiclass_small | replay")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     args = ap.parse_args()
     if args.no_retile:

@@ -292,6 +292,8 @@ class Mix:
         front = ["probe_steer"]
         if self.cfg.T_max > 2048 and self.cfg.C_max > 1:
             front.append("probe_multiclass")
+            if self.cfg.n_groups_max == 0:
+                front.append("probe_tc")
         if self.cfg.n_groups_max == 0:
             return front
         tail = ["edit_only"] if self.cfg.flags & MIX_FLAG_SAE_EDIT_ONLY else []

@@ -76,7 +76,7 @@ void free_all(mix_ctx* c) {
   cudaFree(c->d_edit_idx); cudaFree(c->d_edit_val); cudaFree(c->d_edit_mode); cudaFree(c->d_status);
   cudaFree(c->d_tmp_req); cudaFree(c->d_tmp_req_slot); cudaFree(c->d_panel); cudaFree(c->d_panel_row);
   cudaFree(c->d_mtile_group); cudaFree(c->d_row_group); cudaFree(c->d_route); cudaFree(c->d_z); cudaFree(c->d_topk_idx);
-  cudaFree(c->d_topk_val); cudaFree(c->d_tmap_w); cudaFree(c->d_cand_val); cudaFree(c->d_cand_idx);
+  cudaFree(c->d_topk_val); cudaFree(c->d_tmap_w); cudaFree(c->d_tmap_probe); cudaFree(c->d_mc_dense); cudaFree(c->d_cand_val); cudaFree(c->d_cand_idx);
   cudaFree(c->d_row_delta); cudaFree(c->d_edit_coef);
   cudaFree(c->d_cand_ninth); cudaFree(c->d_row_flag); cudaFree(c->d_mtile_flag); cudaFree(c->d_n_flagged);
   if (c->owned_b_eff)
@@ -269,6 +269,15 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
       if (e == cudaSuccess) e = encode_tc_prepare();
     }
   }
+  if (e == cudaSuccess && has_tc_probe_stage(c)) {
+    // large batches with multi-class probes: the tensor-core probe kernel needs a map per probe matrix
+    if (dev_alloc(&c->d_tmap_probe, NS) != cudaSuccess || dev_alloc(&c->d_mc_dense, 1) != cudaSuccess) {
+      cudaGetLastError(); free_all(c); free(c); return MIX_ERR_NO_MEMORY;
+    }
+    e = cudaMemset(c->d_mc_dense, 0, sizeof(int));
+    if (load_encode_fn() != MIX_OK) e = cudaErrorUnknown;
+    if (e == cudaSuccess) e = probe_tc_prepare();
+  }
   if (e == cudaSuccess && G > 0) {
     e = cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->body_stream, cudaStreamNonBlocking);
@@ -402,6 +411,13 @@ int mix_register_app(mix_ctx* c, int slot, int kind, const void* desc, void* str
     e.act = p->act;
     e.W = p->W;
     e.b = p->b;
+    if (c->d_tmap_probe && p->n_classes > 1 && p->n_classes <= 32) {
+      // rows of the probe matrix beyond n_classes lie outside the tensor: TMA fills them with zeros
+      CUtensorMap tm;
+      if (make_tmap(&tm, p->W, (unsigned long long)p->n_classes, c->cfg.d_model, 32) != MIX_OK)
+        MIX_FAIL(c, MIX_ERR_CUDA, "cuTensorMapEncodeTiled failed for the probe matrix of slot %d", slot);
+      MIX_CUDA(c, cudaMemcpyAsync(c->d_tmap_probe + slot, &tm, sizeof(tm), cudaMemcpyHostToDevice, s));
+    }
   } else if (kind == MIX_STEER) {
     const mix_steer* p = static_cast<const mix_steer*>(desc);
     if (!p->v || !aligned16(p->v)) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "steering vector is NULL or not 16-byte aligned");
@@ -684,8 +700,18 @@ int apply_impl(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream,
   MIX_CUDA(c, launch_probe_steer(c, h, T, scores_out, ps));
   MIX_CUDA(c, tap());
   if (has_multiclass_stage(c)) {
+    // Multi-class probes of a large batch.  With the tensor-core kernel in play, exactly one of the two does
+    // the work (device-side choice made by probe_steer_kernel, see mc_batch_is_dense): the 16-row kernel takes batches sparse in such
+    // rows, the tensor-core kernel dense ones.
     MIX_CUDA(c, launch_probe_multiclass(c, h, T, scores_out, ps));
     MIX_CUDA(c, tap());
+    if (has_tc_probe_stage(c)) {
+      CUtensorMap tm_hidden;                     // host-side encoding only: no device work, fine under capture
+      if (make_tmap(&tm_hidden, h, (unsigned long long)c->cfg.T_max, c->cfg.d_model, kTileM) != MIX_OK)
+        MIX_FAIL(c, MIX_ERR_CUDA, "cuTensorMapEncodeTiled failed for hidden");
+      MIX_CUDA(c, launch_probe_tc(c, tm_hidden, T, scores_out, ps));
+      MIX_CUDA(c, tap());
+    }
   }
   if (fork) MIX_CUDA(c, cudaEventRecord(c->ev_join, ps));
   if (c->cfg.n_groups_max > 0) {
@@ -726,7 +752,7 @@ int mix_apply_router(mix_ctx* c, float* logits, int n_experts, int T, void* stre
 
 int mix_launches_per_apply(const mix_ctx* c) {
   if (!c) return 0;
-  const int front = has_multiclass_stage(c) ? 2 : 1;
+  const int front = 1 + (has_multiclass_stage(c) ? 1 : 0) + (has_tc_probe_stage(c) ? 1 : 0);
   if (c->cfg.n_groups_max == 0) return front;
   return front + ((c->cfg.flags & MIX_FLAG_ENCODE_SIMT) ? 6 : 8) + ((c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) ? 1 : 0);
 }

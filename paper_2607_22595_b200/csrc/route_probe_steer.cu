@@ -3,6 +3,7 @@
 // probe_steer_kernel is the bandwidth kernel of the hook: one warp per token row, 16-byte
 // loads, fp32 FMA, shuffle reductions.  A row whose slot is -1 costs one 4-byte load.
 #include "mix_internal.h"
+#include "row_lookup.cuh"
 
 namespace mix {
 
@@ -142,62 +143,6 @@ __device__ __forceinline__ void finish_probe(const float* logit, int C, int act,
   if (lane + 32 < C) out[lane + 32] = z1;
 }
 
-struct RowApp {
-  bool gated;           // the slot has a gate (whether or not it let this row through)
-  bool chained;         // another app follows on the same row (set even when the gate is closed)
-  int raw_kind;         // the slot's kind even when the gate is closed (0: no valid app)
-  int kind, C, act;     // kind 0: nothing to do
-  float alpha;
-  const uint4* W;
-  const float* b;
-};
-
-// Does row t pass the gate of its slot?  (NaN fails both comparisons.)
-__device__ __forceinline__ bool gate_open(const GateEntry* __restrict__ gates, int s, int t) {
-  const int4 g0 = __ldg(reinterpret_cast<const int4*>(gates + s));        // scores ptr, stride, col
-  const int4 g1 = __ldg(reinterpret_cast<const int4*>(gates + s) + 1);    // cmp, thr
-  const float* sc = reinterpret_cast<const float*>(((unsigned long long)(unsigned)g0.y << 32) | (unsigned)g0.x);
-  const float v = __ldg(sc + (size_t)t * g0.z + g0.w);
-  const float thr = __int_as_float(g1.y);
-  return g1.x == MIX_GATE_GE ? v >= thr : v < thr;
-}
-
-// Slot -> app for row t; flags bad slot ids; applies the slot's gate.  `leader` is the one
-// thread that may raise status.
-__device__ __forceinline__ RowApp lookup(int s, int t, const AppEntry* __restrict__ apps,
-                                         const GateEntry* __restrict__ gates, int n_slots,
-                                         unsigned* __restrict__ status, bool leader, bool eval_gate = true) {
-  RowApp r;
-  r.kind = 0;
-  r.raw_kind = 0;
-  r.C = 0;
-  r.gated = false;
-  r.chained = false;
-  if (s == -1) return r;
-  if (s < -1 || s >= n_slots) {
-    if (leader) atomicOr(status, MIX_STATUS_BAD_SLOT);
-    return r;
-  }
-  // the whole 48-byte entry in three independent 16-byte loads (one round trip)
-  const int4* e = reinterpret_cast<const int4*>(apps + s);
-  const int4 q0 = __ldg(e), q1 = __ldg(e + 1), q2 = __ldg(e + 2);
-  if (!q0.x) {                                   // valid
-    if (leader) atomicOr(status, MIX_STATUS_BAD_SLOT);
-    return r;
-  }
-  r.gated = (q0.y & kKindGated) != 0;
-  r.chained = (q0.y & kKindChained) != 0;
-  r.raw_kind = q0.y & kKindMask;
-  r.C = q0.z;
-  if (eval_gate && r.gated && !gate_open(gates, s, t)) return r;  // gate closed: the row passes through
-  r.kind = q0.y & kKindMask;
-  r.act = q0.w;
-  r.alpha = __int_as_float(q1.x);
-  r.W = reinterpret_cast<const uint4*>(((unsigned long long)(unsigned)q2.y << 32) | (unsigned)q2.x);
-  r.b = reinterpret_cast<const float*>(((unsigned long long)(unsigned)q2.w << 32) | (unsigned)q2.z);
-  return r;
-}
-
 constexpr int kWarpsPerBlock = 8;      // = rows per CTA of the large-batch kernel
 constexpr int kCoopMaxClasses = 32;    // widest probe the cooperative tensor-core pass takes
 
@@ -246,16 +191,24 @@ __device__ __forceinline__ void warp_row(const RowApp& a, __nv_bfloat16* __restr
 
 // Large batches: a CTA owns 8 consecutive rows, one warp per row: streaming work (steering,
 // single-class probes).  Multi-class probes up to kCoopMaxClasses classes are left to
-// probe_multiclass_kernel when `multiclass_elsewhere` is set.
+// probe_tc_kernel (probe_tc.cu) when `multiclass_elsewhere` is set.
 __global__ void __launch_bounds__(kWarpsPerBlock * 32, 3)
 probe_steer_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
                    const AppEntry* __restrict__ apps, const GateEntry* __restrict__ gates, int n_slots,
                    __nv_bfloat16* __restrict__ hidden, int d,
-                   float* __restrict__ scores, int C_max, unsigned* __restrict__ status, int multiclass_elsewhere) {
+                   float* __restrict__ scores, int C_max, unsigned* __restrict__ status, int multiclass_elsewhere,
+                   int* __restrict__ mc_dense_flag) {
   __shared__ float s_logit[kWarpsPerBlock][kMaxClasses];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t = blockIdx.x * kWarpsPerBlock + warp;
   const int n_live = __ldg(n_live_p);            // issued together with the slot id: one round trip, not two
+  if (mc_dense_flag != nullptr && blockIdx.x == 0) {
+    // this CTA also decides, for the two multi-class probe kernels that follow in the stream, which of
+    // them takes the batch
+    const int live = min(T, n_live);
+    const bool dense = live > 0 && mc_batch_is_dense(token_slot, apps, n_slots, live);
+    if (threadIdx.x == 0) *mc_dense_flag = dense ? 1 : 0;
+  }
   const int slot = t < T ? __ldg(token_slot + t) : -1;
   if (t >= min(T, n_live)) return;
   const RowApp a = lookup(slot, t, apps, gates, n_slots, status, lane == 0);
@@ -349,7 +302,8 @@ struct McRow {
 __global__ void __launch_bounds__(kMcWarps * 32, 2)
 probe_multiclass_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
                         const AppEntry* __restrict__ apps, const GateEntry* __restrict__ gates, int n_slots,
-                        const __nv_bfloat16* __restrict__ hidden, int d, float* __restrict__ scores, int C_max) {
+                        const __nv_bfloat16* __restrict__ hidden, int d, float* __restrict__ scores, int C_max,
+                        const int* __restrict__ mc_dense_flag) {
   __shared__ float s_part[kMcWarps][kMcRows][kCoopMaxClasses];   // [warp][row][class]
   __shared__ float s_logit[kMcWarps][kCoopMaxClasses];
   __shared__ McRow s_row[kMcRows];
@@ -358,6 +312,7 @@ probe_multiclass_kernel(const int* __restrict__ token_slot, const int* __restric
   const int t0 = blockIdx.x * kMcRows;
   const int n_live = min(T, __ldg(n_live_p));
   if (t0 >= n_live || scores == nullptr) return;
+  if (mc_dense_flag != nullptr && *mc_dense_flag) return;   // a batch dense in these rows is probe_tc_kernel's
   if (threadIdx.x == 0) s_any = 0;
   __syncthreads();
   if (threadIdx.x < kMcRows) {           // one thread per row: slot -> entry -> gate
@@ -922,6 +877,10 @@ bool has_multiclass_stage(const Ctx* c) {
   return c->cfg.T_max > kTeamMaxRows && c->cfg.C_max > 1 && !(c->cfg.flags & MIX_FLAG_SLOT_CHAINS);
 }
 
+// The tensor-core probe kernel holds a whole SM's shared memory, as the SAE encode does: beside an encode
+// it could only wait, so contexts with SAE weight sets leave every batch to the 16-row kernel.
+bool has_tc_probe_stage(const Ctx* c) { return has_multiclass_stage(c) && c->cfg.n_groups_max == 0; }
+
 cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s) {
   if (c->cfg.flags & MIX_FLAG_SLOT_CHAINS) {
     probe_steer_chain_kernel<<<c->cfg.T_max, kChainWarps * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps,
@@ -937,7 +896,8 @@ cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float
     const int blocks = (c->cfg.T_max + kWarpsPerBlock - 1) / kWarpsPerBlock;
     probe_steer_kernel<<<blocks, kWarpsPerBlock * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates,
                                                               c->cfg.n_slots_max, hidden, c->cfg.d_model, scores,
-                                                              c->cfg.C_max, c->d_status, has_multiclass_stage(c) ? 1 : 0);
+                                                              c->cfg.C_max, c->d_status, has_multiclass_stage(c) ? 1 : 0,
+                                                              has_tc_probe_stage(c) ? c->d_mc_dense : nullptr);
   }
   return cudaGetLastError();
 }
@@ -946,7 +906,7 @@ cudaError_t launch_probe_multiclass(const Ctx* c, const __nv_bfloat16* hidden, i
   const int blocks = (c->cfg.T_max + kMcRows - 1) / kMcRows;
   probe_multiclass_kernel<<<blocks, kMcWarps * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates,
                                                                  c->cfg.n_slots_max, hidden, c->cfg.d_model, scores,
-                                                                 c->cfg.C_max);
+                                                                 c->cfg.C_max, has_tc_probe_stage(c) ? c->d_mc_dense : nullptr);
   return cudaGetLastError();
 }
 

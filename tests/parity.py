@@ -15,6 +15,7 @@ from oracle import mi_hook as O
 #   TopK index sets                                   : equal, except members whose pre-activation is within
 #                                                       1e-3 of the oracle's k-th value may be swapped
 SCORE_RTOL = 1e-3
+LOGIT_ACC_TOL = 4e-6        # ~64 fp32 unit roundoffs (2^-24) of sum |w_i h_i|: raw logits only, see check_parity
 HIDDEN_TOL_FRAC = 1e-2
 TOPK_TIE_TOL = 1e-3
 CANARY_F32 = np.uint32(0x7FC0DEAD)          # a NaN payload nobody computes
@@ -90,6 +91,14 @@ def check_parity(wh, out, rows=None, expect_status=0, check_features=True, scale
             C = len(s_ref)
             s_gpu = out["scores"][t, :C].astype(np.float64)
             rel = np.abs(s_gpu - s_ref) / np.abs(s_ref)
+            app = wh.apps[int(wh.token_slot[t])]
+            if app.act == O.ACT_NONE:
+                # A raw logit can be arbitrarily close to zero, where a relative bound says nothing about an
+                # fp32-accumulated sum: such an entry may instead be within LOGIT_ACC_TOL * sum_i |w_i h_i|
+                # (a few dozen fp32 roundings of the summed magnitudes; sigmoid / softmax scores, the quantity
+                # the 1e-3 bound is stated for, keep the pure relative test).
+                mag = np.abs(O.bf16_to_f64(app.W)) @ np.abs(O.bf16_to_f64(wh.hidden[t]))
+                rel = np.where(np.abs(s_gpu - s_ref) <= LOGIT_ACC_TOL * mag, 0.0, rel)
             assert (rel <= SCORE_RTOL).all(), "row %d probe scores off: rel %g" % (t, rel.max())
             assert (scores_bits[t, C:] == CANARY_F32).all()
             stats["max_score_rel"] = max(stats["max_score_rel"], float(rel.max()))
