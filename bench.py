@@ -683,6 +683,7 @@ def run_mix(args, rank, world, local_rank):
             try:
                 ex["decode_variants"] = extras_decode_variants(w, hiddens, scores, mixlib)
                 ex["sweep"] = extras_sweep(peaks, mixlib)
+                ex["multiclass_probes"] = extras_multiclass(peaks, mixlib)
                 tiny = extras_sae("tiny (config 0)", W.make_tiny("cuda"), peaks, mixlib)
                 ex["tiny"] = {"t_call_ms_graph": tiny["t_call_ms_graph"], "status": tiny["status"],
                               "note": "correctness config: the call sits on the launch-latency floor of its kernel chain"}

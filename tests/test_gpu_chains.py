@@ -19,9 +19,11 @@ def _mixlib():
     return mixlib
 
 
-def check_chain_parity(wh, out):
+def check_chain_parity(wh, out, scale_with_output=False, expect_status=0):
     ref = O.apply_chain_hook(wh)
     hmax = float(np.abs(O.bf16_to_f64(wh.hidden)).max())
+    if scale_with_output:      # an app's output may dwarf the hidden state (see parity.check_parity)
+        hmax = max([hmax] + [float(np.abs(ref.y[t]).max()) for t in range(wh.T_max) if ref.modified[t]])
     sb = out["scores"].view(np.uint32)
     redo = {}
     for t in range(wh.T_max):
@@ -55,7 +57,8 @@ def check_chain_parity(wh, out):
             assert int(out["n_active"][t]) == ref.n_active[t]
         elif t not in ref.n_active:
             assert int(out["n_active"][t]) == int(CANARY_I32)
-    assert out["status"] == 0
+    if expect_status is not None:
+        assert out["status"] == expect_status
     return dict(modified=n_mod, scores=n_scores, swaps=len(redo))
 
 
@@ -167,3 +170,38 @@ def test_set_chain_error_codes():
     ref_rows_slot1 = np.nonzero(w.token_slot[:w.T_live] == 1)[0]
     assert np.array_equal(out["hidden"][ref_rows_slot1], W.bits(w.hidden)[ref_rows_slot1])
     m.destroy()
+
+
+# ------------------------------------------------------------------ seeded random chains
+def _random_chained_workload(seed):
+    from test_gpu_fuzz import random_workload
+    w = random_workload(seed)
+    rng = np.random.default_rng(seed + 77)
+    light = [s for s, a in w.apps.items() if a.kind in (W.KIND_PROBE, W.KIND_STEER, W.KIND_PROJECT)]
+    sae = [s for s, a in w.apps.items() if a.kind == W.KIND_SAE]
+    rng.shuffle(light)
+    chains, C_need = {}, w.C_max
+    i = 0
+    while i < len(light):
+        n = int(rng.integers(1, 4))                                   # 1..3 light apps, then maybe an SAE app
+        members = light[i:i + n]
+        i += n
+        if sae and rng.random() < 0.5:
+            members = members + [int(rng.choice(sae))]
+        classes = sum(w.apps[s].W.shape[0] for s in members if w.apps[s].kind == W.KIND_PROBE)
+        if classes > 64 or len(members) < 2:
+            continue
+        for a, b in zip(members[:-1], members[1:]):
+            chains[a] = b
+        C_need = max(C_need, classes)
+    return W.Workload(w.name + "c", w.d_model, w.T_max, w.T_live, w.hidden, w.token_slot, w.apps, w.groups, w.n_slots_max,
+                      w.n_groups_max, C_need, w.k_max, w.r_max, w.d_sae_max, chains=chains)
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_chains(seed):
+    mixlib = _mixlib()
+    w = _random_chained_workload(3000 + seed)
+    out = run_gpu(w, flags=mixlib.MIX_FLAG_SLOT_CHAINS, graph=bool(seed % 2), conditional=bool(seed % 4 == 1))
+    check_chain_parity(W.host(w), out, scale_with_output=True, expect_status=None)
+    assert out["status"] & ~mixlib.MIX_STATUS_TOPK_GENERAL == 0
