@@ -327,7 +327,8 @@ int mix_launches_per_apply(const mix_ctx* ctx);
    array of mix_launches_per_apply() + 1 cudaEvent_t handles created by the caller with timing
    enabled, or NULL to switch the taps off.  Every later mix_apply() records events[0] before
    its first kernel and events[i] after its i-th kernel, on the call's stream; the array is
-   copied.  Kernel order: probe_steer, [probe_multiclass: only if T_max > 2048 and C_max > 1; then probe_tc if also n_groups_max == 0,]
+   copied.  Kernel order: [probe_decide,] probe_steer, [probe_multiclass: only if T_max > 2048 and C_max > 1;
+   probe_decide before and probe_tc after it if also n_groups_max == 0,]
    route, pack, encode, merge, encode (flagged row tiles), select, decode; with
    MIX_FLAG_ENCODE_SIMT the SAE part is route, pack, encode, select, decode; with
    MIX_FLAG_SAE_EDIT_ONLY an edit_only kernel comes last. */

@@ -290,10 +290,10 @@ class Mix:
     @property
     def STAGES(self):
         front = ["probe_steer"]
-        if self.cfg.T_max > 2048 and self.cfg.C_max > 1:
+        if self.cfg.T_max > 2048 and self.cfg.C_max > 1 and not (self.cfg.flags & MIX_FLAG_SLOT_CHAINS):
             front.append("probe_multiclass")
             if self.cfg.n_groups_max == 0:
-                front.append("probe_tc")
+                front = ["probe_decide"] + front + ["probe_tc"]
         if self.cfg.n_groups_max == 0:
             return front
         tail = ["edit_only"] if self.cfg.flags & MIX_FLAG_SAE_EDIT_ONLY else []

@@ -278,7 +278,7 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
     if (load_encode_fn() != MIX_OK) e = cudaErrorUnknown;
     if (e == cudaSuccess) e = probe_tc_prepare();
   }
-  if (e == cudaSuccess && G > 0) {
+  if (e == cudaSuccess && (G > 0 || has_tc_probe_stage(c))) {
     e = cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->body_stream, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming);
@@ -697,22 +697,37 @@ int apply_impl(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream,
     MIX_CUDA(c, cudaStreamWaitEvent(ps, c->ev_fork, 0));
   }
   MIX_CUDA(c, tap());
+  // Multi-class probes of a large batch have two kernels of which exactly one does the work: the 16-row
+  // kernel takes batches sparse in such rows (and every batch of a context with SAE weight sets), the
+  // tensor-core kernel dense ones.  Where both exist, a one-CTA kernel makes the choice first and the
+  // tensor-core kernel -- whose rows no other kernel of this call touches -- runs on the context's side
+  // stream, beside the streaming kernel's pass over the batch.
+  const bool tc = has_tc_probe_stage(c);
+  const bool tc_fork = tc && !c->stage_events_on;
+  CUtensorMap tm_hidden;                         // host-side encoding only: no device work, fine under capture
+  if (tc) {
+    if (make_tmap(&tm_hidden, h, (unsigned long long)c->cfg.T_max, c->cfg.d_model, kTileM) != MIX_OK)
+      MIX_FAIL(c, MIX_ERR_CUDA, "cuTensorMapEncodeTiled failed for hidden");
+    MIX_CUDA(c, launch_mc_decide(c, T, ps));
+    MIX_CUDA(c, tap());
+    if (tc_fork) {
+      MIX_CUDA(c, cudaEventRecord(c->ev_fork, ps));
+      MIX_CUDA(c, cudaStreamWaitEvent(c->side_stream, c->ev_fork, 0));
+      MIX_CUDA(c, launch_probe_tc(c, tm_hidden, T, scores_out, c->side_stream));
+      MIX_CUDA(c, cudaEventRecord(c->ev_join, c->side_stream));
+    }
+  }
   MIX_CUDA(c, launch_probe_steer(c, h, T, scores_out, ps));
   MIX_CUDA(c, tap());
   if (has_multiclass_stage(c)) {
-    // Multi-class probes of a large batch.  With the tensor-core kernel in play, exactly one of the two does
-    // the work (device-side choice made by probe_steer_kernel, see mc_batch_is_dense): the 16-row kernel takes batches sparse in such
-    // rows, the tensor-core kernel dense ones.
     MIX_CUDA(c, launch_probe_multiclass(c, h, T, scores_out, ps));
     MIX_CUDA(c, tap());
-    if (has_tc_probe_stage(c)) {
-      CUtensorMap tm_hidden;                     // host-side encoding only: no device work, fine under capture
-      if (make_tmap(&tm_hidden, h, (unsigned long long)c->cfg.T_max, c->cfg.d_model, kTileM) != MIX_OK)
-        MIX_FAIL(c, MIX_ERR_CUDA, "cuTensorMapEncodeTiled failed for hidden");
-      MIX_CUDA(c, launch_probe_tc(c, tm_hidden, T, scores_out, ps));
-      MIX_CUDA(c, tap());
-    }
   }
+  if (tc && !tc_fork) {
+    MIX_CUDA(c, launch_probe_tc(c, tm_hidden, T, scores_out, ps));
+    MIX_CUDA(c, tap());
+  }
+  if (tc_fork) MIX_CUDA(c, cudaStreamWaitEvent(ps, c->ev_join, 0));
   if (fork) MIX_CUDA(c, cudaEventRecord(c->ev_join, ps));
   if (c->cfg.n_groups_max > 0) {
     MIX_CUDA(c, launch_route(c, T, s, handle, conditional ? 1 : 0));
@@ -752,7 +767,7 @@ int mix_apply_router(mix_ctx* c, float* logits, int n_experts, int T, void* stre
 
 int mix_launches_per_apply(const mix_ctx* c) {
   if (!c) return 0;
-  const int front = 1 + (has_multiclass_stage(c) ? 1 : 0) + (has_tc_probe_stage(c) ? 1 : 0);
+  const int front = 1 + (has_multiclass_stage(c) ? 1 : 0) + (has_tc_probe_stage(c) ? 2 : 0);
   if (c->cfg.n_groups_max == 0) return front;
   return front + ((c->cfg.flags & MIX_FLAG_ENCODE_SIMT) ? 6 : 8) + ((c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) ? 1 : 0);
 }

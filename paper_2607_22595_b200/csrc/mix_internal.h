@@ -137,7 +137,7 @@ struct Ctx {
   int* d_n_flagged;         // [1]
   CUtensorMap* d_tmap_w;    // [n_groups_max] W_enc maps (box kTileK x kTileN, 128B swizzle)
   CUtensorMap* d_tmap_probe;   // [n_slots_max] maps of multi-class probe matrices (box kTileK x 32), large-batch contexts only
-  int* d_mc_dense;          // [1] is this call's batch dense in multi-class probe rows?  written by probe_steer_kernel
+  int* d_mc_dense;          // [1] is this call's batch dense in multi-class probe rows?  written by mc_decide_kernel
   CUtensorMap tmap_panel;   // panel map (box kTileK x kTileM, 128B swizzle)
 
   // probe/steer kernels run beside the SAE chain on this stream (created with the context)
@@ -189,9 +189,10 @@ cudaError_t launch_pdl(int which, void (*kernel)(KArgs...), dim3 grid, dim3 bloc
 // kernel launchers (each returns the CUDA error of the launch)
 cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s);
 // Multi-class probes of large batches have two kernels; both are launched and exactly one does the work, chosen
-// on the device (block 0 of probe_steer_kernel samples the slot map, mc_batch_is_dense in row_lookup.cuh, and
-// leaves the answer in d_mc_dense): probe_tc (tcgen05, streams whole 128-row tiles: batches
+// on the device (mc_decide_kernel samples the slot map, mc_batch_is_dense in row_lookup.cuh, and leaves the
+// answer in d_mc_dense): probe_tc (tcgen05, streams whole 128-row tiles: batches
 // dense in such rows) or probe_multiclass (mma.sync, 16-row tiles: sparse ones).
+cudaError_t launch_mc_decide(const Ctx* c, int T, cudaStream_t s);
 cudaError_t launch_probe_tc(const Ctx* c, const CUtensorMap& tmap_hidden, int T, float* scores, cudaStream_t s);
 cudaError_t launch_probe_multiclass(const Ctx* c, const __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s);
 cudaError_t probe_tc_prepare();   // opt in to the large dynamic shared memory size

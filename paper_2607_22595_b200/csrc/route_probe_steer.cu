@@ -196,19 +196,11 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32, 3)
 probe_steer_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
                    const AppEntry* __restrict__ apps, const GateEntry* __restrict__ gates, int n_slots,
                    __nv_bfloat16* __restrict__ hidden, int d,
-                   float* __restrict__ scores, int C_max, unsigned* __restrict__ status, int multiclass_elsewhere,
-                   int* __restrict__ mc_dense_flag) {
+                   float* __restrict__ scores, int C_max, unsigned* __restrict__ status, int multiclass_elsewhere) {
   __shared__ float s_logit[kWarpsPerBlock][kMaxClasses];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t = blockIdx.x * kWarpsPerBlock + warp;
   const int n_live = __ldg(n_live_p);            // issued together with the slot id: one round trip, not two
-  if (mc_dense_flag != nullptr && blockIdx.x == 0) {
-    // this CTA also decides, for the two multi-class probe kernels that follow in the stream, which of
-    // them takes the batch
-    const int live = min(T, n_live);
-    const bool dense = live > 0 && mc_batch_is_dense(token_slot, apps, n_slots, live);
-    if (threadIdx.x == 0) *mc_dense_flag = dense ? 1 : 0;
-  }
   const int slot = t < T ? __ldg(token_slot + t) : -1;
   if (t >= min(T, n_live)) return;
   const RowApp a = lookup(slot, t, apps, gates, n_slots, status, lane == 0);
@@ -870,11 +862,25 @@ __global__ void fold_bias_kernel(const __nv_bfloat16* __restrict__ W_enc, const 
   if (lane == 0) b_eff[j] = b_enc[j] - acc;
 }
 
+// One small CTA decides, for the two multi-class probe kernels, which of them takes this call's batch.
+__global__ void __launch_bounds__(64)
+mc_decide_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
+                 const AppEntry* __restrict__ apps, int n_slots, int* __restrict__ mc_dense_flag) {
+  const int live = min(T, __ldg(n_live_p));
+  const bool dense = mc_batch_is_dense(token_slot, apps, n_slots, max(live, 1)) && live > 0;
+  if (threadIdx.x == 0) *mc_dense_flag = dense ? 1 : 0;
+}
+
 }  // namespace
 
 
 bool has_multiclass_stage(const Ctx* c) {
   return c->cfg.T_max > kTeamMaxRows && c->cfg.C_max > 1 && !(c->cfg.flags & MIX_FLAG_SLOT_CHAINS);
+}
+
+cudaError_t launch_mc_decide(const Ctx* c, int T, cudaStream_t s) {
+  mc_decide_kernel<<<1, 64, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->cfg.n_slots_max, c->d_mc_dense);
+  return cudaGetLastError();
 }
 
 // The tensor-core probe kernel holds a whole SM's shared memory, as the SAE encode does: beside an encode
@@ -896,8 +902,7 @@ cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float
     const int blocks = (c->cfg.T_max + kWarpsPerBlock - 1) / kWarpsPerBlock;
     probe_steer_kernel<<<blocks, kWarpsPerBlock * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates,
                                                               c->cfg.n_slots_max, hidden, c->cfg.d_model, scores,
-                                                              c->cfg.C_max, c->d_status, has_multiclass_stage(c) ? 1 : 0,
-                                                              has_tc_probe_stage(c) ? c->d_mc_dense : nullptr);
+                                                              c->cfg.C_max, c->d_status, has_multiclass_stage(c) ? 1 : 0);
   }
   return cudaGetLastError();
 }

@@ -45,7 +45,7 @@ def test_dense_batch_many_probes_per_tile(graph):
     w = _probe_workload(T_max, T_live, d, slot, classes, acts)
     out = run_gpu(w, graph=graph)
     st = check_parity(W.host(w), out)
-    assert st["rows"] == T_max and out["mix"].STAGES == ["probe_steer", "probe_multiclass", "probe_tc"]
+    assert st["rows"] == T_max and out["mix"].STAGES == ["probe_decide", "probe_steer", "probe_multiclass", "probe_tc"]
 
 
 def test_dense_batch_with_other_kinds_unhooked_rows_and_a_gate():
