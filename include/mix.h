@@ -20,8 +20,10 @@
  *   MIX_PROJECT directional ablation, the usual statement of "subtract a vector" for a refusal-style
  *              direction (Section 3 "Write"; Table 1, row 1): h[t,:] <- bf16( h - beta (h . r) r ),
  *              in place; r is used as given (pass a unit vector for an orthogonal projection).
- *   slot -1    no app: the row is neither read nor written (Section 4.2 "Toggling
- *              semantics": an inactive app costs a request nothing).
+ *   slot -1    no app: the row is never written and stays bit-identical (Section 4.2 "Toggling
+ *              semantics": an inactive app costs a request nothing).  It is not read either, with one
+ *              exception: in a batch of more than 2048 rows that is dense in multi-class probe rows,
+ *              the probe kernel streams whole 128-row tiles and discards the rows that are not its own.
  *
  * Rows are independent.  Activation of an app for a request is data (the slot map and the
  * small device tables), never launch structure: mix_apply() only enqueues kernels with a
