@@ -489,6 +489,17 @@ def extras_decode_variants(w, hiddens, scores, mixlib):
             mb.apply(h, sc, stream=stream)
     out["probe_then_steer_two_calls_us_per_step"] = measure(Two())
     ma.destroy(); mb.destroy()
+    # 32 hooked layers: 32 contexts (one per layer, same apps) applied one after the other to the decode step's
+    # hidden state, all in the captured graph; per decode step, i.e. per 32 hook calls
+    layers = [W.make_context(mixlib.Mix, w) for _ in range(32)]
+
+    class Stack:
+        def apply(self, h, sc, stream=None):
+            for mm in layers:
+                mm.apply(h, sc, stream=stream)
+    out["32_hooked_layers_us_per_decode_step"] = measure(Stack())
+    for mm in layers:
+        mm.destroy()
     return out
 
 
