@@ -533,3 +533,37 @@ def test_maximum_k_and_edit_list(add_error):
     out = run_gpu(w)
     check_parity(W.host(w), out, expect_status=None)
     assert out["status"] & ~_mixlib().MIX_STATUS_TOPK_GENERAL == 0
+
+
+def test_create_destroy_returns_all_device_memory():
+    """Every allocation of every kind of context (SAE with both encoder forms, chains, the large-batch probe
+    kernels, registrations that make the library keep copies) is released by mix_destroy."""
+    mixlib = _mixlib()
+    g = torch.Generator(device=DEV); g.manual_seed(0)
+
+    def cycle():
+        w = W.make_tiny(DEV)
+        m = W.make_context(mixlib.Mix, w, flags=mixlib.MIX_FLAG_RETILE_W_ENC | mixlib.MIX_FLAG_SLOT_CHAINS)
+        m.apply(w.hidden.clone()); m.destroy()
+        sae = W.make_sae_weights(g, DEV, 128, 512, W.SAE_TOPK, k=4, fp8=True)
+        m = mixlib.Mix(d_model=128, T_max=8, n_slots_max=1, n_groups_max=1, k_max=4, r_max=1, d_sae_max=512,
+                       flags=mixlib.MIX_FLAG_FP8_W_ENC)
+        m.register_sae_weights(0, 512, sae.act, 4, sae.W_enc, sae.b_enc, sae.W_dec, w_scale=sae.w_scale)
+        m.destroy()
+        sae = W.make_sae_weights(g, DEV, 128, 512, W.SAE_RELU)
+        m = mixlib.Mix(d_model=128, T_max=8, n_slots_max=1, n_groups_max=1, r_max=1, d_sae_max=512)
+        m.register_sae_weights(0, 512, sae.act, 0, sae.W_enc, sae.b_enc, sae.W_dec, b_dec=torch.zeros(128, device=DEV),
+                               center_input=True)
+        m.destroy()
+        m = mixlib.Mix(d_model=128, T_max=4096, n_slots_max=4, C_max=8)          # both multi-class probe kernels
+        m.register_probe(0, torch.zeros((8, 128), device=DEV, dtype=torch.bfloat16), None, mixlib.MIX_ACT_SOFTMAX)
+        m.destroy()
+
+    cycle()                                              # first use may load modules and grow caches
+    torch.cuda.synchronize(); torch.cuda.empty_cache()
+    free0, _ = torch.cuda.mem_get_info()
+    for _ in range(20):
+        cycle()
+    torch.cuda.synchronize(); torch.cuda.empty_cache()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free0 - free1 < (8 << 20), "device memory shrank by %d bytes over 20 create/destroy cycles" % (free0 - free1)
