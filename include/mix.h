@@ -289,7 +289,9 @@ int mix_set_feature_out(mix_ctx* ctx, int* topk_idx, float* topk_val, int* n_act
    device fp32 [T_max, C_max] or NULL; only the first n_classes entries of probe rows are
    written.  Enqueues kernels on `stream` (when the context has SAE weight sets, the probe /
    steering kernels run on a context-owned side stream forked from and joined back into `stream`
-   by events, so they overlap the SAE chain) and returns; safe to capture.  Device-side
+   by events, so they overlap the SAE chain; in a context for more than 2048 rows with multi-class
+   probes and no SAE weight sets, the tensor-core probe kernel runs on that side stream beside the
+   streaming kernel) and returns; safe to capture.  Device-side
    problems (bad slot ids, ...) are reported through the status word, never by faulting.
    Errors: INVALID_ARG (NULL hidden, misaligned), OUT_OF_RANGE (T), CUDA (launch failure). */
 int mix_apply(mix_ctx* ctx, void* hidden, int T, float* scores_out, void* stream);
