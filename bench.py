@@ -498,6 +498,10 @@ def extras_decode_variants(w, hiddens, scores, mixlib):
             for mm in layers:
                 mm.apply(h, sc, stream=stream)
     out["32_hooked_layers_us_per_decode_step"] = measure(Stack())
+    # changing one per-request parameter between replays, host cost per replay of a one-kernel graph: a 4-byte
+    # write into a device table (what this library does) vs a kernel-node parameter update (the paper's way)
+    tab, node = layers[0].bench_param_update(iters=3000)
+    out["param_change_plus_graph_launch_us"] = {"device_table_write": tab, "kernel_node_param_update": node}
     for mm in layers:
         mm.destroy()
     return out

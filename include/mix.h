@@ -338,6 +338,19 @@ int mix_launches_per_apply(const mix_ctx* ctx);
    MIX_FLAG_SAE_EDIT_ONLY an edit_only kernel comes last. */
 int mix_set_stage_events(mix_ctx* ctx, void* const* events);
 
+/* Measurement aid for the paper's "CUDA-graph-safe kernel design" paragraph (separate static graph
+   structure from per-request dynamic parameters; reuse the instantiated graph and update only the
+   affected kernel-node parameters before launch).  This library never updates node parameters: all
+   dynamic state lives in device tables written by stream-ordered copies.  The call times both
+   mechanisms on a one-kernel graph, `iters` times each, host wall clock per iteration including the
+   graph launch, with one synchronisation at the end: (a) a 4-byte cudaMemcpyAsync into a device table
+   the kernel reads, then cudaGraphLaunch; (b) cudaGraphExecKernelNodeSetParams with the new value
+   as a kernel argument, then cudaGraphLaunch.  Both kernels add the value to an accumulator and
+   the two sums are compared.  us_table / us_node: host floats, microseconds per iteration.
+   Synchronises `stream`; not capturable; allocates and frees 8 bytes of device memory.
+   Errors: INVALID_ARG (NULL outputs, iters < 1), CUDA (API failure or the two sums differ). */
+int mix_bench_param_update(mix_ctx* ctx, int iters, float* us_table, float* us_node, void* stream);
+
 /* Test / profiling taps into the SAE workspace after a mix_apply (device pointers owned by
    the context; valid until mix_destroy):  panel_rows int32 [n_panel_rows] gives the token
    index of each packed panel row (-1 = padding), z the fp32 pre-activations

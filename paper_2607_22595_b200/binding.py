@@ -33,6 +33,7 @@ EXPORTS = [
     "mix_register_app", "mix_unregister_app", "mix_set_gate", "mix_set_chain", "mix_update_steer_alpha", "mix_update_sae_edits",
     "mix_set_slot_map", "mix_set_request_map", "mix_set_feature_out", "mix_apply", "mix_apply_conditional", "mix_apply_router", "mix_get_status",
     "mix_launches_per_apply", "mix_set_stage_events", "mix_debug_workspace", "mix_sae_apply_static",
+    "mix_bench_param_update",
 ]
 
 
@@ -105,6 +106,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.mix_get_status.argtypes = [vp, C.POINTER(C.c_uint), vp]
     lib.mix_launches_per_apply.argtypes = [vp]
     lib.mix_set_stage_events.argtypes = [vp, C.POINTER(vp)]
+    lib.mix_bench_param_update.argtypes = [vp, ci, C.POINTER(C.c_float), C.POINTER(C.c_float), vp]
     lib.mix_sae_apply_static.argtypes = [vp, ci, ci, C.POINTER(MixSaeWeights), C.POINTER(MixSaeApp), vp, vp, vp,
                                          C.c_char_p, ci]
     lib.mix_debug_workspace.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(C.c_longlong), C.POINTER(ci)]
@@ -312,6 +314,12 @@ class Mix:
         arr = (C.c_void_p * len(events))(*[e.cuda_event for e in events])
         self._check(self.lib.mix_set_stage_events(self.ctx, arr))
         self._keep["ev"] = events
+
+    def bench_param_update(self, iters=2000, stream=None):
+        """(us per iteration with a device-table write, us per iteration with a kernel-node parameter update)."""
+        a, b = C.c_float(0), C.c_float(0)
+        self._check(self.lib.mix_bench_param_update(self.ctx, int(iters), C.byref(a), C.byref(b), _stream(stream)))
+        return float(a.value), float(b.value)
 
     def debug_workspace(self):
         pr, z, ld, n = C.c_void_p(), C.c_void_p(), C.c_longlong(), C.c_int()

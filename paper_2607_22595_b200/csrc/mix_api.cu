@@ -4,6 +4,7 @@
 #include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
+#include <time.h>
 
 #include "mix_internal.h"
 
@@ -24,6 +25,13 @@ namespace {
     cudaError_t e_ = (expr);                                                                 \
     if (e_ != cudaSuccess) MIX_FAIL(ctx, MIX_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e_)); \
   } while (0)
+
+__global__ void bench_add_from_table(const float* __restrict__ table, float* __restrict__ acc) {
+  if (threadIdx.x == 0) acc[0] += table[0];
+}
+__global__ void bench_add_from_param(float v, float* __restrict__ acc) {
+  if (threadIdx.x == 0) acc[0] += v;
+}
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -793,6 +801,64 @@ int mix_set_stage_events(mix_ctx* c, void* const* events) {
     }
     c->stage_events_on = 1;
   }
+  return MIX_OK;
+}
+
+int mix_bench_param_update(mix_ctx* c, int iters, float* us_table, float* us_node, void* stream) {
+  if (!c) return MIX_ERR_INVALID_ARG;
+  if (!us_table || !us_node || iters < 1) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "NULL output or iters < 1");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  float* d = nullptr;                                   // d[0]: table entry / unused, d[1]: accumulator
+  MIX_CUDA(c, cudaMalloc(reinterpret_cast<void**>(&d), 2 * sizeof(float)));
+  cudaGraph_t graph[2] = {nullptr, nullptr};
+  cudaGraphExec_t exec[2] = {nullptr, nullptr};
+  cudaGraphNode_t node[2];
+  float sums[2] = {0.f, 0.f};
+  double us[2] = {0.0, 0.0};
+  cudaError_t e = cudaSuccess;
+  for (int v = 0; v < 2 && e == cudaSuccess; ++v) {
+    const float* table = d;
+    float* acc = d + 1;
+    float value = 0.f;
+    void* args_table[2] = {&table, &acc};
+    void* args_param[2] = {&value, &acc};
+    cudaKernelNodeParams kp;
+    memset(&kp, 0, sizeof(kp));
+    kp.func = v == 0 ? reinterpret_cast<void*>(bench_add_from_table) : reinterpret_cast<void*>(bench_add_from_param);
+    kp.gridDim = dim3(1);
+    kp.blockDim = dim3(32);
+    kp.kernelParams = v == 0 ? args_table : args_param;
+    e = cudaGraphCreate(&graph[v], 0);
+    if (e == cudaSuccess) e = cudaGraphAddKernelNode(&node[v], graph[v], nullptr, 0, &kp);
+    if (e == cudaSuccess) e = cudaGraphInstantiate(&exec[v], graph[v], 0);
+    if (e == cudaSuccess) e = cudaMemsetAsync(d, 0, 2 * sizeof(float), s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) break;
+    timespec t0, t1;
+    clock_gettime(CLOCK_MONOTONIC, &t0);
+    for (int i = 0; i < iters && e == cudaSuccess; ++i) {
+      value = (float)(i % 7);                           // small integers: the sums are exact in fp32
+      if (v == 0) {
+        e = cudaMemcpyAsync(d, &value, sizeof(float), cudaMemcpyHostToDevice, s);   // pageable source: staged at once
+      } else {
+        e = cudaGraphExecKernelNodeSetParams(exec[v], node[v], &kp);
+      }
+      if (e == cudaSuccess) e = cudaGraphLaunch(exec[v], s);
+    }
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    clock_gettime(CLOCK_MONOTONIC, &t1);
+    us[v] = ((t1.tv_sec - t0.tv_sec) * 1e9 + (t1.tv_nsec - t0.tv_nsec)) / 1e3 / iters;
+    if (e == cudaSuccess) e = cudaMemcpy(&sums[v], d + 1, sizeof(float), cudaMemcpyDeviceToHost);
+  }
+  for (int v = 0; v < 2; ++v) {
+    if (exec[v]) cudaGraphExecDestroy(exec[v]);
+    if (graph[v]) cudaGraphDestroy(graph[v]);
+  }
+  cudaFree(d);
+  MIX_CUDA(c, e);
+  if (sums[0] != sums[1]) MIX_FAIL(c, MIX_ERR_CUDA, "the two mechanisms disagree: %g vs %g", (double)sums[0], (double)sums[1]);
+  *us_table = (float)us[0];
+  *us_node = (float)us[1];
   return MIX_OK;
 }
 

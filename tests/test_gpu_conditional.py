@@ -91,3 +91,16 @@ def test_conditional_outside_capture_is_an_error_and_no_sae_context_is_plain():
     ref = run_gpu(wd)
     assert np.array_equal(W.bits(hd), ref["hidden"])
     md.destroy()
+
+
+def test_param_update_measurement_entry_runs_and_agrees():
+    """mix_bench_param_update: the two mechanisms (device-table write, kernel-node parameter update) accumulate
+    the same sum; both times are positive; bad arguments are rejected."""
+    mixlib = _mixlib()
+    m = mixlib.Mix(d_model=64, T_max=8, n_slots_max=1)
+    a, b = m.bench_param_update(iters=300)
+    assert 0.0 < a < 1e4 and 0.0 < b < 1e4
+    with pytest.raises(mixlib.MixError) as e:
+        m.bench_param_update(iters=0)
+    assert e.value.code == -1
+    m.destroy()
