@@ -87,7 +87,8 @@ enum {
                                          streams whole DRAM pages instead of 128-byte pieces of 256 different rows.  Costs
                                          2 * d_sae * d bytes per weight set, allocated at registration (W_enc itself is no
                                          longer read by mix_apply and need not stay alive) */,
-  MIX_FLAG_TEST_STALL_ENCODE = 1u << 2 /* test hook for the time-out path: the encode kernel's producer never delivers a
+  MIX_FLAG_TEST_STALL_ENCODE = 1u << 2 /* test hook for the time-out path: the producer of the encode kernel (and of the
+                                         tensor-core probe kernel) never delivers a
                                          tile and every bounded wait is capped at ~1 ms, so each CTA gives up, raises
                                          MIX_STATUS_WAIT_TIMEOUT, frees its tensor memory and returns; the SAE rows of that
                                          call are not meaningful.  Nothing hangs and the context stays usable */,

@@ -35,7 +35,8 @@ constexpr int kPBBytes = kPBlocks * kPBlockBytes;      // 8 KiB
 constexpr int kPStageBytes = kPABytes + kPBBytes;
 constexpr int kPThreads = 7 * 32;
 constexpr int kPTmemCols = 2 * kPBlocks * kPBlockCols; // 128: two accumulators of 64 columns
-__device__ const long long kPWaitCycles = 4000000000ll;   // ~2 s at 2 GHz
+constexpr long long kPWaitCycles = 4000000000ll;       // ~2 s at 2 GHz
+constexpr long long kPWaitCyclesTest = 2000000ll;      // ~1 ms: the cap under MIX_FLAG_TEST_STALL_ENCODE
 
 struct PDesc {
   int t0;                       // first row of the tile
@@ -53,6 +54,7 @@ struct __align__(8) PShared {
   unsigned long long desc_empty[2];
   unsigned tmem_base;
   volatile int abort_flag;
+  long long wait_cycles;        // cap of every bounded wait in this launch
   PDesc desc[2];
 };
 constexpr int kPSmemBytes = kPStages * kPStageBytes + 1024 /* alignment slack */ + 1024 /* PShared */;
@@ -60,14 +62,15 @@ static_assert(kPSmemBytes <= 227 * 1024, "shared memory per CTA");
 static_assert(sizeof(PShared) <= 1024, "PShared must fit the space reserved for it");
 
 __device__ __forceinline__ bool pwait(unsigned bar, unsigned parity, PShared* sh, unsigned* status) {
-  return mbar_wait_bounded(bar, parity, &sh->abort_flag, &kPWaitCycles, status);
+  return mbar_wait_bounded(bar, parity, &sh->abort_flag, &sh->wait_cycles, status);
 }
 
 __global__ void __launch_bounds__(kPThreads, 1)
 probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const CUtensorMap* __restrict__ tmap_probe,
                 const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
                 const AppEntry* __restrict__ apps, const GateEntry* __restrict__ gates, int n_slots, int d,
-                float* __restrict__ scores, int C_max, unsigned* __restrict__ status, const int* __restrict__ mc_dense_flag) {
+                float* __restrict__ scores, int C_max, unsigned* __restrict__ status, const int* __restrict__ mc_dense_flag,
+                int test_stall) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   PShared* sh = reinterpret_cast<PShared*>(tiles + kPStages * kPStageBytes);
@@ -88,6 +91,7 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const CUtensorM
       mbar_init(smem_u32(&sh->desc_empty[a]), 6);      // producer, MMA issuer, four epilogue warps
     }
     sh->abort_flag = 0;
+    sh->wait_cycles = test_stall ? kPWaitCyclesTest : kPWaitCycles;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -186,6 +190,9 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const CUtensorM
         bool ok = true;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!pwait(smem_u32(&sh->empty[stage]), phase ^ 1u, sh, status)) { ok = false; break; }
+          // Test hook (MIX_FLAG_TEST_STALL_ENCODE): the producer never fills a stage, so the consumers' bounded
+          // waits run out and the whole CTA leaves through the time-out path.
+          if (test_stall) { ok = false; break; }
           const unsigned bar = smem_u32(&sh->full[stage]);
           mbar_expect_tx(bar, kPABytes + nb * kPBlockBytes);
           const unsigned sa = smem_u32(tiles + stage * kPStageBytes);
@@ -320,7 +327,8 @@ cudaError_t launch_probe_tc(const Ctx* c, const CUtensorMap& tmap_hidden, int T,
   if (scores == nullptr) return cudaSuccess;
   probe_tc_kernel<<<c->n_sms, kPThreads, kPSmemBytes, s>>>(tmap_hidden, c->d_tmap_probe, c->d_token_slot, c->d_n_live, T,
                                                            c->d_apps, c->d_gates, c->cfg.n_slots_max, c->cfg.d_model, scores,
-                                                           c->cfg.C_max, c->d_status, c->d_mc_dense);
+                                                           c->cfg.C_max, c->d_status, c->d_mc_dense,
+                                                           (c->cfg.flags & MIX_FLAG_TEST_STALL_ENCODE) ? 1 : 0);
   return cudaGetLastError();
 }
 

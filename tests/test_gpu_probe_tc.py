@@ -95,3 +95,20 @@ def test_same_scores_from_both_kernels():
     assert np.array_equal(written, ~np.isnan(b["scores"])) and written.any()
     assert np.abs(a["scores"][written] - b["scores"][written]).max() <= 2e-6
     assert np.array_equal(a["hidden"], b["hidden"])
+
+
+def test_time_out_path_of_the_tensor_core_probe_kernel():
+    """With the test hook the producer delivers nothing and every wait is capped at about a millisecond: each
+    CTA gives up, raises the status bit, frees its tensor memory and returns; nothing hangs, no row is written,
+    and the device runs an ordinary call right afterwards."""
+    mixlib = _mixlib()
+    T_max, d = 2304, 256
+    slot = (np.arange(T_max) // 64) % 2
+    w = _probe_workload(T_max, T_max, d, slot, [4, 12], [W.ACT_SOFTMAX, W.ACT_SOFTMAX])
+    out = run_gpu(w, flags=mixlib.MIX_FLAG_TEST_STALL_ENCODE)
+    assert out["status"] & mixlib.MIX_STATUS_WAIT_TIMEOUT
+    assert np.array_equal(out["hidden"], W.bits(w.hidden))
+    assert np.isnan(out["scores"]).all()                               # the canary: no score was written
+    good = run_gpu(w)
+    assert good["status"] == 0
+    check_parity(W.host(w), good)
