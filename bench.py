@@ -357,9 +357,10 @@ def extras_multiclass(peaks, mixlib, small=False):
     round-robin over the probes): the tensor-core probe kernel plus the pass of the streaming kernel that
     skips these rows.  Bytes counted: the hidden state once."""
     out = {}
-    shapes = [(5120, 16384, 16, 8)] if small else [(4096, 65536, 2, 4), (4096, 65536, 16, 8), (4096, 65536, 32, 4),
-                                                   (8192, 32768, 8, 4), (5120, 16384, 16, 8)]
-    for d, T, C, n_probe in shapes:
+    shapes = [(5120, 16384, 16, 8, 1.0)] if small else [(4096, 65536, 2, 4, 1.0), (4096, 65536, 16, 8, 1.0),
+                                                        (4096, 65536, 32, 4, 1.0), (8192, 32768, 8, 4, 1.0),
+                                                        (5120, 16384, 16, 8, 1.0), (4096, 65536, 16, 8, 0.25)]
+    for d, T, C, n_probe, density in shapes:
         g = torch.Generator(device="cuda"); g.manual_seed(1)
         hidden = torch.randn((T, d), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
         m = mixlib.Mix(d_model=d, T_max=T, n_slots_max=n_probe, C_max=C)
@@ -367,17 +368,21 @@ def extras_multiclass(peaks, mixlib, small=False):
         for s_ in range(n_probe):
             Wp = (torch.randn((C, d), generator=g, device="cuda") * d ** -0.5).to(torch.bfloat16); keep.append(Wp)
             m.register_probe(s_, Wp, None, mixlib.MIX_ACT_SOFTMAX)
-        m.set_slot_map(torch.from_numpy(((np.arange(T) // 256) % n_probe).astype(np.int32)).cuda())
+        req = np.arange(T) // 256                                           # requests of 256 rows
+        slot_map = (req % n_probe).astype(np.int32)
+        if density < 1.0:                                                    # every (1/density)-th request is hooked
+            slot_map = np.where(req % int(round(1 / density)) == 0, (req // int(round(1 / density))) % n_probe, -1).astype(np.int32)
+        m.set_slot_map(torch.from_numpy(slot_map).cuda())
         scores = torch.zeros((T, C), dtype=torch.float32, device="cuda")
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         best = 1e9
         for _ in range(6):
             e0.record(); m.apply(hidden, scores); e1.record(); torch.cuda.synchronize()
             best = min(best, e0.elapsed_time(e1))
-        nbytes = T * d * 2
+        nbytes = int((slot_map >= 0).sum()) * d * 2                        # hooked rows only
         st = time_stages(m, lambda: m.apply(hidden, scores))
         tc_ms = st["probe_tc"]
-        out["d=%d T=%d C=%d probes=%d" % (d, T, C, n_probe)] = {
+        out["d=%d T=%d C=%d probes=%d hooked=%d%%" % (d, T, C, n_probe, round(100 * density))] = {
             "ms": best, "gbs": nbytes / best / 1e6, "frac_hbm_peak": nbytes / best / 1e6 / peaks["hbm_gbs"],
             "frac_hbm_nominal": nbytes / best / 1e6 / NOMINAL_HBM_GBS, "stage_ms": st,
             "probe_tc_kernel_alone": {"gbs": nbytes / tc_ms / 1e6, "frac_hbm_peak": nbytes / tc_ms / 1e6 / peaks["hbm_gbs"]},
