@@ -91,3 +91,65 @@ def test_bf16_rounding_is_nearest_and_monotone(x):
         for nb in (up, dn):
             if np.isfinite(nb) and (nb > 0) == (y > 0) and y != 0:
                 assert abs(y - x) <= abs(nb - x) + 0.0        # no neighbour is closer
+
+
+@settings(max_examples=40, deadline=None)
+@given(st.integers(0, 2 ** 32 - 1), st.integers(1, 4), st.booleans())
+def test_chain_is_hook_after_hook_and_commutes_with_row_permutation(seed, length, with_gate):
+    """Random chains of read / write apps: the chained hook equals the single-app hook applied once per app to
+    the bf16 output of the previous one; probe columns follow the static layout; permuting the rows permutes
+    the results."""
+    rng = np.random.default_rng(seed)
+    d, T = 32, 9
+    apps, chains, cols = {}, {}, []
+    C_total = 0
+    for s in range(length):
+        kind = int(rng.integers(0, 3))
+        if kind == 0:
+            C = int(rng.integers(1, 4))
+            apps[s] = W.Probe(_bf(rng.standard_normal((C, d))), rng.standard_normal(C).astype(np.float32),
+                              W.ACT_SOFTMAX if C > 1 else W.ACT_SIGMOID)
+            cols.append((s, C_total, C)); C_total += C
+        elif kind == 1:
+            apps[s] = W.Steer(_bf(rng.standard_normal(d)), float(np.float32(rng.uniform(-3, 3))))
+        else:
+            r = rng.standard_normal(d); apps[s] = W.Project(_bf(r / np.linalg.norm(r)), 1.0)
+        if s + 1 < length:
+            chains[s] = s + 1
+    hidden = _bf(rng.standard_normal((T, d)))
+    if with_gate:
+        sc = rng.standard_normal((T, 1)).astype(np.float32)
+        apps[0].gate = W.Gate(sc, 0, W.GATE_GE, 0.0)
+    slot = np.where(rng.random(T) < 0.7, 0, -1).astype(np.int32)
+    w = W.Workload("c", d, T, T, hidden, slot, apps, {}, n_slots_max=length, C_max=max(C_total, 1), chains=chains)
+    r = O.apply_chain_hook(w)
+    for t in range(T):
+        cur = hidden[t:t + 1].copy()
+        want_scores = {}
+        if slot[t] == 0:
+            for s in range(length):
+                one_apps = {0: apps[s]}
+                if getattr(apps[s], "gate", None) is not None:       # the gate indexes rows of the full batch
+                    if not O.gate_open(apps[s].gate, t):
+                        continue
+                    import copy
+                    a2 = copy.copy(apps[s]); a2.gate = None
+                    one_apps = {0: a2}
+                w1 = W.Workload("s", d, 1, 1, cur, np.array([0], np.int32), one_apps, {}, n_slots_max=1, C_max=4)
+                one = O.apply_hook(w1)
+                cur = one.out_bits[0][None, :].copy()
+                if 0 in one.scores:
+                    c0 = [c for (ss, c, n) in cols if ss == s][0]
+                    for j, v in enumerate(one.scores[0]):
+                        want_scores[c0 + j] = float(v)
+        assert np.array_equal(r.out_bits[t], cur[0])
+        assert r.scores[t] == want_scores
+    perm = rng.permutation(T)
+    wp = W.Workload("p", d, T, T, hidden[perm], slot[perm], apps, {}, n_slots_max=length, C_max=max(C_total, 1), chains=chains)
+    if with_gate:
+        import copy
+        apps_p = dict(apps); g0 = copy.copy(apps[0]); g0.gate = W.Gate(sc[perm], 0, W.GATE_GE, 0.0); apps_p[0] = g0
+        wp.apps = apps_p
+    rp = O.apply_chain_hook(wp)
+    for i, t in enumerate(perm):
+        assert np.array_equal(rp.out_bits[i], r.out_bits[int(t)]) and rp.scores[i] == r.scores[int(t)]
