@@ -567,3 +567,47 @@ def test_create_destroy_returns_all_device_memory():
     torch.cuda.synchronize(); torch.cuda.empty_cache()
     free1, _ = torch.cuda.mem_get_info()
     assert free0 - free1 < (8 << 20), "device memory shrank by %d bytes over 20 create/destroy cycles" % (free0 - free1)
+
+
+@pytest.mark.parametrize("which", ["tiny", "mixed", "dense_probes"])
+def test_guard_bands_around_the_callers_buffers_stay_intact(which):
+    """hidden, scores and the feature read-out buffers sit inside larger allocations whose extra rows before and
+    after carry a canary pattern: no kernel of the call may write (or, for hidden, change) a byte outside the
+    [T_max, ...] window it was given."""
+    mixlib = _mixlib()
+    if which == "tiny":
+        w = W.make_tiny(DEV)
+    elif which == "mixed":
+        w = W.make_mixed(DEV, d=320, T=2601, R=48, d_sae=1024, cap=300, mu=4.0, edit_hint=oracle_edit_hint)
+    else:
+        T, d = 2560, 256
+        g = torch.Generator(device=DEV); g.manual_seed(5)
+        apps = {s: W.Probe((torch.randn((C, d), generator=g, device=DEV) * d ** -0.5).to(torch.bfloat16), None, W.ACT_SOFTMAX)
+                for s, C in enumerate([3, 17])}
+        hidden = torch.randn((T, d), generator=g, device=DEV, dtype=torch.float32).to(torch.bfloat16)
+        w = W.Workload("dense", d, T, T, hidden, ((np.arange(T) // 100) % 2).astype(np.int32), apps, {}, n_slots_max=2, C_max=17)
+    T, d, C, k_max = w.T_max, w.d_model, max(w.C_max, 1), max(w.k_max, 1)
+    G = 3                                                   # guard rows on each side
+    def guarded(cols, dtype, fill):
+        big = torch.full((T + 2 * G, cols), fill, dtype=dtype, device=DEV)
+        return big, big[G:G + T]
+    h_big, h = guarded(d, torch.bfloat16, 0.0)
+    h_big[:G] = 123.0; h_big[G + T:] = -77.0
+    h.copy_(w.hidden)
+    s_big, scores = guarded(C, torch.float32, 4242.0)
+    i_big, tk_idx = guarded(k_max, torch.int32, -99)
+    v_big, tk_val = guarded(k_max, torch.float32, 4242.0)
+    n_big, n_act = guarded(1, torch.int32, -99)
+    m = W.make_context(mixlib.Mix, w)
+    if w.n_groups_max > 0:
+        m.set_feature_out(tk_idx, tk_val, n_act.view(-1))
+    m.apply(h, scores)
+    torch.cuda.synchronize()
+    assert (h_big[:G] == 123.0).all() and (h_big[G + T:] == -77.0).all()
+    for big, fill in ((s_big, 4242.0), (i_big, -99), (v_big, 4242.0), (n_big, -99)):
+        assert (big[:G] == fill).all() and (big[G + T:] == fill).all()
+    assert m.get_status() == 0
+    # and inside the window the result is the usual one
+    ref = run_gpu(w)
+    assert np.array_equal(W.bits(h), ref["hidden"])
+    m.destroy()
