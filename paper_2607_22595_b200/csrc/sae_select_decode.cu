@@ -460,6 +460,66 @@ __device__ __forceinline__ void accumulate_list(float (*acc)[8], const float* co
   }
 }
 
+constexpr int kDecRows = kDecThreads / 32;     // packed rows per CTA of decode_kernel: one per warp
+
+// A row that keeps the error term: one warp works out f'_j - f_j for each of its edit entries and leaves
+// them, with the row's slot (-1 when no edit changes anything: the row then stays bit-exact) and the
+// decoder pointer, for decode_delta_kernel.
+__device__ __forceinline__ void warp_edit_coefs(int p, int slot, const AppEntry& app, const GroupEntry& ge,
+                                                const float* __restrict__ z, const int* __restrict__ K,
+                                                const float* __restrict__ Kv, const int* __restrict__ edit_idx,
+                                                const float* __restrict__ edit_val,
+                                                const unsigned char* __restrict__ edit_mode, int r_max,
+                                                RowDelta* __restrict__ row_delta, float* __restrict__ edit_coef,
+                                                int* s_e, float* s_f, int lane) {
+  const int n_edit = app.n_edit;
+  for (int e = lane; e < n_edit; e += 32) {
+    s_e[e] = edit_idx[slot * r_max + e];
+    s_f[e] = 0.f;
+  }
+  __syncwarp();
+  if (ge.act == MIX_SAE_TOPK) {
+    // the value of a selected feature comes from the row's TopK list (the Z scratch is not written for
+    // TopK sets unless the row took the fallback selection); an unselected one is 0
+    for (int i = lane; i < ge.k; i += 32) {
+      const int id = K[i];
+      for (int e = 0; e < n_edit; ++e)
+        if (s_e[e] == id) s_f[e] = fmaxf(Kv[i], 0.f);
+    }
+    __syncwarp();
+  }
+  bool any = false;
+  for (int e = lane; e < n_edit; e += 32) {
+    const int j = s_e[e];
+    bool alive = true;                                   // a later entry for the same feature wins
+    for (int e2 = e + 1; e2 < n_edit; ++e2) alive = alive && (s_e[e2] != j);
+    float f;
+    if (ge.act == MIX_SAE_RELU) {
+      f = fmaxf(z[j], 0.f);
+    } else if (ge.act == MIX_SAE_JUMPRELU) {
+      const float zj = z[j];
+      f = zj > ge.theta[j] ? zj : 0.f;
+    } else {
+      f = s_f[e];
+    }
+    const float fnew = edit_mode[slot * r_max + e] == MIX_EDIT_CLAMP ? edit_val[slot * r_max + e] : 0.f;
+    const float delta = alive ? fnew - f : 0.f;
+    edit_coef[(size_t)p * r_max + e] = delta;
+    any = any || delta != 0.f;
+  }
+  any = __any_sync(0xffffffffu, any);
+  if (lane == 0) {
+    RowDelta rd;
+    rd.slot = any ? slot : -1;
+    rd.n_edit = n_edit;
+    rd.W_dec = ge.W_dec;
+    row_delta[p] = rd;
+  }
+}
+
+// decode_kernel: a CTA owns kDecRows consecutive packed rows.  Rows that keep the error term only get
+// their edit coefficients (one warp per row, all at once); rows whose app replaces the residual are
+// then rebuilt one after the other by the whole CTA:  h' = b_dec + sum_j f'_j W_dec[j].
 __global__ void __launch_bounds__(kDecThreads)
 decode_kernel(__nv_bfloat16* __restrict__ hidden, int d, const float* __restrict__ Z, long long ldz,
               const int* __restrict__ panel_row, const int* __restrict__ row_slot,
@@ -472,97 +532,68 @@ decode_kernel(__nv_bfloat16* __restrict__ hidden, int d, const float* __restrict
   pdl_launch_dependents();
   __shared__ float s_coef[kDecList];
   __shared__ int s_feat[kDecList];
-  __shared__ float s_fnew[kMaxEdits];
-  __shared__ int s_eidx[kMaxEdits];
-  __shared__ int s_alive[kMaxEdits];
-  __shared__ float s_fold[kMaxEdits];
-  __shared__ int s_any, s_n;
-  const int p = blockIdx.x;
-  const int tid = threadIdx.x;
-  if (p >= rs->n_panel_rows) return;
-  const int t = panel_row[p];
-  if (t < 0) {
-    if (tid == 0) row_delta[p].slot = -1;             // padding row of a tile
-    return;
-  }
-  const int slot = row_slot[t];                       // the SAE app's slot (the row's own, or the last of its chain)
-  const AppEntry app = apps[slot];
-  const GroupEntry ge = groups[app.group];
-  const int n_edit = app.n_edit;
-  const int S = (int)ge.d_sae;
-  const float* z = Z + (size_t)p * ldz;
-  const int* K = ws_idx + (size_t)p * k_max;
-  const float* Kv = ws_val + (size_t)p * k_max;
-  const int nvec = d >> 3;
-
-  if (tid == 0) { s_any = 0; s_n = 0; }
-  if (tid < n_edit) {
-    s_eidx[tid] = edit_idx[slot * r_max + tid];
-    s_fold[tid] = 0.f;
-  }
-  __syncthreads();
-  if (ge.act == MIX_SAE_TOPK) {
-    // TopK: the value of a selected feature comes from the row's TopK list (the Z scratch is not
-    // written for TopK sets unless the row took the fallback selection); an unselected one is 0.
-    // The list is scanned element-parallel against the edit list.
-    for (int i = tid; i < ge.k; i += kDecThreads) {
-      const int id = K[i];
-      for (int e = 0; e < n_edit; ++e)
-        if (s_eidx[e] == id) s_fold[e] = fmaxf(Kv[i], 0.f);
-    }
-    __syncthreads();
-  }
-  // edits: f_j before and after; a later entry for the same feature overrides an earlier one
-  if (tid < n_edit) {
-    const int j = s_eidx[tid];
-    bool alive = true;
-    for (int e2 = tid + 1; e2 < n_edit; ++e2) alive = alive && (s_eidx[e2] != j);
-    float f;
-    if (ge.act == MIX_SAE_RELU) {
-      f = fmaxf(z[j], 0.f);
-    } else if (ge.act == MIX_SAE_JUMPRELU) {
-      const float zj = z[j];
-      f = zj > ge.theta[j] ? zj : 0.f;
-    } else {
-      f = s_fold[tid];
-    }
-    const float fnew = edit_mode[slot * r_max + tid] == MIX_EDIT_CLAMP ? edit_val[slot * r_max + tid] : 0.f;
-    s_alive[tid] = alive;
-    s_fnew[tid] = fnew;
-    if (app.add_error) {
-      const float delta = alive ? fnew - f : 0.f;
-      edit_coef[(size_t)p * r_max + tid] = delta;
-      if (delta != 0.f) s_any = 1;
-    }
-  }
-  __syncthreads();
-
-  if (app.add_error) {
-    // the row keeps the error term: decode_delta_kernel adds the deltas, eight rows at a time.
-    // No effective edit: the row is left alone and stays bit-exact.
-    if (tid == 0) {
-      RowDelta rd;
-      rd.slot = s_any ? slot : -1;
-      rd.n_edit = n_edit;
-      rd.W_dec = ge.W_dec;
-      row_delta[p] = rd;
-    }
-    return;
-  }
-  if (tid == 0) row_delta[p].slot = -1;
-  float acc[kDecU][8];
-  uint4* hrow = reinterpret_cast<uint4*>(hidden + (size_t)t * d);
+  __shared__ int s_we[kDecRows][kMaxEdits];
+  __shared__ float s_wf[kDecRows][kMaxEdits];
+  __shared__ int s_replace[kDecRows];                  // token row of a replace-mode row, else -1
+  __shared__ int s_n;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int p0 = blockIdx.x * kDecRows;
+  const int n_rows = rs->n_panel_rows;
+  if (p0 >= n_rows) return;
   {
+    const int p = p0 + warp;
+    const int t = p < n_rows ? panel_row[p] : -1;
+    int replace_t = -1;
+    if (t < 0) {
+      if (p < n_rows && lane == 0) row_delta[p].slot = -1;           // padding row of a tile
+    } else {
+      const int slot = row_slot[t];                    // the SAE app's slot (the row's own, or the last of its chain)
+      const AppEntry app = apps[slot];
+      if (!app.add_error) {
+        replace_t = t;
+        if (lane == 0) row_delta[p].slot = -1;
+      } else {
+        const GroupEntry ge = groups[app.group];
+        warp_edit_coefs(p, slot, app, ge, Z + (size_t)p * ldz, ws_idx + (size_t)p * k_max, ws_val + (size_t)p * k_max,
+                        edit_idx, edit_val, edit_mode, r_max, row_delta, edit_coef, s_we[warp], s_wf[warp], lane);
+      }
+    }
+    if (lane == 0) s_replace[warp] = replace_t;
+  }
+  __syncthreads();
+  const int nvec = d >> 3;
+  for (int r = 0; r < kDecRows; ++r) {                 // CTA-uniform
+    const int t = s_replace[r];
+    if (t < 0) continue;
+    const int p = p0 + r;
+    const int slot = row_slot[t];
+    const AppEntry app = apps[slot];
+    const GroupEntry ge = groups[app.group];
+    const int n_edit = app.n_edit;
+    const int S = (int)ge.d_sae;
+    const float* z = Z + (size_t)p * ldz;
+    const int* K = ws_idx + (size_t)p * k_max;
+    const float* Kv = ws_val + (size_t)p * k_max;
+    int* s_eidx = s_we[0];                             // the per-warp scratch is free again
+    if (tid == 0) s_n = 0;
+    if (tid < n_edit) s_eidx[tid] = edit_idx[slot * r_max + tid];
+    __syncthreads();
+    // edited features contribute f' (live entries only: a later entry for the same feature wins)
+    if (tid < n_edit) {
+      const int j = s_eidx[tid];
+      bool alive = true;
+      for (int e2 = tid + 1; e2 < n_edit; ++e2) alive = alive && (s_eidx[e2] != j);
+      const float fnew = edit_mode[slot * r_max + tid] == MIX_EDIT_CLAMP ? edit_val[slot * r_max + tid] : 0.f;
+      s_coef[tid] = alive ? fnew : 0.f;
+      s_feat[tid] = j;
+    }
+    float acc[kDecU][8];
+    uint4* hrow = reinterpret_cast<uint4*>(hidden + (size_t)t * d);
 #pragma unroll
     for (int u = 0; u < kDecU; ++u) {
       const int v = tid + u * kDecThreads;
 #pragma unroll
       for (int i = 0; i < 8; ++i) acc[u][i] = (ge.b_dec && v < nvec) ? ge.b_dec[v * 8 + i] : 0.f;
-    }
-    // edited features contribute f' (live entries only)
-    if (tid < n_edit) {
-      s_coef[tid] = s_alive[tid] ? s_fnew[tid] : 0.f;
-      s_feat[tid] = s_eidx[tid];
     }
     __syncthreads();
     accumulate_list(acc, s_coef, s_feat, n_edit, ge.W_dec, d, nvec);
@@ -603,17 +634,18 @@ decode_kernel(__nv_bfloat16* __restrict__ hidden, int d, const float* __restrict
         __syncthreads();
       }
     }
-  }
 #pragma unroll
-  for (int u = 0; u < kDecU; ++u) {
-    const int v = tid + u * kDecThreads;
-    if (v < nvec) {
-      uint4 q;
-      __nv_bfloat162* pp = reinterpret_cast<__nv_bfloat162*>(&q);
+    for (int u = 0; u < kDecU; ++u) {
+      const int v = tid + u * kDecThreads;
+      if (v < nvec) {
+        uint4 q;
+        __nv_bfloat162* pp = reinterpret_cast<__nv_bfloat162*>(&q);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) pp[i] = __floats2bfloat162_rn(acc[u][2 * i], acc[u][2 * i + 1]);
-      hrow[v] = q;
+        for (int i = 0; i < 4; ++i) pp[i] = __floats2bfloat162_rn(acc[u][2 * i], acc[u][2 * i + 1]);
+        hrow[v] = q;
+      }
     }
+    __syncthreads();                                   // the shared lists are reused by the next row
   }
 }
 
@@ -884,7 +916,7 @@ cudaError_t launch_edit_only(const Ctx* c, __nv_bfloat16* hidden, int T, cudaStr
 // the rows that keep the error term, only works out the coefficients of their edits; decode_delta_kernel
 // then adds those rows' deltas, eight rows per CTA.
 cudaError_t launch_decode(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s) {
-  return launch_pdl(kPdlTail, decode_kernel, dim3(c->panel_rows_cap), dim3(kDecThreads), 0, s, hidden, c->cfg.d_model, c->d_z, c->cfg.d_sae_max,
+  return launch_pdl(kPdlTail, decode_kernel, dim3((c->panel_rows_cap + kDecRows - 1) / kDecRows), dim3(kDecThreads), 0, s, hidden, c->cfg.d_model, c->d_z, c->cfg.d_sae_max,
                                                           c->d_panel_row, c->d_row_slot, c->d_route, c->d_apps,
                                                           c->d_groups, c->d_edit_idx, c->d_edit_val, c->d_edit_mode,
                                                           c->cfg.r_max, c->cfg.k_max, c->d_topk_idx, c->d_topk_val,
