@@ -108,7 +108,20 @@ enum {
                                          contraction) and the scale is applied to the fp32 accumulator.  A memory option:
                                          the widening costs more time than the halved stream saves.  The paper has no
                                          counterpart.  Not together with MIX_FLAG_ENCODE_SIMT, MIX_FLAG_SAE_EDIT_ONLY or
-                                         center_input */
+                                         center_input */,
+  MIX_FLAG_FP8_ACT = 1u << 6          /* only with MIX_FLAG_FP8_W_ENC: the encoder's INPUT is 8-bit too, so the encode is
+                                         an E4M3 x E4M3 tensor-core contraction (kind::f8f6f4) that streams half the
+                                         bytes and needs no widening.  Each SAE row of `hidden` is quantised when it is
+                                         packed: s = the smallest power of two with max|h_i| / s <= 448 (2^0 for a zero
+                                         row, never below 2^-100), code_i = E4M3 nearest to h_i / s, ties to the even
+                                         code; the encoder then sees s * e4m3(code_i) in place of h_i:
+                                           z_j = s * W_enc_scale[j] * sum_i e4m3(code_i) e4m3(W_enc[j, i]) + b_enc[j].
+                                         Everything after the pre-activations (selection, edits, decode, the error term
+                                         and the write-back) works on the unquantised bf16 row as before.  This changes
+                                         the pre-activations by up to the quantisation step of the row (2^-4 relative per
+                                         element): an accuracy / speed trade the caller opts into; the paper has no
+                                         counterpart.  Needs d_model to be a multiple of 128; rows with non-finite
+                                         entries are not supported */
 };
 
 typedef struct {

@@ -23,10 +23,12 @@ memory (each pre-activation is still one full-length dot product).
 Parity pins: every function here is pinned by tests/test_oracle_pins.py
 (closed forms, hand-worked values under tests/golden/, brute force, library
 routines, algebraic invariants), tests/test_oracle_chain.py (slot chains) and
-tests/test_oracle_fp8.py (8-bit encoder).  Nothing is "parity unpinned".
+tests/test_oracle_fp8.py (8-bit encoder) and tests/test_oracle_fp8_act.py (8-bit encoder
+input).  Nothing is "parity unpinned".
 """
 from __future__ import annotations
 
+import math
 from dataclasses import dataclass, field
 from typing import Dict, Iterable, List, Optional
 
@@ -148,6 +150,49 @@ def encoder_rows_f64(W_enc_bits: np.ndarray, w_scale: Optional[np.ndarray] = Non
     if w_scale is None:
         return bf16_to_f64(W_enc_bits)
     return e4m3_to_f64(W_enc_bits) * np.asarray(w_scale, dtype=np.float64)[:, None]
+
+
+E4M3_MAX = 448.0                                  # largest finite E4M3 magnitude (code 0x7E)
+ACT_SCALE_MIN_EXP = -100                          # the row scale of the 8-bit input is never below 2^-100
+_E4M3_GRID = _E4M3_VALUES[:127]                   # magnitudes of codes 0x00 .. 0x7E, ascending with the code
+
+
+def e4m3_quantize(x: np.ndarray) -> np.ndarray:
+    """Nearest E4M3 code of each entry of x (float64, |x| <= 448); a value half-way between two
+    neighbouring codes goes to the even code (round-to-nearest-even of the 3-bit mantissa)."""
+    x = np.asarray(x, dtype=np.float64)
+    a = np.abs(x)
+    if np.any(a > E4M3_MAX):
+        raise ValueError("e4m3_quantize takes magnitudes up to 448")
+    hi = np.searchsorted(_E4M3_GRID, a, side="left")          # first code with value >= a
+    hi = np.minimum(hi, 126)
+    lo = np.maximum(hi - 1, 0)
+    d_lo, d_hi = a - _E4M3_GRID[lo], _E4M3_GRID[hi] - a
+    take_hi = (d_hi < d_lo) | ((d_hi == d_lo) & (hi % 2 == 0))
+    code = np.where(take_hi, hi, lo).astype(np.uint8)
+    return np.where(np.signbit(x), code | 0x80, code).astype(np.uint8)
+
+
+def act_row_scale(x: np.ndarray) -> float:
+    """Scale of a row quantised to 8 bits: the smallest power of two s with max|x_i| / s <= 448,
+    never below 2^-100; 1 for a row of zeros."""
+    amax = float(np.max(np.abs(x))) if np.size(x) else 0.0
+    if amax == 0.0:
+        return 1.0
+    m, E = math.frexp(amax)                          # amax = m 2^E, 0.5 <= m < 1;  448 = 0.875 * 2^9
+    e = E - 9 if m <= 0.875 else E - 8
+    return math.ldexp(1.0, max(e, ACT_SCALE_MIN_EXP))
+
+
+def quantize_rows_e4m3(X: np.ndarray) -> np.ndarray:
+    """What the 8-bit encoder sees in place of each row x of X: s * e4m3(code_i), with s = act_row_scale(x)
+    and code_i the E4M3 code nearest to x_i / s."""
+    X = np.atleast_2d(np.asarray(X, dtype=np.float64))
+    out = np.empty_like(X)
+    for n in range(X.shape[0]):
+        s = act_row_scale(X[n])
+        out[n] = e4m3_to_f64(e4m3_quantize(X[n] / s)) * s
+    return out
 
 
 def sae_preact(X: np.ndarray, W_enc_bits: np.ndarray, b_enc: np.ndarray,
@@ -319,7 +364,8 @@ def apply_hook(w, rows: Optional[Iterable[int]] = None, keep_z: bool = False,
     for g, ts in sae_rows.items():
         sae = w.groups[g]
         X = bf16_to_f64(hidden_bits[np.asarray(ts)])
-        Z = sae_preact(X, sae.W_enc, sae.b_enc, sae.b_dec, sae.center_input, getattr(sae, "w_scale", None))
+        X_enc = quantize_rows_e4m3(X) if getattr(w, "fp8_act", False) else X      # 8-bit input: the encode alone sees it
+        Z = sae_preact(X_enc, sae.W_enc, sae.b_enc, sae.b_dec, sae.center_input, getattr(sae, "w_scale", None))
         for n, t in enumerate(ts):
             app = w.apps[int(w.token_slot[t])]
             Ko = None if topk_override is None else topk_override.get(t)
@@ -406,7 +452,8 @@ def apply_chain_hook(w, rows: Optional[Iterable[int]] = None,
                 y = project(h, bf16_to_f64(app.r), app.beta)
             elif app.kind == KIND_SAE:
                 sae = w.groups[app.group]
-                z = sae_preact(h[None, :], sae.W_enc, sae.b_enc, sae.b_dec, sae.center_input,
+                h_enc = quantize_rows_e4m3(h[None, :]) if getattr(w, "fp8_act", False) else h[None, :]
+                z = sae_preact(h_enc, sae.W_enc, sae.b_enc, sae.b_dec, sae.center_input,
                                getattr(sae, "w_scale", None))[0]
                 Ko = None if topk_override is None else topk_override.get(t)
                 y, K, n_act, _ = sae_row(h, z, sae, app, Ko)

@@ -1,6 +1,6 @@
 // Thin wrappers around the sm_100a instructions the tensor-core kernels of this library share:
 // mbarriers with bounded waits, TMA tile loads (never multicast), shared-memory and instruction
-// descriptors of tcgen05.mma (kind::f16, operands K-major with the 128-byte swizzle), commit,
+// descriptors of tcgen05.mma (kind::f16 and kind::f8f6f4, operands K-major with the 128-byte swizzle), commit,
 // fences, and the 32-lane x 32-column tensor-memory load.
 #pragma once
 
@@ -86,6 +86,20 @@ __device__ __forceinline__ void umma_f16(unsigned d_tmem, unsigned long long a, 
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// kind::f8f6f4 with both operands E4M3 (format code 0), D fp32, both K-major: one instruction takes
+// K = 32 elements = 32 bytes, so a 128-byte swizzled row holds four steps (bf16: 16 elements, same bytes).
+__host__ __device__ constexpr unsigned idesc_e4m3(int m, int n) {
+  return (1u << 4) | ((unsigned)(n >> 3) << 17) | ((unsigned)(m >> 4) << 24);
+}
+__device__ __forceinline__ void umma_e4m3(unsigned d_tmem, unsigned long long a, unsigned long long b, unsigned idesc,
+                                          unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
       : "memory");
 }

@@ -119,6 +119,7 @@ class Workload:
     d_sae_max: int = 0
     meta: dict = field(default_factory=dict)
     chains: Dict[int, int] = field(default_factory=dict)   # slot -> next slot applied to the same row
+    fp8_act: bool = False               # SAE rows reach the (8-bit) encoder quantised to E4M3 with a power-of-two row scale
 
 
 def bits(t):
@@ -161,4 +162,4 @@ def host(w: Workload, only_groups=None) -> Workload:
     }
     return Workload(w.name, w.d_model, w.T_max, w.T_live, bits(w.hidden), w.token_slot.copy(),
                     apps, groups, w.n_slots_max, w.n_groups_max, w.C_max, w.k_max, w.r_max,
-                    w.d_sae_max, dict(w.meta), dict(w.chains))
+                    w.d_sae_max, dict(w.meta), dict(w.chains), w.fp8_act)
