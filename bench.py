@@ -250,7 +250,8 @@ def extras_sae(name, w, peaks, mixlib, extra_flags=0, w_enc_bytes_per_el=2.0):
     enc_s = st["encode"] * 1e-3
     status = m.get_status()
     m.destroy()
-    layout = "8-bit E4M3 codes, tile-ordered copy" if extra_flags & 32 else (
+    layout = "8-bit E4M3 codes in blocks of 128, tile-ordered copy; 8-bit input" if extra_flags & 64 else (
+        "8-bit E4M3 codes, tile-ordered copy") if extra_flags & 32 else (
         "tile-contiguous copy" if SAE_FLAGS & 2 else "as registered")
     return {"workload": name, "w_enc_layout": layout,
             "t_call_ms_graph": min(times), "t_call_ms_graph_median_of_11": float(np.median(times)),
@@ -415,6 +416,20 @@ def run_workload(args):
         out = extras_sae("sae_small, 8-bit encoder (d=4096, d_sae=16384, 2 sets, T=256)",
                          W.make_sae_heavy("cuda", d_sae=16384, T=256, R=16, G=2, fp8=True), peaks, mixlib,
                          extra_flags=32, w_enc_bytes_per_el=1.0)
+    elif name == "sae_heavy_fp8a":  # config 2, 8-bit encoder AND 8-bit encoder input (E4M3 x E4M3 contraction)
+        out = extras_sae("sae_heavy (config 2), 8-bit encoder and input", W.make_sae_heavy("cuda", fp8=True, fp8_act=True),
+                         peaks, mixlib, extra_flags=32 | 64, w_enc_bytes_per_el=1.0)
+    elif name == "mixed_fp8a":
+        out = extras_sae("mixed (config 3), 8-bit encoder and input", W.make_mixed("cuda", fp8=True, fp8_act=True),
+                         peaks, mixlib, extra_flags=32 | 64, w_enc_bytes_per_el=1.0)
+    elif name == "sae_small_fp8a":  # profiling case for the 8-bit contraction
+        out = extras_sae("sae_small, 8-bit encoder and input (d=4096, d_sae=16384, 2 sets, T=256)",
+                         W.make_sae_heavy("cuda", d_sae=16384, T=256, R=16, G=2, fp8=True, fp8_act=True), peaks, mixlib,
+                         extra_flags=32 | 64, w_enc_bytes_per_el=1.0)
+    elif name == "mixed_small_fp8a":
+        out = extras_sae("mixed_small, 8-bit encoder and input (d=5120, d_sae=8192, T=4096)",
+                         W.make_mixed("cuda", T=4096, d_sae=8192, R=32, fp8=True, fp8_act=True), peaks, mixlib,
+                         extra_flags=32 | 64, w_enc_bytes_per_el=1.0)
     elif name == "sae_small":     # profiling case: weights (256 MiB) exceed L2, < 1 GiB on the device
         out = extras_sae("sae_small (d=4096, d_sae=16384, 2 sets, T=256)",
                          W.make_sae_heavy("cuda", d_sae=16384, T=256, R=16, G=2), peaks, mixlib)
@@ -740,7 +755,7 @@ def main():
     ap.add_argument("--no-retile", action="store_true",
                     help="SAE contexts stream W_enc as registered instead of a tile-contiguous copy (MIX_FLAG_RETILE_W_ENC)")
     ap.add_argument("--workload", default="decode",
-                    help="decode (the contract line) | sweep | sae_heavy | sae_heavy_fp8 | sae_small | sae_small_fp8 | mixed | mixed_fp8 | mixed_small | conditional | conditional_small | multiclass | multiclass_small | replay")
+                    help="decode (the contract line) | sweep | sae_heavy | sae_heavy_fp8 | sae_heavy_fp8a | sae_small | sae_small_fp8 | sae_small_fp8a | mixed | mixed_fp8 | mixed_fp8a | mixed_small | mixed_small_fp8a | conditional | conditional_small | multiclass | multiclass_small | replay")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     args = ap.parse_args()
     if args.no_retile:

@@ -27,6 +27,7 @@ MIX_FLAG_TEST_STALL_ENCODE = 4
 MIX_FLAG_SAE_EDIT_ONLY = 8
 MIX_FLAG_SLOT_CHAINS = 16
 MIX_FLAG_FP8_W_ENC = 32
+MIX_FLAG_FP8_ACT = 64
 
 EXPORTS = [
     "mix_create", "mix_destroy", "mix_last_error", "mix_register_sae_weights", "mix_unregister_sae_weights",

@@ -61,6 +61,18 @@ int make_tmap_u8(CUtensorMap* out, const void* base, unsigned long long rows) {
   return r == CUDA_SUCCESS ? MIX_OK : MIX_ERR_CUDA;
 }
 
+// E4M3 codes [rows, width] row-major for the 8-bit contraction: box = 128 bytes x box_rows rows; 128-byte swizzle.
+int make_tmap_e4m3(CUtensorMap* out, const void* base, unsigned long long rows, unsigned long long width, int box_rows) {
+  cuuint64_t dims[2] = {(cuuint64_t)width, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)width};
+  cuuint32_t box[2] = {(cuuint32_t)(2 * kTileK), (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = g_encode(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? MIX_OK : MIX_ERR_CUDA;
+}
+
 int make_tmap(CUtensorMap* out, const void* base, unsigned long long rows, int d, int box_rows) {
   cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)d * 2};
@@ -82,7 +94,7 @@ cudaError_t dev_alloc(T** p, size_t n) {
 void free_all(mix_ctx* c) {
   cudaFree(c->d_token_slot); cudaFree(c->d_n_live); cudaFree(c->d_apps); cudaFree(c->d_groups); cudaFree(c->d_gates); cudaFree(c->d_vec_arena); cudaFree(c->d_chain_next); cudaFree(c->d_row_slot);
   cudaFree(c->d_edit_idx); cudaFree(c->d_edit_val); cudaFree(c->d_edit_mode); cudaFree(c->d_status);
-  cudaFree(c->d_tmp_req); cudaFree(c->d_tmp_req_slot); cudaFree(c->d_panel); cudaFree(c->d_panel_row);
+  cudaFree(c->d_tmp_req); cudaFree(c->d_tmp_req_slot); cudaFree(c->d_panel); cudaFree(c->d_panel_row); cudaFree(c->d_act_scale);
   cudaFree(c->d_mtile_group); cudaFree(c->d_row_group); cudaFree(c->d_route); cudaFree(c->d_z); cudaFree(c->d_topk_idx);
   cudaFree(c->d_topk_val); cudaFree(c->d_tmap_w); cudaFree(c->d_tmap_probe); cudaFree(c->d_mc_dense); cudaFree(c->d_cand_val); cudaFree(c->d_cand_idx);
   cudaFree(c->d_row_delta); cudaFree(c->d_edit_coef);
@@ -200,6 +212,8 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
   }
   if ((cfg->flags & MIX_FLAG_SLOT_CHAINS) && (cfg->flags & MIX_FLAG_SAE_EDIT_ONLY)) return MIX_ERR_INVALID_ARG;
   if ((cfg->flags & MIX_FLAG_FP8_W_ENC) && (cfg->flags & (MIX_FLAG_ENCODE_SIMT | MIX_FLAG_SAE_EDIT_ONLY))) return MIX_ERR_INVALID_ARG;
+  if ((cfg->flags & MIX_FLAG_FP8_ACT) && !(cfg->flags & MIX_FLAG_FP8_W_ENC)) return MIX_ERR_INVALID_ARG;
+  if ((cfg->flags & MIX_FLAG_FP8_ACT) && cfg->d_model % (2 * kTileK)) return MIX_ERR_UNSUPPORTED;
   mix_ctx* c = static_cast<mix_ctx*>(calloc(1, sizeof(mix_ctx)));
   if (!c) return MIX_ERR_NO_MEMORY;
   c->cfg = *cfg;
@@ -235,6 +249,7 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
     const size_t P = c->panel_rows_cap;
     ok = ok && dev_alloc(&c->d_panel, P * cfg->d_model) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_panel_row, P) == cudaSuccess;
+    if (cfg->flags & MIX_FLAG_FP8_ACT) ok = ok && dev_alloc(&c->d_act_scale, P) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_mtile_group, P / kTileM) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_row_group, T) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_row_slot, T) == cudaSuccess;
@@ -271,9 +286,13 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
     if (e == cudaSuccess) e = cudaMemset(c->d_panel_row, 0xff, c->panel_rows_cap * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(c->d_mtile_group, 0xff, c->panel_rows_cap / kTileM * sizeof(int));
     if (e == cudaSuccess && !(cfg->flags & MIX_FLAG_ENCODE_SIMT)) {
-      if (load_encode_fn() != MIX_OK ||
-          make_tmap(&c->tmap_panel, c->d_panel, c->panel_rows_cap, cfg->d_model, kTileM) != MIX_OK)
+      if (load_encode_fn() != MIX_OK)
         e = cudaErrorUnknown;
+      else if ((cfg->flags & MIX_FLAG_FP8_ACT)
+                   ? make_tmap_e4m3(&c->tmap_panel, c->d_panel, c->panel_rows_cap, cfg->d_model, kTileM) != MIX_OK
+                   : make_tmap(&c->tmap_panel, c->d_panel, c->panel_rows_cap, cfg->d_model, kTileM) != MIX_OK)
+        e = cudaErrorUnknown;
+      if (e == cudaSuccess && c->d_act_scale) e = cudaMemset(c->d_act_scale, 0, c->panel_rows_cap * sizeof(float));
       if (e == cudaSuccess) e = encode_tc_prepare();
     }
   }
@@ -361,8 +380,12 @@ int mix_register_sae_weights(mix_ctx* c, int group, const mix_sae_weights* w, vo
         MIX_FAIL(c, MIX_ERR_NO_MEMORY, "cannot allocate the tile-ordered copy of the 8-bit W_enc");
       }
       unsigned char* tiled = reinterpret_cast<unsigned char*>(c->owned_w_tiled[group]);
-      MIX_CUDA(c, launch_retile_fp8(static_cast<const unsigned char*>(w->W_enc), tiled, w->d_sae, c->cfg.d_model, s));
-      if (make_tmap_u8(&tm, tiled, (unsigned long long)(n_el / kTileK)) != MIX_OK)
+      // (8-bit input as well: blocks of 128 codes per row, [S/256][d/128][256][128], 128-byte swizzled boxes)
+      const bool e4 = (c->cfg.flags & MIX_FLAG_FP8_ACT) != 0;
+      MIX_CUDA(c, launch_retile_fp8(static_cast<const unsigned char*>(w->W_enc), tiled, w->d_sae, c->cfg.d_model,
+                                    e4 ? 2 * kTileK : kTileK, s));
+      if ((e4 ? make_tmap_e4m3(&tm, tiled, (unsigned long long)(n_el / (2 * kTileK)), 2 * kTileK, kTileN)
+              : make_tmap_u8(&tm, tiled, (unsigned long long)(n_el / kTileK))) != MIX_OK)
         MIX_FAIL(c, MIX_ERR_CUDA, "cuTensorMapEncodeTiled failed for the 8-bit W_enc");
     } else if (c->cfg.flags & MIX_FLAG_RETILE_W_ENC) {
       // library-owned tile-contiguous copy: [S/256][d/64][256][64], seen by TMA as a 64-column matrix

@@ -117,7 +117,8 @@ struct Ctx {
 
   // SAE workspace
   int panel_rows_cap;       // P
-  __nv_bfloat16* d_panel;   // [P, d]
+  __nv_bfloat16* d_panel;   // [P, d]  (MIX_FLAG_FP8_ACT: the same memory holds E4M3 codes, uint8 [P, d])
+  float* d_act_scale;       // [P] row scales of the 8-bit panel (MIX_FLAG_FP8_ACT only)
   int* d_panel_row;         // [P] token index or -1
   int* d_mtile_group;       // [P / kTileM] group of each m-tile or -1
   int* d_row_group;         // [T_max] routing scratch: weight set of each token row or -1
@@ -213,7 +214,7 @@ cudaError_t launch_compose_map(const Ctx* c, int T_live, int n_req, cudaStream_t
 cudaError_t launch_fold_bias(const __nv_bfloat16* W_enc, const float* b_enc, const float* b_dec, float* b_eff,
                              long long d_sae, int d, cudaStream_t s);
 cudaError_t launch_retile(const __nv_bfloat16* W_enc, __nv_bfloat16* W_tiled, long long d_sae, int d, cudaStream_t s);
-cudaError_t launch_retile_fp8(const unsigned char* W_enc, unsigned char* W_tiled, long long d_sae, int d, cudaStream_t s);
+cudaError_t launch_retile_fp8(const unsigned char* W_enc, unsigned char* W_tiled, long long d_sae, int d, int kb_bytes, cudaStream_t s);
 cudaError_t encode_tc_prepare();   // opt in to the large dynamic shared memory size
 
 }  // namespace mix

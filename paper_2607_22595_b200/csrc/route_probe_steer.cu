@@ -2,6 +2,8 @@
 //
 // probe_steer_kernel is the bandwidth kernel of the hook: one warp per token row, 16-byte
 // loads, fp32 FMA, shuffle reductions.  A row whose slot is -1 costs one 4-byte load.
+#include <cuda_fp8.h>
+
 #include "mix_internal.h"
 #include "row_lookup.cuh"
 
@@ -829,6 +831,55 @@ pack_kernel(const __nv_bfloat16* __restrict__ hidden, const int* __restrict__ pa
   for (int i = lane; i < nvec; i += 32) dst[i] = __ldg(src + i);
 }
 
+// 8-bit encoder input: every routed row is quantised on its way into the panel.  s = the smallest
+// power of two with max|h_i| / s <= 448 (never below 2^-100; 1 for a row of zeros), code_i = E4M3
+// nearest to h_i / s (the division is exact, the conversion rounds to nearest even).  One warp per row:
+// a first pass for the largest magnitude, a second one (the row is in L1 by then) for the codes.
+__global__ void __launch_bounds__(256)
+pack_e4m3_kernel(const __nv_bfloat16* __restrict__ hidden, const int* __restrict__ panel_row,
+                 const RouteState* __restrict__ rs, unsigned char* __restrict__ panel, float* __restrict__ act_scale, int d) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int p = blockIdx.x * 8 + warp;
+  if (p >= rs->n_panel_rows) return;
+  const int t = panel_row[p];
+  uint2* dst = reinterpret_cast<uint2*>(panel + (size_t)p * d);
+  const int nvec = d >> 3;
+  if (t < 0) {   // padding rows of a tile
+    for (int i = lane; i < nvec; i += 32) dst[i] = make_uint2(0u, 0u);
+    if (lane == 0) act_scale[p] = 0.f;
+    return;
+  }
+  const uint4* src = reinterpret_cast<const uint4*>(hidden + (size_t)t * d);
+  unsigned m2 = 0u;                                     // two 15-bit magnitudes, compared as integers
+  for (int i = lane; i < nvec; i += 32) {
+    const uint4 q = __ldg(src + i);
+    m2 = __vmaxu2(m2, __vmaxu2(__vmaxu2(q.x & 0x7fff7fffu, q.y & 0x7fff7fffu), __vmaxu2(q.z & 0x7fff7fffu, q.w & 0x7fff7fffu)));
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m2 = __vmaxu2(m2, __shfl_xor_sync(0xffffffffu, m2, o));
+  const unsigned a = max(m2 & 0xffffu, m2 >> 16);       // bf16 bits of max|h_i|: (1 + frac / 128) * 2^(E - 127)
+  int e = 0;
+  if (a != 0u) {
+    const int E = (int)(a >> 7) - 127, frac = (int)(a & 0x7fu);
+    e = max(E - (frac <= 96 ? 8 : 7), -100);            // 448 = 1.75 * 2^8, and 1.75 = 1 + 96 / 128
+  }
+  const float inv = __uint_as_float((unsigned)(127 - e) << 23);
+  if (lane == 0) act_scale[p] = __uint_as_float((unsigned)(127 + e) << 23);
+  for (int i = lane; i < nvec; i += 32) {
+    const uint4 q = __ldg(src + i);
+    const unsigned w[4] = {q.x, q.y, q.z, q.w};
+    unsigned short c[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const float lo = __uint_as_float(w[u] << 16) * inv, hi = __uint_as_float(w[u] & 0xffff0000u) * inv;
+      c[u] = __nv_cvt_float2_to_fp8x2(make_float2(lo, hi), __NV_SATFINITE, __NV_E4M3);
+    }
+    dst[i] = make_uint2((unsigned)c[0] | ((unsigned)c[1] << 16), (unsigned)c[2] | ((unsigned)c[3] << 16));
+  }
+}
+
 // Router-logit steering: one thread per (row, expert).
 __global__ void __launch_bounds__(256)
 router_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
@@ -937,6 +988,9 @@ cudaError_t launch_route(const Ctx* c, int T, cudaStream_t s, unsigned long long
 
 cudaError_t launch_pack(const Ctx* c, const __nv_bfloat16* hidden, cudaStream_t s) {
   const int blocks = (c->panel_rows_cap + 7) / 8;
+  if (c->cfg.flags & MIX_FLAG_FP8_ACT)
+    return launch_pdl(kPdlPack, pack_e4m3_kernel, dim3(blocks), dim3(256), 0, s, hidden, c->d_panel_row, c->d_route,
+                      reinterpret_cast<unsigned char*>(c->d_panel), c->d_act_scale, c->cfg.d_model);
   return launch_pdl(kPdlPack, pack_kernel, dim3(blocks), dim3(256), 0, s, hidden, c->d_panel_row, c->d_route, c->d_panel, c->cfg.d_model);
 }
 

@@ -6,14 +6,16 @@
 // Warp roles:  warp 0 = TMA producer (panel tile 128x64 and W_enc tile 256x64 per k-block into
 // a 4-stage ring of 128-byte-swizzled shared memory), warp 1 = MMA issuer (tcgen05.mma
 // 128x256x16, fp32 accumulators in tensor memory, double buffered so the epilogue of one tile
-// overlaps the main loop of the next), warps 2..5 = epilogue (tcgen05.ld, + bias, then either
+// overlaps the main loop of the next), warps 2..9 = epilogue, two per tensor-memory lane quarter
+// with 128 columns of the tile each (tcgen05.ld, + bias, then either
 // the fp32 pre-activations to the Z scratch, or -- for TopK weight sets -- only the tile's 8
-// largest values per row plus its 9th, which the merge step turns into the exact TopK).
+// largest values per row plus its 9th, which the merge step turns into the exact TopK; the two
+// warps of a quarter merge their lists through shared memory).
 // No TMA multicast and no clusters.  Every wait is bounded: on expiry the CTA raises
 // MIX_STATUS_WAIT_TIMEOUT, lets its copies land, frees its tensor memory and returns.
 //
 // 8-bit encoder (kFp8): the W_enc tile arrives as 256 x 64 E4M3 codes (16 KiB, half the bytes);
-// warps 6..13 (two teams on alternate k-blocks) widen it to bf16 -- exactly: every E4M3 value is
+// eight more warps behind four epilogue warps (two teams on alternate k-blocks) widen it to bf16 -- exactly: every E4M3 value is
 // a bf16 value -- into the same 128-byte-swizzled layout TMA would have produced, and only then
 // is the k-block handed to the MMA warp; the per-feature scale is applied to the fp32
 // accumulator in the epilogue.  The copies land in a ring of 5 stages of 32 KiB (panel 16,
@@ -21,6 +23,13 @@
 // halves the encoder's footprint in HBM but is NOT faster than the bf16 form: the widening adds
 // 48 KiB of load/store traffic per k-block to a shared memory that the copies (32 KiB) and the
 // tensor core's operand reads (48 KiB) already keep busy, and the widening warps wait on it.
+//
+// 8-bit encoder AND 8-bit input (kEnc == 2): the panel holds E4M3 codes too (quantised per row with
+// a power-of-two scale by the pack step), so both operands go to the tensor core as they arrive:
+// tcgen05.mma kind::f8f6f4, 128 x 256 x 32 per instruction.  A k-block is 128 elements (the same
+// 128-byte swizzled rows, 16 + 32 KiB per stage, four instructions), so the kernel is the bf16
+// kernel with half as many k-blocks; the epilogue multiplies the accumulator by row scale x
+// feature scale.
 #include "mix_internal.h"
 #include "tc_common.cuh"
 
@@ -35,12 +44,19 @@ constexpr int kBBytes = kTileN * kTileK * 2;   // 32 KiB
 constexpr int kRawBytes = kTileN * kTileK;     // 16 KiB of E4M3 codes (8-bit encoder only)
 constexpr int kConvWarps = 4;                  // warps per widening team (8-bit encoder only)
 constexpr int kConvTeams = 2;                  // team g (warps 6 + 4g ..) widens every k-block with index = g mod 2, into slot g
-template <bool kFp8> struct TcCfg {
+// kEnc: 0 = bf16 encoder and input; 1 = 8-bit encoder widened to bf16; 2 = 8-bit encoder and 8-bit input
+template <int kEnc> struct TcCfg {
+  static constexpr bool kFp8 = kEnc == 1;
   static constexpr int kStages = kFp8 ? 5 : 4;
   static constexpr int kStageBytes = kABytes + (kFp8 ? kRawBytes : kBBytes);
   static constexpr int kRingBytes = kStages * kStageBytes + (kFp8 ? kBRing * kBBytes : 0);
-  static constexpr int kThreads = 192 + (kFp8 ? kConvTeams * kConvWarps * 32 : 0);
-  static constexpr int kSmemBytes = kRingBytes + 1024 /* alignment slack */ + 1024 /* TcShared */;
+  // epilogue warps: 4 (one per tensor-memory lane quarter, all 256 columns) or 8 (two per quarter, 128 columns
+  // each; the two top-9 lists of a row meet in shared memory).  One warp per scheduler runs the epilogue's
+  // dependent compare/select chains at a fraction of the issue rate; two interleave.
+  static constexpr int kEpiWarps = kFp8 ? 4 : 8;
+  static constexpr int kXchgBytes = kEpiWarps == 8 ? 2 * 4 * (kCandPerTile + 1) * 32 * 8 : 0;   // [acc][quarter][entry][lane] x (value, column)
+  static constexpr int kThreads = 64 + kEpiWarps * 32 + (kFp8 ? kConvTeams * kConvWarps * 32 : 0);
+  static constexpr int kSmemBytes = kRingBytes + 1024 /* alignment slack */ + 1024 /* TcShared */ + kXchgBytes;
   static_assert(kSmemBytes <= 227 * 1024, "shared memory per CTA");
 };
 constexpr int kTmemCols = 512;                 // two 128 x 256 fp32 accumulators
@@ -54,6 +70,7 @@ struct __align__(8) TcShared {
   unsigned long long b_empty[kBRing];     // 8-bit encoder: the MMAs that read the slot are done
   unsigned long long tmem_full[2];
   unsigned long long tmem_empty[2];
+  unsigned long long xchg_full[2][4];     // 8 epilogue warps: the upper-half warp's list of (accumulator, quarter) is in shared memory
   unsigned tmem_base;
   volatile int abort_flag;
   long long wait_cycles;      // cap of every bounded wait in this launch
@@ -69,6 +86,7 @@ __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, TcShare
 }
 
 constexpr unsigned kIdesc = idesc_f16(kTileM, kTileN);     // D fp32, A and B bf16, K-major, N = 256, M = 128
+constexpr unsigned kIdescE4 = idesc_e4m3(kTileM, kTileN);  // D fp32, A and B E4M3, K-major, N = 256, M = 128
 
 __device__ __forceinline__ void umma(unsigned d_tmem, unsigned long long a, unsigned long long b, unsigned accumulate) {
   umma_f16(d_tmem, a, b, kIdesc, accumulate);
@@ -140,24 +158,32 @@ __device__ __forceinline__ void e4m3x4_to_bf16x4(unsigned w, unsigned& lo, unsig
   hi = *reinterpret_cast<const unsigned*>(&r1);
 }
 
-template <bool kFp8>
-__global__ void __launch_bounds__(TcCfg<kFp8>::kThreads, 1)
+template <int kEnc>
+__global__ void __launch_bounds__(TcCfg<kEnc>::kThreads, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorMap* __restrict__ tmap_w,
                  const RouteState* __restrict__ rs_g, const GroupEntry* __restrict__ groups, int n_groups,
                  float* __restrict__ Z, long long ldz, int d, unsigned* __restrict__ status, int mode,
                  const int* __restrict__ mtile_flag, const int* __restrict__ n_flagged, float* __restrict__ cand_val,
-                 int* __restrict__ cand_idx, float* __restrict__ cand_ninth, int cand_tiles, int w_tiled, int test_stall) {
-  constexpr int kStages = TcCfg<kFp8>::kStages;
-  constexpr int kStageBytes = TcCfg<kFp8>::kStageBytes;
-  constexpr int kTcThreads = TcCfg<kFp8>::kThreads;
+                 int* __restrict__ cand_idx, float* __restrict__ cand_ninth, int cand_tiles, int w_tiled, int test_stall,
+                 const float* __restrict__ act_scale) {
+  constexpr bool kFp8 = kEnc == 1;                     // codes widened to bf16 in shared memory
+  constexpr bool kE4 = kEnc == 2;                      // E4M3 x E4M3 contraction
+  constexpr int kBlockK = kE4 ? 2 * kTileK : kTileK;   // elements per 128-byte row of either operand
+  constexpr int kStages = TcCfg<kEnc>::kStages;
+  constexpr int kStageBytes = TcCfg<kEnc>::kStageBytes;
+  constexpr int kTcThreads = TcCfg<kEnc>::kThreads;
+  constexpr int kEpiWarps = TcCfg<kEnc>::kEpiWarps;
+  constexpr int kEpiCols = kTileN / (kEpiWarps / 4);   // columns of a tile per epilogue warp
   pdl_wait();
   pdl_launch_dependents();
   if (mode == 1 && *n_flagged == 0) return;
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment: required by the 128-byte swizzle atoms
   unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  TcShared* sh = reinterpret_cast<TcShared*>(tiles + TcCfg<kFp8>::kRingBytes);
+  TcShared* sh = reinterpret_cast<TcShared*>(tiles + TcCfg<kEnc>::kRingBytes);
   unsigned char* bring = tiles + kStages * kStageBytes;      // 8-bit encoder: the ring of widened tiles
+  float* xchg_val = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(sh) + 1024);
+  int* xchg_idx = reinterpret_cast<int*>(xchg_val + 2 * 4 * (kCandPerTile + 1) * 32);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   for (int i = threadIdx.x; i < (int)(sizeof(RouteState) / sizeof(int)); i += kTcThreads)
@@ -173,7 +199,8 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&sh->tmem_full[a]), 1);
-      mbar_init(smem_u32(&sh->tmem_empty[a]), 4);
+      mbar_init(smem_u32(&sh->tmem_empty[a]), kEpiWarps);
+      for (int q = 0; q < 4; ++q) mbar_init(smem_u32(&sh->xchg_full[a][q]), 1);
     }
     sh->abort_flag = 0;
     sh->wait_cycles = test_stall ? kWaitCyclesTest : kWaitCycles;
@@ -194,7 +221,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
   __syncthreads();
   tc_fence_after();
   const unsigned tmem_base = sh->tmem_base;
-  const int num_kb = d / kTileK;
+  const int num_kb = d / kBlockK;
 
   if (warp == 0) {
     if (lane == 0) {
@@ -213,10 +240,10 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
           const unsigned bar = smem_u32(&sh->full[stage]);
           mbar_expect_tx(bar, kFp8 ? kABytes + kRawBytes : kABytes + kBBytes);
           const unsigned sa = smem_u32(tiles + stage * kStageBytes);
-          tma_load_2d(sa, &tmap_panel, kb * kTileK, t.m_tile_global * kTileM, bar);
+          tma_load_2d(sa, &tmap_panel, kb * kBlockK, t.m_tile_global * kTileM, bar);
           // W_enc tile: rows n_tile*256.. of the row-major matrix, or -- when the weights were re-laid
           // out at registration -- block (n_tile, kb) of the tile-contiguous copy [S/256][d/64][256][64]
-          if (kFp8)   // block (n_tile, kb) of the tile-ordered codes, into the stage's staging area
+          if (kFp8 || kE4)   // block (n_tile, kb) of the tile-ordered codes (kFp8: into the stage's staging area)
             tma_load_2d(sa + kABytes, tw, 0, (t.n_tile * num_kb + kb) * kTileN, bar);
           else if (w_tiled)
             tma_load_2d(sa + kABytes, tw, 0, (t.n_tile * num_kb + kb) * kTileN, bar);
@@ -245,8 +272,10 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
           const unsigned sb = kFp8 ? smem_u32(bring + bs * kBBytes) : sa + kABytes;
           const unsigned long long da = umma_desc(sa), db = umma_desc(sb);
 #pragma unroll
-          for (int k = 0; k < kTileK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per step
-            umma(d_tmem, da + 2ull * k, db + 2ull * k, (unsigned)((kb | k) != 0));
+          for (int k = 0; k < 4; ++k) {   // 16 bf16 or 32 codes = 32 bytes = 2 descriptor units per step
+            if (kE4) umma_e4m3(d_tmem, da + 2ull * k, db + 2ull * k, kIdescE4, (unsigned)((kb | k) != 0));
+            else umma(d_tmem, da + 2ull * k, db + 2ull * k, (unsigned)((kb | k) != 0));
+          }
           umma_commit(smem_u32(&sh->empty[stage]));
           if (kFp8) {
             umma_commit(smem_u32(&sh->b_empty[bs]));
@@ -261,14 +290,14 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
         if (acc == 0) acc_phase ^= 1u;
       }
     }
-  } else if (kFp8 && warp >= 6) {
+  } else if (kFp8 && warp >= 2 + kEpiWarps) {
     // widen the stage's 256 x 64 codes to bf16.  Thread c of 128 takes the 16-byte pieces c, c + 128, ...
     // (piece = row * 4 + quarter of the row): 16 codes in, two 16-byte chunks of the row's 128 bytes out,
     // stored where the 128-byte swizzle puts them (chunk index XOR row mod 8).
     // Two teams of four warps take alternate k-blocks (team = slot of the widened-tile ring), so one
     // team's stores and proxy fence overlap the other team's arithmetic.
-    const int team = (warp - 6) / kConvWarps;
-    const int ct = threadIdx.x - (6 + team * kConvWarps) * 32;
+    const int team = (warp - (2 + kEpiWarps)) / kConvWarps;
+    const int ct = threadIdx.x - (2 + kEpiWarps + team * kConvWarps) * 32;
     int stage = 0, bs = 0;
     unsigned phase = 0, bphase = 0;
     bool ok = true;
@@ -312,7 +341,10 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
     }
   } else {
     const int q = warp & 3;                  // tensor-memory lane quarter this warp may read
+    const int half = (warp - 2) >> 2;        // 8 epilogue warps: which 128 columns of the tile
+    const int c_lo = half * kEpiCols;
     unsigned acc = 0, acc_phase = 0;
+    unsigned xchg_phase = 0;                 // bit a: phase of the next hand-over through xchg_full[a][q] (TopK tiles only)
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
       const Tile t = decode_tile(sh->rs, groups, n_groups, tile);
       if (!tile_wanted(t, groups, mode, mtile_flag)) continue;
@@ -323,7 +355,9 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
       const bool valid = row_local < t.rows_valid;
       const size_t p = (size_t)t.m_tile_global * kTileM + row_local;
       const float* bias = groups[t.group].b_eff + (size_t)t.n_tile * kTileN;
-      const float* wsc = kFp8 ? groups[t.group].w_scale + (size_t)t.n_tile * kTileN : nullptr;
+      constexpr bool kScaled = kEnc != 0;      // the accumulator is in units of the codes
+      const float* wsc = kScaled ? groups[t.group].w_scale + (size_t)t.n_tile * kTileN : nullptr;
+      const float ars = kE4 ? (valid ? __ldg(act_scale + p) : 0.f) : 1.f;     // power of two: the products below are exact
       const unsigned taddr = tmem_base + ((unsigned)(q * 32) << 16) + acc * kTileN;
       if (mode == 0 && groups[t.group].act == MIX_SAE_TOPK) {
         float tv[kCandPerTile + 1];
@@ -334,21 +368,44 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
           ti[s] = 0;
         }
 #pragma unroll 1
-        for (int c = 0; c < kTileN; c += 32) {
+        for (int c = c_lo; c < c_lo + kEpiCols; c += 32) {
           float v[32];
           tmem_ld32(taddr + c, v);
 #pragma unroll
           for (int i = 0; i < 32; i += 4) {
             const float4 b4 = __ldg(reinterpret_cast<const float4*>(bias + c + i));
             float4 s4 = make_float4(1.f, 1.f, 1.f, 1.f);
-            if (kFp8) s4 = __ldg(reinterpret_cast<const float4*>(wsc + c + i));
-            top9_insert(tv, ti, kFp8 ? fmaf(v[i], s4.x, b4.x) : v[i] + b4.x, c + i);
-            top9_insert(tv, ti, kFp8 ? fmaf(v[i + 1], s4.y, b4.y) : v[i + 1] + b4.y, c + i + 1);
-            top9_insert(tv, ti, kFp8 ? fmaf(v[i + 2], s4.z, b4.z) : v[i + 2] + b4.z, c + i + 2);
-            top9_insert(tv, ti, kFp8 ? fmaf(v[i + 3], s4.w, b4.w) : v[i + 3] + b4.w, c + i + 3);
+            if (kScaled) s4 = __ldg(reinterpret_cast<const float4*>(wsc + c + i));
+            if (kE4) { s4.x *= ars; s4.y *= ars; s4.z *= ars; s4.w *= ars; }
+            top9_insert(tv, ti, kScaled ? fmaf(v[i], s4.x, b4.x) : v[i] + b4.x, c + i);
+            top9_insert(tv, ti, kScaled ? fmaf(v[i + 1], s4.y, b4.y) : v[i + 1] + b4.y, c + i + 1);
+            top9_insert(tv, ti, kScaled ? fmaf(v[i + 2], s4.z, b4.z) : v[i + 2] + b4.z, c + i + 2);
+            top9_insert(tv, ti, kScaled ? fmaf(v[i + 3], s4.w, b4.w) : v[i + 3] + b4.w, c + i + 3);
           }
         }
-        if (valid) {
+        bool writer = true;
+        if (kEpiWarps == 8) {
+          // the upper-half warp hands its list over; the lower-half warp merges it into its own (its columns
+          // come first, so equal values keep the lower column in front) and writes the tile's candidates
+          float* xv = xchg_val + (size_t)((acc * 4 + q) * (kCandPerTile + 1)) * 32 + lane;
+          int* xi = xchg_idx + (size_t)((acc * 4 + q) * (kCandPerTile + 1)) * 32 + lane;
+          if (half == 1) {
+#pragma unroll
+            for (int s = 0; s <= kCandPerTile; ++s) {
+              xv[s * 32] = tv[s];
+              xi[s * 32] = ti[s];
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->xchg_full[acc][q]));
+            writer = false;
+          } else {
+            if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&sh->xchg_full[acc][q]), (xchg_phase >> acc) & 1u, sh, status))) break;
+#pragma unroll
+            for (int s = 0; s <= kCandPerTile; ++s) top9_insert(tv, ti, xv[s * 32], xi[s * 32]);
+          }
+        }
+        xchg_phase ^= 1u << acc;
+        if (valid && writer) {
           const size_t slot = p * (size_t)cand_tiles + (size_t)t.n_tile;
           float4* cv = reinterpret_cast<float4*>(cand_val + slot * kCandPerTile);
           int4* ci = reinterpret_cast<int4*>(cand_idx + slot * kCandPerTile);
@@ -362,7 +419,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
       } else {
         float* out = Z + p * (size_t)ldz + (size_t)t.n_tile * kTileN;
 #pragma unroll 1
-        for (int c = 0; c < kTileN; c += 32) {
+        for (int c = c_lo; c < c_lo + kEpiCols; c += 32) {
           float v[32];
           tmem_ld32(taddr + c, v);
           if (valid) {
@@ -370,12 +427,13 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
             for (int i = 0; i < 32; i += 4) {
               const float4 b4 = __ldg(reinterpret_cast<const float4*>(bias + c + i));
               float4 s4 = make_float4(1.f, 1.f, 1.f, 1.f);
-              if (kFp8) s4 = __ldg(reinterpret_cast<const float4*>(wsc + c + i));
+              if (kScaled) s4 = __ldg(reinterpret_cast<const float4*>(wsc + c + i));
+              if (kE4) { s4.x *= ars; s4.y *= ars; s4.z *= ars; s4.w *= ars; }
               float4 o;
-              o.x = kFp8 ? fmaf(v[i], s4.x, b4.x) : v[i] + b4.x;
-              o.y = kFp8 ? fmaf(v[i + 1], s4.y, b4.y) : v[i + 1] + b4.y;
-              o.z = kFp8 ? fmaf(v[i + 2], s4.z, b4.z) : v[i + 2] + b4.z;
-              o.w = kFp8 ? fmaf(v[i + 3], s4.w, b4.w) : v[i + 3] + b4.w;
+              o.x = kScaled ? fmaf(v[i], s4.x, b4.x) : v[i] + b4.x;
+              o.y = kScaled ? fmaf(v[i + 1], s4.y, b4.y) : v[i + 1] + b4.y;
+              o.z = kScaled ? fmaf(v[i + 2], s4.z, b4.z) : v[i + 2] + b4.z;
+              o.w = kScaled ? fmaf(v[i + 3], s4.w, b4.w) : v[i + 3] + b4.w;
               *reinterpret_cast<float4*>(out + c + i) = o;
             }
           }
@@ -417,27 +475,30 @@ __global__ void retile_kernel(const uint4* __restrict__ src, uint4* __restrict__
   dst[i] = src[((n_tile * kTileN + r) * (long long)d + (long long)kb * kTileK) / 8 + piece];
 }
 
-// The same for 8-bit codes: [S, d] bytes -> [S/256][d/64][256][64] bytes, one thread per 16 bytes.
-__global__ void retile_fp8_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, long long d_sae, int d) {
+// The same for 8-bit codes: [S, d] bytes -> [S/256][d/kb_bytes][256][kb_bytes] bytes (kb_bytes = 64 for the
+// widening kernel, 128 for the 8-bit contraction), one thread per 16 bytes.
+__global__ void retile_fp8_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, long long d_sae, int d, int kb_bytes) {
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  const int num_kb = d / kTileK;
+  const int num_kb = d / kb_bytes;
+  const int ppr = kb_bytes / 16;                        // 16-byte pieces per block row
   const long long total = d_sae * (long long)d / 16;
   if (i >= total) return;
-  const int piece = (int)(i & 3);                       // 4 pieces per 64-byte row
-  const long long row_in_all = i >> 2;
+  const int piece = (int)(i % ppr);
+  const long long row_in_all = i / ppr;
   const int r = (int)(row_in_all % kTileN);
   const long long blk = row_in_all / kTileN;
   const int kb = (int)(blk % num_kb);
   const long long n_tile = blk / num_kb;
-  dst[i] = src[((n_tile * kTileN + r) * (long long)d + (long long)kb * kTileK) / 16 + piece];
+  dst[i] = src[((n_tile * kTileN + r) * (long long)d + (long long)kb * kb_bytes) / 16 + piece];
 }
 
 }  // namespace
 
-cudaError_t launch_retile_fp8(const unsigned char* W_enc, unsigned char* W_tiled, long long d_sae, int d, cudaStream_t s) {
+cudaError_t launch_retile_fp8(const unsigned char* W_enc, unsigned char* W_tiled, long long d_sae, int d, int kb_bytes,
+                              cudaStream_t s) {
   const long long total = d_sae * (long long)d / 16;
   retile_fp8_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(reinterpret_cast<const uint4*>(W_enc),
-                                                                    reinterpret_cast<uint4*>(W_tiled), d_sae, d);
+                                                                    reinterpret_cast<uint4*>(W_tiled), d_sae, d, kb_bytes);
   return cudaGetLastError();
 }
 
@@ -449,25 +510,28 @@ cudaError_t launch_retile(const __nv_bfloat16* W_enc, __nv_bfloat16* W_tiled, lo
 }
 
 cudaError_t encode_tc_prepare() {
-  cudaError_t e = cudaFuncSetAttribute(encode_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       TcCfg<false>::kSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(encode_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<0>::kSmemBytes);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(encode_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<true>::kSmemBytes);
+    e = cudaFuncSetAttribute(encode_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<1>::kSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(encode_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<2>::kSmemBytes);
   return e;
 }
 
-cudaError_t launch_encode_tc(const Ctx* c, int mode, cudaStream_t s) {
+template <int kEnc>
+static cudaError_t launch_encode_tc_as(const Ctx* c, int mode, cudaStream_t s) {
   const int w_tiled = (c->cfg.flags & MIX_FLAG_RETILE_W_ENC) ? 1 : 0;
   const int stall = (c->cfg.flags & MIX_FLAG_TEST_STALL_ENCODE) ? 1 : 0;
-  if (c->cfg.flags & MIX_FLAG_FP8_W_ENC)
-    return launch_pdl(mode == 0 ? kPdlEncode : kPdlTail, encode_tc_kernel<true>, dim3(c->n_sms), dim3(TcCfg<true>::kThreads), TcCfg<true>::kSmemBytes, s,
-                      c->tmap_panel, c->d_tmap_w, c->d_route, c->d_groups, c->cfg.n_groups_max, c->d_z, c->cfg.d_sae_max,
-                      c->cfg.d_model, c->d_status, mode, c->d_mtile_flag, c->d_n_flagged, c->d_cand_val, c->d_cand_idx,
-                      c->d_cand_ninth, c->cand_tiles, w_tiled, stall);
-  return launch_pdl(mode == 0 ? kPdlEncode : kPdlTail, encode_tc_kernel<false>, dim3(c->n_sms), dim3(TcCfg<false>::kThreads), TcCfg<false>::kSmemBytes, s,
-                    c->tmap_panel, c->d_tmap_w, c->d_route, c->d_groups, c->cfg.n_groups_max, c->d_z, c->cfg.d_sae_max,
-                    c->cfg.d_model, c->d_status, mode, c->d_mtile_flag, c->d_n_flagged, c->d_cand_val, c->d_cand_idx,
-                    c->d_cand_ninth, c->cand_tiles, w_tiled, stall);
+  return launch_pdl(mode == 0 ? kPdlEncode : kPdlTail, encode_tc_kernel<kEnc>, dim3(c->n_sms), dim3(TcCfg<kEnc>::kThreads),
+                    TcCfg<kEnc>::kSmemBytes, s, c->tmap_panel, c->d_tmap_w, c->d_route, c->d_groups, c->cfg.n_groups_max, c->d_z,
+                    c->cfg.d_sae_max, c->cfg.d_model, c->d_status, mode, c->d_mtile_flag, c->d_n_flagged, c->d_cand_val,
+                    c->d_cand_idx, c->d_cand_ninth, c->cand_tiles, w_tiled, stall, c->d_act_scale);
+}
+
+cudaError_t launch_encode_tc(const Ctx* c, int mode, cudaStream_t s) {
+  if (c->cfg.flags & MIX_FLAG_FP8_ACT) return launch_encode_tc_as<2>(c, mode, s);
+  if (c->cfg.flags & MIX_FLAG_FP8_W_ENC) return launch_encode_tc_as<1>(c, mode, s);
+  return launch_encode_tc_as<0>(c, mode, s);
 }
 
 }  // namespace mix

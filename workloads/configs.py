@@ -261,7 +261,7 @@ def make_decode(device="cpu", d=4096, T=256, n_probe=64, n_steer=32, seed=None):
 # config 2: SAE-heavy
 # --------------------------------------------------------------------------
 def make_sae_heavy(device="cpu", d=4096, d_sae=65536, k=64, T=512, R=32, G=4, n_edit=16,
-                   edit_hint: Optional[EditHint] = None, seed=None, fp8=False):
+                   edit_hint: Optional[EditHint] = None, seed=None, fp8=False, fp8_act=False):
     seed = BASE_SEED + 2000 if seed is None else seed
     g, rng = _gen(device, seed), np.random.default_rng(seed)
     hidden = _hidden(g, device, T, d)
@@ -281,7 +281,8 @@ def make_sae_heavy(device="cpu", d=4096, d_sae=65536, k=64, T=512, R=32, G=4, n_
         apps[r] = SaeApp(gi, idx, val, mode, add_error=True)
     return Workload("sae_heavy", d, T, T, hidden, token_slot, apps, groups, n_slots_max=R,
                     n_groups_max=G, C_max=1, k_max=k, r_max=n_edit, d_sae_max=d_sae,
-                    meta={"lengths": lengths, "token_req": token_req, "req_group": req_group, "seed": seed})
+                    meta={"lengths": lengths, "token_req": token_req, "req_group": req_group, "seed": seed},
+                    fp8_act=bool(fp8_act))
 
 
 # --------------------------------------------------------------------------
@@ -289,7 +290,7 @@ def make_sae_heavy(device="cpu", d=4096, d_sae=65536, k=64, T=512, R=32, G=4, n_
 # --------------------------------------------------------------------------
 def make_mixed(device="cpu", d=5120, T=8192, R=64, d_sae=32768, C=16, n_probe=8, n_steer=8, G=2,
                n_edit=16, cap=2048, mu=5.0, b_enc_mean=-0.1,
-               edit_hint: Optional[EditHint] = None, seed=None, fp8=False):
+               edit_hint: Optional[EditHint] = None, seed=None, fp8=False, fp8_act=False):
     seed = BASE_SEED + 3000 if seed is None else seed
     g, rng = _gen(device, seed), np.random.default_rng(seed)
     hidden = _hidden(g, device, T, d)
@@ -341,7 +342,7 @@ def make_mixed(device="cpu", d=5120, T=8192, R=64, d_sae=32768, C=16, n_probe=8,
                     n_slots_max=base_sae + max(n_a, 1), n_groups_max=G, C_max=C, k_max=0,
                     r_max=n_edit, d_sae_max=d_sae,
                     meta={"lengths": lengths, "token_req": token_req, "req_kind": req_kind,
-                          "req_group": req_group, "seed": seed})
+                          "req_group": req_group, "seed": seed}, fp8_act=bool(fp8_act))
 
 
 # --------------------------------------------------------------------------
