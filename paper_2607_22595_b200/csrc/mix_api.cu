@@ -94,7 +94,7 @@ cudaError_t dev_alloc(T** p, size_t n) {
 void free_all(mix_ctx* c) {
   cudaFree(c->d_token_slot); cudaFree(c->d_n_live); cudaFree(c->d_apps); cudaFree(c->d_groups); cudaFree(c->d_gates); cudaFree(c->d_vec_arena); cudaFree(c->d_chain_next); cudaFree(c->d_row_slot);
   cudaFree(c->d_edit_idx); cudaFree(c->d_edit_val); cudaFree(c->d_edit_mode); cudaFree(c->d_status);
-  cudaFree(c->d_tmp_req); cudaFree(c->d_tmp_req_slot); cudaFree(c->d_panel); cudaFree(c->d_panel_row); cudaFree(c->d_act_scale);
+  cudaFree(c->d_tmp_req); cudaFree(c->d_tmp_req_slot); cudaFree(c->d_panel); cudaFree(c->d_panel_row); cudaFree(c->d_act_scale); cudaFree(c->d_tau); cudaFree(c->d_tau_min);
   cudaFree(c->d_mtile_group); cudaFree(c->d_row_group); cudaFree(c->d_route); cudaFree(c->d_z); cudaFree(c->d_topk_idx);
   cudaFree(c->d_topk_val); cudaFree(c->d_tmap_w); cudaFree(c->d_tmap_probe); cudaFree(c->d_mc_dense); cudaFree(c->d_cand_val); cudaFree(c->d_cand_idx);
   cudaFree(c->d_row_delta); cudaFree(c->d_edit_coef);
@@ -269,6 +269,8 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
       ok = ok && dev_alloc(&c->d_row_flag, P) == cudaSuccess;
       ok = ok && dev_alloc(&c->d_mtile_flag, P / kTileM) == cudaSuccess;
       ok = ok && dev_alloc(&c->d_n_flagged, 1) == cudaSuccess;
+      ok = ok && dev_alloc(&c->d_tau, P * (size_t)kTauSlots) == cudaSuccess;
+      ok = ok && dev_alloc(&c->d_tau_min, P) == cudaSuccess;
     }
   }
   if (!ok) { cudaGetLastError(); free_all(c); free(c); return MIX_ERR_NO_MEMORY; }

@@ -21,6 +21,7 @@ constexpr int kTeamMaxRows = 2048;  // contexts up to this T_max run probes / st
 constexpr int kMaxClasses = 64;
 constexpr int kMaxK = 1024;
 constexpr int kMaxEdits = 64;
+constexpr int kTauSlots = 128;      // per packed row: slots of the running lower bound on the row's k-th largest pre-activation (k <= 128)
 constexpr int kCandPerTile = 8;     // TopK candidates the encode epilogue keeps per (row, feature tile)
 constexpr int kCandMax = 4096;      // candidates per row the merge step can sort in shared memory
 
@@ -132,6 +133,8 @@ struct Ctx {
   float* d_cand_val;        // [P, cand_tiles, kCandPerTile] per-tile TopK candidates (fused epilogue)
   int* d_cand_idx;          // same shape: feature ids
   float* d_cand_ninth;      // [P, cand_tiles] the (kCandPerTile+1)-th largest value of each tile
+  unsigned* d_tau_min;      // [P] the smallest of the row's first k slots, as last computed by a publisher
+  unsigned* d_tau;          // [P, kTauSlots] order-preserving keys of pre-activations seen so far in this call (0 = empty)
   int cand_tiles;           // d_sae_max / kTileN
   int* d_row_flag;          // [P] row needs the exact fallback selection
   int* d_mtile_flag;        // [P / kTileM] some row of the tile is flagged
@@ -184,6 +187,17 @@ cudaError_t launch_pdl(int which, void (*kernel)(KArgs...), dim3 grid, dim3 bloc
   cfg.attrs = at;
   cfg.numAttrs = (pdl_mask() & which) ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
+#ifdef __CUDACC__
+// Order-preserving 32-bit key of a float (larger value, larger key; -0 and +0 share one key; 0 is below every value).
+__device__ __forceinline__ unsigned f2key(float f) {
+  const unsigned b = __float_as_uint(f + 0.f);          // -0.0 -> +0.0: equal values, equal keys
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float key2f(unsigned k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 #endif
 

@@ -814,12 +814,16 @@ route_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_
 // Copy every routed row into the packed K-major panel (one warp per panel row).
 __global__ void __launch_bounds__(256)
 pack_kernel(const __nv_bfloat16* __restrict__ hidden, const int* __restrict__ panel_row,
-            const RouteState* __restrict__ rs, __nv_bfloat16* __restrict__ panel, int d) {
+            const RouteState* __restrict__ rs, __nv_bfloat16* __restrict__ panel, int d, unsigned* __restrict__ tau_slots, unsigned* __restrict__ tau_min) {
   pdl_wait();
   pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int p = blockIdx.x * 8 + warp;
   if (p >= rs->n_panel_rows) return;
+  if (tau_slots) {                                     // the encode's TopK bound starts empty
+    reinterpret_cast<uint4*>(tau_slots + (size_t)p * kTauSlots)[lane] = make_uint4(0u, 0u, 0u, 0u);
+    if (lane == 0) tau_min[p] = 0u;
+  }
   const int t = panel_row[p];
   uint4* dst = reinterpret_cast<uint4*>(panel + (size_t)p * d);
   const int nvec = d >> 3;
@@ -837,12 +841,17 @@ pack_kernel(const __nv_bfloat16* __restrict__ hidden, const int* __restrict__ pa
 // a first pass for the largest magnitude, a second one (the row is in L1 by then) for the codes.
 __global__ void __launch_bounds__(256)
 pack_e4m3_kernel(const __nv_bfloat16* __restrict__ hidden, const int* __restrict__ panel_row,
-                 const RouteState* __restrict__ rs, unsigned char* __restrict__ panel, float* __restrict__ act_scale, int d) {
+                 const RouteState* __restrict__ rs, unsigned char* __restrict__ panel, float* __restrict__ act_scale, int d,
+                 unsigned* __restrict__ tau_slots, unsigned* __restrict__ tau_min) {
   pdl_wait();
   pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int p = blockIdx.x * 8 + warp;
   if (p >= rs->n_panel_rows) return;
+  if (tau_slots) {                                     // the encode's TopK bound starts empty
+    reinterpret_cast<uint4*>(tau_slots + (size_t)p * kTauSlots)[lane] = make_uint4(0u, 0u, 0u, 0u);
+    if (lane == 0) tau_min[p] = 0u;
+  }
   const int t = panel_row[p];
   uint2* dst = reinterpret_cast<uint2*>(panel + (size_t)p * d);
   const int nvec = d >> 3;
@@ -990,8 +999,8 @@ cudaError_t launch_pack(const Ctx* c, const __nv_bfloat16* hidden, cudaStream_t 
   const int blocks = (c->panel_rows_cap + 7) / 8;
   if (c->cfg.flags & MIX_FLAG_FP8_ACT)
     return launch_pdl(kPdlPack, pack_e4m3_kernel, dim3(blocks), dim3(256), 0, s, hidden, c->d_panel_row, c->d_route,
-                      reinterpret_cast<unsigned char*>(c->d_panel), c->d_act_scale, c->cfg.d_model);
-  return launch_pdl(kPdlPack, pack_kernel, dim3(blocks), dim3(256), 0, s, hidden, c->d_panel_row, c->d_route, c->d_panel, c->cfg.d_model);
+                      reinterpret_cast<unsigned char*>(c->d_panel), c->d_act_scale, c->cfg.d_model, c->d_tau, c->d_tau_min);
+  return launch_pdl(kPdlPack, pack_kernel, dim3(blocks), dim3(256), 0, s, hidden, c->d_panel_row, c->d_route, c->d_panel, c->cfg.d_model, c->d_tau, c->d_tau_min);
 }
 
 cudaError_t launch_compose_map(const Ctx* c, int T_live, int n_req, cudaStream_t s) {

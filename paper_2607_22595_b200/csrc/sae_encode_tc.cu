@@ -43,9 +43,11 @@ constexpr int kABytes = kTileM * kTileK * 2;   // 16 KiB
 constexpr int kBBytes = kTileN * kTileK * 2;   // 32 KiB
 constexpr int kRawBytes = kTileN * kTileK;     // 16 KiB of E4M3 codes (8-bit encoder only)
 constexpr int kConvWarps = 4;                  // warps per widening team (8-bit encoder only)
+constexpr int kXchgEntries = kCandPerTile + 2;  // a top-9 list and the bound it was collected under
 constexpr int kConvTeams = 2;                  // team g (warps 6 + 4g ..) widens every k-block with index = g mod 2, into slot g
 // kEnc: 0 = bf16 encoder and input; 1 = 8-bit encoder widened to bf16; 2 = 8-bit encoder and 8-bit input
-template <int kEnc> struct TcCfg {
+template <int kEnc, int kEpi> struct TcCfg {
+  static_assert(kEpi == 4 || (kEpi == 8 && kEnc != 1), "epilogue warps");
   static constexpr bool kFp8 = kEnc == 1;
   static constexpr int kStages = kFp8 ? 5 : 4;
   static constexpr int kStageBytes = kABytes + (kFp8 ? kRawBytes : kBBytes);
@@ -53,8 +55,8 @@ template <int kEnc> struct TcCfg {
   // epilogue warps: 4 (one per tensor-memory lane quarter, all 256 columns) or 8 (two per quarter, 128 columns
   // each; the two top-9 lists of a row meet in shared memory).  One warp per scheduler runs the epilogue's
   // dependent compare/select chains at a fraction of the issue rate; two interleave.
-  static constexpr int kEpiWarps = kFp8 ? 4 : 8;
-  static constexpr int kXchgBytes = kEpiWarps == 8 ? 2 * 4 * (kCandPerTile + 1) * 32 * 8 : 0;   // [acc][quarter][entry][lane] x (value, column)
+  static constexpr int kEpiWarps = kEpi;
+  static constexpr int kXchgBytes = kEpiWarps == 8 ? 2 * 4 * kXchgEntries * 32 * 8 : 0;   // [acc][quarter][entry][lane] x (value, column)
   static constexpr int kThreads = 64 + kEpiWarps * 32 + (kFp8 ? kConvTeams * kConvWarps * 32 : 0);
   static constexpr int kSmemBytes = kRingBytes + 1024 /* alignment slack */ + 1024 /* TcShared */ + kXchgBytes;
   static_assert(kSmemBytes <= 227 * 1024, "shared memory per CTA");
@@ -96,13 +98,39 @@ struct Tile {
   int group, n_tile, m_tile_global, rows_valid;
 };
 
-__device__ __forceinline__ Tile decode_tile(const RouteState& rs, const GroupEntry* groups, int n_groups, int tile) {
+// Number of feature tiles per row tile if it is the same for every weight set that has rows (the usual
+// case: one SAE width per context), else 0.
+__device__ __forceinline__ int uniform_feature_tiles(const RouteState& rs, int n_groups) {
+  int nt = -1;
+  for (int g = 0; g < n_groups; ++g) {
+    const int mt = rs.group_mtile0[g + 1] - rs.group_mtile0[g];
+    if (mt == 0) continue;
+    const int nt_g = (rs.group_tile0[g + 1] - rs.group_tile0[g]) / mt;
+    if (nt >= 0 && nt_g != nt) return 0;
+    nt = nt_g;
+  }
+  return nt > 0 && nt * rs.n_mtiles == rs.total_tiles ? nt : 0;
+}
+
+// Linear tile id -> (weight set, feature tile, row tile).  With one SAE width the order is feature tile by
+// feature tile over ALL row tiles of the panel, so every row sees its first feature tiles finished early in
+// the launch (the TopK epilogue's running bound needs that); otherwise weight set by weight set.
+__device__ __forceinline__ Tile decode_tile(const RouteState& rs, const GroupEntry* groups, int n_groups, int tile,
+                                            int uniform_nt) {
+  Tile t;
   int g = 0;
+  if (uniform_nt > 0) {
+    t.n_tile = tile / rs.n_mtiles;
+    t.m_tile_global = tile - t.n_tile * rs.n_mtiles;
+    while (g + 1 < n_groups && t.m_tile_global >= rs.group_mtile0[g + 1]) ++g;
+    t.group = g;
+    t.rows_valid = min(kTileM, rs.group_count[g] - (t.m_tile_global - rs.group_mtile0[g]) * kTileM);
+    return t;
+  }
   while (g + 1 < n_groups && tile >= rs.group_tile0[g + 1]) ++g;
   const int local = tile - rs.group_tile0[g];
   const int count = rs.group_count[g];
   const int mt = (count + kTileM - 1) / kTileM;
-  Tile t;
   t.group = g;
   t.n_tile = local / mt;
   const int m_local = local - t.n_tile * mt;
@@ -121,22 +149,20 @@ __device__ __forceinline__ bool tile_wanted(const Tile& t, const GroupEntry* __r
 }
 
 // Insert (x, c) into the descending list tv[0..8] if it beats the 9th entry.  Equal values keep
-// the earlier (lower) column in front, which is the tie rule of the selection.
+// the earlier (lower) column in front, which is the tie rule of the selection: the new element goes
+// in front of the first entry it strictly beats, and everything from there on moves down one place.
 __device__ __forceinline__ void top9_insert(float (&tv)[kCandPerTile + 1], int (&ti)[kCandPerTile + 1], float x, int c) {
   if (!(x > tv[kCandPerTile])) return;
-  bool placed = false;
+  bool moving = false;
 #pragma unroll
-  for (int s = kCandPerTile; s >= 1; --s) {
-    const bool gt = x > tv[s - 1];
-    const float nv = gt ? tv[s - 1] : (placed ? tv[s] : x);
-    const int ni = gt ? ti[s - 1] : (placed ? ti[s] : c);
-    placed = placed || !gt;
-    tv[s] = nv;
-    ti[s] = ni;
-  }
-  if (!placed) {
-    tv[0] = x;
-    ti[0] = c;
+  for (int s = 0; s <= kCandPerTile; ++s) {
+    moving = moving || x > tv[s];
+    const float t = tv[s];
+    const int u = ti[s];
+    tv[s] = moving ? x : t;
+    ti[s] = moving ? c : u;
+    x = moving ? t : x;
+    c = moving ? u : c;
   }
 }
 
@@ -158,21 +184,21 @@ __device__ __forceinline__ void e4m3x4_to_bf16x4(unsigned w, unsigned& lo, unsig
   hi = *reinterpret_cast<const unsigned*>(&r1);
 }
 
-template <int kEnc>
-__global__ void __launch_bounds__(TcCfg<kEnc>::kThreads, 1)
+template <int kEnc, int kEpi>
+__global__ void __launch_bounds__(TcCfg<kEnc, kEpi>::kThreads, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorMap* __restrict__ tmap_w,
                  const RouteState* __restrict__ rs_g, const GroupEntry* __restrict__ groups, int n_groups,
                  float* __restrict__ Z, long long ldz, int d, unsigned* __restrict__ status, int mode,
                  const int* __restrict__ mtile_flag, const int* __restrict__ n_flagged, float* __restrict__ cand_val,
                  int* __restrict__ cand_idx, float* __restrict__ cand_ninth, int cand_tiles, int w_tiled, int test_stall,
-                 const float* __restrict__ act_scale) {
+                 const float* __restrict__ act_scale, unsigned* __restrict__ tau_slots, unsigned* __restrict__ tau_min) {
   constexpr bool kFp8 = kEnc == 1;                     // codes widened to bf16 in shared memory
   constexpr bool kE4 = kEnc == 2;                      // E4M3 x E4M3 contraction
   constexpr int kBlockK = kE4 ? 2 * kTileK : kTileK;   // elements per 128-byte row of either operand
-  constexpr int kStages = TcCfg<kEnc>::kStages;
-  constexpr int kStageBytes = TcCfg<kEnc>::kStageBytes;
-  constexpr int kTcThreads = TcCfg<kEnc>::kThreads;
-  constexpr int kEpiWarps = TcCfg<kEnc>::kEpiWarps;
+  constexpr int kStages = TcCfg<kEnc, kEpi>::kStages;
+  constexpr int kStageBytes = TcCfg<kEnc, kEpi>::kStageBytes;
+  constexpr int kTcThreads = TcCfg<kEnc, kEpi>::kThreads;
+  constexpr int kEpiWarps = TcCfg<kEnc, kEpi>::kEpiWarps;
   constexpr int kEpiCols = kTileN / (kEpiWarps / 4);   // columns of a tile per epilogue warp
   pdl_wait();
   pdl_launch_dependents();
@@ -180,10 +206,10 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment: required by the 128-byte swizzle atoms
   unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  TcShared* sh = reinterpret_cast<TcShared*>(tiles + TcCfg<kEnc>::kRingBytes);
+  TcShared* sh = reinterpret_cast<TcShared*>(tiles + TcCfg<kEnc, kEpi>::kRingBytes);
   unsigned char* bring = tiles + kStages * kStageBytes;      // 8-bit encoder: the ring of widened tiles
   float* xchg_val = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(sh) + 1024);
-  int* xchg_idx = reinterpret_cast<int*>(xchg_val + 2 * 4 * (kCandPerTile + 1) * 32);
+  int* xchg_idx = reinterpret_cast<int*>(xchg_val + 2 * 4 * kXchgEntries * 32);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   for (int i = threadIdx.x; i < (int)(sizeof(RouteState) / sizeof(int)); i += kTcThreads)
@@ -221,6 +247,8 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
   __syncthreads();
   tc_fence_after();
   const unsigned tmem_base = sh->tmem_base;
+  // (the interleaved order serves the TopK epilogue's running bound; without TopK rows the plain order is a little faster)
+  const int uniform_nt = sh->rs.n_topk_rows > 0 ? uniform_feature_tiles(sh->rs, n_groups) : 0;
   const int num_kb = d / kBlockK;
 
   if (warp == 0) {
@@ -229,7 +257,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
       unsigned phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const Tile t = decode_tile(sh->rs, groups, n_groups, tile);
+        const Tile t = decode_tile(sh->rs, groups, n_groups, tile, uniform_nt);
         if (!tile_wanted(t, groups, mode, mtile_flag)) continue;
         const CUtensorMap* tw = tmap_w + t.group;
         for (int kb = 0; kb < num_kb; ++kb) {
@@ -259,7 +287,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
       unsigned phase = 0, bphase = 0, acc = 0, acc_phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        if (mode != 0 && !tile_wanted(decode_tile(sh->rs, groups, n_groups, tile), groups, mode, mtile_flag)) continue;
+        if (mode != 0 && !tile_wanted(decode_tile(sh->rs, groups, n_groups, tile, uniform_nt), groups, mode, mtile_flag)) continue;
         if (!mbar_wait(smem_u32(&sh->tmem_empty[acc]), acc_phase ^ 1u, sh, status)) break;
         tc_fence_after();
         const unsigned d_tmem = tmem_base + acc * kTileN;
@@ -302,7 +330,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
     unsigned phase = 0, bphase = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-      if (mode != 0 && !tile_wanted(decode_tile(sh->rs, groups, n_groups, tile), groups, mode, mtile_flag)) continue;
+      if (mode != 0 && !tile_wanted(decode_tile(sh->rs, groups, n_groups, tile, uniform_nt), groups, mode, mtile_flag)) continue;
       for (int kb = 0; kb < num_kb; ++kb) {
         if (bs != team) {                      // the other team's k-block
           bs ^= 1;
@@ -346,25 +374,38 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
     unsigned acc = 0, acc_phase = 0;
     unsigned xchg_phase = 0;                 // bit a: phase of the next hand-over through xchg_full[a][q] (TopK tiles only)
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-      const Tile t = decode_tile(sh->rs, groups, n_groups, tile);
+      const Tile t = decode_tile(sh->rs, groups, n_groups, tile, uniform_nt);
       if (!tile_wanted(t, groups, mode, mtile_flag)) continue;
-      // warp-uniform decision: tcgen05.ld below needs the whole warp
-      if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&sh->tmem_full[acc]), acc_phase, sh, status))) break;
-      tc_fence_after();
       const int row_local = q * 32 + lane;
       const bool valid = row_local < t.rows_valid;
       const size_t p = (size_t)t.m_tile_global * kTileM + row_local;
+      // TopK tiles: a lower bound on the row's k-th largest pre-activation, from what every CTA has seen of the
+      // row so far in this call.  The row's k slots each hold the largest of a disjoint share of the values that
+      // tiles already finished published (distinct elements of the row), so once no slot is empty there are k
+      // elements >= the smallest slot: nothing below it can be in the TopK, and nearly everything is below it
+      // after the first tiles.  Read before the wait for the accumulator; a stale value is merely a lower bound.
+      const bool topk_tile = mode == 0 && groups[t.group].act == MIX_SAE_TOPK;
+      const int k_row = groups[t.group].k;
+      const bool use_tau = topk_tile && valid && tau_slots != nullptr && k_row <= kTauSlots;
+      unsigned tau_key = 0u;                   // 0: no bound yet
+      if (use_tau) tau_key = __ldcg(tau_min + p);     // the smallest slot, as of the last time a publisher looked
+      // warp-uniform decision: tcgen05.ld below needs the whole warp
+      if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&sh->tmem_full[acc]), acc_phase, sh, status))) break;
+      tc_fence_after();
       const float* bias = groups[t.group].b_eff + (size_t)t.n_tile * kTileN;
       constexpr bool kScaled = kEnc != 0;      // the accumulator is in units of the codes
       const float* wsc = kScaled ? groups[t.group].w_scale + (size_t)t.n_tile * kTileN : nullptr;
       const float ars = kE4 ? (valid ? __ldg(act_scale + p) : 0.f) : 1.f;     // power of two: the products below are exact
       const unsigned taddr = tmem_base + ((unsigned)(q * 32) << 16) + acc * kTileN;
-      if (mode == 0 && groups[t.group].act == MIX_SAE_TOPK) {
+      if (topk_tile) {
+        // the list starts out filled with a value just below the bound: whatever is not collected is at most that
+        const float tau = tau_key > 1u ? key2f(tau_key) : -INFINITY;
+        const float below_tau = tau_key > 1u ? key2f(tau_key - 1u) : -INFINITY;
         float tv[kCandPerTile + 1];
         int ti[kCandPerTile + 1];
 #pragma unroll
         for (int s = 0; s <= kCandPerTile; ++s) {
-          tv[s] = -INFINITY;
+          tv[s] = below_tau;
           ti[s] = 0;
         }
 #pragma unroll 1
@@ -377,24 +418,29 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
             float4 s4 = make_float4(1.f, 1.f, 1.f, 1.f);
             if (kScaled) s4 = __ldg(reinterpret_cast<const float4*>(wsc + c + i));
             if (kE4) { s4.x *= ars; s4.y *= ars; s4.z *= ars; s4.w *= ars; }
-            top9_insert(tv, ti, kScaled ? fmaf(v[i], s4.x, b4.x) : v[i] + b4.x, c + i);
-            top9_insert(tv, ti, kScaled ? fmaf(v[i + 1], s4.y, b4.y) : v[i + 1] + b4.y, c + i + 1);
-            top9_insert(tv, ti, kScaled ? fmaf(v[i + 2], s4.z, b4.z) : v[i + 2] + b4.z, c + i + 2);
-            top9_insert(tv, ti, kScaled ? fmaf(v[i + 3], s4.w, b4.w) : v[i + 3] + b4.w, c + i + 3);
+            v[i] = kScaled ? fmaf(v[i], s4.x, b4.x) : v[i] + b4.x;
+            v[i + 1] = kScaled ? fmaf(v[i + 1], s4.y, b4.y) : v[i + 1] + b4.y;
+            v[i + 2] = kScaled ? fmaf(v[i + 2], s4.z, b4.z) : v[i + 2] + b4.z;
+            v[i + 3] = kScaled ? fmaf(v[i + 3], s4.w, b4.w) : v[i + 3] + b4.w;
           }
+          // (the list's 9th value is at least below_tau, so the test inside top9_insert covers the bound too)
+#pragma unroll
+          for (int i = 0; i < 32; ++i) top9_insert(tv, ti, v[i], c + i);
         }
         bool writer = true;
+        unsigned tau_pub = tau_key;
         if (kEpiWarps == 8) {
           // the upper-half warp hands its list over; the lower-half warp merges it into its own (its columns
           // come first, so equal values keep the lower column in front) and writes the tile's candidates
-          float* xv = xchg_val + (size_t)((acc * 4 + q) * (kCandPerTile + 1)) * 32 + lane;
-          int* xi = xchg_idx + (size_t)((acc * 4 + q) * (kCandPerTile + 1)) * 32 + lane;
+          float* xv = xchg_val + (size_t)((acc * 4 + q) * kXchgEntries) * 32 + lane;
+          int* xi = xchg_idx + (size_t)((acc * 4 + q) * kXchgEntries) * 32 + lane;
           if (half == 1) {
 #pragma unroll
             for (int s = 0; s <= kCandPerTile; ++s) {
               xv[s * 32] = tv[s];
               xi[s * 32] = ti[s];
             }
+            xi[(kCandPerTile + 1) * 32] = (int)tau_key;
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh->xchg_full[acc][q]));
             writer = false;
@@ -402,6 +448,9 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
             if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&sh->xchg_full[acc][q]), (xchg_phase >> acc) & 1u, sh, status))) break;
 #pragma unroll
             for (int s = 0; s <= kCandPerTile; ++s) top9_insert(tv, ti, xv[s * 32], xi[s * 32]);
+            // the two warps may have read the bound at different times: what is at or above the larger one is a
+            // real element of the row (each warp's fillers lie below its own bound)
+            tau_pub = max(tau_key, (unsigned)xi[(kCandPerTile + 1) * 32]);
           }
         }
         xchg_phase ^= 1u << acc;
@@ -415,6 +464,35 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
           ci[0] = make_int4(j0 + ti[0], j0 + ti[1], j0 + ti[2], j0 + ti[3]);
           ci[1] = make_int4(j0 + ti[4], j0 + ti[5], j0 + ti[6], j0 + ti[7]);
           cand_ninth[slot] = tv[kCandPerTile];
+          if (use_tau) {
+            // this tile's r-th largest goes to slot (n_tile + r k/8) mod k: no two (tile, rank) pairs are the same
+            // element, eight consecutive feature tiles fill every slot, and every slot sees all ranks over time
+            unsigned* sp = tau_slots + p * kTauSlots;
+            bool raised_min = false;
+            const int rank_step = max(k_row / kCandPerTile, 1);
+            int slot_r = t.n_tile % k_row;
+#pragma unroll
+            for (int r = 0; r < kCandPerTile; ++r) {
+              const unsigned key = f2key(tv[r]);
+              if (key >= tau_pub && tv[r] > -INFINITY) {
+                const unsigned old = atomicMax(sp + slot_r, key);
+                raised_min = raised_min || old < key;      // the smallest slot may have moved up
+              }
+              slot_r += rank_step;
+              if (slot_r >= k_row) slot_r -= k_row;
+            }
+            if (raised_min) {
+              unsigned m = 0xffffffffu;
+              for (int j = 0; j < k_row; j += 4) {
+                const uint4 w = __ldcg(reinterpret_cast<const uint4*>(sp) + (j >> 2));
+                m = min(m, w.x);
+                if (j + 1 < k_row) m = min(m, w.y);
+                if (j + 2 < k_row) m = min(m, w.z);
+                if (j + 3 < k_row) m = min(m, w.w);
+              }
+              if (m > tau_pub) atomicMax(tau_min + p, m);
+            }
+          }
         }
       } else {
         float* out = Z + p * (size_t)ldz + (size_t)t.n_tile * kTileN;
@@ -509,29 +587,41 @@ cudaError_t launch_retile(const __nv_bfloat16* W_enc, __nv_bfloat16* W_tiled, lo
   return cudaGetLastError();
 }
 
+template <int kEnc, int kEpi>
+static cudaError_t encode_tc_prepare_as() {
+  return cudaFuncSetAttribute(encode_tc_kernel<kEnc, kEpi>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              TcCfg<kEnc, kEpi>::kSmemBytes);
+}
+
 cudaError_t encode_tc_prepare() {
-  cudaError_t e = cudaFuncSetAttribute(encode_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<0>::kSmemBytes);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(encode_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<1>::kSmemBytes);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(encode_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<2>::kSmemBytes);
+  cudaError_t e = encode_tc_prepare_as<0, 4>();
+  if (e == cudaSuccess) e = encode_tc_prepare_as<0, 8>();
+  if (e == cudaSuccess) e = encode_tc_prepare_as<1, 4>();
+  if (e == cudaSuccess) e = encode_tc_prepare_as<2, 4>();
+  if (e == cudaSuccess) e = encode_tc_prepare_as<2, 8>();
   return e;
 }
 
-template <int kEnc>
+template <int kEnc, int kEpi>
 static cudaError_t launch_encode_tc_as(const Ctx* c, int mode, cudaStream_t s) {
   const int w_tiled = (c->cfg.flags & MIX_FLAG_RETILE_W_ENC) ? 1 : 0;
   const int stall = (c->cfg.flags & MIX_FLAG_TEST_STALL_ENCODE) ? 1 : 0;
-  return launch_pdl(mode == 0 ? kPdlEncode : kPdlTail, encode_tc_kernel<kEnc>, dim3(c->n_sms), dim3(TcCfg<kEnc>::kThreads),
-                    TcCfg<kEnc>::kSmemBytes, s, c->tmap_panel, c->d_tmap_w, c->d_route, c->d_groups, c->cfg.n_groups_max, c->d_z,
-                    c->cfg.d_sae_max, c->cfg.d_model, c->d_status, mode, c->d_mtile_flag, c->d_n_flagged, c->d_cand_val,
-                    c->d_cand_idx, c->d_cand_ninth, c->cand_tiles, w_tiled, stall, c->d_act_scale);
+  return launch_pdl(mode == 0 ? kPdlEncode : kPdlTail, encode_tc_kernel<kEnc, kEpi>, dim3(c->n_sms),
+                    dim3(TcCfg<kEnc, kEpi>::kThreads), TcCfg<kEnc, kEpi>::kSmemBytes, s, c->tmap_panel, c->d_tmap_w, c->d_route,
+                    c->d_groups, c->cfg.n_groups_max, c->d_z, c->cfg.d_sae_max, c->cfg.d_model, c->d_status, mode,
+                    c->d_mtile_flag, c->d_n_flagged, c->d_cand_val, c->d_cand_idx, c->d_cand_ninth, c->cand_tiles, w_tiled,
+                    stall, c->d_act_scale, c->d_tau, c->d_tau_min);
 }
 
+// Eight epilogue warps pay off for the TopK epilogue (selection work per element); the plain store of the
+// pre-activations is a little faster with four.  Either form is correct for any mix of weight sets; the choice
+// is made from the sets registered when the call is enqueued (or captured).
 cudaError_t launch_encode_tc(const Ctx* c, int mode, cudaStream_t s) {
-  if (c->cfg.flags & MIX_FLAG_FP8_ACT) return launch_encode_tc_as<2>(c, mode, s);
-  if (c->cfg.flags & MIX_FLAG_FP8_W_ENC) return launch_encode_tc_as<1>(c, mode, s);
-  return launch_encode_tc_as<0>(c, mode, s);
+  bool topk = false;
+  for (int g = 0; g < c->cfg.n_groups_max; ++g) topk = topk || (c->h_groups[g].valid && c->h_groups[g].act == MIX_SAE_TOPK);
+  if (c->cfg.flags & MIX_FLAG_FP8_ACT) return topk ? launch_encode_tc_as<2, 8>(c, mode, s) : launch_encode_tc_as<2, 4>(c, mode, s);
+  if (c->cfg.flags & MIX_FLAG_FP8_W_ENC) return launch_encode_tc_as<1, 4>(c, mode, s);
+  return topk ? launch_encode_tc_as<0, 8>(c, mode, s) : launch_encode_tc_as<0, 4>(c, mode, s);
 }
 
 }  // namespace mix

@@ -80,14 +80,6 @@ constexpr int kCand = 1024;        // composites sorted in shared memory (>= k_m
 constexpr int kBins = 2048;
 static_assert(kCand >= kMaxK, "the sort buffer must hold a full TopK list");
 
-__device__ __forceinline__ unsigned f2key(float f) {
-  const unsigned b = __float_as_uint(f + 0.f);          // -0.0 -> +0.0: equal values, equal keys
-  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
-}
-__device__ __forceinline__ float key2f(unsigned k) {
-  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
-}
-
 // In-place bitonic sort of the first n entries of `a` (shared memory), descending.  Entries up
 // to the next power of two are overwritten with 0 (the smallest composite key).
 __device__ void bitonic_sort_desc(unsigned long long* a, int n) {
