@@ -265,10 +265,12 @@ def extras_sae(name, w, peaks, mixlib, extra_flags=0, w_enc_bytes_per_el=2.0):
             "token_rows_per_s": w.T_live / (min(times) * 1e-3), "status": status}
 
 
-def run_replay(peaks, mixlib, n_replays):
-    """Config 4: one captured graph at T_max = 2048, a fresh slot map and live count per replay."""
-    w = W.make_replay("cuda")
-    m = W.make_context(mixlib.Mix, w, flags=SAE_FLAGS)
+def run_replay(peaks, mixlib, n_replays, fp8a=False):
+    """Config 4: one captured graph at T_max = 2048, a fresh slot map and live count per replay.
+    fp8a: 8-bit encoder and 8-bit encoder input (half the W_enc bytes; the tensor bound is taken at twice the
+    measured bf16 rate, the nominal ratio of the two formats)."""
+    w = W.make_replay("cuda", fp8=fp8a, fp8_act=fp8a)
+    m = W.make_context(mixlib.Mix, w, flags=SAE_FLAGS | (32 | 64 if fp8a else 0))
     T = w.T_max
     h = w.hidden.clone()
     scores = torch.zeros((T, 1), dtype=torch.float32, device="cuda")
@@ -296,9 +298,10 @@ def run_replay(peaks, mixlib, n_replays):
             a = w.apps.get(int(token_slot[t]))
             if a is not None and a.kind == W.KIND_SAE:
                 counts[a.group] = counts.get(a.group, 0) + 1
-        wbytes = sum(2.0 * w.d_model * w.groups[gi].d_sae for gi in counts)
+        wbytes = sum((1.0 if fp8a else 2.0) * w.d_model * w.groups[gi].d_sae for gi in counts)
         flops = sum(2.0 * n * w.d_model * w.groups[gi].d_sae for gi, n in counts.items())
-        bound_ms = max(wbytes / (peaks["hbm_gbs"] * 1e9), flops / (peaks["bf16_tflops"] * 1e12)) * 1e3
+        bound_ms = max(wbytes / (peaks["hbm_gbs"] * 1e9),
+                       flops / ((2.0 if fp8a else 1.0) * peaks["bf16_tflops"] * 1e12)) * 1e3
         rec.append((n_live, sum(counts.values()), len(counts), ms, bound_ms))
         if r % 50 == 49 or r == n_replays - 1:
             bad_status |= m.get_status()
@@ -306,7 +309,7 @@ def run_replay(peaks, mixlib, n_replays):
     a = np.array(rec)
     live = a[a[:, 2] > 0]
     ratio = live[:, 4] / live[:, 3] if len(live) else np.array([0.0])
-    return {"workload": "replay (config 4)", "replays": n_replays, "status_or": bad_status,
+    return {"workload": "replay (config 4)" + (", 8-bit encoder and input" if fp8a else ""), "replays": n_replays, "status_or": bad_status,
             "t_call_ms": {"min": float(a[:, 3].min()), "p50": float(np.median(a[:, 3])), "p90": float(np.quantile(a[:, 3], 0.9)),
                           "max": float(a[:, 3].max())},
             "empty_replay_ms": float(a[a[:, 0] == 0][:, 3].min()) if (a[:, 0] == 0).any() else None,
@@ -448,6 +451,8 @@ def run_workload(args):
         out = extras_multiclass(peaks, mixlib, small=True)
     elif name == "replay":
         out = run_replay(peaks, mixlib, args.steps or 200)
+    elif name == "replay_fp8a":
+        out = run_replay(peaks, mixlib, args.steps or 200, fp8a=True)
     else:
         raise SystemExit("unknown workload %r" % name)
     print(json.dumps(out), flush=True)
@@ -755,7 +760,7 @@ def main():
     ap.add_argument("--no-retile", action="store_true",
                     help="SAE contexts stream W_enc as registered instead of a tile-contiguous copy (MIX_FLAG_RETILE_W_ENC)")
     ap.add_argument("--workload", default="decode",
-                    help="decode (the contract line) | sweep | sae_heavy | sae_heavy_fp8 | sae_heavy_fp8a | sae_small | sae_small_fp8 | sae_small_fp8a | mixed | mixed_fp8 | mixed_fp8a | mixed_small | mixed_small_fp8a | conditional | conditional_small | multiclass | multiclass_small | replay")
+                    help="decode (the contract line) | sweep | sae_heavy | sae_heavy_fp8 | sae_heavy_fp8a | sae_small | sae_small_fp8 | sae_small_fp8a | mixed | mixed_fp8 | mixed_fp8a | mixed_small | mixed_small_fp8a | conditional | conditional_small | replay_fp8a | multiclass | multiclass_small | replay")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     args = ap.parse_args()
     if args.no_retile:

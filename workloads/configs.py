@@ -349,7 +349,7 @@ def make_mixed(device="cpu", d=5120, T=8192, R=64, d_sae=32768, C=16, n_probe=8,
 # config 4: fixed-size graph replay
 # --------------------------------------------------------------------------
 def make_replay(device="cpu", d=8192, T_max=2048, d_sae=131072, k=128, G=8, n_probe=64, n_steer=16,
-                n_sae_slots=64, n_edit=16, seed=None):
+                n_sae_slots=64, n_edit=16, seed=None, fp8=False, fp8_act=False):
     """Apps for the replay config; the slot map of each replay comes from `replay_map`."""
     seed = BASE_SEED + 4000 if seed is None else seed
     g, rng = _gen(device, seed), np.random.default_rng(seed)
@@ -363,7 +363,7 @@ def make_replay(device="cpu", d=8192, T_max=2048, d_sae=131072, k=128, G=8, n_pr
     alphas = rng.uniform(1.0, 8.0, size=n_steer)
     for i in range(n_steer):
         apps[n_probe + i] = Steer(v=Vs[i].contiguous(), alpha=float(np.float32(alphas[i])))
-    groups = {gi: make_sae_weights(g, device, d, d_sae, SAE_TOPK, k=k) for gi in range(G)}
+    groups = {gi: make_sae_weights(g, device, d, d_sae, SAE_TOPK, k=k, fp8=fp8) for gi in range(G)}
     base = n_probe + n_steer
     for i in range(n_sae_slots):
         idx, val, mode = _edits(rng, d_sae, n_edit, None)
@@ -371,7 +371,7 @@ def make_replay(device="cpu", d=8192, T_max=2048, d_sae=131072, k=128, G=8, n_pr
     token_slot = np.full(T_max, -1, dtype=np.int32)
     w = Workload("replay", d, T_max, 0, hidden, token_slot, apps, groups,
                  n_slots_max=base + n_sae_slots, n_groups_max=G, C_max=1, k_max=k, r_max=n_edit,
-                 d_sae_max=d_sae, meta={"seed": seed})
+                 d_sae_max=d_sae, meta={"seed": seed}, fp8_act=bool(fp8_act))
     return w
 
 
