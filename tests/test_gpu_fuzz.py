@@ -15,10 +15,10 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
-def random_workload(seed):
+def random_workload(seed, fp8=False, fp8_act=False):
     rng = np.random.default_rng(seed)
     g = torch.Generator(device=DEV); g.manual_seed(int(seed))
-    d = int(rng.choice([64, 128, 192, 320, 512]))
+    d = int(rng.choice([128, 256, 384, 512] if fp8_act else [64, 128, 192, 320, 512]))   # 8-bit input: k-blocks of 128
     T = int(rng.choice([1, 7, 33, 128, 129, 300, 2100]))       # 2100 > 2048: the large-batch kernels
     n_groups = int(rng.integers(0, 4))
     hidden = (torch.randn((T, d), generator=g, device=DEV) * float(rng.choice([0.1, 1.0, 8.0]))).to(torch.bfloat16)
@@ -44,8 +44,8 @@ def random_workload(seed):
         act = int(rng.choice([W.SAE_RELU, W.SAE_JUMPRELU, W.SAE_TOPK]))
         k = int(rng.integers(1, min(48, S // 8))) if act == W.SAE_TOPK else 0
         sae = W.make_sae_weights(g, DEV, d, S, act, k=k, theta_range=(0.05, 0.3),
-                                 b_enc_mean=float(rng.choice([-0.1, -1.5])))
-        if rng.random() < 0.5:
+                                 b_enc_mean=float(rng.choice([-0.1, -1.5])), fp8=fp8)
+        if rng.random() < 0.5 and not fp8:                      # (an 8-bit encoder takes no input centring)
             sae.b_dec = torch.randn(d, generator=g, device=DEV) * 0.2
             sae.center_input = bool(rng.random() < 0.5)
         groups[gi] = sae
@@ -75,7 +75,8 @@ def random_workload(seed):
         for s in rng.choice(slots, size=min(2, len(slots)), replace=False):
             apps[int(s)].gate = W.Gate(sc, int(rng.integers(0, 2)), int(rng.integers(0, 2)), float(rng.normal()))
     return W.Workload("fuzz%d" % seed, d, T, T_live, hidden, token_slot, apps, groups, n_slots_max=n_slots,
-                      n_groups_max=n_groups, C_max=C_max, k_max=k_max, r_max=r_max, d_sae_max=d_sae_max)
+                      n_groups_max=n_groups, C_max=C_max, k_max=k_max, r_max=r_max, d_sae_max=d_sae_max,
+                      fp8_act=fp8_act)
 
 
 @pytest.mark.parametrize("seed", range(40))
@@ -89,4 +90,17 @@ def test_random_small_workload(seed):
     st = check_parity(W.host(w), out, expect_status=None, scale_with_output=True,
                       check_features=not (flags & mixlib.MIX_FLAG_SAE_EDIT_ONLY))
     assert out["status"] & ~mixlib.MIX_STATUS_TOPK_GENERAL == 0       # no bad slots, groups or timeouts
+    assert st["rows"] == w.T_max
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_small_workload_8bit(seed):
+    """The same sweep with the encoder as E4M3 codes, and (odd seeds) the encoder's input quantised as well."""
+    import paper_2607_22595_b200 as mixlib
+    fp8_act = bool(seed % 2)
+    w = random_workload(3000 + seed, fp8=True, fp8_act=fp8_act)
+    flags = mixlib.MIX_FLAG_FP8_W_ENC | (mixlib.MIX_FLAG_FP8_ACT if fp8_act else 0)
+    out = run_gpu(w, flags=flags, graph=bool(seed % 4 >= 2))
+    st = check_parity(W.host(w), out, expect_status=None, scale_with_output=True)
+    assert out["status"] & ~mixlib.MIX_STATUS_TOPK_GENERAL == 0
     assert st["rows"] == w.T_max
