@@ -153,3 +153,14 @@ def test_fp8_act_sae_heavy_full_size_sampled_rows():
     rows = [t for t in sample_rows(wh, per_kind=6) if w.apps[int(w.token_slot[t])].group == 1][:8]
     assert len(rows) >= 4
     check_parity(wh, out, rows=rows)
+
+
+def test_fp8_act_mixed_full_size_sampled_rows():
+    # config 3 in the launch configuration bench.py times (JumpReLU sets: the plain-store epilogue, four warps)
+    w = W.make_mixed(DEV, edit_hint=oracle_edit_hint, fp8=True, fp8_act=True)
+    out = run_gpu(w, flags=_flags() | _mixlib().MIX_FLAG_RETILE_W_ENC, graph=True)
+    wh = W.host(w)
+    unh = np.nonzero(wh.token_slot < 0)[0]
+    assert np.array_equal(out["hidden"][unh], wh.hidden[unh])        # every unhooked row is bit-identical
+    rows = sample_rows(wh, per_kind=12, seed=5)
+    check_parity(wh, out, rows=rows)
