@@ -744,6 +744,17 @@ def run_mix(args, rank, world, local_rank):
                             "per row instead); an algorithmic shortcut, not counted toward any tensor-pipe fraction",
                     "t_call_ms_graph": eo["t_call_ms_graph"], "stage_ms": eo["stage_ms"],
                     "token_rows_per_s": eo["token_rows_per_s"], "status": eo["status"]}
+                del wm
+                torch.cuda.empty_cache()
+                # opt-in 8-bit contraction (quantised encoder and encoder input: a different numerical method)
+                for key, mk, label in (("sae_heavy_8bit", W.make_sae_heavy, "sae_heavy (config 2), 8-bit encoder and input"),
+                                       ("mixed_8bit", W.make_mixed, "mixed (config 3), 8-bit encoder and input")):
+                    r8 = extras_sae(label, mk("cuda", fp8=True, fp8_act=True), peaks, mixlib, extra_flags=32 | 64,
+                                    w_enc_bytes_per_el=1.0)
+                    r8["note"] = ("MIX_FLAG_FP8_W_ENC | MIX_FLAG_FP8_ACT; tensor fractions here are against the bf16 peaks: "
+                                  "halve them for the 8-bit peak (nominal ratio 2)")
+                    ex[key] = r8
+                    torch.cuda.empty_cache()
             except Exception as e:                       # extras never break the contract line
                 ex["error"] = repr(e)
             line["extras"] = ex
