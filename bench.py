@@ -639,6 +639,22 @@ def run_mix(args, rank, world, local_rank):
     torch.cuda.synchronize()
     warm_us = e0.elapsed_time(e1) * 1e3 / (4 * min(R, 256))
 
+    # the cold protocol again with the hook kernels launched the ordinary way (no programmatic dependent launch):
+    # what a step costs behind a kernel that does not let its successor start early
+    old_mask = mixlib.set_pdl_mask(-1)
+    mixlib.set_pdl_mask(old_mask & ~8)
+    with torch.cuda.stream(stream):
+        g_plain = capture_steps(m, hiddens, scores, range(R), stream)
+        g_plain.replay()
+        e0.record(stream)
+        for _ in range(4):
+            g_plain.replay()
+        e1.record(stream)
+    torch.cuda.synchronize()
+    plain_us = e0.elapsed_time(e1) * 1e3 / (4 * R)
+    mixlib.set_pdl_mask(old_mask)
+    del g_plain
+
     # launch floor: the same graph with zero live rows (every CTA exits after one 4-byte load)
     m.set_slot_map(torch.from_numpy(w.token_slot.copy()).cuda(), 0)
     with torch.cuda.stream(stream):
@@ -709,6 +725,11 @@ def run_mix(args, rank, world, local_rank):
                    "us_added_per_decode_step": ms_per_step * 1e3, "us_added_per_decode_step_warm_l2": warm_us,
                    "us_added_per_decode_step_32_hooked_layers": 32 * ms_per_step * 1e3,
                    "us_per_step_zero_live_rows": floor_us,
+                   "us_added_per_decode_step_without_programmatic_launch": plain_us,
+                   "launch": "hook kernels are launched with programmatic stream serialization: in this back-to-back "
+                             "protocol a step's live-count / slot-map / app-table / vector lookups overlap the previous "
+                             "step's kernel, and `hidden` is read after the in-kernel wait; behind a kernel that does not "
+                             "signal early the step costs the 'without' figure",
                    "status_word": status},
         "clocks": clocks,
         "e2e": {"value": e2e_rows / e2e_s, "unit": UNIT, "h2d_bytes_per_step": T * d * 2 + 4 * T,

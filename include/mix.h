@@ -305,7 +305,13 @@ int mix_set_feature_out(mix_ctx* ctx, int* topk_idx, float* topk_val, int* n_act
    steering kernels run on a context-owned side stream forked from and joined back into `stream`
    by events, so they overlap the SAE chain; in a context for more than 2048 rows with multi-class
    probes and no SAE weight sets, the tensor-core probe kernel runs on that side stream beside the
-   streaming kernel) and returns; safe to capture.  Device-side
+   streaming kernel) and returns; safe to capture.  In a context without SAE weight sets and
+   T_max <= 2048 the kernel is launched with programmatic stream serialization (see
+   mix_set_pdl_mask): if the kernel in front of it in `stream` lets its successor start early, the
+   part that looks up the live count, slot map, app entry and single-vector weights -- tables the
+   library owns and only copies write -- overlaps that kernel; `hidden`, gate scores and
+   multi-class probe weights are read only after the predecessor has completed and flushed, and the
+   grid does not end before it.  Behind any other kernel nothing changes.  Device-side
    problems (bad slot ids, ...) are reported through the status word, never by faulting.
    Errors: INVALID_ARG (NULL hidden, misaligned), OUT_OF_RANGE (T), CUDA (launch failure). */
 int mix_apply(mix_ctx* ctx, void* hidden, int T, float* scores_out, void* stream);
@@ -364,6 +370,16 @@ int mix_set_stage_events(mix_ctx* ctx, void* const* events);
    Synchronises `stream`; not capturable; allocates and frees 8 bytes of device memory.
    Errors: INVALID_ARG (NULL outputs, iters < 1), CUDA (API failure or the two sums differ). */
 int mix_bench_param_update(mix_ctx* ctx, int iters, float* us_table, float* us_node, void* stream);
+
+/* Which launches of the library use programmatic dependent launch (a kernel's CTAs may become resident,
+   and run the part of the kernel that reads only library-owned tables, while the kernel in front of
+   it in the stream is still running; everything the predecessor may have written is read after an
+   in-kernel wait).  Bits: 1 the row-packing kernel, 2 the full SAE encode pass, 4 the kernels
+   after it, 8 the one-CTA-per-row probe / steering kernel of a context that has no SAE weight sets
+   (T_max <= 2048).  Default 1 | 4 | 8, or the value of MIX_PDL_MASK in the environment when the
+   library first launches.  Process-wide; affects launches (and captures) made afterwards; meant
+   for A/B measurement.  Returns the previous mask.  mask < 0 only queries. */
+int mix_set_pdl_mask(int mask);
 
 /* Test / profiling taps into the SAE workspace after a mix_apply (device pointers owned by
    the context; valid until mix_destroy):  panel_rows int32 [n_panel_rows] gives the token

@@ -34,7 +34,7 @@ EXPORTS = [
     "mix_register_app", "mix_unregister_app", "mix_set_gate", "mix_set_chain", "mix_update_steer_alpha", "mix_update_sae_edits",
     "mix_set_slot_map", "mix_set_request_map", "mix_set_feature_out", "mix_apply", "mix_apply_conditional", "mix_apply_router", "mix_get_status",
     "mix_launches_per_apply", "mix_set_stage_events", "mix_debug_workspace", "mix_sae_apply_static",
-    "mix_bench_param_update",
+    "mix_bench_param_update", "mix_set_pdl_mask",
 ]
 
 
@@ -107,6 +107,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.mix_get_status.argtypes = [vp, C.POINTER(C.c_uint), vp]
     lib.mix_launches_per_apply.argtypes = [vp]
     lib.mix_set_stage_events.argtypes = [vp, C.POINTER(vp)]
+    lib.mix_set_pdl_mask.argtypes = [ci]
     lib.mix_bench_param_update.argtypes = [vp, ci, C.POINTER(C.c_float), C.POINTER(C.c_float), vp]
     lib.mix_sae_apply_static.argtypes = [vp, ci, ci, C.POINTER(MixSaeWeights), C.POINTER(MixSaeApp), vp, vp, vp,
                                          C.c_char_p, ci]
@@ -117,6 +118,11 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     if path == _build.LIB_PATH:
         _lib = lib
     return lib
+
+
+def set_pdl_mask(mask: int) -> int:
+    """Which launches use programmatic dependent launch (see mix_set_pdl_mask); returns the previous mask."""
+    return int(load_library().mix_set_pdl_mask(int(mask)))
 
 
 def _ptr(t) -> Optional[int]:

@@ -187,14 +187,21 @@ int upload_chain(mix_ctx* c, int slot, cudaStream_t s) {
 }  // namespace
 
 namespace mix {
+static int g_pdl_mask = -1;        // -1: not yet read from the environment
 int pdl_mask() {
   // default: not the full encode pass -- measured, its early-resident CTAs cost config 3 about 7 us
-  static const int mask = getenv("MIX_PDL_MASK") ? atoi(getenv("MIX_PDL_MASK")) : (kPdlPack | kPdlTail);
-  return mask;
+  if (g_pdl_mask < 0) g_pdl_mask = getenv("MIX_PDL_MASK") ? (atoi(getenv("MIX_PDL_MASK")) & 15) : (kPdlPack | kPdlTail | kPdlHook);
+  return g_pdl_mask;
 }
 }  // namespace mix
 
 extern "C" {
+
+int mix_set_pdl_mask(int mask) {
+  const int old = mix::pdl_mask();
+  if (mask >= 0) mix::g_pdl_mask = mask & 15;
+  return old;
+}
 
 int mix_create(mix_ctx** out, const mix_config* cfg) {
   if (!out || !cfg) return MIX_ERR_INVALID_ARG;
@@ -628,6 +635,7 @@ int mix_set_request_map(mix_ctx* c, const int* token_req, int T_live, const int*
     MIX_CUDA(c, cudaMemcpyAsync(c->d_tmp_req, token_req, (size_t)T_live * sizeof(int), kind, s));
     if (n_req > 0) MIX_CUDA(c, cudaMemcpyAsync(c->d_tmp_req_slot, req_slot, (size_t)n_req * sizeof(int), kind, s));
     MIX_CUDA(c, launch_compose_map(c, T_live, n_req, s));
+    c->map_from_kernel = 1;
   }
   MIX_CUDA(c, cudaMemcpyAsync(c->d_n_live, &T_live, sizeof(int), cudaMemcpyHostToDevice, s));
   return MIX_OK;
@@ -750,7 +758,10 @@ int apply_impl(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream,
       MIX_CUDA(c, cudaEventRecord(c->ev_join, c->side_stream));
     }
   }
-  MIX_CUDA(c, launch_probe_steer(c, h, T, scores_out, ps));
+  // (programmatic launch only where this kernel directly follows the caller's work in the caller's stream)
+  const bool hook_pdl = !fork && !tc && !c->stage_events_on && !c->map_from_kernel;
+  c->map_from_kernel = 0;
+  MIX_CUDA(c, launch_probe_steer(c, h, T, scores_out, ps, hook_pdl));
   MIX_CUDA(c, tap());
   if (has_multiclass_stage(c)) {
     MIX_CUDA(c, launch_probe_multiclass(c, h, T, scores_out, ps));

@@ -150,6 +150,8 @@ struct Ctx {
   cudaEvent_t ev_fork, ev_join;
 
   // profiling taps
+  int map_from_kernel;      // the slot map was last written by compose_map_kernel, not by a copy: the next hook kernel
+                            // must not read it ahead of its predecessor
   int stage_events_on;
   cudaEvent_t stage_events[16];
 
@@ -170,8 +172,9 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // Which launches use programmatic dependent launch: bit 0 pack, bit 1 the full encode pass, bit 2 everything after
-// it (merge ... decode_delta).  MIX_PDL_MASK in the environment overrides the default (A/B timing); read once.
-enum { kPdlPack = 1, kPdlEncode = 2, kPdlTail = 4 };
+// it (merge ... decode_delta), bit 3 the one-CTA-per-row probe / steering kernel of a context without weight sets.
+// MIX_PDL_MASK in the environment overrides the default (A/B timing); read once.
+enum { kPdlPack = 1, kPdlEncode = 2, kPdlTail = 4, kPdlHook = 8 };
 int pdl_mask();
 
 template <typename... KArgs, typename... Args>
@@ -202,7 +205,7 @@ __device__ __forceinline__ float key2f(unsigned k) {
 #endif
 
 // kernel launchers (each returns the CUDA error of the launch)
-cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s);
+cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s, bool allow_pdl);
 // Multi-class probes of large batches have two kernels; both are launched and exactly one does the work, chosen
 // on the device (mc_decide_kernel samples the slot map, mc_batch_is_dense in row_lookup.cuh, and leaves the
 // answer in d_mc_dense): probe_tc (tcgen05, streams whole 128-row tiles: batches

@@ -377,26 +377,43 @@ probe_steer_team_kernel(const int* __restrict__ token_slot, const int* __restric
   constexpr int NT = NW * 32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t = blockIdx.x;                      // < T_max: the slot map has an entry for every row
+  // Programmatic dependent launch (when the launch asked for it; otherwise the two instructions do nothing):
+  // everything up to pdl_wait() reads only tables the LIBRARY owns and that only copies write -- live count,
+  // slot map, app entry, vector arena -- so it may run while the kernel in front of this one in the stream (the
+  // layer that produces `hidden`, or the previous hook) is still running.  Memory the caller owns (`hidden`,
+  // multi-class probe weights, gate scores) is read after the wait only, and every thread waits before it
+  // leaves, so that this grid cannot end -- and release ITS successor -- before its predecessor has.
+  pdl_launch_dependents();
   const int n_live = __ldg(n_live_p);            // both loads issue together: one round trip, not two
   const int slot = __ldg(token_slot + t);
-  if (t >= min(T, n_live) || slot == -1) return;
+  if (t >= min(T, n_live) || slot == -1) {
+    pdl_wait();
+    return;
+  }
   const int nvec = d >> 3;
   uint4* hrow = reinterpret_cast<uint4*>(hidden + (size_t)t * d);
   // Single-vector weights (steering, projection, one-class probe) were copied at registration
   // into row `slot` of the context's vector arena, so their address follows from the slot id
   // alone: the row AND its vector are requested together, before the app entry is known.
   uint4 hq[kTeamVec], vq[kTeamVec];
-  if (slot >= 0 && slot < n_slots) {
+  const bool slot_ok = slot >= 0 && slot < n_slots;
+  if (slot_ok) {
 #pragma unroll
     for (int u = 0; u < kTeamVec; ++u) {
       const int v = threadIdx.x + u * NT;
-      if (v < nvec) {
-        hq[u] = __ldcs(hrow + v);
-        vq[u] = __ldg(vec_arena + (size_t)slot * nvec + v);
-      }
+      if (v < nvec) vq[u] = __ldg(vec_arena + (size_t)slot * nvec + v);
     }
   }
-  const RowApp a = lookup(slot, t, apps, gates, n_slots, status, threadIdx.x == 0);
+  RowApp a = lookup(slot, t, apps, gates, n_slots, status, threadIdx.x == 0, /*eval_gate=*/false);
+  pdl_wait();
+  if (slot_ok) {
+#pragma unroll
+    for (int u = 0; u < kTeamVec; ++u) {
+      const int v = threadIdx.x + u * NT;
+      if (v < nvec) hq[u] = __ldcs(hrow + v);
+    }
+  }
+  if (a.gated && a.kind != 0 && !gate_open(gates, slot, t)) return;       // gate closed: the row passes through
   if (a.kind == MIX_STEER) {
     if (a.alpha == 0.f) return;                  // identity; the row stays bit-exact
 #pragma unroll
@@ -528,8 +545,13 @@ probe_steer_chain_kernel(const int* __restrict__ token_slot, const int* __restri
   constexpr int NT = kChainWarps * 32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t = blockIdx.x;                      // < T_max: the slot map has an entry for every row
+  // programmatic dependent launch, as in probe_steer_team_kernel: the live count and the slot id (library-owned,
+  // written only by copies) may be read while the predecessor still runs; everything else comes after the wait,
+  // and every thread waits before it leaves
+  pdl_launch_dependents();
   const int n_live = __ldg(n_live_p);
   int slot = __ldg(token_slot + t);
+  pdl_wait();
   if (t >= min(T, n_live) || slot == -1) return;
   const int nvec = d >> 3;
   uint4* hrow = reinterpret_cast<uint4*>(hidden + (size_t)t * d);
@@ -947,17 +969,15 @@ cudaError_t launch_mc_decide(const Ctx* c, int T, cudaStream_t s) {
 // it could only wait, so contexts with SAE weight sets leave every batch to the 16-row kernel.
 bool has_tc_probe_stage(const Ctx* c) { return has_multiclass_stage(c) && c->cfg.n_groups_max == 0; }
 
-cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s) {
+cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s, bool allow_pdl) {
   if (c->cfg.flags & MIX_FLAG_SLOT_CHAINS) {
-    probe_steer_chain_kernel<<<c->cfg.T_max, kChainWarps * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps,
-                                                                       c->d_gates, c->d_chain_next, c->cfg.n_slots_max,
-                                                                       hidden, c->cfg.d_model, scores, c->cfg.C_max,
-                                                                       c->d_status);
+    return launch_pdl(allow_pdl ? kPdlHook : 0, probe_steer_chain_kernel, dim3(c->cfg.T_max), dim3(kChainWarps * 32), 0, s,
+                      c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates, c->d_chain_next, c->cfg.n_slots_max, hidden,
+                      c->cfg.d_model, scores, c->cfg.C_max, c->d_status);
   } else if (c->cfg.T_max <= kTeamMaxRows) {
-    probe_steer_team_kernel<8><<<c->cfg.T_max, 8 * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates,
-                                                              c->cfg.n_slots_max, hidden, c->cfg.d_model, scores,
-                                                              c->cfg.C_max, c->d_status,
-                                                              reinterpret_cast<const uint4*>(c->d_vec_arena));
+    return launch_pdl(allow_pdl ? kPdlHook : 0, probe_steer_team_kernel<8>, dim3(c->cfg.T_max), dim3(8 * 32), 0, s,
+                      c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates, c->cfg.n_slots_max, hidden, c->cfg.d_model,
+                      scores, c->cfg.C_max, c->d_status, reinterpret_cast<const uint4*>(c->d_vec_arena));
   } else {
     const int blocks = (c->cfg.T_max + kWarpsPerBlock - 1) / kWarpsPerBlock;
     probe_steer_kernel<<<blocks, kWarpsPerBlock * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates,
