@@ -611,3 +611,35 @@ def test_guard_bands_around_the_callers_buffers_stay_intact(which):
     ref = run_gpu(w)
     assert np.array_equal(W.bits(h), ref["hidden"])
     m.destroy()
+
+
+# ------------------------------------------------------------------ the encode epilogue's running TopK bound
+@pytest.mark.parametrize("k", [1, 7, 64, 128, 129])
+@pytest.mark.parametrize("case", ["plain", "all_negative", "winners_in_one_tile", "equal_across_tiles"])
+def test_topk_running_bound_adversarial(k, case):
+    """Many feature tiles per CTA-wave on few rows, so later tiles start from the bound earlier tiles published:
+    k at the slot count's edges (128 slots; 129 switches the bound off), pre-activations that are all negative,
+    more than eight winners inside one tile (the candidate lists overflow: flagged rows, exact fallback), and
+    values repeated exactly in every tile (ties across tiles: the lower feature id wins)."""
+    d, S, T = 128, 256 * 40, 70                          # 40 feature tiles, one ragged row tile
+    g = torch.Generator(device=DEV); g.manual_seed(100 + k)
+    We = (torch.randn((S, d), generator=g, device=DEV) * d ** -0.5).to(torch.bfloat16)
+    be = torch.randn((S,), generator=g, device=DEV) * 0.05
+    if case == "all_negative":
+        be = be - 50.0
+    elif case == "winners_in_one_tile":
+        be[256 * 17 + 3: 256 * 17 + 3 + 12] += 30.0       # twelve of the largest values sit in tile 17
+    elif case == "equal_across_tiles":
+        We[256:] = We[:256].repeat(39, 1)                 # every tile repeats tile 0: 40-fold exact ties
+        be[256:] = be[:256].repeat(39)
+    w = _one_sae_workload(d, S, W.SAE_TOPK, k, T, True, ([3, 256 * 17 + 5], [2.0, 0.0], [0, 1]), W_enc=We, b_enc=be)
+    out = run_gpu(w, graph=True, replays=2)
+    check_parity(W.host(w), out, expect_status=None)
+    assert out["status"] & ~_mixlib().MIX_STATUS_TOPK_GENERAL == 0
+    if case == "equal_across_tiles":
+        # the tie rule across tiles, free of fp32-vs-fp64 near-ties between DIFFERENT base features: a copy in
+        # tile m is selected only if the copies in all lower tiles are
+        for t in range(T):
+            ids = set(out["topk_idx"][t, :k].tolist())
+            for j in ids:
+                assert all((j % 256) + 256 * m in ids for m in range(j // 256)), "row %d id %d" % (t, j)
