@@ -509,9 +509,12 @@ __device__ __forceinline__ void warp_edit_coefs(int p, int slot, const AppEntry&
   }
 }
 
-// decode_kernel: a CTA owns kDecRows consecutive packed rows.  Rows that keep the error term only get
-// their edit coefficients (one warp per row, all at once); rows whose app replaces the residual are
-// then rebuilt one after the other by the whole CTA:  h' = b_dec + sum_j f'_j W_dec[j].
+// decode_kernel: a CTA owns `rows_per_cta` (kDecRows or 1) consecutive packed rows.  Rows that keep the error
+// term only get their edit coefficients (one warp per row, all at once); rows whose app replaces the
+// residual are then rebuilt one after the other by the whole CTA:  h' = b_dec + sum_j f'_j W_dec[j].
+// Eight rows per CTA is the form for contexts whose apps all keep the error term (an eighth of the CTAs);
+// where a replacing app is registered the launch gives every row its own CTA, so that those rows -- a
+// CTA-wide gather each -- run side by side.  Either form handles every kind of row.
 __global__ void __launch_bounds__(kDecThreads)
 decode_kernel(__nv_bfloat16* __restrict__ hidden, int d, const float* __restrict__ Z, long long ldz,
               const int* __restrict__ panel_row, const int* __restrict__ row_slot,
@@ -519,7 +522,7 @@ decode_kernel(__nv_bfloat16* __restrict__ hidden, int d, const float* __restrict
               const GroupEntry* __restrict__ groups, const int* __restrict__ edit_idx,
               const float* __restrict__ edit_val, const unsigned char* __restrict__ edit_mode, int r_max, int k_max,
               const int* __restrict__ ws_idx, const float* __restrict__ ws_val,
-              RowDelta* __restrict__ row_delta, float* __restrict__ edit_coef) {
+              RowDelta* __restrict__ row_delta, float* __restrict__ edit_coef, int rows_per_cta) {
   pdl_wait();
   pdl_launch_dependents();
   __shared__ float s_coef[kDecList];
@@ -529,10 +532,10 @@ decode_kernel(__nv_bfloat16* __restrict__ hidden, int d, const float* __restrict
   __shared__ int s_replace[kDecRows];                  // token row of a replace-mode row, else -1
   __shared__ int s_n;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int p0 = blockIdx.x * kDecRows;
+  const int p0 = blockIdx.x * rows_per_cta;
   const int n_rows = rs->n_panel_rows;
   if (p0 >= n_rows) return;
-  {
+  if (warp < rows_per_cta) {
     const int p = p0 + warp;
     const int t = p < n_rows ? panel_row[p] : -1;
     int replace_t = -1;
@@ -554,7 +557,7 @@ decode_kernel(__nv_bfloat16* __restrict__ hidden, int d, const float* __restrict
   }
   __syncthreads();
   const int nvec = d >> 3;
-  for (int r = 0; r < kDecRows; ++r) {                 // CTA-uniform
+  for (int r = 0; r < rows_per_cta; ++r) {             // CTA-uniform
     const int t = s_replace[r];
     if (t < 0) continue;
     const int p = p0 + r;
@@ -904,15 +907,20 @@ cudaError_t launch_edit_only(const Ctx* c, __nv_bfloat16* hidden, int T, cudaStr
                                                             c->d_edit_mode, c->cfg.r_max);
 }
 
-// Two kernels: decode_kernel (one CTA per row) rebuilds the rows whose app replaces the residual and, for
-// the rows that keep the error term, only works out the coefficients of their edits; decode_delta_kernel
-// then adds those rows' deltas, eight rows per CTA.
+// Two kernels: decode_kernel rebuilds the rows whose app replaces the residual and, for the rows that keep
+// the error term, only works out the coefficients of their edits; decode_delta_kernel then adds those
+// rows' deltas, eight rows per CTA.  decode_kernel's rows per CTA follow from the apps registered when the
+// call is enqueued (or captured): eight where every SAE app keeps the error term, one as soon as a
+// replacing app exists (the sae_static path, whose context keeps no host copy of the app table, takes one).
 cudaError_t launch_decode(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s) {
-  return launch_pdl(kPdlTail, decode_kernel, dim3((c->panel_rows_cap + kDecRows - 1) / kDecRows), dim3(kDecThreads), 0, s, hidden, c->cfg.d_model, c->d_z, c->cfg.d_sae_max,
-                                                          c->d_panel_row, c->d_row_slot, c->d_route, c->d_apps,
-                                                          c->d_groups, c->d_edit_idx, c->d_edit_val, c->d_edit_mode,
-                                                          c->cfg.r_max, c->cfg.k_max, c->d_topk_idx, c->d_topk_val,
-                                                          c->d_row_delta, c->d_edit_coef);
+  bool replacing = c->h_apps == nullptr;
+  for (int i = 0; c->h_apps != nullptr && i < c->cfg.n_slots_max; ++i)
+    replacing = replacing || (c->h_apps[i].valid && (c->h_apps[i].kind & kKindMask) == MIX_SAE && !c->h_apps[i].add_error);
+  const int rows_per_cta = replacing ? 1 : kDecRows;
+  return launch_pdl(kPdlTail, decode_kernel, dim3((c->panel_rows_cap + rows_per_cta - 1) / rows_per_cta), dim3(kDecThreads), 0, s,
+                    hidden, c->cfg.d_model, c->d_z, c->cfg.d_sae_max, c->d_panel_row, c->d_row_slot, c->d_route, c->d_apps,
+                    c->d_groups, c->d_edit_idx, c->d_edit_val, c->d_edit_mode, c->cfg.r_max, c->cfg.k_max, c->d_topk_idx,
+                    c->d_topk_val, c->d_row_delta, c->d_edit_coef, rows_per_cta);
 }
 
 cudaError_t launch_decode_delta(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s) {
