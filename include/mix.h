@@ -311,7 +311,11 @@ int mix_set_feature_out(mix_ctx* ctx, int* topk_idx, float* topk_val, int* n_act
    part that looks up the live count, slot map, app entry and single-vector weights -- tables the
    library owns and only copies write -- overlaps that kernel; `hidden`, gate scores and
    multi-class probe weights are read only after the predecessor has completed and flushed, and the
-   grid does not end before it.  Behind any other kernel nothing changes.  Device-side
+   grid does not end before it.  Behind any other kernel nothing changes.  Two launch shapes follow
+   from what is registered when the call is enqueued or captured -- the encode's epilogue warps
+   (TopK weight set present or not) and the decode's rows per CTA (a replacing SAE app present or
+   not); this is performance only: every shape handles every registration, so tables rewritten
+   after a capture are still applied correctly.  Device-side
    problems (bad slot ids, ...) are reported through the status word, never by faulting.
    Errors: INVALID_ARG (NULL hidden, misaligned), OUT_OF_RANGE (T), CUDA (launch failure). */
 int mix_apply(mix_ctx* ctx, void* hidden, int T, float* scores_out, void* stream);
