@@ -49,18 +49,6 @@ int load_encode_fn() {
 }
 
 // bf16 [rows, d] row-major; box = kTileK columns x box_rows rows; 128-byte swizzle.
-// 8-bit encoder tiles: rows of 64 bytes, plain (unswizzled) boxes of 256 rows
-int make_tmap_u8(CUtensorMap* out, const void* base, unsigned long long rows) {
-  cuuint64_t dims[2] = {(cuuint64_t)kTileK, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)kTileK};
-  cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)kTileN};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = g_encode(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? MIX_OK : MIX_ERR_CUDA;
-}
-
 // E4M3 codes [rows, width] row-major for the 8-bit contraction: box = 128 bytes x box_rows rows; 128-byte swizzle.
 int make_tmap_e4m3(CUtensorMap* out, const void* base, unsigned long long rows, unsigned long long width, int box_rows) {
   cuuint64_t dims[2] = {(cuuint64_t)width, (cuuint64_t)rows};
@@ -220,7 +208,7 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
   if ((cfg->flags & MIX_FLAG_SLOT_CHAINS) && (cfg->flags & MIX_FLAG_SAE_EDIT_ONLY)) return MIX_ERR_INVALID_ARG;
   if ((cfg->flags & MIX_FLAG_FP8_W_ENC) && (cfg->flags & (MIX_FLAG_ENCODE_SIMT | MIX_FLAG_SAE_EDIT_ONLY))) return MIX_ERR_INVALID_ARG;
   if ((cfg->flags & MIX_FLAG_FP8_ACT) && !(cfg->flags & MIX_FLAG_FP8_W_ENC)) return MIX_ERR_INVALID_ARG;
-  if ((cfg->flags & MIX_FLAG_FP8_ACT) && cfg->d_model % (2 * kTileK)) return MIX_ERR_UNSUPPORTED;
+  if ((cfg->flags & MIX_FLAG_FP8_W_ENC) && cfg->d_model % (2 * kTileK)) return MIX_ERR_UNSUPPORTED;   // k-blocks of 128 codes
   mix_ctx* c = static_cast<mix_ctx*>(calloc(1, sizeof(mix_ctx)));
   if (!c) return MIX_ERR_NO_MEMORY;
   c->cfg = *cfg;
@@ -256,7 +244,7 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
     const size_t P = c->panel_rows_cap;
     ok = ok && dev_alloc(&c->d_panel, P * cfg->d_model) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_panel_row, P) == cudaSuccess;
-    if (cfg->flags & MIX_FLAG_FP8_ACT) ok = ok && dev_alloc(&c->d_act_scale, P) == cudaSuccess;
+    if (cfg->flags & MIX_FLAG_FP8_W_ENC) ok = ok && dev_alloc(&c->d_act_scale, P) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_mtile_group, P / kTileM) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_row_group, T) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_row_slot, T) == cudaSuccess;
@@ -297,8 +285,8 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
     if (e == cudaSuccess && !(cfg->flags & MIX_FLAG_ENCODE_SIMT)) {
       if (load_encode_fn() != MIX_OK)
         e = cudaErrorUnknown;
-      else if ((cfg->flags & MIX_FLAG_FP8_ACT)
-                   ? make_tmap_e4m3(&c->tmap_panel, c->d_panel, c->panel_rows_cap, cfg->d_model, kTileM) != MIX_OK
+      else if ((cfg->flags & MIX_FLAG_FP8_W_ENC)    // codes: P rows (8-bit input) or 2 P rows (hi, lo) in the same buffer
+                   ? make_tmap_e4m3(&c->tmap_panel, c->d_panel, 2ull * c->panel_rows_cap, cfg->d_model, kTileM) != MIX_OK
                    : make_tmap(&c->tmap_panel, c->d_panel, c->panel_rows_cap, cfg->d_model, kTileM) != MIX_OK)
         e = cudaErrorUnknown;
       if (e == cudaSuccess && c->d_act_scale) e = cudaMemset(c->d_act_scale, 0, c->panel_rows_cap * sizeof(float));
@@ -381,7 +369,8 @@ int mix_register_sae_weights(mix_ctx* c, int group, const mix_sae_weights* w, vo
   if (!(c->cfg.flags & MIX_FLAG_ENCODE_SIMT)) {
     CUtensorMap tm;
     if (fp8) {
-      // library-owned tile-ordered copy of the codes: [S/256][d/64][256][64] bytes, seen by TMA as a 64-byte-wide matrix
+      // library-owned tile-ordered copy of the codes: [S/256][d/128][256][128] bytes, seen by TMA as a 128-byte-wide
+      // matrix (128-byte swizzled boxes of 256 rows)
       if (c->owned_w_tiled[group]) { cudaStreamSynchronize(s); cudaFree(c->owned_w_tiled[group]); c->owned_w_tiled[group] = nullptr; }
       const size_t n_el = (size_t)w->d_sae * c->cfg.d_model;
       if (cudaMalloc(reinterpret_cast<void**>(&c->owned_w_tiled[group]), n_el) != cudaSuccess) {
@@ -389,12 +378,8 @@ int mix_register_sae_weights(mix_ctx* c, int group, const mix_sae_weights* w, vo
         MIX_FAIL(c, MIX_ERR_NO_MEMORY, "cannot allocate the tile-ordered copy of the 8-bit W_enc");
       }
       unsigned char* tiled = reinterpret_cast<unsigned char*>(c->owned_w_tiled[group]);
-      // (8-bit input as well: blocks of 128 codes per row, [S/256][d/128][256][128], 128-byte swizzled boxes)
-      const bool e4 = (c->cfg.flags & MIX_FLAG_FP8_ACT) != 0;
-      MIX_CUDA(c, launch_retile_fp8(static_cast<const unsigned char*>(w->W_enc), tiled, w->d_sae, c->cfg.d_model,
-                                    e4 ? 2 * kTileK : kTileK, s));
-      if ((e4 ? make_tmap_e4m3(&tm, tiled, (unsigned long long)(n_el / (2 * kTileK)), 2 * kTileK, kTileN)
-              : make_tmap_u8(&tm, tiled, (unsigned long long)(n_el / kTileK))) != MIX_OK)
+      MIX_CUDA(c, launch_retile_fp8(static_cast<const unsigned char*>(w->W_enc), tiled, w->d_sae, c->cfg.d_model, 2 * kTileK, s));
+      if (make_tmap_e4m3(&tm, tiled, (unsigned long long)(n_el / (2 * kTileK)), 2 * kTileK, kTileN) != MIX_OK)
         MIX_FAIL(c, MIX_ERR_CUDA, "cuTensorMapEncodeTiled failed for the 8-bit W_enc");
     } else if (c->cfg.flags & MIX_FLAG_RETILE_W_ENC) {
       // library-owned tile-contiguous copy: [S/256][d/64][256][64], seen by TMA as a 64-column matrix

@@ -2,6 +2,7 @@
 //
 // probe_steer_kernel is the bandwidth kernel of the hook: one warp per token row, 16-byte
 // loads, fp32 FMA, shuffle reductions.  A row whose slot is -1 costs one 4-byte load.
+#include <cuda_fp16.h>
 #include <cuda_fp8.h>
 
 #include "mix_internal.h"
@@ -857,14 +858,21 @@ pack_kernel(const __nv_bfloat16* __restrict__ hidden, const int* __restrict__ pa
   for (int i = lane; i < nvec; i += 32) dst[i] = __ldg(src + i);
 }
 
-// 8-bit encoder input: every routed row is quantised on its way into the panel.  s = the smallest
-// power of two with max|h_i| / s <= 448 (never below 2^-100; 1 for a row of zeros), code_i = E4M3
-// nearest to h_i / s (the division is exact, the conversion rounds to nearest even).  One warp per row:
-// a first pass for the largest magnitude, a second one (the row is in L1 by then) for the codes.
+// 8-bit encoder: every routed row goes into the panel as E4M3 codes with a power-of-two row scale.
+// s = the smallest power of two with max|h_i| / s <= 448 (never below 2^-100; 1 for a row of zeros); h_i / s is
+// exact in fp32, the conversion rounds to nearest even.  One warp per row: a first pass for the largest
+// magnitude, a second one (the row is in L1 by then) for the codes.
+//   kSplit = false (MIX_FLAG_FP8_ACT): code_i = E4M3 nearest to h_i / s -- the encoder's input IS quantised.
+//   kSplit = true  (MIX_FLAG_FP8_W_ENC alone): the bf16 row is kept, as the sum of two E4M3 operands with the same
+//     scale: hi_i = E4M3 nearest to x = h_i / s, lo_i = E4M3 nearest to x - hi_i (exact subtraction).  A bf16 value
+//     has 8 significant bits, hi takes the leading 4 and the remainder has at most 4, so hi + lo = x exactly
+//     unless bits of x lie below 2^-9 (the subnormal step of E4M3), i.e. the error per element is at most
+//     2^-10 s <= 4.4e-6 max|h_i| and zero for |h_i| >= 2^-2 s.  The lo codes go to rows [lo_row0 + p] of the panel.
+template <bool kSplit>
 __global__ void __launch_bounds__(256)
 pack_e4m3_kernel(const __nv_bfloat16* __restrict__ hidden, const int* __restrict__ panel_row,
                  const RouteState* __restrict__ rs, unsigned char* __restrict__ panel, float* __restrict__ act_scale, int d,
-                 unsigned* __restrict__ tau_slots, unsigned* __restrict__ tau_min) {
+                 unsigned* __restrict__ tau_slots, unsigned* __restrict__ tau_min, int lo_row0) {
   pdl_wait();
   pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -876,9 +884,13 @@ pack_e4m3_kernel(const __nv_bfloat16* __restrict__ hidden, const int* __restrict
   }
   const int t = panel_row[p];
   uint2* dst = reinterpret_cast<uint2*>(panel + (size_t)p * d);
+  uint2* dst_lo = reinterpret_cast<uint2*>(panel + ((size_t)lo_row0 + p) * d);
   const int nvec = d >> 3;
   if (t < 0) {   // padding rows of a tile
-    for (int i = lane; i < nvec; i += 32) dst[i] = make_uint2(0u, 0u);
+    for (int i = lane; i < nvec; i += 32) {
+      dst[i] = make_uint2(0u, 0u);
+      if (kSplit) dst_lo[i] = make_uint2(0u, 0u);
+    }
     if (lane == 0) act_scale[p] = 0.f;
     return;
   }
@@ -901,13 +913,18 @@ pack_e4m3_kernel(const __nv_bfloat16* __restrict__ hidden, const int* __restrict
   for (int i = lane; i < nvec; i += 32) {
     const uint4 q = __ldg(src + i);
     const unsigned w[4] = {q.x, q.y, q.z, q.w};
-    unsigned short c[4];
+    unsigned short c[4], cl[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const float lo = __uint_as_float(w[u] << 16) * inv, hi = __uint_as_float(w[u] & 0xffff0000u) * inv;
       c[u] = __nv_cvt_float2_to_fp8x2(make_float2(lo, hi), __NV_SATFINITE, __NV_E4M3);
+      if (kSplit) {
+        const float2 back = __half22float2(__half2(__nv_cvt_fp8x2_to_halfraw2(c[u], __NV_E4M3)));   // exact: E4M3 fits fp16
+        cl[u] = __nv_cvt_float2_to_fp8x2(make_float2(lo - back.x, hi - back.y), __NV_SATFINITE, __NV_E4M3);
+      }
     }
     dst[i] = make_uint2((unsigned)c[0] | ((unsigned)c[1] << 16), (unsigned)c[2] | ((unsigned)c[3] << 16));
+    if (kSplit) dst_lo[i] = make_uint2((unsigned)cl[0] | ((unsigned)cl[1] << 16), (unsigned)cl[2] | ((unsigned)cl[3] << 16));
   }
 }
 
@@ -1017,9 +1034,13 @@ cudaError_t launch_route(const Ctx* c, int T, cudaStream_t s, unsigned long long
 
 cudaError_t launch_pack(const Ctx* c, const __nv_bfloat16* hidden, cudaStream_t s) {
   const int blocks = (c->panel_rows_cap + 7) / 8;
+  unsigned char* codes = reinterpret_cast<unsigned char*>(c->d_panel);
   if (c->cfg.flags & MIX_FLAG_FP8_ACT)
-    return launch_pdl(kPdlPack, pack_e4m3_kernel, dim3(blocks), dim3(256), 0, s, hidden, c->d_panel_row, c->d_route,
-                      reinterpret_cast<unsigned char*>(c->d_panel), c->d_act_scale, c->cfg.d_model, c->d_tau, c->d_tau_min);
+    return launch_pdl(kPdlPack, pack_e4m3_kernel<false>, dim3(blocks), dim3(256), 0, s, hidden, c->d_panel_row, c->d_route,
+                      codes, c->d_act_scale, c->cfg.d_model, c->d_tau, c->d_tau_min, 0);
+  if (c->cfg.flags & MIX_FLAG_FP8_W_ENC)      // hi codes in rows [0, P), lo codes in rows [P, 2P) of the same buffer
+    return launch_pdl(kPdlPack, pack_e4m3_kernel<true>, dim3(blocks), dim3(256), 0, s, hidden, c->d_panel_row, c->d_route,
+                      codes, c->d_act_scale, c->cfg.d_model, c->d_tau, c->d_tau_min, c->panel_rows_cap);
   return launch_pdl(kPdlPack, pack_kernel, dim3(blocks), dim3(256), 0, s, hidden, c->d_panel_row, c->d_route, c->d_panel, c->cfg.d_model, c->d_tau, c->d_tau_min);
 }
 

@@ -14,22 +14,17 @@
 // No TMA multicast and no clusters.  Every wait is bounded: on expiry the CTA raises
 // MIX_STATUS_WAIT_TIMEOUT, lets its copies land, frees its tensor memory and returns.
 //
-// 8-bit encoder (kFp8): the W_enc tile arrives as 256 x 64 E4M3 codes (16 KiB, half the bytes);
-// eight more warps behind four epilogue warps (two teams on alternate k-blocks) widen it to bf16 -- exactly: every E4M3 value is
-// a bf16 value -- into the same 128-byte-swizzled layout TMA would have produced, and only then
-// is the k-block handed to the MMA warp; the per-feature scale is applied to the fp32
-// accumulator in the epilogue.  The copies land in a ring of 5 stages of 32 KiB (panel 16,
-// codes 16) and the widened tiles go through a separate ring of two 32 KiB slots.  This form
-// halves the encoder's footprint in HBM but is NOT faster than the bf16 form: the widening adds
-// 48 KiB of load/store traffic per k-block to a shared memory that the copies (32 KiB) and the
-// tensor core's operand reads (48 KiB) already keep busy, and the widening warps wait on it.
-//
-// 8-bit encoder AND 8-bit input (kEnc == 2): the panel holds E4M3 codes too (quantised per row with
-// a power-of-two scale by the pack step), so both operands go to the tensor core as they arrive:
-// tcgen05.mma kind::f8f6f4, 128 x 256 x 32 per instruction.  A k-block is 128 elements (the same
-// 128-byte swizzled rows, 16 + 32 KiB per stage, four instructions), so the kernel is the bf16
-// kernel with half as many k-blocks; the epilogue multiplies the accumulator by row scale x
-// feature scale.
+// 8-bit encoder (kEnc != 0): W_enc is E4M3 codes with one fp32 scale per feature, and the contraction is
+// tcgen05.mma kind::f8f6f4 (both operands E4M3), 128 x 256 x 32 per instruction.  A k-block is 128 elements
+// (the same 128-byte swizzled rows: 16 KiB of panel, 32 KiB of W_enc, four instructions), so the kernel is the
+// bf16 kernel with half as many k-blocks; the epilogue multiplies the accumulator by row scale x feature scale.
+//   kEnc == 2 (8-bit input): the panel holds the row quantised to E4M3 with a power-of-two scale.
+//   kEnc == 1 (the hidden state stays bf16): the pack step split each row EXACTLY (down to 2^-10 of the scale)
+//     into two E4M3 operands hi + lo with one common power-of-two scale; a stage carries both panel tiles
+//     (16 + 16 + 32 KiB, three stages) and the eight instructions of a k-block accumulate hi W and lo W into
+//     the same accumulator.  Per element of K that is the tensor time of the bf16 kernel with half the W_enc
+//     bytes: as fast as kEnc == 2 where the stream of W_enc is the bound, as fast as bf16 where the tensor
+//     pipe is.
 #include "mix_internal.h"
 #include "tc_common.cuh"
 
@@ -37,27 +32,23 @@ namespace mix {
 
 namespace {
 
-constexpr int kMaxStages = 5;
-constexpr int kBRing = 2;                      // 8-bit encoder: widened W_enc tiles in flight between the widening warps and the MMA
-constexpr int kABytes = kTileM * kTileK * 2;   // 16 KiB
-constexpr int kBBytes = kTileN * kTileK * 2;   // 32 KiB
-constexpr int kRawBytes = kTileN * kTileK;     // 16 KiB of E4M3 codes (8-bit encoder only)
-constexpr int kConvWarps = 4;                  // warps per widening team (8-bit encoder only)
+constexpr int kMaxStages = 4;
+constexpr int kABytes = kTileM * kTileK * 2;   // 16 KiB: 128 rows of 128 bytes
+constexpr int kBBytes = kTileN * kTileK * 2;   // 32 KiB: 256 rows of 128 bytes
 constexpr int kXchgEntries = kCandPerTile + 2;  // a top-9 list and the bound it was collected under
-constexpr int kConvTeams = 2;                  // team g (warps 6 + 4g ..) widens every k-block with index = g mod 2, into slot g
-// kEnc: 0 = bf16 encoder and input; 1 = 8-bit encoder widened to bf16; 2 = 8-bit encoder and 8-bit input
+// kEnc: 0 = bf16 encoder and input; 1 = 8-bit encoder, bf16 input as two E4M3 operands; 2 = 8-bit encoder and 8-bit input
 template <int kEnc, int kEpi> struct TcCfg {
-  static_assert(kEpi == 4 || (kEpi == 8 && kEnc != 1), "epilogue warps");
-  static constexpr bool kFp8 = kEnc == 1;
-  static constexpr int kStages = kFp8 ? 5 : 4;
-  static constexpr int kStageBytes = kABytes + (kFp8 ? kRawBytes : kBBytes);
-  static constexpr int kRingBytes = kStages * kStageBytes + (kFp8 ? kBRing * kBBytes : 0);
+  static_assert(kEpi == 4 || kEpi == 8, "epilogue warps");
+  static constexpr bool kSplit = kEnc == 1;            // two panel tiles (hi, lo) per stage
+  static constexpr int kStages = kSplit ? 3 : 4;
+  static constexpr int kStageBytes = (kSplit ? 2 : 1) * kABytes + kBBytes;
+  static constexpr int kRingBytes = kStages * kStageBytes;
   // epilogue warps: 4 (one per tensor-memory lane quarter, all 256 columns) or 8 (two per quarter, 128 columns
   // each; the two top-9 lists of a row meet in shared memory).  One warp per scheduler runs the epilogue's
   // dependent compare/select chains at a fraction of the issue rate; two interleave.
   static constexpr int kEpiWarps = kEpi;
   static constexpr int kXchgBytes = kEpiWarps == 8 ? 2 * 4 * kXchgEntries * 32 * 8 : 0;   // [acc][quarter][entry][lane] x (value, column)
-  static constexpr int kThreads = 64 + kEpiWarps * 32 + (kFp8 ? kConvTeams * kConvWarps * 32 : 0);
+  static constexpr int kThreads = 64 + kEpiWarps * 32;
   static constexpr int kSmemBytes = kRingBytes + 1024 /* alignment slack */ + 1024 /* TcShared */ + kXchgBytes;
   static_assert(kSmemBytes <= 227 * 1024, "shared memory per CTA");
 };
@@ -68,8 +59,6 @@ constexpr long long kWaitCyclesTest = 2000000ll;  // ~1 ms: the cap under MIX_FL
 struct __align__(8) TcShared {
   unsigned long long full[kMaxStages];
   unsigned long long empty[kMaxStages];
-  unsigned long long conv[kBRing];        // 8-bit encoder: slot holds a widened W_enc tile
-  unsigned long long b_empty[kBRing];     // 8-bit encoder: the MMAs that read the slot are done
   unsigned long long tmem_full[2];
   unsigned long long tmem_empty[2];
   unsigned long long xchg_full[2][4];     // 8 epilogue warps: the upper-half warp's list of (accumulator, quarter) is in shared memory
@@ -166,24 +155,6 @@ __device__ __forceinline__ void top9_insert(float (&tv)[kCandPerTile + 1], int (
   }
 }
 
-// Four packed E4M3 codes -> four bf16 values, exactly, without conversion instructions (those
-// run at a fraction of the ALU rate and would make the widening the bottleneck).  A code byte
-// s.eeee.mmm placed as s.0000eeee.mmm0000 IS the bf16 number 2^-120 times the code's value --
-// bf16 has 8 exponent bits, so the 4-bit exponent field and the 3 mantissa bits drop into place,
-// and the codes with e = 0 become bf16 subnormals with the right value -- and one bf16x2
-// multiplication by 2^120 (exact: a power of two, result in range) finishes the job.
-__device__ __forceinline__ void e4m3x4_to_bf16x4(unsigned w, unsigned& lo, unsigned& hi) {
-  const unsigned t0 = __byte_perm(w, 0u, 0x1404);        // (b1 << 24) | (b0 << 8)
-  const unsigned t1 = __byte_perm(w, 0u, 0x3424);        // (b3 << 24) | (b2 << 8)
-  const unsigned u0 = (t0 & 0x80008000u) | ((t0 >> 4) & 0x07f007f0u);
-  const unsigned u1 = (t1 & 0x80008000u) | ((t1 >> 4) & 0x07f007f0u);
-  const unsigned k2 = 0x7B807B80u;                        // bf16 2^120, twice
-  const __nv_bfloat162 r0 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&u0), *reinterpret_cast<const __nv_bfloat162*>(&k2));
-  const __nv_bfloat162 r1 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&u1), *reinterpret_cast<const __nv_bfloat162*>(&k2));
-  lo = *reinterpret_cast<const unsigned*>(&r0);
-  hi = *reinterpret_cast<const unsigned*>(&r1);
-}
-
 template <int kEnc, int kEpi>
 __global__ void __launch_bounds__(TcCfg<kEnc, kEpi>::kThreads, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorMap* __restrict__ tmap_w,
@@ -191,9 +162,10 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
                  float* __restrict__ Z, long long ldz, int d, unsigned* __restrict__ status, int mode,
                  const int* __restrict__ mtile_flag, const int* __restrict__ n_flagged, float* __restrict__ cand_val,
                  int* __restrict__ cand_idx, float* __restrict__ cand_ninth, int cand_tiles, int w_tiled, int test_stall,
-                 const float* __restrict__ act_scale, unsigned* __restrict__ tau_slots, unsigned* __restrict__ tau_min) {
-  constexpr bool kFp8 = kEnc == 1;                     // codes widened to bf16 in shared memory
-  constexpr bool kE4 = kEnc == 2;                      // E4M3 x E4M3 contraction
+                 const float* __restrict__ act_scale, unsigned* __restrict__ tau_slots, unsigned* __restrict__ tau_min,
+                 int lo_row0) {
+  constexpr bool kE4 = kEnc != 0;                      // E4M3 x E4M3 contraction
+  constexpr bool kSplit = kEnc == 1;                   // the panel row is hi + lo: two operand tiles per k-block
   constexpr int kBlockK = kE4 ? 2 * kTileK : kTileK;   // elements per 128-byte row of either operand
   constexpr int kStages = TcCfg<kEnc, kEpi>::kStages;
   constexpr int kStageBytes = TcCfg<kEnc, kEpi>::kStageBytes;
@@ -207,7 +179,6 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
   // 1024-byte alignment: required by the 128-byte swizzle atoms
   unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   TcShared* sh = reinterpret_cast<TcShared*>(tiles + TcCfg<kEnc, kEpi>::kRingBytes);
-  unsigned char* bring = tiles + kStages * kStageBytes;      // 8-bit encoder: the ring of widened tiles
   float* xchg_val = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(sh) + 1024);
   int* xchg_idx = reinterpret_cast<int*>(xchg_val + 2 * 4 * kXchgEntries * 32);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -218,10 +189,6 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&sh->full[s]), 1);
       mbar_init(smem_u32(&sh->empty[s]), 1);
-    }
-    for (int j = 0; j < kBRing; ++j) {
-      mbar_init(smem_u32(&sh->conv[j]), kConvWarps);
-      mbar_init(smem_u32(&sh->b_empty[j]), 1);
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&sh->tmem_full[a]), 1);
@@ -266,25 +233,26 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
           // bounded wait runs out and the whole CTA leaves through the time-out path.
           if (test_stall) { ok = false; break; }
           const unsigned bar = smem_u32(&sh->full[stage]);
-          mbar_expect_tx(bar, kFp8 ? kABytes + kRawBytes : kABytes + kBBytes);
+          mbar_expect_tx(bar, kStageBytes);
           const unsigned sa = smem_u32(tiles + stage * kStageBytes);
+          const unsigned sw = sa + (kSplit ? 2 : 1) * kABytes;
           tma_load_2d(sa, &tmap_panel, kb * kBlockK, t.m_tile_global * kTileM, bar);
+          if (kSplit) tma_load_2d(sa + kABytes, &tmap_panel, kb * kBlockK, lo_row0 + t.m_tile_global * kTileM, bar);   // the lo codes
           // W_enc tile: rows n_tile*256.. of the row-major matrix, or -- when the weights were re-laid
-          // out at registration -- block (n_tile, kb) of the tile-contiguous copy [S/256][d/64][256][64]
-          if (kFp8 || kE4)   // block (n_tile, kb) of the tile-ordered codes (kFp8: into the stage's staging area)
-            tma_load_2d(sa + kABytes, tw, 0, (t.n_tile * num_kb + kb) * kTileN, bar);
-          else if (w_tiled)
-            tma_load_2d(sa + kABytes, tw, 0, (t.n_tile * num_kb + kb) * kTileN, bar);
+          // out at registration (always, for codes) -- block (n_tile, kb) of the tile-contiguous copy
+          // [S/256][d/kBlockK][256][kBlockK]
+          if (kE4 || w_tiled)
+            tma_load_2d(sw, tw, 0, (t.n_tile * num_kb + kb) * kTileN, bar);
           else
-            tma_load_2d(sa + kABytes, tw, kb * kTileK, t.n_tile * kTileN, bar);
+            tma_load_2d(sw, tw, kb * kTileK, t.n_tile * kTileN, bar);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      int stage = 0, bs = 0;
-      unsigned phase = 0, bphase = 0, acc = 0, acc_phase = 0;
+      int stage = 0;
+      unsigned phase = 0, acc = 0, acc_phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
         if (mode != 0 && !tile_wanted(decode_tile(sh->rs, groups, n_groups, tile, uniform_nt), groups, mode, mtile_flag)) continue;
@@ -292,79 +260,28 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
         tc_fence_after();
         const unsigned d_tmem = tmem_base + acc * kTileN;
         for (int kb = 0; kb < num_kb; ++kb) {
-          // 8-bit encoder: the widening warps waited for the stage's copies and arrive on conv[] after
-          // their bf16 tile is visible to the tensor core's (async-proxy) reads
-          if (!mbar_wait(smem_u32(kFp8 ? &sh->conv[bs] : &sh->full[stage]), kFp8 ? bphase : phase, sh, status)) { ok = false; break; }
+          if (!mbar_wait(smem_u32(&sh->full[stage]), phase, sh, status)) { ok = false; break; }
           tc_fence_after();
           const unsigned sa = smem_u32(tiles + stage * kStageBytes);
-          const unsigned sb = kFp8 ? smem_u32(bring + bs * kBBytes) : sa + kABytes;
+          const unsigned sb = sa + (kSplit ? 2 : 1) * kABytes;
           const unsigned long long da = umma_desc(sa), db = umma_desc(sb);
 #pragma unroll
           for (int k = 0; k < 4; ++k) {   // 16 bf16 or 32 codes = 32 bytes = 2 descriptor units per step
             if (kE4) umma_e4m3(d_tmem, da + 2ull * k, db + 2ull * k, kIdescE4, (unsigned)((kb | k) != 0));
             else umma(d_tmem, da + 2ull * k, db + 2ull * k, (unsigned)((kb | k) != 0));
           }
-          umma_commit(smem_u32(&sh->empty[stage]));
-          if (kFp8) {
-            umma_commit(smem_u32(&sh->b_empty[bs]));
-            bs ^= 1;
-            if (bs == 0) bphase ^= 1u;
+          if (kSplit) {                   // + lo W into the same accumulator
+            const unsigned long long dl = umma_desc(sa + kABytes);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) umma_e4m3(d_tmem, dl + 2ull * k, db + 2ull * k, kIdescE4, 1u);
           }
+          umma_commit(smem_u32(&sh->empty[stage]));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
         umma_commit(smem_u32(&sh->tmem_full[acc]));
         acc ^= 1u;
         if (acc == 0) acc_phase ^= 1u;
-      }
-    }
-  } else if (kFp8 && warp >= 2 + kEpiWarps) {
-    // widen the stage's 256 x 64 codes to bf16.  Thread c of 128 takes the 16-byte pieces c, c + 128, ...
-    // (piece = row * 4 + quarter of the row): 16 codes in, two 16-byte chunks of the row's 128 bytes out,
-    // stored where the 128-byte swizzle puts them (chunk index XOR row mod 8).
-    // Two teams of four warps take alternate k-blocks (team = slot of the widened-tile ring), so one
-    // team's stores and proxy fence overlap the other team's arithmetic.
-    const int team = (warp - (2 + kEpiWarps)) / kConvWarps;
-    const int ct = threadIdx.x - (2 + kEpiWarps + team * kConvWarps) * 32;
-    int stage = 0, bs = 0;
-    unsigned phase = 0, bphase = 0;
-    bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-      if (mode != 0 && !tile_wanted(decode_tile(sh->rs, groups, n_groups, tile, uniform_nt), groups, mode, mtile_flag)) continue;
-      for (int kb = 0; kb < num_kb; ++kb) {
-        if (bs != team) {                      // the other team's k-block
-          bs ^= 1;
-          if (bs == 0) bphase ^= 1u;
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
-          continue;
-        }
-        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&sh->full[stage]), phase, sh, status))) { ok = false; break; }
-        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&sh->b_empty[bs]), bphase ^ 1u, sh, status))) { ok = false; break; }
-        const uint4* raw = reinterpret_cast<const uint4*>(tiles + stage * kStageBytes + kABytes);
-        unsigned char* bt = bring + bs * kBBytes;
-        constexpr int kPieces = kTileN * 4 / (kConvWarps * 32);    // 16-byte pieces of codes per thread: 8
-        uint4 in[kPieces];
-#pragma unroll
-        for (int it = 0; it < kPieces; ++it) in[it] = raw[it * (kConvWarps * 32) + ct];   // all loads first
-#pragma unroll
-        for (int it = 0; it < kPieces; ++it) {
-          const int piece = it * (kConvWarps * 32) + ct;
-          const int r = piece >> 2, qr = piece & 3;
-          uint4 lo, hi;
-          e4m3x4_to_bf16x4(in[it].x, lo.x, lo.y);
-          e4m3x4_to_bf16x4(in[it].y, lo.z, lo.w);
-          e4m3x4_to_bf16x4(in[it].z, hi.x, hi.y);
-          e4m3x4_to_bf16x4(in[it].w, hi.z, hi.w);
-          unsigned char* row = bt + r * 128;
-          *reinterpret_cast<uint4*>(row + (((2 * qr) ^ (r & 7)) << 4)) = lo;
-          *reinterpret_cast<uint4*>(row + (((2 * qr + 1) ^ (r & 7)) << 4)) = hi;
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> async-proxy reads
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&sh->conv[bs]));
-        bs ^= 1;
-        if (bs == 0) bphase ^= 1u;
-        if (++stage == kStages) { stage = 0; phase ^= 1u; }
       }
     }
   } else {
@@ -597,6 +514,7 @@ cudaError_t encode_tc_prepare() {
   cudaError_t e = encode_tc_prepare_as<0, 4>();
   if (e == cudaSuccess) e = encode_tc_prepare_as<0, 8>();
   if (e == cudaSuccess) e = encode_tc_prepare_as<1, 4>();
+  if (e == cudaSuccess) e = encode_tc_prepare_as<1, 8>();
   if (e == cudaSuccess) e = encode_tc_prepare_as<2, 4>();
   if (e == cudaSuccess) e = encode_tc_prepare_as<2, 8>();
   return e;
@@ -610,7 +528,7 @@ static cudaError_t launch_encode_tc_as(const Ctx* c, int mode, cudaStream_t s) {
                     dim3(TcCfg<kEnc, kEpi>::kThreads), TcCfg<kEnc, kEpi>::kSmemBytes, s, c->tmap_panel, c->d_tmap_w, c->d_route,
                     c->d_groups, c->cfg.n_groups_max, c->d_z, c->cfg.d_sae_max, c->cfg.d_model, c->d_status, mode,
                     c->d_mtile_flag, c->d_n_flagged, c->d_cand_val, c->d_cand_idx, c->d_cand_ninth, c->cand_tiles, w_tiled,
-                    stall, c->d_act_scale, c->d_tau, c->d_tau_min);
+                    stall, c->d_act_scale, c->d_tau, c->d_tau_min, c->panel_rows_cap);
 }
 
 // Eight epilogue warps pay off for the TopK epilogue (selection work per element); the plain store of the
@@ -620,7 +538,7 @@ cudaError_t launch_encode_tc(const Ctx* c, int mode, cudaStream_t s) {
   bool topk = false;
   for (int g = 0; g < c->cfg.n_groups_max; ++g) topk = topk || (c->h_groups[g].valid && c->h_groups[g].act == MIX_SAE_TOPK);
   if (c->cfg.flags & MIX_FLAG_FP8_ACT) return topk ? launch_encode_tc_as<2, 8>(c, mode, s) : launch_encode_tc_as<2, 4>(c, mode, s);
-  if (c->cfg.flags & MIX_FLAG_FP8_W_ENC) return launch_encode_tc_as<1, 4>(c, mode, s);
+  if (c->cfg.flags & MIX_FLAG_FP8_W_ENC) return topk ? launch_encode_tc_as<1, 8>(c, mode, s) : launch_encode_tc_as<1, 4>(c, mode, s);
   return topk ? launch_encode_tc_as<0, 8>(c, mode, s) : launch_encode_tc_as<0, 4>(c, mode, s);
 }
 

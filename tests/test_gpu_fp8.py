@@ -1,5 +1,6 @@
-"""GPU: 8-bit (E4M3 codes x per-feature scale) encoder weights, widened to bf16 in shared memory in front
-of the tcgen05 contraction, against the oracle evaluated on the same codes and scales."""
+"""GPU: 8-bit (E4M3 codes x per-feature scale) encoder weights with the hidden state kept in bf16 (each row goes
+to the 8-bit tcgen05 contraction as the exact sum of two E4M3 operands), against the oracle evaluated on the same
+codes and scales."""
 import numpy as np
 import pytest
 import torch
@@ -19,8 +20,8 @@ def _mixlib():
 
 @pytest.mark.parametrize("graph", [False, True])
 def test_fp8_sae_heavy_small(graph):
-    # TopK sets, two row tiles with a ragged tail per weight set, 5 k-blocks, 4 feature tiles
-    w = W.make_sae_heavy(DEV, d=320, d_sae=1024, k=16, T=400, R=12, G=2, n_edit=6, edit_hint=oracle_edit_hint, fp8=True)
+    # TopK sets, two row tiles with a ragged tail per weight set, 3 k-blocks of 128, 4 feature tiles
+    w = W.make_sae_heavy(DEV, d=384, d_sae=1024, k=16, T=400, R=12, G=2, n_edit=6, edit_hint=oracle_edit_hint, fp8=True)
     out = run_gpu(w, flags=_mixlib().MIX_FLAG_FP8_W_ENC, graph=graph)
     st = check_parity(W.host(w), out)
     assert st["rows"] == 400
@@ -34,13 +35,13 @@ def test_fp8_mixed_small_jumprelu_and_probes():
 
 
 def test_fp8_wide_rows_many_stages():
-    # d = 4096: 64 k-blocks per tile, so every stage of the ring is reused 21 times per tile
+    # d = 4096: 32 k-blocks per tile, so every stage of the ring is reused 10 times per tile
     w = W.make_sae_heavy(DEV, d=4096, d_sae=512, k=8, T=130, R=5, G=1, n_edit=4, edit_hint=oracle_edit_hint, fp8=True)
     out = run_gpu(w, flags=_mixlib().MIX_FLAG_FP8_W_ENC)
     check_parity(W.host(w), out)
 
 
-def test_fp8_every_code_is_widened_exactly():
+def test_fp8_every_code_contracts_exactly():
     """One-hot rows read single encoder entries back: every one of the 254 finite codes, subnormal ones
     included, must come out of the contraction with exactly its value."""
     from oracle import mi_hook as O
@@ -116,3 +117,37 @@ def test_fp8_sae_heavy_full_size_sampled_rows():
     rows = [t for t in sample_rows(wh, per_kind=6) if w.apps[int(w.token_slot[t])].group == 1][:8]
     assert len(rows) >= 4
     check_parity(wh, out, rows=rows)
+
+
+def test_fp8_bf16_rows_reach_the_encoder_exactly():
+    """The hidden state is NOT quantised by MIX_FLAG_FP8_W_ENC alone: with an identity encoder (code 0x38 = 1 on the
+    diagonal) the TopK list of a row is the row itself, to the last bit for entries of at least 2^-10 of the row's
+    largest magnitude (hi + lo is exact there) and within 2^-10 of the row scale below that."""
+    from oracle import mi_hook as O
+    d = 256
+    codes = np.zeros((d, d), dtype=np.uint8)
+    codes[np.arange(d), np.arange(d)] = 0x38
+    g = torch.Generator(device=DEV); g.manual_seed(0)
+    W_dec = torch.randn((d, d), generator=g, device=DEV).to(torch.bfloat16)
+    sae = W.SaeWeights(d, W.SAE_TOPK, d, torch.from_numpy(codes).to(DEV), torch.zeros(d, device=DEV), W_dec,
+                       w_scale=torch.ones(d, device=DEV))
+    rng = np.random.default_rng(9)
+    rows = [rng.standard_normal(d), rng.standard_normal(d) * 2.0 ** 30, rng.standard_normal(d) * 2.0 ** -40, np.zeros(d),
+            rng.standard_normal(d) * np.exp(rng.uniform(-12, 12, d))]
+    X = O.bf16_to_f64(O.f64_to_bf16_bits(np.stack(rows)))
+    T = X.shape[0]
+    hidden = W.from_bits(O.f64_to_bf16_bits(X), DEV)
+    app = W.SaeApp(0, np.zeros(0, np.int32), np.zeros(0, np.float32), np.zeros(0, np.uint8), True)
+    w = W.Workload("rows", d, T, T, hidden, np.zeros(T, dtype=np.int32), {0: app}, {0: sae}, n_slots_max=1,
+                   n_groups_max=1, C_max=1, k_max=d, r_max=1, d_sae_max=d)
+    out = run_gpu(w, flags=_mixlib().MIX_FLAG_FP8_W_ENC)
+    for t in range(T):
+        idx = out["topk_idx"][t]
+        assert sorted(idx.tolist()) == list(range(d))
+        got = np.empty(d); got[idx] = out["topk_val"][t].astype(np.float64)
+        amax = np.abs(X[t]).max()
+        s = O.act_row_scale(X[t])                       # the same power-of-two scale the split uses
+        big = np.abs(X[t]) >= 0.25 * s
+        assert np.array_equal(got[big], X[t][big]), "row %d" % t
+        assert np.all(np.abs(got - X[t]) <= 2.0 ** -10 * s), "row %d" % t
+        assert amax == 0 or np.abs(got - X[t]).max() <= 4.5e-6 * amax

@@ -18,7 +18,7 @@ DEV = "cuda"
 def random_workload(seed, fp8=False, fp8_act=False):
     rng = np.random.default_rng(seed)
     g = torch.Generator(device=DEV); g.manual_seed(int(seed))
-    d = int(rng.choice([128, 256, 384, 512] if fp8_act else [64, 128, 192, 320, 512]))   # 8-bit input: k-blocks of 128
+    d = int(rng.choice([128, 256, 384, 512] if fp8 else [64, 128, 192, 320, 512]))   # 8-bit encoder: k-blocks of 128
     T = int(rng.choice([1, 7, 33, 128, 129, 300, 2100]))       # 2100 > 2048: the large-batch kernels
     n_groups = int(rng.integers(0, 4))
     hidden = (torch.randn((T, d), generator=g, device=DEV) * float(rng.choice([0.1, 1.0, 8.0]))).to(torch.bfloat16)
