@@ -265,12 +265,13 @@ def extras_sae(name, w, peaks, mixlib, extra_flags=0, w_enc_bytes_per_el=2.0):
             "token_rows_per_s": w.T_live / (min(times) * 1e-3), "status": status}
 
 
-def run_replay(peaks, mixlib, n_replays, fp8a=False):
+def run_replay(peaks, mixlib, n_replays, fp8a=False, fp8w=False):
     """Config 4: one captured graph at T_max = 2048, a fresh slot map and live count per replay.
+    fp8w: 8-bit encoder, bf16 rows as two E4M3 operands (half the W_enc bytes, the bf16 tensor time).
     fp8a: 8-bit encoder and 8-bit encoder input (half the W_enc bytes; the tensor bound is taken at twice the
     measured bf16 rate, the nominal ratio of the two formats)."""
-    w = W.make_replay("cuda", fp8=fp8a, fp8_act=fp8a)
-    m = W.make_context(mixlib.Mix, w, flags=SAE_FLAGS | (32 | 64 if fp8a else 0))
+    w = W.make_replay("cuda", fp8=fp8a or fp8w, fp8_act=fp8a)
+    m = W.make_context(mixlib.Mix, w, flags=SAE_FLAGS | (32 | 64 if fp8a else (32 if fp8w else 0)))
     T = w.T_max
     h = w.hidden.clone()
     scores = torch.zeros((T, 1), dtype=torch.float32, device="cuda")
@@ -298,7 +299,7 @@ def run_replay(peaks, mixlib, n_replays, fp8a=False):
             a = w.apps.get(int(token_slot[t]))
             if a is not None and a.kind == W.KIND_SAE:
                 counts[a.group] = counts.get(a.group, 0) + 1
-        wbytes = sum((1.0 if fp8a else 2.0) * w.d_model * w.groups[gi].d_sae for gi in counts)
+        wbytes = sum((1.0 if (fp8a or fp8w) else 2.0) * w.d_model * w.groups[gi].d_sae for gi in counts)
         flops = sum(2.0 * n * w.d_model * w.groups[gi].d_sae for gi, n in counts.items())
         bound_ms = max(wbytes / (peaks["hbm_gbs"] * 1e9),
                        flops / ((2.0 if fp8a else 1.0) * peaks["bf16_tflops"] * 1e12)) * 1e3
@@ -309,7 +310,8 @@ def run_replay(peaks, mixlib, n_replays, fp8a=False):
     a = np.array(rec)
     live = a[a[:, 2] > 0]
     ratio = live[:, 4] / live[:, 3] if len(live) else np.array([0.0])
-    return {"workload": "replay (config 4)" + (", 8-bit encoder and input" if fp8a else ""), "replays": n_replays, "status_or": bad_status,
+    return {"workload": "replay (config 4)" + (", 8-bit encoder and input" if fp8a else (", 8-bit encoder, bf16 rows" if fp8w else "")),
+            "replays": n_replays, "status_or": bad_status,
             "t_call_ms": {"min": float(a[:, 3].min()), "p50": float(np.median(a[:, 3])), "p90": float(np.quantile(a[:, 3], 0.9)),
                           "max": float(a[:, 3].max())},
             "empty_replay_ms": float(a[a[:, 0] == 0][:, 3].min()) if (a[:, 0] == 0).any() else None,
@@ -453,6 +455,8 @@ def run_workload(args):
         out = run_replay(peaks, mixlib, args.steps or 200)
     elif name == "replay_fp8a":
         out = run_replay(peaks, mixlib, args.steps or 200, fp8a=True)
+    elif name == "replay_fp8":
+        out = run_replay(peaks, mixlib, args.steps or 200, fp8w=True)
     else:
         raise SystemExit("unknown workload %r" % name)
     print(json.dumps(out), flush=True)
@@ -767,13 +771,18 @@ def run_mix(args, rank, world, local_rank):
                     "token_rows_per_s": eo["token_rows_per_s"], "status": eo["status"]}
                 del wm
                 torch.cuda.empty_cache()
-                # opt-in 8-bit contraction (quantised encoder and encoder input: a different numerical method)
-                for key, mk, label in (("sae_heavy_8bit", W.make_sae_heavy, "sae_heavy (config 2), 8-bit encoder and input"),
-                                       ("mixed_8bit", W.make_mixed, "mixed (config 3), 8-bit encoder and input")):
-                    r8 = extras_sae(label, mk("cuda", fp8=True, fp8_act=True), peaks, mixlib, extra_flags=32 | 64,
+                # opt-in 8-bit encoder: with the bf16 hidden state kept exact (two E4M3 operands per row), and with the
+                # encoder's input quantised as well (a different numerical method)
+                for key, mk, label, act in (
+                        ("sae_heavy_8bit_encoder", W.make_sae_heavy, "sae_heavy (config 2), 8-bit encoder, bf16 rows", False),
+                        ("mixed_8bit_encoder", W.make_mixed, "mixed (config 3), 8-bit encoder, bf16 rows", False),
+                        ("sae_heavy_8bit", W.make_sae_heavy, "sae_heavy (config 2), 8-bit encoder and input", True),
+                        ("mixed_8bit", W.make_mixed, "mixed (config 3), 8-bit encoder and input", True)):
+                    r8 = extras_sae(label, mk("cuda", fp8=True, fp8_act=act), peaks, mixlib, extra_flags=32 | (64 if act else 0),
                                     w_enc_bytes_per_el=1.0)
-                    r8["note"] = ("MIX_FLAG_FP8_W_ENC | MIX_FLAG_FP8_ACT; tensor fractions here are against the bf16 peaks: "
-                                  "halve them for the 8-bit peak (nominal ratio 2)")
+                    r8["note"] = ("MIX_FLAG_FP8_W_ENC" + (" | MIX_FLAG_FP8_ACT" if act else "") + "; tensor fractions here are "
+                                  "against the bf16 peaks" + (": halve them for the 8-bit peak (nominal ratio 2)" if act else
+                                                              " (two 8-bit instructions per element of K: the bf16 tensor time)"))
                     ex[key] = r8
                     torch.cuda.empty_cache()
             except Exception as e:                       # extras never break the contract line
@@ -792,7 +801,7 @@ def main():
     ap.add_argument("--no-retile", action="store_true",
                     help="SAE contexts stream W_enc as registered instead of a tile-contiguous copy (MIX_FLAG_RETILE_W_ENC)")
     ap.add_argument("--workload", default="decode",
-                    help="decode (the contract line) | sweep | sae_heavy | sae_heavy_fp8 | sae_heavy_fp8a | sae_small | sae_small_fp8 | sae_small_fp8a | mixed | mixed_fp8 | mixed_fp8a | mixed_small | mixed_small_fp8a | conditional | conditional_small | replay_fp8a | multiclass | multiclass_small | replay")
+                    help="decode (the contract line) | sweep | sae_heavy | sae_heavy_fp8 | sae_heavy_fp8a | sae_small | sae_small_fp8 | sae_small_fp8a | mixed | mixed_fp8 | mixed_fp8a | mixed_small | mixed_small_fp8a | conditional | conditional_small | replay_fp8 | replay_fp8a | multiclass | multiclass_small | replay")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     args = ap.parse_args()
     if args.no_retile:
