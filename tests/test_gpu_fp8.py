@@ -94,6 +94,10 @@ def test_fp8_api_errors():
             mixlib.Mix(d_model=128, T_max=8, n_slots_max=1, n_groups_max=1, k_max=4, r_max=1, d_sae_max=256,
                        flags=mixlib.MIX_FLAG_FP8_W_ENC | bad)
         assert e.value.code == -1
+    with pytest.raises(mixlib.MixError) as e:          # k-blocks of 128 codes: d_model must be a multiple of 128
+        mixlib.Mix(d_model=192, T_max=8, n_slots_max=1, n_groups_max=1, k_max=4, r_max=1, d_sae_max=256,
+                   flags=mixlib.MIX_FLAG_FP8_W_ENC)
+    assert e.value.code == -3
     m = mixlib.Mix(d_model=128, T_max=8, n_slots_max=1, n_groups_max=1, k_max=4, r_max=1, d_sae_max=256,
                    flags=mixlib.MIX_FLAG_FP8_W_ENC)
     g = torch.Generator(device=DEV); g.manual_seed(0)
