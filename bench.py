@@ -38,7 +38,7 @@ SAE_FLAGS = 2            # mix_config.flags of the SAE contexts of the extras / 
 # dram__bytes_read.sum + dram__bytes_write.sum of one probe_steer_team_kernel launch on this workload,
 # from the ncu capture summarised in profiles/probe_steer_kernel_decode.md (reads 2.40 MB, writes 0:
 # the steered rows are still dirty in L2 when the kernel ends).
-DECODE_DRAM_BYTES_PER_LAUNCH = 2399232
+DECODE_DRAM_BYTES_PER_LAUNCH = 2404352
 
 
 NOMINAL_HBM_GBS = 8000.0        # B200 HBM3e (DGX figure; HGX 7.7 TB/s): context beside the measured peak
