@@ -82,7 +82,7 @@ cudaError_t dev_alloc(T** p, size_t n) {
 void free_all(mix_ctx* c) {
   cudaFree(c->d_token_slot); cudaFree(c->d_n_live); cudaFree(c->d_apps); cudaFree(c->d_groups); cudaFree(c->d_gates); cudaFree(c->d_vec_arena); cudaFree(c->d_chain_next); cudaFree(c->d_row_slot);
   cudaFree(c->d_edit_idx); cudaFree(c->d_edit_val); cudaFree(c->d_edit_mode); cudaFree(c->d_status);
-  cudaFree(c->d_tmp_req); cudaFree(c->d_tmp_req_slot); cudaFree(c->d_panel); cudaFree(c->d_panel_row); cudaFree(c->d_act_scale); cudaFree(c->d_tau); cudaFree(c->d_tau_min);
+  cudaFree(c->d_tmp_req); cudaFree(c->d_tmp_req_slot); cudaFree(c->d_panel); cudaFree(c->d_panel_row); cudaFree(c->d_act_scale); cudaFree(c->d_tau); cudaFree(c->d_tau_min); cudaFree(c->d_eo_row_delta); cudaFree(c->d_eo_coef);
   cudaFree(c->d_mtile_group); cudaFree(c->d_row_group); cudaFree(c->d_route); cudaFree(c->d_z); cudaFree(c->d_topk_idx);
   cudaFree(c->d_topk_val); cudaFree(c->d_tmap_w); cudaFree(c->d_tmap_probe); cudaFree(c->d_mc_dense); cudaFree(c->d_cand_val); cudaFree(c->d_cand_idx);
   cudaFree(c->d_row_delta); cudaFree(c->d_edit_coef);
@@ -255,6 +255,10 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
     ok = ok && dev_alloc(&c->d_tmap_w, G) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_row_delta, P) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_edit_coef, P * (size_t)(cfg->r_max > 0 ? cfg->r_max : 1)) == cudaSuccess;
+    if (cfg->flags & MIX_FLAG_SAE_EDIT_ONLY) {
+      ok = ok && dev_alloc(&c->d_eo_row_delta, (size_t)T) == cudaSuccess;
+      ok = ok && dev_alloc(&c->d_eo_coef, (size_t)T * (size_t)(cfg->r_max > 0 ? cfg->r_max : 1)) == cudaSuccess;
+    }
     if (!(cfg->flags & MIX_FLAG_ENCODE_SIMT)) {
       c->cand_tiles = (int)(cfg->d_sae_max / kTileN);
       const size_t nc = P * (size_t)c->cand_tiles;
@@ -291,6 +295,9 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
         e = cudaErrorUnknown;
       if (e == cudaSuccess && c->d_act_scale) e = cudaMemset(c->d_act_scale, 0, c->panel_rows_cap * sizeof(float));
       if (e == cudaSuccess) e = encode_tc_prepare();
+    }
+    if (e == cudaSuccess && (cfg->flags & MIX_FLAG_SAE_EDIT_ONLY)) {
+      e = edit_only_prepare();
     }
   }
   if (e == cudaSuccess && has_tc_probe_stage(c)) {
@@ -798,7 +805,7 @@ int mix_launches_per_apply(const mix_ctx* c) {
   if (!c) return 0;
   const int front = 1 + (has_multiclass_stage(c) ? 1 : 0) + (has_tc_probe_stage(c) ? 2 : 0);
   if (c->cfg.n_groups_max == 0) return front;
-  return front + ((c->cfg.flags & MIX_FLAG_ENCODE_SIMT) ? 6 : 8) + ((c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) ? 1 : 0);
+  return front + ((c->cfg.flags & MIX_FLAG_ENCODE_SIMT) ? 6 : 8) + ((c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) ? 2 : 0);   // coefficient kernel + delta kernel
 }
 
 int mix_get_status(mix_ctx* c, unsigned* bits, void* stream) {

@@ -133,6 +133,8 @@ struct Ctx {
   float* d_cand_val;        // [P, cand_tiles, kCandPerTile] per-tile TopK candidates (fused epilogue)
   int* d_cand_idx;          // same shape: feature ids
   float* d_cand_ninth;      // [P, cand_tiles] the (kCandPerTile+1)-th largest value of each tile
+  RowDelta* d_eo_row_delta; // [T_max] edit-only shortcut: per token row, what decode_delta_kernel adds (MIX_FLAG_SAE_EDIT_ONLY)
+  float* d_eo_coef;         // [T_max, r_max]
   unsigned* d_tau_min;      // [P] the smallest of the row's first k slots, as last computed by a publisher
   unsigned* d_tau;          // [P, kTauSlots] order-preserving keys of pre-activations seen so far in this call (0 = empty)
   int cand_tiles;           // d_sae_max / kTileN
@@ -227,6 +229,7 @@ cudaError_t launch_select(const Ctx* c, bool flagged_only, cudaStream_t s);
 cudaError_t launch_decode(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s);         // rows without the error term
 cudaError_t launch_decode_delta(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s);   // rows with it
 cudaError_t launch_edit_only(const Ctx* c, __nv_bfloat16* hidden, int T, cudaStream_t s);
+cudaError_t edit_only_prepare();   // opt in to the dynamic shared memory of the edit-only kernel
 cudaError_t launch_compose_map(const Ctx* c, int T_live, int n_req, cudaStream_t s);
 cudaError_t launch_fold_bias(const __nv_bfloat16* W_enc, const float* b_enc, const float* b_dec, float* b_eff,
                              long long d_sae, int d, cudaStream_t s);

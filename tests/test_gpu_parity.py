@@ -643,3 +643,40 @@ def test_topk_running_bound_adversarial(k, case):
             ids = set(out["topk_idx"][t, :k].tolist())
             for j in ids:
                 assert all((j % 256) + 256 * m in ids for m in range(j // 256)), "row %d id %d" % (t, j)
+
+
+def test_edit_only_rows_of_different_slots_share_a_cta():
+    """The edit-only kernel takes eight consecutive token rows per CTA and shares the edited encoder / decoder rows
+    among rows of one slot: here the slot changes every one to three rows, two weight sets (ReLU and JumpReLU)
+    alternate, unhooked, probe and steering rows sit in between, the batch ends in the middle of a CTA's rows, and
+    d = 8192 uses the largest shared-memory layout."""
+    mixlib = _mixlib()
+    d, S, T = 8192, 512, 77
+    g = torch.Generator(device=DEV); g.manual_seed(21)
+    rng = np.random.default_rng(21)
+    groups = {0: W.make_sae_weights(g, DEV, d, S, W.SAE_RELU, b_enc_mean=-0.05),
+              1: W.make_sae_weights(g, DEV, d, S, W.SAE_JUMPRELU, theta_range=(0.05, 0.3))}
+    apps = {}
+    for s in range(6):                                   # six SAE apps, three per weight set, different edit lists
+        n_edit = int(rng.integers(1, 9))
+        idx = rng.integers(0, S, size=n_edit).astype(np.int32)
+        if n_edit >= 3:
+            idx[-1] = idx[0]                             # a repeated feature: the later entry wins
+        mode = rng.integers(0, 2, size=n_edit).astype(np.uint8)
+        val = np.where(mode == W.EDIT_CLAMP, rng.uniform(0.5, 6, size=n_edit), 0).astype(np.float32)
+        apps[s] = W.SaeApp(s % 2, idx, val, mode, True)
+    apps[6] = W.Steer((torch.randn(d, generator=g, device=DEV) * d ** -0.5).to(torch.bfloat16), 3.0)
+    apps[7] = W.Probe((torch.randn((1, d), generator=g, device=DEV) * d ** -0.5).to(torch.bfloat16), None, W.ACT_SIGMOID)
+    token_slot = np.full(T, -1, dtype=np.int32)
+    t = 0
+    while t < T:
+        seg = int(rng.integers(1, 4))
+        token_slot[t:t + seg] = int(rng.choice([-1, 0, 1, 2, 3, 4, 5, 6, 7]))
+        t += seg
+    hidden = torch.randn((T, d), generator=g, device=DEV).to(torch.bfloat16)
+    w = W.Workload("eo8", d, T, T - 3, hidden, token_slot, apps, groups, n_slots_max=8, n_groups_max=2, C_max=1,
+                   k_max=1, r_max=8, d_sae_max=S)
+    out = run_gpu(w, flags=mixlib.MIX_FLAG_SAE_EDIT_ONLY, graph=True)
+    st = check_parity(W.host(w), out, check_features=False)
+    assert st["rows"] == T
+    assert (token_slot[:T - 3] <= 5).sum() > 20 and len(set(token_slot[:T - 3].tolist())) >= 6
