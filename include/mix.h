@@ -352,7 +352,7 @@ int mix_get_status(mix_ctx* ctx, unsigned* bits, void* stream);
 
 /* Number of kernels one mix_apply() call launches on this context (fixed at mix_create):
    1 without SAE weight sets, else 8 (6 with MIX_FLAG_ENCODE_SIMT); one more when T_max > 2048
-   and C_max > 1 (multi-class probes of large batches run in a kernel of their own), and one more
+   and C_max > 1 (multi-class probes of large batches run in a kernel of their own), and two more
    with MIX_FLAG_SAE_EDIT_ONLY. */
 int mix_launches_per_apply(const mix_ctx* ctx);
 
@@ -364,7 +364,7 @@ int mix_launches_per_apply(const mix_ctx* ctx);
    probe_decide before and probe_tc after it if also n_groups_max == 0,]
    route, pack, encode, merge, encode (flagged row tiles), select, decode; with
    MIX_FLAG_ENCODE_SIMT the SAE part is route, pack, encode, select, decode; with
-   MIX_FLAG_SAE_EDIT_ONLY an edit_only kernel comes last. */
+   MIX_FLAG_SAE_EDIT_ONLY an edit_only and an edit_only_delta kernel come last. */
 int mix_set_stage_events(mix_ctx* ctx, void* const* events);
 
 /* Measurement aid for the paper's "CUDA-graph-safe kernel design" paragraph (separate static graph

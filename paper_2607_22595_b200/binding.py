@@ -305,7 +305,7 @@ class Mix:
                 front = ["probe_decide"] + front + ["probe_tc"]
         if self.cfg.n_groups_max == 0:
             return front
-        tail = ["edit_only"] if self.cfg.flags & MIX_FLAG_SAE_EDIT_ONLY else []
+        tail = ["edit_only", "edit_only_delta"] if self.cfg.flags & MIX_FLAG_SAE_EDIT_ONLY else []
         if self.cfg.flags & MIX_FLAG_ENCODE_SIMT:
             return front + ["route", "pack", "encode", "select", "decode", "decode_delta"] + tail
         return front + ["route", "pack", "encode", "merge", "encode_flagged", "select", "decode", "decode_delta"] + tail

@@ -776,6 +776,8 @@ int apply_impl(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream,
     if (c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) {
       MIX_CUDA(c, launch_edit_only(c, h, T, s));
       MIX_CUDA(c, tap());
+      MIX_CUDA(c, launch_edit_only_delta(c, h, s));
+      MIX_CUDA(c, tap());
     }
   }
   if (fork) MIX_CUDA(c, cudaStreamWaitEvent(s, c->ev_join, 0));

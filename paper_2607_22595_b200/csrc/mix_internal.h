@@ -229,6 +229,7 @@ cudaError_t launch_select(const Ctx* c, bool flagged_only, cudaStream_t s);
 cudaError_t launch_decode(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s);         // rows without the error term
 cudaError_t launch_decode_delta(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s);   // rows with it
 cudaError_t launch_edit_only(const Ctx* c, __nv_bfloat16* hidden, int T, cudaStream_t s);
+cudaError_t launch_edit_only_delta(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s);   // decode_delta_kernel on the shortcut's token-indexed records
 cudaError_t edit_only_prepare();   // opt in to the dynamic shared memory of the edit-only kernel
 cudaError_t launch_compose_map(const Ctx* c, int T_live, int n_req, cudaStream_t s);
 cudaError_t launch_fold_bias(const __nv_bfloat16* W_enc, const float* b_enc, const float* b_dec, float* b_eff,

@@ -1017,7 +1017,10 @@ cudaError_t launch_edit_only(const Ctx* c, __nv_bfloat16* hidden, int T, cudaStr
                              hidden, c->cfg.d_model, c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates, c->cfg.n_slots_max,
                              c->d_groups, c->cfg.n_groups_max, c->d_edit_idx, c->d_edit_val, c->d_edit_mode, c->cfg.r_max,
                              c->d_eo_row_delta, c->d_eo_coef, c->cfg.T_max);
-  if (e != cudaSuccess) return e;
+  return e;
+}
+
+cudaError_t launch_edit_only_delta(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s) {
   dim3 grid((unsigned)((c->cfg.T_max + kDdRows - 1) / kDdRows), (unsigned)((c->cfg.d_model / 8 + kDdThreads - 1) / kDdThreads));
   return launch_pdl(kPdlTail, decode_delta_kernel, dim3(grid), dim3(kDdThreads), 0, s, hidden, c->cfg.d_model,
                     static_cast<const int*>(nullptr), c->d_route, c->d_eo_row_delta, c->d_eo_coef, c->d_edit_idx, c->cfg.r_max,
