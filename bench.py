@@ -214,8 +214,9 @@ def time_stages(m, fn, reps=5):
     return dict(zip(m.STAGES[:n], best))
 
 
-def extras_sae(name, w, peaks, mixlib, extra_flags=0, w_enc_bytes_per_el=2.0):
-    """SAE-carrying config: per-kernel times, encode flop rate and weight-stream bandwidth."""
+def extras_sae(name, w, peaks, mixlib, extra_flags=0, w_enc_bytes_per_el=2.0, conditional=False):
+    """SAE-carrying config: per-kernel times, encode flop rate and weight-stream bandwidth.
+    conditional: the graph is captured with mix_apply_conditional (the SAE chain under a graph IF node)."""
     m = W.make_context(mixlib.Mix, w, flags=SAE_FLAGS | extra_flags)
     h = w.hidden.clone()
     scores = torch.zeros((w.T_max, max(w.C_max, 1)), dtype=torch.float32, device="cuda")
@@ -232,7 +233,7 @@ def extras_sae(name, w, peaks, mixlib, extra_flags=0, w_enc_bytes_per_el=2.0):
         m.apply(h, scores, stream=s)
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g, stream=s):
-            m.apply(h, scores, stream=s)
+            (m.apply_conditional if conditional else m.apply)(h, scores, stream=s)
     torch.cuda.current_stream().wait_stream(s)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     times = []
@@ -769,6 +770,12 @@ def run_mix(args, rank, world, local_rank):
                             "per row instead); an algorithmic shortcut, not counted toward any tensor-pipe fraction",
                     "t_call_ms_graph": eo["t_call_ms_graph"], "stage_ms": eo["stage_ms"],
                     "token_rows_per_s": eo["token_rows_per_s"], "status": eo["status"]}
+                eoc = extras_sae("mixed (config 3), edit-only shortcut, conditional graph", wm, peaks, mixlib, extra_flags=8,
+                                 conditional=True)
+                ex["mixed_edit_only_shortcut"]["t_call_ms_graph_with_mix_apply_conditional"] = eoc["t_call_ms_graph"]
+                ex["mixed_edit_only_shortcut"]["note_conditional"] = (
+                    "every SAE row takes the shortcut here, so the packed panel is empty and the graph IF node of "
+                    "mix_apply_conditional skips the seven kernels of the SAE chain")
                 del wm
                 torch.cuda.empty_cache()
                 # opt-in 8-bit encoder: with the bf16 hidden state kept exact (two E4M3 operands per row), and with the
