@@ -441,6 +441,8 @@ def run_workload(args):
                          W.make_sae_heavy("cuda", d_sae=16384, T=256, R=16, G=2), peaks, mixlib)
     elif name == "mixed":
         out = extras_sae("mixed (config 3)", W.make_mixed("cuda"), peaks, mixlib)
+    elif name == "mixed_edit_only":   # config 3 with MIX_FLAG_SAE_EDIT_ONLY (an algorithmic shortcut, never a tensor-pipe figure)
+        out = extras_sae("mixed (config 3), edit-only shortcut", W.make_mixed("cuda"), peaks, mixlib, extra_flags=8)
     elif name == "mixed_small":   # profiling case for the tensor-bound regime
         out = extras_sae("mixed_small (d=5120, d_sae=8192, T=4096)",
                          W.make_mixed("cuda", T=4096, d_sae=8192, R=32), peaks, mixlib)
@@ -808,7 +810,7 @@ def main():
     ap.add_argument("--no-retile", action="store_true",
                     help="SAE contexts stream W_enc as registered instead of a tile-contiguous copy (MIX_FLAG_RETILE_W_ENC)")
     ap.add_argument("--workload", default="decode",
-                    help="decode (the contract line) | sweep | sae_heavy | sae_heavy_fp8 | sae_heavy_fp8a | sae_small | sae_small_fp8 | sae_small_fp8a | mixed | mixed_fp8 | mixed_fp8a | mixed_small | mixed_small_fp8a | conditional | conditional_small | replay_fp8 | replay_fp8a | multiclass | multiclass_small | replay")
+                    help="decode (the contract line) | sweep | sae_heavy | sae_heavy_fp8 | sae_heavy_fp8a | sae_small | sae_small_fp8 | sae_small_fp8a | mixed | mixed_fp8 | mixed_fp8a | mixed_edit_only | mixed_small | mixed_small_fp8a | conditional | conditional_small | replay_fp8 | replay_fp8a | multiclass | multiclass_small | replay")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     args = ap.parse_args()
     if args.no_retile:
