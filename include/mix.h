@@ -212,6 +212,9 @@ typedef struct {
 
 /* Create a context on the CURRENT CUDA device and allocate every table and workspace the
    hook will ever need (the only allocating call besides registration of a centred SAE).
+   (Paper, Section 4.2 "State and dataflow": an app's state -- parameters, buffers -- is set up ahead
+   of time and lives on the device; "CUDA-graph-safe kernel design": the static part of the launch
+   structure is fixed once, here, at the capture size T_max.)
    Workspace: a bf16 panel of (T_max + 128*n_groups_max) x d and an fp32 pre-activation
    scratch of the same rows x d_sae_max, when n_groups_max > 0.
    Errors: INVALID_ARG (NULL, non-positive sizes), UNSUPPORTED (d_model % 64, d_sae_max % 256,
@@ -225,8 +228,12 @@ int mix_destroy(mix_ctx* ctx);
 const char* mix_last_error(const mix_ctx* ctx);
 
 /* Register / replace SAE weight set `group` (stream-ordered table write).  Not captured.
+   Replacing a set while SAE apps are attached to it is allowed as long as the new d_sae still
+   covers every feature those apps edit; otherwise the call fails and changes nothing (unregister
+   the apps or give them new edit lists first).
    Errors: OUT_OF_RANGE (group, d_sae > d_sae_max, k), UNSUPPORTED (d_sae % 256), INVALID_ARG
-   (NULL or pointers not 16-byte aligned, JumpReLU without theta, centring without b_dec). */
+   (NULL or pointers not 16-byte aligned, JumpReLU without theta, centring without b_dec, a
+   replacement too narrow for an attached app's edits). */
 int mix_register_sae_weights(mix_ctx* ctx, int group, const mix_sae_weights* w, void* stream);
 int mix_unregister_sae_weights(mix_ctx* ctx, int group, void* stream);
 
@@ -242,7 +249,8 @@ int mix_register_app(mix_ctx* ctx, int slot, int kind, const void* desc, void* s
 int mix_unregister_app(mix_ctx* ctx, int slot, void* stream);
 
 /* Cheap toggles that never touch launch structure (Section 4.2 "Toggling semantics").
-   mix_update_steer_alpha also sets beta of a MIX_PROJECT app. */
+   mix_update_steer_alpha also sets beta of a MIX_PROJECT app.  mix_update_sae_edits validates the
+   whole list first: a call that fails has changed nothing, on the host or on the device. */
 int mix_update_steer_alpha(mix_ctx* ctx, int slot, float alpha, void* stream);
 int mix_update_sae_edits(mix_ctx* ctx, int slot, int n_edit, const int* idx, const float* val,
                          const unsigned char* mode, void* stream);
@@ -282,19 +290,26 @@ int mix_set_gate(mix_ctx* ctx, int slot, const float* scores, int row_stride, in
    there; a cycle; a chain longer than 4; class columns beyond C_max), OUT_OF_RANGE (slot ids). */
 int mix_set_chain(mix_ctx* ctx, int slot, int next_slot, void* stream);
 
-/* Install the token->slot map for the next mix_apply calls: token_slot int32[T_live]
+/* (Paper, Section 4.2 "Toggling semantics" and "Graph-level toggling and continuous batching":
+   which requests of the running batch an app is active for is per-request data that changes from
+   step to step while the captured launch structure stays as it is.)
+   Install the token->slot map for the next mix_apply calls: token_slot int32[T_live]
    (host if src_is_device == 0, else device), -1 = no app.  Rows >= T_live are pass-through.
    One async copy + a 4-byte store into fixed device buffers; never captured in a graph.
    A host source must stay valid until the stream reaches the copy (use pinned memory for a
    truly asynchronous copy).  Errors: OUT_OF_RANGE (T_live < 0 or > T_max). */
 int mix_set_slot_map(mix_ctx* ctx, const int* token_slot, int T_live, int src_is_device, void* stream);
 
-/* Two-level form: slot of token t = req_slot[token_req[t]] (token_req < 0 or >= n_req -> -1),
-   composed on the device.  Both arrays host or both device. */
+/* Two-level form of the same map (Section 4.2 "Toggling semantics": activation is per REQUEST; a
+   continuous-batching engine already holds token -> request): slot of token t =
+   req_slot[token_req[t]] (token_req < 0 or >= n_req -> -1), composed on the device.  Both arrays
+   host or both device. */
 int mix_set_request_map(mix_ctx* ctx, const int* token_req, int T_live, const int* req_slot, int n_req,
                         int src_is_device, void* stream);
 
-/* Optional feature read-out (device buffers, NULL = off): topk_idx int32 [T_max, k_max] and
+/* Optional feature read-out (Section 3 "Read" applied to SAE features; Section 4.2 "State and
+   dataflow": values read at a hook go to buffers the app owns) (device buffers, NULL = off):
+   topk_idx int32 [T_max, k_max] and
    topk_val fp32 [T_max, k_max] receive, for every TopK-SAE row, the selected feature ids
    in order of decreasing pre-activation (ties: lower id first) and those pre-activations
    (before ReLU and before edits); entries k..k_max-1 and other rows are not written.
@@ -303,7 +318,10 @@ int mix_set_request_map(mix_ctx* ctx, const int* token_req, int T_live, const in
    pointers it was captured with. */
 int mix_set_feature_out(mix_ctx* ctx, int* topk_idx, float* topk_val, int* n_active);
 
-/* Apply the hook.  hidden: device bf16 [T_max, d], modified in place.  T: number of rows of
+/* Apply the hook (Section 4.2 "Executable units": the functions attached at a hook run as GPU
+   kernels on the hidden states that pass it; Section 3: read, write, conditional write; "CUDA-
+   graph-safe kernel design": capturable, nothing about a request is baked into the launch).
+   hidden: device bf16 [T_max, d], modified in place.  T: number of rows of
    `hidden` that may be live (<= T_max; rows >= min(T, T_live) are pass-through).  scores_out:
    device fp32 [T_max, C_max] or NULL; only the first n_classes entries of probe rows are
    written.  Enqueues kernels on `stream` (when the context has SAE weight sets, the probe /
@@ -347,7 +365,9 @@ int mix_apply_conditional(mix_ctx* ctx, void* hidden, int T, float* scores_out, 
 int mix_apply_router(mix_ctx* ctx, float* logits, int n_experts, int T, void* stream);
 
 /* Copy the device status word (bits MIX_STATUS_*) to *bits and clear it on the device.
-   Synchronises `stream`. */
+   Synchronises `stream`.  (Section 4.2 "CUDA-graph-safe kernel design" rules out a host check in
+   the middle of a replayed graph: device-side problems are therefore recorded in a word the host
+   reads when it chooses to, never raised as a fault.) */
 int mix_get_status(mix_ctx* ctx, unsigned* bits, void* stream);
 
 /* Number of kernels one mix_apply() call launches on this context (fixed at mix_create):
@@ -429,7 +449,13 @@ int mix_debug_workspace(mix_ctx* ctx, const int** panel_rows, const float** z, l
  * independent, but two calls that overlap on the GPU (different streams, or different host
  * threads) race on it -- serialise them.  The first call on each device looks up the
  * array's device address (no allocation); make that first call before any stream capture
- * begins.  Enqueues on `stream` and returns; results are ready when the stream reaches them. */
+ * begins.  The look-up stores one pointer per device without a lock: two host threads whose
+ * first calls on one device coincide both store the same value, which is harmless, but the
+ * calls themselves still race on the array as said above.  `w`, `app` and the edit arrays are
+ * read before the call returns and reach the GPU as kernel arguments; no host memory of the
+ * caller is referenced afterwards.  Enqueues on `stream` and returns; results are ready when
+ * the stream reaches them.  The path has no status word the caller could read: every argument
+ * that could raise a device-side status bit is rejected on the host instead. */
 #define MIX_STATIC_MAX_ROWS 128
 #define MIX_STATIC_MAX_D_MODEL 4096
 #define MIX_STATIC_MAX_D_SAE 8192

@@ -92,7 +92,7 @@ void free_all(mix_ctx* c) {
   if (c->owned_w_tiled)
     for (int g = 0; g < c->cfg.n_groups_max; ++g) cudaFree(c->owned_w_tiled[g]);
   free(c->owned_w_tiled);
-  free(c->owned_b_eff); free(c->h_apps); free(c->h_groups); free(c->h_chain_next);
+  free(c->owned_b_eff); free(c->h_apps); free(c->h_groups); free(c->h_chain_next); free(c->h_edit_idx);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->ev_join) cudaEventDestroy(c->ev_join);
   if (c->side_stream) cudaStreamDestroy(c->side_stream);
@@ -114,8 +114,8 @@ int publish_app(mix_ctx* c, int slot, cudaStream_t s) {
   return MIX_OK;
 }
 
-int upload_edits(mix_ctx* c, int slot, int group, int n_edit, const int* idx, const float* val,
-                 const unsigned char* mode, cudaStream_t s) {
+// Range and mode checks of an edit list against weight set `group`; changes nothing.
+int check_edits(mix_ctx* c, int group, int n_edit, const int* idx, const float* val, const unsigned char* mode) {
   if (n_edit < 0 || n_edit > c->cfg.r_max) MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "n_edit %d outside [0, r_max=%d]", n_edit, c->cfg.r_max);
   if (n_edit > 0 && (!idx || !val || !mode)) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "edit arrays are NULL");
   const long long S = c->h_groups[group].d_sae;
@@ -123,8 +123,15 @@ int upload_edits(mix_ctx* c, int slot, int group, int n_edit, const int* idx, co
     if (idx[e] < 0 || idx[e] >= S) MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "edit %d: feature %d outside [0, %lld)", e, idx[e], S);
     if (mode[e] != MIX_EDIT_CLAMP && mode[e] != MIX_EDIT_ABLATE) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "edit %d: bad mode %d", e, mode[e]);
   }
+  return MIX_OK;
+}
+
+// Copies a checked edit list into the slot's rows of the device tables and into the host mirror of the
+// indices (kept so that a weight set can be replaced only by one that still covers every edited feature).
+int upload_edits(mix_ctx* c, int slot, int n_edit, const int* idx, const float* val, const unsigned char* mode, cudaStream_t s) {
   if (n_edit > 0) {
     const size_t off = (size_t)slot * c->cfg.r_max;
+    memcpy(c->h_edit_idx + off, idx, n_edit * sizeof(int));
     MIX_CUDA(c, cudaMemcpyAsync(c->d_edit_idx + off, idx, n_edit * sizeof(int), cudaMemcpyHostToDevice, s));
     MIX_CUDA(c, cudaMemcpyAsync(c->d_edit_val + off, val, n_edit * sizeof(float), cudaMemcpyHostToDevice, s));
     MIX_CUDA(c, cudaMemcpyAsync(c->d_edit_mode + off, mode, n_edit, cudaMemcpyHostToDevice, s));
@@ -221,10 +228,11 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
   c->h_apps = static_cast<AppEntry*>(calloc(NS, sizeof(AppEntry)));
   c->h_groups = static_cast<GroupEntry*>(calloc(G > 0 ? G : 1, sizeof(GroupEntry)));
   c->h_chain_next = static_cast<int*>(malloc(NS * sizeof(int)));
+  c->h_edit_idx = static_cast<int*>(calloc((size_t)NS * c->cfg.r_max, sizeof(int)));
   if (c->h_chain_next) memset(c->h_chain_next, 0xff, NS * sizeof(int));
   c->owned_b_eff = static_cast<float**>(calloc(G > 0 ? G : 1, sizeof(float*)));
   c->owned_w_tiled = static_cast<__nv_bfloat16**>(calloc(G > 0 ? G : 1, sizeof(__nv_bfloat16*)));
-  if (!c->h_apps || !c->h_groups || !c->h_chain_next || !c->owned_b_eff || !c->owned_w_tiled) { free_all(c); free(c); return MIX_ERR_NO_MEMORY; }
+  if (!c->h_apps || !c->h_groups || !c->h_chain_next || !c->h_edit_idx || !c->owned_b_eff || !c->owned_w_tiled) { free_all(c); free(c); return MIX_ERR_NO_MEMORY; }
   bool ok = true;
   ok = ok && dev_alloc(&c->d_token_slot, T) == cudaSuccess;
   ok = ok && dev_alloc(&c->d_n_live, 1) == cudaSuccess;
@@ -350,6 +358,16 @@ int mix_register_sae_weights(mix_ctx* c, int group, const mix_sae_weights* w, vo
   const bool fp8 = (c->cfg.flags & MIX_FLAG_FP8_W_ENC) != 0;
   if (fp8 && (!w->W_enc_scale || w->center_input))
     MIX_FAIL(c, MIX_ERR_INVALID_ARG, "an 8-bit encoder needs W_enc_scale and does not take center_input");
+  // Replacing a weight set: the edit lists of the apps attached to it were range-checked against the old
+  // d_sae and index W_enc / W_dec rows on the device, so the new set must still cover every edited feature.
+  for (int sl = 0; sl < c->cfg.n_slots_max; ++sl) {
+    const AppEntry& a = c->h_apps[sl];
+    if (!a.valid || (a.kind & kKindMask) != MIX_SAE || a.group != group) continue;
+    for (int e = 0; e < a.n_edit; ++e)
+      if (c->h_edit_idx[(size_t)sl * c->cfg.r_max + e] >= w->d_sae)
+        MIX_FAIL(c, MIX_ERR_INVALID_ARG, "slot %d edits feature %d of weight set %d: the new d_sae %lld does not cover it "
+                 "(unregister the app or change its edits first)", sl, c->h_edit_idx[(size_t)sl * c->cfg.r_max + e], group, w->d_sae);
+  }
 
   GroupEntry ge;
   memset(&ge, 0, sizeof(ge));
@@ -470,7 +488,8 @@ int mix_register_app(mix_ctx* c, int slot, int kind, const void* desc, void* str
     const mix_sae_app* p = static_cast<const mix_sae_app*>(desc);
     if (p->group < 0 || p->group >= c->cfg.n_groups_max || !c->h_groups[p->group].valid)
       MIX_FAIL(c, MIX_ERR_OUT_OF_RANGE, "SAE weight set %d is not registered", p->group);
-    rc = upload_edits(c, slot, p->group, p->n_edit, p->idx, p->val, p->mode, s);
+    rc = check_edits(c, p->group, p->n_edit, p->idx, p->val, p->mode);
+    if (rc == MIX_OK) rc = upload_edits(c, slot, p->n_edit, p->idx, p->val, p->mode, s);
     if (rc != MIX_OK) return rc;
     e.group = p->group;
     e.n_edit = p->n_edit;
@@ -592,11 +611,14 @@ int mix_update_sae_edits(mix_ctx* c, int slot, int n_edit, const int* idx, const
   int rc = check_slot(c, slot);
   if (rc != MIX_OK) return rc;
   if (!c->h_apps[slot].valid || (c->h_apps[slot].kind & kKindMask) != MIX_SAE) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "slot %d is not an SAE app", slot);
+  // validate before anything is enqueued: a failed call changes nothing, on the host or on the device
+  rc = check_edits(c, c->h_apps[slot].group, n_edit, idx, val, mode);
+  if (rc != MIX_OK) return rc;
   // shrink first, grow last, so a concurrent reader never sees a count beyond valid entries
   const int old_n = c->h_apps[slot].n_edit;
-  if (n_edit < old_n && n_edit >= 0)
+  if (n_edit < old_n)
     MIX_CUDA(c, cudaMemcpyAsync(&c->d_apps[slot].n_edit, &n_edit, sizeof(int), cudaMemcpyHostToDevice, s));
-  rc = upload_edits(c, slot, c->h_apps[slot].group, n_edit, idx, val, mode, s);
+  rc = upload_edits(c, slot, n_edit, idx, val, mode, s);
   if (rc != MIX_OK) return rc;
   c->h_apps[slot].n_edit = n_edit;
   MIX_CUDA(c, cudaMemcpyAsync(&c->d_apps[slot].n_edit, &n_edit, sizeof(int), cudaMemcpyHostToDevice, s));

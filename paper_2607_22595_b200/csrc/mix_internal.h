@@ -102,6 +102,7 @@ struct Ctx {
   GateEntry* d_gates;       // [n_slots_max]
   int* d_chain_next;        // [n_slots_max] next slot applied to the same row, or -1 (MIX_FLAG_SLOT_CHAINS)
   int* h_chain_next;        // host mirror
+  int* h_edit_idx;          // host mirror of d_edit_idx (validation when a weight set is replaced)
   __nv_bfloat16* d_vec_arena;   // [n_slots_max, d] copies of single-vector weights (T_max <= kTeamMaxRows), else null
   int* d_edit_idx;          // [n_slots_max * r_max]
   float* d_edit_val;

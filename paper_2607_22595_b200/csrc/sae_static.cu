@@ -55,6 +55,40 @@ static __device__ __align__(256) unsigned char g_static_scratch[kScratchBytes];
 constexpr int kMaxDevices = 64;
 unsigned char* g_scratch_addr[kMaxDevices];     // device address of the array, per device, once resolved
 
+// Everything the call's tables need, passed to the set-up kernel BY VALUE (well under the 4 KiB of kernel
+// parameters): no host pointer is handed to the stream, so nothing the stream does later depends on the
+// caller's stack or on the caller's edit arrays staying alive.
+struct StaticSetup {
+  int n_rows;
+  int n_edit;
+  AppEntry app;
+  GroupEntry group;
+  int edit_idx[kMaxEdits];
+  float edit_val[kMaxEdits];
+  unsigned char edit_mode[kMaxEdits];
+};
+
+// Rewrites every table of the scratch array that this call's kernels read before writing.
+__global__ void __launch_bounds__(128)
+static_setup_kernel(const StaticSetup su, int* __restrict__ token_slot, int* __restrict__ n_live,
+                    unsigned* __restrict__ status, AppEntry* __restrict__ app, GroupEntry* __restrict__ group,
+                    int* __restrict__ edit_idx, float* __restrict__ edit_val, unsigned char* __restrict__ edit_mode) {
+  const int tid = threadIdx.x;
+  if (tid < su.n_rows) token_slot[tid] = 0;             // every row -> slot 0 (n_rows <= 128 = blockDim.x)
+  if (tid < su.n_edit) {
+    edit_idx[tid] = su.edit_idx[tid];
+    edit_val[tid] = su.edit_val[tid];
+    edit_mode[tid] = su.edit_mode[tid];
+  }
+  if (tid == 0) {
+    *n_live = su.n_rows;
+    *status = 0u;
+    *app = su.app;
+    *group = su.group;
+  }
+}
+static_assert(kStaticRows <= 128 && kMaxEdits <= 128, "one thread per row / per edit entry in the set-up kernel");
+
 int fail(char* errbuf, int errbuf_len, int code, const char* fmt, long long a = 0, long long b = 0) {
   if (errbuf && errbuf_len > 0) snprintf(errbuf, (size_t)errbuf_len, fmt, a, b);
   return code;
@@ -167,19 +201,23 @@ extern "C" int mix_sae_apply_static(void* hidden, int n_rows, int d_model, const
   ge.W_dec = static_cast<const __nv_bfloat16*>(w->W_dec);
   ge.b_dec = w->b_dec;
 
-  // The array keeps whatever the previous call left: rewrite every table this call reads.
-  // (Routing rewrites the row lists and counters itself; the panel, Z and TopK lists are
-  // fully rewritten for the rows in use before they are read.)
-  cudaError_t e = cudaMemsetAsync(c.d_token_slot, 0, (size_t)n_rows * sizeof(int), s);   // every row -> slot 0
-  if (e == cudaSuccess) e = cudaMemcpyAsync(c.d_n_live, &n_rows, sizeof(int), cudaMemcpyHostToDevice, s);
-  if (e == cudaSuccess) e = cudaMemsetAsync(c.d_status, 0, sizeof(unsigned), s);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(c.d_apps, &ae, sizeof(ae), cudaMemcpyHostToDevice, s);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(c.d_groups, &ge, sizeof(ge), cudaMemcpyHostToDevice, s);
-  if (e == cudaSuccess && app->n_edit > 0) {
-    e = cudaMemcpyAsync(c.d_edit_idx, app->idx, app->n_edit * sizeof(int), cudaMemcpyHostToDevice, s);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(c.d_edit_val, app->val, app->n_edit * sizeof(float), cudaMemcpyHostToDevice, s);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(c.d_edit_mode, app->mode, (size_t)app->n_edit, cudaMemcpyHostToDevice, s);
+  // The array keeps whatever the previous call left: one small kernel rewrites every table this call reads,
+  // from values it received as kernel parameters.  (Routing rewrites the row lists and counters itself; the
+  // panel, Z and TopK lists are fully rewritten for the rows in use before they are read.)
+  StaticSetup su;
+  memset(&su, 0, sizeof(su));
+  su.n_rows = n_rows;
+  su.n_edit = app->n_edit;
+  su.app = ae;
+  su.group = ge;
+  for (int i = 0; i < app->n_edit; ++i) {
+    su.edit_idx[i] = app->idx[i];
+    su.edit_val[i] = app->val[i];
+    su.edit_mode[i] = app->mode[i];
   }
+  static_setup_kernel<<<1, 128, 0, s>>>(su, c.d_token_slot, c.d_n_live, c.d_status, c.d_apps, c.d_groups, c.d_edit_idx,
+                                        c.d_edit_val, c.d_edit_mode);
+  cudaError_t e = cudaGetLastError();
   __nv_bfloat16* h = static_cast<__nv_bfloat16*>(hidden);
   if (e == cudaSuccess) e = launch_route(&c, n_rows, s);
   if (e == cudaSuccess) e = launch_pack(&c, h, s);

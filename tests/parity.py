@@ -18,6 +18,14 @@ SCORE_RTOL = 1e-3
 LOGIT_ACC_TOL = 4e-6        # ~64 fp32 unit roundoffs (2^-24) of sum |w_i h_i|: raw logits only, see check_parity
 HIDDEN_TOL_FRAC = 1e-2
 TOPK_TIE_TOL = 1e-3
+# Beside the mandated bound above, every written element is held to a TIGHT bound (tight_bound below):
+#   1 bf16 ulp at max(|y_i|, |h_i|)  +  the fp32 accumulation allowance of the sums that feed it.
+# The first term is the final rounding to bf16 (half an ulp) with room for a rounding decision taken on a value
+# perturbed by the second; taking the ulp at max(|y_i|, |h_i|) rather than at |y_i| alone covers elements where
+# h_i and the update cancel.  The second term bounds what fp32 accumulation (tensor core or FMA chain) can move:
+# LOGIT_ACC_TOL * sum|w_i x_i| per pre-activation or dot product, carried through the coefficient it enters, and
+# (n + 2) * 2^-24 * sum|terms| for an n-term fp32 sum.
+THRESHOLD_SLACK = 1e-4      # a ReLU / JumpReLU pre-activation this close to its threshold may fall either way in fp32
 CANARY_F32 = np.uint32(0x7FC0DEAD)          # a NaN payload nobody computes
 CANARY_I32 = np.int32(-559038737)
 
@@ -67,6 +75,53 @@ def bf16_ulp(x):
     return 2.0 ** (np.floor(np.log2(a)) - 7)
 
 
+def tight_bound(wh, t, ref, K_override=None):
+    """Per-element bound on |gpu - oracle| for a written row (see the header), or None where it does not apply:
+    8-bit encoders (their own error model), rows where a pre-activation that decides a coefficient lies within
+    THRESHOLD_SLACK of its JumpReLU threshold (the step there is not a rounding effect), very wide supports."""
+    kind = ref.kind[t]
+    app = wh.apps[int(wh.token_slot[t])]
+    h = O.bf16_to_f64(wh.hidden[t])
+    y = ref.y[t]
+    eps = 2.0 ** -24
+    if kind == O.KIND_STEER:
+        return bf16_ulp(np.maximum(np.abs(y), np.abs(h))) + 2 * eps * (np.abs(h) + np.abs(y))
+    if kind == O.KIND_PROJECT:
+        r = np.abs(O.bf16_to_f64(app.r))
+        return bf16_ulp(np.maximum(np.abs(y), np.abs(h))) + LOGIT_ACC_TOL * abs(app.beta) * float(np.abs(h) @ r) * r + \
+            2 * eps * (np.abs(h) + np.abs(y))
+    if kind != O.KIND_SAE or t not in ref.z:
+        return None
+    sae = wh.groups[app.group]
+    if getattr(sae, "w_scale", None) is not None or getattr(wh, "fp8_act", False):
+        return None
+    z = ref.z[t]
+    f, _ = O.sae_activate(z, sae.act, sae.k, sae.theta, K_override)
+    f2 = O.sae_edit(f, app.edit_idx, app.edit_val, app.edit_mode)
+    if app.add_error:
+        F = np.unique(np.asarray(app.edit_idx, dtype=np.int64))
+        coef = f2[F] - f[F]
+        base = np.abs(h)
+    else:
+        F = np.nonzero((f2 != 0) | (f != 0))[0]
+        coef = f2[F]
+        base = np.zeros_like(h) if sae.b_dec is None else np.abs(np.asarray(sae.b_dec, dtype=np.float64))
+    if len(F) > 4096:
+        return None
+    if sae.act == O.SAE_JUMPRELU:
+        watch = F if app.add_error else np.arange(len(z))
+        if (np.abs(z[watch] - np.asarray(sae.theta, dtype=np.float64)[watch]) <= THRESHOLD_SLACK).any():
+            return None
+    if len(F) == 0:
+        return bf16_ulp(np.maximum(np.abs(y), base)) + 2 * eps * base
+    x_enc = h - np.asarray(sae.b_dec, dtype=np.float64) if (sae.center_input and sae.b_dec is not None) else h
+    Wd = np.abs(O.bf16_to_f64(sae.W_dec[F]))
+    magz = np.abs(O.bf16_to_f64(sae.W_enc[F])) @ np.abs(x_enc) + np.abs(np.asarray(sae.b_enc, dtype=np.float64)[F])
+    acc = LOGIT_ACC_TOL * (magz @ Wd) + (len(F) + 2) * eps * (np.abs(coef) @ Wd + base)
+    at = np.maximum(np.abs(y), np.abs(h)) if app.add_error else np.abs(y)
+    return bf16_ulp(at) + acc
+
+
 def check_parity(wh, out, rows=None, expect_status=0, check_features=True, scale_with_output=False):
     """wh: host workload (numpy); out: run_gpu result.  Asserts parity on `rows` (default all).
     scale_with_output: take the hidden-state bound as 1e-2 * max(|h_in|, |y_ref|) -- for inputs where
@@ -78,7 +133,8 @@ def check_parity(wh, out, rows=None, expect_status=0, check_features=True, scale
     hmax = float(np.abs(O.bf16_to_f64(wh.hidden)).max())
     hid = out["hidden"]
     scores_bits = out["scores"].view(np.uint32)
-    stats = dict(max_score_rel=0.0, max_hidden_err=0.0, max_hidden_ulp=0.0, topk_swaps=0, rows=len(rows))
+    stats = dict(max_score_rel=0.0, max_hidden_err=0.0, max_hidden_ulp=0.0, topk_swaps=0, rows=len(rows), tight_rows=0,
+                 max_tight_frac=0.0)
     redo = {}
     for t in rows:
         kind = ref.kind[t]
@@ -136,14 +192,21 @@ def check_parity(wh, out, rows=None, expect_status=0, check_features=True, scale
                 t, kind, err.max(), HIDDEN_TOL_FRAC * hmax)
             stats["max_hidden_err"] = max(stats["max_hidden_err"], float(err.max()))
             stats["max_hidden_ulp"] = max(stats["max_hidden_ulp"], float((err / bf16_ulp(ref.y[t])).max()))
+            bound = tight_bound(wh, t, ref, redo.get(t))
+            if bound is not None:
+                worst = int(np.argmax(err - bound))
+                assert (err <= bound).all(), "row %d (kind %d) element %d off by %g: tight bound %g (1 bf16 ulp + fp32 accumulation)" % (
+                    t, kind, worst, err[worst], bound[worst])
+                stats["tight_rows"] += 1
+                stats["max_tight_frac"] = max(stats["max_tight_frac"], float((err / bound).max()))
         if kind == O.KIND_SAE and check_features:
             na = int(out["n_active"][t])
             if t in ref.topk:
                 assert na == ref.n_active[t], "row %d n_active %d != %d" % (t, na, ref.n_active[t])
-            else:   # ReLU / JumpReLU: entries within 1e-4 of their threshold may fall either way
+            else:   # ReLU / JumpReLU: entries within THRESHOLD_SLACK of their threshold may fall either way
                 sae = wh.groups[wh.apps[int(wh.token_slot[t])].group]
                 thr = np.zeros_like(ref.z[t]) if sae.theta is None else np.maximum(sae.theta.astype(np.float64), 0)
-                slack = int((np.abs(ref.z[t] - thr) <= 1e-4).sum())
+                slack = int((np.abs(ref.z[t] - thr) <= THRESHOLD_SLACK).sum())
                 assert abs(na - ref.n_active[t]) <= slack, "row %d n_active %d vs %d" % (t, na, ref.n_active[t])
         elif check_features:
             assert int(out["n_active"][t]) == int(CANARY_I32)

@@ -417,6 +417,38 @@ def test_api_error_codes():
     m.destroy()
 
 
+def test_replacing_a_weight_set_and_failed_edit_updates_change_nothing():
+    """A weight set may be replaced under attached apps only if the new width still covers their edited
+    features (the device indexes W_enc / W_dec rows with them), and an edit update that fails validation
+    leaves the app exactly as it was.  API checks only: no call here reaches a kernel with a bad index."""
+    mixlib = _mixlib()
+    d, S = 128, 512
+    g = torch.Generator(device=DEV); g.manual_seed(5)
+    sae = W.make_sae_weights(g, DEV, d, S, W.SAE_TOPK, k=4)
+    hidden = torch.randn((8, d), generator=g, device=DEV, dtype=torch.float32).to(torch.bfloat16)
+    m = mixlib.Mix(d_model=d, T_max=8, n_slots_max=2, n_groups_max=1, C_max=1, k_max=4, r_max=4, d_sae_max=S)
+    m.register_sae_weights(0, S, sae.act, sae.k, sae.W_enc, sae.b_enc, sae.W_dec)
+    m.register_sae_app(0, 0, [3, 300], [2.0, 0.0], [0, 1], True)
+    with pytest.raises(mixlib.MixError) as e:           # 256 features no longer cover feature 300
+        m.register_sae_weights(0, 256, sae.act, sae.k, sae.W_enc, sae.b_enc, sae.W_dec)
+    assert e.value.code == -1 and "300" in str(e.value)
+    m.set_slot_map(np.zeros(8, dtype=np.int32))
+    h1 = hidden.clone(); m.apply(h1); torch.cuda.synchronize()
+    with pytest.raises(mixlib.MixError) as e:           # second entry out of range: nothing may change
+        m.update_sae_edits(0, [5, 512], [1.0, 1.0], [0, 0])
+    assert e.value.code == -2
+    with pytest.raises(mixlib.MixError) as e:
+        m.update_sae_edits(0, [5], [1.0], [7])          # bad mode, shorter list: the count must not shrink
+    assert e.value.code == -1
+    h2 = hidden.clone(); m.apply(h2); torch.cuda.synchronize()
+    assert torch.equal(h1, h2) and not torch.equal(h1, hidden)
+    m.update_sae_edits(0, [3], [2.0], [0])              # feature 300 is gone from the list ...
+    m.register_sae_weights(0, 256, sae.act, sae.k, sae.W_enc, sae.b_enc, sae.W_dec)   # ... so the narrower set fits
+    h3 = hidden.clone(); m.apply(h3); torch.cuda.synchronize()
+    assert m.get_status() == 0
+    m.destroy()
+
+
 # ------------------------------------------------------------------ full-size configs, sampled rows
 def test_sae_heavy_full_size_sampled_rows():
     w = W.make_sae_heavy(DEV, edit_hint=oracle_edit_hint)

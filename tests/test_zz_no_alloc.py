@@ -3,9 +3,10 @@
 mix_sae_apply_static() serves callers that are not allowed to allocate device memory (a
 plugin inside a serving engine that owns all of HBM, a latency-critical path that cannot
 afford cudaMalloc's implicit synchronisation).  Its scratch is one fixed array inside the
-library, shared by all calls and never cleared between them, so the test makes two different
-calls in a row and checks each against mix_apply() on an ordinary context given the same
-inputs.  This file sorts last on purpose: a run that stops at the first failure has then
+library, shared by all calls and never cleared between them, so the test makes different calls in
+a row (a large one, a small one of another kind, a large one again) and checks each against
+mix_apply() on an ordinary context given the same inputs and, row by row, against the float64
+oracle.  This file sorts last on purpose: a run that stops at the first failure has then
 already run every other test.
 """
 import numpy as np
@@ -15,7 +16,7 @@ import torch
 import workloads as W
 from oracle import mi_hook as O
 
-from parity import HIDDEN_TOL_FRAC
+from parity import CANARY_F32, HIDDEN_TOL_FRAC, check_parity
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -61,6 +62,23 @@ def _via_static(mixlib, sae, hidden, edits, add_error):
     return h, ti, tv
 
 
+def _oracle_check(case, out):
+    """Every row of one static call against the float64 oracle: hidden state and, for TopK, ids and values."""
+    sae, hidden, edits, add_error = case
+    h_s, ti_s, tv_s = out
+    n = hidden.shape[0]
+    app = W.SaeApp(0, *edits, add_error)
+    wl = W.Workload("static", hidden.shape[1], n, n, hidden, np.zeros(n, dtype=np.int32), {0: app}, {0: sae},
+                    n_slots_max=1, n_groups_max=1, C_max=1, k_max=sae.k, r_max=8, d_sae_max=sae.d_sae)
+    wh = W.host(wl)
+    n_act = np.zeros(n, dtype=np.int32)
+    if sae.k:
+        n_act = (tv_s.cpu().numpy() > 0).sum(axis=1).astype(np.int32)    # what mix_apply would report for TopK rows
+    res = dict(hidden=W.bits(h_s), scores=np.full((n, 1), CANARY_F32, dtype=np.uint32).view(np.float32),
+               topk_idx=ti_s.cpu().numpy(), topk_val=tv_s.cpu().numpy(), n_active=n_act, status=0)
+    return check_parity(wh, res, check_features=bool(sae.k))
+
+
 def test_static_entry_point_matches_context_path_on_two_calls_in_a_row():
     import paper_2607_22595_b200 as mixlib
     cases = [
@@ -68,6 +86,8 @@ def test_static_entry_point_matches_context_path_on_two_calls_in_a_row():
         # fewer rows, narrower SAE, other activation, no error term: stale rows, stale TopK
         # lists and a stale edit list from the first call must not show through
         _case(22, 37, 128, 1024, W.SAE_JUMPRELU, 0, ([7], [1.5], [0]), False),
+        # and back to a full tile of rows after the small call, with the longer edit list again
+        _case(24, 128, 256, 2048, W.SAE_TOPK, 16, ([11, 12, 2047, 0, 11], [2.0, 0.0, 4.0, 1.0, 7.0], [0, 1, 0, 0, 0]), False),
     ]
     static_out = [_via_static(mixlib, *c) for c in cases]          # back to back, same scratch
     for c, (h_s, ti_s, tv_s) in zip(cases, static_out):
@@ -80,17 +100,11 @@ def test_static_entry_point_matches_context_path_on_two_calls_in_a_row():
         if sae.k:
             assert torch.equal(ti_s, ti_c)
             assert (tv_s - tv_c).abs().max().item() <= 1e-3
-    # and the static path stands on its own against the oracle (first case, a few rows)
-    sae, hidden, edits, add_error = cases[0]
-    app = W.SaeApp(0, *edits, add_error)
-    wl = W.Workload("static", hidden.shape[1], hidden.shape[0], hidden.shape[0], hidden,
-                    np.zeros(hidden.shape[0], dtype=np.int32), {0: app}, {0: sae}, n_slots_max=1, n_groups_max=1,
-                    C_max=1, k_max=sae.k, r_max=4, d_sae_max=sae.d_sae)
-    ref = O.apply_hook(W.host(wl), rows=[0, 50, 99])
-    got = O.bf16_to_f64(W.bits(static_out[0][0]))
-    hmax = float(hidden.float().abs().max())
-    for t in (0, 50, 99):
-        assert np.abs(got[t] - ref.y[t]).max() <= HIDDEN_TOL_FRAC * hmax
+    # and every call stands on its own against the float64 oracle, on every row (the last row of the short
+    # second call included: the case that exists to catch scratch left over from the first)
+    for c, out in zip(cases, static_out):
+        stats = _oracle_check(c, out)
+        assert stats["rows"] == c[1].shape[0]
 
 
 def test_static_entry_point_rejects_sizes_beyond_its_fixed_scratch():
