@@ -4,10 +4,12 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl mix|reference] [--no-extras]
 
 A step is one mix_apply() over one synthetic decode batch (d = 4096, 256 one-token requests,
-64 probes + 32 steering vectors, 25 % of rows unhooked).  The timed region replays CUDA graphs
-whose nodes are consecutive steps on ROTATING hidden-state buffers (512 MiB in total, four
-times the L2), so every step finds its activations cold in L2; inputs are resident in HBM.
-One JSON line goes to stdout (rank 0).  With N > 1 every rank runs its own replica on its own
+64 probes + 32 steering vectors, 25 % of rows unhooked).  A repeat is EXACTLY K such steps, replayed
+as a CUDA graph on ROTATING hidden-state buffers (>= 512 MiB in total, four times the L2), so every
+step finds its activations cold in L2; inputs are resident in HBM.  The repeat is timed again and
+again (one CUDA event between repeats) until the region is at least 0.35 s long; `ms_per_step` is
+the median repeat time / K, so the figure does not depend on K.  One JSON line goes to stdout
+(rank 0); the roofline fractions of the other configurations are under `roofline.targets`.  With N > 1 every rank runs its own replica on its own
 batch (rows are independent: no collective on the data path), time = max over ranks.
 """
 from __future__ import annotations
@@ -35,9 +37,9 @@ WORKLOAD = "decode: d=4096, T=256 (256 requests x 1 token), 64 probes + 32 steer
 ROTATE_BYTES = 512 << 20
 SAE_FLAGS = 2            # mix_config.flags of the SAE contexts of the extras / --workload runs: MIX_FLAG_RETILE_W_ENC
                          # (tile-contiguous copy of W_enc made at registration); --no-retile streams W_enc as given
-# dram__bytes_read.sum + dram__bytes_write.sum of one probe_steer_team_kernel launch on this workload,
-# from the ncu capture summarised in profiles/probe_steer_kernel_decode.md (reads 2.40 MB, writes 0:
-# the steered rows are still dirty in L2 when the kernel ends).
+# dram__bytes_read.sum + dram__bytes_write.sum of one probe_steer_team_kernel launch on the decode workload, from an
+# ncu capture of this kernel (reads only: the steered rows are still dirty in L2 when the kernel ends).  Reported as
+# `roofline.traffic`, labelled as not re-measured; the fraction itself uses the algorithmic bytes.
 DECODE_DRAM_BYTES_PER_LAUNCH = 2404352
 
 
@@ -158,6 +160,21 @@ def barrier(world):
 
 
 # ------------------------------------------------------------------------------ oracle legs
+def host_threads():
+    """Threads the oracle may use: the process's affinity mask.  numpy's BLAS pool (the oracle's matrix
+    products) is set to exactly that many, so the printed count is the one that ran."""
+    n = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    used = n
+    try:
+        from threadpoolctl import threadpool_info, threadpool_limits
+        threadpool_limits(limits=n)
+        pools = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        used = max(pools) if pools else 1
+    except Exception:
+        pass
+    return n, used
+
+
 def oracle_leg(seconds_target=10.0, max_batches=10000):
     """Time the float64 oracle, as it stands, on whole decode batches for about `seconds_target` s."""
     from oracle import mi_hook as O
@@ -173,12 +190,59 @@ def oracle_leg(seconds_target=10.0, max_batches=10000):
     return dict(rows_per_s=n * wh.T_max / dt, batches=n, seconds=dt, rows=n * wh.T_max)
 
 
+def oracle_sae_sample(w, n_sae_rows=4, n_other_rows=8, seed=0):
+    """The oracle on a bounded sample of an SAE-carrying configuration (tensors on cuda are copied to the host
+    first): `n_sae_rows` SAE rows of weight set 0 -- the oracle converts a whole encoder to float64 for however
+    few rows it is given, so rows/s on a sample UNDERSTATES a full pass -- and a few rows of every other kind."""
+    from oracle import mi_hook as O
+    wh = W.host(w, only_groups={0})
+    rng = np.random.default_rng(seed)
+    sae_rows, other = [], []
+    for t in range(w.T_live):
+        a = w.apps.get(int(w.token_slot[t]))
+        if a is not None and a.kind == W.KIND_SAE and a.group == 0:
+            sae_rows.append(t)
+        elif a is not None and a.kind != W.KIND_SAE:
+            other.append(t)
+    rows = list(rng.choice(sae_rows, size=min(n_sae_rows, len(sae_rows)), replace=False)) if sae_rows else []
+    rows += list(rng.choice(other, size=min(n_other_rows, len(other)), replace=False)) if other else []
+    t0 = time.perf_counter()
+    O.apply_hook(wh, rows)
+    dt = time.perf_counter() - t0
+    n_sae_total = sum(1 for t in range(w.T_live) if (w.apps.get(int(w.token_slot[t])) is not None
+                                                        and w.apps[int(w.token_slot[t])].kind == W.KIND_SAE))
+    return {"rows": len(rows), "sae_rows": min(n_sae_rows, len(sae_rows)), "seconds": dt, "rows_per_s": len(rows) / dt,
+            "extrapolated_full_batch_s": dt / max(len(rows), 1) * w.T_live,
+            "extrapolation": "sample seconds per row x %d live rows (%d of them SAE rows); an upper estimate, the per-weight-set "
+                             "float64 conversion of the encoder is spread over few rows in the sample" % (w.T_live, n_sae_total)}
+
+
+def cpu_baseline_block(seconds_target):
+    """cpu_baseline of the contract line: the oracle on whole decode batches (the line's own workload), plus its
+    time on sampled rows of configs 2 and 3."""
+    avail, used = host_threads()
+    cb = oracle_leg(seconds_target)
+    out = {"value": cb["rows_per_s"], "unit": UNIT, "cores": used, "cores_available": avail, "kind": "oracle",
+           "threads": "numpy BLAS pool set to the affinity mask (%d); the row loop itself is one Python thread" % avail,
+           "sample": "%d whole decode batches (%d rows) in %.1f s" % (cb["batches"], cb["rows"], cb["seconds"])}
+    if torch.cuda.is_available():
+        try:
+            out["cfg2_sae_heavy_sample"] = oracle_sae_sample(W.make_sae_heavy("cuda"), n_sae_rows=4, n_other_rows=0)
+            torch.cuda.empty_cache()
+            out["cfg3_mixed_sample"] = oracle_sae_sample(W.make_mixed("cuda"), n_sae_rows=4, n_other_rows=8)
+            torch.cuda.empty_cache()
+        except Exception as e:
+            out["sae_sample_error"] = repr(e)
+    return out
+
+
 def run_reference(args, rank, world):
     """--impl reference: the oracle on the host cores, same metric and config."""
     if rank != 0:
         return
     steps, warm = args.steps or 20, args.warmup if args.warmup is not None else 3
     from oracle import mi_hook as O
+    avail, used = host_threads()
     wh = W.host(W.make_decode("cpu"))
     for _ in range(max(warm, 1)):
         O.apply_hook(wh)
@@ -189,10 +253,9 @@ def run_reference(args, rank, world):
     val = steps * wh.T_max / dt
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
             "warmup": warm, "ms_per_step": 1e3 * dt / steps, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "note": "float64 CPU oracle, one whole batch per step"},
-            "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle",
-                             "sample": "%d whole decode batches (256 rows each)" % steps},
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": contract_config(),
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": used, "cores_available": avail, "kind": "oracle",
+                             "sample": "%d whole decode batches (256 rows each); float64 CPU oracle, one whole batch per step" % steps},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
@@ -305,7 +368,7 @@ def run_replay(peaks, mixlib, n_replays, fp8a=False, fp8w=False):
         bound_ms = max(wbytes / (peaks["hbm_gbs"] * 1e9),
                        flops / ((2.0 if fp8a else 1.0) * peaks["bf16_tflops"] * 1e12)) * 1e3
         rec.append((n_live, sum(counts.values()), len(counts), ms, bound_ms))
-        if r % 50 == 49 or r == n_replays - 1:
+        if r % 10 == 9 or r == n_replays - 1:
             bad_status |= m.get_status()
     m.destroy()
     a = np.array(rec)
@@ -313,6 +376,10 @@ def run_replay(peaks, mixlib, n_replays, fp8a=False, fp8w=False):
     ratio = live[:, 4] / live[:, 3] if len(live) else np.array([0.0])
     return {"workload": "replay (config 4)" + (", 8-bit encoder and input" if fp8a else (", 8-bit encoder, bf16 rows" if fp8w else "")),
             "replays": n_replays, "status_or": bad_status,
+            "n_live_covered": {"min": int(a[:, 0].min()), "max": int(a[:, 0].max()), "zero": bool((a[:, 0] == 0).any()),
+                               "full": bool((a[:, 0] == T).any())},
+            "below_0p75": [{"n_live": int(x[0]), "sae_rows": int(x[1]), "groups_live": int(x[2]), "ms": float(x[3]),
+                            "bound_ms": float(x[4])} for x in live[np.argsort(ratio)[:8]] if x[4] / x[3] < 0.75],
             "t_call_ms": {"min": float(a[:, 3].min()), "p50": float(np.median(a[:, 3])), "p90": float(np.quantile(a[:, 3], 0.9)),
                           "max": float(a[:, 3].max())},
             "empty_replay_ms": float(a[a[:, 0] == 0][:, 3].min()) if (a[:, 0] == 0).any() else None,
@@ -322,6 +389,35 @@ def run_replay(peaks, mixlib, n_replays, fp8a=False, fp8w=False):
             "worst": {"n_live": int(a[a[:, 3].argmax(), 0]), "sae_rows": int(a[a[:, 3].argmax(), 1]),
                       "groups_live": int(a[a[:, 3].argmax(), 2]), "ms": float(a[:, 3].max()),
                       "bound_ms": float(a[a[:, 3].argmax(), 4])}}
+
+
+def extras_replace_decode(peaks, mixlib, small=False):
+    """The decode as a gather: config 2 with the error term OFF, so every row is rebuilt from b_dec and the k = 64
+    selected plus 16 edited W_dec rows (512 rows x 80 rows x 8 KiB = 320 MiB gathered).  Reported: the decode
+    kernel's time between stage events and the gather's bytes over it.  small: a 4096-wide case for profiling."""
+    w = W.make_sae_heavy("cuda", d_sae=16384, T=256, R=16, G=2) if small else W.make_sae_heavy("cuda", edit_hint=gpu_edit_hint)
+    for a in w.apps.values():
+        a.add_error = False
+    m = W.make_context(mixlib.Mix, w, flags=SAE_FLAGS)
+    h = w.hidden.clone()
+    def fn():
+        h.copy_(w.hidden)
+        m.apply(h)
+    for _ in range(2):
+        fn()
+    torch.cuda.synchronize()
+    st = time_stages(m, fn)
+    key = "tail" if "tail" in st else "decode"
+    n_rows = int(sum(1 for t in range(w.T_live) if w.apps.get(int(w.token_slot[t])) is not None))
+    k = max(sw.k for sw in w.groups.values())
+    nbytes = float(n_rows) * (k + w.r_max) * w.d_model * 2 + float(n_rows) * w.d_model * 2
+    status = m.get_status()
+    m.destroy()
+    return {"what": "config 2 with add_error = 0: %d rows x (k=%d + %d edited) W_dec rows of %d B gathered, row written" % (
+                n_rows, k, w.r_max, w.d_model * 2),
+            "stage": key, "decode_us": st[key] * 1e3, "bytes": nbytes, "gather_gbs": nbytes / st[key] / 1e6,
+            "frac_hbm_peak": nbytes / st[key] / 1e6 / peaks["hbm_gbs"], "stage_ms": st, "status": status,
+            "note": "the merge of the TopK candidates runs in the same kernel when the stage is `tail`"}
 
 
 def extras_conditional(w, mixlib):
@@ -454,6 +550,10 @@ def run_workload(args):
         out = extras_multiclass(peaks, mixlib)
     elif name == "multiclass_small":   # profiling case: 168 MB of hidden state
         out = extras_multiclass(peaks, mixlib, small=True)
+    elif name == "replace_decode":
+        out = extras_replace_decode(peaks, mixlib)
+    elif name == "replace_decode_small":   # profiling case
+        out = extras_replace_decode(peaks, mixlib, small=True)
     elif name == "replay":
         out = run_replay(peaks, mixlib, args.steps or 200)
     elif name == "replay_fp8a":
@@ -587,6 +687,54 @@ def extras_sweep(peaks, mixlib):
 
 
 # ------------------------------------------------------------------------------ main arm
+MIN_REGION_S = 0.35        # the timed region is repeated until it is at least this long
+
+
+def plan_pass(m, hiddens, scores, K, stream):
+    """Graphs whose replay, one after the other, is a whole number of repeats of EXACTLY K consecutive steps on
+    rotating hidden buffers: returns (graphs, repeats per pass).  K <= number of buffers R (a multiple of K): one
+    graph that walks all R buffers = R / K repeats back to back -- a K-step graph launched on its own would add
+    the launch latency of a whole graph to every K steps, which belongs to the engine's graph, not to the hook
+    kernel inside it; this way the per-step figure is the same for every K.  Larger K: the all-buffers graph
+    replayed K // R times plus a remainder graph = one repeat.  Either way a buffer comes round again only after
+    all the others (>= 4x L2) have been touched."""
+    R = len(hiddens)
+    if K <= R:
+        return [capture_steps(m, hiddens, scores, range(R), stream)], R // K
+    graphs = [capture_steps(m, hiddens, scores, range(R), stream)] * (K // R)
+    if K % R:
+        graphs.append(capture_steps(m, hiddens, scores, range(K % R), stream))
+    return graphs, 1
+
+
+def time_passes(graphs, n_pass, stream):
+    """Replays the pass n_pass times back to back on `stream`, one CUDA event between consecutive passes.
+    Returns the per-pass milliseconds."""
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_pass + 1)]
+    with torch.cuda.stream(stream):
+        evs[0].record(stream)
+        for r in range(n_pass):
+            for g in graphs:
+                g.replay()
+            evs[r + 1].record(stream)
+    torch.cuda.synchronize()
+    return [evs[r].elapsed_time(evs[r + 1]) for r in range(n_pass)]
+
+
+def passes_for(graphs, stream, min_region_s=MIN_REGION_S):
+    """Untimed: the pass twice (uploads the graphs), then a short estimate of its time."""
+    time_passes(graphs, 2, stream)
+    est_ms = float(np.median(time_passes(graphs, 3, stream)))
+    return int(min(max(np.ceil(min_region_s * 1e3 / max(est_ms, 1e-3)), 5), 20000))
+
+
+def contract_config():
+    """The same in both arms (the driver compares them)."""
+    return {"workload": WORKLOAD,
+            "l2": "inputs larger than L2: the hidden states of successive steps rotate over >= 512 MiB of buffers "
+                  "(4x L2), so every step finds its rows cold; the 0.75 MiB of weights stay warm, as in serving"}
+
+
 def run_mix(args, rank, world, local_rank):
     import paper_2607_22595_b200 as mixlib
     from paper_2607_22595_b200 import _build
@@ -596,90 +744,75 @@ def run_mix(args, rank, world, local_rank):
     w = W.make_decode("cuda", seed=W.BASE_SEED + 1000 + rank)
     m = W.make_context(mixlib.Mix, w)
     T, d = w.T_max, w.d_model
+    K = args.steps or 256                      # steps per repeat
+    Wm = max(args.warmup if args.warmup is not None else 5, 3)
     R = max(2, -(-ROTATE_BYTES // (T * d * 2)))
+    if K < R:
+        R = -(-R // K) * K                     # a whole number of K-step graphs
     hiddens = [w.hidden.clone() for _ in range(R)]
     scores = [torch.zeros((T, 1), dtype=torch.float32, device="cuda") for _ in range(R)]
-    K = args.steps or 400 * R
-    Wm = args.warmup if args.warmup is not None else 3 * R
-    Wm = max(Wm, 3)
 
     stream = torch.cuda.Stream()
     stream.wait_stream(torch.cuda.current_stream())
+    # `value` is the step as it costs behind ANY predecessor kernel: the hook kernel launched the ordinary way.
+    # (With programmatic dependent launch, hook calls placed back to back hide each other's table look-ups; that
+    # figure is measured afterwards and reported beside it.)
+    pdl_default = mixlib.set_pdl_mask(-1)
+    mixlib.set_pdl_mask(pdl_default & ~8)
     with torch.cuda.stream(stream):
-        for i in range(min(Wm, R)):
-            m.apply(hiddens[i], scores[i], stream=stream)            # untimed warm-up, eager
-        g_full = capture_steps(m, hiddens, scores, range(R), stream) if K >= R else None
-        rem = K % R
-        g_rem = capture_steps(m, hiddens, scores, range(rem), stream) if rem else None
-        for _ in range(max(0, (Wm - R) // R)):
-            if g_full is not None:
-                g_full.replay()
+        for i in range(Wm):
+            m.apply(hiddens[i % R], scores[i % R], stream=stream)   # W untimed warm-up steps, eager
+        graphs, reps_per_pass = plan_pass(m, hiddens, scores, K, stream)
     torch.cuda.synchronize()
+    n_pass = passes_for(graphs, stream)
+    n_rep = n_pass * reps_per_pass
 
     sampler = ClockSampler(local_rank)
     time.sleep(0.3)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier(world); torch.cuda.synchronize()
     t0 = time.time()
-    with torch.cuda.stream(stream):
-        e0.record(stream)
-        for _ in range(K // R):
-            g_full.replay()
-        if g_rem is not None:
-            g_rem.replay()
-        e1.record(stream)
-    torch.cuda.synchronize(); barrier(world)
+    per_rep = [x / reps_per_pass for x in time_passes(graphs, n_pass, stream)]     # ms per K steps
+    barrier(world)
     t1 = time.time()
-    ms_local = e0.elapsed_time(e1)
-    ms = dist_max(ms_local, world)
-    rows_total = dist_sum(float(K) * w.T_live, world)
+    ms_rep = dist_max(float(np.median(per_rep)), world)          # K steps, median over repeats, slowest rank
+    ms_per_step = ms_rep / K
+    rows_per_rep = dist_sum(float(K) * w.T_live, world)
     clocks = sampler.summary(t0, t1)
+    region_s = float(np.sum(per_rep)) * reps_per_pass * 1e-3
+    spread = {"p10": float(np.quantile(per_rep, 0.1)) / K * 1e3, "p50": float(np.median(per_rep)) / K * 1e3,
+              "p90": float(np.quantile(per_rep, 0.9)) / K * 1e3, "mean": float(np.mean(per_rep)) / K * 1e3}
 
-    # warm-L2 variant (one buffer), for context
+    def us_per_step(gs, steps_per_pass):
+        n = passes_for(gs, stream, MIN_REGION_S / 3)
+        return float(np.median(time_passes(gs, n, stream))) / steps_per_pass * 1e3
+
+    # side figures, same protocol: (a) programmatic dependent launch of the hook kernel, calls back to back
+    mixlib.set_pdl_mask(pdl_default)
     with torch.cuda.stream(stream):
-        g_warm = capture_steps(m, hiddens, scores, [0] * min(R, 256), stream)
-        g_warm.replay()
-        e0.record(stream)
-        for _ in range(4):
-            g_warm.replay()
-        e1.record(stream)
+        graphs_pdl, _ = plan_pass(m, hiddens, scores, K, stream)
     torch.cuda.synchronize()
-    warm_us = e0.elapsed_time(e1) * 1e3 / (4 * min(R, 256))
-
-    # the cold protocol again with the hook kernels launched the ordinary way (no programmatic dependent launch):
-    # what a step costs behind a kernel that does not let its successor start early
-    old_mask = mixlib.set_pdl_mask(-1)
-    mixlib.set_pdl_mask(old_mask & ~8)
+    pdl_us = us_per_step(graphs_pdl, K * reps_per_pass)
+    del graphs_pdl
+    mixlib.set_pdl_mask(pdl_default & ~8)
+    # (b) warm L2: every step on the same buffer
+    Kw = 256
     with torch.cuda.stream(stream):
-        g_plain = capture_steps(m, hiddens, scores, range(R), stream)
-        g_plain.replay()
-        e0.record(stream)
-        for _ in range(4):
-            g_plain.replay()
-        e1.record(stream)
+        graphs_warm = [capture_steps(m, hiddens, scores, [0] * Kw, stream)]
     torch.cuda.synchronize()
-    plain_us = e0.elapsed_time(e1) * 1e3 / (4 * R)
-    mixlib.set_pdl_mask(old_mask)
-    del g_plain
-
-    # launch floor: the same graph with zero live rows (every CTA exits after one 4-byte load)
+    warm_us = us_per_step(graphs_warm, Kw)
+    # (c) launch floor: the same graphs with zero live rows (every CTA exits after one 4-byte load)
     m.set_slot_map(torch.from_numpy(w.token_slot.copy()).cuda(), 0)
-    with torch.cuda.stream(stream):
-        g_warm.replay()
-        e0.record(stream)
-        for _ in range(4):
-            g_warm.replay()
-        e1.record(stream)
-    torch.cuda.synchronize()
-    floor_us = e0.elapsed_time(e1) * 1e3 / (4 * min(R, 256))
+    floor_us = us_per_step(graphs, K * reps_per_pass)
     m.set_slot_map(torch.from_numpy(w.token_slot.copy()).cuda(), w.T_live)
+    torch.cuda.synchronize()
+    del graphs_warm
+    mixlib.set_pdl_mask(pdl_default)
 
     # end to end through the public API with host buffers: every step copies its hidden states
     # and slot map from pinned host memory, applies the hook, and copies hidden + scores back.
     # Steps are independent batches, so they are pipelined over a few contexts (one stream and
     # one device buffer each): the H2D of one step overlaps the D2H of another, as a serving
     # engine with several batches in flight would do.
-    K_e2e = min(K, 2000)
     n_pipe = 3
     pipes = []
     for i in range(n_pipe):
@@ -701,18 +834,17 @@ def run_mix(args, rank, world, local_rank):
     for i in range(2 * n_pipe):
         e2e_step(i)
     # host <-> device copies share the PCIe link and the host's memory system with other tenants of the box:
-    # three rounds, the fastest is reported
-    n_round, K_round = 3, max(K_e2e // 3, 1)
+    # three rounds of max(K, 200) steps each, the fastest is reported
+    n_round, K_e2e = 3, max(K, 200)
     e2e_s = None
     for _ in range(n_round):
         torch.cuda.synchronize(); barrier(world)
         te = time.perf_counter()
-        for i in range(K_round):
+        for i in range(K_e2e):
             e2e_step(i)
         torch.cuda.synchronize()
         dt = dist_max(time.perf_counter() - te, world)
         e2e_s = dt if e2e_s is None else min(e2e_s, dt)
-    K_e2e = K_round
     torch.cuda.set_stream(torch.cuda.default_stream())
     sampler.stop()
     e2e_rows = dist_sum(float(K_e2e) * w.T_live, world)
@@ -721,83 +853,114 @@ def run_mix(args, rank, world, local_rank):
     if rank != 0:
         return
     nbytes, rows_p, rows_s = decode_bytes(w)
-    ms_per_step = ms / K
     achieved = nbytes / (ms_per_step * 1e-3) / 1e9
     line = {
-        "metric": METRIC, "value": rows_total / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "metric": METRIC, "value": rows_per_rep / (ms_rep * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "l2": "inputs rotate over %d hidden buffers (%d MiB > 4x L2); weights (0.75 MiB) stay warm" % (R, R * T * d * 2 >> 20),
-                   "graph": "CUDA-graph replay, %d steps per graph" % R, "probe_rows": rows_p, "steer_rows": rows_s,
-                   "us_added_per_decode_step": ms_per_step * 1e3, "us_added_per_decode_step_warm_l2": warm_us,
-                   "us_added_per_decode_step_32_hooked_layers": 32 * ms_per_step * 1e3,
-                   "us_per_step_zero_live_rows": floor_us,
-                   "us_added_per_decode_step_without_programmatic_launch": plain_us,
-                   "launch": "hook kernels are launched with programmatic stream serialization: in this back-to-back "
-                             "protocol a step's live-count / slot-map / app-table / vector lookups overlap the previous "
-                             "step's kernel, and `hidden` is read after the in-kernel wait; behind a kernel that does not "
-                             "signal early the step costs the 'without' figure",
-                   "status_word": status},
+        "dtype": "bf16", "data": "synthetic", "config": contract_config(),
         "clocks": clocks,
         "e2e": {"value": e2e_rows / e2e_s, "unit": UNIT, "h2d_bytes_per_step": T * d * 2 + 4 * T,
-                "d2h_bytes_per_step": T * d * 2 + 4 * T, "steps": K_e2e, "rounds": "fastest of 3", "pipeline_depth": n_pipe},
-        "gpu_launches": K * m.launches_per_apply(),
+                "d2h_bytes_per_step": T * d * 2 + 4 * T, "steps": K_e2e, "rounds": "fastest of %d" % n_round,
+                "pipeline_depth": n_pipe},
+        "gpu_launches": n_rep * K * m.launches_per_apply(),
         "roofline": {"bound": "hbm", "kernel": "probe_steer_team_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": DECODE_DRAM_BYTES_PER_LAUNCH,
+                     "traffic_source": "dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel on this "
+                                       "workload in an earlier ncu capture (not re-measured by this run)",
                      "frac_of_nominal_8000_gbs": achieved / NOMINAL_HBM_GBS,
                      "peak_source": peaks["source"],
                      "algorithmic_bytes_per_launch": nbytes,
-                     "note": "2.9 MB per launch: launch-latency-bound, not bandwidth-bound; see extras.sweep for the same kernel on 2 GiB"},
+                     "note": "2.9 MB per launch: launch-latency-bound by construction; the bandwidth- and tensor-bound "
+                             "kernels of the other configs are in `targets`",
+                     "protocol": {"steps_per_repeat": K, "repeats": n_rep, "timed_region_s": region_s,
+                                  "ms_per_step": "median over timed passes of (pass time / steps in the pass)",
+                                  "repeats_per_timed_pass": reps_per_pass, "us_per_step_over_passes": spread,
+                                  "graph": "CUDA-graph replay; a graph launch holds %d consecutive steps (%d repeats of %d) over %d "
+                                           "hidden buffers (%d MiB)" % (min(K, R) if K > R else R, reps_per_pass, K, R,
+                                                                        R * T * d * 2 >> 20),
+                                  "launch": "ordinary kernel launch (what a step costs behind any predecessor kernel)"},
+                     "decode_step": {"probe_rows": rows_p, "steer_rows": rows_s,
+                                     "us_added_per_decode_step": ms_per_step * 1e3,
+                                     "us_added_per_decode_step_32_hooked_layers": 32 * ms_per_step * 1e3,
+                                     "us_per_step_warm_l2": warm_us, "us_per_step_zero_live_rows": floor_us,
+                                     "us_per_step_programmatic_launch_back_to_back": pdl_us,
+                                     "status_word": status}},
     }
     if world == 1:
-        cb = oracle_leg(args.cpu_seconds)
-        line["cpu_baseline"] = {"value": cb["rows_per_s"], "unit": UNIT, "cores": 1, "kind": "oracle",
-                                "sample": "%d whole decode batches (%d rows) in %.1f s" % (cb["batches"], cb["rows"], cb["seconds"])}
+        line["cpu_baseline"] = cpu_baseline_block(args.cpu_seconds)
         if not args.no_extras:
-            ex = {}
+            targets, ex = {}, {}
             try:
-                ex["decode_variants"] = extras_decode_variants(w, hiddens, scores, mixlib)
-                ex["sweep"] = extras_sweep(peaks, mixlib)
-                ex["multiclass_probes"] = extras_multiclass(peaks, mixlib)
-                tiny = extras_sae("tiny (config 0)", W.make_tiny("cuda"), peaks, mixlib)
-                ex["tiny"] = {"t_call_ms_graph": tiny["t_call_ms_graph"], "status": tiny["status"],
-                              "note": "correctness config: the call sits on the launch-latency floor of its kernel chain"}
-                ex["sae_heavy"] = extras_sae("sae_heavy (config 2)", W.make_sae_heavy("cuda"), peaks, mixlib)
-                torch.cuda.empty_cache()
-                wm = W.make_mixed("cuda")
-                ex["mixed"] = extras_sae("mixed (config 3)", wm, peaks, mixlib)
-                eo = extras_sae("mixed (config 3), edit-only shortcut", wm, peaks, mixlib, extra_flags=8)
-                ex["mixed_edit_only_shortcut"] = {
-                    "note": "MIX_FLAG_SAE_EDIT_ONLY: JumpReLU rows with the error term skip the encode (16 dot products "
-                            "per row instead); an algorithmic shortcut, not counted toward any tensor-pipe fraction",
-                    "t_call_ms_graph": eo["t_call_ms_graph"], "stage_ms": eo["stage_ms"],
-                    "token_rows_per_s": eo["token_rows_per_s"], "status": eo["status"]}
-                eoc = extras_sae("mixed (config 3), edit-only shortcut, conditional graph", wm, peaks, mixlib, extra_flags=8,
-                                 conditional=True)
-                ex["mixed_edit_only_shortcut"]["t_call_ms_graph_with_mix_apply_conditional"] = eoc["t_call_ms_graph"]
-                ex["mixed_edit_only_shortcut"]["note_conditional"] = (
-                    "every SAE row takes the shortcut here, so the packed panel is empty and the graph IF node of "
-                    "mix_apply_conditional skips the seven kernels of the SAE chain")
-                del wm
-                torch.cuda.empty_cache()
-                # opt-in 8-bit encoder: with the bf16 hidden state kept exact (two E4M3 operands per row), and with the
-                # encoder's input quantised as well (a different numerical method)
-                for key, mk, label, act in (
-                        ("sae_heavy_8bit_encoder", W.make_sae_heavy, "sae_heavy (config 2), 8-bit encoder, bf16 rows", False),
-                        ("mixed_8bit_encoder", W.make_mixed, "mixed (config 3), 8-bit encoder, bf16 rows", False),
-                        ("sae_heavy_8bit", W.make_sae_heavy, "sae_heavy (config 2), 8-bit encoder and input", True),
-                        ("mixed_8bit", W.make_mixed, "mixed (config 3), 8-bit encoder and input", True)):
-                    r8 = extras_sae(label, mk("cuda", fp8=True, fp8_act=act), peaks, mixlib, extra_flags=32 | (64 if act else 0),
-                                    w_enc_bytes_per_el=1.0)
-                    r8["note"] = ("MIX_FLAG_FP8_W_ENC" + (" | MIX_FLAG_FP8_ACT" if act else "") + "; tensor fractions here are "
-                                  "against the bf16 peaks" + (": halve them for the 8-bit peak (nominal ratio 2)" if act else
-                                                              " (two 8-bit instructions per element of K: the bf16 tensor time)"))
-                    ex[key] = r8
-                    torch.cuda.empty_cache()
-            except Exception as e:                       # extras never break the contract line
+                collect_targets(targets, ex, w, hiddens, scores, peaks, mixlib, args)
+            except Exception as e:                       # the other configs never break the contract line
                 ex["error"] = repr(e)
+            line["roofline"]["targets"] = targets
             line["extras"] = ex
     print(json.dumps(line), flush=True)
+
+
+def gpu_edit_hint(gi, sae, h_row):
+    """Input recipe of configs 2 and 3 (outside every timed region): the features that fire on one row, so
+    that half of a request's edits land on features it actually uses.  A plain torch product in row chunks."""
+    x = h_row.float()
+    z = torch.empty(sae.d_sae, dtype=torch.float32, device=x.device)
+    for j0 in range(0, sae.d_sae, 8192):
+        j1 = min(sae.d_sae, j0 + 8192)
+        Wc = sae.W_enc[j0:j1]
+        Wc = Wc.view(torch.float8_e4m3fn).float() * sae.w_scale[j0:j1, None] if sae.w_scale is not None else Wc.float()
+        z[j0:j1] = Wc @ x + sae.b_enc[j0:j1]
+    if sae.act == W.SAE_TOPK:
+        top = torch.topk(z, sae.k)
+        return top.indices[top.values > 0].cpu().numpy()
+    thr = sae.theta if sae.theta is not None else torch.zeros_like(z)
+    return torch.nonzero((z > thr) & (z > 0)).flatten().cpu().numpy()
+
+
+def collect_targets(targets, ex, w, hiddens, scores, peaks, mixlib, args):
+    """The other configurations: what the roofline targets are judged on goes to `targets` (compact), the
+    per-kernel detail to `extras`."""
+    sw = extras_sweep(peaks, mixlib)
+    ex["sweep"] = sw
+    targets["steer_stream"] = {"what": "steering alone, d=8192, T=65536 (2 GiB read + written)", "gbs": sw["steer"]["gbs"],
+                               "frac_hbm": sw["steer"]["frac_hbm_peak"]}
+    targets["probe_stream"] = {"what": "one-class probe alone, d=8192, T=65536 (1 GiB read)", "gbs": sw["probe"]["gbs"],
+                               "frac_hbm": sw["probe"]["frac_hbm_peak"]}
+    targets["encode_alone"] = {"what": sw["encode"]["shape"], "tflops": sw["encode"]["tflops"],
+                               "frac_bf16_burst": sw["encode"]["frac_bf16_peak"]}
+    tiny = extras_sae("tiny (config 0)", W.make_tiny("cuda"), peaks, mixlib)
+    targets["cfg0_tiny"] = {"call_us": tiny["t_call_ms_graph"] * 1e3, "status": tiny["status"]}
+    r2 = extras_sae("sae_heavy (config 2)", W.make_sae_heavy("cuda", edit_hint=gpu_edit_hint), peaks, mixlib)
+    ex["sae_heavy"] = r2
+    targets["cfg2_sae_heavy"] = {"call_us": r2["t_call_ms_graph"] * 1e3, "encode_us": r2["stage_ms"]["encode"] * 1e3,
+                                 "encode_w_enc_gbs": r2["encode_weight_stream_gbs"], "encode_frac_hbm": r2["encode_frac_hbm_peak"],
+                                 "call_over_encode": r2["t_call_ms_graph"] / r2["stage_ms"]["encode"], "status": r2["status"]}
+    torch.cuda.empty_cache()
+    wm = W.make_mixed("cuda", edit_hint=gpu_edit_hint)
+    r3 = extras_sae("mixed (config 3)", wm, peaks, mixlib)
+    ex["mixed"] = r3
+    targets["cfg3_mixed"] = {"call_us": r3["t_call_ms_graph"] * 1e3, "encode_us": r3["stage_ms"]["encode"] * 1e3,
+                             "encode_tflops": r3["encode_tflops"], "encode_frac_bf16_burst": r3["encode_frac_bf16_peak"],
+                             "encode_frac_bf16_sustained": r3["encode_frac_bf16_sustained"],
+                             "call_over_encode": r3["t_call_ms_graph"] / r3["stage_ms"]["encode"], "status": r3["status"]}
+    eo = extras_sae("mixed (config 3), edit-only shortcut", wm, peaks, mixlib, extra_flags=8)
+    ex["mixed_edit_only_shortcut"] = {
+        "note": "MIX_FLAG_SAE_EDIT_ONLY: JumpReLU rows with the error term skip the encode (16 dot products per row "
+                "instead); an algorithmic shortcut, not counted toward any tensor-pipe fraction",
+        "t_call_ms_graph": eo["t_call_ms_graph"], "stage_ms": eo["stage_ms"], "status": eo["status"]}
+    del wm
+    torch.cuda.empty_cache()
+    rd = extras_replace_decode(peaks, mixlib)
+    ex["replace_decode"] = rd
+    targets["replace_decode"] = {"what": rd["what"], "decode_us": rd["decode_us"], "gather_gbs": rd["gather_gbs"],
+                                 "frac_hbm": rd["frac_hbm_peak"], "status": rd["status"]}
+    r4 = run_replay(peaks, mixlib, args.replays)
+    ex["replay"] = r4
+    targets["cfg4_replay"] = {"replays": r4["replays"], "bound_over_time": r4["bound_over_time"],
+                              "t_call_ms": r4["t_call_ms"], "empty_replay_us": None if r4["empty_replay_ms"] is None else r4["empty_replay_ms"] * 1e3,
+                              "n_live_covered": r4["n_live_covered"], "status_or": r4["status_or"]}
+    torch.cuda.empty_cache()
+    ex["multiclass_probes"] = extras_multiclass(peaks, mixlib)
+    ex["decode_variants"] = extras_decode_variants(w, hiddens[:256], scores[:256], mixlib)
 
 
 def main():
@@ -811,7 +974,8 @@ def main():
                     help="SAE contexts stream W_enc as registered instead of a tile-contiguous copy (MIX_FLAG_RETILE_W_ENC)")
     ap.add_argument("--workload", default="decode",
                     help="decode (the contract line) | sweep | sae_heavy | sae_heavy_fp8 | sae_heavy_fp8a | sae_small | sae_small_fp8 | sae_small_fp8a | mixed | mixed_fp8 | mixed_fp8a | mixed_edit_only | mixed_small | mixed_small_fp8a | conditional | conditional_small | replay_fp8 | replay_fp8a | multiclass | multiclass_small | replay")
-    ap.add_argument("--cpu-seconds", type=float, default=10.0)
+    ap.add_argument("--cpu-seconds", type=float, default=8.0)
+    ap.add_argument("--replays", type=int, default=60, help="replays of config 4 in the default run")
     args = ap.parse_args()
     if args.no_retile:
         global SAE_FLAGS
