@@ -506,6 +506,8 @@ def run_workload(args):
     name = args.workload
     if name == "sweep":
         out = extras_sweep(peaks, mixlib)
+    elif name == "sweep_small":       # profiling case for the streaming probe / steering kernel
+        out = extras_sweep(peaks, mixlib, small=True)
     elif name == "sae_heavy":
         out = extras_sae("sae_heavy (config 2)", W.make_sae_heavy("cuda"), peaks, mixlib)
     elif name == "sae_heavy_fp8":   # config 2 with the encoder as 8-bit codes (MIX_FLAG_FP8_W_ENC)
@@ -639,9 +641,10 @@ def extras_decode_variants(w, hiddens, scores, mixlib):
     return out
 
 
-def extras_sweep(peaks, mixlib):
-    """Bandwidth kernels alone at a size that cannot hide in L2: d = 8192, T = 65536, every row hooked."""
-    d, T = 8192, 65536
+def extras_sweep(peaks, mixlib, small=False):
+    """Bandwidth kernels alone at a size that cannot hide in L2: d = 8192, T = 65536, every row hooked.
+    small: T = 16384 (256 MiB of hidden state) and no encode -- the profiling case."""
+    d, T = 8192, (16384 if small else 65536)
     g = torch.Generator(device="cuda"); g.manual_seed(1)
     hidden = torch.randn((T, d), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
     v = torch.randn((d,), generator=g, device="cuda").to(torch.bfloat16)
@@ -663,6 +666,8 @@ def extras_sweep(peaks, mixlib):
     m.destroy()
     del hidden
     torch.cuda.empty_cache()
+    if small:
+        return out
     # the encode alone in the tensor-bound regime: one TopK weight set, every row an SAE row
     d, T, S = 4096, 4096, 65536
     sae = W.make_sae_weights(g, "cuda", d, S, W.SAE_TOPK, k=64)

@@ -334,11 +334,10 @@ int mix_set_feature_out(mix_ctx* ctx, int* topk_idx, float* topk_val, int* n_act
    part that looks up the live count, slot map, app entry and single-vector weights -- tables the
    library owns and only copies write -- overlaps that kernel; `hidden`, gate scores and
    multi-class probe weights are read only after the predecessor has completed and flushed, and the
-   grid does not end before it.  Behind any other kernel nothing changes.  Two launch shapes follow
+   grid does not end before it.  Behind any other kernel nothing changes.  One launch shape follows
    from what is registered when the call is enqueued or captured -- the encode's epilogue warps
-   (TopK weight set present or not) and the decode's rows per CTA (a replacing SAE app present or
-   not); this is performance only: every shape handles every registration, so tables rewritten
-   after a capture are still applied correctly.  Device-side
+   (TopK weight set present or not); this is performance only: either shape handles every
+   registration, so tables rewritten after a capture are still applied correctly.  Device-side
    problems (bad slot ids, ...) are reported through the status word, never by faulting.
    Errors: INVALID_ARG (NULL hidden, misaligned), OUT_OF_RANGE (T), CUDA (launch failure). */
 int mix_apply(mix_ctx* ctx, void* hidden, int T, float* scores_out, void* stream);
@@ -347,10 +346,10 @@ int mix_apply(mix_ctx* ctx, void* hidden, int T, float* scores_out, void* stream
    paper, paragraph "Graph-level toggling and continuous batching": for true data-dependent
    control flow an upstream GPU computation decides whether a downstream intervention body
    executes, as with CUDA conditional nodes, with no CPU in the loop).  `stream` MUST be capturing: the call adds to
-   the graph being captured the probe / steering kernels and the route kernel as mix_apply() does,
-   then one conditional IF node whose body holds the rest of the SAE chain (pack, encode,
-   selection, decode); the route kernel sets the node's condition to (SAE rows routed > 0).  A
-   replay with no SAE row live therefore launches none of the body's kernels, instead of eight
+   the graph being captured the probe / steering kernels and the routing kernel as mix_apply() does,
+   then one conditional IF node whose body holds the rest of the SAE chain (encode, selection,
+   decode); the routing kernel sets the node's condition to (SAE rows routed > 0).  A
+   replay with no SAE row live therefore launches none of the body's kernels, instead of four
    kernels that each find nothing to do.  Results are identical to mix_apply()'s.  The capture
    continues after the node; work captured later on `stream` depends on it.  A context without
    weight sets behaves exactly like mix_apply() (and then `stream` need not be capturing).
@@ -371,7 +370,7 @@ int mix_apply_router(mix_ctx* ctx, float* logits, int n_experts, int T, void* st
 int mix_get_status(mix_ctx* ctx, unsigned* bits, void* stream);
 
 /* Number of kernels one mix_apply() call launches on this context (fixed at mix_create):
-   1 without SAE weight sets, else 8 (6 with MIX_FLAG_ENCODE_SIMT); one more when T_max > 2048
+   1 without SAE weight sets, else 6 (4 with MIX_FLAG_ENCODE_SIMT); one more when T_max > 2048
    and C_max > 1 (multi-class probes of large batches run in a kernel of their own), and two more
    with MIX_FLAG_SAE_EDIT_ONLY. */
 int mix_launches_per_apply(const mix_ctx* ctx);
@@ -382,9 +381,10 @@ int mix_launches_per_apply(const mix_ctx* ctx);
    its first kernel and events[i] after its i-th kernel, on the call's stream; the array is
    copied.  Kernel order: [probe_decide,] probe_steer, [probe_multiclass: only if T_max > 2048 and C_max > 1;
    probe_decide before and probe_tc after it if also n_groups_max == 0,]
-   route, pack, encode, merge, encode (flagged row tiles), select, decode; with
-   MIX_FLAG_ENCODE_SIMT the SAE part is route, pack, encode, select, decode; with
-   MIX_FLAG_SAE_EDIT_ONLY an edit_only and an edit_only_delta kernel come last. */
+   front (routing + row pack), encode, tail (selection, edits, decode, write-back), encode (row tiles
+   flagged for the exact fallback selection), tail (the flagged rows); with MIX_FLAG_ENCODE_SIMT the
+   SAE part is front, encode, tail; with MIX_FLAG_SAE_EDIT_ONLY an edit_only and an edit_only_delta
+   kernel come last. */
 int mix_set_stage_events(mix_ctx* ctx, void* const* events);
 
 /* Measurement aid for the paper's "CUDA-graph-safe kernel design" paragraph (separate static graph
@@ -403,8 +403,8 @@ int mix_bench_param_update(mix_ctx* ctx, int iters, float* us_table, float* us_n
 /* Which launches of the library use programmatic dependent launch (a kernel's CTAs may become resident,
    and run the part of the kernel that reads only library-owned tables, while the kernel in front of
    it in the stream is still running; everything the predecessor may have written is read after an
-   in-kernel wait).  Bits: 1 the row-packing kernel, 2 the full SAE encode pass, 4 the kernels
-   after it, 8 the one-CTA-per-row probe / steering kernel of a context that has no SAE weight sets
+   in-kernel wait).  Bits: 1 unused (the row pack is part of the first kernel of the SAE chain),
+   2 the full SAE encode pass, 4 the kernels after it, 8 the one-CTA-per-row probe / steering kernel of a context that has no SAE weight sets
    (T_max <= 2048).  Default 1 | 4 | 8, or the value of MIX_PDL_MASK in the environment when the
    library first launches.  Process-wide; affects launches (and captures) made afterwards; meant
    for A/B measurement.  Returns the previous mask.  mask < 0 only queries. */

@@ -307,8 +307,8 @@ class Mix:
             return front
         tail = ["edit_only", "edit_only_delta"] if self.cfg.flags & MIX_FLAG_SAE_EDIT_ONLY else []
         if self.cfg.flags & MIX_FLAG_ENCODE_SIMT:
-            return front + ["route", "pack", "encode", "select", "decode", "decode_delta"] + tail
-        return front + ["route", "pack", "encode", "merge", "encode_flagged", "select", "decode", "decode_delta"] + tail
+            return front + ["front", "encode", "tail"] + tail
+        return front + ["front", "encode", "tail", "encode_flagged", "tail_flagged"] + tail
 
     def set_stage_events(self, events=None):
         """events: list of launches_per_apply() + 1 torch.cuda.Event(enable_timing=True), or None."""

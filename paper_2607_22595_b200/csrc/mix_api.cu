@@ -80,12 +80,11 @@ cudaError_t dev_alloc(T** p, size_t n) {
 }
 
 void free_all(mix_ctx* c) {
-  cudaFree(c->d_token_slot); cudaFree(c->d_n_live); cudaFree(c->d_apps); cudaFree(c->d_groups); cudaFree(c->d_gates); cudaFree(c->d_vec_arena); cudaFree(c->d_chain_next); cudaFree(c->d_row_slot);
+  cudaFree(c->d_token_slot); cudaFree(c->d_n_live); cudaFree(c->d_apps); cudaFree(c->d_groups); cudaFree(c->d_gates); cudaFree(c->d_vec_arena); cudaFree(c->d_chain_next); cudaFree(c->d_row_slot); cudaFree(c->d_row_rec);
   cudaFree(c->d_edit_idx); cudaFree(c->d_edit_val); cudaFree(c->d_edit_mode); cudaFree(c->d_status);
   cudaFree(c->d_tmp_req); cudaFree(c->d_tmp_req_slot); cudaFree(c->d_panel); cudaFree(c->d_panel_row); cudaFree(c->d_act_scale); cudaFree(c->d_tau); cudaFree(c->d_tau_min); cudaFree(c->d_eo_row_delta); cudaFree(c->d_eo_coef);
-  cudaFree(c->d_mtile_group); cudaFree(c->d_row_group); cudaFree(c->d_route); cudaFree(c->d_z); cudaFree(c->d_topk_idx);
-  cudaFree(c->d_topk_val); cudaFree(c->d_tmap_w); cudaFree(c->d_tmap_probe); cudaFree(c->d_mc_dense); cudaFree(c->d_cand_val); cudaFree(c->d_cand_idx);
-  cudaFree(c->d_row_delta); cudaFree(c->d_edit_coef);
+  cudaFree(c->d_mtile_group); cudaFree(c->d_row_group); cudaFree(c->d_route); cudaFree(c->d_z);
+  cudaFree(c->d_tmap_w); cudaFree(c->d_tmap_probe); cudaFree(c->d_mc_dense); cudaFree(c->d_cand_val); cudaFree(c->d_cand_idx);
   cudaFree(c->d_cand_ninth); cudaFree(c->d_row_flag); cudaFree(c->d_mtile_flag); cudaFree(c->d_n_flagged);
   if (c->owned_b_eff)
     for (int g = 0; g < c->cfg.n_groups_max; ++g) cudaFree(c->owned_b_eff[g]);
@@ -258,11 +257,8 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
     ok = ok && dev_alloc(&c->d_row_slot, T) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_route, 1) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_z, P * (size_t)cfg->d_sae_max) == cudaSuccess;
-    ok = ok && dev_alloc(&c->d_topk_idx, P * (size_t)c->cfg.k_max) == cudaSuccess;
-    ok = ok && dev_alloc(&c->d_topk_val, P * (size_t)c->cfg.k_max) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_tmap_w, G) == cudaSuccess;
-    ok = ok && dev_alloc(&c->d_row_delta, P) == cudaSuccess;
-    ok = ok && dev_alloc(&c->d_edit_coef, P * (size_t)(cfg->r_max > 0 ? cfg->r_max : 1)) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_row_rec, P) == cudaSuccess;
     if (cfg->flags & MIX_FLAG_SAE_EDIT_ONLY) {
       ok = ok && dev_alloc(&c->d_eo_row_delta, (size_t)T) == cudaSuccess;
       ok = ok && dev_alloc(&c->d_eo_coef, (size_t)T * (size_t)(cfg->r_max > 0 ? cfg->r_max : 1)) == cudaSuccess;
@@ -666,30 +662,24 @@ int mix_set_feature_out(mix_ctx* c, int* topk_idx, float* topk_val, int* n_activ
 extern "C++" {
 namespace {
 
-// The SAE chain after routing: pack ... decode.  `tap` records a stage event after each launch.
+// The SAE chain behind the front kernel: encode ... write-back.  `tap` records a stage event after each launch.
 template <class Tap>
 int sae_chain(mix_ctx* c, __nv_bfloat16* h, cudaStream_t s, Tap&& tap) {
-  MIX_CUDA(c, launch_pack(c, h, s));
-  MIX_CUDA(c, tap());
   if (c->cfg.flags & MIX_FLAG_ENCODE_SIMT) {
     MIX_CUDA(c, launch_encode_simt(c, s));
     MIX_CUDA(c, tap());
-    MIX_CUDA(c, launch_select(c, false, s));
+    MIX_CUDA(c, launch_tail(c, h, 1, s));        // TopK from Z, edits, decode
     MIX_CUDA(c, tap());
   } else {
     MIX_CUDA(c, launch_encode_tc(c, 0, s));      // TopK sets -> candidates, other sets -> Z
     MIX_CUDA(c, tap());
-    MIX_CUDA(c, launch_merge(c, s));             // exact TopK from candidates, or a flag
+    MIX_CUDA(c, launch_tail(c, h, 0, s));        // exact TopK from candidates (or a flag), edits, decode
     MIX_CUDA(c, tap());
     MIX_CUDA(c, launch_encode_tc(c, 1, s));      // flagged row tiles -> Z (returns at once if none)
     MIX_CUDA(c, tap());
-    MIX_CUDA(c, launch_select(c, true, s));      // flagged TopK rows; active counts of the other sets
+    MIX_CUDA(c, launch_tail(c, h, 2, s));        // the flagged rows (returns at once if none)
     MIX_CUDA(c, tap());
   }
-  MIX_CUDA(c, launch_decode(c, h, s));           // rows that replace the residual; edit coefficients
-  MIX_CUDA(c, tap());
-  MIX_CUDA(c, launch_decode_delta(c, h, s));     // rows that keep the error term
-  MIX_CUDA(c, tap());
   return MIX_OK;
 }
 
@@ -788,11 +778,11 @@ int apply_impl(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream,
   if (tc_fork) MIX_CUDA(c, cudaStreamWaitEvent(ps, c->ev_join, 0));
   if (fork) MIX_CUDA(c, cudaEventRecord(c->ev_join, ps));
   if (c->cfg.n_groups_max > 0) {
-    MIX_CUDA(c, launch_route(c, T, s, handle, conditional ? 1 : 0));
-    MIX_CUDA(c, tap());
     // with slot chains a steering app may precede an SAE app on the same row: the SAE chain reads
-    // the hidden state only after the probe / steering kernel is done
+    // the hidden state (first in the front kernel's row pack) only after the probe / steering kernel is done
     if (fork && (c->cfg.flags & MIX_FLAG_SLOT_CHAINS)) MIX_CUDA(c, cudaStreamWaitEvent(s, c->ev_join, 0));
+    MIX_CUDA(c, launch_front(c, h, T, s, handle, conditional ? 1 : 0));   // routing + row pack
+    MIX_CUDA(c, tap());
     const int rc = conditional ? sae_chain_conditional(c, h, s, graph, handle) : sae_chain(c, h, s, tap);
     if (rc != MIX_OK) return rc;
     if (c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) {
@@ -829,7 +819,7 @@ int mix_launches_per_apply(const mix_ctx* c) {
   if (!c) return 0;
   const int front = 1 + (has_multiclass_stage(c) ? 1 : 0) + (has_tc_probe_stage(c) ? 2 : 0);
   if (c->cfg.n_groups_max == 0) return front;
-  return front + ((c->cfg.flags & MIX_FLAG_ENCODE_SIMT) ? 6 : 8) + ((c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) ? 2 : 0);   // coefficient kernel + delta kernel
+  return front + ((c->cfg.flags & MIX_FLAG_ENCODE_SIMT) ? 3 : 5) + ((c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) ? 2 : 0);   // coefficient kernel + delta kernel
 }
 
 int mix_get_status(mix_ctx* c, unsigned* bits, void* stream) {

@@ -68,7 +68,18 @@ struct __align__(16) GroupEntry {
   const void* pad2_;
 };
 
-// What decode_kernel leaves for decode_delta_kernel about one packed row that keeps the error term.
+// What the front kernel leaves about one packed panel row for the kernels behind the encode: one 16-byte load
+// instead of the chain panel row -> slot map -> app entry.
+struct __align__(16) RowRec {
+  int t;                            // token row, or -1: padding row of a tile
+  int slot;                         // slot of the SAE app that acts on the row (the row's own, or the last of its chain)
+  int n_edit;                       // length of that app's edit list
+  int group_flags;                  // low byte: weight set; kRecAddError: the app keeps the error term
+};
+constexpr int kRecGroupMask = 0xff;
+constexpr int kRecAddError = 0x100;
+
+// What sae_edit_only_kernel leaves for decode_delta_kernel about one token row.
 struct __align__(16) RowDelta {
   int slot;                         // the row's slot, or -1: nothing to add (no effective edit, other kind of row)
   int n_edit;
@@ -124,13 +135,10 @@ struct Ctx {
   int* d_panel_row;         // [P] token index or -1
   int* d_mtile_group;       // [P / kTileM] group of each m-tile or -1
   int* d_row_group;         // [T_max] routing scratch: weight set of each token row or -1
-  int* d_row_slot;          // [T_max] slot of the SAE app that acts on the row (the row's own slot, or the last of its chain), or -1
+  int* d_row_slot;          // [T_max] routing scratch: slot of the SAE app that acts on the row (batches beyond the first 8192 rows)
+  RowRec* d_row_rec;        // [P] per packed row: token row, slot, edit count, weight set, error-term flag
   RouteState* d_route;
   float* d_z;               // [P, d_sae_max]
-  RowDelta* d_row_delta;    // [P]
-  float* d_edit_coef;       // [P, r_max] f'_j - f_j of each edit entry of the row's slot
-  int* d_topk_idx;          // [P, k_max]
-  float* d_topk_val;        // [P, k_max]
   float* d_cand_val;        // [P, cand_tiles, kCandPerTile] per-tile TopK candidates (fused epilogue)
   int* d_cand_idx;          // same shape: feature ids
   float* d_cand_ninth;      // [P, cand_tiles] the (kCandPerTile+1)-th largest value of each tile
@@ -220,15 +228,16 @@ cudaError_t probe_tc_prepare();   // opt in to the large dynamic shared memory s
 bool has_multiclass_stage(const Ctx* c);   // large batches with multi-class probes get a kernel of their own
 bool has_tc_probe_stage(const Ctx* c);     // ... and, in contexts without SAE weight sets, the tensor-core kernel for dense batches
 cudaError_t launch_router(const Ctx* c, float* logits, int n_experts, int T, cudaStream_t s);
-// cond/use_cond: graph-conditional handle the kernel sets to (SAE rows routed > 0); plain calls pass 0, 0
-cudaError_t launch_route(const Ctx* c, int T, cudaStream_t s, unsigned long long cond = 0, int use_cond = 0);
-cudaError_t launch_pack(const Ctx* c, const __nv_bfloat16* hidden, cudaStream_t s);
+// Routing + row pack in one launch.  cond/use_cond: graph-conditional handle the kernel sets to (SAE rows
+// routed > 0); plain calls pass 0, 0
+cudaError_t launch_front(const Ctx* c, const __nv_bfloat16* hidden, int T, cudaStream_t s, unsigned long long cond = 0,
+                         int use_cond = 0);
 cudaError_t launch_encode_simt(const Ctx* c, cudaStream_t s);
 cudaError_t launch_encode_tc(const Ctx* c, int mode, cudaStream_t s);   // 0: all tiles; 1: flagged row tiles -> Z
-cudaError_t launch_merge(const Ctx* c, cudaStream_t s);
-cudaError_t launch_select(const Ctx* c, bool flagged_only, cudaStream_t s);
-cudaError_t launch_decode(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s);         // rows without the error term
-cudaError_t launch_decode_delta(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s);   // rows with it
+// Selection, edits, decode and write-back of every SAE row.  mode 0: behind the tensor-core encode (TopK from its
+// candidates; rows it cannot settle are flagged); 1: behind the CUDA-core encode (TopK from Z); 2: the flagged
+// rows, after their row tiles were re-encoded to Z (returns at once when nothing is flagged).
+cudaError_t launch_tail(const Ctx* c, __nv_bfloat16* hidden, int mode, cudaStream_t s);
 cudaError_t launch_edit_only(const Ctx* c, __nv_bfloat16* hidden, int T, cudaStream_t s);
 cudaError_t launch_edit_only_delta(const Ctx* c, __nv_bfloat16* hidden, cudaStream_t s);   // decode_delta_kernel on the shortcut's token-indexed records
 cudaError_t edit_only_prepare();   // opt in to the dynamic shared memory of the edit-only kernel

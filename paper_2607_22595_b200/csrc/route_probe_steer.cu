@@ -1,10 +1,7 @@
-// Slot routing, the read (probe) and write (steering) primitives, and the SAE row pack.
+// The read (probe) and write (steering) primitives of the hook, and the small kernels around the slot map.
 //
 // probe_steer_kernel is the bandwidth kernel of the hook: one warp per token row, 16-byte
 // loads, fp32 FMA, shuffle reductions.  A row whose slot is -1 costs one 4-byte load.
-#include <cuda_fp16.h>
-#include <cuda_fp8.h>
-
 #include "mix_internal.h"
 #include "row_lookup.cuh"
 
@@ -657,277 +654,6 @@ probe_steer_chain_kernel(const int* __restrict__ token_slot, const int* __restri
   }
 }
 
-// ---------------------------------------------------------------------------------------
-// SAE routing: one CTA builds, in ascending row order, the packed-panel position of every
-// SAE row, the per-group counts and the encode tile schedule.  Integer work only.
-// ---------------------------------------------------------------------------------------
-constexpr int kRouteThreads = 1024;
-constexpr int kRouteWarps = kRouteThreads / 32;
-constexpr int kRouteBatch = 8;          // chunks of 1024 rows whose lookups are in flight together
-
-__global__ void __launch_bounds__(kRouteThreads)
-route_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
-             const AppEntry* __restrict__ apps, const GateEntry* __restrict__ gates, int n_slots,
-             const GroupEntry* __restrict__ groups, int n_groups,
-             int* __restrict__ panel_row, int panel_cap, int* __restrict__ mtile_group, RouteState* __restrict__ rs,
-             unsigned* __restrict__ status, int* __restrict__ row_flag, int* __restrict__ mtile_flag,
-             int* __restrict__ n_flagged, int* __restrict__ row_group, int edit_only,
-             cudaGraphConditionalHandle cond, int use_cond, const int* __restrict__ chain_next,
-             int* __restrict__ row_slot) {
-  extern __shared__ int s_cnt[];                      // [n_chunks * kRouteWarps][n_groups]
-  __shared__ int s_total[kMaxGroups], s_base[kMaxGroups + 1];
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int n_live = min(T, __ldg(n_live_p));
-  const int n_chunks = (n_live + kRouteThreads - 1) / kRouteThreads;
-
-  for (int p = tid; p < panel_cap; p += kRouteThreads) panel_row[p] = -1;
-  for (int m = tid; m < panel_cap / kTileM; m += kRouteThreads) mtile_group[m] = -1;
-  if (row_flag) {             // fallback-selection flags of the fused TopK path start clear every call
-    for (int p = tid; p < panel_cap; p += kRouteThreads) row_flag[p] = 0;
-    for (int m = tid; m < panel_cap / kTileM; m += kRouteThreads) mtile_flag[m] = 0;
-    if (tid == 0) *n_flagged = 0;
-  }
-
-  // phase A: the group of every row this thread owns (row c * 1024 + tid of chunk c), resolved
-  // stage by stage for kRouteBatch chunks at a time so that their loads are in flight together
-  // (slot ids, then app entries, then weight-set entries: three round trips per batch instead
-  // of three per chunk); then per (chunk, warp) counts per group.
-  for (int c0 = 0; c0 < n_chunks; c0 += kRouteBatch) {
-    int slot[kRouteBatch], grp[kRouteBatch];
-#pragma unroll
-    for (int c = 0; c < kRouteBatch; ++c) {
-      const int t = (c0 + c) * kRouteThreads + tid;
-      slot[c] = (c0 + c < n_chunks && t < n_live) ? __ldg(token_slot + t) : -1;
-      if (slot[c] >= n_slots) slot[c] = -1;
-    }
-    int2 head[kRouteBatch];
-    int group_id[kRouteBatch];
-#pragma unroll
-    for (int c = 0; c < kRouteBatch; ++c) {
-      head[c] = make_int2(0, 0);
-      group_id[c] = -1;
-      if (slot[c] >= 0) {
-        head[c] = __ldg(reinterpret_cast<const int2*>(apps + slot[c]));          // valid, kind
-        group_id[c] = __ldg(&apps[slot[c]].group);
-      }
-    }
-    // a row whose slot starts a chain is an SAE row if the chain ends in an SAE app: follow the
-    // links (rare, so the dependent loads are not batched) and carry on with that app's slot
-#pragma unroll
-    for (int c = 0; c < kRouteBatch; ++c) {
-      if (head[c].x && (head[c].y & kKindChained) && (head[c].y & kKindMask) != MIX_SAE) {
-        int s2 = slot[c];
-        int2 h2 = head[c];
-        for (int depth = 1; depth < kMaxChain && s2 >= 0; ++depth) {
-          s2 = (h2.y & kKindChained) ? __ldg(chain_next + s2) : -1;
-          if (s2 < 0 || s2 >= n_slots) { s2 = -1; break; }
-          h2 = __ldg(reinterpret_cast<const int2*>(apps + s2));
-          if (!h2.x) { s2 = -1; break; }
-          if ((h2.y & kKindMask) == MIX_SAE) break;
-        }
-        if (s2 >= 0 && (h2.y & kKindMask) != MIX_SAE) s2 = -1;
-        slot[c] = s2;
-        head[c] = s2 >= 0 ? h2 : make_int2(0, 0);
-        group_id[c] = s2 >= 0 ? __ldg(&apps[s2].group) : -1;
-      }
-    }
-#pragma unroll
-    for (int c = 0; c < kRouteBatch; ++c) {
-      grp[c] = -1;
-      if (head[c].x && (head[c].y & kKindMask) == MIX_SAE) {
-        const int g = group_id[c];
-        if (g < 0 || g >= n_groups || !__ldg(&groups[g].valid)) {
-          atomicOr(status, MIX_STATUS_BAD_GROUP);
-        } else if (edit_only && __ldg(&apps[slot[c]].add_error) && __ldg(&groups[g].act) != MIX_SAE_TOPK) {
-          // handled by sae_edit_only_kernel: with the error term on, a ReLU / JumpReLU row needs
-          // only the pre-activations of its edited features, not the whole encode
-        } else if (!(head[c].y & kKindGated) || gate_open(gates, slot[c], (c0 + c) * kRouteThreads + tid)) {
-          grp[c] = g;
-        }
-      }
-    }
-#pragma unroll
-    for (int c = 0; c < kRouteBatch; ++c) {
-      if (c0 + c < n_chunks) {                       // uniform across the CTA
-        const int t = (c0 + c) * kRouteThreads + tid;
-        if (t < n_live) {
-          row_group[t] = grp[c];                     // read back by this same thread in phase C
-          row_slot[t] = grp[c] >= 0 ? slot[c] : -1;  // the SAE app's slot, for the decode kernels
-        }
-        for (int q = 0; q < n_groups; ++q) {
-          const unsigned m = __ballot_sync(0xffffffffu, grp[c] == q);
-          if (lane == 0) s_cnt[((c0 + c) * kRouteWarps + warp) * n_groups + q] = __popc(m);
-        }
-      }
-    }
-  }
-  __syncthreads();
-  // phase B: exclusive scan over (chunk, warp) for each group; warp q owns group q
-  const int n_seg = n_chunks * kRouteWarps;
-  for (int q = warp; q < n_groups; q += kRouteWarps) {
-    int carry = 0;
-    for (int s0 = 0; s0 < n_seg; s0 += 32) {
-      const int i = s0 + lane;
-      const int v = i < n_seg ? s_cnt[i * n_groups + q] : 0;
-      int incl = v;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int y = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += y;
-      }
-      if (i < n_seg) s_cnt[i * n_groups + q] = carry + incl - v;
-      carry += __shfl_sync(0xffffffffu, incl, 31);
-    }
-    if (lane == 0) s_total[q] = carry;
-  }
-  __syncthreads();
-  if (tid == 0) {
-    int mt = 0, tiles = 0, rows = 0, topk_rows = 0;
-    for (int q = 0; q < n_groups; ++q) {
-      s_base[q] = mt * kTileM;
-      rs->group_count[q] = s_total[q];
-      rs->group_mtile0[q] = mt;
-      rs->group_tile0[q] = tiles;
-      const int m_tiles = (s_total[q] + kTileM - 1) / kTileM;
-      for (int m = 0; m < m_tiles; ++m) mtile_group[mt + m] = q;
-      mt += m_tiles;
-      rows += s_total[q];
-      if (s_total[q] > 0 && groups[q].act == MIX_SAE_TOPK) topk_rows += s_total[q];
-      tiles += s_total[q] > 0 ? m_tiles * (int)(groups[q].d_sae / kTileN) : 0;
-    }
-    s_base[n_groups] = mt * kTileM;
-    for (int q = n_groups; q <= kMaxGroups; ++q) {
-      rs->group_mtile0[q] = mt;
-      rs->group_tile0[q] = tiles;
-      if (q < kMaxGroups) rs->group_count[q] = 0;
-    }
-    rs->n_panel_rows = mt * kTileM;
-    rs->n_mtiles = mt;
-    rs->n_sae_rows = rows;
-    rs->total_tiles = tiles;
-    rs->n_topk_rows = topk_rows;
-    // graph-conditional form: the SAE chain sits in the body of an IF node that runs only when a row needs it
-    if (use_cond) cudaGraphSetConditional(cond, rows > 0 ? 1u : 0u);
-  }
-  __syncthreads();
-  // phase C: stable scatter
-  for (int c0 = 0; c0 < n_chunks; c0 += kRouteBatch) {
-    int grp[kRouteBatch];
-#pragma unroll
-    for (int c = 0; c < kRouteBatch; ++c) {
-      const int t = (c0 + c) * kRouteThreads + tid;
-      grp[c] = t < n_live ? row_group[t] : -1;
-    }
-#pragma unroll
-    for (int c = 0; c < kRouteBatch; ++c) {
-      if (c0 + c < n_chunks) {
-        for (int q = 0; q < n_groups; ++q) {
-          const unsigned m = __ballot_sync(0xffffffffu, grp[c] == q);
-          if (grp[c] == q) {
-            const int pos = s_base[q] + s_cnt[((c0 + c) * kRouteWarps + warp) * n_groups + q] +
-                            __popc(m & ((1u << lane) - 1u));
-            panel_row[pos] = (c0 + c) * kRouteThreads + tid;
-          }
-        }
-      }
-    }
-  }
-}
-
-// Copy every routed row into the packed K-major panel (one warp per panel row).
-__global__ void __launch_bounds__(256)
-pack_kernel(const __nv_bfloat16* __restrict__ hidden, const int* __restrict__ panel_row,
-            const RouteState* __restrict__ rs, __nv_bfloat16* __restrict__ panel, int d, unsigned* __restrict__ tau_slots, unsigned* __restrict__ tau_min) {
-  pdl_wait();
-  pdl_launch_dependents();
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int p = blockIdx.x * 8 + warp;
-  if (p >= rs->n_panel_rows) return;
-  if (tau_slots) {                                     // the encode's TopK bound starts empty
-    reinterpret_cast<uint4*>(tau_slots + (size_t)p * kTauSlots)[lane] = make_uint4(0u, 0u, 0u, 0u);
-    if (lane == 0) tau_min[p] = 0u;
-  }
-  const int t = panel_row[p];
-  uint4* dst = reinterpret_cast<uint4*>(panel + (size_t)p * d);
-  const int nvec = d >> 3;
-  if (t < 0) {   // padding rows of a tile: keep them finite
-    for (int i = lane; i < nvec; i += 32) dst[i] = make_uint4(0, 0, 0, 0);
-    return;
-  }
-  const uint4* src = reinterpret_cast<const uint4*>(hidden + (size_t)t * d);
-  for (int i = lane; i < nvec; i += 32) dst[i] = __ldg(src + i);
-}
-
-// 8-bit encoder: every routed row goes into the panel as E4M3 codes with a power-of-two row scale.
-// s = the smallest power of two with max|h_i| / s <= 448 (never below 2^-100; 1 for a row of zeros); h_i / s is
-// exact in fp32, the conversion rounds to nearest even.  One warp per row: a first pass for the largest
-// magnitude, a second one (the row is in L1 by then) for the codes.
-//   kSplit = false (MIX_FLAG_FP8_ACT): code_i = E4M3 nearest to h_i / s -- the encoder's input IS quantised.
-//   kSplit = true  (MIX_FLAG_FP8_W_ENC alone): the bf16 row is kept, as the sum of two E4M3 operands with the same
-//     scale: hi_i = E4M3 nearest to x = h_i / s, lo_i = E4M3 nearest to x - hi_i (exact subtraction).  A bf16 value
-//     has 8 significant bits, hi takes the leading 4 and the remainder has at most 4, so hi + lo = x exactly
-//     unless bits of x lie below 2^-9 (the subnormal step of E4M3), i.e. the error per element is at most
-//     2^-10 s <= 4.4e-6 max|h_i| and zero for |h_i| >= 2^-2 s.  The lo codes go to rows [lo_row0 + p] of the panel.
-template <bool kSplit>
-__global__ void __launch_bounds__(256)
-pack_e4m3_kernel(const __nv_bfloat16* __restrict__ hidden, const int* __restrict__ panel_row,
-                 const RouteState* __restrict__ rs, unsigned char* __restrict__ panel, float* __restrict__ act_scale, int d,
-                 unsigned* __restrict__ tau_slots, unsigned* __restrict__ tau_min, int lo_row0) {
-  pdl_wait();
-  pdl_launch_dependents();
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int p = blockIdx.x * 8 + warp;
-  if (p >= rs->n_panel_rows) return;
-  if (tau_slots) {                                     // the encode's TopK bound starts empty
-    reinterpret_cast<uint4*>(tau_slots + (size_t)p * kTauSlots)[lane] = make_uint4(0u, 0u, 0u, 0u);
-    if (lane == 0) tau_min[p] = 0u;
-  }
-  const int t = panel_row[p];
-  uint2* dst = reinterpret_cast<uint2*>(panel + (size_t)p * d);
-  uint2* dst_lo = reinterpret_cast<uint2*>(panel + ((size_t)lo_row0 + p) * d);
-  const int nvec = d >> 3;
-  if (t < 0) {   // padding rows of a tile
-    for (int i = lane; i < nvec; i += 32) {
-      dst[i] = make_uint2(0u, 0u);
-      if (kSplit) dst_lo[i] = make_uint2(0u, 0u);
-    }
-    if (lane == 0) act_scale[p] = 0.f;
-    return;
-  }
-  const uint4* src = reinterpret_cast<const uint4*>(hidden + (size_t)t * d);
-  unsigned m2 = 0u;                                     // two 15-bit magnitudes, compared as integers
-  for (int i = lane; i < nvec; i += 32) {
-    const uint4 q = __ldg(src + i);
-    m2 = __vmaxu2(m2, __vmaxu2(__vmaxu2(q.x & 0x7fff7fffu, q.y & 0x7fff7fffu), __vmaxu2(q.z & 0x7fff7fffu, q.w & 0x7fff7fffu)));
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) m2 = __vmaxu2(m2, __shfl_xor_sync(0xffffffffu, m2, o));
-  const unsigned a = max(m2 & 0xffffu, m2 >> 16);       // bf16 bits of max|h_i|: (1 + frac / 128) * 2^(E - 127)
-  int e = 0;
-  if (a != 0u) {
-    const int E = (int)(a >> 7) - 127, frac = (int)(a & 0x7fu);
-    e = max(E - (frac <= 96 ? 8 : 7), -100);            // 448 = 1.75 * 2^8, and 1.75 = 1 + 96 / 128
-  }
-  const float inv = __uint_as_float((unsigned)(127 - e) << 23);
-  if (lane == 0) act_scale[p] = __uint_as_float((unsigned)(127 + e) << 23);
-  for (int i = lane; i < nvec; i += 32) {
-    const uint4 q = __ldg(src + i);
-    const unsigned w[4] = {q.x, q.y, q.z, q.w};
-    unsigned short c[4], cl[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const float lo = __uint_as_float(w[u] << 16) * inv, hi = __uint_as_float(w[u] & 0xffff0000u) * inv;
-      c[u] = __nv_cvt_float2_to_fp8x2(make_float2(lo, hi), __NV_SATFINITE, __NV_E4M3);
-      if (kSplit) {
-        const float2 back = __half22float2(__half2(__nv_cvt_fp8x2_to_halfraw2(c[u], __NV_E4M3)));   // exact: E4M3 fits fp16
-        cl[u] = __nv_cvt_float2_to_fp8x2(make_float2(lo - back.x, hi - back.y), __NV_SATFINITE, __NV_E4M3);
-      }
-    }
-    dst[i] = make_uint2((unsigned)c[0] | ((unsigned)c[1] << 16), (unsigned)c[2] | ((unsigned)c[3] << 16));
-    if (kSplit) dst_lo[i] = make_uint2((unsigned)cl[0] | ((unsigned)cl[1] << 16), (unsigned)cl[2] | ((unsigned)cl[3] << 16));
-  }
-}
-
 // Router-logit steering: one thread per (row, expert).
 __global__ void __launch_bounds__(256)
 router_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
@@ -1017,31 +743,6 @@ cudaError_t launch_router(const Ctx* c, float* logits, int n_experts, int T, cud
   router_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates,
                                                             c->cfg.n_slots_max, logits, n_experts);
   return cudaGetLastError();
-}
-
-cudaError_t launch_route(const Ctx* c, int T, cudaStream_t s, unsigned long long cond, int use_cond) {
-  const int n_chunks = (c->cfg.T_max + kRouteThreads - 1) / kRouteThreads;
-  const size_t smem = (size_t)n_chunks * kRouteWarps * c->cfg.n_groups_max * sizeof(int);
-  route_kernel<<<1, kRouteThreads, smem, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates, c->cfg.n_slots_max,
-                                              c->d_groups, c->cfg.n_groups_max, c->d_panel_row, c->panel_rows_cap,
-                                              c->d_mtile_group, c->d_route, c->d_status, c->d_row_flag,
-                                              c->d_mtile_flag, c->d_n_flagged, c->d_row_group,
-                                              (c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) ? 1 : 0,
-                                              static_cast<cudaGraphConditionalHandle>(cond), use_cond, c->d_chain_next,
-                                              c->d_row_slot);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_pack(const Ctx* c, const __nv_bfloat16* hidden, cudaStream_t s) {
-  const int blocks = (c->panel_rows_cap + 7) / 8;
-  unsigned char* codes = reinterpret_cast<unsigned char*>(c->d_panel);
-  if (c->cfg.flags & MIX_FLAG_FP8_ACT)
-    return launch_pdl(kPdlPack, pack_e4m3_kernel<false>, dim3(blocks), dim3(256), 0, s, hidden, c->d_panel_row, c->d_route,
-                      codes, c->d_act_scale, c->cfg.d_model, c->d_tau, c->d_tau_min, 0);
-  if (c->cfg.flags & MIX_FLAG_FP8_W_ENC)      // hi codes in rows [0, P), lo codes in rows [P, 2P) of the same buffer
-    return launch_pdl(kPdlPack, pack_e4m3_kernel<true>, dim3(blocks), dim3(256), 0, s, hidden, c->d_panel_row, c->d_route,
-                      codes, c->d_act_scale, c->cfg.d_model, c->d_tau, c->d_tau_min, c->panel_rows_cap);
-  return launch_pdl(kPdlPack, pack_kernel, dim3(blocks), dim3(256), 0, s, hidden, c->d_panel_row, c->d_route, c->d_panel, c->cfg.d_model, c->d_tau, c->d_tau_min);
 }
 
 cudaError_t launch_compose_map(const Ctx* c, int T_live, int n_req, cudaStream_t s) {

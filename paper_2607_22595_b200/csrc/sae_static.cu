@@ -1,10 +1,10 @@
 // mix_sae_apply_static(): the SAE function of the hook for callers that must not allocate.
 //
 // Everything mix_create() would cudaMalloc for the SAE path (slot map, app / weight-set
-// tables, edit lists, routing state, the packed bf16 panel, the fp32 pre-activation scratch
-// and the TopK lists) lives here in ONE file-scope device array of fixed size.  The array is
+// tables, edit lists, routing state, the packed bf16 panel and the fp32 pre-activation
+// scratch) lives here in ONE file-scope device array of fixed size.  The array is
 // part of the library image: every GPU that loads libmix.so holds it until the process exits.
-// The call then runs the same routing, pack, encode (CUDA-core kernel), select and decode
+// The call then runs the same routing / pack, encode (CUDA-core kernel) and selection / decode
 // kernels as mix_apply(), pointed at that array.
 #include <stdio.h>
 #include <string.h>
@@ -39,11 +39,8 @@ constexpr size_t kOffMtileGroup = kOffPanelRow + align256(kStaticRows * sizeof(i
 constexpr size_t kOffRowGroup = kOffMtileGroup + 256;
 constexpr size_t kOffRowSlot = kOffRowGroup + align256(kStaticRows * sizeof(int));
 constexpr size_t kOffChainNext = kOffRowSlot + align256(kStaticRows * sizeof(int));
-constexpr size_t kOffRowDelta = kOffChainNext + 256;
-constexpr size_t kOffEditCoef = kOffRowDelta + align256(kStaticRows * sizeof(RowDelta));
-constexpr size_t kOffTopkIdx = kOffEditCoef + align256((size_t)kStaticRows * kMaxEdits * sizeof(float));
-constexpr size_t kOffTopkVal = kOffTopkIdx + align256((size_t)kStaticRows * kStaticK * sizeof(int));
-constexpr size_t kOffPanel = kOffTopkVal + align256((size_t)kStaticRows * kStaticK * sizeof(float));
+constexpr size_t kOffRowRec = kOffChainNext + 256;
+constexpr size_t kOffPanel = kOffRowRec + align256(kStaticRows * sizeof(RowRec));
 constexpr size_t kOffZ = kOffPanel + align256((size_t)kStaticRows * kStaticD * sizeof(__nv_bfloat16));
 constexpr size_t kScratchBytes = kOffZ + align256((size_t)kStaticRows * kStaticDsae * sizeof(float));
 static_assert(kScratchBytes < (6u << 20), "the header promises less than 6 MiB");
@@ -172,10 +169,7 @@ extern "C" int mix_sae_apply_static(void* hidden, int n_rows, int d_model, const
   c.d_row_group = reinterpret_cast<int*>(base + kOffRowGroup);
   c.d_row_slot = reinterpret_cast<int*>(base + kOffRowSlot);
   c.d_chain_next = reinterpret_cast<int*>(base + kOffChainNext);   // never read: the app entry carries no chain flag
-  c.d_row_delta = reinterpret_cast<RowDelta*>(base + kOffRowDelta);
-  c.d_edit_coef = reinterpret_cast<float*>(base + kOffEditCoef);
-  c.d_topk_idx = reinterpret_cast<int*>(base + kOffTopkIdx);
-  c.d_topk_val = reinterpret_cast<float*>(base + kOffTopkVal);
+  c.d_row_rec = reinterpret_cast<RowRec*>(base + kOffRowRec);
   c.d_panel = reinterpret_cast<__nv_bfloat16*>(base + kOffPanel);
   c.d_z = reinterpret_cast<float*>(base + kOffZ);
   c.panel_rows_cap = kStaticRows;
@@ -219,12 +213,9 @@ extern "C" int mix_sae_apply_static(void* hidden, int n_rows, int d_model, const
                                         c.d_edit_val, c.d_edit_mode);
   cudaError_t e = cudaGetLastError();
   __nv_bfloat16* h = static_cast<__nv_bfloat16*>(hidden);
-  if (e == cudaSuccess) e = launch_route(&c, n_rows, s);
-  if (e == cudaSuccess) e = launch_pack(&c, h, s);
+  if (e == cudaSuccess) e = launch_front(&c, h, n_rows, s);       // routing + row pack
   if (e == cudaSuccess) e = launch_encode_simt(&c, s);
-  if (e == cudaSuccess) e = launch_select(&c, false, s);
-  if (e == cudaSuccess) e = launch_decode(&c, h, s);
-  if (e == cudaSuccess) e = launch_decode_delta(&c, h, s);
+  if (e == cudaSuccess) e = launch_tail(&c, h, 1, s);             // selection, edits, decode, write-back
   if (e != cudaSuccess) return fail(errbuf, errbuf_len, MIX_ERR_CUDA, "CUDA error %lld while enqueuing the static SAE call", (long long)e);
   return MIX_OK;
 }

@@ -1,0 +1,748 @@
+// Everything behind the SAE encode, in one launch: activation / selection, per-feature edits, sparse decode,
+// error term and write-back (with a second launch of the same kernel for rows that need the exact fallback).
+//
+//   tail_kernel, row role (one CTA per packed row, grid-stride):
+//     TopK row   : exact TopK -- from the per-tile candidates of the fused encode epilogue (radix refinement on
+//                  order-preserving keys, then a sort of the few composites left; ties go to the lower feature
+//                  id), or from the fp32 pre-activations Z when the encode wrote those -- then, with the list
+//                  still in shared memory, the edits and the decode of the row:
+//                    error term on : h' = h + sum over edited j of (f'_j - f_j) W_dec[j]
+//                    error term off: h' = b_dec + sum_j f'_j W_dec[j]
+//                  A row whose candidates cannot prove the TopK is flagged and left to the fallback launch.
+//     other rows : the active count if asked for; rows whose app replaces the residual are rebuilt from Z.
+//   tail_kernel, delta role (a CTA owns 4 consecutive packed rows x 2048 columns):
+//     ReLU / JumpReLU rows that keep the error term: f_j of the edited features from Z, then the deltas.
+//     Neighbouring packed rows mostly share a request, hence an edit list, so each edited W_dec row is
+//     fetched once per CTA and applied to its rows with per-row coefficients.
+// The two roles own disjoint rows, so they run side by side in one grid.
+#include "mix_internal.h"
+
+namespace mix {
+
+namespace {
+
+// ---------------------------------------------------------------------------------------
+// selection
+// ---------------------------------------------------------------------------------------
+constexpr int kTailThreads = 256;
+constexpr int kCand = 1024;        // composites sorted in shared memory (>= k_max)
+constexpr int kBins = 2048;
+static_assert(kCand >= kMaxK, "the sort buffer must hold a full TopK list");
+
+// In-place bitonic sort of the first n entries of `a` (shared memory), descending.  Entries up
+// to the next power of two are overwritten with 0 (the smallest composite key).
+__device__ void bitonic_sort_desc(unsigned long long* a, int n) {
+  const int tid = threadIdx.x;
+  int n2 = 1;
+  while (n2 < n) n2 <<= 1;
+  for (int i = n + tid; i < n2; i += kTailThreads) a[i] = 0ull;
+  __syncthreads();
+  for (int size = 2; size <= n2; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int i = tid; i < n2 / 2; i += kTailThreads) {
+        const int lo = 2 * i - (i & (stride - 1));
+        const int hi = lo + stride;
+        const bool desc = ((lo & size) == 0);
+        const unsigned long long x = a[lo], y = a[hi];
+        if ((x < y) == desc) {
+          a[lo] = y;
+          a[hi] = x;
+        }
+      }
+      __syncthreads();
+    }
+  }
+}
+
+// Largest digit D with count(digit >= D) >= need, and the count of digits > D.  One warp, two
+// levels: each lane sums a run of n_bins / 32 bins (largest digits in lane 0) and a warp scan
+// finds the run where the running count reaches `need`; then the 32 lanes split that run.
+__device__ void find_digit(const int* hist, int n_bins, int need, int* s_out) {
+  const int lane = threadIdx.x & 31;
+  const int per = n_bins / 32;                  // 64 or 32: a multiple of 4
+  const int hi = n_bins - lane * per;           // this lane's run is [hi - per, hi)
+  int sum = 0;
+  const int4* h4 = reinterpret_cast<const int4*>(hist + hi - per);
+  for (int i = 0; i < per / 4; ++i) {
+    const int4 v = h4[i];
+    sum += v.x + v.y + v.z + v.w;
+  }
+  int incl = sum;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  const int excl = incl - sum;                  // elements in bins above this lane's run
+  const unsigned hit = __ballot_sync(0xffffffffu, excl < need && incl >= need);
+  const int L = __ffs(hit) - 1;                 // exactly one lane (need <= total count)
+  const int run_hi = n_bins - L * per;
+  const int above_run = __shfl_sync(0xffffffffu, excl, L);
+  // level 2: lane l takes bins run_hi - 1 - l*w .. run_hi - (l+1)*w, w = per / 32 (2 or 1), descending
+  const int w = per / 32;
+  int c0 = hist[run_hi - 1 - lane * w], c1 = w == 2 ? hist[run_hi - 2 - lane * w] : 0;
+  int inc2 = c0 + c1;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, inc2, o);
+    if (lane >= o) inc2 += y;
+  }
+  const int before = above_run + inc2 - (c0 + c1);     // elements in bins above this lane's bins
+  if (before < need && before + c0 + c1 >= need) {
+    if (before + c0 >= need) {
+      s_out[0] = run_hi - 1 - lane * w;
+      s_out[1] = before;
+    } else {
+      s_out[0] = run_hi - 2 - lane * w;
+      s_out[1] = before + c0;
+    }
+  }
+}
+
+// The two places a row's values can come from.
+struct ZRow {            // all pre-activations of the row; position = feature id
+  const float* z;
+  int n;
+  __device__ __forceinline__ unsigned key(int i) const { return f2key(z[i]); }
+  __device__ __forceinline__ unsigned id(int i) const { return (unsigned)i; }
+};
+struct CandRow {         // per-tile candidates of the fused encode epilogue
+  const float* v;
+  const int* j;
+  int n;
+  __device__ __forceinline__ unsigned key(int i) const { return f2key(v[i]); }
+  __device__ __forceinline__ unsigned id(int i) const { return (unsigned)j[i]; }
+};
+
+struct SelShared {
+  __align__(16) int hist[kBins];            // radix histogram; afterwards the output of the counting sort (kBins / 2 composites)
+  unsigned long long cand[kCand];
+  int n, res[2], count;
+};
+
+// Append `c` to sh.cand for every thread whose `take` is set: one shared-memory atomic per warp
+// (the lanes of a warp are ranked by ballot), not one per element on a single hot counter.
+// Every thread of the warp must call this.
+__device__ __forceinline__ void push_cand(SelShared& sh, bool take, unsigned long long c) {
+  const unsigned m = __ballot_sync(0xffffffffu, take);
+  if (m == 0u) return;
+  const int lane = threadIdx.x & 31, leader = __ffs(m) - 1;
+  int base = 0;
+  if (lane == leader) base = atomicAdd(&sh.n, __popc(m));
+  base = __shfl_sync(0xffffffffu, base, leader);
+  if (take) {
+    const int pos = base + __popc(m & ((1u << lane) - 1u));
+    if (pos < kCand) sh.cand[pos] = c;
+  }
+}
+
+// Collect into sh.cand (unsorted composites key << 32 | ~id) a set that contains the k largest
+// entries of `src` under the order (value descending, id ascending): radix refinement on the
+// order-preserving keys, up to 11 bits at a time, until what is still undecided fits the buffer.
+// The first digit starts at the highest bit in which the keys differ at all (the candidates of a
+// row are its largest values: they share sign, exponent and often leading mantissa bits, and a
+// digit taken from those bits would put them all into a handful of bins -- thousands of atomic
+// increments on the same few counters).  If more than the buffer's worth of entries tie EXACTLY
+// with the k-th value:
+//   ORDERED sources (position order = id order) finish with an index-ordered pass and return 2;
+//   other sources return 0 (the caller falls back).
+// Returns 1 in the ordinary case.  Every thread of the CTA must call this.
+template <bool ORDERED, class Src>
+__device__ int radix_collect(const Src& src, int k, SelShared& sh) {
+  const int tid = threadIdx.x, n = src.n;
+  // range of the keys
+  unsigned kmin = 0xffffffffu, kmax = 0u;
+  for (int i = tid; i < n; i += kTailThreads) {
+    const unsigned key = src.key(i);
+    kmin = min(kmin, key);
+    kmax = max(kmax, key);
+  }
+  kmin = __reduce_min_sync(0xffffffffu, kmin);
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+  if ((tid & 31) == 0) {
+    sh.hist[tid >> 5] = (int)kmin;
+    sh.hist[32 + (tid >> 5)] = (int)kmax;
+  }
+  __syncthreads();
+  for (int w = 0; w < kTailThreads / 32; ++w) {
+    kmin = min(kmin, (unsigned)sh.hist[w]);
+    kmax = max(kmax, (unsigned)sh.hist[32 + w]);
+  }
+  __syncthreads();
+  int hi_bit = (kmax ^ kmin) ? 32 - __clz(kmax ^ kmin) : 0;     // bits [0, hi_bit) vary; the rest is common
+  unsigned prefix = hi_bit >= 32 ? 0u : (kmax >> hi_bit);       // digits fixed so far (= key >> hi_bit of the k-th)
+  int need = k;                 // winners still to be found inside the prefix set
+  // Refinement goes on while the undecided set is much larger than k, even if it would already fit
+  // the buffer: one more histogram pass costs far less than sorting a thousand composites.
+  const int enough = max(2 * k, 128);
+  bool done = false;
+  while (hi_bit > 0) {
+    const int width = min(11, hi_bit), shift = hi_bit - width, nb = 1 << width;
+    for (int b = tid; b < kBins; b += kTailThreads) sh.hist[b] = 0;     // digits >= nb do not occur: their bins stay 0
+    __syncthreads();
+    for (int i = tid; i < n; i += kTailThreads) {
+      const unsigned key = src.key(i);
+      if (hi_bit >= 32 || (key >> hi_bit) == prefix) atomicAdd(&sh.hist[(key >> shift) & (nb - 1)], 1);
+    }
+    __syncthreads();
+    if (tid < 32) find_digit(sh.hist, kBins, need, sh.res);
+    __syncthreads();
+    const int D = sh.res[0], above = sh.res[1];
+    const int in_bin = sh.hist[D];
+    need -= above;
+    prefix = (prefix << width) | (unsigned)D;
+    hi_bit = shift;
+    done = (k - need) + in_bin <= kCand;
+    __syncthreads();
+    if (done && (k - need) + in_bin <= enough) break;
+  }
+  if (tid == 0) sh.n = 0;
+  __syncthreads();
+  const int n_up = (n + kTailThreads - 1) / kTailThreads * kTailThreads;    // whole warps take part in every ballot
+  if (done) {
+    for (int i = tid; i < n_up; i += kTailThreads) {
+      const unsigned key = i < n ? src.key(i) : 0u;
+      const bool take = i < n && (key >> hi_bit) >= prefix;
+      push_cand(sh, take, take ? (((unsigned long long)key << 32) | (0xffffffffu - src.id(i))) : 0ull);
+    }
+    __syncthreads();
+    return 1;
+  }
+  if constexpr (!ORDERED) {
+    return 0;
+  } else {
+  // every larger key, then the `need` lowest ids among the exact ties, in index order
+  for (int i = tid; i < n_up; i += kTailThreads) {
+    const unsigned key = i < n ? src.key(i) : 0u;
+    const bool take = i < n && key > prefix;
+    push_cand(sh, take, take ? (((unsigned long long)key << 32) | (0xffffffffu - src.id(i))) : 0ull);
+  }
+  __syncthreads();
+  int taken = 0;               // uniform across the block
+  for (int i0 = 0; i0 < n && taken < need; i0 += kTailThreads) {
+    const int i = i0 + tid;
+    const bool eq = i < n && src.key(i) == prefix;
+    const unsigned m = __ballot_sync(0xffffffffu, eq);
+    if ((tid & 31) == 0) sh.hist[tid >> 5] = __popc(m);
+    __syncthreads();
+    int before = 0, total = 0;
+    for (int w = 0; w < kTailThreads / 32; ++w) {
+      const int c = sh.hist[w];
+      if (w < (tid >> 5)) before += c;
+      total += c;
+    }
+    const int rank = taken + before + __popc(m & ((1u << (tid & 31)) - 1u));
+    if (eq && rank < need) {
+      const int pos = atomicAdd(&sh.n, 1);
+      sh.cand[pos] = ((unsigned long long)prefix << 32) | (0xffffffffu - src.id(i));
+    }
+    taken += total;
+    __syncthreads();
+  }
+  __syncthreads();
+  return 2;
+  }
+}
+
+
+// The sh.n composites of sh.cand in descending order.  Up to one composite per thread they are sorted by
+// counting (composites are distinct: the rank of one is the number of larger ones; one pass over shared memory
+// and one barrier, where the bitonic network needs dozens of barriers); longer lists take the network.
+// Returns where the sorted list is.  Every thread of the CTA must call this.
+__device__ const unsigned long long* sort_desc(SelShared& sh) {
+  const int tid = threadIdx.x, n = sh.n;
+  if (n <= kTailThreads) {
+    unsigned long long* out = reinterpret_cast<unsigned long long*>(sh.hist);
+    if (tid < n) {
+      const unsigned long long c = sh.cand[tid];
+      int rank = 0;
+      for (int j = 0; j < n; ++j) rank += sh.cand[j] > c;
+      out[rank] = c;
+    }
+    __syncthreads();
+    return out;
+  }
+  bitonic_sort_desc(sh.cand, n);
+  return sh.cand;
+}
+
+__device__ __forceinline__ int comp_id(unsigned long long c) { return (int)(0xffffffffu - (unsigned)(c & 0xffffffffull)); }
+__device__ __forceinline__ float comp_val(unsigned long long c) { return key2f((unsigned)(c >> 32)); }
+
+// Read-out of a row's TopK: ids in order of decreasing pre-activation, the pre-activations, the active count.
+__device__ void emit_topk(const unsigned long long* a, int k, int k_max, int t, int* __restrict__ out_idx,
+                          float* __restrict__ out_val, int* __restrict__ out_n_active, int* s_count) {
+  const int tid = threadIdx.x;
+  if (out_idx == nullptr && out_val == nullptr && out_n_active == nullptr) return;
+  int pos_cnt = 0;
+  for (int i = tid; i < k; i += kTailThreads) {
+    const unsigned long long c = a[i];
+    const float v = comp_val(c);
+    if (out_idx) out_idx[(size_t)t * k_max + i] = comp_id(c);
+    if (out_val) out_val[(size_t)t * k_max + i] = v;
+    pos_cnt += v > 0.f;
+  }
+  if (out_n_active) {
+    if (tid == 0) *s_count = 0;
+    __syncthreads();
+    pos_cnt = __reduce_add_sync(0xffffffffu, pos_cnt);
+    if ((tid & 31) == 0) atomicAdd(s_count, pos_cnt);
+    __syncthreads();
+    if (tid == 0) out_n_active[t] = *s_count;
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// decode
+// ---------------------------------------------------------------------------------------
+constexpr int kDecList = 1024 + kMaxEdits;     // >= k_max + r_max
+constexpr int kDecU = 4;                       // 16-byte column vectors per thread: 256 x 4 x 8 = 8192 columns
+
+__device__ __forceinline__ void axpy8(float* acc, float c, const uint4& q) {
+  const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&q);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 t = __bfloat1622float2(p[i]);
+    acc[2 * i] = fmaf(c, t.x, acc[2 * i]);
+    acc[2 * i + 1] = fmaf(c, t.y, acc[2 * i + 1]);
+  }
+}
+
+// acc += sum_e coef[e] * W_dec[feat[e], :] over this thread's column vectors (four 16-byte loads in flight per
+// thread and entry; the CTA's other warps and the SM's other CTAs cover the latency).  Entries with a zero
+// coefficient are not fetched.
+__device__ __forceinline__ void accumulate_list(float (*acc)[8], const float* coef, const int* feat, int n,
+                                                const __nv_bfloat16* __restrict__ W_dec, int d, int nvec) {
+  const int tid = threadIdx.x;
+#pragma unroll 1
+  for (int e = 0; e < n; ++e) {
+    const float c = coef[e];
+    if (c == 0.f) continue;
+    const uint4* row = reinterpret_cast<const uint4*>(W_dec + (size_t)feat[e] * d);
+    uint4 q[kDecU];
+#pragma unroll
+    for (int u = 0; u < kDecU; ++u) {
+      const int v = tid + u * kTailThreads;
+      q[u] = v < nvec ? __ldg(row + v) : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int u = 0; u < kDecU; ++u) axpy8(acc[u], c, q[u]);
+  }
+}
+
+__device__ __forceinline__ void store_row(uint4* hrow, float (*acc)[8], int nvec) {
+#pragma unroll
+  for (int u = 0; u < kDecU; ++u) {
+    const int v = threadIdx.x + u * kTailThreads;
+    if (v < nvec) {
+      uint4 q;
+      __nv_bfloat162* pp = reinterpret_cast<__nv_bfloat162*>(&q);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) pp[i] = __floats2bfloat162_rn(acc[u][2 * i], acc[u][2 * i + 1]);
+      hrow[v] = q;
+    }
+  }
+}
+
+enum { kTailCand = 0, kTailZ = 1, kTailFallback = 2 };
+
+struct TailArgs {
+  __nv_bfloat16* hidden;
+  int d;
+  const float* Z;
+  long long ldz;
+  const RowRec* row_rec;
+  const RouteState* rs;
+  const GroupEntry* groups;
+  const int* edit_idx;
+  const float* edit_val;
+  const unsigned char* edit_mode;
+  int r_max, k_max;
+  const float* cand_val;
+  const int* cand_idx;
+  const float* cand_ninth;
+  int cand_tiles;
+  int* out_idx;
+  float* out_val;
+  int* out_n_active;
+  int* row_flag;
+  int* mtile_flag;
+  int* n_flagged;
+  unsigned* status;
+  int mode;                 // kTailCand: TopK from the encode's candidates; kTailZ: TopK from Z; kTailFallback: flagged rows only, from Z
+  int n_row_ctas;           // CTAs [0, n_row_ctas) take the row role, the rest the delta role
+  int n_col_slices;         // delta role: ceil(d / 2048)
+};
+
+struct RowShared {
+  SelShared sel;
+  float coef[kDecList];
+  int feat[kDecList];
+  int eidx[kMaxEdits];
+  float ef[kMaxEdits];
+  int n_list;
+};
+
+// Row role.
+__device__ void tail_rows(const TailArgs& a, RowShared& sh) {
+  const int tid = threadIdx.x;
+  const int n_rows = a.rs->n_panel_rows;
+  const int d = a.d, nvec = d >> 3;
+  for (int p = blockIdx.x; p < n_rows; p += a.n_row_ctas) {
+    const RowRec rec = a.row_rec[p];
+    const int t = rec.t;
+    if (t < 0) continue;                               // padding row of a tile (uniform across the CTA, like every branch below)
+    // (the weight-set entry field by field, not as a struct held in registers across the whole row)
+    const GroupEntry* gp = a.groups + (rec.group_flags & kRecGroupMask);
+    const int act = gp->act;
+    const bool add_error = (rec.group_flags & kRecAddError) != 0;
+    const bool topk = act == MIX_SAE_TOPK;
+    if (a.mode == kTailFallback && !(topk && a.row_flag[p])) continue;
+    const int S = (int)gp->d_sae, k = gp->k;
+    const float* z = a.Z + (size_t)p * a.ldz;
+    const unsigned long long* sorted = nullptr;
+    if (topk) {
+      if (a.mode == kTailCand) {
+        // Every (row, feature tile) contributed its 8 largest pre-activations and its 9th.  The k largest
+        // candidates are the row's TopK unless some tile's 9th value reaches the k-th candidate, i.e. that tile
+        // may hide a winner (or an exact tie whose order matters): such rows are flagged, their row tiles are
+        // re-encoded to Z and the fallback launch selects exactly.
+        const int n_tiles = S / kTileN, n = n_tiles * kCandPerTile;
+        bool flag = n < k;                             // uniform
+        if (!flag) {
+          CandRow src{a.cand_val + (size_t)p * a.cand_tiles * kCandPerTile, a.cand_idx + (size_t)p * a.cand_tiles * kCandPerTile, n};
+          flag = radix_collect<false>(src, k, sh.sel) == 0;
+        }
+        if (!flag) {
+          sorted = sort_desc(sh.sel);
+          const unsigned kth = (unsigned)(sorted[k - 1] >> 32);
+          const float* ninth = a.cand_ninth + (size_t)p * a.cand_tiles;
+          int over = 0;
+          for (int i = tid; i < n_tiles; i += kTailThreads) over |= f2key(ninth[i]) >= kth;
+          flag = __syncthreads_or(over) != 0;
+        }
+        if (flag) {
+          if (tid == 0) {
+            a.row_flag[p] = 1;
+            a.mtile_flag[p / kTileM] = 1;
+            atomicAdd(a.n_flagged, 1);
+          }
+          __syncthreads();
+          continue;
+        }
+      } else {
+        ZRow src{z, S};
+        const int how = radix_collect<true>(src, k, sh.sel);
+        if (how == 2 && tid == 0) atomicOr(a.status, MIX_STATUS_TOPK_GENERAL);
+        sorted = sort_desc(sh.sel);
+      }
+      emit_topk(sorted, k, a.k_max, t, a.out_idx, a.out_val, a.out_n_active, &sh.sel.count);
+    } else {
+      if (a.out_n_active != nullptr) {
+        int cnt = 0;
+        const float* theta = gp->theta;
+        for (int j = tid; j < S; j += kTailThreads) {
+          const float v = z[j];
+          cnt += act == MIX_SAE_RELU ? v > 0.f : (v > theta[j] && v > 0.f);
+        }
+        if (tid == 0) sh.sel.count = 0;
+        __syncthreads();
+        cnt = __reduce_add_sync(0xffffffffu, cnt);
+        if ((tid & 31) == 0) atomicAdd(&sh.sel.count, cnt);
+        __syncthreads();
+        if (tid == 0) a.out_n_active[t] = sh.sel.count;
+      }
+      if (add_error) {                                 // the delta role's row
+        __syncthreads();
+        continue;
+      }
+    }
+    // ---- edits and decode of this row
+    const int slot = rec.slot, n_edit = rec.n_edit;
+    uint4* hrow = reinterpret_cast<uint4*>(a.hidden + (size_t)t * d);
+    const __nv_bfloat16* W_dec = gp->W_dec;
+    if (tid < n_edit) {
+      sh.eidx[tid] = a.edit_idx[slot * a.r_max + tid];
+      sh.ef[tid] = 0.f;
+    }
+    __syncthreads();
+    float acc[kDecU][8];
+    if (add_error) {
+      // (TopK rows only.)  f_j of an edited feature comes from the row's TopK list, 0 if it was not selected
+      for (int i = tid; i < k; i += kTailThreads) {
+        const int id = comp_id(sorted[i]);
+        for (int e = 0; e < n_edit; ++e)
+          if (sh.eidx[e] == id) sh.ef[e] = fmaxf(comp_val(sorted[i]), 0.f);
+      }
+      __syncthreads();
+      float delta = 0.f;
+      if (tid < n_edit) {
+        const int j = sh.eidx[tid];
+        bool alive = true;                             // a later entry for the same feature wins
+        for (int e2 = tid + 1; e2 < n_edit; ++e2) alive = alive && (sh.eidx[e2] != j);
+        const float fnew = a.edit_mode[slot * a.r_max + tid] == MIX_EDIT_CLAMP ? a.edit_val[slot * a.r_max + tid] : 0.f;
+        delta = alive ? fnew - sh.ef[tid] : 0.f;
+        sh.coef[tid] = delta;
+        sh.feat[tid] = j;
+      }
+      if (__syncthreads_or(delta != 0.f)) {            // no effective edit: the row stays as it is, bit for bit
+#pragma unroll
+        for (int u = 0; u < kDecU; ++u) {
+          const int v = tid + u * kTailThreads;
+          const uint4 hq = v < nvec ? hrow[v] : make_uint4(0u, 0u, 0u, 0u);
+          const __nv_bfloat162* pp = reinterpret_cast<const __nv_bfloat162*>(&hq);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float2 f2 = __bfloat1622float2(pp[i]);
+            acc[u][2 * i] = f2.x;
+            acc[u][2 * i + 1] = f2.y;
+          }
+        }
+        accumulate_list(acc, sh.coef, sh.feat, n_edit, W_dec, d, nvec);
+        store_row(hrow, acc, nvec);
+      }
+      __syncthreads();
+      continue;
+    }
+    // the app replaces the residual: h' = b_dec + sum_j f'_j W_dec[j]
+    if (tid < n_edit) {       // edited features contribute f' (live entries only)
+      const int j = sh.eidx[tid];
+      bool alive = true;
+      for (int e2 = tid + 1; e2 < n_edit; ++e2) alive = alive && (sh.eidx[e2] != j);
+      const float fnew = a.edit_mode[slot * a.r_max + tid] == MIX_EDIT_CLAMP ? a.edit_val[slot * a.r_max + tid] : 0.f;
+      sh.coef[tid] = alive ? fnew : 0.f;
+      sh.feat[tid] = j;
+    }
+    {
+      const float* b_dec = gp->b_dec;
+#pragma unroll
+      for (int u = 0; u < kDecU; ++u) {
+        const int v = tid + u * kTailThreads;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[u][i] = (b_dec && v < nvec) ? b_dec[v * 8 + i] : 0.f;
+      }
+    }
+    if (topk) {
+      for (int i = tid; i < k; i += kTailThreads) {
+        const int j = comp_id(sorted[i]);
+        bool edited = false;
+        for (int e = 0; e < n_edit; ++e) edited = edited || (sh.eidx[e] == j);
+        // an id outside the SAE can only come from a call whose encode timed out: never address with it
+        const bool in_range = (unsigned)j < (unsigned)S;
+        sh.coef[n_edit + i] = (edited || !in_range) ? 0.f : fmaxf(comp_val(sorted[i]), 0.f);
+        sh.feat[n_edit + i] = in_range ? j : 0;
+      }
+      __syncthreads();
+      accumulate_list(acc, sh.coef, sh.feat, n_edit + k, W_dec, d, nvec);
+    } else {
+      const float* theta = gp->theta;
+      __syncthreads();
+      accumulate_list(acc, sh.coef, sh.feat, n_edit, W_dec, d, nvec);
+      // dense scan of the activations in chunks; active, unedited features are compacted
+      // into shared memory and applied chunk by chunk
+      if (tid == 0) sh.n_list = 0;
+      __syncthreads();
+      for (int c0 = 0; c0 < S; c0 += 1024) {
+        for (int j = c0 + tid; j < min(S, c0 + 1024); j += kTailThreads) {
+          const float zj = z[j];
+          const float f = act == MIX_SAE_RELU ? fmaxf(zj, 0.f) : (zj > theta[j] ? zj : 0.f);
+          if (f != 0.f) {
+            bool edited = false;
+            for (int e = 0; e < n_edit; ++e) edited = edited || (sh.eidx[e] == j);
+            if (!edited) {
+              const int pos = atomicAdd(&sh.n_list, 1);
+              sh.coef[pos] = f;
+              sh.feat[pos] = j;
+            }
+          }
+        }
+        __syncthreads();
+        accumulate_list(acc, sh.coef, sh.feat, sh.n_list, W_dec, d, nvec);
+        __syncthreads();
+        if (tid == 0) sh.n_list = 0;
+        __syncthreads();
+      }
+    }
+    store_row(hrow, acc, nvec);
+    __syncthreads();                                   // the shared lists are reused by the next row
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// delta role: ReLU / JumpReLU rows with the error term
+// ---------------------------------------------------------------------------------------
+constexpr int kDlRows = 4;
+constexpr int kDlBatch = 8;
+constexpr int kDlEntries = kDlRows * kMaxEdits;
+
+struct DeltaShared {
+  __align__(16) float coef[kDlEntries + kDlBatch][kDlRows];
+  const uint4* wrow[kDlEntries + kDlBatch];
+  int idx[kMaxEdits];
+  int t[kDlRows], slot[kDlRows], n_edit[kDlRows], grp[kDlRows], changed[kDlRows];
+};
+
+__device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int cta) {
+  const int tid = threadIdx.x;
+  const int rg = cta / a.n_col_slices, cs = cta - rg * a.n_col_slices;
+  const int p0 = rg * kDlRows;
+  const int n_rows = a.rs->n_panel_rows;
+  if (p0 >= n_rows) return;
+  if (tid < kDlRows) {
+    const int p = p0 + tid;                              // in bounds: the panel capacity is a multiple of 128
+    const RowRec rec = a.row_rec[p];
+    const int g = rec.group_flags & kRecGroupMask;
+    bool on = p < n_rows && rec.t >= 0 && (rec.group_flags & kRecAddError) && rec.n_edit > 0;
+    if (on) on = a.groups[g].act != MIX_SAE_TOPK;
+    sh.t[tid] = on ? rec.t : -1;
+    sh.slot[tid] = on ? rec.slot : -1;
+    sh.n_edit[tid] = rec.n_edit;
+    sh.grp[tid] = g;
+    sh.changed[tid] = 0;
+  }
+  __syncthreads();
+  bool any = false;
+#pragma unroll
+  for (int r = 0; r < kDlRows; ++r) any = any || sh.slot[r] >= 0;
+  if (!any) return;
+  const int d = a.d;
+  const int v = cs * kTailThreads + tid;                 // this thread's 16-byte column vector
+  const bool in_cols = v < (d >> 3);
+  uint4 hraw[kDlRows];
+#pragma unroll
+  for (int r = 0; r < kDlRows; ++r) {
+    const int t = sh.t[r];
+    hraw[r] = make_uint4(0u, 0u, 0u, 0u);
+    if (t >= 0 && in_cols) hraw[r] = reinterpret_cast<const uint4*>(a.hidden + (size_t)t * d)[v];
+  }
+  // entries: the edit lists of the distinct slots, one after the other; thread e of a slot works out entry e
+  // for every row of that slot (the coefficient of a row of another slot is zero)
+  int n_entries = 0;                                    // CTA-uniform
+  for (int r = 0; r < kDlRows; ++r) {
+    const int slot = sh.slot[r];
+    bool first = slot >= 0;
+    for (int r2 = 0; r2 < r; ++r2) first = first && sh.slot[r2] != slot;
+    if (!first) continue;
+    const int n_edit = sh.n_edit[r];
+    if (tid < n_edit) sh.idx[tid] = a.edit_idx[slot * a.r_max + tid];
+    __syncthreads();
+    if (tid < n_edit) {
+      const GroupEntry ge = a.groups[sh.grp[r]];
+      const int j = sh.idx[tid];
+      bool alive = true;                                 // a later entry for the same feature wins
+      for (int e2 = tid + 1; e2 < n_edit; ++e2) alive = alive && (sh.idx[e2] != j);
+      const float fnew = a.edit_mode[slot * a.r_max + tid] == MIX_EDIT_CLAMP ? a.edit_val[slot * a.r_max + tid] : 0.f;
+      const float theta = ge.act == MIX_SAE_JUMPRELU ? ge.theta[j] : 0.f;
+      float c[kDlRows];
+#pragma unroll
+      for (int r2 = 0; r2 < kDlRows; ++r2) {
+        c[r2] = 0.f;
+        if (sh.slot[r2] == slot && alive) {
+          const float zj = a.Z[(size_t)(p0 + r2) * a.ldz + j];
+          const float f = ge.act == MIX_SAE_RELU ? fmaxf(zj, 0.f) : (zj > theta ? zj : 0.f);
+          c[r2] = fnew - f;
+          if (c[r2] != 0.f) sh.changed[r2] = 1;
+        }
+      }
+#pragma unroll
+      for (int r2 = 0; r2 < kDlRows; ++r2) sh.coef[n_entries + tid][r2] = c[r2];
+      sh.wrow[n_entries + tid] = reinterpret_cast<const uint4*>(ge.W_dec + (size_t)j * d);
+    }
+    n_entries += n_edit;
+    __syncthreads();
+  }
+  // pad to a whole batch: repeats of the last decoder row with zero coefficients
+  if (tid < kDlBatch) {
+    sh.wrow[n_entries + tid] = sh.wrow[n_entries - 1];
+#pragma unroll
+    for (int r2 = 0; r2 < kDlRows; ++r2) sh.coef[n_entries + tid][r2] = 0.f;
+  }
+  __syncthreads();
+  if (!in_cols) return;
+  float acc[kDlRows][8];
+#pragma unroll
+  for (int r = 0; r < kDlRows; ++r) {
+    const __nv_bfloat162* pp = reinterpret_cast<const __nv_bfloat162*>(&hraw[r]);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 f2 = __bfloat1622float2(pp[i]);
+      acc[r][2 * i] = f2.x;
+      acc[r][2 * i + 1] = f2.y;
+    }
+  }
+  // kDlBatch decoder rows in flight per thread: the loop is bound by load latency, not arithmetic
+  for (int e0 = 0; e0 < n_entries; e0 += kDlBatch) {
+    uint4 q[kDlBatch];
+#pragma unroll
+    for (int u = 0; u < kDlBatch; ++u) q[u] = __ldg(sh.wrow[e0 + u] + v);
+#pragma unroll
+    for (int u = 0; u < kDlBatch; ++u) {
+      const float4 c4 = *reinterpret_cast<const float4*>(&sh.coef[e0 + u][0]);
+      axpy8(acc[0], c4.x, q[u]);
+      axpy8(acc[1], c4.y, q[u]);
+      axpy8(acc[2], c4.z, q[u]);
+      axpy8(acc[3], c4.w, q[u]);
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < kDlRows; ++r) {
+    if (sh.slot[r] < 0 || !sh.changed[r]) continue;     // no effective edit: the row stays bit-exact
+    uint4 o;
+    __nv_bfloat162* pp = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) pp[i] = __floats2bfloat162_rn(acc[r][2 * i], acc[r][2 * i + 1]);
+    reinterpret_cast<uint4*>(a.hidden + (size_t)sh.t[r] * d)[v] = o;
+  }
+}
+
+__global__ void __launch_bounds__(kTailThreads, 3)
+tail_kernel(const TailArgs a) {
+  pdl_wait();
+  pdl_launch_dependents();
+  __shared__ RowShared s_row;
+  __shared__ DeltaShared s_delta;
+  if (a.mode == kTailFallback && *a.n_flagged == 0) return;   // nothing was flagged: the usual case
+  if ((int)blockIdx.x < a.n_row_ctas)
+    tail_rows(a, s_row);
+  else
+    tail_delta(a, s_delta, (int)blockIdx.x - a.n_row_ctas);
+}
+
+}  // namespace
+
+// mode: 0 the main launch behind the tensor-core encode, 1 the main launch behind the CUDA-core encode (TopK
+// straight from Z), 2 the fallback launch (flagged rows only; returns at once when there are none).
+cudaError_t launch_tail(const Ctx* c, __nv_bfloat16* hidden, int mode, cudaStream_t s) {
+  TailArgs a;
+  a.hidden = hidden;
+  a.d = c->cfg.d_model;
+  a.Z = c->d_z;
+  a.ldz = c->cfg.d_sae_max;
+  a.row_rec = c->d_row_rec;
+  a.rs = c->d_route;
+  a.groups = c->d_groups;
+  a.edit_idx = c->d_edit_idx;
+  a.edit_val = c->d_edit_val;
+  a.edit_mode = c->d_edit_mode;
+  a.r_max = c->cfg.r_max;
+  a.k_max = c->cfg.k_max;
+  a.cand_val = c->d_cand_val;
+  a.cand_idx = c->d_cand_idx;
+  a.cand_ninth = c->d_cand_ninth;
+  a.cand_tiles = c->cand_tiles;
+  a.out_idx = c->out_topk_idx;
+  a.out_val = c->out_topk_val;
+  a.out_n_active = c->out_n_active;
+  a.row_flag = c->d_row_flag;
+  a.mtile_flag = c->d_mtile_flag;
+  a.n_flagged = c->d_n_flagged;
+  a.status = c->d_status;
+  a.mode = mode;
+  const int n_sms = c->n_sms > 0 ? c->n_sms : 148;
+  a.n_row_ctas = c->panel_rows_cap < n_sms * 6 ? c->panel_rows_cap : n_sms * 6;
+  a.n_col_slices = (c->cfg.d_model / 8 + kTailThreads - 1) / kTailThreads;
+  const int n_delta = mode == kTailFallback ? 0 : (c->panel_rows_cap / kDlRows) * a.n_col_slices;
+  return launch_pdl(kPdlTail, tail_kernel, dim3(a.n_row_ctas + n_delta), dim3(kTailThreads), 0, s, a);
+}
+
+}  // namespace mix
