@@ -74,10 +74,11 @@ struct __align__(16) RowRec {
   int t;                            // token row, or -1: padding row of a tile
   int slot;                         // slot of the SAE app that acts on the row (the row's own, or the last of its chain)
   int n_edit;                       // length of that app's edit list
-  int group_flags;                  // low byte: weight set; kRecAddError: the app keeps the error term
+  int group_flags;                  // low byte: weight set; kRecAddError: the app keeps the error term; bits 16..17: the set's activation
 };
 constexpr int kRecGroupMask = 0xff;
 constexpr int kRecAddError = 0x100;
+constexpr int kRecActShift = 16;
 
 // What sae_edit_only_kernel leaves for decode_delta_kernel about one token row.
 struct __align__(16) RowDelta {

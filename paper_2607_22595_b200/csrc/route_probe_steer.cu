@@ -370,22 +370,23 @@ __global__ void __launch_bounds__(NW * 32)
 probe_steer_team_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
                         const AppEntry* __restrict__ apps, const GateEntry* __restrict__ gates, int n_slots,
                         __nv_bfloat16* __restrict__ hidden, int d, float* __restrict__ scores, int C_max,
-                        unsigned* __restrict__ status, const uint4* __restrict__ vec_arena) {
+                        unsigned* __restrict__ status, const uint4* __restrict__ vec_arena, int pdl) {
   __shared__ float s_part[NW][kMaxClasses];
   constexpr int NT = NW * 32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t = blockIdx.x;                      // < T_max: the slot map has an entry for every row
-  // Programmatic dependent launch (when the launch asked for it; otherwise the two instructions do nothing):
-  // everything up to pdl_wait() reads only tables the LIBRARY owns and that only copies write -- live count,
-  // slot map, app entry, vector arena -- so it may run while the kernel in front of this one in the stream (the
-  // layer that produces `hidden`, or the previous hook) is still running.  Memory the caller owns (`hidden`,
-  // multi-class probe weights, gate scores) is read after the wait only, and every thread waits before it
-  // leaves, so that this grid cannot end -- and release ITS successor -- before its predecessor has.
-  pdl_launch_dependents();
+  // Programmatic dependent launch (`pdl`: the launch asked for it): everything up to pdl_wait() reads only
+  // tables the LIBRARY owns and that only copies write -- live count, slot map, app entry, vector arena -- so it
+  // may run while the kernel in front of this one in the stream (the layer that produces `hidden`, or the
+  // previous hook) is still running.  Memory the caller owns (`hidden`, multi-class probe weights, gate scores)
+  // is read after the wait only, and every thread waits before it leaves, so that this grid cannot end -- and
+  // release ITS successor -- before its predecessor has.  Launched the ordinary way, nothing has to wait: the
+  // row is then requested together with the vector and the app entry, one round trip earlier.
+  if (pdl) pdl_launch_dependents();
   const int n_live = __ldg(n_live_p);            // both loads issue together: one round trip, not two
   const int slot = __ldg(token_slot + t);
   if (t >= min(T, n_live) || slot == -1) {
-    pdl_wait();
+    if (pdl) pdl_wait();
     return;
   }
   const int nvec = d >> 3;
@@ -402,13 +403,22 @@ probe_steer_team_kernel(const int* __restrict__ token_slot, const int* __restric
       if (v < nvec) vq[u] = __ldg(vec_arena + (size_t)slot * nvec + v);
     }
   }
-  RowApp a = lookup(slot, t, apps, gates, n_slots, status, threadIdx.x == 0, /*eval_gate=*/false);
-  pdl_wait();
-  if (slot_ok) {
+  if (!pdl && slot_ok) {
 #pragma unroll
     for (int u = 0; u < kTeamVec; ++u) {
       const int v = threadIdx.x + u * NT;
       if (v < nvec) hq[u] = __ldcs(hrow + v);
+    }
+  }
+  RowApp a = lookup(slot, t, apps, gates, n_slots, status, threadIdx.x == 0, /*eval_gate=*/false);
+  if (pdl) {
+    pdl_wait();
+    if (slot_ok) {
+#pragma unroll
+      for (int u = 0; u < kTeamVec; ++u) {
+        const int v = threadIdx.x + u * NT;
+        if (v < nvec) hq[u] = __ldcs(hrow + v);
+      }
     }
   }
   if (a.gated && a.kind != 0 && !gate_open(gates, slot, t)) return;       // gate closed: the row passes through
@@ -718,9 +728,10 @@ cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float
                       c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates, c->d_chain_next, c->cfg.n_slots_max, hidden,
                       c->cfg.d_model, scores, c->cfg.C_max, c->d_status);
   } else if (c->cfg.T_max <= kTeamMaxRows) {
+    const int pdl = (allow_pdl && (pdl_mask() & kPdlHook)) ? 1 : 0;
     return launch_pdl(allow_pdl ? kPdlHook : 0, probe_steer_team_kernel<8>, dim3(c->cfg.T_max), dim3(8 * 32), 0, s,
                       c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates, c->cfg.n_slots_max, hidden, c->cfg.d_model,
-                      scores, c->cfg.C_max, c->d_status, reinterpret_cast<const uint4*>(c->d_vec_arena));
+                      scores, c->cfg.C_max, c->d_status, reinterpret_cast<const uint4*>(c->d_vec_arena), pdl);
   } else {
     const int blocks = (c->cfg.T_max + kWarpsPerBlock - 1) / kWarpsPerBlock;
     probe_steer_kernel<<<blocks, kWarpsPerBlock * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps, c->d_gates,

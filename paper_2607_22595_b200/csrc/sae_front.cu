@@ -36,12 +36,12 @@ __device__ __forceinline__ void pack_row_bf16(const __nv_bfloat16* __restrict__ 
   }
   const uint4* src = reinterpret_cast<const uint4*>(hidden + (size_t)t * d);
   int i = lane;
-  for (; i + 96 < nvec; i += 128) {                      // four loads in flight per lane
-    const uint4 a = __ldg(src + i), b = __ldg(src + i + 32), c = __ldg(src + i + 64), e = __ldg(src + i + 96);
-    dst[i] = a;
-    dst[i + 32] = b;
-    dst[i + 64] = c;
-    dst[i + 96] = e;
+  for (; i + 224 < nvec; i += 256) {                     // eight loads in flight per lane
+    uint4 q[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) q[u] = __ldg(src + i + 32 * u);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) dst[i + 32 * u] = q[u];
   }
   for (; i < nvec; i += 32) dst[i] = __ldg(src + i);
 }
@@ -149,6 +149,7 @@ front_kernel(const FrontArgs a) {
   __shared__ int s_total[kMaxGroups], s_base[kMaxGroups + 1];
   __shared__ int s_tok[kFrontRowsMax], s_slot[kFrontRowsMax], s_grp[kFrontRowsMax];
   __shared__ int s_n_panel_rows;
+  __shared__ int s_gact[kMaxGroups], s_gtiles[kMaxGroups];   // per weight set: activation, feature tiles (0: not registered)
   pdl_launch_dependents();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool first_cta = blockIdx.x == 0;
@@ -158,6 +159,11 @@ front_kernel(const FrontArgs a) {
   const int n_own = a.rows_per_cta;
   const int p0 = blockIdx.x * n_own;
   if (tid < n_own) s_tok[tid] = -1;
+  if (tid < n_groups) {                                // requested now, needed after the scan
+    const bool valid = __ldg(&a.groups[tid].valid) != 0;
+    s_gact[tid] = __ldg(&a.groups[tid].act);
+    s_gtiles[tid] = valid ? (int)(__ldg(&a.groups[tid].d_sae) / kTileN) : 0;
+  }
 
   // phase A: the weight set (or -1) of every row this thread owns (row c * 1024 + tid of chunk c), resolved
   // stage by stage for kRouteBatch chunks at a time so that their loads are in flight together (slot ids, then
@@ -267,12 +273,7 @@ front_kernel(const FrontArgs a) {
     for (int q = 0; q < n_groups; ++q) {
       s_base[q] = mt * kTileM;
       const int m_tiles = (s_total[q] + kTileM - 1) / kTileM;
-      int act = 0;
-      long long d_sae = 0;
-      if (s_total[q] > 0) {
-        act = __ldg(&a.groups[q].act);
-        d_sae = __ldg(&a.groups[q].d_sae);
-      }
+      const int act = s_gact[q];
       if (first_cta) {
         a.rs->group_count[q] = s_total[q];
         a.rs->group_mtile0[q] = mt;
@@ -282,7 +283,7 @@ front_kernel(const FrontArgs a) {
       mt += m_tiles;
       rows += s_total[q];
       if (s_total[q] > 0 && act == MIX_SAE_TOPK) topk_rows += s_total[q];
-      tiles += s_total[q] > 0 ? m_tiles * (int)(d_sae / kTileN) : 0;
+      tiles += s_total[q] > 0 ? m_tiles * s_gtiles[q] : 0;
     }
     s_base[n_groups] = mt * kTileM;
     s_n_panel_rows = mt * kTileM;
@@ -344,31 +345,32 @@ front_kernel(const FrontArgs a) {
     const int p = p0 + r;
     if (p >= a.panel_cap) break;
     const int t = s_tok[r];
+    // the row's record first requested, last written: its two table entries arrive while the row is copied
+    int n_edit = 0, add_error = 0;
+    if (lane == 0 && t >= 0) {
+      n_edit = __ldg(&a.apps[s_slot[r]].n_edit);
+      add_error = __ldg(&a.apps[s_slot[r]].add_error);
+    }
+    if (p < s_n_panel_rows) {
+      if (a.tau_slots) {                                 // the encode's TopK bound starts empty
+        reinterpret_cast<uint4*>(a.tau_slots + (size_t)p * kTauSlots)[lane] = make_uint4(0u, 0u, 0u, 0u);
+        if (lane == 0) a.tau_min[p] = 0u;
+      }
+      if (kPack == 0)
+        pack_row_bf16(a.hidden, t, static_cast<__nv_bfloat16*>(a.panel), (size_t)p, a.d, lane);
+      else
+        pack_row_e4m3<kPack == 1>(a.hidden, t, static_cast<unsigned char*>(a.panel), a.act_scale, (size_t)p, a.d, a.lo_row0, lane);
+    }
     if (lane == 0) {
       RowRec rec;
       rec.t = t;
-      rec.slot = -1;
-      rec.n_edit = 0;
-      rec.group_flags = 0;
-      if (t >= 0) {
-        const int slot = s_slot[r];
-        rec.slot = slot;
-        rec.n_edit = __ldg(&a.apps[slot].n_edit);
-        rec.group_flags = s_grp[r] | (__ldg(&a.apps[slot].add_error) ? kRecAddError : 0);
-      }
+      rec.slot = t >= 0 ? s_slot[r] : -1;
+      rec.n_edit = n_edit;
+      rec.group_flags = t >= 0 ? (s_grp[r] | (add_error ? kRecAddError : 0) | (s_gact[s_grp[r]] << kRecActShift)) : 0;
       a.row_rec[p] = rec;
       a.panel_row[p] = t;
       if (a.row_flag) a.row_flag[p] = 0;
     }
-    if (p >= s_n_panel_rows) continue;
-    if (a.tau_slots) {                                   // the encode's TopK bound starts empty
-      reinterpret_cast<uint4*>(a.tau_slots + (size_t)p * kTauSlots)[lane] = make_uint4(0u, 0u, 0u, 0u);
-      if (lane == 0) a.tau_min[p] = 0u;
-    }
-    if (kPack == 0)
-      pack_row_bf16(a.hidden, t, static_cast<__nv_bfloat16*>(a.panel), (size_t)p, a.d, lane);
-    else
-      pack_row_e4m3<kPack == 1>(a.hidden, t, static_cast<unsigned char*>(a.panel), a.act_scale, (size_t)p, a.d, a.lo_row0, lane);
   }
 }
 

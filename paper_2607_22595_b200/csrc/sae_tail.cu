@@ -296,7 +296,7 @@ __device__ void emit_topk(const unsigned long long* a, int k, int k_max, int t, 
 // decode
 // ---------------------------------------------------------------------------------------
 constexpr int kDecList = 1024 + kMaxEdits;     // >= k_max + r_max
-constexpr int kDecU = 4;                       // 16-byte column vectors per thread: 256 x 4 x 8 = 8192 columns
+constexpr int kGatherBatch = 8;                // decoder rows in flight per thread
 
 __device__ __forceinline__ void axpy8(float* acc, float c, const uint4& q) {
   const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&q);
@@ -308,40 +308,44 @@ __device__ __forceinline__ void axpy8(float* acc, float c, const uint4& q) {
   }
 }
 
-// acc += sum_e coef[e] * W_dec[feat[e], :] over this thread's column vectors (four 16-byte loads in flight per
-// thread and entry; the CTA's other warps and the SM's other CTAs cover the latency).  Entries with a zero
-// coefficient are not fetched.
-__device__ __forceinline__ void accumulate_list(float (*acc)[8], const float* coef, const int* feat, int n,
-                                                const __nv_bfloat16* __restrict__ W_dec, int d, int nvec) {
-  const int tid = threadIdx.x;
+// The gather of the decode.  A row is rebuilt in passes of 2048 columns: thread `tid` owns the 16-byte column
+// vector v = pass * 256 + tid, so one decoder row is read as 4 KiB of contiguous 16-byte loads per pass, and
+// acc (8 columns) += sum_e coef[e] * W_dec[feat[e], 8v .. 8v+7] with kGatherBatch decoder rows in flight per
+// thread -- the loop is bound by load latency, not arithmetic.  Entries with a zero coefficient are not fetched.
+__device__ __forceinline__ void gather_list(float (&acc)[8], const float* coef, const int* feat, int n,
+                                            const __nv_bfloat16* __restrict__ W_dec, int d, int v, bool in_cols) {
 #pragma unroll 1
-  for (int e = 0; e < n; ++e) {
-    const float c = coef[e];
-    if (c == 0.f) continue;
-    const uint4* row = reinterpret_cast<const uint4*>(W_dec + (size_t)feat[e] * d);
-    uint4 q[kDecU];
+  for (int e0 = 0; e0 < n; e0 += kGatherBatch) {
+    uint4 q[kGatherBatch];
+    float c[kGatherBatch];
 #pragma unroll
-    for (int u = 0; u < kDecU; ++u) {
-      const int v = tid + u * kTailThreads;
-      q[u] = v < nvec ? __ldg(row + v) : make_uint4(0u, 0u, 0u, 0u);
+    for (int u = 0; u < kGatherBatch; ++u) {
+      const int e = e0 + u;
+      c[u] = e < n ? coef[e] : 0.f;
+      q[u] = make_uint4(0u, 0u, 0u, 0u);
+      if (c[u] != 0.f && in_cols) q[u] = __ldg(reinterpret_cast<const uint4*>(W_dec + (size_t)feat[e] * d) + v);
     }
 #pragma unroll
-    for (int u = 0; u < kDecU; ++u) axpy8(acc[u], c, q[u]);
+    for (int u = 0; u < kGatherBatch; ++u) axpy8(acc, c[u], q[u]);
   }
 }
 
-__device__ __forceinline__ void store_row(uint4* hrow, float (*acc)[8], int nvec) {
+__device__ __forceinline__ void load8(float (&acc)[8], const uint4& q) {
+  const __nv_bfloat162* pp = reinterpret_cast<const __nv_bfloat162*>(&q);
 #pragma unroll
-  for (int u = 0; u < kDecU; ++u) {
-    const int v = threadIdx.x + u * kTailThreads;
-    if (v < nvec) {
-      uint4 q;
-      __nv_bfloat162* pp = reinterpret_cast<__nv_bfloat162*>(&q);
-#pragma unroll
-      for (int i = 0; i < 4; ++i) pp[i] = __floats2bfloat162_rn(acc[u][2 * i], acc[u][2 * i + 1]);
-      hrow[v] = q;
-    }
+  for (int i = 0; i < 4; ++i) {
+    const float2 f2 = __bfloat1622float2(pp[i]);
+    acc[2 * i] = f2.x;
+    acc[2 * i + 1] = f2.y;
   }
+}
+
+__device__ __forceinline__ uint4 pack8(const float (&acc)[8]) {
+  uint4 q;
+  __nv_bfloat162* pp = reinterpret_cast<__nv_bfloat162*>(&q);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) pp[i] = __floats2bfloat162_rn(acc[2 * i], acc[2 * i + 1]);
+  return q;
 }
 
 enum { kTailCand = 0, kTailZ = 1, kTailFallback = 2 };
@@ -394,7 +398,7 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh) {
     if (t < 0) continue;                               // padding row of a tile (uniform across the CTA, like every branch below)
     // (the weight-set entry field by field, not as a struct held in registers across the whole row)
     const GroupEntry* gp = a.groups + (rec.group_flags & kRecGroupMask);
-    const int act = gp->act;
+    const int act = (rec.group_flags >> kRecActShift) & 3;
     const bool add_error = (rec.group_flags & kRecAddError) != 0;
     const bool topk = act == MIX_SAE_TOPK;
     if (a.mode == kTailFallback && !(topk && a.row_flag[p])) continue;
@@ -466,7 +470,6 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh) {
       sh.ef[tid] = 0.f;
     }
     __syncthreads();
-    float acc[kDecU][8];
     if (add_error) {
       // (TopK rows only.)  f_j of an edited feature comes from the row's TopK list, 0 if it was not selected
       for (int i = tid; i < k; i += kTailThreads) {
@@ -486,20 +489,12 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh) {
         sh.feat[tid] = j;
       }
       if (__syncthreads_or(delta != 0.f)) {            // no effective edit: the row stays as it is, bit for bit
-#pragma unroll
-        for (int u = 0; u < kDecU; ++u) {
-          const int v = tid + u * kTailThreads;
-          const uint4 hq = v < nvec ? hrow[v] : make_uint4(0u, 0u, 0u, 0u);
-          const __nv_bfloat162* pp = reinterpret_cast<const __nv_bfloat162*>(&hq);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float2 f2 = __bfloat1622float2(pp[i]);
-            acc[u][2 * i] = f2.x;
-            acc[u][2 * i + 1] = f2.y;
-          }
+        for (int v = tid; v < nvec; v += kTailThreads) {
+          float acc[8];
+          load8(acc, hrow[v]);
+          gather_list(acc, sh.coef, sh.feat, n_edit, W_dec, d, v, true);
+          hrow[v] = pack8(acc);
         }
-        accumulate_list(acc, sh.coef, sh.feat, n_edit, W_dec, d, nvec);
-        store_row(hrow, acc, nvec);
       }
       __syncthreads();
       continue;
@@ -513,15 +508,7 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh) {
       sh.coef[tid] = alive ? fnew : 0.f;
       sh.feat[tid] = j;
     }
-    {
-      const float* b_dec = gp->b_dec;
-#pragma unroll
-      for (int u = 0; u < kDecU; ++u) {
-        const int v = tid + u * kTailThreads;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) acc[u][i] = (b_dec && v < nvec) ? b_dec[v * 8 + i] : 0.f;
-      }
-    }
+    const float* b_dec = gp->b_dec;
     if (topk) {
       for (int i = tid; i < k; i += kTailThreads) {
         const int j = comp_id(sorted[i]);
@@ -533,37 +520,49 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh) {
         sh.feat[n_edit + i] = in_range ? j : 0;
       }
       __syncthreads();
-      accumulate_list(acc, sh.coef, sh.feat, n_edit + k, W_dec, d, nvec);
+      for (int v = tid; v < nvec; v += kTailThreads) {
+        float acc[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] = b_dec ? b_dec[v * 8 + i] : 0.f;
+        gather_list(acc, sh.coef, sh.feat, n_edit + k, W_dec, d, v, true);
+        hrow[v] = pack8(acc);
+      }
     } else {
+      // ReLU / JumpReLU: per pass of 2048 columns, the edited features first, then a dense scan of the
+      // activations in chunks of 1024 -- active, unedited features are compacted into shared memory and
+      // applied chunk by chunk.  (Every thread walks every pass: the scan needs the whole CTA.)
       const float* theta = gp->theta;
-      __syncthreads();
-      accumulate_list(acc, sh.coef, sh.feat, n_edit, W_dec, d, nvec);
-      // dense scan of the activations in chunks; active, unedited features are compacted
-      // into shared memory and applied chunk by chunk
-      if (tid == 0) sh.n_list = 0;
-      __syncthreads();
-      for (int c0 = 0; c0 < S; c0 += 1024) {
-        for (int j = c0 + tid; j < min(S, c0 + 1024); j += kTailThreads) {
-          const float zj = z[j];
-          const float f = act == MIX_SAE_RELU ? fmaxf(zj, 0.f) : (zj > theta[j] ? zj : 0.f);
-          if (f != 0.f) {
-            bool edited = false;
-            for (int e = 0; e < n_edit; ++e) edited = edited || (sh.eidx[e] == j);
-            if (!edited) {
-              const int pos = atomicAdd(&sh.n_list, 1);
-              sh.coef[pos] = f;
-              sh.feat[pos] = j;
+      for (int v0 = 0; v0 < nvec; v0 += kTailThreads) {
+        const int v = v0 + tid;
+        const bool in_cols = v < nvec;
+        float acc[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] = (b_dec && in_cols) ? b_dec[v * 8 + i] : 0.f;
+        __syncthreads();
+        gather_list(acc, sh.coef, sh.feat, n_edit, W_dec, d, v, in_cols);
+        for (int c0 = 0; c0 < S; c0 += 1024) {
+          if (tid == 0) sh.n_list = 0;
+          __syncthreads();
+          for (int j = c0 + tid; j < min(S, c0 + 1024); j += kTailThreads) {
+            const float zj = z[j];
+            const float f = act == MIX_SAE_RELU ? fmaxf(zj, 0.f) : (zj > theta[j] ? zj : 0.f);
+            if (f != 0.f) {
+              bool edited = false;
+              for (int e = 0; e < n_edit; ++e) edited = edited || (sh.eidx[e] == j);
+              if (!edited) {
+                const int pos = atomicAdd(&sh.n_list, 1);
+                sh.coef[kMaxEdits + pos] = f;
+                sh.feat[kMaxEdits + pos] = j;
+              }
             }
           }
+          __syncthreads();
+          gather_list(acc, sh.coef + kMaxEdits, sh.feat + kMaxEdits, sh.n_list, W_dec, d, v, in_cols);
+          __syncthreads();
         }
-        __syncthreads();
-        accumulate_list(acc, sh.coef, sh.feat, sh.n_list, W_dec, d, nvec);
-        __syncthreads();
-        if (tid == 0) sh.n_list = 0;
-        __syncthreads();
+        if (in_cols) hrow[v] = pack8(acc);
       }
     }
-    store_row(hrow, acc, nvec);
     __syncthreads();                                   // the shared lists are reused by the next row
   }
 }
@@ -592,8 +591,8 @@ __device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int cta) {
     const int p = p0 + tid;                              // in bounds: the panel capacity is a multiple of 128
     const RowRec rec = a.row_rec[p];
     const int g = rec.group_flags & kRecGroupMask;
-    bool on = p < n_rows && rec.t >= 0 && (rec.group_flags & kRecAddError) && rec.n_edit > 0;
-    if (on) on = a.groups[g].act != MIX_SAE_TOPK;
+    const bool on = p < n_rows && rec.t >= 0 && (rec.group_flags & kRecAddError) && rec.n_edit > 0 &&
+                    ((rec.group_flags >> kRecActShift) & 3) != MIX_SAE_TOPK;
     sh.t[tid] = on ? rec.t : -1;
     sh.slot[tid] = on ? rec.slot : -1;
     sh.n_edit[tid] = rec.n_edit;
