@@ -417,6 +417,14 @@ int mix_set_pdl_mask(int mask);
 int mix_debug_workspace(mix_ctx* ctx, const int** panel_rows, const float** z, long long* ld_z,
                         int* n_panel_rows);
 
+/* Profiling aid (no counterpart in the paper).  A context created while MIX_PHASE_CLOCKS=1 is set in the
+   environment keeps 32 words in which the first CTA of the SAE chain's front and tail kernels stamps the GPU's
+   nanosecond timer at its phase boundaries (0..4 front: start, rows classified, routing scanned, positions
+   found, rows packed; 7..15 tail: launched, predecessor done, row 0 read, candidates narrowed, sorted, TopK
+   known, coefficients known, row written, CTA done).  out32: HOST array of 32 words, zeros when the context
+   was created without the variable.  Synchronises the device. */
+int mix_debug_phase_clocks(mix_ctx* ctx, unsigned long long* out32);
+
 /* ---------------------------------------------------------------------------------------
  * SAE function for callers that cannot allocate device memory.  (The paper has no counterpart
  * to this call; it exists for integration reasons only.)

@@ -34,7 +34,7 @@ EXPORTS = [
     "mix_register_app", "mix_unregister_app", "mix_set_gate", "mix_set_chain", "mix_update_steer_alpha", "mix_update_sae_edits",
     "mix_set_slot_map", "mix_set_request_map", "mix_set_feature_out", "mix_apply", "mix_apply_conditional", "mix_apply_router", "mix_get_status",
     "mix_launches_per_apply", "mix_set_stage_events", "mix_debug_workspace", "mix_sae_apply_static",
-    "mix_bench_param_update", "mix_set_pdl_mask",
+    "mix_bench_param_update", "mix_set_pdl_mask", "mix_debug_phase_clocks",
 ]
 
 
@@ -112,6 +112,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.mix_sae_apply_static.argtypes = [vp, ci, ci, C.POINTER(MixSaeWeights), C.POINTER(MixSaeApp), vp, vp, vp,
                                          C.c_char_p, ci]
     lib.mix_debug_workspace.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(C.c_longlong), C.POINTER(ci)]
+    lib.mix_debug_phase_clocks.argtypes = [vp, C.POINTER(C.c_ulonglong)]
     for name in EXPORTS:
         if name != "mix_last_error":
             getattr(lib, name).restype = ci
@@ -327,6 +328,12 @@ class Mix:
         a, b = C.c_float(0), C.c_float(0)
         self._check(self.lib.mix_bench_param_update(self.ctx, int(iters), C.byref(a), C.byref(b), _stream(stream)))
         return float(a.value), float(b.value)
+
+    def debug_phase_clocks(self):
+        """32 nanosecond stamps of the front / tail kernels' phases (zeros unless MIX_PHASE_CLOCKS=1 at creation)."""
+        out = (C.c_ulonglong * 32)()
+        self._check(self.lib.mix_debug_phase_clocks(self.ctx, out))
+        return [int(x) for x in out]
 
     def debug_workspace(self):
         pr, z, ld, n = C.c_void_p(), C.c_void_p(), C.c_longlong(), C.c_int()

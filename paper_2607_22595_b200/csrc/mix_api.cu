@@ -84,7 +84,7 @@ void free_all(mix_ctx* c) {
   cudaFree(c->d_edit_idx); cudaFree(c->d_edit_val); cudaFree(c->d_edit_mode); cudaFree(c->d_status);
   cudaFree(c->d_tmp_req); cudaFree(c->d_tmp_req_slot); cudaFree(c->d_panel); cudaFree(c->d_panel_row); cudaFree(c->d_act_scale); cudaFree(c->d_tau); cudaFree(c->d_tau_min); cudaFree(c->d_eo_row_delta); cudaFree(c->d_eo_coef);
   cudaFree(c->d_mtile_group); cudaFree(c->d_row_group); cudaFree(c->d_route); cudaFree(c->d_z);
-  cudaFree(c->d_tmap_w); cudaFree(c->d_tmap_probe); cudaFree(c->d_mc_dense); cudaFree(c->d_cand_val); cudaFree(c->d_cand_idx);
+  cudaFree(c->d_tmap_w); cudaFree(c->d_tmap_w_half); cudaFree(c->d_phase_clk); cudaFree(c->d_tmap_probe); cudaFree(c->d_mc_dense); cudaFree(c->d_cand_val); cudaFree(c->d_cand_idx);
   cudaFree(c->d_cand_ninth); cudaFree(c->d_row_flag); cudaFree(c->d_mtile_flag); cudaFree(c->d_n_flagged);
   if (c->owned_b_eff)
     for (int g = 0; g < c->cfg.n_groups_max; ++g) cudaFree(c->owned_b_eff[g]);
@@ -258,7 +258,10 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
     ok = ok && dev_alloc(&c->d_route, 1) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_z, P * (size_t)cfg->d_sae_max) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_tmap_w, G) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_tmap_w_half, G) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_row_rec, P) == cudaSuccess;
+    if (getenv("MIX_PHASE_CLOCKS") && atoi(getenv("MIX_PHASE_CLOCKS")))
+      ok = ok && dev_alloc(&c->d_phase_clk, 32) == cudaSuccess && cudaMemset(c->d_phase_clk, 0, 32 * sizeof(unsigned long long)) == cudaSuccess;
     if (cfg->flags & MIX_FLAG_SAE_EDIT_ONLY) {
       ok = ok && dev_alloc(&c->d_eo_row_delta, (size_t)T) == cudaSuccess;
       ok = ok && dev_alloc(&c->d_eo_coef, (size_t)T * (size_t)(cfg->r_max > 0 ? cfg->r_max : 1)) == cudaSuccess;
@@ -388,7 +391,7 @@ int mix_register_sae_weights(mix_ctx* c, int group, const mix_sae_weights* w, vo
     ge.b_eff = c->owned_b_eff[group];
   }
   if (!(c->cfg.flags & MIX_FLAG_ENCODE_SIMT)) {
-    CUtensorMap tm;
+    CUtensorMap tm, tm_half;       // boxes of 256 features, and of 128 (one CTA's share when a CTA pair works on the tile)
     if (fp8) {
       // library-owned tile-ordered copy of the codes: [S/256][d/128][256][128] bytes, seen by TMA as a 128-byte-wide
       // matrix (128-byte swizzled boxes of 256 rows)
@@ -400,7 +403,8 @@ int mix_register_sae_weights(mix_ctx* c, int group, const mix_sae_weights* w, vo
       }
       unsigned char* tiled = reinterpret_cast<unsigned char*>(c->owned_w_tiled[group]);
       MIX_CUDA(c, launch_retile_fp8(static_cast<const unsigned char*>(w->W_enc), tiled, w->d_sae, c->cfg.d_model, 2 * kTileK, s));
-      if (make_tmap_e4m3(&tm, tiled, (unsigned long long)(n_el / (2 * kTileK)), 2 * kTileK, kTileN) != MIX_OK)
+      if (make_tmap_e4m3(&tm, tiled, (unsigned long long)(n_el / (2 * kTileK)), 2 * kTileK, kTileN) != MIX_OK ||
+          make_tmap_e4m3(&tm_half, tiled, (unsigned long long)(n_el / (2 * kTileK)), 2 * kTileK, kTileN / 2) != MIX_OK)
         MIX_FAIL(c, MIX_ERR_CUDA, "cuTensorMapEncodeTiled failed for the 8-bit W_enc");
     } else if (c->cfg.flags & MIX_FLAG_RETILE_W_ENC) {
       // library-owned tile-contiguous copy: [S/256][d/64][256][64], seen by TMA as a 64-column matrix
@@ -411,12 +415,15 @@ int mix_register_sae_weights(mix_ctx* c, int group, const mix_sae_weights* w, vo
         MIX_FAIL(c, MIX_ERR_NO_MEMORY, "cannot allocate the re-tiled copy of W_enc");
       }
       MIX_CUDA(c, launch_retile(ge.W_enc, c->owned_w_tiled[group], w->d_sae, c->cfg.d_model, s));
-      if (make_tmap(&tm, c->owned_w_tiled[group], (unsigned long long)(n_el / kTileK), kTileK, kTileN) != MIX_OK)
+      if (make_tmap(&tm, c->owned_w_tiled[group], (unsigned long long)(n_el / kTileK), kTileK, kTileN) != MIX_OK ||
+          make_tmap(&tm_half, c->owned_w_tiled[group], (unsigned long long)(n_el / kTileK), kTileK, kTileN / 2) != MIX_OK)
         MIX_FAIL(c, MIX_ERR_CUDA, "cuTensorMapEncodeTiled failed for the re-tiled W_enc");
-    } else if (make_tmap(&tm, w->W_enc, (unsigned long long)w->d_sae, c->cfg.d_model, kTileN) != MIX_OK) {
+    } else if (make_tmap(&tm, w->W_enc, (unsigned long long)w->d_sae, c->cfg.d_model, kTileN) != MIX_OK ||
+               make_tmap(&tm_half, w->W_enc, (unsigned long long)w->d_sae, c->cfg.d_model, kTileN / 2) != MIX_OK) {
       MIX_FAIL(c, MIX_ERR_CUDA, "cuTensorMapEncodeTiled failed for W_enc");
     }
     MIX_CUDA(c, cudaMemcpyAsync(c->d_tmap_w + group, &tm, sizeof(tm), cudaMemcpyHostToDevice, s));
+    MIX_CUDA(c, cudaMemcpyAsync(c->d_tmap_w_half + group, &tm_half, sizeof(tm_half), cudaMemcpyHostToDevice, s));
   }
   c->h_groups[group] = ge;
   GroupEntry tmp = ge;
@@ -901,6 +908,14 @@ int mix_bench_param_update(mix_ctx* c, int iters, float* us_table, float* us_nod
   if (sums[0] != sums[1]) MIX_FAIL(c, MIX_ERR_CUDA, "the two mechanisms disagree: %g vs %g", (double)sums[0], (double)sums[1]);
   *us_table = (float)us[0];
   *us_node = (float)us[1];
+  return MIX_OK;
+}
+
+int mix_debug_phase_clocks(mix_ctx* c, unsigned long long* out32) {
+  if (!c) return MIX_ERR_INVALID_ARG;
+  if (!out32) MIX_FAIL(c, MIX_ERR_INVALID_ARG, "out32 is NULL");
+  memset(out32, 0, 32 * sizeof(unsigned long long));
+  if (c->d_phase_clk) MIX_CUDA(c, cudaMemcpy(out32, c->d_phase_clk, 32 * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
   return MIX_OK;
 }
 

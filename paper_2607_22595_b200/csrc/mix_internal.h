@@ -94,7 +94,8 @@ struct RouteState {
   int n_mtiles;                     // = n_panel_rows / kTileM
   int total_tiles;                  // encode tiles over all groups
   int n_topk_rows;                  // SAE rows whose weight set is TopK
-  int pad_[3];
+  int n_delta_rows;                 // ReLU / JumpReLU rows that keep the error term and have edits (the tail kernel's delta role)
+  int pad_[2];
   int group_count[kMaxGroups];      // M_g
   int group_mtile0[kMaxGroups + 1]; // first m-tile of group g in the panel
   int group_tile0[kMaxGroups + 1];  // first linear encode tile of group g
@@ -152,6 +153,7 @@ struct Ctx {
   int* d_mtile_flag;        // [P / kTileM] some row of the tile is flagged
   int* d_n_flagged;         // [1]
   CUtensorMap* d_tmap_w;    // [n_groups_max] W_enc maps (box kTileK x kTileN, 128B swizzle)
+  CUtensorMap* d_tmap_w_half;   // [n_groups_max] the same with boxes of kTileN / 2 rows: what one CTA of a pair fetches
   CUtensorMap* d_tmap_probe;   // [n_slots_max] maps of multi-class probe matrices (box kTileK x 32), large-batch contexts only
   int* d_mc_dense;          // [1] is this call's batch dense in multi-class probe rows?  written by mc_decide_kernel
   CUtensorMap tmap_panel;   // panel map (box kTileK x kTileM, 128B swizzle)
@@ -166,6 +168,8 @@ struct Ctx {
                             // must not read it ahead of its predecessor
   int stage_events_on;
   cudaEvent_t stage_events[16];
+
+  unsigned long long* d_phase_clk;   // [32] profiling aid (MIX_PHASE_CLOCKS=1 at mix_create): globaltimer stamps of kernel phases, else null
 
   // optional outputs
   int* out_topk_idx;
@@ -206,6 +210,15 @@ cudaError_t launch_pdl(int which, void (*kernel)(KArgs...), dim3 grid, dim3 bloc
 #endif
 
 #ifdef __CUDACC__
+// Profiling aid: thread `who` (a bool) stamps slot i of the phase-clock array with the global nanosecond timer.
+__device__ __forceinline__ void phase_stamp(unsigned long long* clk, int i, bool who) {
+  if (clk != nullptr && who) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    clk[i] = t;
+  }
+}
+
 // Order-preserving 32-bit key of a float (larger value, larger key; -0 and +0 share one key; 0 is below every value).
 __device__ __forceinline__ unsigned f2key(float f) {
   const unsigned b = __float_as_uint(f + 0.f);          // -0.0 -> +0.0: equal values, equal keys
@@ -248,5 +261,7 @@ cudaError_t launch_fold_bias(const __nv_bfloat16* W_enc, const float* b_enc, con
 cudaError_t launch_retile(const __nv_bfloat16* W_enc, __nv_bfloat16* W_tiled, long long d_sae, int d, cudaStream_t s);
 cudaError_t launch_retile_fp8(const unsigned char* W_enc, unsigned char* W_tiled, long long d_sae, int d, int kb_bytes, cudaStream_t s);
 cudaError_t encode_tc_prepare();   // opt in to the large dynamic shared memory size
+constexpr int kEncodePairDefault = 0;   // the encode on CTA pairs (tcgen05 cta_group::2) unless MIX_ENCODE_PAIR says otherwise
+int encode_pair_mode(int set);     // returns the mode in force; set >= 0 changes it (A/B timing)
 
 }  // namespace mix

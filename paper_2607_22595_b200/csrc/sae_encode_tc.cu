@@ -25,6 +25,8 @@
 //     the same accumulator.  Per element of K that is the tensor time of the bf16 kernel with half the W_enc
 //     bytes: as fast as kEnc == 2 where the stream of W_enc is the bound, as fast as bf16 where the tensor
 //     pipe is.
+#include <stdlib.h>
+
 #include "mix_internal.h"
 #include "tc_common.cuh"
 
@@ -32,16 +34,20 @@ namespace mix {
 
 namespace {
 
-constexpr int kMaxStages = 4;
+constexpr int kMaxStages = 6;
 constexpr int kABytes = kTileM * kTileK * 2;   // 16 KiB: 128 rows of 128 bytes
 constexpr int kBBytes = kTileN * kTileK * 2;   // 32 KiB: 256 rows of 128 bytes
 constexpr int kXchgEntries = kCandPerTile + 2;  // a top-9 list and the bound it was collected under
 // kEnc: 0 = bf16 encoder and input; 1 = 8-bit encoder, bf16 input as two E4M3 operands; 2 = 8-bit encoder and 8-bit input
-template <int kEnc, int kEpi> struct TcCfg {
+// kPair: two CTAs (a cluster) share one 256-row x 256-feature tile: each loads its own 128 panel rows and HALF of the
+//        W_enc tile, and one tcgen05.mma.cta_group::2 instruction feeds both SMs' tensor cores -- a third less
+//        shared-memory fill per SM and flop than a CTA working alone (32 instead of 48 KiB per k-block).
+template <int kEnc, int kEpi, bool kPair> struct TcCfg {
   static_assert(kEpi == 4 || kEpi == 8, "epilogue warps");
   static constexpr bool kSplit = kEnc == 1;            // two panel tiles (hi, lo) per stage
-  static constexpr int kStages = kSplit ? 3 : 4;
-  static constexpr int kStageBytes = (kSplit ? 2 : 1) * kABytes + kBBytes;
+  static constexpr int kBBytesCta = kPair ? kBBytes / 2 : kBBytes;
+  static constexpr int kStageBytes = (kSplit ? 2 : 1) * kABytes + kBBytesCta;
+  static constexpr int kStages = kPair ? (kSplit ? 4 : 6) : (kSplit ? 3 : 4);
   static constexpr int kRingBytes = kStages * kStageBytes;
   // epilogue warps: 4 (one per tensor-memory lane quarter, all 256 columns) or 8 (two per quarter, 128 columns
   // each; the two top-9 lists of a row meet in shared memory).  One warp per scheduler runs the epilogue's
@@ -57,7 +63,7 @@ constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz
 constexpr long long kWaitCyclesTest = 2000000ll;  // ~1 ms: the cap under MIX_FLAG_TEST_STALL_ENCODE
 
 struct __align__(8) TcShared {
-  unsigned long long full[kMaxStages];
+  unsigned long long full[kMaxStages];      // (a pair's leader: filled by both CTAs' copies)
   unsigned long long empty[kMaxStages];
   unsigned long long tmem_full[2];
   unsigned long long tmem_empty[2];
@@ -66,6 +72,9 @@ struct __align__(8) TcShared {
   volatile int abort_flag;
   long long wait_cycles;      // cap of every bounded wait in this launch
   RouteState rs;
+  // CTA pairs: first row-tile pair / first pair-tile of each weight set, totals
+  short pair0[kMaxGroups + 1];
+  int ptile0[kMaxGroups + 1];
 };
 static_assert(sizeof(TcShared) <= 1024, "TcShared must fit the space reserved for it");
 
@@ -78,13 +87,12 @@ __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, TcShare
 
 constexpr unsigned kIdesc = idesc_f16(kTileM, kTileN);     // D fp32, A and B bf16, K-major, N = 256, M = 128
 constexpr unsigned kIdescE4 = idesc_e4m3(kTileM, kTileN);  // D fp32, A and B E4M3, K-major, N = 256, M = 128
-
-__device__ __forceinline__ void umma(unsigned d_tmem, unsigned long long a, unsigned long long b, unsigned accumulate) {
-  umma_f16(d_tmem, a, b, kIdesc, accumulate);
-}
+constexpr unsigned kIdescPair = idesc_f16(2 * kTileM, kTileN);     // the pair's instruction: M = 256
+constexpr unsigned kIdescE4Pair = idesc_e4m3(2 * kTileM, kTileN);
 
 struct Tile {
   int group, n_tile, m_tile_global, rows_valid;
+  int m_tile_peer;      // CTA pairs: the row tile the other CTA of the pair works on (the same one when the weight set has an odd tile left over)
 };
 
 // Number of feature tiles per row tile if it is the same for every weight set that has rows (the usual
@@ -114,6 +122,7 @@ __device__ __forceinline__ Tile decode_tile(const RouteState& rs, const GroupEnt
     while (g + 1 < n_groups && t.m_tile_global >= rs.group_mtile0[g + 1]) ++g;
     t.group = g;
     t.rows_valid = min(kTileM, rs.group_count[g] - (t.m_tile_global - rs.group_mtile0[g]) * kTileM);
+    t.m_tile_peer = t.m_tile_global;
     return t;
   }
   while (g + 1 < n_groups && tile >= rs.group_tile0[g + 1]) ++g;
@@ -125,6 +134,36 @@ __device__ __forceinline__ Tile decode_tile(const RouteState& rs, const GroupEnt
   const int m_local = local - t.n_tile * mt;
   t.m_tile_global = rs.group_mtile0[g] + m_local;
   t.rows_valid = min(kTileM, count - m_local * kTileM);
+  t.m_tile_peer = t.m_tile_global;
+  return t;
+}
+
+// The same for CTA pairs: linear pair-tile id -> (weight set, feature tile, pair of row tiles) and, for the CTA of
+// rank `rank`, its own row tile.  A weight set with an odd number of row tiles leaves its last pair half empty:
+// the CTA without a tile of its own repeats the other one's loads and keeps nothing (rows_valid = 0).
+__device__ __forceinline__ Tile decode_pair_tile(const TcShared& sh, int n_groups, int tile, int uniform_nt, int rank) {
+  const RouteState& rs = sh.rs;
+  Tile t;
+  int g = 0, pl;
+  if (uniform_nt > 0) {
+    const int n_pairs = sh.pair0[n_groups];
+    t.n_tile = tile / n_pairs;
+    const int pr = tile - t.n_tile * n_pairs;
+    while (g + 1 < n_groups && pr >= sh.pair0[g + 1]) ++g;
+    pl = pr - sh.pair0[g];
+  } else {
+    while (g + 1 < n_groups && tile >= sh.ptile0[g + 1]) ++g;
+    const int local = tile - sh.ptile0[g];
+    const int mp = sh.pair0[g + 1] - sh.pair0[g];
+    t.n_tile = local / mp;
+    pl = local - t.n_tile * mp;
+  }
+  const int mt = rs.group_mtile0[g + 1] - rs.group_mtile0[g];
+  const int m_own = 2 * pl + rank, m_peer = 2 * pl + (1 - rank);
+  t.group = g;
+  t.m_tile_global = rs.group_mtile0[g] + min(m_own, mt - 1);
+  t.m_tile_peer = rs.group_mtile0[g] + min(m_peer, mt - 1);
+  t.rows_valid = m_own < mt ? min(kTileM, rs.group_count[g] - m_own * kTileM) : 0;
   return t;
 }
 
@@ -134,7 +173,7 @@ __device__ __forceinline__ Tile decode_tile(const RouteState& rs, const GroupEnt
 __device__ __forceinline__ bool tile_wanted(const Tile& t, const GroupEntry* __restrict__ groups, int mode,
                                             const int* __restrict__ mtile_flag) {
   if (mode == 0) return true;
-  return groups[t.group].act == MIX_SAE_TOPK && mtile_flag[t.m_tile_global] != 0;
+  return groups[t.group].act == MIX_SAE_TOPK && (mtile_flag[t.m_tile_global] | mtile_flag[t.m_tile_peer]) != 0;   // same answer in both CTAs of a pair
 }
 
 // Insert (x, c) into the descending list tv[0..8] if it beats the 9th entry.  Equal values keep
@@ -155,8 +194,8 @@ __device__ __forceinline__ void top9_insert(float (&tv)[kCandPerTile + 1], int (
   }
 }
 
-template <int kEnc, int kEpi>
-__global__ void __launch_bounds__(TcCfg<kEnc, kEpi>::kThreads, 1)
+template <int kEnc, int kEpi, bool kPair>
+__global__ void __launch_bounds__(TcCfg<kEnc, kEpi, kPair>::kThreads, 1)
 encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorMap* __restrict__ tmap_w,
                  const RouteState* __restrict__ rs_g, const GroupEntry* __restrict__ groups, int n_groups,
                  float* __restrict__ Z, long long ldz, int d, unsigned* __restrict__ status, int mode,
@@ -167,10 +206,11 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
   constexpr bool kE4 = kEnc != 0;                      // E4M3 x E4M3 contraction
   constexpr bool kSplit = kEnc == 1;                   // the panel row is hi + lo: two operand tiles per k-block
   constexpr int kBlockK = kE4 ? 2 * kTileK : kTileK;   // elements per 128-byte row of either operand
-  constexpr int kStages = TcCfg<kEnc, kEpi>::kStages;
-  constexpr int kStageBytes = TcCfg<kEnc, kEpi>::kStageBytes;
-  constexpr int kTcThreads = TcCfg<kEnc, kEpi>::kThreads;
-  constexpr int kEpiWarps = TcCfg<kEnc, kEpi>::kEpiWarps;
+  using Cfg = TcCfg<kEnc, kEpi, kPair>;
+  constexpr int kStages = Cfg::kStages;
+  constexpr int kStageBytes = Cfg::kStageBytes;
+  constexpr int kTcThreads = Cfg::kThreads;
+  constexpr int kEpiWarps = Cfg::kEpiWarps;
   constexpr int kEpiCols = kTileN / (kEpiWarps / 4);   // columns of a tile per epilogue warp
   pdl_wait();
   pdl_launch_dependents();
@@ -178,21 +218,43 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment: required by the 128-byte swizzle atoms
   unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  TcShared* sh = reinterpret_cast<TcShared*>(tiles + TcCfg<kEnc, kEpi>::kRingBytes);
+  TcShared* sh = reinterpret_cast<TcShared*>(tiles + Cfg::kRingBytes);
   float* xchg_val = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(sh) + 1024);
   int* xchg_idx = reinterpret_cast<int*>(xchg_val + 2 * 4 * kXchgEntries * 32);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // CTA pairs: rank 0 leads (it issues the pair's tensor-core instructions and owns the barriers both CTAs' copies
+  // complete on); `worker` numbers the units that walk the tile list -- pairs, or single CTAs
+  const int rank = kPair ? (int)cluster_ctarank() : 0;
+  const bool leader = rank == 0;
+  const int worker = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int n_workers = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
   for (int i = threadIdx.x; i < (int)(sizeof(RouteState) / sizeof(int)); i += kTcThreads)
     reinterpret_cast<int*>(&sh->rs)[i] = reinterpret_cast<const int*>(rs_g)[i];
+  if (kPair) __syncthreads();
   if (threadIdx.x == 0) {
+    if (kPair) {      // pairs of row tiles per weight set
+      int np = 0, pt = 0;
+      for (int g = 0; g < n_groups; ++g) {
+        const int mt = sh->rs.group_mtile0[g + 1] - sh->rs.group_mtile0[g];
+        const int nt = mt > 0 ? (sh->rs.group_tile0[g + 1] - sh->rs.group_tile0[g]) / mt : 0;
+        sh->pair0[g] = (short)np;
+        sh->ptile0[g] = pt;
+        np += (mt + 1) / 2;
+        pt += ((mt + 1) / 2) * nt;
+      }
+      for (int g = n_groups; g <= kMaxGroups; ++g) {
+        sh->pair0[g] = (short)np;
+        sh->ptile0[g] = pt;
+      }
+    }
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&sh->full[s]), 1);
       mbar_init(smem_u32(&sh->empty[s]), 1);
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&sh->tmem_full[a]), 1);
-      mbar_init(smem_u32(&sh->tmem_empty[a]), kEpiWarps);
+      mbar_init(smem_u32(&sh->tmem_empty[a]), kPair ? 2 * kEpiWarps : kEpiWarps);   // a pair's leader hears from both CTAs' epilogues
       for (int q = 0; q < 4; ++q) mbar_init(smem_u32(&sh->xchg_full[a][q]), 1);
     }
     sh->abort_flag = 0;
@@ -201,30 +263,32 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
-  const int total_tiles = sh->rs.total_tiles;
-  if (total_tiles == 0) return;            // nothing routed to any SAE: no tensor memory is taken
+  if (sh->rs.total_tiles == 0) return;     // nothing routed to any SAE: no tensor memory is taken (both CTAs of a pair see the same)
+  const int total_tiles = kPair ? sh->ptile0[n_groups] : sh->rs.total_tiles;
 
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
-                 "r"(kTmemCols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (kPair) tmem_alloc_pair(smem_u32(&sh->tmem_base), kTmemCols);
+    else tmem_alloc(smem_u32(&sh->tmem_base), kTmemCols);
   }
   tc_fence_before();
-  __syncthreads();
+  if (kPair) cluster_sync_all();           // the peer's barriers are initialised before anything is sent to them
+  else __syncthreads();
   tc_fence_after();
   const unsigned tmem_base = sh->tmem_base;
   // (the interleaved order serves the TopK epilogue's running bound; without TopK rows the plain order is a little faster)
   const int uniform_nt = sh->rs.n_topk_rows > 0 ? uniform_feature_tiles(sh->rs, n_groups) : 0;
   const int num_kb = d / kBlockK;
+  auto tile_of = [&](int tile) {
+    return kPair ? decode_pair_tile(*sh, n_groups, tile, uniform_nt, rank) : decode_tile(sh->rs, groups, n_groups, tile, uniform_nt);
+  };
 
   if (warp == 0) {
     if (lane == 0) {
       int stage = 0;
       unsigned phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const Tile t = decode_tile(sh->rs, groups, n_groups, tile, uniform_nt);
+      for (int tile = worker; tile < total_tiles && ok; tile += n_workers) {
+        const Tile t = tile_of(tile);
         if (!tile_wanted(t, groups, mode, mtile_flag)) continue;
         const CUtensorMap* tw = tmap_w + t.group;
         for (int kb = 0; kb < num_kb; ++kb) {
@@ -233,29 +297,42 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
           // bounded wait runs out and the whole CTA leaves through the time-out path.
           if (test_stall) { ok = false; break; }
           const unsigned bar = smem_u32(&sh->full[stage]);
-          mbar_expect_tx(bar, kStageBytes);
           const unsigned sa = smem_u32(tiles + stage * kStageBytes);
           const unsigned sw = sa + (kSplit ? 2 : 1) * kABytes;
-          tma_load_2d(sa, &tmap_panel, kb * kBlockK, t.m_tile_global * kTileM, bar);
-          if (kSplit) tma_load_2d(sa + kABytes, &tmap_panel, kb * kBlockK, lo_row0 + t.m_tile_global * kTileM, bar);   // the lo codes
-          // W_enc tile: rows n_tile*256.. of the row-major matrix, or -- when the weights were re-laid
-          // out at registration (always, for codes) -- block (n_tile, kb) of the tile-contiguous copy
-          // [S/256][d/kBlockK][256][kBlockK]
-          if (kE4 || w_tiled)
-            tma_load_2d(sw, tw, 0, (t.n_tile * num_kb + kb) * kTileN, bar);
-          else
-            tma_load_2d(sw, tw, kb * kTileK, t.n_tile * kTileN, bar);
+          if (kPair) {
+            // both CTAs' copies complete on the LEADER's barrier, which expects the bytes of both; this CTA
+            // fetches its own 128 panel rows and its half (128 features) of the W_enc tile
+            if (leader) mbar_expect_tx(bar, 2 * kStageBytes);
+            const unsigned bar_c = mapa_cluster(bar, 0);
+            tma_load_2d_pair(sa, &tmap_panel, kb * kBlockK, t.m_tile_global * kTileM, bar_c);
+            if (kSplit) tma_load_2d_pair(sa + kABytes, &tmap_panel, kb * kBlockK, lo_row0 + t.m_tile_global * kTileM, bar_c);
+            if (kE4 || w_tiled)
+              tma_load_2d_pair(sw, tw, 0, (t.n_tile * num_kb + kb) * kTileN + rank * (kTileN / 2), bar_c);
+            else
+              tma_load_2d_pair(sw, tw, kb * kTileK, t.n_tile * kTileN + rank * (kTileN / 2), bar_c);
+          } else {
+            mbar_expect_tx(bar, kStageBytes);
+            tma_load_2d(sa, &tmap_panel, kb * kBlockK, t.m_tile_global * kTileM, bar);
+            if (kSplit) tma_load_2d(sa + kABytes, &tmap_panel, kb * kBlockK, lo_row0 + t.m_tile_global * kTileM, bar);   // the lo codes
+            // W_enc tile: rows n_tile*256.. of the row-major matrix, or -- when the weights were re-laid
+            // out at registration (always, for codes) -- block (n_tile, kb) of the tile-contiguous copy
+            // [S/256][d/kBlockK][256][kBlockK]
+            if (kE4 || w_tiled)
+              tma_load_2d(sw, tw, 0, (t.n_tile * num_kb + kb) * kTileN, bar);
+            else
+              tma_load_2d(sw, tw, kb * kTileK, t.n_tile * kTileN, bar);
+          }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    if (lane == 0 && leader) {
       int stage = 0;
       unsigned phase = 0, acc = 0, acc_phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        if (mode != 0 && !tile_wanted(decode_tile(sh->rs, groups, n_groups, tile, uniform_nt), groups, mode, mtile_flag)) continue;
+      for (int tile = worker; tile < total_tiles && ok; tile += n_workers) {
+        if (mode != 0 && !tile_wanted(tile_of(tile), groups, mode, mtile_flag)) continue;
         if (!mbar_wait(smem_u32(&sh->tmem_empty[acc]), acc_phase ^ 1u, sh, status)) break;
         tc_fence_after();
         const unsigned d_tmem = tmem_base + acc * kTileN;
@@ -267,19 +344,31 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
           const unsigned long long da = umma_desc(sa), db = umma_desc(sb);
 #pragma unroll
           for (int k = 0; k < 4; ++k) {   // 16 bf16 or 32 codes = 32 bytes = 2 descriptor units per step
-            if (kE4) umma_e4m3(d_tmem, da + 2ull * k, db + 2ull * k, kIdescE4, (unsigned)((kb | k) != 0));
-            else umma(d_tmem, da + 2ull * k, db + 2ull * k, (unsigned)((kb | k) != 0));
+            const unsigned accum = (unsigned)((kb | k) != 0);
+            if (kPair) {
+              if (kE4) umma_e4m3_pair(d_tmem, da + 2ull * k, db + 2ull * k, kIdescE4Pair, accum);
+              else umma_f16_pair(d_tmem, da + 2ull * k, db + 2ull * k, kIdescPair, accum);
+            } else {
+              if (kE4) umma_e4m3(d_tmem, da + 2ull * k, db + 2ull * k, kIdescE4, accum);
+              else umma_f16(d_tmem, da + 2ull * k, db + 2ull * k, kIdesc, accum);
+            }
           }
           if (kSplit) {                   // + lo W into the same accumulator
             const unsigned long long dl = umma_desc(sa + kABytes);
 #pragma unroll
-            for (int k = 0; k < 4; ++k) umma_e4m3(d_tmem, dl + 2ull * k, db + 2ull * k, kIdescE4, 1u);
+            for (int k = 0; k < 4; ++k) {
+              if (kPair) umma_e4m3_pair(d_tmem, dl + 2ull * k, db + 2ull * k, kIdescE4Pair, 1u);
+              else umma_e4m3(d_tmem, dl + 2ull * k, db + 2ull * k, kIdescE4, 1u);
+            }
           }
-          umma_commit(smem_u32(&sh->empty[stage]));
+          // the stage is free again -- in both CTAs of a pair
+          if (kPair) umma_commit_pair(smem_u32(&sh->empty[stage]));
+          else umma_commit(smem_u32(&sh->empty[stage]));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        umma_commit(smem_u32(&sh->tmem_full[acc]));
+        if (kPair) umma_commit_pair(smem_u32(&sh->tmem_full[acc]));
+        else umma_commit(smem_u32(&sh->tmem_full[acc]));
         acc ^= 1u;
         if (acc == 0) acc_phase ^= 1u;
       }
@@ -290,8 +379,8 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
     const int c_lo = half * kEpiCols;
     unsigned acc = 0, acc_phase = 0;
     unsigned xchg_phase = 0;                 // bit a: phase of the next hand-over through xchg_full[a][q] (TopK tiles only)
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-      const Tile t = decode_tile(sh->rs, groups, n_groups, tile, uniform_nt);
+    for (int tile = worker; tile < total_tiles; tile += n_workers) {
+      const Tile t = tile_of(tile);
       if (!tile_wanted(t, groups, mode, mtile_flag)) continue;
       const int row_local = q * 32 + lane;
       const bool valid = row_local < t.rows_valid;
@@ -436,7 +525,10 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[acc]));
+      if (lane == 0) {     // the accumulator is free: tell the CTA that issues the instructions
+        if (kPair && !leader) mbar_arrive_cluster(mapa_cluster(smem_u32(&sh->tmem_empty[acc]), 0));
+        else mbar_arrive(smem_u32(&sh->tmem_empty[acc]));
+      }
       acc ^= 1u;
       if (acc == 0) acc_phase ^= 1u;
     }
@@ -449,9 +541,12 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
     const long long t0 = clock64();
     while (clock64() - t0 < 2000000ll) __nanosleep(1000);
   }
+  // a pair leaves together: neither CTA's barriers or tensor memory go away while the other may still reach them
+  if (kPair) cluster_sync_all();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    if (kPair) tmem_dealloc_pair(tmem_base, kTmemCols);
+    else tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 
@@ -504,31 +599,70 @@ cudaError_t launch_retile(const __nv_bfloat16* W_enc, __nv_bfloat16* W_tiled, lo
   return cudaGetLastError();
 }
 
-template <int kEnc, int kEpi>
+template <int kEnc, int kEpi, bool kPair>
 static cudaError_t encode_tc_prepare_as() {
-  return cudaFuncSetAttribute(encode_tc_kernel<kEnc, kEpi>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              TcCfg<kEnc, kEpi>::kSmemBytes);
+  return cudaFuncSetAttribute(encode_tc_kernel<kEnc, kEpi, kPair>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              TcCfg<kEnc, kEpi, kPair>::kSmemBytes);
 }
 
 cudaError_t encode_tc_prepare() {
-  cudaError_t e = encode_tc_prepare_as<0, 4>();
-  if (e == cudaSuccess) e = encode_tc_prepare_as<0, 8>();
-  if (e == cudaSuccess) e = encode_tc_prepare_as<1, 4>();
-  if (e == cudaSuccess) e = encode_tc_prepare_as<1, 8>();
-  if (e == cudaSuccess) e = encode_tc_prepare_as<2, 4>();
-  if (e == cudaSuccess) e = encode_tc_prepare_as<2, 8>();
+  cudaError_t e = encode_tc_prepare_as<0, 4, false>();
+  if (e == cudaSuccess) e = encode_tc_prepare_as<0, 8, false>();
+  if (e == cudaSuccess) e = encode_tc_prepare_as<1, 4, false>();
+  if (e == cudaSuccess) e = encode_tc_prepare_as<1, 8, false>();
+  if (e == cudaSuccess) e = encode_tc_prepare_as<2, 4, false>();
+  if (e == cudaSuccess) e = encode_tc_prepare_as<2, 8, false>();
+  if (e == cudaSuccess) e = encode_tc_prepare_as<0, 4, true>();
+  if (e == cudaSuccess) e = encode_tc_prepare_as<0, 8, true>();
+  if (e == cudaSuccess) e = encode_tc_prepare_as<1, 4, true>();
+  if (e == cudaSuccess) e = encode_tc_prepare_as<1, 8, true>();
+  if (e == cudaSuccess) e = encode_tc_prepare_as<2, 4, true>();
+  if (e == cudaSuccess) e = encode_tc_prepare_as<2, 8, true>();
   return e;
 }
 
-template <int kEnc, int kEpi>
+// CTA pairs or single CTAs: MIX_ENCODE_PAIR in the environment (0 / 1), read once; set by mix_set_encode_pair for A/B timing.
+static int g_encode_pair = -1;
+int encode_pair_mode(int set) {
+  if (g_encode_pair < 0) g_encode_pair = getenv("MIX_ENCODE_PAIR") ? (atoi(getenv("MIX_ENCODE_PAIR")) != 0) : kEncodePairDefault;
+  const int old = g_encode_pair;
+  if (set >= 0) g_encode_pair = set != 0;
+  return old;
+}
+
+template <int kEnc, int kEpi, bool kPair>
 static cudaError_t launch_encode_tc_as(const Ctx* c, int mode, cudaStream_t s) {
+  using Cfg = TcCfg<kEnc, kEpi, kPair>;
   const int w_tiled = (c->cfg.flags & MIX_FLAG_RETILE_W_ENC) ? 1 : 0;
   const int stall = (c->cfg.flags & MIX_FLAG_TEST_STALL_ENCODE) ? 1 : 0;
-  return launch_pdl(mode == 0 ? kPdlEncode : kPdlTail, encode_tc_kernel<kEnc, kEpi>, dim3(c->n_sms),
-                    dim3(TcCfg<kEnc, kEpi>::kThreads), TcCfg<kEnc, kEpi>::kSmemBytes, s, c->tmap_panel, c->d_tmap_w, c->d_route,
-                    c->d_groups, c->cfg.n_groups_max, c->d_z, c->cfg.d_sae_max, c->cfg.d_model, c->d_status, mode,
-                    c->d_mtile_flag, c->d_n_flagged, c->d_cand_val, c->d_cand_idx, c->d_cand_ninth, c->cand_tiles, w_tiled,
-                    stall, c->d_act_scale, c->d_tau, c->d_tau_min, c->panel_rows_cap);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(kPair ? (c->n_sms & ~1) : c->n_sms);
+  cfg.blockDim = dim3(Cfg::kThreads);
+  cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+  cfg.stream = s;
+  cudaLaunchAttribute at[2];
+  int n_at = 0;
+  if (kPair) {
+    at[n_at].id = cudaLaunchAttributeClusterDimension;
+    at[n_at].val.clusterDim.x = 2;
+    at[n_at].val.clusterDim.y = 1;
+    at[n_at].val.clusterDim.z = 1;
+    ++n_at;
+  }
+  if (pdl_mask() & (mode == 0 ? kPdlEncode : kPdlTail)) {
+    at[n_at].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[n_at].val.programmaticStreamSerializationAllowed = 1;
+    ++n_at;
+  }
+  cfg.attrs = at;
+  cfg.numAttrs = n_at;
+  const CUtensorMap* tmap_w = kPair ? c->d_tmap_w_half : c->d_tmap_w;
+  return cudaLaunchKernelEx(&cfg, encode_tc_kernel<kEnc, kEpi, kPair>, c->tmap_panel, tmap_w,
+                            static_cast<const RouteState*>(c->d_route), static_cast<const GroupEntry*>(c->d_groups),
+                            c->cfg.n_groups_max, c->d_z, (long long)c->cfg.d_sae_max, c->cfg.d_model, c->d_status, mode,
+                            static_cast<const int*>(c->d_mtile_flag), static_cast<const int*>(c->d_n_flagged), c->d_cand_val,
+                            c->d_cand_idx, c->d_cand_ninth, c->cand_tiles, w_tiled, stall,
+                            static_cast<const float*>(c->d_act_scale), c->d_tau, c->d_tau_min, c->panel_rows_cap);
 }
 
 // Eight epilogue warps pay off for the TopK epilogue (selection work per element); the plain store of the
@@ -537,9 +671,14 @@ static cudaError_t launch_encode_tc_as(const Ctx* c, int mode, cudaStream_t s) {
 cudaError_t launch_encode_tc(const Ctx* c, int mode, cudaStream_t s) {
   bool topk = false;
   for (int g = 0; g < c->cfg.n_groups_max; ++g) topk = topk || (c->h_groups[g].valid && c->h_groups[g].act == MIX_SAE_TOPK);
-  if (c->cfg.flags & MIX_FLAG_FP8_ACT) return topk ? launch_encode_tc_as<2, 8>(c, mode, s) : launch_encode_tc_as<2, 4>(c, mode, s);
-  if (c->cfg.flags & MIX_FLAG_FP8_W_ENC) return topk ? launch_encode_tc_as<1, 8>(c, mode, s) : launch_encode_tc_as<1, 4>(c, mode, s);
-  return topk ? launch_encode_tc_as<0, 8>(c, mode, s) : launch_encode_tc_as<0, 4>(c, mode, s);
+  if (encode_pair_mode(-1)) {
+    if (c->cfg.flags & MIX_FLAG_FP8_ACT) return topk ? launch_encode_tc_as<2, 8, true>(c, mode, s) : launch_encode_tc_as<2, 4, true>(c, mode, s);
+    if (c->cfg.flags & MIX_FLAG_FP8_W_ENC) return topk ? launch_encode_tc_as<1, 8, true>(c, mode, s) : launch_encode_tc_as<1, 4, true>(c, mode, s);
+    return topk ? launch_encode_tc_as<0, 8, true>(c, mode, s) : launch_encode_tc_as<0, 4, true>(c, mode, s);
+  }
+  if (c->cfg.flags & MIX_FLAG_FP8_ACT) return topk ? launch_encode_tc_as<2, 8, false>(c, mode, s) : launch_encode_tc_as<2, 4, false>(c, mode, s);
+  if (c->cfg.flags & MIX_FLAG_FP8_W_ENC) return topk ? launch_encode_tc_as<1, 8, false>(c, mode, s) : launch_encode_tc_as<1, 4, false>(c, mode, s);
+  return topk ? launch_encode_tc_as<0, 8, false>(c, mode, s) : launch_encode_tc_as<0, 4, false>(c, mode, s);
 }
 
 }  // namespace mix

@@ -139,6 +139,7 @@ struct FrontArgs {
   unsigned* tau_slots;
   unsigned* tau_min;
   int lo_row0;
+  unsigned long long* clk;   // profiling aid or null
 };
 
 // kPack: 0 the bf16 row, 1 E4M3 hi + lo (exact split), 2 E4M3 quantised.
@@ -150,15 +151,18 @@ front_kernel(const FrontArgs a) {
   __shared__ int s_tok[kFrontRowsMax], s_slot[kFrontRowsMax], s_grp[kFrontRowsMax];
   __shared__ int s_n_panel_rows;
   __shared__ int s_gact[kMaxGroups], s_gtiles[kMaxGroups];   // per weight set: activation, feature tiles (0: not registered)
+  __shared__ int s_n_delta;
   pdl_launch_dependents();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool first_cta = blockIdx.x == 0;
   const int n_groups = a.n_groups, n_slots = a.n_slots;
   const int n_live = min(a.T, __ldg(a.n_live_p));
   const int n_chunks = (n_live + kFrontThreads - 1) / kFrontThreads;
+  phase_stamp(a.clk, 0, first_cta && tid == 0);
   const int n_own = a.rows_per_cta;
   const int p0 = blockIdx.x * n_own;
   if (tid < n_own) s_tok[tid] = -1;
+  if (tid == 0) s_n_delta = 0;
   if (tid < n_groups) {                                // requested now, needed after the scan
     const bool valid = __ldg(&a.groups[tid].valid) != 0;
     s_gact[tid] = __ldg(&a.groups[tid].act);
@@ -166,37 +170,52 @@ front_kernel(const FrontArgs a) {
   }
 
   // phase A: the weight set (or -1) of every row this thread owns (row c * 1024 + tid of chunk c), resolved
-  // stage by stage for kRouteBatch chunks at a time so that their loads are in flight together (slot ids, then
-  // app entries, then weight-set entries: three round trips per batch); then per (chunk, warp) counts per set.
-  // The first batch (8192 rows: every configuration in use) stays in registers for phase C; later batches go
-  // through the row_group / row_slot scratch (every CTA writes the same values there and reads back its own).
-  int grp0[kRouteBatch], slot0[kRouteBatch];
-  for (int c0 = 0; c0 < n_chunks; c0 += kRouteBatch) {
-    int slot[kRouteBatch], grp[kRouteBatch];
+  // stage by stage for kRouteBatch chunks at a time so that their loads are in flight together: the slot ids
+  // (requested together with the live count), then bytes 0..31 of the app entries -- valid, kind, weight set,
+  // edit count, error-term flag in one round trip; the weight sets' own entries were requested at the top of
+  // the kernel.  Then per (chunk, warp) counts per set.  The first batch (8192 rows: every configuration in use)
+  // stays in registers for phase C; later batches go through the row_group / row_slot scratch (every CTA writes
+  // the same values there and reads back its own).
+  // meta: (weight set + 1) | edit count << 8 | error-term flag << 16; 0 = not an SAE row of this call
+  int meta0[kRouteBatch], slot0[kRouteBatch];
+  const int T_cap = a.T;
+  const int n_chunks_cap = (T_cap + kFrontThreads - 1) / kFrontThreads;
+  bool groups_ready = false;
+  for (int c0 = 0; c0 < n_chunks_cap; c0 += kRouteBatch) {
+    int slot[kRouteBatch], meta[kRouteBatch];
 #pragma unroll
     for (int c = 0; c < kRouteBatch; ++c) {
       const int t = (c0 + c) * kFrontThreads + tid;
-      slot[c] = (c0 + c < n_chunks && t < n_live) ? __ldg(a.token_slot + t) : -1;
-      if (slot[c] >= n_slots) slot[c] = -1;
+      slot[c] = t < T_cap ? __ldg(a.token_slot + t) : -1;      // does not wait for the live count
     }
-    int2 head[kRouteBatch];
-    int group_id[kRouteBatch];
+    if (c0 >= n_chunks) break;                                  // (uniform) nothing live from here on
 #pragma unroll
     for (int c = 0; c < kRouteBatch; ++c) {
-      head[c] = make_int2(0, 0);
-      group_id[c] = -1;
+      const int t = (c0 + c) * kFrontThreads + tid;
+      if (t >= n_live || slot[c] >= n_slots) slot[c] = -1;
+    }
+    int2 q0[kRouteBatch];                 // valid, kind
+    int3 q1[kRouteBatch];                 // weight set, edit count, error-term flag
+#pragma unroll
+    for (int c = 0; c < kRouteBatch; ++c) {
+      q0[c] = make_int2(0, 0);
+      q1[c] = make_int3(0, 0, 0);
       if (slot[c] >= 0) {
-        head[c] = __ldg(reinterpret_cast<const int2*>(a.apps + slot[c]));          // valid, kind
-        group_id[c] = __ldg(&a.apps[slot[c]].group);
+        const AppEntry* e = a.apps + slot[c];
+        q0[c] = __ldg(reinterpret_cast<const int2*>(e));
+        q1[c].x = __ldg(&e->group);
+        const int2 ne = __ldg(reinterpret_cast<const int2*>(&e->n_edit));
+        q1[c].y = ne.x;
+        q1[c].z = ne.y;
       }
     }
     // a row whose slot starts a chain is an SAE row if the chain ends in an SAE app: follow the
     // links (rare, so the dependent loads are not batched) and carry on with that app's slot
 #pragma unroll
     for (int c = 0; c < kRouteBatch; ++c) {
-      if (head[c].x && (head[c].y & kKindChained) && (head[c].y & kKindMask) != MIX_SAE) {
+      if (q0[c].x && (q0[c].y & kKindChained) && (q0[c].y & kKindMask) != MIX_SAE) {
         int s2 = slot[c];
-        int2 h2 = head[c];
+        int2 h2 = q0[c];
         for (int depth = 1; depth < kMaxChain && s2 >= 0; ++depth) {
           s2 = (h2.y & kKindChained) ? __ldg(a.chain_next + s2) : -1;
           if (s2 < 0 || s2 >= n_slots) { s2 = -1; break; }
@@ -206,47 +225,66 @@ front_kernel(const FrontArgs a) {
         }
         if (s2 >= 0 && (h2.y & kKindMask) != MIX_SAE) s2 = -1;
         slot[c] = s2;
-        head[c] = s2 >= 0 ? h2 : make_int2(0, 0);
-        group_id[c] = s2 >= 0 ? __ldg(&a.apps[s2].group) : -1;
-      }
-    }
-#pragma unroll
-    for (int c = 0; c < kRouteBatch; ++c) {
-      grp[c] = -1;
-      if (head[c].x && (head[c].y & kKindMask) == MIX_SAE) {
-        const int g = group_id[c];
-        if (g < 0 || g >= n_groups || !__ldg(&a.groups[g].valid)) {
-          if (first_cta) atomicOr(a.status, MIX_STATUS_BAD_GROUP);
-        } else if (a.edit_only && __ldg(&a.apps[slot[c]].add_error) && __ldg(&a.groups[g].act) != MIX_SAE_TOPK) {
-          // handled by sae_edit_only_kernel: with the error term on, a ReLU / JumpReLU row needs
-          // only the pre-activations of its edited features, not the whole encode
-        } else if (!(head[c].y & kKindGated) || gate_open(a.gates, slot[c], (c0 + c) * kFrontThreads + tid)) {
-          grp[c] = g;
+        q0[c] = s2 >= 0 ? h2 : make_int2(0, 0);
+        q1[c] = make_int3(0, 0, 0);
+        if (s2 >= 0) {
+          q1[c].x = __ldg(&a.apps[s2].group);
+          q1[c].y = __ldg(&a.apps[s2].n_edit);
+          q1[c].z = __ldg(&a.apps[s2].add_error);
         }
       }
     }
+    if (!groups_ready) {                   // the weight-set table requested at the top has long arrived
+      __syncthreads();
+      groups_ready = true;
+    }
+    int n_delta = 0;
+#pragma unroll
+    for (int c = 0; c < kRouteBatch; ++c) {
+      meta[c] = 0;
+      if (q0[c].x && (q0[c].y & kKindMask) == MIX_SAE) {
+        const int g = q1[c].x, n_edit = q1[c].y, add_error = q1[c].z != 0;
+        if (g < 0 || g >= n_groups || s_gtiles[g] == 0) {
+          if (first_cta) atomicOr(a.status, MIX_STATUS_BAD_GROUP);
+        } else if (a.edit_only && add_error && s_gact[g] != MIX_SAE_TOPK) {
+          // handled by sae_edit_only_kernel: with the error term on, a ReLU / JumpReLU row needs
+          // only the pre-activations of its edited features, not the whole encode
+        } else if (!(q0[c].y & kKindGated) || gate_open(a.gates, slot[c], (c0 + c) * kFrontThreads + tid)) {
+          meta[c] = (g + 1) | (n_edit << 8) | (add_error << 16);
+          n_delta += add_error && n_edit > 0 && s_gact[g] != MIX_SAE_TOPK;
+        }
+      }
+    }
+    n_delta = __reduce_add_sync(0xffffffffu, n_delta);
+    if (lane == 0 && n_delta) atomicAdd(&s_n_delta, n_delta);
 #pragma unroll
     for (int c = 0; c < kRouteBatch; ++c) {
       if (c0 == 0) {
-        grp0[c] = grp[c];
+        meta0[c] = meta[c];
         slot0[c] = slot[c];
       }
       if (c0 + c < n_chunks) {                       // uniform across the CTA
         const int t = (c0 + c) * kFrontThreads + tid;
         if (c0 > 0 && t < n_live) {
-          a.row_group[t] = grp[c];
+          a.row_group[t] = meta[c];
           a.row_slot[t] = slot[c];
         }
+        const int grp = (meta[c] & 0xff) - 1;
         for (int q = 0; q < n_groups; ++q) {
-          const unsigned m = __ballot_sync(0xffffffffu, grp[c] == q);
+          const unsigned m = __ballot_sync(0xffffffffu, grp == q);
           if (lane == 0) s_cnt[((c0 + c) * kFrontWarps + warp) * n_groups + q] = __popc(m);
         }
       }
     }
   }
+  if (!groups_ready) __syncthreads();
+  phase_stamp(a.clk, 1, first_cta && tid == 0);
   if (n_chunks == 0) {
 #pragma unroll
-    for (int c = 0; c < kRouteBatch; ++c) grp0[c] = slot0[c] = -1;
+    for (int c = 0; c < kRouteBatch; ++c) {
+      meta0[c] = 0;
+      slot0[c] = -1;
+    }
   }
   __syncthreads();
   // phase B: exclusive scan over (chunk, warp) for each weight set; warp q owns set q
@@ -299,6 +337,7 @@ front_kernel(const FrontArgs a) {
       a.rs->n_sae_rows = rows;
       a.rs->total_tiles = tiles;
       a.rs->n_topk_rows = topk_rows;
+      a.rs->n_delta_rows = s_n_delta;
       if (a.n_flagged) *a.n_flagged = 0;       // fallback-selection flags of the fused TopK path start clear every call
       // graph-conditional form: the rest of the SAE chain sits in the body of an IF node that runs only when a row needs it
       if (a.use_cond) cudaGraphSetConditional(a.cond, rows > 0 ? 1u : 0u);
@@ -307,32 +346,34 @@ front_kernel(const FrontArgs a) {
   if (first_cta && a.mtile_flag)
     for (int m = tid; m < a.panel_cap / kTileM; m += kFrontThreads) a.mtile_flag[m] = 0;
   __syncthreads();
+  phase_stamp(a.clk, 2, first_cta && tid == 0);
   // phase C: stable positions; a row that lands in this CTA's share of the panel leaves its token here
   for (int c0 = 0; c0 < n_chunks; c0 += kRouteBatch) {
-    int grp[kRouteBatch], slot[kRouteBatch];
+    int meta[kRouteBatch], slot[kRouteBatch];
 #pragma unroll
     for (int c = 0; c < kRouteBatch; ++c) {
       const int t = (c0 + c) * kFrontThreads + tid;
       if (c0 == 0) {
-        grp[c] = grp0[c];
+        meta[c] = meta0[c];
         slot[c] = slot0[c];
       } else {
-        grp[c] = (c0 + c < n_chunks && t < n_live) ? a.row_group[t] : -1;
-        slot[c] = grp[c] >= 0 ? a.row_slot[t] : -1;
+        meta[c] = (c0 + c < n_chunks && t < n_live) ? a.row_group[t] : 0;
+        slot[c] = meta[c] ? a.row_slot[t] : -1;
       }
     }
 #pragma unroll
     for (int c = 0; c < kRouteBatch; ++c) {
       if (c0 + c < n_chunks) {
+        const int grp = (meta[c] & 0xff) - 1;
         for (int q = 0; q < n_groups; ++q) {
-          const unsigned m = __ballot_sync(0xffffffffu, grp[c] == q);
-          if (grp[c] == q) {
+          const unsigned m = __ballot_sync(0xffffffffu, grp == q);
+          if (grp == q) {
             const int pos = s_base[q] + s_cnt[((c0 + c) * kFrontWarps + warp) * n_groups + q] +
                             __popc(m & ((1u << lane) - 1u));
             if (pos >= p0 && pos < p0 + n_own) {
               s_tok[pos - p0] = (c0 + c) * kFrontThreads + tid;
               s_slot[pos - p0] = slot[c];
-              s_grp[pos - p0] = q;
+              s_grp[pos - p0] = meta[c];
             }
           }
         }
@@ -340,17 +381,12 @@ front_kernel(const FrontArgs a) {
     }
   }
   __syncthreads();
+  phase_stamp(a.clk, 3, first_cta && tid == 0);
   // this CTA's panel rows, one per warp and round: the row's record for the kernels behind the encode, then the row itself
   for (int r = warp; r < n_own; r += kFrontWarps) {
     const int p = p0 + r;
     if (p >= a.panel_cap) break;
     const int t = s_tok[r];
-    // the row's record first requested, last written: its two table entries arrive while the row is copied
-    int n_edit = 0, add_error = 0;
-    if (lane == 0 && t >= 0) {
-      n_edit = __ldg(&a.apps[s_slot[r]].n_edit);
-      add_error = __ldg(&a.apps[s_slot[r]].add_error);
-    }
     if (p < s_n_panel_rows) {
       if (a.tau_slots) {                                 // the encode's TopK bound starts empty
         reinterpret_cast<uint4*>(a.tau_slots + (size_t)p * kTauSlots)[lane] = make_uint4(0u, 0u, 0u, 0u);
@@ -365,13 +401,15 @@ front_kernel(const FrontArgs a) {
       RowRec rec;
       rec.t = t;
       rec.slot = t >= 0 ? s_slot[r] : -1;
-      rec.n_edit = n_edit;
-      rec.group_flags = t >= 0 ? (s_grp[r] | (add_error ? kRecAddError : 0) | (s_gact[s_grp[r]] << kRecActShift)) : 0;
+      const int meta = t >= 0 ? s_grp[r] : 0, g = (meta & 0xff) - 1;
+      rec.n_edit = (meta >> 8) & 0xff;
+      rec.group_flags = t >= 0 ? (g | ((meta >> 16) & 1 ? kRecAddError : 0) | (s_gact[g] << kRecActShift)) : 0;
       a.row_rec[p] = rec;
       a.panel_row[p] = t;
       if (a.row_flag) a.row_flag[p] = 0;
     }
   }
+  phase_stamp(a.clk, 4, first_cta && tid == 0);
 }
 
 }  // namespace
@@ -408,6 +446,7 @@ cudaError_t launch_front(const Ctx* c, const __nv_bfloat16* hidden, int T, cudaS
   a.tau_slots = c->d_tau;
   a.tau_min = c->d_tau_min;
   a.lo_row0 = c->panel_rows_cap;
+  a.clk = c->d_phase_clk;
   const int n_chunks = (c->cfg.T_max + kFrontThreads - 1) / kFrontThreads;
   const size_t smem = (size_t)n_chunks * kFrontWarps * c->cfg.n_groups_max * sizeof(int);
   // one wave of CTAs where the panel allows it (a CTA of 1024 threads has an SM to itself)

@@ -374,8 +374,8 @@ struct TailArgs {
   int* n_flagged;
   unsigned* status;
   int mode;                 // kTailCand: TopK from the encode's candidates; kTailZ: TopK from Z; kTailFallback: flagged rows only, from Z
-  int n_row_ctas;           // CTAs [0, n_row_ctas) take the row role, the rest the delta role
   int n_col_slices;         // delta role: ceil(d / 2048)
+  unsigned long long* clk;  // profiling aid or null
 };
 
 struct RowShared {
@@ -392,7 +392,9 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh) {
   const int tid = threadIdx.x;
   const int n_rows = a.rs->n_panel_rows;
   const int d = a.d, nvec = d >> 3;
-  for (int p = blockIdx.x; p < n_rows; p += a.n_row_ctas) {
+  for (int p = blockIdx.x; p < n_rows; p += gridDim.x) {
+    const bool stamp = p == 0 && tid == 0 && a.mode != kTailFallback;
+    phase_stamp(a.clk, 9, stamp);
     const RowRec rec = a.row_rec[p];
     const int t = rec.t;
     if (t < 0) continue;                               // padding row of a tile (uniform across the CTA, like every branch below)
@@ -417,8 +419,10 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh) {
           CandRow src{a.cand_val + (size_t)p * a.cand_tiles * kCandPerTile, a.cand_idx + (size_t)p * a.cand_tiles * kCandPerTile, n};
           flag = radix_collect<false>(src, k, sh.sel) == 0;
         }
+        phase_stamp(a.clk, 10, stamp);
         if (!flag) {
           sorted = sort_desc(sh.sel);
+          phase_stamp(a.clk, 11, stamp);
           const unsigned kth = (unsigned)(sorted[k - 1] >> 32);
           const float* ninth = a.cand_ninth + (size_t)p * a.cand_tiles;
           int over = 0;
@@ -440,6 +444,7 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh) {
         if (how == 2 && tid == 0) atomicOr(a.status, MIX_STATUS_TOPK_GENERAL);
         sorted = sort_desc(sh.sel);
       }
+      phase_stamp(a.clk, 12, stamp);
       emit_topk(sorted, k, a.k_max, t, a.out_idx, a.out_val, a.out_n_active, &sh.sel.count);
     } else {
       if (a.out_n_active != nullptr) {
@@ -488,6 +493,7 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh) {
         sh.coef[tid] = delta;
         sh.feat[tid] = j;
       }
+      phase_stamp(a.clk, 13, stamp);
       if (__syncthreads_or(delta != 0.f)) {            // no effective edit: the row stays as it is, bit for bit
         for (int v = tid; v < nvec; v += kTailThreads) {
           float acc[8];
@@ -497,6 +503,7 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh) {
         }
       }
       __syncthreads();
+      phase_stamp(a.clk, 14, stamp);
       continue;
     }
     // the app replaces the residual: h' = b_dec + sum_j f'_j W_dec[j]
@@ -581,12 +588,12 @@ struct DeltaShared {
   int t[kDlRows], slot[kDlRows], n_edit[kDlRows], grp[kDlRows], changed[kDlRows];
 };
 
-__device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int cta) {
+// One work item of the delta role: row group `item / n_col_slices`, column slice `item % n_col_slices`.
+__device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int item, int n_rows) {
   const int tid = threadIdx.x;
-  const int rg = cta / a.n_col_slices, cs = cta - rg * a.n_col_slices;
+  const int rg = item / a.n_col_slices, cs = item - rg * a.n_col_slices;
   const int p0 = rg * kDlRows;
-  const int n_rows = a.rs->n_panel_rows;
-  if (p0 >= n_rows) return;
+  __syncthreads();                                       // the shared lists of the previous item are free
   if (tid < kDlRows) {
     const int p = p0 + tid;                              // in bounds: the panel capacity is a multiple of 128
     const RowRec rec = a.row_rec[p];
@@ -694,17 +701,26 @@ __device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int cta) {
   }
 }
 
+// A fixed grid of CTAs (a few per SM, all resident at once or nearly) walks the work of the call: first the
+// packed rows that need the row role, then the row groups x column slices of the delta role.  Both lists are as
+// long as THIS call's routing made them, not as long as the context's capacity, and a role with no rows this
+// call (no TopK / replacing row; no ReLU / JumpReLU row with edits) is skipped without looking at a single row.
 __global__ void __launch_bounds__(kTailThreads, 3)
 tail_kernel(const TailArgs a) {
+  phase_stamp(a.clk, 7, blockIdx.x == 0 && threadIdx.x == 0 && a.mode != kTailFallback);
   pdl_wait();
   pdl_launch_dependents();
+  phase_stamp(a.clk, 8, blockIdx.x == 0 && threadIdx.x == 0 && a.mode != kTailFallback);
   __shared__ RowShared s_row;
   __shared__ DeltaShared s_delta;
   if (a.mode == kTailFallback && *a.n_flagged == 0) return;   // nothing was flagged: the usual case
-  if ((int)blockIdx.x < a.n_row_ctas)
-    tail_rows(a, s_row);
-  else
-    tail_delta(a, s_delta, (int)blockIdx.x - a.n_row_ctas);
+  const int n_rows = a.rs->n_panel_rows, n_delta = a.rs->n_delta_rows, n_sae = a.rs->n_sae_rows;
+  if (a.mode == kTailFallback || n_sae > n_delta || (a.out_n_active != nullptr && n_sae > 0)) tail_rows(a, s_row);
+  if (a.mode != kTailFallback && n_delta > 0) {
+    const int n_items = (n_rows / kDlRows) * a.n_col_slices;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x) tail_delta(a, s_delta, item, n_rows);
+  }
+  phase_stamp(a.clk, 15, blockIdx.x == 0 && threadIdx.x == 0 && a.mode != kTailFallback);
 }
 
 }  // namespace
@@ -737,11 +753,13 @@ cudaError_t launch_tail(const Ctx* c, __nv_bfloat16* hidden, int mode, cudaStrea
   a.n_flagged = c->d_n_flagged;
   a.status = c->d_status;
   a.mode = mode;
+  a.clk = c->d_phase_clk;
   const int n_sms = c->n_sms > 0 ? c->n_sms : 148;
-  a.n_row_ctas = c->panel_rows_cap < n_sms * 6 ? c->panel_rows_cap : n_sms * 6;
   a.n_col_slices = (c->cfg.d_model / 8 + kTailThreads - 1) / kTailThreads;
-  const int n_delta = mode == kTailFallback ? 0 : (c->panel_rows_cap / kDlRows) * a.n_col_slices;
-  return launch_pdl(kPdlTail, tail_kernel, dim3(a.n_row_ctas + n_delta), dim3(kTailThreads), 0, s, a);
+  const int work_cap = c->panel_rows_cap > (c->panel_rows_cap / kDlRows) * a.n_col_slices ? c->panel_rows_cap
+                                                                                          : (c->panel_rows_cap / kDlRows) * a.n_col_slices;
+  const int grid = work_cap < n_sms * 6 ? work_cap : n_sms * 6;
+  return launch_pdl(kPdlTail, tail_kernel, dim3(grid), dim3(kTailThreads), 0, s, a);
 }
 
 }  // namespace mix
