@@ -311,7 +311,7 @@ def extras_sae(name, w, peaks, mixlib, extra_flags=0, w_enc_bytes_per_el=2.0, co
             counts[a.group] = counts.get(a.group, 0) + 1
     flops = sum(2.0 * n * w.d_model * w.groups[g].d_sae for g, n in counts.items())
     wbytes = sum(w_enc_bytes_per_el * w.d_model * w.groups[g].d_sae for g in counts)
-    enc_s = st["encode"] * 1e-3
+    enc_s = max(st["encode"], st.get("encode_pair", 0.0)) * 1e-3      # (of the two encode kernels one works, the other returns at once)
     status = m.get_status()
     m.destroy()
     layout = "8-bit E4M3 codes in blocks of 128, tile-ordered copy; 8-bit input" if extra_flags & 64 else (
@@ -682,8 +682,8 @@ def extras_sweep(peaks, mixlib, small=False):
     torch.cuda.synchronize()
     st = time_stages(m, lambda: m.apply(h))
     flops = 2.0 * T * d * S
-    enc_s = st["encode"] * 1e-3
-    out["encode"] = {"shape": "M=4096, d=4096, S=65536, one TopK weight set", "ms": st["encode"], "tflops": flops / enc_s / 1e12,
+    enc_s = max(st["encode"], st.get("encode_pair", 0.0)) * 1e-3      # (of the two encode kernels one works, the other returns at once)
+    out["encode"] = {"shape": "M=4096, d=4096, S=65536, one TopK weight set", "ms": enc_s * 1e3, "tflops": flops / enc_s / 1e12,
                      "frac_bf16_peak": flops / enc_s / 1e12 / peaks["bf16_tflops"],
                      "frac_bf16_sustained": flops / enc_s / 1e12 / peaks["bf16_tflops_sustained"],
                      "frac_bf16_nominal": flops / enc_s / 1e12 / NOMINAL_BF16_TFLOPS, "status": m.get_status()}
@@ -936,17 +936,18 @@ def collect_targets(targets, ex, w, hiddens, scores, peaks, mixlib, args):
     targets["cfg0_tiny"] = {"call_us": tiny["t_call_ms_graph"] * 1e3, "status": tiny["status"]}
     r2 = extras_sae("sae_heavy (config 2)", W.make_sae_heavy("cuda", edit_hint=gpu_edit_hint), peaks, mixlib)
     ex["sae_heavy"] = r2
-    targets["cfg2_sae_heavy"] = {"call_us": r2["t_call_ms_graph"] * 1e3, "encode_us": r2["stage_ms"]["encode"] * 1e3,
+    enc_ms = lambda r: max(r["stage_ms"]["encode"], r["stage_ms"].get("encode_pair", 0.0))
+    targets["cfg2_sae_heavy"] = {"call_us": r2["t_call_ms_graph"] * 1e3, "encode_us": enc_ms(r2) * 1e3,
                                  "encode_w_enc_gbs": r2["encode_weight_stream_gbs"], "encode_frac_hbm": r2["encode_frac_hbm_peak"],
-                                 "call_over_encode": r2["t_call_ms_graph"] / r2["stage_ms"]["encode"], "status": r2["status"]}
+                                 "call_over_encode": r2["t_call_ms_graph"] / enc_ms(r2), "status": r2["status"]}
     torch.cuda.empty_cache()
     wm = W.make_mixed("cuda", edit_hint=gpu_edit_hint)
     r3 = extras_sae("mixed (config 3)", wm, peaks, mixlib)
     ex["mixed"] = r3
-    targets["cfg3_mixed"] = {"call_us": r3["t_call_ms_graph"] * 1e3, "encode_us": r3["stage_ms"]["encode"] * 1e3,
+    targets["cfg3_mixed"] = {"call_us": r3["t_call_ms_graph"] * 1e3, "encode_us": enc_ms(r3) * 1e3,
                              "encode_tflops": r3["encode_tflops"], "encode_frac_bf16_burst": r3["encode_frac_bf16_peak"],
                              "encode_frac_bf16_sustained": r3["encode_frac_bf16_sustained"],
-                             "call_over_encode": r3["t_call_ms_graph"] / r3["stage_ms"]["encode"], "status": r3["status"]}
+                             "call_over_encode": r3["t_call_ms_graph"] / enc_ms(r3), "status": r3["status"]}
     eo = extras_sae("mixed (config 3), edit-only shortcut", wm, peaks, mixlib, extra_flags=8)
     ex["mixed_edit_only_shortcut"] = {
         "note": "MIX_FLAG_SAE_EDIT_ONLY: JumpReLU rows with the error term skip the encode (16 dot products per row "

@@ -370,7 +370,7 @@ int mix_apply_router(mix_ctx* ctx, float* logits, int n_experts, int T, void* st
 int mix_get_status(mix_ctx* ctx, unsigned* bits, void* stream);
 
 /* Number of kernels one mix_apply() call launches on this context (fixed at mix_create):
-   1 without SAE weight sets, else 6 (4 with MIX_FLAG_ENCODE_SIMT); one more when T_max > 2048
+   1 without SAE weight sets, else 7 (4 with MIX_FLAG_ENCODE_SIMT); one more when T_max > 2048
    and C_max > 1 (multi-class probes of large batches run in a kernel of their own), and two more
    with MIX_FLAG_SAE_EDIT_ONLY. */
 int mix_launches_per_apply(const mix_ctx* ctx);
@@ -381,9 +381,12 @@ int mix_launches_per_apply(const mix_ctx* ctx);
    its first kernel and events[i] after its i-th kernel, on the call's stream; the array is
    copied.  Kernel order: [probe_decide,] probe_steer, [probe_multiclass: only if T_max > 2048 and C_max > 1;
    probe_decide before and probe_tc after it if also n_groups_max == 0,]
-   front (routing + row pack), encode, tail (selection, edits, decode, write-back), encode (row tiles
-   flagged for the exact fallback selection), tail (the flagged rows); with MIX_FLAG_ENCODE_SIMT the
-   SAE part is front, encode, tail; with MIX_FLAG_SAE_EDIT_ONLY an edit_only and an edit_only_delta
+   front (routing + row pack), encode on single CTAs, encode on CTA pairs (the front kernel picks one of
+   the two per call from the routing result -- pairs when the weight sets average well over one 128-row
+   tile each -- and the other returns at once; a stage event is recorded for both even where one is
+   never launched), tail (selection, edits, decode, write-back), encode (row tiles flagged for the exact
+   fallback selection), tail (the flagged rows); with MIX_FLAG_ENCODE_SIMT the SAE part is front, encode,
+   tail; with MIX_FLAG_SAE_EDIT_ONLY an edit_only and an edit_only_delta
    kernel come last. */
 int mix_set_stage_events(mix_ctx* ctx, void* const* events);
 

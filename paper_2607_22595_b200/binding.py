@@ -309,7 +309,7 @@ class Mix:
         tail = ["edit_only", "edit_only_delta"] if self.cfg.flags & MIX_FLAG_SAE_EDIT_ONLY else []
         if self.cfg.flags & MIX_FLAG_ENCODE_SIMT:
             return front + ["front", "encode", "tail"] + tail
-        return front + ["front", "encode", "tail", "encode_flagged", "tail_flagged"] + tail
+        return front + ["front", "encode", "encode_pair", "tail", "encode_flagged", "tail_flagged"] + tail
 
     def set_stage_events(self, events=None):
         """events: list of launches_per_apply() + 1 torch.cuda.Event(enable_timing=True), or None."""

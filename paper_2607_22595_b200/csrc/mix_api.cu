@@ -80,10 +80,10 @@ cudaError_t dev_alloc(T** p, size_t n) {
 }
 
 void free_all(mix_ctx* c) {
-  cudaFree(c->d_token_slot); cudaFree(c->d_n_live); cudaFree(c->d_apps); cudaFree(c->d_groups); cudaFree(c->d_gates); cudaFree(c->d_vec_arena); cudaFree(c->d_chain_next); cudaFree(c->d_row_slot); cudaFree(c->d_row_rec);
+  cudaFree(c->d_token_slot); cudaFree(c->d_n_live); cudaFree(c->d_apps); cudaFree(c->d_groups); cudaFree(c->d_gates); cudaFree(c->d_vec_arena); cudaFree(c->d_chain_next); cudaFree(c->d_row_meta); cudaFree(c->d_front_counts); cudaFree(c->d_front_sync); cudaFree(c->d_row_rec);
   cudaFree(c->d_edit_idx); cudaFree(c->d_edit_val); cudaFree(c->d_edit_mode); cudaFree(c->d_status);
   cudaFree(c->d_tmp_req); cudaFree(c->d_tmp_req_slot); cudaFree(c->d_panel); cudaFree(c->d_panel_row); cudaFree(c->d_act_scale); cudaFree(c->d_tau); cudaFree(c->d_tau_min); cudaFree(c->d_eo_row_delta); cudaFree(c->d_eo_coef);
-  cudaFree(c->d_mtile_group); cudaFree(c->d_row_group); cudaFree(c->d_route); cudaFree(c->d_z);
+  cudaFree(c->d_mtile_group); cudaFree(c->d_route); cudaFree(c->d_z);
   cudaFree(c->d_tmap_w); cudaFree(c->d_tmap_w_half); cudaFree(c->d_phase_clk); cudaFree(c->d_tmap_probe); cudaFree(c->d_mc_dense); cudaFree(c->d_cand_val); cudaFree(c->d_cand_idx);
   cudaFree(c->d_cand_ninth); cudaFree(c->d_row_flag); cudaFree(c->d_mtile_flag); cudaFree(c->d_n_flagged);
   if (c->owned_b_eff)
@@ -207,9 +207,9 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
       cfg->r_max > kMaxEdits || cfg->n_groups_max > kMaxGroups || cfg->d_sae_max % kTileN ||
       cfg->d_sae_max > 0x7fffffffll || (cfg->n_groups_max > 0 && cfg->d_sae_max == 0))
     return MIX_ERR_UNSUPPORTED;
-  {  // the routing kernel keeps (T_max / 32) x n_groups counters in static-size shared memory
-    const long long chunks = (cfg->T_max + 1023) / 1024;
-    if (chunks * 32 * cfg->n_groups_max * 4 > 40 * 1024) return MIX_ERR_UNSUPPORTED;
+  {  // the routing kernel keeps (chunks of 256 rows) x (n_groups + 1) counters in shared memory
+    const long long chunks = (cfg->T_max + 255) / 256;
+    if (chunks * (cfg->n_groups_max + 1) * 4 > 40 * 1024) return MIX_ERR_UNSUPPORTED;
   }
   if ((cfg->flags & MIX_FLAG_SLOT_CHAINS) && (cfg->flags & MIX_FLAG_SAE_EDIT_ONLY)) return MIX_ERR_INVALID_ARG;
   if ((cfg->flags & MIX_FLAG_FP8_W_ENC) && (cfg->flags & (MIX_FLAG_ENCODE_SIMT | MIX_FLAG_SAE_EDIT_ONLY))) return MIX_ERR_INVALID_ARG;
@@ -253,8 +253,9 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
     ok = ok && dev_alloc(&c->d_panel_row, P) == cudaSuccess;
     if (cfg->flags & MIX_FLAG_FP8_W_ENC) ok = ok && dev_alloc(&c->d_act_scale, P) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_mtile_group, P / kTileM) == cudaSuccess;
-    ok = ok && dev_alloc(&c->d_row_group, T) == cudaSuccess;
-    ok = ok && dev_alloc(&c->d_row_slot, T) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_row_meta, T) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_front_counts, (size_t)front_chunks(T) * (G + 1)) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_front_sync, (size_t)front_chunks(T) + 2) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_route, 1) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_z, P * (size_t)cfg->d_sae_max) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_tmap_w, G) == cudaSuccess;
@@ -291,6 +292,7 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
   if (e == cudaSuccess && G > 0) {
     e = cudaMemset(c->d_panel, 0, (size_t)c->panel_rows_cap * cfg->d_model * sizeof(__nv_bfloat16));
     if (e == cudaSuccess) e = cudaMemset(c->d_route, 0, sizeof(RouteState));
+    if (e == cudaSuccess) e = cudaMemset(c->d_front_sync, 0, ((size_t)front_chunks(T) + 2) * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(c->d_panel_row, 0xff, c->panel_rows_cap * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(c->d_mtile_group, 0xff, c->panel_rows_cap / kTileM * sizeof(int));
     if (e == cudaSuccess && !(cfg->flags & MIX_FLAG_ENCODE_SIMT)) {
@@ -678,11 +680,15 @@ int sae_chain(mix_ctx* c, __nv_bfloat16* h, cudaStream_t s, Tap&& tap) {
     MIX_CUDA(c, launch_tail(c, h, 1, s));        // TopK from Z, edits, decode
     MIX_CUDA(c, tap());
   } else {
-    MIX_CUDA(c, launch_encode_tc(c, 0, s));      // TopK sets -> candidates, other sets -> Z
+    // TopK sets -> candidates, other sets -> Z.  Two kernels, of which the one the front kernel chose for this
+    // call does the work: single CTAs on 128-row tiles, CTA pairs on 256-row tiles (contexts of more than 128 rows)
+    if (encode_pair_mode(-1) != 1 || c->cfg.T_max <= kTileM) MIX_CUDA(c, launch_encode_tc(c, 0, false, s));
+    MIX_CUDA(c, tap());
+    if (encode_pair_possible(c)) MIX_CUDA(c, launch_encode_tc(c, 0, true, s));
     MIX_CUDA(c, tap());
     MIX_CUDA(c, launch_tail(c, h, 0, s));        // exact TopK from candidates (or a flag), edits, decode
     MIX_CUDA(c, tap());
-    MIX_CUDA(c, launch_encode_tc(c, 1, s));      // flagged row tiles -> Z (returns at once if none)
+    MIX_CUDA(c, launch_encode_tc(c, 1, false, s));   // flagged row tiles -> Z (returns at once if none)
     MIX_CUDA(c, tap());
     MIX_CUDA(c, launch_tail(c, h, 2, s));        // the flagged rows (returns at once if none)
     MIX_CUDA(c, tap());
@@ -826,7 +832,7 @@ int mix_launches_per_apply(const mix_ctx* c) {
   if (!c) return 0;
   const int front = 1 + (has_multiclass_stage(c) ? 1 : 0) + (has_tc_probe_stage(c) ? 2 : 0);
   if (c->cfg.n_groups_max == 0) return front;
-  return front + ((c->cfg.flags & MIX_FLAG_ENCODE_SIMT) ? 3 : 5) + ((c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) ? 2 : 0);   // coefficient kernel + delta kernel
+  return front + ((c->cfg.flags & MIX_FLAG_ENCODE_SIMT) ? 3 : 6) + ((c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) ? 2 : 0);   // coefficient kernel + delta kernel
 }
 
 int mix_get_status(mix_ctx* c, unsigned* bits, void* stream) {

@@ -95,7 +95,8 @@ struct RouteState {
   int total_tiles;                  // encode tiles over all groups
   int n_topk_rows;                  // SAE rows whose weight set is TopK
   int n_delta_rows;                 // ReLU / JumpReLU rows that keep the error term and have edits (the tail kernel's delta role)
-  int pad_[2];
+  int use_pair;                     // this call's encode runs on CTA pairs (256-row tiles) rather than on single CTAs
+  int pad_;
   int group_count[kMaxGroups];      // M_g
   int group_mtile0[kMaxGroups + 1]; // first m-tile of group g in the panel
   int group_tile0[kMaxGroups + 1];  // first linear encode tile of group g
@@ -136,8 +137,9 @@ struct Ctx {
   float* d_act_scale;       // [P] row scales of the 8-bit panel (MIX_FLAG_FP8_ACT only)
   int* d_panel_row;         // [P] token index or -1
   int* d_mtile_group;       // [P / kTileM] group of each m-tile or -1
-  int* d_row_group;         // [T_max] routing scratch: weight set of each token row or -1
-  int* d_row_slot;          // [T_max] routing scratch: slot of the SAE app that acts on the row (batches beyond the first 8192 rows)
+  int2* d_row_meta;         // [T_max] front kernel: per token row, what its chunk's CTA found out (weight set, edit count, flags; slot)
+  int* d_front_counts;      // [chunks of 256 token rows][n_groups_max + 1] front kernel: SAE rows per weight set and chunk
+  int* d_front_sync;        // [2 + chunks] front kernel: epoch, CTAs done, per-chunk publication epoch
   RowRec* d_row_rec;        // [P] per packed row: token row, slot, edit count, weight set, error-term flag
   RouteState* d_route;
   float* d_z;               // [P, d_sae_max]
@@ -210,11 +212,14 @@ cudaError_t launch_pdl(int which, void (*kernel)(KArgs...), dim3 grid, dim3 bloc
 #endif
 
 #ifdef __CUDACC__
-// Profiling aid: thread `who` (a bool) stamps slot i of the phase-clock array with the global nanosecond timer.
+// Profiling aid: thread `who` (a bool) stamps slot i of the phase-clock array: slots 0, 7, 8 and 15 (a kernel's
+// first and last stamps) with the global nanosecond timer, the others with the SM's cycle counter -- cheap to
+// read, and comparable between stamps of the same CTA.
 __device__ __forceinline__ void phase_stamp(unsigned long long* clk, int i, bool who) {
   if (clk != nullptr && who) {
     unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    if (i == 0 || i == 7 || i == 8 || i == 15) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    else t = (unsigned long long)clock64();
     clk[i] = t;
   }
 }
@@ -246,8 +251,10 @@ cudaError_t launch_router(const Ctx* c, float* logits, int n_experts, int T, cud
 // routed > 0); plain calls pass 0, 0
 cudaError_t launch_front(const Ctx* c, const __nv_bfloat16* hidden, int T, cudaStream_t s, unsigned long long cond = 0,
                          int use_cond = 0);
+int front_chunks(int T_max);       // chunks of token rows the front kernel classifies: sizes d_front_counts / d_front_sync
 cudaError_t launch_encode_simt(const Ctx* c, cudaStream_t s);
-cudaError_t launch_encode_tc(const Ctx* c, int mode, cudaStream_t s);   // 0: all tiles; 1: flagged row tiles -> Z
+cudaError_t launch_encode_tc(const Ctx* c, int mode, bool pair, cudaStream_t s);   // 0: all tiles; 1: flagged row tiles -> Z
+bool encode_pair_possible(const Ctx* c);   // the CTA-pair encode kernel is part of this context's launch sequence
 // Selection, edits, decode and write-back of every SAE row.  mode 0: behind the tensor-core encode (TopK from its
 // candidates; rows it cannot settle are flagged); 1: behind the CUDA-core encode (TopK from Z); 2: the flagged
 // rows, after their row tiles were re-encoded to Z (returns at once when nothing is flagged).
@@ -261,7 +268,10 @@ cudaError_t launch_fold_bias(const __nv_bfloat16* W_enc, const float* b_enc, con
 cudaError_t launch_retile(const __nv_bfloat16* W_enc, __nv_bfloat16* W_tiled, long long d_sae, int d, cudaStream_t s);
 cudaError_t launch_retile_fp8(const unsigned char* W_enc, unsigned char* W_tiled, long long d_sae, int d, int kb_bytes, cudaStream_t s);
 cudaError_t encode_tc_prepare();   // opt in to the large dynamic shared memory size
-constexpr int kEncodePairDefault = 0;   // the encode on CTA pairs (tcgen05 cta_group::2) unless MIX_ENCODE_PAIR says otherwise
+// The encode has two kernels -- single CTAs on 128-row tiles, CTA pairs (tcgen05 cta_group::2) on 256-row tiles --
+// and the front kernel decides per call, from the routing result, which of them works (the other returns at once).
+// MIX_ENCODE_PAIR in the environment forces one: 0 single CTAs, 1 pairs; unset (or 2) = decided on the device.
+constexpr int kEncodePairDefault = 2;
 int encode_pair_mode(int set);     // returns the mode in force; set >= 0 changes it (A/B timing)
 
 }  // namespace mix

@@ -264,6 +264,8 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
   }
   __syncthreads();
   if (sh->rs.total_tiles == 0) return;     // nothing routed to any SAE: no tensor memory is taken (both CTAs of a pair see the same)
+  // the full pass has two kernels, single CTAs and CTA pairs; the front kernel chose one for this call
+  if (mode == 0 && (sh->rs.use_pair != 0) != kPair) return;
   const int total_tiles = kPair ? sh->ptile0[n_groups] : sh->rs.total_tiles;
 
   if (warp == 1) {
@@ -624,9 +626,12 @@ cudaError_t encode_tc_prepare() {
 // CTA pairs or single CTAs: MIX_ENCODE_PAIR in the environment (0 / 1), read once; set by mix_set_encode_pair for A/B timing.
 static int g_encode_pair = -1;
 int encode_pair_mode(int set) {
-  if (g_encode_pair < 0) g_encode_pair = getenv("MIX_ENCODE_PAIR") ? (atoi(getenv("MIX_ENCODE_PAIR")) != 0) : kEncodePairDefault;
+  if (g_encode_pair < 0) {
+    const int v = getenv("MIX_ENCODE_PAIR") ? atoi(getenv("MIX_ENCODE_PAIR")) : kEncodePairDefault;
+    g_encode_pair = v == 0 || v == 1 ? v : 2;
+  }
   const int old = g_encode_pair;
-  if (set >= 0) g_encode_pair = set != 0;
+  if (set >= 0) g_encode_pair = set == 0 || set == 1 ? set : 2;
   return old;
 }
 
@@ -668,10 +673,12 @@ static cudaError_t launch_encode_tc_as(const Ctx* c, int mode, cudaStream_t s) {
 // Eight epilogue warps pay off for the TopK epilogue (selection work per element); the plain store of the
 // pre-activations is a little faster with four.  Either form is correct for any mix of weight sets; the choice
 // is made from the sets registered when the call is enqueued (or captured).
-cudaError_t launch_encode_tc(const Ctx* c, int mode, cudaStream_t s) {
+// pair: the CTA-pair kernel (256-row tiles) or the single-CTA kernel; a full pass (mode 0) launches both, and
+// the one the front kernel did not choose for this call returns at once.
+cudaError_t launch_encode_tc(const Ctx* c, int mode, bool pair, cudaStream_t s) {
   bool topk = false;
   for (int g = 0; g < c->cfg.n_groups_max; ++g) topk = topk || (c->h_groups[g].valid && c->h_groups[g].act == MIX_SAE_TOPK);
-  if (encode_pair_mode(-1)) {
+  if (pair) {
     if (c->cfg.flags & MIX_FLAG_FP8_ACT) return topk ? launch_encode_tc_as<2, 8, true>(c, mode, s) : launch_encode_tc_as<2, 4, true>(c, mode, s);
     if (c->cfg.flags & MIX_FLAG_FP8_W_ENC) return topk ? launch_encode_tc_as<1, 8, true>(c, mode, s) : launch_encode_tc_as<1, 4, true>(c, mode, s);
     return topk ? launch_encode_tc_as<0, 8, true>(c, mode, s) : launch_encode_tc_as<0, 4, true>(c, mode, s);
@@ -680,5 +687,7 @@ cudaError_t launch_encode_tc(const Ctx* c, int mode, cudaStream_t s) {
   if (c->cfg.flags & MIX_FLAG_FP8_W_ENC) return topk ? launch_encode_tc_as<1, 8, false>(c, mode, s) : launch_encode_tc_as<1, 4, false>(c, mode, s);
   return topk ? launch_encode_tc_as<0, 8, false>(c, mode, s) : launch_encode_tc_as<0, 4, false>(c, mode, s);
 }
+
+bool encode_pair_possible(const Ctx* c) { return encode_pair_mode(-1) != 0 && c->cfg.T_max > kTileM; }
 
 }  // namespace mix

@@ -2,11 +2,10 @@
 //
 // Routing is integer work on the slot map: which rows carry an SAE app, of which weight set, and where each of
 // them goes in the packed panel (weight set by weight set, ascending token order inside a set, every set
-// starting on a 128-row tile).  It used to be a one-CTA kernel followed by a pack kernel that waited for it.
-// Here EVERY CTA repeats the routing for itself -- the slot map and the small tables are a few tens of KiB, L2
-// hits after the first CTA -- and then packs its own 32 panel rows, one per warp: no CTA waits for another, and
-// one launch and one dependent kernel boundary disappear from the front of every SAE call.  CTA 0 alone writes
-// what exists once (the routing result the encode reads, the tile -> weight-set map, the conditional handle).
+// starting on a 128-row tile).  The kernel does it as a chunked scan inside one grid -- every CTA classifies 256
+// token rows and publishes their counts, every CTA then reads the small count table -- and packs the rows right
+// after, each CTA the eight panel rows it owns, found through the published per-row records.  The only waiting
+// between CTAs is a bounded wait for the published chunks; see front_kernel.
 //
 // Pack forms: the bf16 row as it is; with an 8-bit encoder the row as E4M3 codes with a power-of-two row
 // scale -- quantised (MIX_FLAG_FP8_ACT), or split exactly into two E4M3 operands hi + lo.
@@ -20,10 +19,8 @@ namespace mix {
 
 namespace {
 
-constexpr int kFrontThreads = 1024;
-constexpr int kFrontWarps = kFrontThreads / 32;
-constexpr int kFrontRowsMax = 512;        // most panel rows one CTA packs (a multiple of 32: whole rounds of one row per warp)
-constexpr int kRouteBatch = 8;            // chunks of 1024 rows whose look-ups are in flight together
+constexpr int kFrontThreads = 256;        // = token rows a CTA classifies
+constexpr int kFrontWarps = kFrontThreads / 32;   // = panel rows a CTA packs
 
 // bf16 row -> panel row (or zeros for the padding rows of a tile: they must be finite).
 __device__ __forceinline__ void pack_row_bf16(const __nv_bfloat16* __restrict__ hidden, int t, __nv_bfloat16* __restrict__ panel,
@@ -116,19 +113,20 @@ struct FrontArgs {
   int n_groups;
   const int* chain_next;
   int edit_only;
+  // exchange between the CTAs of one launch
+  int2* row_meta;          // [T_max] per token row: (weight set + 1) | edit count << 8 | error-term flag << 16 (0: not an SAE row), slot
+  int* counts;             // [chunks][n_groups + 1] SAE rows per weight set in each chunk of 256 token rows; last column: delta-role rows
+  int* sync;               // [0] epoch of the last finished call, [1] CTAs of this call that are done, [2 + c] epoch in which chunk c was published
   // routing results (written)
   int* panel_row;
   RowRec* row_rec;
   int panel_cap;
-  int rows_per_cta;        // panel rows packed by one CTA: a multiple of 32, <= kFrontRowsMax
   int* mtile_group;
   RouteState* rs;
   unsigned* status;
   int* row_flag;
   int* mtile_flag;
   int* n_flagged;
-  int* row_group;          // scratch, used only by batches beyond the first 8192 rows
-  int* row_slot;           // scratch, likewise
   cudaGraphConditionalHandle cond;
   int use_cond;
   // pack
@@ -140,279 +138,282 @@ struct FrontArgs {
   unsigned* tau_min;
   int lo_row0;
   unsigned long long* clk;   // profiling aid or null
+  int pair_mode;             // 0: the encode runs on single CTAs, 1: on CTA pairs, 2: decided here from the routing result
 };
 
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release(int* p, int v) { asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory"); }
+
+constexpr long long kFrontWaitCycles = 2000000000ll;   // ~1 s: cap of the wait for the other CTAs' chunks
+
+// One launch, three steps, no CTA doing another's work:
+//   1. CTA c < chunks classifies token rows [256 c, 256 c + 256) -- slot -> app entry -> SAE row of which weight set --
+//      and PUBLISHES the chunk: per-row records, per-set counts, then a flag carrying this call's epoch.
+//   2. Every CTA waits (bounded) until all chunks carry the epoch, reads the small count table and scans it: totals
+//      per weight set, the sets' first panel rows, and for every chunk the rank of its first row within each set.
+//      The publishing CTAs never wait before they publish, and CTAs are dispatched in index order, so whoever waits,
+//      waits for work that is already running.
+//   3. CTA b packs panel rows [8 b, 8 b + 8), one per warp: the row's set and rank follow from its position, the
+//      chunk that holds that rank from the scan, the token from that chunk's published records.
+// CTA 0 alone writes what exists once (the routing result the encode reads, the tile -> weight-set map, the
+// conditional handle).  The epoch advances when the last CTA of the launch leaves.
 // kPack: 0 the bf16 row, 1 E4M3 hi + lo (exact split), 2 E4M3 quantised.
 template <int kPack>
 __global__ void __launch_bounds__(kFrontThreads)
 front_kernel(const FrontArgs a) {
-  extern __shared__ int s_cnt[];                      // [n_chunks * kFrontWarps][n_groups]
-  __shared__ int s_total[kMaxGroups], s_base[kMaxGroups + 1];
-  __shared__ int s_tok[kFrontRowsMax], s_slot[kFrontRowsMax], s_grp[kFrontRowsMax];
-  __shared__ int s_n_panel_rows;
+  extern __shared__ int s_tab[];                      // [chunks][n_groups + 1]: counts, then exclusive prefixes over the chunks
+  __shared__ int s_total[kMaxGroups + 1], s_base[kMaxGroups + 1];
   __shared__ int s_gact[kMaxGroups], s_gtiles[kMaxGroups];   // per weight set: activation, feature tiles (0: not registered)
-  __shared__ int s_n_delta;
+  __shared__ int s_wcnt[kFrontWarps][kMaxGroups + 1];
+  __shared__ int s_n_panel_rows;
   pdl_launch_dependents();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const bool first_cta = blockIdx.x == 0;
-  const int n_groups = a.n_groups, n_slots = a.n_slots;
-  const int n_live = min(a.T, __ldg(a.n_live_p));
-  const int n_chunks = (n_live + kFrontThreads - 1) / kFrontThreads;
+  const int cta = blockIdx.x;
+  const bool first_cta = cta == 0;
+  const int n_groups = a.n_groups, n_slots = a.n_slots, ncol = n_groups + 1;
+  const int n_chunks = (a.T + kFrontThreads - 1) / kFrontThreads;     // the same in every CTA: who publishes is fixed by the launch
   phase_stamp(a.clk, 0, first_cta && tid == 0);
-  const int n_own = a.rows_per_cta;
-  const int p0 = blockIdx.x * n_own;
-  if (tid < n_own) s_tok[tid] = -1;
-  if (tid == 0) s_n_delta = 0;
-  if (tid < n_groups) {                                // requested now, needed after the scan
+  const int target = ld_acquire(a.sync) + 1;          // this call's epoch
+  if (tid < n_groups) {                                // requested now, needed after the first barrier
     const bool valid = __ldg(&a.groups[tid].valid) != 0;
     s_gact[tid] = __ldg(&a.groups[tid].act);
     s_gtiles[tid] = valid ? (int)(__ldg(&a.groups[tid].d_sae) / kTileN) : 0;
   }
-
-  // phase A: the weight set (or -1) of every row this thread owns (row c * 1024 + tid of chunk c), resolved
-  // stage by stage for kRouteBatch chunks at a time so that their loads are in flight together: the slot ids
-  // (requested together with the live count), then bytes 0..31 of the app entries -- valid, kind, weight set,
-  // edit count, error-term flag in one round trip; the weight sets' own entries were requested at the top of
-  // the kernel.  Then per (chunk, warp) counts per set.  The first batch (8192 rows: every configuration in use)
-  // stays in registers for phase C; later batches go through the row_group / row_slot scratch (every CTA writes
-  // the same values there and reads back its own).
-  // meta: (weight set + 1) | edit count << 8 | error-term flag << 16; 0 = not an SAE row of this call
-  int meta0[kRouteBatch], slot0[kRouteBatch];
-  const int T_cap = a.T;
-  const int n_chunks_cap = (T_cap + kFrontThreads - 1) / kFrontThreads;
-  bool groups_ready = false;
-  for (int c0 = 0; c0 < n_chunks_cap; c0 += kRouteBatch) {
-    int slot[kRouteBatch], meta[kRouteBatch];
-#pragma unroll
-    for (int c = 0; c < kRouteBatch; ++c) {
-      const int t = (c0 + c) * kFrontThreads + tid;
-      slot[c] = t < T_cap ? __ldg(a.token_slot + t) : -1;      // does not wait for the live count
+  // ---- step 1: classify and publish one chunk
+  if (cta < n_chunks) {
+    const int t = cta * kFrontThreads + tid;
+    const int n_live = min(a.T, __ldg(a.n_live_p));   // both loads issue together
+    int slot = t < a.T ? __ldg(a.token_slot + t) : -1;
+    if (t >= n_live || slot >= n_slots) slot = -1;
+    int2 q0 = make_int2(0, 0);                         // valid, kind
+    int g = -1, n_edit = 0, add_error = 0;
+    if (slot >= 0) {
+      const AppEntry* e = a.apps + slot;
+      q0 = __ldg(reinterpret_cast<const int2*>(e));
+      g = __ldg(&e->group);
+      const int2 ne = __ldg(reinterpret_cast<const int2*>(&e->n_edit));
+      n_edit = ne.x;
+      add_error = ne.y != 0;
     }
-    if (c0 >= n_chunks) break;                                  // (uniform) nothing live from here on
-#pragma unroll
-    for (int c = 0; c < kRouteBatch; ++c) {
-      const int t = (c0 + c) * kFrontThreads + tid;
-      if (t >= n_live || slot[c] >= n_slots) slot[c] = -1;
-    }
-    int2 q0[kRouteBatch];                 // valid, kind
-    int3 q1[kRouteBatch];                 // weight set, edit count, error-term flag
-#pragma unroll
-    for (int c = 0; c < kRouteBatch; ++c) {
-      q0[c] = make_int2(0, 0);
-      q1[c] = make_int3(0, 0, 0);
-      if (slot[c] >= 0) {
-        const AppEntry* e = a.apps + slot[c];
-        q0[c] = __ldg(reinterpret_cast<const int2*>(e));
-        q1[c].x = __ldg(&e->group);
-        const int2 ne = __ldg(reinterpret_cast<const int2*>(&e->n_edit));
-        q1[c].y = ne.x;
-        q1[c].z = ne.y;
+    // a row whose slot starts a chain is an SAE row if the chain ends in an SAE app: follow the links
+    if (q0.x && (q0.y & kKindChained) && (q0.y & kKindMask) != MIX_SAE) {
+      int s2 = slot;
+      int2 h2 = q0;
+      for (int depth = 1; depth < kMaxChain && s2 >= 0; ++depth) {
+        s2 = (h2.y & kKindChained) ? __ldg(a.chain_next + s2) : -1;
+        if (s2 < 0 || s2 >= n_slots) { s2 = -1; break; }
+        h2 = __ldg(reinterpret_cast<const int2*>(a.apps + s2));
+        if (!h2.x) { s2 = -1; break; }
+        if ((h2.y & kKindMask) == MIX_SAE) break;
+      }
+      if (s2 >= 0 && (h2.y & kKindMask) != MIX_SAE) s2 = -1;
+      slot = s2;
+      q0 = s2 >= 0 ? h2 : make_int2(0, 0);
+      if (s2 >= 0) {
+        g = __ldg(&a.apps[s2].group);
+        n_edit = __ldg(&a.apps[s2].n_edit);
+        add_error = __ldg(&a.apps[s2].add_error) != 0;
       }
     }
-    // a row whose slot starts a chain is an SAE row if the chain ends in an SAE app: follow the
-    // links (rare, so the dependent loads are not batched) and carry on with that app's slot
-#pragma unroll
-    for (int c = 0; c < kRouteBatch; ++c) {
-      if (q0[c].x && (q0[c].y & kKindChained) && (q0[c].y & kKindMask) != MIX_SAE) {
-        int s2 = slot[c];
-        int2 h2 = q0[c];
-        for (int depth = 1; depth < kMaxChain && s2 >= 0; ++depth) {
-          s2 = (h2.y & kKindChained) ? __ldg(a.chain_next + s2) : -1;
-          if (s2 < 0 || s2 >= n_slots) { s2 = -1; break; }
-          h2 = __ldg(reinterpret_cast<const int2*>(a.apps + s2));
-          if (!h2.x) { s2 = -1; break; }
-          if ((h2.y & kKindMask) == MIX_SAE) break;
-        }
-        if (s2 >= 0 && (h2.y & kKindMask) != MIX_SAE) s2 = -1;
-        slot[c] = s2;
-        q0[c] = s2 >= 0 ? h2 : make_int2(0, 0);
-        q1[c] = make_int3(0, 0, 0);
-        if (s2 >= 0) {
-          q1[c].x = __ldg(&a.apps[s2].group);
-          q1[c].y = __ldg(&a.apps[s2].n_edit);
-          q1[c].z = __ldg(&a.apps[s2].add_error);
-        }
+    __syncthreads();                                   // the weight-set table is in shared memory
+    int meta = 0, is_delta = 0;
+    if (q0.x && (q0.y & kKindMask) == MIX_SAE) {
+      if (g < 0 || g >= n_groups || s_gtiles[g] == 0) {
+        atomicOr(a.status, MIX_STATUS_BAD_GROUP);
+      } else if (a.edit_only && add_error && s_gact[g] != MIX_SAE_TOPK) {
+        // handled by sae_edit_only_kernel: with the error term on, a ReLU / JumpReLU row needs
+        // only the pre-activations of its edited features, not the whole encode
+      } else if (!(q0.y & kKindGated) || gate_open(a.gates, slot, t)) {
+        meta = (g + 1) | (n_edit << 8) | (add_error << 16);
+        is_delta = add_error && n_edit > 0 && s_gact[g] != MIX_SAE_TOPK;
       }
     }
-    if (!groups_ready) {                   // the weight-set table requested at the top has long arrived
-      __syncthreads();
-      groups_ready = true;
-    }
-    int n_delta = 0;
-#pragma unroll
-    for (int c = 0; c < kRouteBatch; ++c) {
-      meta[c] = 0;
-      if (q0[c].x && (q0[c].y & kKindMask) == MIX_SAE) {
-        const int g = q1[c].x, n_edit = q1[c].y, add_error = q1[c].z != 0;
-        if (g < 0 || g >= n_groups || s_gtiles[g] == 0) {
-          if (first_cta) atomicOr(a.status, MIX_STATUS_BAD_GROUP);
-        } else if (a.edit_only && add_error && s_gact[g] != MIX_SAE_TOPK) {
-          // handled by sae_edit_only_kernel: with the error term on, a ReLU / JumpReLU row needs
-          // only the pre-activations of its edited features, not the whole encode
-        } else if (!(q0[c].y & kKindGated) || gate_open(a.gates, slot[c], (c0 + c) * kFrontThreads + tid)) {
-          meta[c] = (g + 1) | (n_edit << 8) | (add_error << 16);
-          n_delta += add_error && n_edit > 0 && s_gact[g] != MIX_SAE_TOPK;
-        }
-      }
-    }
-    n_delta = __reduce_add_sync(0xffffffffu, n_delta);
-    if (lane == 0 && n_delta) atomicAdd(&s_n_delta, n_delta);
-#pragma unroll
-    for (int c = 0; c < kRouteBatch; ++c) {
-      if (c0 == 0) {
-        meta0[c] = meta[c];
-        slot0[c] = slot[c];
-      }
-      if (c0 + c < n_chunks) {                       // uniform across the CTA
-        const int t = (c0 + c) * kFrontThreads + tid;
-        if (c0 > 0 && t < n_live) {
-          a.row_group[t] = meta[c];
-          a.row_slot[t] = slot[c];
-        }
-        const int grp = (meta[c] & 0xff) - 1;
-        for (int q = 0; q < n_groups; ++q) {
-          const unsigned m = __ballot_sync(0xffffffffu, grp == q);
-          if (lane == 0) s_cnt[((c0 + c) * kFrontWarps + warp) * n_groups + q] = __popc(m);
-        }
-      }
-    }
-  }
-  if (!groups_ready) __syncthreads();
-  phase_stamp(a.clk, 1, first_cta && tid == 0);
-  if (n_chunks == 0) {
-#pragma unroll
-    for (int c = 0; c < kRouteBatch; ++c) {
-      meta0[c] = 0;
-      slot0[c] = -1;
-    }
-  }
-  __syncthreads();
-  // phase B: exclusive scan over (chunk, warp) for each weight set; warp q owns set q
-  const int n_seg = n_chunks * kFrontWarps;
-  for (int q = warp; q < n_groups; q += kFrontWarps) {
-    int carry = 0;
-    for (int s0 = 0; s0 < n_seg; s0 += 32) {
-      const int i = s0 + lane;
-      const int v = i < n_seg ? s_cnt[i * n_groups + q] : 0;
-      int incl = v;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int y = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += y;
-      }
-      if (i < n_seg) s_cnt[i * n_groups + q] = carry + incl - v;
-      carry += __shfl_sync(0xffffffffu, incl, 31);
-    }
-    if (lane == 0) s_total[q] = carry;
-  }
-  __syncthreads();
-  if (tid == 0) {
-    int mt = 0, tiles = 0, rows = 0, topk_rows = 0;
+    if (t < a.T) a.row_meta[t] = make_int2(meta, slot);
+    const int grp = (meta & 0xff) - 1;
     for (int q = 0; q < n_groups; ++q) {
-      s_base[q] = mt * kTileM;
-      const int m_tiles = (s_total[q] + kTileM - 1) / kTileM;
-      const int act = s_gact[q];
-      if (first_cta) {
-        a.rs->group_count[q] = s_total[q];
-        a.rs->group_mtile0[q] = mt;
-        a.rs->group_tile0[q] = tiles;
-        for (int m = 0; m < m_tiles; ++m) a.mtile_group[mt + m] = q;
-      }
-      mt += m_tiles;
-      rows += s_total[q];
-      if (s_total[q] > 0 && act == MIX_SAE_TOPK) topk_rows += s_total[q];
-      tiles += s_total[q] > 0 ? m_tiles * s_gtiles[q] : 0;
+      const unsigned m = __ballot_sync(0xffffffffu, grp == q);
+      if (lane == 0) s_wcnt[warp][q] = __popc(m);
     }
-    s_base[n_groups] = mt * kTileM;
-    s_n_panel_rows = mt * kTileM;
-    if (first_cta) {
-      for (int q = n_groups; q <= kMaxGroups; ++q) {
-        a.rs->group_mtile0[q] = mt;
-        a.rs->group_tile0[q] = tiles;
-        if (q < kMaxGroups) a.rs->group_count[q] = 0;
-      }
-      for (int m = mt; m < a.panel_cap / kTileM; ++m) a.mtile_group[m] = -1;
-      a.rs->n_panel_rows = mt * kTileM;
-      a.rs->n_mtiles = mt;
-      a.rs->n_sae_rows = rows;
-      a.rs->total_tiles = tiles;
-      a.rs->n_topk_rows = topk_rows;
-      a.rs->n_delta_rows = s_n_delta;
-      if (a.n_flagged) *a.n_flagged = 0;       // fallback-selection flags of the fused TopK path start clear every call
-      // graph-conditional form: the rest of the SAE chain sits in the body of an IF node that runs only when a row needs it
-      if (a.use_cond) cudaGraphSetConditional(a.cond, rows > 0 ? 1u : 0u);
+    {
+      const unsigned m = __ballot_sync(0xffffffffu, is_delta != 0);
+      if (lane == 0) s_wcnt[warp][n_groups] = __popc(m);
+    }
+    __syncthreads();
+    if (tid < ncol) {
+      int sum = 0;
+#pragma unroll
+      for (int w = 0; w < kFrontWarps; ++w) sum += s_wcnt[w][tid];
+      a.counts[cta * ncol + tid] = sum;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) st_release(a.sync + 2 + cta, target);
+  } else {
+    __syncthreads();                                   // (the weight-set table)
+  }
+  phase_stamp(a.clk, 1, first_cta && tid == 0);
+  // ---- step 2: wait for every chunk, scan the counts
+  bool ok = true;
+  for (int c = tid; c < n_chunks; c += kFrontThreads) {
+    if (ld_acquire(a.sync + 2 + c) == target) continue;
+    const long long t0 = clock64();
+    while (ld_acquire(a.sync + 2 + c) != target) {
+      if (clock64() - t0 > kFrontWaitCycles) { ok = false; break; }
+      __nanosleep(64);
     }
   }
-  if (first_cta && a.mtile_flag)
-    for (int m = tid; m < a.panel_cap / kTileM; m += kFrontThreads) a.mtile_flag[m] = 0;
-  __syncthreads();
-  phase_stamp(a.clk, 2, first_cta && tid == 0);
-  // phase C: stable positions; a row that lands in this CTA's share of the panel leaves its token here
-  for (int c0 = 0; c0 < n_chunks; c0 += kRouteBatch) {
-    int meta[kRouteBatch], slot[kRouteBatch];
+  ok = __syncthreads_and(ok) != 0;
+  if (ok) {
+    for (int i = tid; i < n_chunks * ncol; i += kFrontThreads) s_tab[i] = __ldcg(a.counts + i);   // (never through L1: written by other SMs)
+    __syncthreads();
+    for (int q = warp; q < ncol; q += kFrontWarps) {   // exclusive scan over the chunks, one column per warp
+      int carry = 0;
+      for (int c0 = 0; c0 < n_chunks; c0 += 32) {
+        const int c = c0 + lane;
+        const int v = c < n_chunks ? s_tab[c * ncol + q] : 0;
+        int incl = v;
 #pragma unroll
-    for (int c = 0; c < kRouteBatch; ++c) {
-      const int t = (c0 + c) * kFrontThreads + tid;
-      if (c0 == 0) {
-        meta[c] = meta0[c];
-        slot[c] = slot0[c];
-      } else {
-        meta[c] = (c0 + c < n_chunks && t < n_live) ? a.row_group[t] : 0;
-        slot[c] = meta[c] ? a.row_slot[t] : -1;
+        for (int o = 1; o < 32; o <<= 1) {
+          const int y = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += y;
+        }
+        if (c < n_chunks) s_tab[c * ncol + q] = carry + incl - v;
+        carry += __shfl_sync(0xffffffffu, incl, 31);
+      }
+      if (lane == 0) s_total[q] = carry;
+    }
+    __syncthreads();
+    phase_stamp(a.clk, 2, first_cta && tid == 0);
+    if (tid == 0) {
+      int mt = 0, tiles = 0, rows = 0, topk_rows = 0, pair_tiles = 0;
+      for (int q = 0; q < n_groups; ++q) {
+        s_base[q] = mt * kTileM;
+        const int m_tiles = (s_total[q] + kTileM - 1) / kTileM;
+        if (first_cta) {
+          a.rs->group_count[q] = s_total[q];
+          a.rs->group_mtile0[q] = mt;
+          a.rs->group_tile0[q] = tiles;
+          for (int m = 0; m < m_tiles; ++m) a.mtile_group[mt + m] = q;
+        }
+        mt += m_tiles;
+        rows += s_total[q];
+        if (s_total[q] > 0 && s_gact[q] == MIX_SAE_TOPK) topk_rows += s_total[q];
+        tiles += s_total[q] > 0 ? m_tiles * s_gtiles[q] : 0;
+        pair_tiles += s_total[q] > 0 ? ((m_tiles + 1) / 2) * s_gtiles[q] : 0;
+      }
+      s_base[n_groups] = mt * kTileM;
+      s_n_panel_rows = mt * kTileM;
+      if (first_cta) {
+        for (int q = n_groups; q <= kMaxGroups; ++q) {
+          a.rs->group_mtile0[q] = mt;
+          a.rs->group_tile0[q] = tiles;
+          if (q < kMaxGroups) a.rs->group_count[q] = 0;
+        }
+        for (int m = mt; m < a.panel_cap / kTileM; ++m) a.mtile_group[m] = -1;
+        a.rs->n_panel_rows = mt * kTileM;
+        a.rs->n_mtiles = mt;
+        a.rs->n_sae_rows = rows;
+        a.rs->total_tiles = tiles;
+        a.rs->n_topk_rows = topk_rows;
+        a.rs->n_delta_rows = s_total[n_groups];
+        // A pair-tile keeps two SMs busy for about 3/4 of the time one SM needs for a 128-row tile (a third less
+        // shared-memory fill per SM), so pairs win when the weight sets average well over one row tile each, and lose
+        // where most sets have a single row tile (half of every pair would repeat the other half's work).
+        a.rs->use_pair = a.pair_mode == 2 ? (3 * pair_tiles <= 2 * tiles) : a.pair_mode;
+        if (a.n_flagged) *a.n_flagged = 0;       // fallback-selection flags of the fused TopK path start clear every call
+        // graph-conditional form: the rest of the SAE chain sits in the body of an IF node that runs only when a row needs it
+        if (a.use_cond) cudaGraphSetConditional(a.cond, rows > 0 ? 1u : 0u);
       }
     }
+    if (first_cta && a.mtile_flag)
+      for (int m = tid; m < a.panel_cap / kTileM; m += kFrontThreads) a.mtile_flag[m] = 0;
+    __syncthreads();
+    phase_stamp(a.clk, 3, first_cta && tid == 0);
+    // ---- step 3: this CTA's panel rows, one per warp
+    const int p = cta * kFrontWarps + warp;
+    if (p < a.panel_cap) {
+      int t = -1, meta = 0, slot = -1;
+      if (p < s_n_panel_rows) {
+        int g = 0;
+        while (g + 1 < n_groups && p >= s_base[g + 1]) ++g;
+        const int r = p - s_base[g];                   // rank of the row within its weight set
+        if (r < s_total[g]) {
+          // the chunk that holds rank r: the last one whose first rank is <= r
+          int c_hit = 0;
+          for (int c0 = 0; c0 < n_chunks; c0 += 32) {
+            const int c = c0 + lane;
+            const unsigned m = __ballot_sync(0xffffffffu, c < n_chunks && s_tab[c * ncol + g] <= r);
+            if (m) c_hit = c0 + 31 - __clz(m);
+          }
+          int left = r - s_tab[c_hit * ncol + g];      // rank inside the chunk
+          int2 mm[kFrontThreads / 32];
 #pragma unroll
-    for (int c = 0; c < kRouteBatch; ++c) {
-      if (c0 + c < n_chunks) {
-        const int grp = (meta[c] & 0xff) - 1;
-        for (int q = 0; q < n_groups; ++q) {
-          const unsigned m = __ballot_sync(0xffffffffu, grp == q);
-          if (grp == q) {
-            const int pos = s_base[q] + s_cnt[((c0 + c) * kFrontWarps + warp) * n_groups + q] +
-                            __popc(m & ((1u << lane) - 1u));
-            if (pos >= p0 && pos < p0 + n_own) {
-              s_tok[pos - p0] = (c0 + c) * kFrontThreads + tid;
-              s_slot[pos - p0] = slot[c];
-              s_grp[pos - p0] = meta[c];
+          for (int i = 0; i < kFrontThreads / 32; ++i) {
+            const int tt = c_hit * kFrontThreads + i * 32 + lane;
+            mm[i] = tt < a.T ? __ldcg(a.row_meta + tt) : make_int2(0, -1);
+          }
+          bool found = false;
+#pragma unroll
+          for (int i = 0; i < kFrontThreads / 32; ++i) {
+            const unsigned m = __ballot_sync(0xffffffffu, (mm[i].x & 0xff) - 1 == g);
+            const int cnt = __popc(m);
+            if (!found) {
+              if (left < cnt) {
+                const int src = __fns(m, 0, left + 1);
+                t = c_hit * kFrontThreads + i * 32 + src;
+                meta = __shfl_sync(0xffffffffu, mm[i].x, src);
+                slot = __shfl_sync(0xffffffffu, mm[i].y, src);
+                found = true;
+              } else {
+                left -= cnt;
+              }
             }
           }
         }
+        if (a.tau_slots) {                               // the encode's TopK bound starts empty
+          reinterpret_cast<uint4*>(a.tau_slots + (size_t)p * kTauSlots)[lane] = make_uint4(0u, 0u, 0u, 0u);
+          if (lane == 0) a.tau_min[p] = 0u;
+        }
+        if (kPack == 0)
+          pack_row_bf16(a.hidden, t, static_cast<__nv_bfloat16*>(a.panel), (size_t)p, a.d, lane);
+        else
+          pack_row_e4m3<kPack == 1>(a.hidden, t, static_cast<unsigned char*>(a.panel), a.act_scale, (size_t)p, a.d, a.lo_row0, lane);
+      }
+      if (lane == 0) {
+        RowRec rec;
+        const int g = (meta & 0xff) - 1;
+        rec.t = t;
+        rec.slot = t >= 0 ? slot : -1;
+        rec.n_edit = (meta >> 8) & 0xff;
+        rec.group_flags = t >= 0 ? (g | ((meta >> 16) & 1 ? kRecAddError : 0) | (s_gact[g] << kRecActShift)) : 0;
+        a.row_rec[p] = rec;
+        a.panel_row[p] = t;
+        if (a.row_flag) a.row_flag[p] = 0;
       }
     }
-  }
-  __syncthreads();
-  phase_stamp(a.clk, 3, first_cta && tid == 0);
-  // this CTA's panel rows, one per warp and round: the row's record for the kernels behind the encode, then the row itself
-  for (int r = warp; r < n_own; r += kFrontWarps) {
-    const int p = p0 + r;
-    if (p >= a.panel_cap) break;
-    const int t = s_tok[r];
-    if (p < s_n_panel_rows) {
-      if (a.tau_slots) {                                 // the encode's TopK bound starts empty
-        reinterpret_cast<uint4*>(a.tau_slots + (size_t)p * kTauSlots)[lane] = make_uint4(0u, 0u, 0u, 0u);
-        if (lane == 0) a.tau_min[p] = 0u;
-      }
-      if (kPack == 0)
-        pack_row_bf16(a.hidden, t, static_cast<__nv_bfloat16*>(a.panel), (size_t)p, a.d, lane);
-      else
-        pack_row_e4m3<kPack == 1>(a.hidden, t, static_cast<unsigned char*>(a.panel), a.act_scale, (size_t)p, a.d, a.lo_row0, lane);
-    }
-    if (lane == 0) {
-      RowRec rec;
-      rec.t = t;
-      rec.slot = t >= 0 ? s_slot[r] : -1;
-      const int meta = t >= 0 ? s_grp[r] : 0, g = (meta & 0xff) - 1;
-      rec.n_edit = (meta >> 8) & 0xff;
-      rec.group_flags = t >= 0 ? (g | ((meta >> 16) & 1 ? kRecAddError : 0) | (s_gact[g] << kRecActShift)) : 0;
-      a.row_rec[p] = rec;
-      a.panel_row[p] = t;
-      if (a.row_flag) a.row_flag[p] = 0;
-    }
+  } else if (tid == 0) {
+    atomicOr(a.status, MIX_STATUS_WAIT_TIMEOUT);
   }
   phase_stamp(a.clk, 4, first_cta && tid == 0);
+  // the last CTA to leave closes the call: the next launch reads the new epoch
+  __syncthreads();
+  if (tid == 0) {
+    __threadfence();
+    if (atomicAdd(a.sync + 1, 1) == (int)gridDim.x - 1) {
+      a.sync[1] = 0;
+      __threadfence();
+      st_release(a.sync, target);
+    }
+  }
 }
 
 }  // namespace
+
+int front_chunks(int T_max) { return (T_max + kFrontThreads - 1) / kFrontThreads; }
 
 cudaError_t launch_front(const Ctx* c, const __nv_bfloat16* hidden, int T, cudaStream_t s, unsigned long long cond, int use_cond) {
   FrontArgs a;
@@ -426,6 +427,9 @@ cudaError_t launch_front(const Ctx* c, const __nv_bfloat16* hidden, int T, cudaS
   a.n_groups = c->cfg.n_groups_max;
   a.chain_next = c->d_chain_next;
   a.edit_only = (c->cfg.flags & MIX_FLAG_SAE_EDIT_ONLY) ? 1 : 0;
+  a.row_meta = c->d_row_meta;
+  a.counts = c->d_front_counts;
+  a.sync = c->d_front_sync;
   a.panel_row = c->d_panel_row;
   a.row_rec = c->d_row_rec;
   a.panel_cap = c->panel_rows_cap;
@@ -435,8 +439,6 @@ cudaError_t launch_front(const Ctx* c, const __nv_bfloat16* hidden, int T, cudaS
   a.row_flag = c->d_row_flag;
   a.mtile_flag = c->d_mtile_flag;
   a.n_flagged = c->d_n_flagged;
-  a.row_group = c->d_row_group;
-  a.row_slot = c->d_row_slot;
   a.cond = static_cast<cudaGraphConditionalHandle>(cond);
   a.use_cond = use_cond;
   a.hidden = hidden;
@@ -447,14 +449,11 @@ cudaError_t launch_front(const Ctx* c, const __nv_bfloat16* hidden, int T, cudaS
   a.tau_min = c->d_tau_min;
   a.lo_row0 = c->panel_rows_cap;
   a.clk = c->d_phase_clk;
-  const int n_chunks = (c->cfg.T_max + kFrontThreads - 1) / kFrontThreads;
-  const size_t smem = (size_t)n_chunks * kFrontWarps * c->cfg.n_groups_max * sizeof(int);
-  // one wave of CTAs where the panel allows it (a CTA of 1024 threads has an SM to itself)
-  const int n_sms = c->n_sms > 0 ? c->n_sms : 148;
-  int rows = ((c->panel_rows_cap + n_sms - 1) / n_sms + 31) / 32 * 32;
-  rows = rows < 32 ? 32 : (rows > kFrontRowsMax ? kFrontRowsMax : rows);
-  a.rows_per_cta = rows;
-  const dim3 grid((c->panel_rows_cap + rows - 1) / rows);
+  a.pair_mode = ((c->cfg.flags & MIX_FLAG_ENCODE_SIMT) || !encode_pair_possible(c)) ? 0 : encode_pair_mode(-1);
+  const int chunks = front_chunks(T);
+  const size_t smem = (size_t)front_chunks(c->cfg.T_max) * (c->cfg.n_groups_max + 1) * sizeof(int);
+  const int pack_ctas = (c->panel_rows_cap + kFrontWarps - 1) / kFrontWarps;
+  const dim3 grid(chunks > pack_ctas ? chunks : pack_ctas);
   if (c->cfg.flags & MIX_FLAG_FP8_ACT)
     front_kernel<2><<<grid, kFrontThreads, smem, s>>>(a);
   else if (c->cfg.flags & MIX_FLAG_FP8_W_ENC)      // hi codes in rows [0, P), lo codes in rows [P, 2P) of the same buffer

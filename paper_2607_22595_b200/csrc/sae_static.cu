@@ -36,9 +36,10 @@ constexpr size_t kOffEditMode = kOffEditVal + align256(kMaxEdits * sizeof(float)
 constexpr size_t kOffRoute = kOffEditMode + align256(kMaxEdits);
 constexpr size_t kOffPanelRow = kOffRoute + align256(sizeof(RouteState));
 constexpr size_t kOffMtileGroup = kOffPanelRow + align256(kStaticRows * sizeof(int));
-constexpr size_t kOffRowGroup = kOffMtileGroup + 256;
-constexpr size_t kOffRowSlot = kOffRowGroup + align256(kStaticRows * sizeof(int));
-constexpr size_t kOffChainNext = kOffRowSlot + align256(kStaticRows * sizeof(int));
+constexpr size_t kOffRowMeta = kOffMtileGroup + 256;
+constexpr size_t kOffFrontCounts = kOffRowMeta + align256(kStaticRows * sizeof(int2));
+constexpr size_t kOffFrontSync = kOffFrontCounts + 256;      // one chunk: a count per weight set + one, then epoch words
+constexpr size_t kOffChainNext = kOffFrontSync + 256;
 constexpr size_t kOffRowRec = kOffChainNext + 256;
 constexpr size_t kOffPanel = kOffRowRec + align256(kStaticRows * sizeof(RowRec));
 constexpr size_t kOffZ = kOffPanel + align256((size_t)kStaticRows * kStaticD * sizeof(__nv_bfloat16));
@@ -166,8 +167,10 @@ extern "C" int mix_sae_apply_static(void* hidden, int n_rows, int d_model, const
   c.d_route = reinterpret_cast<RouteState*>(base + kOffRoute);
   c.d_panel_row = reinterpret_cast<int*>(base + kOffPanelRow);
   c.d_mtile_group = reinterpret_cast<int*>(base + kOffMtileGroup);
-  c.d_row_group = reinterpret_cast<int*>(base + kOffRowGroup);
-  c.d_row_slot = reinterpret_cast<int*>(base + kOffRowSlot);
+  c.d_row_meta = reinterpret_cast<int2*>(base + kOffRowMeta);
+  c.d_front_counts = reinterpret_cast<int*>(base + kOffFrontCounts);
+  c.d_front_sync = reinterpret_cast<int*>(base + kOffFrontSync);   // epoch words: zero when the library is loaded, then only ever
+                                                                   // advanced by the routing kernel itself, one step per call
   c.d_chain_next = reinterpret_cast<int*>(base + kOffChainNext);   // never read: the app entry carries no chain flag
   c.d_row_rec = reinterpret_cast<RowRec*>(base + kOffRowRec);
   c.d_panel = reinterpret_cast<__nv_bfloat16*>(base + kOffPanel);

@@ -106,13 +106,37 @@ struct ZRow {            // all pre-activations of the row; position = feature i
   __device__ __forceinline__ unsigned key(int i) const { return f2key(z[i]); }
   __device__ __forceinline__ unsigned id(int i) const { return (unsigned)i; }
 };
-struct CandRow {         // per-tile candidates of the fused encode epilogue
-  const float* v;
-  const int* j;
+struct CandRow {         // per-tile candidates of the fused encode epilogue, their keys staged in shared memory.
+  // The id of a candidate is its POSITION in the row's candidate array: positions run tile by tile, and inside a
+  // tile by decreasing value with the lower column first among equal values, so among equal keys position order
+  // is feature-id order -- the tie rule -- and the feature ids are fetched for the k winners only.
+  const unsigned* key_s;
   int n;
-  __device__ __forceinline__ unsigned key(int i) const { return f2key(v[i]); }
-  __device__ __forceinline__ unsigned id(int i) const { return (unsigned)j[i]; }
+  __device__ __forceinline__ unsigned key(int i) const { return key_s[i]; }
+  __device__ __forceinline__ unsigned id(int i) const { return (unsigned)i; }
 };
+
+// f(i, key, valid) for i = tid, tid + 256, ... < n_up (n_up: n rounded up to whole CTAs, so that whole warps take
+// part), the keys of four steps requested before the first is used: a source in global memory is then read
+// with four loads in flight per thread instead of one (a loop that mixes loads with shared-memory atomics is
+// not reordered by the compiler).
+template <class Src, class F>
+__device__ __forceinline__ void scan_keys(const Src& src, int n, int n_up, F&& f) {
+  constexpr int U = 4;
+  for (int i0 = threadIdx.x; i0 < n_up; i0 += U * kTailThreads) {
+    unsigned key[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int i = i0 + u * kTailThreads;
+      key[u] = i < n ? src.key(i) : 0u;
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int i = i0 + u * kTailThreads;
+      if (i < n_up) f(i, key[u], i < n);
+    }
+  }
+}
 
 struct SelShared {
   __align__(16) int hist[kBins];            // radix histogram; afterwards the output of the counting sort (kBins / 2 composites)
@@ -148,15 +172,17 @@ __device__ __forceinline__ void push_cand(SelShared& sh, bool take, unsigned lon
 //   other sources return 0 (the caller falls back).
 // Returns 1 in the ordinary case.  Every thread of the CTA must call this.
 template <bool ORDERED, class Src>
-__device__ int radix_collect(const Src& src, int k, SelShared& sh) {
+__device__ int radix_collect(const Src& src, int k, SelShared& sh, unsigned long long* clk = nullptr, bool stamp = false) {
   const int tid = threadIdx.x, n = src.n;
+  const int n_up = (n + kTailThreads - 1) / kTailThreads * kTailThreads;    // whole warps take part in every ballot
   // range of the keys
   unsigned kmin = 0xffffffffu, kmax = 0u;
-  for (int i = tid; i < n; i += kTailThreads) {
-    const unsigned key = src.key(i);
-    kmin = min(kmin, key);
-    kmax = max(kmax, key);
-  }
+  scan_keys(src, n, n_up, [&](int, unsigned key, bool valid) {
+    if (valid) {
+      kmin = min(kmin, key);
+      kmax = max(kmax, key);
+    }
+  });
   kmin = __reduce_min_sync(0xffffffffu, kmin);
   kmax = __reduce_max_sync(0xffffffffu, kmax);
   if ((tid & 31) == 0) {
@@ -169,6 +195,8 @@ __device__ int radix_collect(const Src& src, int k, SelShared& sh) {
     kmax = max(kmax, (unsigned)sh.hist[32 + w]);
   }
   __syncthreads();
+  phase_stamp(clk, 16, stamp);
+  int n_pass = 0;
   int hi_bit = (kmax ^ kmin) ? 32 - __clz(kmax ^ kmin) : 0;     // bits [0, hi_bit) vary; the rest is common
   unsigned prefix = hi_bit >= 32 ? 0u : (kmax >> hi_bit);       // digits fixed so far (= key >> hi_bit of the k-th)
   int need = k;                 // winners still to be found inside the prefix set
@@ -180,10 +208,9 @@ __device__ int radix_collect(const Src& src, int k, SelShared& sh) {
     const int width = min(11, hi_bit), shift = hi_bit - width, nb = 1 << width;
     for (int b = tid; b < kBins; b += kTailThreads) sh.hist[b] = 0;     // digits >= nb do not occur: their bins stay 0
     __syncthreads();
-    for (int i = tid; i < n; i += kTailThreads) {
-      const unsigned key = src.key(i);
-      if (hi_bit >= 32 || (key >> hi_bit) == prefix) atomicAdd(&sh.hist[(key >> shift) & (nb - 1)], 1);
-    }
+    scan_keys(src, n, n_up, [&](int, unsigned key, bool valid) {
+      if (valid && (hi_bit >= 32 || (key >> hi_bit) == prefix)) atomicAdd(&sh.hist[(key >> shift) & (nb - 1)], 1);
+    });
     __syncthreads();
     if (tid < 32) find_digit(sh.hist, kBins, need, sh.res);
     __syncthreads();
@@ -194,17 +221,17 @@ __device__ int radix_collect(const Src& src, int k, SelShared& sh) {
     hi_bit = shift;
     done = (k - need) + in_bin <= kCand;
     __syncthreads();
+    phase_stamp(clk, 17 + min(n_pass, 3), stamp);
+    ++n_pass;
     if (done && (k - need) + in_bin <= enough) break;
   }
   if (tid == 0) sh.n = 0;
   __syncthreads();
-  const int n_up = (n + kTailThreads - 1) / kTailThreads * kTailThreads;    // whole warps take part in every ballot
   if (done) {
-    for (int i = tid; i < n_up; i += kTailThreads) {
-      const unsigned key = i < n ? src.key(i) : 0u;
-      const bool take = i < n && (key >> hi_bit) >= prefix;
+    scan_keys(src, n, n_up, [&](int i, unsigned key, bool valid) {
+      const bool take = valid && (key >> hi_bit) >= prefix;
       push_cand(sh, take, take ? (((unsigned long long)key << 32) | (0xffffffffu - src.id(i))) : 0ull);
-    }
+    });
     __syncthreads();
     return 1;
   }
@@ -212,11 +239,10 @@ __device__ int radix_collect(const Src& src, int k, SelShared& sh) {
     return 0;
   } else {
   // every larger key, then the `need` lowest ids among the exact ties, in index order
-  for (int i = tid; i < n_up; i += kTailThreads) {
-    const unsigned key = i < n ? src.key(i) : 0u;
-    const bool take = i < n && key > prefix;
+  scan_keys(src, n, n_up, [&](int i, unsigned key, bool valid) {
+    const bool take = valid && key > prefix;
     push_cand(sh, take, take ? (((unsigned long long)key << 32) | (0xffffffffu - src.id(i))) : 0ull);
-  }
+  });
   __syncthreads();
   int taken = 0;               // uniform across the block
   for (int i0 = 0; i0 < n && taken < need; i0 += kTailThreads) {
@@ -270,15 +296,14 @@ __device__ __forceinline__ int comp_id(unsigned long long c) { return (int)(0xff
 __device__ __forceinline__ float comp_val(unsigned long long c) { return key2f((unsigned)(c >> 32)); }
 
 // Read-out of a row's TopK: ids in order of decreasing pre-activation, the pre-activations, the active count.
-__device__ void emit_topk(const unsigned long long* a, int k, int k_max, int t, int* __restrict__ out_idx,
+__device__ void emit_topk(const int* ids, const float* vals, int k, int k_max, int t, int* __restrict__ out_idx,
                           float* __restrict__ out_val, int* __restrict__ out_n_active, int* s_count) {
   const int tid = threadIdx.x;
   if (out_idx == nullptr && out_val == nullptr && out_n_active == nullptr) return;
   int pos_cnt = 0;
   for (int i = tid; i < k; i += kTailThreads) {
-    const unsigned long long c = a[i];
-    const float v = comp_val(c);
-    if (out_idx) out_idx[(size_t)t * k_max + i] = comp_id(c);
+    const float v = vals[i];
+    if (out_idx) out_idx[(size_t)t * k_max + i] = ids[i];
     if (out_val) out_val[(size_t)t * k_max + i] = v;
     pos_cnt += v > 0.f;
   }
@@ -380,14 +405,21 @@ struct TailArgs {
 
 struct RowShared {
   SelShared sel;
+  unsigned keys[kCandMax];  // a TopK row's candidate keys (the radix passes run on shared memory)
   float coef[kDecList];
   int feat[kDecList];
   int eidx[kMaxEdits];
-  float ef[kMaxEdits];
+  float ef[kMaxEdits];      // f_j of each edited feature before the edit
+  float enew[kMaxEdits];    // f'_j
   int n_list;
 };
 
-// Row role.
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
+// Row role.  Per row, the dependent round trips are: the row's record; then -- requested together -- the edit
+// list, the candidate keys (into shared memory: the selection passes never go back to global memory) and the
+// tiles' 9th values; then the winners' feature ids; then the gather, whose decoder rows and hidden row were
+// prefetched into L2 as soon as the edit list was known.
 __device__ void tail_rows(const TailArgs& a, RowShared& sh) {
   const int tid = threadIdx.x;
   const int n_rows = a.rs->n_panel_rows;
@@ -404,30 +436,72 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh) {
     const bool add_error = (rec.group_flags & kRecAddError) != 0;
     const bool topk = act == MIX_SAE_TOPK;
     if (a.mode == kTailFallback && !(topk && a.row_flag[p])) continue;
+    if (!topk && add_error && a.out_n_active == nullptr) continue;     // the delta role's row, and nobody wants its active count
+    const int slot = rec.slot, n_edit = rec.n_edit;
+    const bool from_cand = topk && a.mode == kTailCand;
+    // ---- everything the record alone gives the address of, requested together
+    if (tid < n_edit) {
+      sh.eidx[tid] = a.edit_idx[slot * a.r_max + tid];
+      sh.enew[tid] = a.edit_mode[slot * a.r_max + tid] == MIX_EDIT_CLAMP ? a.edit_val[slot * a.r_max + tid] : 0.f;
+      sh.ef[tid] = 0.f;
+    }
     const int S = (int)gp->d_sae, k = gp->k;
+    const __nv_bfloat16* W_dec = gp->W_dec;
     const float* z = a.Z + (size_t)p * a.ldz;
-    const unsigned long long* sorted = nullptr;
+    uint4* hrow = reinterpret_cast<uint4*>(a.hidden + (size_t)t * d);
+    const int n_tiles = S / kTileN, n_cand = n_tiles * kCandPerTile;
+    unsigned ninth_max = 0u;                           // largest key among this thread's share of the tiles' 9th values
+    if (from_cand && n_cand >= k) {
+      const float* cv = a.cand_val + (size_t)p * a.cand_tiles * kCandPerTile;
+      for (int i0 = tid; i0 < n_cand; i0 += 8 * kTailThreads) {
+        float v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int i = i0 + u * kTailThreads;
+          v[u] = i < n_cand ? cv[i] : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int i = i0 + u * kTailThreads;
+          if (i < n_cand) sh.keys[i] = f2key(v[u]);
+        }
+      }
+      const float* ninth = a.cand_ninth + (size_t)p * a.cand_tiles;
+      for (int i = tid; i < n_tiles; i += kTailThreads) ninth_max = max(ninth_max, f2key(ninth[i]));
+    }
+    __syncthreads();
+    phase_stamp(a.clk, 21, stamp);
+    // the decoder rows of the edited features and (error term on) the row itself: on their way into L2 while the
+    // selection runs
+    if (topk || !add_error) {
+      const int lines = d >> 6;                        // 128-byte lines per row
+      for (int x = tid; x < n_edit * lines; x += kTailThreads) {
+        const int e = x / lines;
+        prefetch_l2(W_dec + (size_t)sh.eidx[e] * d + (size_t)(x - e * lines) * 64);
+      }
+      if (add_error)
+        for (int x = tid; x < lines; x += kTailThreads) prefetch_l2(reinterpret_cast<const __nv_bfloat16*>(hrow) + (size_t)x * 64);
+    }
+    int* win_id = sh.feat + n_edit;                    // the winners follow the edit entries in the gather lists
+    float* win_val = sh.coef + n_edit;
     if (topk) {
-      if (a.mode == kTailCand) {
+      const unsigned long long* sorted;
+      if (from_cand) {
         // Every (row, feature tile) contributed its 8 largest pre-activations and its 9th.  The k largest
         // candidates are the row's TopK unless some tile's 9th value reaches the k-th candidate, i.e. that tile
         // may hide a winner (or an exact tie whose order matters): such rows are flagged, their row tiles are
         // re-encoded to Z and the fallback launch selects exactly.
-        const int n_tiles = S / kTileN, n = n_tiles * kCandPerTile;
-        bool flag = n < k;                             // uniform
+        bool flag = n_cand < k;                        // uniform
         if (!flag) {
-          CandRow src{a.cand_val + (size_t)p * a.cand_tiles * kCandPerTile, a.cand_idx + (size_t)p * a.cand_tiles * kCandPerTile, n};
-          flag = radix_collect<false>(src, k, sh.sel) == 0;
+          CandRow src{sh.keys, n_cand};
+          flag = radix_collect<false>(src, k, sh.sel, a.clk, stamp) == 0;
         }
         phase_stamp(a.clk, 10, stamp);
         if (!flag) {
           sorted = sort_desc(sh.sel);
           phase_stamp(a.clk, 11, stamp);
           const unsigned kth = (unsigned)(sorted[k - 1] >> 32);
-          const float* ninth = a.cand_ninth + (size_t)p * a.cand_tiles;
-          int over = 0;
-          for (int i = tid; i < n_tiles; i += kTailThreads) over |= f2key(ninth[i]) >= kth;
-          flag = __syncthreads_or(over) != 0;
+          flag = __syncthreads_or(ninth_max >= kth) != 0;
         }
         if (flag) {
           if (tid == 0) {
@@ -438,14 +512,24 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh) {
           __syncthreads();
           continue;
         }
+        const int* ci = a.cand_idx + (size_t)p * a.cand_tiles * kCandPerTile;
+        for (int i = tid; i < k; i += kTailThreads) {
+          win_id[i] = ci[comp_id(sorted[i])];          // position -> feature id, for the winners only
+          win_val[i] = comp_val(sorted[i]);
+        }
       } else {
         ZRow src{z, S};
         const int how = radix_collect<true>(src, k, sh.sel);
         if (how == 2 && tid == 0) atomicOr(a.status, MIX_STATUS_TOPK_GENERAL);
         sorted = sort_desc(sh.sel);
+        for (int i = tid; i < k; i += kTailThreads) {
+          win_id[i] = comp_id(sorted[i]);
+          win_val[i] = comp_val(sorted[i]);
+        }
       }
+      __syncthreads();
       phase_stamp(a.clk, 12, stamp);
-      emit_topk(sorted, k, a.k_max, t, a.out_idx, a.out_val, a.out_n_active, &sh.sel.count);
+      emit_topk(win_id, win_val, k, a.k_max, t, a.out_idx, a.out_val, a.out_n_active, &sh.sel.count);
     } else {
       if (a.out_n_active != nullptr) {
         int cnt = 0;
@@ -467,31 +551,22 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh) {
       }
     }
     // ---- edits and decode of this row
-    const int slot = rec.slot, n_edit = rec.n_edit;
-    uint4* hrow = reinterpret_cast<uint4*>(a.hidden + (size_t)t * d);
-    const __nv_bfloat16* W_dec = gp->W_dec;
-    if (tid < n_edit) {
-      sh.eidx[tid] = a.edit_idx[slot * a.r_max + tid];
-      sh.ef[tid] = 0.f;
-    }
-    __syncthreads();
+    bool alive = true;                                 // a later entry for the same feature wins
+    if (tid < n_edit)
+      for (int e2 = tid + 1; e2 < n_edit; ++e2) alive = alive && (sh.eidx[e2] != sh.eidx[tid]);
     if (add_error) {
       // (TopK rows only.)  f_j of an edited feature comes from the row's TopK list, 0 if it was not selected
       for (int i = tid; i < k; i += kTailThreads) {
-        const int id = comp_id(sorted[i]);
+        const int id = win_id[i];
         for (int e = 0; e < n_edit; ++e)
-          if (sh.eidx[e] == id) sh.ef[e] = fmaxf(comp_val(sorted[i]), 0.f);
+          if (sh.eidx[e] == id) sh.ef[e] = fmaxf(win_val[i], 0.f);
       }
       __syncthreads();
       float delta = 0.f;
       if (tid < n_edit) {
-        const int j = sh.eidx[tid];
-        bool alive = true;                             // a later entry for the same feature wins
-        for (int e2 = tid + 1; e2 < n_edit; ++e2) alive = alive && (sh.eidx[e2] != j);
-        const float fnew = a.edit_mode[slot * a.r_max + tid] == MIX_EDIT_CLAMP ? a.edit_val[slot * a.r_max + tid] : 0.f;
-        delta = alive ? fnew - sh.ef[tid] : 0.f;
+        delta = alive ? sh.enew[tid] - sh.ef[tid] : 0.f;
         sh.coef[tid] = delta;
-        sh.feat[tid] = j;
+        sh.feat[tid] = sh.eidx[tid];
       }
       phase_stamp(a.clk, 13, stamp);
       if (__syncthreads_or(delta != 0.f)) {            // no effective edit: the row stays as it is, bit for bit
@@ -508,23 +583,19 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh) {
     }
     // the app replaces the residual: h' = b_dec + sum_j f'_j W_dec[j]
     if (tid < n_edit) {       // edited features contribute f' (live entries only)
-      const int j = sh.eidx[tid];
-      bool alive = true;
-      for (int e2 = tid + 1; e2 < n_edit; ++e2) alive = alive && (sh.eidx[e2] != j);
-      const float fnew = a.edit_mode[slot * a.r_max + tid] == MIX_EDIT_CLAMP ? a.edit_val[slot * a.r_max + tid] : 0.f;
-      sh.coef[tid] = alive ? fnew : 0.f;
-      sh.feat[tid] = j;
+      sh.coef[tid] = alive ? sh.enew[tid] : 0.f;
+      sh.feat[tid] = sh.eidx[tid];
     }
     const float* b_dec = gp->b_dec;
     if (topk) {
       for (int i = tid; i < k; i += kTailThreads) {
-        const int j = comp_id(sorted[i]);
+        const int j = win_id[i];
         bool edited = false;
         for (int e = 0; e < n_edit; ++e) edited = edited || (sh.eidx[e] == j);
         // an id outside the SAE can only come from a call whose encode timed out: never address with it
         const bool in_range = (unsigned)j < (unsigned)S;
-        sh.coef[n_edit + i] = (edited || !in_range) ? 0.f : fmaxf(comp_val(sorted[i]), 0.f);
-        sh.feat[n_edit + i] = in_range ? j : 0;
+        win_val[i] = (edited || !in_range) ? 0.f : fmaxf(win_val[i], 0.f);
+        win_id[i] = in_range ? j : 0;
       }
       __syncthreads();
       for (int v = tid; v < nvec; v += kTailThreads) {
@@ -594,6 +665,8 @@ __device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int item, int n_r
   const int rg = item / a.n_col_slices, cs = item - rg * a.n_col_slices;
   const int p0 = rg * kDlRows;
   __syncthreads();                                       // the shared lists of the previous item are free
+  const bool stamp = item == 0 && tid == 0;
+  phase_stamp(a.clk, 22, stamp);
   if (tid < kDlRows) {
     const int p = p0 + tid;                              // in bounds: the panel capacity is a multiple of 128
     const RowRec rec = a.row_rec[p];
@@ -610,6 +683,7 @@ __device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int item, int n_r
   bool any = false;
 #pragma unroll
   for (int r = 0; r < kDlRows; ++r) any = any || sh.slot[r] >= 0;
+  phase_stamp(a.clk, 23, stamp);
   if (!any) return;
   const int d = a.d;
   const int v = cs * kTailThreads + tid;                 // this thread's 16-byte column vector
@@ -657,6 +731,7 @@ __device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int item, int n_r
     n_entries += n_edit;
     __syncthreads();
   }
+  phase_stamp(a.clk, 24, stamp);
   // pad to a whole batch: repeats of the last decoder row with zero coefficients
   if (tid < kDlBatch) {
     sh.wrow[n_entries + tid] = sh.wrow[n_entries - 1];
@@ -690,6 +765,7 @@ __device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int item, int n_r
       axpy8(acc[3], c4.w, q[u]);
     }
   }
+  phase_stamp(a.clk, 25, stamp);
 #pragma unroll
   for (int r = 0; r < kDlRows; ++r) {
     if (sh.slot[r] < 0 || !sh.changed[r]) continue;     // no effective edit: the row stays bit-exact

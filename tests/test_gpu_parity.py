@@ -413,7 +413,7 @@ def test_api_error_codes():
     with pytest.raises(mixlib.MixError) as e:
         m.set_slot_map(np.zeros(9, dtype=np.int32))                       # T_live > T_max
     assert e.value.code == -2
-    assert m.launches_per_apply() == 6                                # hook kernel + front, encode, tail, flagged encode, flagged tail
+    assert m.launches_per_apply() == 7                                # hook kernel + front, encode x 2, tail, flagged encode, flagged tail
     m.destroy()
 
 
