@@ -255,7 +255,7 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
     ok = ok && dev_alloc(&c->d_mtile_group, P / kTileM) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_row_meta, T) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_front_counts, (size_t)front_chunks(T) * (G + 1)) == cudaSuccess;
-    ok = ok && dev_alloc(&c->d_front_sync, (size_t)front_chunks(T) + 2) == cudaSuccess;
+    ok = ok && dev_alloc(&c->d_front_sync, 2) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_route, 1) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_z, P * (size_t)cfg->d_sae_max) == cudaSuccess;
     ok = ok && dev_alloc(&c->d_tmap_w, G) == cudaSuccess;
@@ -292,7 +292,7 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
   if (e == cudaSuccess && G > 0) {
     e = cudaMemset(c->d_panel, 0, (size_t)c->panel_rows_cap * cfg->d_model * sizeof(__nv_bfloat16));
     if (e == cudaSuccess) e = cudaMemset(c->d_route, 0, sizeof(RouteState));
-    if (e == cudaSuccess) e = cudaMemset(c->d_front_sync, 0, ((size_t)front_chunks(T) + 2) * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(c->d_front_sync, 0, 2 * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(c->d_panel_row, 0xff, c->panel_rows_cap * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(c->d_mtile_group, 0xff, c->panel_rows_cap / kTileM * sizeof(int));
     if (e == cudaSuccess && !(cfg->flags & MIX_FLAG_ENCODE_SIMT)) {

@@ -139,7 +139,7 @@ struct Ctx {
   int* d_mtile_group;       // [P / kTileM] group of each m-tile or -1
   int2* d_row_meta;         // [T_max] front kernel: per token row, what its chunk's CTA found out (weight set, edit count, flags; slot)
   int* d_front_counts;      // [chunks of 256 token rows][n_groups_max + 1] front kernel: SAE rows per weight set and chunk
-  int* d_front_sync;        // [2 + chunks] front kernel: epoch, CTAs done, per-chunk publication epoch
+  int* d_front_sync;        // [2] front kernel: chunks published / CTAs done in the running call (zero between calls)
   RowRec* d_row_rec;        // [P] per packed row: token row, slot, edit count, weight set, error-term flag
   RouteState* d_route;
   float* d_z;               // [P, d_sae_max]

@@ -116,7 +116,7 @@ struct FrontArgs {
   // exchange between the CTAs of one launch
   int2* row_meta;          // [T_max] per token row: (weight set + 1) | edit count << 8 | error-term flag << 16 (0: not an SAE row), slot
   int* counts;             // [chunks][n_groups + 1] SAE rows per weight set in each chunk of 256 token rows; last column: delta-role rows
-  int* sync;               // [0] epoch of the last finished call, [1] CTAs of this call that are done, [2 + c] epoch in which chunk c was published
+  int* sync;               // [0] chunks published so far in this call, [1] CTAs of this call that are done (both back to 0 when the call ends)
   // routing results (written)
   int* panel_row;
   RowRec* row_rec;
@@ -146,21 +146,20 @@ __device__ __forceinline__ int ld_acquire(const int* p) {
   asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
-__device__ __forceinline__ void st_release(int* p, int v) { asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory"); }
 
 constexpr long long kFrontWaitCycles = 2000000000ll;   // ~1 s: cap of the wait for the other CTAs' chunks
 
 // One launch, three steps, no CTA doing another's work:
 //   1. CTA c < chunks classifies token rows [256 c, 256 c + 256) -- slot -> app entry -> SAE row of which weight set --
-//      and PUBLISHES the chunk: per-row records, per-set counts, then a flag carrying this call's epoch.
-//   2. Every CTA waits (bounded) until all chunks carry the epoch, reads the small count table and scans it: totals
+//      and PUBLISHES the chunk: per-row records, per-set counts, then one more on the call's counter of published chunks.
+//   2. Every CTA waits (one thread polls, bounded) until the counter says all chunks are there, reads the small count table and scans it: totals
 //      per weight set, the sets' first panel rows, and for every chunk the rank of its first row within each set.
 //      The publishing CTAs never wait before they publish, and CTAs are dispatched in index order, so whoever waits,
 //      waits for work that is already running.
 //   3. CTA b packs panel rows [8 b, 8 b + 8), one per warp: the row's set and rank follow from its position, the
 //      chunk that holds that rank from the scan, the token from that chunk's published records.
 // CTA 0 alone writes what exists once (the routing result the encode reads, the tile -> weight-set map, the
-// conditional handle).  The epoch advances when the last CTA of the launch leaves.
+// conditional handle).  The last CTA of the launch to leave puts the two counters back to zero for the next call.
 // kPack: 0 the bf16 row, 1 E4M3 hi + lo (exact split), 2 E4M3 quantised.
 template <int kPack>
 __global__ void __launch_bounds__(kFrontThreads)
@@ -177,7 +176,6 @@ front_kernel(const FrontArgs a) {
   const int n_groups = a.n_groups, n_slots = a.n_slots, ncol = n_groups + 1;
   const int n_chunks = (a.T + kFrontThreads - 1) / kFrontThreads;     // the same in every CTA: who publishes is fixed by the launch
   phase_stamp(a.clk, 0, first_cta && tid == 0);
-  const int target = ld_acquire(a.sync) + 1;          // this call's epoch
   if (tid < n_groups) {                                // requested now, needed after the first barrier
     const bool valid = __ldg(&a.groups[tid].valid) != 0;
     s_gact[tid] = __ldg(&a.groups[tid].act);
@@ -251,19 +249,20 @@ front_kernel(const FrontArgs a) {
     }
     __threadfence();
     __syncthreads();
-    if (tid == 0) st_release(a.sync + 2 + cta, target);
+    if (tid == 0) atomicAdd(a.sync, 1);                // (fence above + this: the chunk is published)
   } else {
     __syncthreads();                                   // (the weight-set table)
   }
   phase_stamp(a.clk, 1, first_cta && tid == 0);
   // ---- step 2: wait for every chunk, scan the counts
   bool ok = true;
-  for (int c = tid; c < n_chunks; c += kFrontThreads) {
-    if (ld_acquire(a.sync + 2 + c) == target) continue;
+  if (tid == 0 && ld_acquire(a.sync) < n_chunks) {     // one polling thread per CTA, backing off: a thousand CTAs ask about one word
     const long long t0 = clock64();
-    while (ld_acquire(a.sync + 2 + c) != target) {
+    unsigned ns = 32;
+    while (ld_acquire(a.sync) < n_chunks) {
       if (clock64() - t0 > kFrontWaitCycles) { ok = false; break; }
-      __nanosleep(64);
+      __nanosleep(ns);
+      if (ns < 256) ns *= 2;
     }
   }
   ok = __syncthreads_and(ok) != 0;
@@ -399,14 +398,13 @@ front_kernel(const FrontArgs a) {
     atomicOr(a.status, MIX_STATUS_WAIT_TIMEOUT);
   }
   phase_stamp(a.clk, 4, first_cta && tid == 0);
-  // the last CTA to leave closes the call: the next launch reads the new epoch
+  // the last CTA to leave closes the call: both counters are zero again when the next launch starts
   __syncthreads();
   if (tid == 0) {
     __threadfence();
     if (atomicAdd(a.sync + 1, 1) == (int)gridDim.x - 1) {
+      a.sync[0] = 0;
       a.sync[1] = 0;
-      __threadfence();
-      st_release(a.sync, target);
     }
   }
 }

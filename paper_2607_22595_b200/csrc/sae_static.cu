@@ -169,8 +169,8 @@ extern "C" int mix_sae_apply_static(void* hidden, int n_rows, int d_model, const
   c.d_mtile_group = reinterpret_cast<int*>(base + kOffMtileGroup);
   c.d_row_meta = reinterpret_cast<int2*>(base + kOffRowMeta);
   c.d_front_counts = reinterpret_cast<int*>(base + kOffFrontCounts);
-  c.d_front_sync = reinterpret_cast<int*>(base + kOffFrontSync);   // epoch words: zero when the library is loaded, then only ever
-                                                                   // advanced by the routing kernel itself, one step per call
+  c.d_front_sync = reinterpret_cast<int*>(base + kOffFrontSync);   // two counters: zero when the library is loaded, and put back
+                                                                   // to zero by the routing kernel itself at the end of every call
   c.d_chain_next = reinterpret_cast<int*>(base + kOffChainNext);   // never read: the app entry carries no chain flag
   c.d_row_rec = reinterpret_cast<RowRec*>(base + kOffRowRec);
   c.d_panel = reinterpret_cast<__nv_bfloat16*>(base + kOffPanel);

@@ -401,6 +401,7 @@ struct TailArgs {
   int mode;                 // kTailCand: TopK from the encode's candidates; kTailZ: TopK from Z; kTailFallback: flagged rows only, from Z
   int n_col_slices;         // delta role: ceil(d / 2048)
   unsigned long long* clk;  // profiling aid or null
+  int n_groups;
 };
 
 struct RowShared {
@@ -412,6 +413,8 @@ struct RowShared {
   float ef[kMaxEdits];      // f_j of each edited feature before the edit
   float enew[kMaxEdits];    // f'_j
   int n_list;
+  int cum[kMaxGroups + 1];  // SAE rows in the weight sets before each one: work index -> packed row, padding rows skipped
+  int row0[kMaxGroups];     // first packed row of each weight set
 };
 
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
@@ -420,12 +423,26 @@ __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefe
 // list, the candidate keys (into shared memory: the selection passes never go back to global memory) and the
 // tiles' 9th values; then the winners' feature ids; then the gather, whose decoder rows and hidden row were
 // prefetched into L2 as soon as the edit list was known.
-__device__ void tail_rows(const TailArgs& a, RowShared& sh) {
+__device__ void tail_rows(const TailArgs& a, RowShared& sh, int n_groups) {
   const int tid = threadIdx.x;
-  const int n_rows = a.rs->n_panel_rows;
   const int d = a.d, nvec = d >> 3;
-  for (int p = blockIdx.x; p < n_rows; p += gridDim.x) {
-    const bool stamp = p == 0 && tid == 0 && a.mode != kTailFallback;
+  // the call's SAE rows, numbered through the weight sets without the padding rows of their last tiles
+  if (tid == 0) {
+    int cum = 0;
+    for (int g = 0; g < n_groups; ++g) {
+      sh.cum[g] = cum;
+      sh.row0[g] = a.rs->group_mtile0[g] * kTileM;
+      cum += a.rs->group_count[g];
+    }
+    sh.cum[n_groups] = cum;
+  }
+  __syncthreads();
+  const int n_work = sh.cum[n_groups];
+  for (int w = blockIdx.x; w < n_work; w += gridDim.x) {
+    int g_w = 0;
+    while (g_w + 1 < n_groups && w >= sh.cum[g_w + 1]) ++g_w;
+    const int p = sh.row0[g_w] + (w - sh.cum[g_w]);
+    const bool stamp = w == 0 && tid == 0 && a.mode != kTailFallback;
     phase_stamp(a.clk, 9, stamp);
     const RowRec rec = a.row_rec[p];
     const int t = rec.t;
@@ -781,17 +798,21 @@ __device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int item, int n_r
 // packed rows that need the row role, then the row groups x column slices of the delta role.  Both lists are as
 // long as THIS call's routing made them, not as long as the context's capacity, and a role with no rows this
 // call (no TopK / replacing row; no ReLU / JumpReLU row with edits) is skipped without looking at a single row.
-__global__ void __launch_bounds__(kTailThreads, 3)
+__global__ void __launch_bounds__(kTailThreads, 4)
 tail_kernel(const TailArgs a) {
   phase_stamp(a.clk, 7, blockIdx.x == 0 && threadIdx.x == 0 && a.mode != kTailFallback);
   pdl_wait();
   pdl_launch_dependents();
   phase_stamp(a.clk, 8, blockIdx.x == 0 && threadIdx.x == 0 && a.mode != kTailFallback);
-  __shared__ RowShared s_row;
-  __shared__ DeltaShared s_delta;
+  __shared__ union TailShared {     // a CTA finishes its rows before it turns to the delta role: the two share the space
+    RowShared row;
+    DeltaShared delta;
+  } s_u;
+  RowShared& s_row = s_u.row;
+  DeltaShared& s_delta = s_u.delta;
   if (a.mode == kTailFallback && *a.n_flagged == 0) return;   // nothing was flagged: the usual case
   const int n_rows = a.rs->n_panel_rows, n_delta = a.rs->n_delta_rows, n_sae = a.rs->n_sae_rows;
-  if (a.mode == kTailFallback || n_sae > n_delta || (a.out_n_active != nullptr && n_sae > 0)) tail_rows(a, s_row);
+  if (a.mode == kTailFallback || n_sae > n_delta || (a.out_n_active != nullptr && n_sae > 0)) tail_rows(a, s_row, a.n_groups);
   if (a.mode != kTailFallback && n_delta > 0) {
     const int n_items = (n_rows / kDlRows) * a.n_col_slices;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x) tail_delta(a, s_delta, item, n_rows);
@@ -830,11 +851,12 @@ cudaError_t launch_tail(const Ctx* c, __nv_bfloat16* hidden, int mode, cudaStrea
   a.status = c->d_status;
   a.mode = mode;
   a.clk = c->d_phase_clk;
+  a.n_groups = c->cfg.n_groups_max;
   const int n_sms = c->n_sms > 0 ? c->n_sms : 148;
   a.n_col_slices = (c->cfg.d_model / 8 + kTailThreads - 1) / kTailThreads;
   const int work_cap = c->panel_rows_cap > (c->panel_rows_cap / kDlRows) * a.n_col_slices ? c->panel_rows_cap
                                                                                           : (c->panel_rows_cap / kDlRows) * a.n_col_slices;
-  const int grid = work_cap < n_sms * 6 ? work_cap : n_sms * 6;
+  const int grid = work_cap < n_sms * 4 ? work_cap : n_sms * 4;      // four CTAs per SM: all of them resident at once
   return launch_pdl(kPdlTail, tail_kernel, dim3(grid), dim3(kTailThreads), 0, s, a);
 }
 

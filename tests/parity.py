@@ -122,14 +122,16 @@ def tight_bound(wh, t, ref, K_override=None):
     return bf16_ulp(at) + acc
 
 
-def check_parity(wh, out, rows=None, expect_status=0, check_features=True, scale_with_output=False):
+def check_parity(wh, out, rows=None, expect_status=0, check_features=True, scale_with_output=False, ref=None):
     """wh: host workload (numpy); out: run_gpu result.  Asserts parity on `rows` (default all).
+    ref: an oracle result for (at least) `rows`, with z kept, computed by the caller; default: apply_hook here.
     scale_with_output: take the hidden-state bound as 1e-2 * max(|h_in|, |y_ref|) -- for inputs where
     an app's output dwarfs the hidden state (a huge steering vector on a tiny h), so that the bf16
     rounding of the output alone would exceed 1e-2 * max|h_in|."""
     T = wh.T_max
     rows = list(range(T)) if rows is None else sorted(set(int(r) for r in rows))
-    ref = O.apply_hook(wh, rows, keep_z=True)
+    if ref is None:
+        ref = O.apply_hook(wh, rows, keep_z=True)
     hmax = float(np.abs(O.bf16_to_f64(wh.hidden)).max())
     hid = out["hidden"]
     scores_bits = out["scores"].view(np.uint32)
