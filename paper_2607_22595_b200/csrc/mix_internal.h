@@ -68,13 +68,15 @@ struct __align__(16) GroupEntry {
   const void* pad2_;
 };
 
-// What the front kernel leaves about one packed panel row for the kernels behind the encode: one 16-byte load
-// instead of the chain panel row -> slot map -> app entry.
+// What the front kernel leaves about one packed panel row for the kernels behind the encode: two 16-byte loads
+// instead of the chain panel row -> slot map -> app entry -> weight-set entry.
 struct __align__(16) RowRec {
   int t;                            // token row, or -1: padding row of a tile
   int slot;                         // slot of the SAE app that acts on the row (the row's own, or the last of its chain)
   int n_edit;                       // length of that app's edit list
   int group_flags;                  // low byte: weight set; kRecAddError: the app keeps the error term; bits 16..17: the set's activation
+  const __nv_bfloat16* W_dec;       // the set's decoder
+  const float* theta;               // the set's JumpReLU thresholds, or null
 };
 constexpr int kRecGroupMask = 0xff;
 constexpr int kRecAddError = 0x100;

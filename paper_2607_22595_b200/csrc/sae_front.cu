@@ -167,6 +167,8 @@ front_kernel(const FrontArgs a) {
   extern __shared__ int s_tab[];                      // [chunks][n_groups + 1]: counts, then exclusive prefixes over the chunks
   __shared__ int s_total[kMaxGroups + 1], s_base[kMaxGroups + 1];
   __shared__ int s_gact[kMaxGroups], s_gtiles[kMaxGroups];   // per weight set: activation, feature tiles (0: not registered)
+  __shared__ const __nv_bfloat16* s_gwdec[kMaxGroups];
+  __shared__ const float* s_gtheta[kMaxGroups];
   __shared__ int s_wcnt[kFrontWarps][kMaxGroups + 1];
   __shared__ int s_n_panel_rows;
   pdl_launch_dependents();
@@ -180,6 +182,8 @@ front_kernel(const FrontArgs a) {
     const bool valid = __ldg(&a.groups[tid].valid) != 0;
     s_gact[tid] = __ldg(&a.groups[tid].act);
     s_gtiles[tid] = valid ? (int)(__ldg(&a.groups[tid].d_sae) / kTileN) : 0;
+    s_gwdec[tid] = a.groups[tid].W_dec;
+    s_gtheta[tid] = a.groups[tid].theta;
   }
   // ---- step 1: classify and publish one chunk
   if (cta < n_chunks) {
@@ -288,7 +292,8 @@ front_kernel(const FrontArgs a) {
     __syncthreads();
     phase_stamp(a.clk, 2, first_cta && tid == 0);
     if (tid == 0) {
-      int mt = 0, tiles = 0, rows = 0, topk_rows = 0, pair_tiles = 0;
+      int mt = 0, tiles = 0, rows = 0, topk_rows = 0;
+      long long cost_single = 0, cost_pair = 0;
       for (int q = 0; q < n_groups; ++q) {
         s_base[q] = mt * kTileM;
         const int m_tiles = (s_total[q] + kTileM - 1) / kTileM;
@@ -302,7 +307,13 @@ front_kernel(const FrontArgs a) {
         rows += s_total[q];
         if (s_total[q] > 0 && s_gact[q] == MIX_SAE_TOPK) topk_rows += s_total[q];
         tiles += s_total[q] > 0 ? m_tiles * s_gtiles[q] : 0;
-        pair_tiles += s_total[q] > 0 ? ((m_tiles + 1) / 2) * s_gtiles[q] : 0;
+        if (s_total[q] > 0) {
+          // per feature tile, in tenths of a microsecond of SM time per k-block (measured): a single CTA needs 0.4 per
+          // 128-row tile, a pair 0.3 on both of its SMs per 256-row tile, and streaming the W_enc tile from HBM at
+          // the rate each form sustains is worth 0.8 resp. 0.9 -- the floor where a weight set has one or two row tiles
+          cost_single += (long long)max(4 * m_tiles, 8) * s_gtiles[q];
+          cost_pair += (long long)max(6 * ((m_tiles + 1) / 2), 9) * s_gtiles[q];
+        }
       }
       s_base[n_groups] = mt * kTileM;
       s_n_panel_rows = mt * kTileM;
@@ -319,10 +330,10 @@ front_kernel(const FrontArgs a) {
         a.rs->total_tiles = tiles;
         a.rs->n_topk_rows = topk_rows;
         a.rs->n_delta_rows = s_total[n_groups];
-        // A pair-tile keeps two SMs busy for about 3/4 of the time one SM needs for a 128-row tile (a third less
-        // shared-memory fill per SM), so pairs win when the weight sets average well over one row tile each, and lose
-        // where most sets have a single row tile (half of every pair would repeat the other half's work).
-        a.rs->use_pair = a.pair_mode == 2 ? (3 * pair_tiles <= 2 * tiles) : a.pair_mode;
+        // Pairs win where the tensor pipe (and the shared-memory fill behind it) is the limit -- weight sets with four or
+        // more row tiles -- and lose where the stream of W_enc is (fewer W_enc bytes in flight per SM) or where half of
+        // every pair would repeat the other half's work (a single row tile).
+        a.rs->use_pair = a.pair_mode == 2 ? (cost_pair < cost_single) : a.pair_mode;
         if (a.n_flagged) *a.n_flagged = 0;       // fallback-selection flags of the fused TopK path start clear every call
         // graph-conditional form: the rest of the SAE chain sits in the body of an IF node that runs only when a row needs it
         if (a.use_cond) cudaGraphSetConditional(a.cond, rows > 0 ? 1u : 0u);
@@ -389,6 +400,8 @@ front_kernel(const FrontArgs a) {
         rec.slot = t >= 0 ? slot : -1;
         rec.n_edit = (meta >> 8) & 0xff;
         rec.group_flags = t >= 0 ? (g | ((meta >> 16) & 1 ? kRecAddError : 0) | (s_gact[g] << kRecActShift)) : 0;
+        rec.W_dec = t >= 0 ? s_gwdec[g] : nullptr;
+        rec.theta = t >= 0 ? s_gtheta[g] : nullptr;
         a.row_rec[p] = rec;
         a.panel_row[p] = t;
         if (a.row_flag) a.row_flag[p] = 0;

@@ -59,7 +59,7 @@ __device__ void bitonic_sort_desc(unsigned long long* a, int n) {
 // finds the run where the running count reaches `need`; then the 32 lanes split that run.
 __device__ void find_digit(const int* hist, int n_bins, int need, int* s_out) {
   const int lane = threadIdx.x & 31;
-  const int per = n_bins / 32;                  // 64 or 32: a multiple of 4
+  const int per = n_bins / 32;                  // 64 (2048 bins) or 8 (256 bins): a multiple of 4
   const int hi = n_bins - lane * per;           // this lane's run is [hi - per, hi)
   int sum = 0;
   const int4* h4 = reinterpret_cast<const int4*>(hist + hi - per);
@@ -78,9 +78,10 @@ __device__ void find_digit(const int* hist, int n_bins, int need, int* s_out) {
   const int L = __ffs(hit) - 1;                 // exactly one lane (need <= total count)
   const int run_hi = n_bins - L * per;
   const int above_run = __shfl_sync(0xffffffffu, excl, L);
-  // level 2: lane l takes bins run_hi - 1 - l*w .. run_hi - (l+1)*w, w = per / 32 (2 or 1), descending
-  const int w = per / 32;
-  int c0 = hist[run_hi - 1 - lane * w], c1 = w == 2 ? hist[run_hi - 2 - lane * w] : 0;
+  // level 2: the run's bins, descending, w = max(per / 32, 1) per lane (lanes beyond the run hold nothing)
+  const int w = per >= 64 ? 2 : 1;
+  const bool in_run = lane * w < per;
+  const int c0 = in_run ? hist[run_hi - 1 - lane * w] : 0, c1 = (in_run && w == 2) ? hist[run_hi - 2 - lane * w] : 0;
   int inc2 = c0 + c1;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -88,7 +89,7 @@ __device__ void find_digit(const int* hist, int n_bins, int need, int* s_out) {
     if (lane >= o) inc2 += y;
   }
   const int before = above_run + inc2 - (c0 + c1);     // elements in bins above this lane's bins
-  if (before < need && before + c0 + c1 >= need) {
+  if (in_run && before < need && before + c0 + c1 >= need) {
     if (before + c0 >= need) {
       s_out[0] = run_hi - 1 - lane * w;
       s_out[1] = before;
@@ -171,18 +172,25 @@ __device__ __forceinline__ void push_cand(SelShared& sh, bool take, unsigned lon
 //   ORDERED sources (position order = id order) finish with an index-ordered pass and return 2;
 //   other sources return 0 (the caller falls back).
 // Returns 1 in the ordinary case.  Every thread of the CTA must call this.
-template <bool ORDERED, class Src>
-__device__ int radix_collect(const Src& src, int k, SelShared& sh, unsigned long long* clk = nullptr, bool stamp = false) {
+// kDigitBits: bits per refinement pass.  11 for a long source (the pre-activations of a whole row: fewer passes over
+// global memory); 8 for a row's candidates (a few thousand keys in shared memory: one pass nearly always settles
+// them, and a 256-bin histogram is cheap to clear and to search).
+// have_range: the caller already holds this thread's share of the keys' minimum and maximum in kmin / kmax.
+template <bool ORDERED, int kDigitBits, class Src>
+__device__ int radix_collect(const Src& src, int k, SelShared& sh, bool have_range = false, unsigned kmin = 0xffffffffu,
+                             unsigned kmax = 0u, unsigned long long* clk = nullptr, bool stamp = false) {
   const int tid = threadIdx.x, n = src.n;
   const int n_up = (n + kTailThreads - 1) / kTailThreads * kTailThreads;    // whole warps take part in every ballot
+  constexpr int kNb = 1 << kDigitBits;
+  static_assert(kNb <= kBins && kNb % 128 == 0, "digit width");
   // range of the keys
-  unsigned kmin = 0xffffffffu, kmax = 0u;
-  scan_keys(src, n, n_up, [&](int, unsigned key, bool valid) {
-    if (valid) {
-      kmin = min(kmin, key);
-      kmax = max(kmax, key);
-    }
-  });
+  if (!have_range)
+    scan_keys(src, n, n_up, [&](int, unsigned key, bool valid) {
+      if (valid) {
+        kmin = min(kmin, key);
+        kmax = max(kmax, key);
+      }
+    });
   kmin = __reduce_min_sync(0xffffffffu, kmin);
   kmax = __reduce_max_sync(0xffffffffu, kmax);
   if ((tid & 31) == 0) {
@@ -205,14 +213,14 @@ __device__ int radix_collect(const Src& src, int k, SelShared& sh, unsigned long
   const int enough = max(2 * k, 128);
   bool done = false;
   while (hi_bit > 0) {
-    const int width = min(11, hi_bit), shift = hi_bit - width, nb = 1 << width;
-    for (int b = tid; b < kBins; b += kTailThreads) sh.hist[b] = 0;     // digits >= nb do not occur: their bins stay 0
+    const int width = min(kDigitBits, hi_bit), shift = hi_bit - width, nb = 1 << width;
+    for (int b = tid; b < kNb; b += kTailThreads) sh.hist[b] = 0;       // digits >= nb do not occur: their bins stay 0
     __syncthreads();
     scan_keys(src, n, n_up, [&](int, unsigned key, bool valid) {
       if (valid && (hi_bit >= 32 || (key >> hi_bit) == prefix)) atomicAdd(&sh.hist[(key >> shift) & (nb - 1)], 1);
     });
     __syncthreads();
-    if (tid < 32) find_digit(sh.hist, kBins, need, sh.res);
+    if (tid < 32) find_digit(sh.hist, kNb, need, sh.res);
     __syncthreads();
     const int D = sh.res[0], above = sh.res[1];
     const int in_bin = sh.hist[D];
@@ -228,9 +236,23 @@ __device__ int radix_collect(const Src& src, int k, SelShared& sh, unsigned long
   if (tid == 0) sh.n = 0;
   __syncthreads();
   if (done) {
+    // every thread counts its survivors, a warp reserves room for all of its lanes with one atomic, then they write
+    int cnt = 0;
+    scan_keys(src, n, n_up, [&](int, unsigned key, bool valid) { cnt += valid && (key >> hi_bit) >= prefix; });
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, incl, o);
+      if ((tid & 31) >= o) incl += y;
+    }
+    int base = 0;
+    if ((tid & 31) == 31 && incl > 0) base = atomicAdd(&sh.n, incl);
+    int pos = __shfl_sync(0xffffffffu, base, 31) + incl - cnt;
     scan_keys(src, n, n_up, [&](int i, unsigned key, bool valid) {
-      const bool take = valid && (key >> hi_bit) >= prefix;
-      push_cand(sh, take, take ? (((unsigned long long)key << 32) | (0xffffffffu - src.id(i))) : 0ull);
+      if (valid && (key >> hi_bit) >= prefix) {
+        if (pos < kCand) sh.cand[pos] = ((unsigned long long)key << 32) | (0xffffffffu - src.id(i));
+        ++pos;
+      }
     });
     __syncthreads();
     return 1;
@@ -417,12 +439,12 @@ struct RowShared {
   int row0[kMaxGroups];     // first packed row of each weight set
 };
 
-__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 // Row role.  Per row, the dependent round trips are: the row's record; then -- requested together -- the edit
 // list, the candidate keys (into shared memory: the selection passes never go back to global memory) and the
-// tiles' 9th values; then the winners' feature ids; then the gather, whose decoder rows and hidden row were
-// prefetched into L2 as soon as the edit list was known.
+// tiles' 9th values; then the winners' feature ids; then the gather.  (Prefetching the edited decoder rows into
+// L2 while the selection runs was tried: one 128-byte line per lane makes 32 memory transactions per warp
+// instruction, and the 1024 prefetches of a row cost more -- 3 us -- than the latency they hid.)
 __device__ void tail_rows(const TailArgs& a, RowShared& sh, int n_groups) {
   const int tid = threadIdx.x;
   const int d = a.d, nvec = d >> 3;
@@ -463,11 +485,12 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh, int n_groups) {
       sh.ef[tid] = 0.f;
     }
     const int S = (int)gp->d_sae, k = gp->k;
-    const __nv_bfloat16* W_dec = gp->W_dec;
+    const __nv_bfloat16* W_dec = rec.W_dec;
     const float* z = a.Z + (size_t)p * a.ldz;
     uint4* hrow = reinterpret_cast<uint4*>(a.hidden + (size_t)t * d);
     const int n_tiles = S / kTileN, n_cand = n_tiles * kCandPerTile;
     unsigned ninth_max = 0u;                           // largest key among this thread's share of the tiles' 9th values
+    unsigned kmin = 0xffffffffu, kmax = 0u;            // range of this thread's share of the candidate keys
     if (from_cand && n_cand >= k) {
       const float* cv = a.cand_val + (size_t)p * a.cand_tiles * kCandPerTile;
       for (int i0 = tid; i0 < n_cand; i0 += 8 * kTailThreads) {
@@ -480,7 +503,12 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh, int n_groups) {
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
           const int i = i0 + u * kTailThreads;
-          if (i < n_cand) sh.keys[i] = f2key(v[u]);
+          if (i < n_cand) {
+            const unsigned key = f2key(v[u]);
+            sh.keys[i] = key;
+            kmin = min(kmin, key);
+            kmax = max(kmax, key);
+          }
         }
       }
       const float* ninth = a.cand_ninth + (size_t)p * a.cand_tiles;
@@ -488,17 +516,6 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh, int n_groups) {
     }
     __syncthreads();
     phase_stamp(a.clk, 21, stamp);
-    // the decoder rows of the edited features and (error term on) the row itself: on their way into L2 while the
-    // selection runs
-    if (topk || !add_error) {
-      const int lines = d >> 6;                        // 128-byte lines per row
-      for (int x = tid; x < n_edit * lines; x += kTailThreads) {
-        const int e = x / lines;
-        prefetch_l2(W_dec + (size_t)sh.eidx[e] * d + (size_t)(x - e * lines) * 64);
-      }
-      if (add_error)
-        for (int x = tid; x < lines; x += kTailThreads) prefetch_l2(reinterpret_cast<const __nv_bfloat16*>(hrow) + (size_t)x * 64);
-    }
     int* win_id = sh.feat + n_edit;                    // the winners follow the edit entries in the gather lists
     float* win_val = sh.coef + n_edit;
     if (topk) {
@@ -511,7 +528,7 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh, int n_groups) {
         bool flag = n_cand < k;                        // uniform
         if (!flag) {
           CandRow src{sh.keys, n_cand};
-          flag = radix_collect<false>(src, k, sh.sel, a.clk, stamp) == 0;
+          flag = radix_collect<false, 8>(src, k, sh.sel, true, kmin, kmax, a.clk, stamp) == 0;
         }
         phase_stamp(a.clk, 10, stamp);
         if (!flag) {
@@ -536,7 +553,7 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh, int n_groups) {
         }
       } else {
         ZRow src{z, S};
-        const int how = radix_collect<true>(src, k, sh.sel);
+        const int how = radix_collect<true, 11>(src, k, sh.sel);
         if (how == 2 && tid == 0) atomicOr(a.status, MIX_STATUS_TOPK_GENERAL);
         sorted = sort_desc(sh.sel);
         for (int i = tid; i < k; i += kTailThreads) {
@@ -672,11 +689,18 @@ constexpr int kDlEntries = kDlRows * kMaxEdits;
 struct DeltaShared {
   __align__(16) float coef[kDlEntries + kDlBatch][kDlRows];
   const uint4* wrow[kDlEntries + kDlBatch];
-  int idx[kMaxEdits];
-  int t[kDlRows], slot[kDlRows], n_edit[kDlRows], grp[kDlRows], changed[kDlRows];
+  int eidx[kDlEntries];               // feature of each entry
+  float enew[kDlEntries];             // f'_j of each entry
+  short efirst[kDlEntries], elen[kDlEntries];   // where the entry's own edit list starts among the entries, and its length
+  short eslot_row[kDlEntries];        // first row of the item that carries the entry's slot
+  int t[kDlRows], slot[kDlRows], n_edit[kDlRows], act[kDlRows], changed[kDlRows];
+  const __nv_bfloat16* wdec[kDlRows];
+  const float* theta[kDlRows];
 };
 
 // One work item of the delta role: row group `item / n_col_slices`, column slice `item % n_col_slices`.
+// Dependent round trips: the rows' records (which carry the decoder and threshold pointers); the edit lists of
+// their slots; the pre-activations and thresholds of the edited features; the decoder rows; the rows themselves.
 __device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int item, int n_rows) {
   const int tid = threadIdx.x;
   const int rg = item / a.n_col_slices, cs = item - rg * a.n_col_slices;
@@ -687,13 +711,14 @@ __device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int item, int n_r
   if (tid < kDlRows) {
     const int p = p0 + tid;                              // in bounds: the panel capacity is a multiple of 128
     const RowRec rec = a.row_rec[p];
-    const int g = rec.group_flags & kRecGroupMask;
-    const bool on = p < n_rows && rec.t >= 0 && (rec.group_flags & kRecAddError) && rec.n_edit > 0 &&
-                    ((rec.group_flags >> kRecActShift) & 3) != MIX_SAE_TOPK;
+    const int act = (rec.group_flags >> kRecActShift) & 3;
+    const bool on = p < n_rows && rec.t >= 0 && (rec.group_flags & kRecAddError) && rec.n_edit > 0 && act != MIX_SAE_TOPK;
     sh.t[tid] = on ? rec.t : -1;
     sh.slot[tid] = on ? rec.slot : -1;
     sh.n_edit[tid] = rec.n_edit;
-    sh.grp[tid] = g;
+    sh.act[tid] = act;
+    sh.wdec[tid] = rec.W_dec;
+    sh.theta[tid] = rec.theta;
     sh.changed[tid] = 0;
   }
   __syncthreads();
@@ -705,15 +730,7 @@ __device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int item, int n_r
   const int d = a.d;
   const int v = cs * kTailThreads + tid;                 // this thread's 16-byte column vector
   const bool in_cols = v < (d >> 3);
-  uint4 hraw[kDlRows];
-#pragma unroll
-  for (int r = 0; r < kDlRows; ++r) {
-    const int t = sh.t[r];
-    hraw[r] = make_uint4(0u, 0u, 0u, 0u);
-    if (t >= 0 && in_cols) hraw[r] = reinterpret_cast<const uint4*>(a.hidden + (size_t)t * d)[v];
-  }
-  // entries: the edit lists of the distinct slots, one after the other; thread e of a slot works out entry e
-  // for every row of that slot (the coefficient of a row of another slot is zero)
+  // entries: the edit lists of the distinct slots, one after the other (the coefficient of a row of another slot is zero)
   int n_entries = 0;                                    // CTA-uniform
   for (int r = 0; r < kDlRows; ++r) {
     const int slot = sh.slot[r];
@@ -721,53 +738,53 @@ __device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int item, int n_r
     for (int r2 = 0; r2 < r; ++r2) first = first && sh.slot[r2] != slot;
     if (!first) continue;
     const int n_edit = sh.n_edit[r];
-    if (tid < n_edit) sh.idx[tid] = a.edit_idx[slot * a.r_max + tid];
-    __syncthreads();
     if (tid < n_edit) {
-      const GroupEntry ge = a.groups[sh.grp[r]];
-      const int j = sh.idx[tid];
+      const int e = n_entries + tid;
+      const int j = a.edit_idx[slot * a.r_max + tid];
+      sh.eidx[e] = j;
+      sh.enew[e] = a.edit_mode[slot * a.r_max + tid] == MIX_EDIT_CLAMP ? a.edit_val[slot * a.r_max + tid] : 0.f;
+      sh.efirst[e] = (short)n_entries;
+      sh.elen[e] = (short)n_edit;
+      sh.eslot_row[e] = (short)r;
+      sh.wrow[e] = reinterpret_cast<const uint4*>(sh.wdec[r] + (size_t)j * d);
+    }
+    n_entries += n_edit;
+  }
+  __syncthreads();
+  if (tid < kDlBatch) sh.wrow[n_entries + tid] = sh.wrow[n_entries - 1];     // pad to a whole batch: repeats of the last decoder row
+  __syncthreads();
+  // thread e works out entry e's coefficient for every row of its slot.  (Requesting the first decoder rows before
+  // this step, so that they are in flight meanwhile, was tried: the registers they hold push the kernel over its
+  // 64-register budget and the spills cost more than the overlap gains.)
+  for (int e = tid; e < n_entries + kDlBatch; e += kTailThreads) {
+    float c[kDlRows] = {0.f, 0.f, 0.f, 0.f};
+    if (e < n_entries) {
+      const int j = sh.eidx[e], r = sh.eslot_row[e], slot = sh.slot[r], act = sh.act[r];
       bool alive = true;                                 // a later entry for the same feature wins
-      for (int e2 = tid + 1; e2 < n_edit; ++e2) alive = alive && (sh.idx[e2] != j);
-      const float fnew = a.edit_mode[slot * a.r_max + tid] == MIX_EDIT_CLAMP ? a.edit_val[slot * a.r_max + tid] : 0.f;
-      const float theta = ge.act == MIX_SAE_JUMPRELU ? ge.theta[j] : 0.f;
-      float c[kDlRows];
+      for (int e2 = e + 1; e2 < sh.efirst[e] + sh.elen[e]; ++e2) alive = alive && (sh.eidx[e2] != j);
+      const float theta = act == MIX_SAE_JUMPRELU ? sh.theta[r][j] : 0.f;
+      const float fnew = sh.enew[e];
 #pragma unroll
       for (int r2 = 0; r2 < kDlRows; ++r2) {
-        c[r2] = 0.f;
         if (sh.slot[r2] == slot && alive) {
           const float zj = a.Z[(size_t)(p0 + r2) * a.ldz + j];
-          const float f = ge.act == MIX_SAE_RELU ? fmaxf(zj, 0.f) : (zj > theta ? zj : 0.f);
+          const float f = act == MIX_SAE_RELU ? fmaxf(zj, 0.f) : (zj > theta ? zj : 0.f);
           c[r2] = fnew - f;
           if (c[r2] != 0.f) sh.changed[r2] = 1;
         }
       }
-#pragma unroll
-      for (int r2 = 0; r2 < kDlRows; ++r2) sh.coef[n_entries + tid][r2] = c[r2];
-      sh.wrow[n_entries + tid] = reinterpret_cast<const uint4*>(ge.W_dec + (size_t)j * d);
     }
-    n_entries += n_edit;
-    __syncthreads();
-  }
-  phase_stamp(a.clk, 24, stamp);
-  // pad to a whole batch: repeats of the last decoder row with zero coefficients
-  if (tid < kDlBatch) {
-    sh.wrow[n_entries + tid] = sh.wrow[n_entries - 1];
 #pragma unroll
-    for (int r2 = 0; r2 < kDlRows; ++r2) sh.coef[n_entries + tid][r2] = 0.f;
+    for (int r2 = 0; r2 < kDlRows; ++r2) sh.coef[e][r2] = c[r2];
   }
   __syncthreads();
+  phase_stamp(a.clk, 24, stamp);
   if (!in_cols) return;
   float acc[kDlRows][8];
 #pragma unroll
-  for (int r = 0; r < kDlRows; ++r) {
-    const __nv_bfloat162* pp = reinterpret_cast<const __nv_bfloat162*>(&hraw[r]);
+  for (int r = 0; r < kDlRows; ++r)
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float2 f2 = __bfloat1622float2(pp[i]);
-      acc[r][2 * i] = f2.x;
-      acc[r][2 * i + 1] = f2.y;
-    }
-  }
+    for (int i = 0; i < 8; ++i) acc[r][i] = 0.f;
   // kDlBatch decoder rows in flight per thread: the loop is bound by load latency, not arithmetic
   for (int e0 = 0; e0 < n_entries; e0 += kDlBatch) {
     uint4 q[kDlBatch];
@@ -783,13 +800,21 @@ __device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int item, int n_r
     }
   }
   phase_stamp(a.clk, 25, stamp);
+  uint4 hraw[kDlRows];
+#pragma unroll
+  for (int r = 0; r < kDlRows; ++r)
+    hraw[r] = sh.t[r] >= 0 ? reinterpret_cast<const uint4*>(a.hidden + (size_t)sh.t[r] * d)[v] : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
   for (int r = 0; r < kDlRows; ++r) {
     if (sh.slot[r] < 0 || !sh.changed[r]) continue;     // no effective edit: the row stays bit-exact
+    const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hraw[r]);
     uint4 o;
     __nv_bfloat162* pp = reinterpret_cast<__nv_bfloat162*>(&o);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) pp[i] = __floats2bfloat162_rn(acc[r][2 * i], acc[r][2 * i + 1]);
+    for (int i = 0; i < 4; ++i) {
+      const float2 h2 = __bfloat1622float2(hp[i]);
+      pp[i] = __floats2bfloat162_rn(h2.x + acc[r][2 * i], h2.y + acc[r][2 * i + 1]);
+    }
     reinterpret_cast<uint4*>(a.hidden + (size_t)sh.t[r] * d)[v] = o;
   }
 }
