@@ -421,6 +421,12 @@ probe_steer_team_kernel(const int* __restrict__ token_slot, const int* __restric
       }
     }
   }
+  // a probe's biases are requested as soon as the entry is here, not after the dot products they are added to
+  float bias_lo = 0.f, bias_hi = 0.f;
+  if (a.kind == MIX_PROBE && a.b != nullptr && warp == 0) {
+    if (lane < a.C) bias_lo = __ldg(a.b + lane);
+    if (lane + 32 < a.C) bias_hi = __ldg(a.b + lane + 32);
+  }
   if (a.gated && a.kind != 0 && !gate_open(gates, slot, t)) return;       // gate closed: the row passes through
   if (a.kind == MIX_STEER) {
     if (a.alpha == 0.f) return;                  // identity; the row stays bit-exact
@@ -526,7 +532,7 @@ probe_steer_team_kernel(const int* __restrict__ token_slot, const int* __restric
   __syncthreads();
   if (warp == 0) {
     for (int c = lane; c < a.C; c += 32) {
-      float z = a.b ? __ldg(a.b + c) : 0.f;
+      float z = c < 32 ? bias_lo : bias_hi;
 #pragma unroll
       for (int w = 0; w < NW; ++w) z += s_part[w][c];
       s_part[0][c] = z;            // only this lane reads or writes column c from here on
