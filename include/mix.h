@@ -42,7 +42,7 @@
  *   - weights are BORROWED: the caller keeps them alive and unchanged until the app /
  *     weight set is unregistered (or the context destroyed) and work already enqueued has
  *     finished.  (The library may also keep its own copy of small weights -- contexts with
- *     T_max <= 2048 copy steering / projection vectors and one-class probe weights at
+ *     T_max <= 2048 copy steering / projection vectors and one-class probe weights and biases at
  *     registration -- so changing borrowed weights in place needs a new registration.)
  *     Everything else (tables, edit lists, slot map) is copied.
  *   - one host thread per context at a time.

@@ -104,11 +104,14 @@ int check_slot(mix_ctx* c, int slot) {
 }
 
 // Publish an app entry: body first with valid = 0, then the valid word.
-int publish_app(mix_ctx* c, int slot, cudaStream_t s) {
+// bias_src: device fp32 whose value goes into the entry's `alpha` word before the entry becomes valid (a one-class
+// probe's bias in contexts whose hook kernel reads it from there), or null.
+int publish_app(mix_ctx* c, int slot, cudaStream_t s, const float* bias_src = nullptr) {
   AppEntry tmp = c->h_apps[slot];
   const int valid = tmp.valid;
   tmp.valid = 0;
   MIX_CUDA(c, cudaMemcpyAsync(c->d_apps + slot, &tmp, sizeof(AppEntry), cudaMemcpyHostToDevice, s));
+  if (bias_src) MIX_CUDA(c, cudaMemcpyAsync(&c->d_apps[slot].alpha, bias_src, sizeof(float), cudaMemcpyDeviceToDevice, s));
   if (valid) MIX_CUDA(c, cudaMemcpyAsync(&c->d_apps[slot].valid, &valid, sizeof(int), cudaMemcpyHostToDevice, s));
   return MIX_OK;
 }
@@ -522,7 +525,10 @@ int mix_register_app(mix_ctx* c, int slot, int kind, const void* desc, void* str
     }
     if (old_next >= 0) MIX_CUDA(c, cudaMemcpyAsync(c->d_chain_next + slot, c->h_chain_next + slot, sizeof(int), cudaMemcpyHostToDevice, s));
   }
-  return publish_app(c, slot, s);
+  // The bias of a one-class probe travels in the entry itself (its `alpha` word is otherwise unused): the
+  // one-CTA-per-row kernel then has it with the entry instead of one dependent load later.
+  const float* bias_src = (c->d_vec_arena && kind == MIX_PROBE && e.n_classes == 1) ? e.b : nullptr;
+  return publish_app(c, slot, s, bias_src);
 }
 
 int mix_unregister_app(mix_ctx* c, int slot, void* stream) {

@@ -122,8 +122,20 @@ __device__ __forceinline__ void probe_dots(const uint4* const* __restrict__ h, c
     for (int c = 0; c < NC; ++c) out[r][c] = warp_sum(acc[r][c]);
 }
 
+// 1 / (1 + e^-z) with the hardware exponential and reciprocal: a few instructions instead of the two library
+// routines' hundred on the one-warp tail of a decode step (0.28 us of a 3 us step); the relative error stays
+// below 1e-5 for |z| < 80, two orders under the 1e-3 the scores are held to.
+__device__ __forceinline__ float fast_sigmoid(float z) { return __frcp_rn(1.f + __expf(-z)); }
+
 // Logits (bias included) of one row in `logit` -> scores.  One warp; C <= 64.
 __device__ __forceinline__ void finish_probe(const float* logit, int C, int act, float* __restrict__ out, int lane) {
+  if (C == 1) {                                  // the decode step's case: one lane, no cross-lane work
+    if (lane == 0) {
+      const float z = logit[0];
+      out[0] = act == MIX_ACT_NONE ? z : (act == MIX_ACT_SOFTMAX ? 1.f : fast_sigmoid(z));
+    }
+    return;
+  }
   float z0 = lane < C ? logit[lane] : -INFINITY;
   float z1 = lane + 32 < C ? logit[lane + 32] : -INFINITY;
   if (act == MIX_ACT_SOFTMAX) {
@@ -136,8 +148,8 @@ __device__ __forceinline__ void finish_probe(const float* logit, int C, int act,
     z0 = e0 / sum;
     z1 = e1 / sum;
   } else if (act == MIX_ACT_SIGMOID) {
-    z0 = 1.f / (1.f + expf(-z0));
-    z1 = 1.f / (1.f + expf(-z1));
+    z0 = fast_sigmoid(z0);
+    z1 = fast_sigmoid(z1);
   }
   if (lane < C) out[lane] = z0;
   if (lane + 32 < C) out[lane + 32] = z1;
@@ -171,7 +183,7 @@ __device__ __forceinline__ void warp_row(const RowApp& a, __nv_bfloat16* __restr
     if (lane == 0) {
       const float zz = z[0][0] + (a.b ? __ldg(a.b) : 0.f);
       // one class: raw logit, sigmoid, or a softmax over a single entry (= 1)
-      out[0] = a.act == MIX_ACT_NONE ? zz : (a.act == MIX_ACT_SOFTMAX ? 1.f : 1.f / (1.f + expf(-zz)));
+      out[0] = a.act == MIX_ACT_NONE ? zz : (a.act == MIX_ACT_SOFTMAX ? 1.f : fast_sigmoid(zz));
     }
     return;
   }
@@ -421,11 +433,16 @@ probe_steer_team_kernel(const int* __restrict__ token_slot, const int* __restric
       }
     }
   }
-  // a probe's biases are requested as soon as the entry is here, not after the dot products they are added to
+  // A one-class probe's bias came with the entry (registration put it into the `alpha` word); the biases of a
+  // wider probe are requested as soon as the entry is here, not after the dot products they are added to.
   float bias_lo = 0.f, bias_hi = 0.f;
-  if (a.kind == MIX_PROBE && a.b != nullptr && warp == 0) {
-    if (lane < a.C) bias_lo = __ldg(a.b + lane);
-    if (lane + 32 < a.C) bias_hi = __ldg(a.b + lane + 32);
+  if (a.kind == MIX_PROBE && warp == 0) {
+    if (a.C == 1) {
+      bias_lo = a.alpha;
+    } else if (a.b != nullptr) {
+      if (lane < a.C) bias_lo = __ldg(a.b + lane);
+      if (lane + 32 < a.C) bias_hi = __ldg(a.b + lane + 32);
+    }
   }
   if (a.gated && a.kind != 0 && !gate_open(gates, slot, t)) return;       // gate closed: the row passes through
   if (a.kind == MIX_STEER) {

@@ -449,6 +449,34 @@ def test_replacing_a_weight_set_and_failed_edit_updates_change_nothing():
     m.destroy()
 
 
+def test_one_class_probe_bias_and_raw_logit_in_a_decode_context():
+    """One-class probes with non-zero biases in a context of at most 2048 rows (the one-CTA-per-row kernel, which
+    takes the bias from the app entry): sigmoid and raw-logit probes, a probe without a bias, and a re-registration
+    with another bias under the same captured graph."""
+    mixlib = _mixlib()
+    d, T = 512, 96
+    g = torch.Generator(device=DEV); g.manual_seed(77)
+    hidden = torch.randn((T, d), generator=g, device=DEV, dtype=torch.float32).to(torch.bfloat16)
+    def probe(bias, act):
+        Wp = (torch.randn((1, d), generator=g, device=DEV) * d ** -0.5).to(torch.bfloat16)
+        b = None if bias is None else torch.tensor([bias], dtype=torch.float32, device=DEV)
+        return W.Probe(W=Wp, b=b, act=act)
+    apps = {0: probe(1.75, W.ACT_SIGMOID), 1: probe(-3.5, W.ACT_NONE), 2: probe(None, W.ACT_SIGMOID), 3: probe(0.25, W.ACT_NONE)}
+    token_slot = (np.arange(T) % 5 - 1).astype(np.int32)
+    w = W.Workload("bias", d, T, T, hidden, token_slot, apps, {}, n_slots_max=4, C_max=1)
+    out = run_gpu(w, graph=True)
+    st = check_parity(W.host(w), out)
+    assert st["max_score_rel"] < 1e-4
+    # a new registration of slot 1 with another bias takes effect without a new capture
+    m = out["mix"]
+    apps[1] = W.Probe(W=apps[1].W, b=torch.tensor([2.0], dtype=torch.float32, device=DEV), act=W.ACT_NONE)
+    m.register_probe(1, apps[1].W, apps[1].b, apps[1].act)
+    w2 = W.Workload("bias2", d, T, T, hidden, token_slot, apps, {}, n_slots_max=4, C_max=1)
+    out2 = run_gpu(w2, mix=m)
+    check_parity(W.host(w2), out2)
+    m.destroy()
+
+
 # ------------------------------------------------------------------ full-size configs, sampled rows
 def test_sae_heavy_full_size_sampled_rows():
     w = W.make_sae_heavy(DEV, edit_hint=oracle_edit_hint)
