@@ -40,7 +40,7 @@ SAE_FLAGS = 2            # mix_config.flags of the SAE contexts of the extras / 
 # dram__bytes_read.sum + dram__bytes_write.sum of one probe_steer_team_kernel launch on the decode workload, from an
 # ncu capture of this kernel (reads only: the steered rows are still dirty in L2 when the kernel ends).  Reported as
 # `roofline.traffic`, labelled as not re-measured; the fraction itself uses the algorithmic bytes.
-DECODE_DRAM_BYTES_PER_LAUNCH = 2404352
+DECODE_DRAM_BYTES_PER_LAUNCH = 2410752
 
 
 NOMINAL_HBM_GBS = 8000.0        # B200 HBM3e (DGX figure; HGX 7.7 TB/s): context beside the measured peak
