@@ -22,8 +22,9 @@
  *              in place; r is used as given (pass a unit vector for an orthogonal projection).
  *   slot -1    no app: the row is never written and stays bit-identical (Section 4.2 "Toggling
  *              semantics": an inactive app costs a request nothing).  It is not read either, with one
- *              exception: in a batch of more than 2048 rows that is dense in multi-class probe rows,
- *              the probe kernel streams whole 128-row tiles and discards the rows that are not its own.
+ *              exception: in a batch of more than 2048 rows, the 128-row tiles that hold multi-class
+ *              probe rows are streamed whole by the probe kernel when those tiles are, together, at
+ *              least half full of such rows; the rows of a tile that are not its own are discarded.
  *
  * Rows are independent.  Activation of an app for a request is data (the slot map and the
  * small device tables), never launch structure: mix_apply() only enqueues kernels with a

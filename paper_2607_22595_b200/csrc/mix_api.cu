@@ -84,7 +84,7 @@ void free_all(mix_ctx* c) {
   cudaFree(c->d_edit_idx); cudaFree(c->d_edit_val); cudaFree(c->d_edit_mode); cudaFree(c->d_status);
   cudaFree(c->d_tmp_req); cudaFree(c->d_tmp_req_slot); cudaFree(c->d_panel); cudaFree(c->d_panel_row); cudaFree(c->d_act_scale); cudaFree(c->d_tau); cudaFree(c->d_tau_min); cudaFree(c->d_eo_row_delta); cudaFree(c->d_eo_coef);
   cudaFree(c->d_mtile_group); cudaFree(c->d_route); cudaFree(c->d_z);
-  cudaFree(c->d_tmap_w); cudaFree(c->d_tmap_w_half); cudaFree(c->d_phase_clk); cudaFree(c->d_tmap_probe); cudaFree(c->d_mc_dense); cudaFree(c->d_cand_val); cudaFree(c->d_cand_idx);
+  cudaFree(c->d_tmap_w); cudaFree(c->d_tmap_w_half); cudaFree(c->d_phase_clk); cudaFree(c->d_tmap_probe); cudaFree(c->d_mc_census); cudaFree(c->d_mc_tiles); cudaFree(c->d_cand_val); cudaFree(c->d_cand_idx);
   cudaFree(c->d_cand_ninth); cudaFree(c->d_row_flag); cudaFree(c->d_mtile_flag); cudaFree(c->d_n_flagged);
   if (c->owned_b_eff)
     for (int g = 0; g < c->cfg.n_groups_max; ++g) cudaFree(c->owned_b_eff[g]);
@@ -314,10 +314,11 @@ int mix_create(mix_ctx** out, const mix_config* cfg) {
   }
   if (e == cudaSuccess && has_tc_probe_stage(c)) {
     // large batches with multi-class probes: the tensor-core probe kernel needs a map per probe matrix
-    if (dev_alloc(&c->d_tmap_probe, NS) != cudaSuccess || dev_alloc(&c->d_mc_dense, 1) != cudaSuccess) {
+    if (dev_alloc(&c->d_tmap_probe, NS) != cudaSuccess || dev_alloc(&c->d_mc_census, 1) != cudaSuccess ||
+        dev_alloc(&c->d_mc_tiles, (size_t)(T + kTileM - 1) / kTileM) != cudaSuccess) {
       cudaGetLastError(); free_all(c); free(c); return MIX_ERR_NO_MEMORY;
     }
-    e = cudaMemset(c->d_mc_dense, 0, sizeof(int));
+    e = cudaMemset(c->d_mc_census, 0, sizeof(McCensus));
     if (load_encode_fn() != MIX_OK) e = cudaErrorUnknown;
     if (e == cudaSuccess) e = probe_tc_prepare();
   }
@@ -772,7 +773,7 @@ int apply_impl(mix_ctx* c, void* hidden, int T, float* scores_out, void* stream,
   if (tc) {
     if (make_tmap(&tm_hidden, h, (unsigned long long)c->cfg.T_max, c->cfg.d_model, kTileM) != MIX_OK)
       MIX_FAIL(c, MIX_ERR_CUDA, "cuTensorMapEncodeTiled failed for hidden");
-    MIX_CUDA(c, launch_mc_decide(c, T, ps));
+    MIX_CUDA(c, launch_mc_census(c, T, ps));
     MIX_CUDA(c, tap());
     if (tc_fork) {
       MIX_CUDA(c, cudaEventRecord(c->ev_fork, ps));

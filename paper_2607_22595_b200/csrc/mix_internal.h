@@ -89,6 +89,13 @@ struct __align__(16) RowDelta {
   const __nv_bfloat16* W_dec;
 };
 
+// Census of a large batch's multi-class probe rows (contexts of more than 2048 rows with such probes and no SAE
+// weight sets): which 128-row tiles hold any, how many rows in all, and which of the two probe kernels takes the call.
+struct McCensus {
+  int n_tiles, n_rows, use_tc, pad_;     // the result the probe kernels read
+  int w_tiles, w_rows, w_done, pad2_;    // counters of the census in progress (zero between calls)
+};
+
 // Result of the routing step for the SAE path (one instance in device memory).
 struct RouteState {
   int n_panel_rows;                 // rows of the packed panel in use (multiple of kTileM)
@@ -159,7 +166,8 @@ struct Ctx {
   CUtensorMap* d_tmap_w;    // [n_groups_max] W_enc maps (box kTileK x kTileN, 128B swizzle)
   CUtensorMap* d_tmap_w_half;   // [n_groups_max] the same with boxes of kTileN / 2 rows: what one CTA of a pair fetches
   CUtensorMap* d_tmap_probe;   // [n_slots_max] maps of multi-class probe matrices (box kTileK x 32), large-batch contexts only
-  int* d_mc_dense;          // [1] is this call's batch dense in multi-class probe rows?  written by mc_decide_kernel
+  McCensus* d_mc_census;    // census of the 128-row tiles that hold multi-class probe rows, taken by mc_census_kernel every call
+  int* d_mc_tiles;          // [ceil(T_max / 128)] those tiles, in no particular order
   CUtensorMap tmap_panel;   // panel map (box kTileK x kTileM, 128B swizzle)
 
   // probe/steer kernels run beside the SAE chain on this stream (created with the context)
@@ -239,10 +247,10 @@ __device__ __forceinline__ float key2f(unsigned k) {
 // kernel launchers (each returns the CUDA error of the launch)
 cudaError_t launch_probe_steer(const Ctx* c, __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s, bool allow_pdl);
 // Multi-class probes of large batches have two kernels; both are launched and exactly one does the work, chosen
-// on the device (mc_decide_kernel samples the slot map, mc_batch_is_dense in row_lookup.cuh, and leaves the
-// answer in d_mc_dense): probe_tc (tcgen05, streams whole 128-row tiles: batches
-// dense in such rows) or probe_multiclass (mma.sync, 16-row tiles: sparse ones).
-cudaError_t launch_mc_decide(const Ctx* c, int T, cudaStream_t s);
+// on the device (mc_census_kernel lists the 128-row tiles that hold such rows and leaves the choice in
+// d_mc_census): probe_tc (tcgen05, streams whole 128-row tiles of that list: batches whose listed tiles are at
+// least half full of such rows) or probe_multiclass (mma.sync, 16-row tiles: rows scattered thinly).
+cudaError_t launch_mc_census(const Ctx* c, int T, cudaStream_t s);
 cudaError_t launch_probe_tc(const Ctx* c, const CUtensorMap& tmap_hidden, int T, float* scores, cudaStream_t s);
 cudaError_t launch_probe_multiclass(const Ctx* c, const __nv_bfloat16* hidden, int T, float* scores, cudaStream_t s);
 cudaError_t probe_tc_prepare();   // opt in to the large dynamic shared memory size

@@ -13,8 +13,8 @@
 // columns, + bias, softmax / sigmoid / identity, scores out), warp 6 = scout (reads the tile's slot
 // ids and app entries, evaluates gates, groups the rows by probe and hands the other roles one
 // descriptor per pass through a small ring).  Rows of other kinds inside a tile are streamed but
-// ignored; tiles without such a probe are skipped -- which is why this kernel only takes batches
-// that are dense in such rows (decided by probe_steer_kernel, see mc_batch_is_dense); sparse ones go to the 16-row mma.sync kernel.  No TMA multicast, no clusters; every wait is
+// ignored.  The CTAs share out the tiles that a census kernel listed as holding such rows (mc_census_kernel), and the
+// kernel takes the call when those tiles are at least half full of such rows; thinly scattered rows go to the 16-row mma.sync kernel.  No TMA multicast, no clusters; every wait is
 // bounded (on expiry: MIX_STATUS_WAIT_TIMEOUT, copies are given time to land, tensor memory freed).
 #include "mix_internal.h"
 #include "row_lookup.cuh"
@@ -69,16 +69,18 @@ __global__ void __launch_bounds__(kPThreads, 1)
 probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const CUtensorMap* __restrict__ tmap_probe,
                 const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
                 const AppEntry* __restrict__ apps, const GateEntry* __restrict__ gates, int n_slots, int d,
-                float* __restrict__ scores, int C_max, unsigned* __restrict__ status, const int* __restrict__ mc_dense_flag,
-                int test_stall) {
+                float* __restrict__ scores, int C_max, unsigned* __restrict__ status, const McCensus* __restrict__ census,
+                const int* __restrict__ census_tiles, int test_stall) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* tiles = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   PShared* sh = reinterpret_cast<PShared*>(tiles + kPStages * kPStageBytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_live = min(T, __ldg(n_live_p));
-  const int n_tiles = (n_live + kTileM - 1) / kTileM;
+  // the tiles of this call that hold multi-class probe rows, as the census listed them (in no particular order):
+  // CTAs share THEM out, so a batch whose hooked requests are clustered still spreads evenly over the SMs
+  if (!census->use_tc) return;                         // rows scattered thinly: probe_multiclass_kernel's call
+  const int n_tiles = census->n_tiles;
   if ((int)blockIdx.x >= n_tiles) return;              // CTA-uniform: this CTA owns no tile
-  if (!*mc_dense_flag) return;                         // a sparse batch is probe_multiclass_kernel's
   if (threadIdx.x == 0) {
     for (int s = 0; s < kPStages; ++s) {
       mbar_init(smem_u32(&sh->full[s]), 1);
@@ -108,7 +110,8 @@ probe_tc_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const CUtensorM
     int di = 0;
     unsigned dphase = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+    for (int ti = blockIdx.x; ti < n_tiles && ok; ti += gridDim.x) {
+      const int tile = __ldg(census_tiles + ti);
       int s[4], blk[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
@@ -327,7 +330,7 @@ cudaError_t launch_probe_tc(const Ctx* c, const CUtensorMap& tmap_hidden, int T,
   if (scores == nullptr) return cudaSuccess;
   probe_tc_kernel<<<c->n_sms, kPThreads, kPSmemBytes, s>>>(tmap_hidden, c->d_tmap_probe, c->d_token_slot, c->d_n_live, T,
                                                            c->d_apps, c->d_gates, c->cfg.n_slots_max, c->cfg.d_model, scores,
-                                                           c->cfg.C_max, c->d_status, c->d_mc_dense,
+                                                           c->cfg.C_max, c->d_status, c->d_mc_census, c->d_mc_tiles,
                                                            (c->cfg.flags & MIX_FLAG_TEST_STALL_ENCODE) ? 1 : 0);
   return cudaGetLastError();
 }

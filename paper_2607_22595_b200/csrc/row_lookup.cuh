@@ -62,32 +62,4 @@ __device__ __forceinline__ RowApp lookup(int s, int t, const AppEntry* __restric
   return r;
 }
 
-// Is the batch dense in multi-class probe rows (2..32 classes)?  256 live rows at scattered, fixed
-// positions are looked at (slot id, then kind and class count of its app; gates are ignored): at least
-// half of them must be such rows.  The positions are a multiplicative hash of 0..255, not an even
-// stride: serving batches are periodic (requests of equal length dealt round-robin over apps) and
-// an even stride can land on one app every time.  Needs n_live >= 1 and at least 64 threads; every
-// thread of the CTA must call it.
-__device__ __forceinline__ bool mc_batch_is_dense(const int* __restrict__ token_slot, const AppEntry* __restrict__ apps,
-                                                  int n_slots, int n_live) {
-  int hit = 0;
-  if (threadIdx.x < 64) {
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const unsigned i = threadIdx.x * 4 + j;
-      const int t = (int)((i * 2654435761u + 0x9E3779B9u) % (unsigned)n_live);
-      const int s = __ldg(token_slot + t);
-      if (s >= 0 && s < n_slots) {
-        const int4 q0 = __ldg(reinterpret_cast<const int4*>(apps + s));    // valid, kind, n_classes, act
-        hit += q0.x && (q0.y & kKindMask) == MIX_PROBE && q0.z > 1 && q0.z <= 32;
-      }
-    }
-  }
-  hit = __reduce_add_sync(0xffffffffu, hit);            // warps 0 and 1 hold the sample
-  __shared__ int s_hits[2];
-  if (threadIdx.x < 64 && (threadIdx.x & 31) == 0) s_hits[threadIdx.x >> 5] = hit;
-  __syncthreads();
-  return 2 * (s_hits[0] + s_hits[1]) >= 256;
-}
-
 }  // namespace mix

@@ -1,5 +1,6 @@
-"""GPU: the tensor-core probe kernel (large batches dense in multi-class probe rows, contexts without SAE weight
-sets) and the device-side choice between it and the 16-row kernel."""
+"""GPU: the tensor-core probe kernel (large batches whose tiles with multi-class probe rows are mostly full,
+contexts without SAE weight sets), the census of those tiles, and the device-side choice between that kernel
+and the 16-row kernel."""
 import numpy as np
 import pytest
 import torch
@@ -65,16 +66,42 @@ def test_dense_batch_with_other_kinds_unhooked_rows_and_a_gate():
     assert np.array_equal(out["hidden"][unhooked], W.bits(w.hidden)[unhooked])
 
 
-@pytest.mark.parametrize("frac", [0.45, 0.55])
-def test_both_sides_of_the_density_threshold(frac):
-    # just below half of the rows are multi-class probes: the 16-row kernel; just above: the tensor-core one.
-    # Either way the result is the oracle's.
+@pytest.mark.parametrize("fill", [0.40, 0.60])
+def test_both_sides_of_the_fill_threshold(fill):
+    # every 128-row tile holds multi-class probe rows in its first `fill` part, nothing in the rest: below half
+    # the 16-row kernel takes the call, above half the tensor-core one.  Either way the result is the oracle's.
     T_max, d = 2304, 256
-    n = int(frac * T_max)
-    slot = np.where(np.arange(T_max) < n, (np.arange(T_max) // 64) % 2, -1)
+    t = np.arange(T_max)
+    slot = np.where((t % 128) < int(fill * 128), (t // 64) % 2, -1)
     w = _probe_workload(T_max, T_max, d, slot, [4, 12], [W.ACT_SOFTMAX, W.ACT_SOFTMAX])
     out = run_gpu(w)
     check_parity(W.host(w), out)
+
+
+@pytest.mark.parametrize("graph", [False, True])
+def test_sparse_batch_of_clustered_requests_takes_the_tile_list(graph):
+    # a quarter of the requests (of 200 rows each) carry a multi-class probe, the rest are unhooked or steered:
+    # the census lists about a third of the tiles, nearly full, and the tensor-core kernel shares THEM out;
+    # replayed twice with another slot map in between, so that the census counters are seen to start from zero
+    T_max, d = 6000, 384
+    req = np.arange(T_max) // 200
+    slot = np.where(req % 4 == 0, (req // 4) % 2, np.where(req % 4 == 1, 2, -1))
+    w = _probe_workload(T_max, T_max - 57, d, slot, [16, 5, 0], [W.ACT_SOFTMAX, W.ACT_SOFTMAX, 0])
+    out = run_gpu(w, graph=graph, replays=2)
+    check_parity(W.host(w), out)
+    m = out["mix"]
+    slot2 = np.where(req % 2 == 0, 1, 0)                                   # every tile full of probe rows now
+    w2 = _probe_workload(T_max, T_max, d, slot2, [16, 5, 0], [W.ACT_SOFTMAX, W.ACT_SOFTMAX, 0])
+    w2.apps = w.apps
+    m.set_slot_map(slot2.astype(np.int32), T_max)
+    w2.hidden = w.hidden
+    out2 = run_gpu(w2, mix=m)
+    check_parity(W.host(w2), out2)
+    m.set_slot_map(slot.astype(np.int32), T_max - 57)
+    out3 = run_gpu(w, mix=m)
+    check_parity(W.host(w), out3)
+    unhooked = np.nonzero(slot < 0)[0]
+    assert np.array_equal(out3["hidden"][unhooked], W.bits(w.hidden)[unhooked])
 
 
 def test_same_scores_from_both_kernels():
