@@ -222,13 +222,13 @@ cudaError_t launch_pdl(int which, void (*kernel)(KArgs...), dim3 grid, dim3 bloc
 #endif
 
 #ifdef __CUDACC__
-// Profiling aid: thread `who` (a bool) stamps slot i of the phase-clock array: slots 0, 7, 8 and 15 (a kernel's
-// first and last stamps) with the global nanosecond timer, the others with the SM's cycle counter -- cheap to
+// Profiling aid: thread `who` (a bool) stamps slot i of the phase-clock array: slots 0, 7, 8, 15 and 26.. (a kernel's
+// first and last stamps; the encode kernel's) with the global nanosecond timer, the others with the SM's cycle counter -- cheap to
 // read, and comparable between stamps of the same CTA.
 __device__ __forceinline__ void phase_stamp(unsigned long long* clk, int i, bool who) {
   if (clk != nullptr && who) {
     unsigned long long t;
-    if (i == 0 || i == 7 || i == 8 || i == 15) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    if (i == 0 || i == 7 || i == 8 || i == 15 || i >= 26) asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     else t = (unsigned long long)clock64();
     clk[i] = t;
   }

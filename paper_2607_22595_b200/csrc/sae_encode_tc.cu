@@ -55,7 +55,10 @@ template <int kEnc, int kEpi, bool kPair> struct TcCfg {
   static constexpr int kEpiWarps = kEpi;
   static constexpr int kXchgBytes = kEpiWarps == 8 ? 2 * 4 * kXchgEntries * 32 * 8 : 0;   // [acc][quarter][entry][lane] x (value, column)
   static constexpr int kThreads = 64 + kEpiWarps * 32;
-  static constexpr int kSmemBytes = kRingBytes + 1024 /* alignment slack */ + 1024 /* TcShared */ + kXchgBytes;
+  // each epilogue warp keeps the bias (and, for codes, the feature scale) of its columns of the current tile in
+  // shared memory, fetched while the tile's main loop still runs
+  static constexpr int kEpiVecBytes = 2 * 4 * kTileN * 4;   // [bias, scale][warp][its columns] floats: 8 KiB with 4 or 8 warps
+  static constexpr int kSmemBytes = kRingBytes + 1024 /* alignment slack */ + 1024 /* TcShared */ + kXchgBytes + kEpiVecBytes;
   static_assert(kSmemBytes <= 227 * 1024, "shared memory per CTA");
 };
 constexpr int kTmemCols = 512;                 // two 128 x 256 fp32 accumulators
@@ -202,7 +205,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
                  const int* __restrict__ mtile_flag, const int* __restrict__ n_flagged, float* __restrict__ cand_val,
                  int* __restrict__ cand_idx, float* __restrict__ cand_ninth, int cand_tiles, int w_tiled, int test_stall,
                  const float* __restrict__ act_scale, unsigned* __restrict__ tau_slots, unsigned* __restrict__ tau_min,
-                 int lo_row0) {
+                 int lo_row0, unsigned long long* __restrict__ clk) {
   constexpr bool kE4 = kEnc != 0;                      // E4M3 x E4M3 contraction
   constexpr bool kSplit = kEnc == 1;                   // the panel row is hi + lo: two operand tiles per k-block
   constexpr int kBlockK = kE4 ? 2 * kTileK : kTileK;   // elements per 128-byte row of either operand
@@ -214,6 +217,8 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
   constexpr int kEpiCols = kTileN / (kEpiWarps / 4);   // columns of a tile per epilogue warp
   pdl_wait();
   pdl_launch_dependents();
+  const bool stamp = clk != nullptr && blockIdx.x == 0 && threadIdx.x == 0 && mode == 0 && !kPair;
+  phase_stamp(clk, 26, stamp);
   if (mode == 1 && *n_flagged == 0) return;
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment: required by the 128-byte swizzle atoms
@@ -221,6 +226,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
   TcShared* sh = reinterpret_cast<TcShared*>(tiles + Cfg::kRingBytes);
   float* xchg_val = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(sh) + 1024);
   int* xchg_idx = reinterpret_cast<int*>(xchg_val + 2 * 4 * kXchgEntries * 32);
+  float* epi_vec = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(sh) + 1024 + Cfg::kXchgBytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // CTA pairs: rank 0 leads (it issues the pair's tensor-core instructions and owns the barriers both CTAs' copies
   // complete on); `worker` numbers the units that walk the tile list -- pairs, or single CTAs
@@ -277,6 +283,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
   else __syncthreads();
   tc_fence_after();
   const unsigned tmem_base = sh->tmem_base;
+  phase_stamp(clk, 27, stamp);
   // (the interleaved order serves the TopK epilogue's running bound; without TopK rows the plain order is a little faster)
   const int uniform_nt = sh->rs.n_topk_rows > 0 ? uniform_feature_tiles(sh->rs, n_groups) : 0;
   const int num_kb = d / kBlockK;
@@ -395,14 +402,28 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
       const bool topk_tile = mode == 0 && groups[t.group].act == MIX_SAE_TOPK;
       const int k_row = groups[t.group].k;
       const bool use_tau = topk_tile && valid && tau_slots != nullptr && k_row <= kTauSlots;
+      // (tiles of the launch's last wave publish nothing: no tile that starts later is left to read it)
+      const bool publish_tau = use_tau && tile + n_workers < total_tiles;
       unsigned tau_key = 0u;                   // 0: no bound yet
       if (use_tau) tau_key = __ldcg(tau_min + p);     // the smallest slot, as of the last time a publisher looked
+      // this warp's columns of the bias (and feature scale) go to shared memory now, while the accumulator is
+      // still being computed: read from global memory inside the loop below, 32 columns at a time between
+      // tensor-memory loads, they were four exposed round trips per tile
+      constexpr bool kScaled = kEnc != 0;      // the accumulator is in units of the codes
+      float* wb = epi_vec + (warp - 2) * kEpiCols;
+      float* ws = wb + kEpiWarps * kEpiCols;
+      {
+        const float* bias_g = groups[t.group].b_eff + (size_t)t.n_tile * kTileN + c_lo;
+        const float* wsc_g = kScaled ? groups[t.group].w_scale + (size_t)t.n_tile * kTileN + c_lo : nullptr;
+        for (int j = lane * 4; j < kEpiCols; j += 128) {
+          *reinterpret_cast<float4*>(wb + j) = __ldg(reinterpret_cast<const float4*>(bias_g + j));
+          if (kScaled) *reinterpret_cast<float4*>(ws + j) = __ldg(reinterpret_cast<const float4*>(wsc_g + j));
+        }
+        __syncwarp();
+      }
       // warp-uniform decision: tcgen05.ld below needs the whole warp
       if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&sh->tmem_full[acc]), acc_phase, sh, status))) break;
       tc_fence_after();
-      const float* bias = groups[t.group].b_eff + (size_t)t.n_tile * kTileN;
-      constexpr bool kScaled = kEnc != 0;      // the accumulator is in units of the codes
-      const float* wsc = kScaled ? groups[t.group].w_scale + (size_t)t.n_tile * kTileN : nullptr;
       const float ars = kE4 ? (valid ? __ldg(act_scale + p) : 0.f) : 1.f;     // power of two: the products below are exact
       const unsigned taddr = tmem_base + ((unsigned)(q * 32) << 16) + acc * kTileN;
       if (topk_tile) {
@@ -422,9 +443,9 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
           tmem_ld32(taddr + c, v);
 #pragma unroll
           for (int i = 0; i < 32; i += 4) {
-            const float4 b4 = __ldg(reinterpret_cast<const float4*>(bias + c + i));
+            const float4 b4 = *reinterpret_cast<const float4*>(wb + (c - c_lo) + i);
             float4 s4 = make_float4(1.f, 1.f, 1.f, 1.f);
-            if (kScaled) s4 = __ldg(reinterpret_cast<const float4*>(wsc + c + i));
+            if (kScaled) s4 = *reinterpret_cast<const float4*>(ws + (c - c_lo) + i);
             if (kE4) { s4.x *= ars; s4.y *= ars; s4.z *= ars; s4.w *= ars; }
             v[i] = kScaled ? fmaf(v[i], s4.x, b4.x) : v[i] + b4.x;
             v[i + 1] = kScaled ? fmaf(v[i + 1], s4.y, b4.y) : v[i + 1] + b4.y;
@@ -472,7 +493,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
           ci[0] = make_int4(j0 + ti[0], j0 + ti[1], j0 + ti[2], j0 + ti[3]);
           ci[1] = make_int4(j0 + ti[4], j0 + ti[5], j0 + ti[6], j0 + ti[7]);
           cand_ninth[slot] = tv[kCandPerTile];
-          if (use_tau) {
+          if (publish_tau) {
             // this tile's r-th largest goes to slot (n_tile + r k/8) mod k: no two (tile, rank) pairs are the same
             // element, eight consecutive feature tiles fill every slot, and every slot sees all ranks over time
             unsigned* sp = tau_slots + p * kTauSlots;
@@ -511,9 +532,9 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
           if (valid) {
 #pragma unroll
             for (int i = 0; i < 32; i += 4) {
-              const float4 b4 = __ldg(reinterpret_cast<const float4*>(bias + c + i));
+              const float4 b4 = *reinterpret_cast<const float4*>(wb + (c - c_lo) + i);
               float4 s4 = make_float4(1.f, 1.f, 1.f, 1.f);
-              if (kScaled) s4 = __ldg(reinterpret_cast<const float4*>(wsc + c + i));
+              if (kScaled) s4 = *reinterpret_cast<const float4*>(ws + (c - c_lo) + i);
               if (kE4) { s4.x *= ars; s4.y *= ars; s4.z *= ars; s4.w *= ars; }
               float4 o;
               o.x = kScaled ? fmaf(v[i], s4.x, b4.x) : v[i] + b4.x;
@@ -538,6 +559,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
 
   tc_fence_before();
   __syncthreads();
+  phase_stamp(clk, 28, stamp);
   if (sh->abort_flag) {
     // give copies that are still in flight time to land before shared memory is released
     const long long t0 = clock64();
@@ -550,6 +572,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
     if (kPair) tmem_dealloc_pair(tmem_base, kTmemCols);
     else tmem_dealloc(tmem_base, kTmemCols);
   }
+  phase_stamp(clk, 29, stamp);
 }
 
 // Registration-time copy of W_enc [S, d] into [S/256][d/64][256][64]: one thread per 16 bytes.
@@ -667,7 +690,8 @@ static cudaError_t launch_encode_tc_as(const Ctx* c, int mode, cudaStream_t s) {
                             c->cfg.n_groups_max, c->d_z, (long long)c->cfg.d_sae_max, c->cfg.d_model, c->d_status, mode,
                             static_cast<const int*>(c->d_mtile_flag), static_cast<const int*>(c->d_n_flagged), c->d_cand_val,
                             c->d_cand_idx, c->d_cand_ninth, c->cand_tiles, w_tiled, stall,
-                            static_cast<const float*>(c->d_act_scale), c->d_tau, c->d_tau_min, c->panel_rows_cap);
+                            static_cast<const float*>(c->d_act_scale), c->d_tau, c->d_tau_min, c->panel_rows_cap,
+                            c->d_phase_clk);
 }
 
 // Eight epilogue warps pay off for the TopK epilogue (selection work per element); the plain store of the

@@ -308,11 +308,12 @@ front_kernel(const FrontArgs a) {
         if (s_total[q] > 0 && s_gact[q] == MIX_SAE_TOPK) topk_rows += s_total[q];
         tiles += s_total[q] > 0 ? m_tiles * s_gtiles[q] : 0;
         if (s_total[q] > 0) {
-          // per feature tile, in tenths of a microsecond of SM time per k-block (measured): a single CTA needs 0.4 per
-          // 128-row tile, a pair 0.3 on both of its SMs per 256-row tile, and streaming the W_enc tile from HBM at
-          // the rate each form sustains is worth 0.8 resp. 0.9 -- the floor where a weight set has one or two row tiles
-          cost_single += (long long)max(4 * m_tiles, 8) * s_gtiles[q];
-          cost_pair += (long long)max(6 * ((m_tiles + 1) / 2), 9) * s_gtiles[q];
+          // per feature tile, in units of 1/40 of the time the W_enc tile takes to stream from HBM (measured on one
+          // weight set with 64 ... 1024 rows): single CTAs stream at the full rate for one row tile, and from two row
+          // tiles on every further tile costs 25 -- each of them fetches the W_enc tile again, from L2; a pair costs 46
+          // per 256-row tile whether its second half has rows or not, streaming at a slightly lower rate
+          cost_single += (long long)(m_tiles == 1 ? 40 : 25 * m_tiles) * s_gtiles[q];
+          cost_pair += (long long)(46 * ((m_tiles + 1) / 2)) * s_gtiles[q];
         }
       }
       s_base[n_groups] = mt * kTileM;
@@ -330,9 +331,9 @@ front_kernel(const FrontArgs a) {
         a.rs->total_tiles = tiles;
         a.rs->n_topk_rows = topk_rows;
         a.rs->n_delta_rows = s_total[n_groups];
-        // Pairs win where the tensor pipe (and the shared-memory fill behind it) is the limit -- weight sets with four or
-        // more row tiles -- and lose where the stream of W_enc is (fewer W_enc bytes in flight per SM) or where half of
-        // every pair would repeat the other half's work (a single row tile).
+        // Pairs win where a weight set has an even number of row tiles (two tiles share one fetch of W_enc, and the
+        // pair's instruction fills less shared memory per flop) and lose where half of a pair would repeat the other
+        // half's work: one row tile, or three.
         a.rs->use_pair = a.pair_mode == 2 ? (cost_pair < cost_single) : a.pair_mode;
         if (a.n_flagged) *a.n_flagged = 0;       // fallback-selection flags of the fused TopK path start clear every call
         // graph-conditional form: the rest of the SAE chain sits in the body of an IF node that runs only when a row needs it

@@ -428,7 +428,8 @@ struct TailArgs {
 
 struct RowShared {
   SelShared sel;
-  unsigned keys[kCandMax];  // a TopK row's candidate keys (the radix passes run on shared memory)
+  __align__(16) unsigned keys[kCandMax];  // a TopK row's candidate keys (the radix passes run on shared memory)
+  GroupEntry grp[kMaxGroups];             // the weight-set table, fetched once per CTA
   float coef[kDecList];
   int feat[kDecList];
   int eidx[kMaxEdits];
@@ -443,12 +444,16 @@ struct RowShared {
 // Row role.  Per row, the dependent round trips are: the row's record; then -- requested together -- the edit
 // list, the candidate keys (into shared memory: the selection passes never go back to global memory) and the
 // tiles' 9th values; then the winners' feature ids; then the gather.  (Prefetching the edited decoder rows into
-// L2 while the selection runs was tried: one 128-byte line per lane makes 32 memory transactions per warp
-// instruction, and the 1024 prefetches of a row cost more -- 3 us -- than the latency they hid.)
+// L2 while the selection runs was tried twice: line by line, one 128-byte line per lane, the 1024 prefetches of a
+// row cost more issue time -- 3 us -- than the latency they hid; one bulk prefetch per decoder row made the
+// staging step 1.5 us slower and the gather no faster.)
 __device__ void tail_rows(const TailArgs& a, RowShared& sh, int n_groups) {
   const int tid = threadIdx.x;
   const int d = a.d, nvec = d >> 3;
   // the call's SAE rows, numbered through the weight sets without the padding rows of their last tiles
+  constexpr int kGrpVecs = (int)(sizeof(GroupEntry) / sizeof(uint4));
+  if (tid >= 32 && tid < 32 + n_groups * kGrpVecs)
+    reinterpret_cast<uint4*>(sh.grp)[tid - 32] = reinterpret_cast<const uint4*>(a.groups)[tid - 32];
   if (tid == 0) {
     int cum = 0;
     for (int g = 0; g < n_groups; ++g) {
@@ -470,7 +475,7 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh, int n_groups) {
     const int t = rec.t;
     if (t < 0) continue;                               // padding row of a tile (uniform across the CTA, like every branch below)
     // (the weight-set entry field by field, not as a struct held in registers across the whole row)
-    const GroupEntry* gp = a.groups + (rec.group_flags & kRecGroupMask);
+    const GroupEntry* gp = sh.grp + (rec.group_flags & kRecGroupMask);
     const int act = (rec.group_flags >> kRecActShift) & 3;
     const bool add_error = (rec.group_flags & kRecAddError) != 0;
     const bool topk = act == MIX_SAE_TOPK;
@@ -478,36 +483,39 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh, int n_groups) {
     if (!topk && add_error && a.out_n_active == nullptr) continue;     // the delta role's row, and nobody wants its active count
     const int slot = rec.slot, n_edit = rec.n_edit;
     const bool from_cand = topk && a.mode == kTailCand;
+    const __nv_bfloat16* W_dec = rec.W_dec;
+    uint4* hrow = reinterpret_cast<uint4*>(a.hidden + (size_t)t * d);
     // ---- everything the record alone gives the address of, requested together
     if (tid < n_edit) {
-      sh.eidx[tid] = a.edit_idx[slot * a.r_max + tid];
+      const int j = a.edit_idx[slot * a.r_max + tid];
+      sh.eidx[tid] = j;
       sh.enew[tid] = a.edit_mode[slot * a.r_max + tid] == MIX_EDIT_CLAMP ? a.edit_val[slot * a.r_max + tid] : 0.f;
       sh.ef[tid] = 0.f;
     }
     const int S = (int)gp->d_sae, k = gp->k;
-    const __nv_bfloat16* W_dec = rec.W_dec;
     const float* z = a.Z + (size_t)p * a.ldz;
-    uint4* hrow = reinterpret_cast<uint4*>(a.hidden + (size_t)t * d);
     const int n_tiles = S / kTileN, n_cand = n_tiles * kCandPerTile;
     unsigned ninth_max = 0u;                           // largest key among this thread's share of the tiles' 9th values
     unsigned kmin = 0xffffffffu, kmax = 0u;            // range of this thread's share of the candidate keys
     if (from_cand && n_cand >= k) {
-      const float* cv = a.cand_val + (size_t)p * a.cand_tiles * kCandPerTile;
-      for (int i0 = tid; i0 < n_cand; i0 += 8 * kTailThreads) {
-        float v[8];
+      // (16-byte pieces, four in flight per thread: 4096 candidates are one round trip)
+      const float4* cv = reinterpret_cast<const float4*>(a.cand_val + (size_t)p * a.cand_tiles * kCandPerTile);
+      const int n_vec = n_cand >> 2;
+      for (int i0 = tid; i0 < n_vec; i0 += 4 * kTailThreads) {
+        float4 v[4];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < 4; ++u) {
           const int i = i0 + u * kTailThreads;
-          v[u] = i < n_cand ? cv[i] : 0.f;
+          v[u] = i < n_vec ? cv[i] : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < 4; ++u) {
           const int i = i0 + u * kTailThreads;
-          if (i < n_cand) {
-            const unsigned key = f2key(v[u]);
-            sh.keys[i] = key;
-            kmin = min(kmin, key);
-            kmax = max(kmax, key);
+          if (i < n_vec) {
+            const uint4 key = make_uint4(f2key(v[u].x), f2key(v[u].y), f2key(v[u].z), f2key(v[u].w));
+            reinterpret_cast<uint4*>(sh.keys)[i] = key;
+            kmin = min(min(kmin, key.x), min(min(key.y, key.z), key.w));
+            kmax = max(max(kmax, key.x), max(max(key.y, key.z), key.w));
           }
         }
       }
