@@ -720,29 +720,54 @@ __global__ void fold_bias_kernel(const __nv_bfloat16* __restrict__ W_enc, const 
   if (lane == 0) b_eff[j] = b_enc[j] - acc;
 }
 
-// Census of the batch's multi-class probe rows (2..32 classes; gates are not looked at): one CTA per 128-row
-// tile counts them and, if there are any, appends the tile to a list; the last CTA to finish publishes the totals
-// and the choice between the two probe kernels, and puts the working counters back to zero for the next call.
+// Census of the batch's multi-class probe rows (2..32 classes; gates are not looked at): a CTA takes 8 tiles of
+// 128 rows, one per warp (four rows per lane, their loads in flight together), counts each tile's such rows and
+// appends the tiles that have any to a list -- one reservation per CTA, so the shared counters see two additions
+// per 1024 rows; the last CTA to finish publishes the totals and the choice between the two probe kernels, and
+// puts the working counters back to zero for the next call.
 // The tensor-core kernel streams whole tiles, the 16-row kernel reaches 38 % of the HBM rate against its 80 %:
 // it takes the call when the listed tiles are, on average, at least half full of such rows.
-__global__ void __launch_bounds__(kTileM)
+constexpr int kCensusWarps = 8;
+__global__ void __launch_bounds__(kCensusWarps * 32)
 mc_census_kernel(const int* __restrict__ token_slot, const int* __restrict__ n_live_p, int T,
                  const AppEntry* __restrict__ apps, int n_slots, McCensus* __restrict__ census, int* __restrict__ tiles) {
+  __shared__ int s_cnt[kCensusWarps];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int live = min(T, __ldg(n_live_p));
-  const int t = blockIdx.x * kTileM + threadIdx.x;
-  int hit = 0;
-  if (t < live) {
-    const int s = __ldg(token_slot + t);
-    if (s >= 0 && s < n_slots) {
-      const int4 q0 = __ldg(reinterpret_cast<const int4*>(apps + s));    // valid, kind, n_classes, act
-      hit = q0.x && (q0.y & kKindMask) == MIX_PROBE && q0.z > 1 && q0.z <= 32;
-    }
+  const int tile = blockIdx.x * kCensusWarps + warp;
+  int slot[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int t = tile * kTileM + i * 32 + lane;
+    slot[i] = t < live ? __ldg(token_slot + t) : -1;
   }
-  const int cnt = __syncthreads_count(hit);
+  int4 q[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    q[i] = make_int4(0, 0, 0, 0);
+    if (slot[i] >= 0 && slot[i] < n_slots) q[i] = __ldg(reinterpret_cast<const int4*>(apps + slot[i]));    // valid, kind, n_classes, act
+  }
+  int cnt = 0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const bool hit = q[i].x && (q[i].y & kKindMask) == MIX_PROBE && q[i].z > 1 && q[i].z <= 32;
+    cnt += __popc(__ballot_sync(0xffffffffu, hit));
+  }
+  if (lane == 0) s_cnt[warp] = cnt;
+  __syncthreads();
   if (threadIdx.x == 0) {
-    if (cnt > 0) {
-      tiles[atomicAdd(&census->w_tiles, 1)] = blockIdx.x;
-      atomicAdd(&census->w_rows, cnt);
+    int n_local = 0, rows = 0;
+#pragma unroll
+    for (int w = 0; w < kCensusWarps; ++w) {
+      n_local += s_cnt[w] > 0;
+      rows += s_cnt[w];
+    }
+    if (n_local > 0) {
+      int pos = atomicAdd(&census->w_tiles, n_local);
+#pragma unroll
+      for (int w = 0; w < kCensusWarps; ++w)
+        if (s_cnt[w] > 0) tiles[pos++] = blockIdx.x * kCensusWarps + w;
+      atomicAdd(&census->w_rows, rows);
     }
     __threadfence();
     if (atomicAdd(&census->w_done, 1) == (int)gridDim.x - 1) {
@@ -765,7 +790,8 @@ bool has_multiclass_stage(const Ctx* c) {
 }
 
 cudaError_t launch_mc_census(const Ctx* c, int T, cudaStream_t s) {
-  mc_census_kernel<<<(c->cfg.T_max + kTileM - 1) / kTileM, kTileM, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps,
+  const int rows_per_cta = kCensusWarps * kTileM;
+  mc_census_kernel<<<(c->cfg.T_max + rows_per_cta - 1) / rows_per_cta, kCensusWarps * 32, 0, s>>>(c->d_token_slot, c->d_n_live, T, c->d_apps,
                                                                            c->cfg.n_slots_max, c->d_mc_census, c->d_mc_tiles);
   return cudaGetLastError();
 }
