@@ -706,12 +706,15 @@ struct DeltaShared {
   const float* theta[kDlRows];
 };
 
-// One work item of the delta role: row group `item / n_col_slices`, column slice `item % n_col_slices`.
+// One work item of the delta role: row group `item / n_cg`, column slices `item % n_cg`, `+ n_cg`, ... (n_cg: into how
+// many items a row group's columns are split this call -- as many as still fit the grid in one wave, because the
+// steps in front of the gather are repeated by every item of a row group).
 // Dependent round trips: the rows' records (which carry the decoder and threshold pointers); the edit lists of
-// their slots; the pre-activations and thresholds of the edited features; the decoder rows; the rows themselves.
-__device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int item, int n_rows) {
+// their slots; the pre-activations and thresholds of the edited features; then, per slice, the decoder rows and
+// the rows themselves.
+__device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int item, int n_rows, int n_cg) {
   const int tid = threadIdx.x;
-  const int rg = item / a.n_col_slices, cs = item - rg * a.n_col_slices;
+  const int rg = item / n_cg, cg = item - rg * n_cg;
   const int p0 = rg * kDlRows;
   __syncthreads();                                       // the shared lists of the previous item are free
   const bool stamp = item == 0 && tid == 0;
@@ -736,8 +739,6 @@ __device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int item, int n_r
   phase_stamp(a.clk, 23, stamp);
   if (!any) return;
   const int d = a.d;
-  const int v = cs * kTailThreads + tid;                 // this thread's 16-byte column vector
-  const bool in_cols = v < (d >> 3);
   // entries: the edit lists of the distinct slots, one after the other (the coefficient of a row of another slot is zero)
   int n_entries = 0;                                    // CTA-uniform
   for (int r = 0; r < kDlRows; ++r) {
@@ -787,7 +788,9 @@ __device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int item, int n_r
   }
   __syncthreads();
   phase_stamp(a.clk, 24, stamp);
-  if (!in_cols) return;
+  for (int cs = cg; cs < a.n_col_slices; cs += n_cg) {
+  const int v = cs * kTailThreads + tid;                 // this thread's 16-byte column vector
+  if (v >= (d >> 3)) break;
   float acc[kDlRows][8];
 #pragma unroll
   for (int r = 0; r < kDlRows; ++r)
@@ -825,6 +828,7 @@ __device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int item, int n_r
     }
     reinterpret_cast<uint4*>(a.hidden + (size_t)sh.t[r] * d)[v] = o;
   }
+  }
 }
 
 // A fixed grid of CTAs (a few per SM, all resident at once or nearly) walks the work of the call: first the
@@ -847,8 +851,10 @@ tail_kernel(const TailArgs a) {
   const int n_rows = a.rs->n_panel_rows, n_delta = a.rs->n_delta_rows, n_sae = a.rs->n_sae_rows;
   if (a.mode == kTailFallback || n_sae > n_delta || (a.out_n_active != nullptr && n_sae > 0)) tail_rows(a, s_row, a.n_groups);
   if (a.mode != kTailFallback && n_delta > 0) {
-    const int n_items = (n_rows / kDlRows) * a.n_col_slices;
-    for (int item = blockIdx.x; item < n_items; item += gridDim.x) tail_delta(a, s_delta, item, n_rows);
+    const int n_rg = n_rows / kDlRows;
+    const int n_cg = min(a.n_col_slices, max(1, (int)gridDim.x / n_rg));
+    const int n_items = n_rg * n_cg;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x) tail_delta(a, s_delta, item, n_rows, n_cg);
   }
   phase_stamp(a.clk, 15, blockIdx.x == 0 && threadIdx.x == 0 && a.mode != kTailFallback);
 }
