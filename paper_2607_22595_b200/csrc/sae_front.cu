@@ -32,15 +32,15 @@ __device__ __forceinline__ void pack_row_bf16(const __nv_bfloat16* __restrict__ 
     return;
   }
   const uint4* src = reinterpret_cast<const uint4*>(hidden + (size_t)t * d);
-  int i = lane;
-  for (; i + 224 < nvec; i += 256) {                     // eight loads in flight per lane
+  for (int i = lane; i < nvec; i += 256) {               // eight loads in flight per lane, the ragged end included
     uint4 q[8];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) q[u] = __ldg(src + i + 32 * u);
+    for (int u = 0; u < 8; ++u)
+      if (i + 32 * u < nvec) q[u] = __ldg(src + i + 32 * u);
 #pragma unroll
-    for (int u = 0; u < 8; ++u) dst[i + 32 * u] = q[u];
+    for (int u = 0; u < 8; ++u)
+      if (i + 32 * u < nvec) dst[i + 32 * u] = q[u];
   }
-  for (; i < nvec; i += 32) dst[i] = __ldg(src + i);
 }
 
 // 8-bit encoder: the row goes into the panel as E4M3 codes with a power-of-two row scale.
