@@ -7,11 +7,14 @@
 // a 4-stage ring of 128-byte-swizzled shared memory), warp 1 = MMA issuer (tcgen05.mma
 // 128x256x16, fp32 accumulators in tensor memory, double buffered so the epilogue of one tile
 // overlaps the main loop of the next), warps 2..9 = epilogue, two per tensor-memory lane quarter
-// with 128 columns of the tile each (tcgen05.ld, + bias, then either
+// with 128 columns of the tile each (tcgen05.ld, + bias -- the warp's columns of it copied to shared
+// memory before the accumulator is waited for -- then either
 // the fp32 pre-activations to the Z scratch, or -- for TopK weight sets -- only the tile's 8
-// largest values per row plus its 9th, which the merge step turns into the exact TopK; the two
+// largest values per row plus its 9th, which the tail kernel turns into the exact TopK; the two
 // warps of a quarter merge their lists through shared memory).
-// No TMA multicast and no clusters.  Every wait is bounded: on expiry the CTA raises
+// A second form (kPair) runs on clusters of two CTAs that share a 256-row tile through
+// tcgen05.mma.cta_group::2; which form works on a call is decided on the device (see TcCfg).
+// No TMA multicast in either form.  Every wait is bounded: on expiry the CTA raises
 // MIX_STATUS_WAIT_TIMEOUT, lets its copies land, frees its tensor memory and returns.
 //
 // 8-bit encoder (kEnc != 0): W_enc is E4M3 codes with one fp32 scale per feature, and the contraction is
@@ -334,6 +337,7 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
+      phase_stamp(clk, 28, stamp);          // the last copy of this CTA has been issued
     }
   } else if (warp == 1) {
     if (lane == 0 && leader) {
@@ -559,7 +563,6 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
 
   tc_fence_before();
   __syncthreads();
-  phase_stamp(clk, 28, stamp);
   if (sh->abort_flag) {
     // give copies that are still in flight time to land before shared memory is released
     const long long t0 = clock64();
