@@ -917,6 +917,10 @@ def run_mix(args, rank, world, local_rank):
                 ex["error"] = repr(e)
             line["roofline"]["targets"] = targets
             line["extras"] = ex
+    # the per-kernel detail first, the contract's own blocks last: whoever keeps only the end of a long line
+    # keeps `roofline` (with `targets`) and `cpu_baseline`
+    tail_keys = [k for k in ("clocks", "e2e", "gpu_launches", "cpu_baseline", "roofline") if k in line]
+    line = {**{k: v for k, v in line.items() if k not in tail_keys}, **{k: line[k] for k in tail_keys}}
     print(json.dumps(line), flush=True)
 
 
@@ -981,7 +985,13 @@ def collect_targets(targets, ex, w, hiddens, scores, peaks, mixlib, args):
                               "t_call_ms": r4["t_call_ms"], "empty_replay_us": None if r4["empty_replay_ms"] is None else r4["empty_replay_ms"] * 1e3,
                               "n_live_covered": r4["n_live_covered"], "status_or": r4["status_or"]}
     torch.cuda.empty_cache()
-    ex["multiclass_probes"] = extras_multiclass(peaks, mixlib)
+    mc = extras_multiclass(peaks, mixlib)
+    ex["multiclass_probes"] = mc
+    targets["multiclass_probes"] = {
+        "what": "whole call replayed from a graph, and the tensor-core probe kernel alone, as fractions of the HBM peak on hooked bytes",
+        **{k: {"call_frac_hbm": round(v["graph_replay"]["frac_hbm_peak"], 3),
+               "kernel_frac_hbm": round(v["probe_tc_kernel_alone"]["frac_hbm_peak"], 3), "status": v["status"]}
+           for k, v in mc.items()}}
     ex["decode_variants"] = extras_decode_variants(w, hiddens[:256], scores[:256], mixlib)
 
 
