@@ -23,7 +23,7 @@ constexpr int kMaxK = 1024;
 constexpr int kMaxEdits = 64;
 constexpr int kTauSlots = 128;      // per packed row: slots of the running lower bound on the row's k-th largest pre-activation (k <= 128)
 constexpr int kCandPerTile = 8;     // TopK candidates the encode epilogue keeps per (row, feature tile)
-constexpr int kCandMax = 4096;      // candidates per row the merge step can sort in shared memory
+constexpr int kCandMax = 4096;      // candidates per row the tail kernel can stage in shared memory
 
 struct __align__(16) AppEntry {
   int valid;          // written last by registration; 0 = slot is pass-through
@@ -199,8 +199,9 @@ struct Ctx {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-// Which launches use programmatic dependent launch: bit 0 pack, bit 1 the full encode pass, bit 2 everything after
-// it (merge ... decode_delta), bit 3 the one-CTA-per-row probe / steering kernel of a context without weight sets.
+// Which launches use programmatic dependent launch: bit 0 unused (the pack step is part of the front kernel now), bit 1
+// the full encode pass, bit 2 everything after it (tail, flagged-tile encode, flagged tail, edit-only kernels), bit 3
+// the one-CTA-per-row probe / steering kernel of a context without weight sets.
 // MIX_PDL_MASK in the environment overrides the default (A/B timing); read once.
 enum { kPdlPack = 1, kPdlEncode = 2, kPdlTail = 4, kPdlHook = 8 };
 int pdl_mask();

@@ -174,7 +174,7 @@ __device__ __forceinline__ Tile decode_pair_tile(const TcShared& sh, int n_group
 }
 
 // mode 0: every tile; TopK weight sets emit candidates, the others write Z.
-// mode 1: only row tiles flagged by the merge step (TopK sets), written to Z for the exact
+// mode 1: only row tiles flagged by the tail kernel (TopK sets), written to Z for the exact
 //         fallback selection; returns at once when nothing is flagged.
 __device__ __forceinline__ bool tile_wanted(const Tile& t, const GroupEntry* __restrict__ groups, int mode,
                                             const int* __restrict__ mtile_flag) {
