@@ -10,7 +10,7 @@ ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libmix.so")
 
-SOURCES = ["mix_api.cu", "route_probe_steer.cu", "probe_tc.cu", "sae_front.cu", "sae_select_decode.cu", "sae_encode_tc.cu", "sae_tail.cu",
+SOURCES = ["mix_api.cu", "route_probe_steer.cu", "probe_tc.cu", "sae_front.cu", "sae_simt_edit_only.cu", "sae_encode_tc.cu", "sae_tail.cu",
            "sae_static.cu"]
 
 
