@@ -423,11 +423,12 @@ int mix_debug_workspace(mix_ctx* ctx, const int** panel_rows, const float** z, l
 
 /* Profiling aid (no counterpart in the paper).  A context created while MIX_PHASE_CLOCKS=1 is set in the
    environment keeps 32 words in which the first CTA of the SAE chain's front, encode and tail kernels stamps
-   the GPU's nanosecond timer (words 0, 7, 8, 15, 26..29) or its SM's cycle counter (the others) at its phase
+   the GPU's nanosecond timer (words 0, 7, 8, 15, 26..31) or its SM's cycle counter (the others) at its phase
    boundaries (0..4 front: start, rows classified, routing scanned, positions found, rows packed; 7..15 tail:
    launched, predecessor done, row 0 read, candidates narrowed, sorted, TopK known, coefficients known, row
    written, CTA done; 16..25 steps inside the tail's selection and its delta role; 26..29 single-CTA encode:
-   predecessor done, tensor memory allocated, last copy issued, CTA done).  out32: HOST array of 32 words,
+   predecessor done, tensor memory allocated, last copy issued, CTA done; 30, 31 the end of the LAST CTA of the
+   tail's main and fallback launches).  out32: HOST array of 32 words,
    zeros when the context was created without the variable.  Synchronises the device. */
 int mix_debug_phase_clocks(mix_ctx* ctx, unsigned long long* out32);
 

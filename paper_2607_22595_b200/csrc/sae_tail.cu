@@ -831,6 +831,16 @@ __device__ void tail_delta(const TailArgs& a, DeltaShared& sh, int item, int n_r
   }
 }
 
+// Profiling aid: the time the LAST CTA of a launch ended (slot 30: main launch, 31: fallback launch), as the
+// largest nanosecond-timer value any CTA saw at its end.
+__device__ __forceinline__ void stamp_launch_end(unsigned long long* clk, int mode) {
+  if (clk != nullptr && threadIdx.x == 0) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    atomicMax(clk + (mode == kTailFallback ? 31 : 30), t);
+  }
+}
+
 // A fixed grid of CTAs (a few per SM, all resident at once or nearly) walks the work of the call: first the
 // packed rows that need the row role, then the row groups x column slices of the delta role.  Both lists are as
 // long as THIS call's routing made them, not as long as the context's capacity, and a role with no rows this
@@ -847,7 +857,10 @@ tail_kernel(const TailArgs a) {
   } s_u;
   RowShared& s_row = s_u.row;
   DeltaShared& s_delta = s_u.delta;
-  if (a.mode == kTailFallback && *a.n_flagged == 0) return;   // nothing was flagged: the usual case
+  if (a.mode == kTailFallback && *a.n_flagged == 0) {   // nothing was flagged: the usual case
+    stamp_launch_end(a.clk, a.mode);
+    return;
+  }
   const int n_rows = a.rs->n_panel_rows, n_delta = a.rs->n_delta_rows, n_sae = a.rs->n_sae_rows;
   if (a.mode == kTailFallback || n_sae > n_delta || (a.out_n_active != nullptr && n_sae > 0)) tail_rows(a, s_row, a.n_groups);
   if (a.mode != kTailFallback && n_delta > 0) {
@@ -857,6 +870,7 @@ tail_kernel(const TailArgs a) {
     for (int item = blockIdx.x; item < n_items; item += gridDim.x) tail_delta(a, s_delta, item, n_rows, n_cg);
   }
   phase_stamp(a.clk, 15, blockIdx.x == 0 && threadIdx.x == 0 && a.mode != kTailFallback);
+  stamp_launch_end(a.clk, a.mode);
 }
 
 }  // namespace
