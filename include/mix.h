@@ -408,8 +408,9 @@ int mix_bench_param_update(mix_ctx* ctx, int iters, float* us_table, float* us_n
    and run the part of the kernel that reads only library-owned tables, while the kernel in front of
    it in the stream is still running; everything the predecessor may have written is read after an
    in-kernel wait).  Bits: 1 unused (the row pack is part of the first kernel of the SAE chain),
-   2 the full SAE encode pass, 4 the kernels after it, 8 the one-CTA-per-row probe / steering kernel of a context that has no SAE weight sets
-   (T_max <= 2048).  Default 1 | 4 | 8, or the value of MIX_PDL_MASK in the environment when the
+   2 the full SAE encode pass (the kernel in front of it lets it start only when its own rows are packed),
+   4 the kernels after it, 8 the one-CTA-per-row probe / steering kernel of a context that has no SAE weight sets
+   (T_max <= 2048).  Default 1 | 2 | 4 | 8, or the value of MIX_PDL_MASK in the environment when the
    library first launches.  Process-wide; affects launches (and captures) made afterwards; meant
    for A/B measurement.  Returns the previous mask.  mask < 0 only queries. */
 int mix_set_pdl_mask(int mask);

@@ -187,7 +187,7 @@ namespace mix {
 static int g_pdl_mask = -1;        // -1: not yet read from the environment
 int pdl_mask() {
   // default: not the full encode pass -- measured, its early-resident CTAs cost config 3 about 7 us
-  if (g_pdl_mask < 0) g_pdl_mask = getenv("MIX_PDL_MASK") ? (atoi(getenv("MIX_PDL_MASK")) & 15) : (kPdlPack | kPdlTail | kPdlHook);
+  if (g_pdl_mask < 0) g_pdl_mask = getenv("MIX_PDL_MASK") ? (atoi(getenv("MIX_PDL_MASK")) & 15) : (kPdlPack | kPdlEncode | kPdlTail | kPdlHook);
   return g_pdl_mask;
 }
 }  // namespace mix

@@ -171,7 +171,6 @@ front_kernel(const FrontArgs a) {
   __shared__ const float* s_gtheta[kMaxGroups];
   __shared__ int s_wcnt[kFrontWarps][kMaxGroups + 1];
   __shared__ int s_n_panel_rows;
-  pdl_launch_dependents();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int cta = blockIdx.x;
   const bool first_cta = cta == 0;
@@ -412,6 +411,9 @@ front_kernel(const FrontArgs a) {
     atomicOr(a.status, MIX_STATUS_WAIT_TIMEOUT);
   }
   phase_stamp(a.clk, 4, first_cta && tid == 0);
+  // Only now may the encode's CTAs be scheduled (where it is launched programmatically): they take most of an SM's
+  // registers and shared memory, and resident any earlier they would crowd out the CTAs that still have rows to pack.
+  pdl_launch_dependents();
   // the last CTA to leave closes the call: both counters are zero again when the next launch starts
   __syncthreads();
   if (tid == 0) {

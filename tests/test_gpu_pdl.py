@@ -122,3 +122,61 @@ def test_request_map_composed_by_a_kernel_is_seen_by_the_next_hook():
                    status=m.get_status())
         check_parity(wh, out, check_features=False)
     m.destroy()
+
+
+def _run_sae_calls(w, n_calls, mask, flags=0):
+    """One graph: n_calls x (copy a fresh batch into `h` -> mix_apply -> copy `h` out); returns the bits of every result."""
+    mixlib = _mixlib()
+    old = mixlib.set_pdl_mask(-1)
+    mixlib.set_pdl_mask(mask)
+    try:
+        m = W.make_context(mixlib.Mix, w, flags=flags)
+        T, C = w.T_max, max(w.C_max, 1)
+        g = torch.Generator(device=DEV); g.manual_seed(5)
+        srcs = [(w.hidden.float() * (1.0 + 0.125 * i) + 0.125 * i * torch.randn(w.hidden.shape, generator=g, device=DEV)).to(torch.bfloat16)
+                for i in range(n_calls)]
+        h = w.hidden.clone()
+        scores = _canary(T, C)
+        outs = [torch.empty_like(h) for _ in range(n_calls)]
+        souts = [torch.empty_like(scores) for _ in range(n_calls)]
+        s = torch.cuda.Stream(); s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s):
+            m.apply(h, scores, stream=s)
+            scores.copy_(_canary(T, C))
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=s):
+                for i in range(n_calls):
+                    h.copy_(srcs[i])
+                    m.apply(h, scores, stream=s)
+                    outs[i].copy_(h)
+                    souts[i].copy_(scores)
+        torch.cuda.current_stream().wait_stream(s)
+        for _ in range(2):                                   # the second replay starts from the first one's device state
+            graph.replay()
+        torch.cuda.synchronize()
+        assert m.get_status() == 0
+        res = [(W.bits(o), x.cpu().numpy()) for o, x in zip(outs, souts)]
+        m.destroy()
+        return res, srcs
+    finally:
+        mixlib.set_pdl_mask(old)
+
+
+@pytest.mark.parametrize("make", ["tiny", "small_mixed"])
+def test_sae_chain_is_bit_identical_with_programmatic_launches_on_and_off(make):
+    """The SAE chain's kernels (front -> encode -> tail -> fallback pair) start early under programmatic launch and
+    wait inside; back-to-back calls in one graph reuse every workspace of the context.  Same bits either way, and
+    right against the oracle."""
+    mixlib = _mixlib()
+    w = W.make_tiny(DEV) if make == "tiny" else W.make_mixed(DEV, T=1024, d=512, d_sae=2048, R=16)
+    default = mixlib.set_pdl_mask(-1)
+    assert default & 2 and default & 4, "encode and tail are launched programmatically by default"
+    a, srcs = _run_sae_calls(w, 3, default)
+    b, _ = _run_sae_calls(w, 3, 0)
+    for i in range(3):
+        assert np.array_equal(a[i][0], b[i][0]), "call %d" % i
+        assert np.array_equal(a[i][1].view(np.uint32), b[i][1].view(np.uint32)), "call %d" % i
+    wh = W.host(w)
+    wh.hidden = W.bits(srcs[2])
+    out = dict(hidden=a[2][0], scores=a[2][1], topk_idx=None, topk_val=None, n_active=None, status=0)
+    check_parity(wh, out, check_features=False)
