@@ -382,10 +382,10 @@ int mix_launches_per_apply(const mix_ctx* ctx);
    its first kernel and events[i] after its i-th kernel, on the call's stream; the array is
    copied.  Kernel order: [probe_decide,] probe_steer, [probe_multiclass: only if T_max > 2048 and C_max > 1;
    probe_decide before and probe_tc after it if also n_groups_max == 0,]
-   front (routing + row pack), encode on single CTAs, encode on CTA pairs (the front kernel picks one of
-   the two per call from the routing result -- pairs when the weight sets average well over one 128-row
-   tile each -- and the other returns at once; a stage event is recorded for both even where one is
-   never launched), tail (selection, edits, decode, write-back), encode (row tiles flagged for the exact
+   front (routing + row pack), encode on single CTAs, encode on CTA pairs (the front kernel deals the
+   call's weight sets between the two from the routing result -- sets with an even number of 128-row
+   tiles to the pairs, when that pays -- and a kernel without a set returns at once; a stage event is
+   recorded for both even where one is never launched), tail (selection, edits, decode, write-back), encode (row tiles flagged for the exact
    fallback selection), tail (the flagged rows); with MIX_FLAG_ENCODE_SIMT the SAE part is front, encode,
    tail; with MIX_FLAG_SAE_EDIT_ONLY an edit_only and an edit_only_delta
    kernel come last. */

@@ -104,8 +104,8 @@ struct RouteState {
   int total_tiles;                  // encode tiles over all groups
   int n_topk_rows;                  // SAE rows whose weight set is TopK
   int n_delta_rows;                 // ReLU / JumpReLU rows that keep the error term and have edits (the tail kernel's delta role)
-  int use_pair;                     // this call's encode runs on CTA pairs (256-row tiles) rather than on single CTAs
-  int pad_;
+  int use_pair;                     // some weight set of this call is encoded by CTA pairs (256-row tiles)
+  int pair_mask;                    // bit g: weight set g is the pair kernel's this call, else the single-CTA kernel's
   int group_count[kMaxGroups];      // M_g
   int group_mtile0[kMaxGroups + 1]; // first m-tile of group g in the panel
   int group_tile0[kMaxGroups + 1];  // first linear encode tile of group g

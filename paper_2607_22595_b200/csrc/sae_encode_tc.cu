@@ -78,9 +78,11 @@ struct __align__(8) TcShared {
   volatile int abort_flag;
   long long wait_cycles;      // cap of every bounded wait in this launch
   RouteState rs;
-  // CTA pairs: first row-tile pair / first pair-tile of each weight set, totals
-  short pair0[kMaxGroups + 1];
-  int ptile0[kMaxGroups + 1];
+  // The weight sets of this call that are THIS kernel's (single CTAs or pairs, as the front kernel dealt them; all
+  // of them in the pass over flagged row tiles), numbered through: first unit -- a 128-row tile, or a pair of
+  // them -- and first tile of each set, totals in entry [n_groups]; sets of the other kernel have no units here
+  short unit0[kMaxGroups + 1];
+  int utile0[kMaxGroups + 1];
 };
 static_assert(sizeof(TcShared) <= 1024, "TcShared must fit the space reserved for it");
 
@@ -101,75 +103,55 @@ struct Tile {
   int m_tile_peer;      // CTA pairs: the row tile the other CTA of the pair works on (the same one when the weight set has an odd tile left over)
 };
 
-// Number of feature tiles per row tile if it is the same for every weight set that has rows (the usual
-// case: one SAE width per context), else 0.
-__device__ __forceinline__ int uniform_feature_tiles(const RouteState& rs, int n_groups) {
+// Number of feature tiles per unit if it is the same for every weight set of this kernel that has rows (the
+// usual case: one SAE width per context), else 0.
+__device__ __forceinline__ int uniform_feature_tiles(const TcShared& sh, int n_groups) {
   int nt = -1;
   for (int g = 0; g < n_groups; ++g) {
-    const int mt = rs.group_mtile0[g + 1] - rs.group_mtile0[g];
-    if (mt == 0) continue;
-    const int nt_g = (rs.group_tile0[g + 1] - rs.group_tile0[g]) / mt;
+    const int units = sh.unit0[g + 1] - sh.unit0[g];
+    if (units == 0) continue;
+    const int nt_g = (sh.utile0[g + 1] - sh.utile0[g]) / units;
     if (nt >= 0 && nt_g != nt) return 0;
     nt = nt_g;
   }
-  return nt > 0 && nt * rs.n_mtiles == rs.total_tiles ? nt : 0;
+  return nt > 0 ? nt : 0;
 }
 
-// Linear tile id -> (weight set, feature tile, row tile).  With one SAE width the order is feature tile by
-// feature tile over ALL row tiles of the panel, so every row sees its first feature tiles finished early in
-// the launch (the TopK epilogue's running bound needs that); otherwise weight set by weight set.
-__device__ __forceinline__ Tile decode_tile(const RouteState& rs, const GroupEntry* groups, int n_groups, int tile,
-                                            int uniform_nt) {
-  Tile t;
-  int g = 0;
-  if (uniform_nt > 0) {
-    t.n_tile = tile / rs.n_mtiles;
-    t.m_tile_global = tile - t.n_tile * rs.n_mtiles;
-    while (g + 1 < n_groups && t.m_tile_global >= rs.group_mtile0[g + 1]) ++g;
-    t.group = g;
-    t.rows_valid = min(kTileM, rs.group_count[g] - (t.m_tile_global - rs.group_mtile0[g]) * kTileM);
-    t.m_tile_peer = t.m_tile_global;
-    return t;
-  }
-  while (g + 1 < n_groups && tile >= rs.group_tile0[g + 1]) ++g;
-  const int local = tile - rs.group_tile0[g];
-  const int count = rs.group_count[g];
-  const int mt = (count + kTileM - 1) / kTileM;
-  t.group = g;
-  t.n_tile = local / mt;
-  const int m_local = local - t.n_tile * mt;
-  t.m_tile_global = rs.group_mtile0[g] + m_local;
-  t.rows_valid = min(kTileM, count - m_local * kTileM);
-  t.m_tile_peer = t.m_tile_global;
-  return t;
-}
-
-// The same for CTA pairs: linear pair-tile id -> (weight set, feature tile, pair of row tiles) and, for the CTA of
-// rank `rank`, its own row tile.  A weight set with an odd number of row tiles leaves its last pair half empty:
-// the CTA without a tile of its own repeats the other one's loads and keeps nothing (rows_valid = 0).
-__device__ __forceinline__ Tile decode_pair_tile(const TcShared& sh, int n_groups, int tile, int uniform_nt, int rank) {
+// Linear tile id of this kernel -> (weight set, feature tile, unit of the set) and, for the CTA of rank `rank` of a
+// pair, its own row tile.  With one SAE width the order is feature tile by feature tile over ALL units, so every
+// row sees its first feature tiles finished early in the launch (the TopK epilogue's running bound needs that);
+// otherwise weight set by weight set.  A weight set with an odd number of row tiles leaves its last pair half
+// empty: the CTA without a tile of its own repeats the other one's loads and keeps nothing (rows_valid = 0).
+template <bool kPair>
+__device__ __forceinline__ Tile decode_tile(const TcShared& sh, int n_groups, int tile, int uniform_nt, int rank) {
   const RouteState& rs = sh.rs;
   Tile t;
-  int g = 0, pl;
+  int g = 0, ul;
   if (uniform_nt > 0) {
-    const int n_pairs = sh.pair0[n_groups];
-    t.n_tile = tile / n_pairs;
-    const int pr = tile - t.n_tile * n_pairs;
-    while (g + 1 < n_groups && pr >= sh.pair0[g + 1]) ++g;
-    pl = pr - sh.pair0[g];
+    const int n_units = sh.unit0[n_groups];
+    t.n_tile = tile / n_units;
+    const int u = tile - t.n_tile * n_units;
+    while (g + 1 < n_groups && u >= sh.unit0[g + 1]) ++g;
+    ul = u - sh.unit0[g];
   } else {
-    while (g + 1 < n_groups && tile >= sh.ptile0[g + 1]) ++g;
-    const int local = tile - sh.ptile0[g];
-    const int mp = sh.pair0[g + 1] - sh.pair0[g];
-    t.n_tile = local / mp;
-    pl = local - t.n_tile * mp;
+    while (g + 1 < n_groups && tile >= sh.utile0[g + 1]) ++g;
+    const int local = tile - sh.utile0[g];
+    const int units = sh.unit0[g + 1] - sh.unit0[g];
+    t.n_tile = local / units;
+    ul = local - t.n_tile * units;
   }
-  const int mt = rs.group_mtile0[g + 1] - rs.group_mtile0[g];
-  const int m_own = 2 * pl + rank, m_peer = 2 * pl + (1 - rank);
   t.group = g;
-  t.m_tile_global = rs.group_mtile0[g] + min(m_own, mt - 1);
-  t.m_tile_peer = rs.group_mtile0[g] + min(m_peer, mt - 1);
-  t.rows_valid = m_own < mt ? min(kTileM, rs.group_count[g] - m_own * kTileM) : 0;
+  if (kPair) {
+    const int mt = rs.group_mtile0[g + 1] - rs.group_mtile0[g];
+    const int m_own = 2 * ul + rank, m_peer = 2 * ul + (1 - rank);
+    t.m_tile_global = rs.group_mtile0[g] + min(m_own, mt - 1);
+    t.m_tile_peer = rs.group_mtile0[g] + min(m_peer, mt - 1);
+    t.rows_valid = m_own < mt ? min(kTileM, rs.group_count[g] - m_own * kTileM) : 0;
+  } else {
+    t.m_tile_global = rs.group_mtile0[g] + ul;
+    t.m_tile_peer = t.m_tile_global;
+    t.rows_valid = min(kTileM, rs.group_count[g] - ul * kTileM);
+  }
   return t;
 }
 
@@ -240,21 +222,23 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
 
   for (int i = threadIdx.x; i < (int)(sizeof(RouteState) / sizeof(int)); i += kTcThreads)
     reinterpret_cast<int*>(&sh->rs)[i] = reinterpret_cast<const int*>(rs_g)[i];
-  if (kPair) __syncthreads();
+  __syncthreads();
   if (threadIdx.x == 0) {
-    if (kPair) {      // pairs of row tiles per weight set
-      int np = 0, pt = 0;
+    {      // this kernel's weight sets: units (row tiles, or pairs of them) and tiles, numbered through
+      int nu = 0, ut = 0;
       for (int g = 0; g < n_groups; ++g) {
         const int mt = sh->rs.group_mtile0[g + 1] - sh->rs.group_mtile0[g];
         const int nt = mt > 0 ? (sh->rs.group_tile0[g + 1] - sh->rs.group_tile0[g]) / mt : 0;
-        sh->pair0[g] = (short)np;
-        sh->ptile0[g] = pt;
-        np += (mt + 1) / 2;
-        pt += ((mt + 1) / 2) * nt;
+        const bool mine = mode != 0 || (((sh->rs.pair_mask >> g) & 1) != 0) == kPair;
+        const int units = !mine ? 0 : (kPair ? (mt + 1) / 2 : mt);
+        sh->unit0[g] = (short)nu;
+        sh->utile0[g] = ut;
+        nu += units;
+        ut += units * nt;
       }
       for (int g = n_groups; g <= kMaxGroups; ++g) {
-        sh->pair0[g] = (short)np;
-        sh->ptile0[g] = pt;
+        sh->unit0[g] = (short)nu;
+        sh->utile0[g] = ut;
       }
     }
     for (int s = 0; s < kStages; ++s) {
@@ -272,10 +256,11 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
-  if (sh->rs.total_tiles == 0) return;     // nothing routed to any SAE: no tensor memory is taken (both CTAs of a pair see the same)
-  // the full pass has two kernels, single CTAs and CTA pairs; the front kernel chose one for this call
-  if (mode == 0 && (sh->rs.use_pair != 0) != kPair) return;
-  const int total_tiles = kPair ? sh->ptile0[n_groups] : sh->rs.total_tiles;
+  // the full pass has two kernels, single CTAs and CTA pairs, and the front kernel dealt this call's weight sets
+  // between them: nothing routed to any SAE, or no set for this kernel -- no tensor memory is taken (both CTAs
+  // of a pair see the same)
+  const int total_tiles = sh->utile0[n_groups];
+  if (total_tiles == 0) return;
 
   if (warp == 1) {
     if (kPair) tmem_alloc_pair(smem_u32(&sh->tmem_base), kTmemCols);
@@ -288,11 +273,9 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
   const unsigned tmem_base = sh->tmem_base;
   phase_stamp(clk, 27, stamp);
   // (the interleaved order serves the TopK epilogue's running bound; without TopK rows the plain order is a little faster)
-  const int uniform_nt = sh->rs.n_topk_rows > 0 ? uniform_feature_tiles(sh->rs, n_groups) : 0;
+  const int uniform_nt = sh->rs.n_topk_rows > 0 ? uniform_feature_tiles(*sh, n_groups) : 0;
   const int num_kb = d / kBlockK;
-  auto tile_of = [&](int tile) {
-    return kPair ? decode_pair_tile(*sh, n_groups, tile, uniform_nt, rank) : decode_tile(sh->rs, groups, n_groups, tile, uniform_nt);
-  };
+  auto tile_of = [&](int tile) { return decode_tile<kPair>(*sh, n_groups, tile, uniform_nt, rank); };
 
   if (warp == 0) {
     if (lane == 0) {

@@ -292,7 +292,8 @@ front_kernel(const FrontArgs a) {
     phase_stamp(a.clk, 2, first_cta && tid == 0);
     if (tid == 0) {
       int mt = 0, tiles = 0, rows = 0, topk_rows = 0;
-      long long cost_single = 0, cost_pair = 0;
+      long long cost_single = 0, cost_pair = 0, cost_split = 0;
+      int live_mask = 0, split_mask = 0, n_even = 0, n_odd3 = 0;
       for (int q = 0; q < n_groups; ++q) {
         s_base[q] = mt * kTileM;
         const int m_tiles = (s_total[q] + kTileM - 1) / kTileM;
@@ -311,8 +312,18 @@ front_kernel(const FrontArgs a) {
           // weight set with 64 ... 1024 rows): single CTAs stream at the full rate for one row tile, and from two row
           // tiles on every further tile costs 25 -- each of them fetches the W_enc tile again, from L2; a pair costs 46
           // per 256-row tile whether its second half has rows or not, streaming at a slightly lower rate
-          cost_single += (long long)(m_tiles == 1 ? 40 : 25 * m_tiles) * s_gtiles[q];
-          cost_pair += (long long)(46 * ((m_tiles + 1) / 2)) * s_gtiles[q];
+          const long long cs = (long long)(m_tiles == 1 ? 40 : 25 * m_tiles) * s_gtiles[q];
+          const long long cp = (long long)(46 * ((m_tiles + 1) / 2)) * s_gtiles[q];
+          cost_single += cs;
+          cost_pair += cp;
+          cost_split += min(cs, cp);
+          live_mask |= 1 << q;
+          if (cp < cs) {
+            split_mask |= 1 << q;
+            ++n_even;
+          } else if (m_tiles >= 3) {
+            ++n_odd3;
+          }
         }
       }
       s_base[n_groups] = mt * kTileM;
@@ -332,8 +343,24 @@ front_kernel(const FrontArgs a) {
         a.rs->n_delta_rows = s_total[n_groups];
         // Pairs win where a weight set has an even number of row tiles (two tiles share one fetch of W_enc, and the
         // pair's instruction fills less shared memory per flop) and lose where half of a pair would repeat the other
-        // half's work: one row tile, or three.
-        a.rs->use_pair = a.pair_mode == 2 ? (cost_pair < cost_single) : a.pair_mode;
+        // half's work: one row tile, or three.  Each weight set may go to the form that is cheaper for it -- the two
+        // encode kernels then both work, one after the other, which costs a second ramp-up and drain (about 25 us:
+        // in the units above 25 x 40 / (time to stream one tile of 512 d bytes at 6.3 TB/s) = 1.23e7 / d).
+        // Measured on config 4's replays, the split pays when two or more sets go to the pairs, or when a set of
+        // three or more row tiles stays with the single CTAs; ONE two-tile set among one-tile sets does not: inside
+        // the single-CTA kernel its second fetch of each W_enc tile and its tensor time hide behind the other sets'
+        // streams (1.67 ms all single against 1.71-1.74 ms split for sets of 1, 1, 1, 1, 2 tiles), so such a call
+        // stays with one form.
+        int mask = a.pair_mode == 1 ? live_mask : 0;
+        if (a.pair_mode == 2) {
+          const bool both = split_mask != 0 && split_mask != live_mask;
+          const long long split_total = cost_split + (both ? 12300000ll / max(a.d, 1) : 0ll);
+          const bool split_pays = !both || n_even >= 2 || n_odd3 >= 1;
+          if (split_pays && split_total <= min(cost_single, cost_pair)) mask = split_mask;
+          else mask = cost_pair < cost_single ? live_mask : 0;
+        }
+        a.rs->pair_mask = mask;
+        a.rs->use_pair = mask != 0;
         if (a.n_flagged) *a.n_flagged = 0;       // fallback-selection flags of the fused TopK path start clear every call
         // graph-conditional form: the rest of the SAE chain sits in the body of an IF node that runs only when a row needs it
         if (a.use_cond) cudaGraphSetConditional(a.cond, rows > 0 ? 1u : 0u);

@@ -740,3 +740,55 @@ def test_edit_only_rows_of_different_slots_share_a_cta():
     st = check_parity(W.host(w), out, check_features=False)
     assert st["rows"] == T
     assert (token_slot[:T - 3] <= 5).sum() > 20 and len(set(token_slot[:T - 3].tolist())) >= 6
+
+
+@pytest.mark.parametrize("rows_per_set", [(100, 200, 256, 300), (130, 40, 0, 0), (256, 256, 0, 0), (512, 100, 300, 0),
+                                          (129, 1, 1, 1), (0, 384, 0, 130)])
+def test_weight_sets_dealt_between_single_ctas_and_cta_pairs(rows_per_set):
+    """A context of more than 128 rows has two encode kernels (single CTAs, CTA pairs) and the front kernel deals
+    the call's weight sets between them by their number of 128-row tiles: two sets of two tiles and one of three
+    beside a one-tile set (both kernels work), one two-tile set beside a one-tile set (single CTAs only), two
+    full pairs (pairs only), four tiles + one + three (both), ... -- one captured graph, a new map per replay,
+    every row against the oracle."""
+    mixlib = _mixlib()
+    w = W.make_replay(DEV, d=256, T_max=1024, d_sae=2048, k=16, G=4, n_probe=4, n_steer=2, n_sae_slots=8, n_edit=4)
+    m = W.make_context(mixlib.Mix, w)
+    T, k_max = w.T_max, w.k_max
+    h_static = w.hidden.clone()
+    scores = torch.empty((T, 1), dtype=torch.float32, device=DEV)
+    tk_idx = torch.empty((T, k_max), dtype=torch.int32, device=DEV)
+    tk_val = torch.empty((T, k_max), dtype=torch.float32, device=DEV)
+    n_act = torch.empty((T,), dtype=torch.int32, device=DEV)
+    m.set_feature_out(tk_idx, tk_val, n_act)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        m.apply(h_static, scores, stream=s)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            m.apply(h_static, scores, stream=s)
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    sae_slots = {gi: [sl for sl, a in w.apps.items() if a.kind == W.KIND_SAE and a.group == gi] for gi in range(4)}
+    other = [sl for sl, a in w.apps.items() if a.kind != W.KIND_SAE]
+    token_slot = np.full(T, -1, dtype=np.int32)
+    t = 0
+    for gi, n in enumerate(rows_per_set):                      # the sets' rows interleaved with a few other rows
+        for j in range(n):
+            token_slot[t] = sae_slots[gi][(j // 37) % len(sae_slots[gi])]
+            t += 1
+        token_slot[t:t + 3] = [other[gi % len(other)], -1, other[(gi + 1) % len(other)]]
+        t += 3
+    n_live = t
+    for rep in range(2):                                       # twice: the second replay starts from the first one's state
+        m.set_slot_map(token_slot, n_live)
+        h_static.copy_(w.hidden)
+        scores.copy_(torch.from_numpy(np.full((T, 1), CANARY_F32, dtype=np.uint32).view(np.float32)))
+        tk_idx.fill_(-559038737); n_act.fill_(-559038737)
+        g.replay()
+        torch.cuda.synchronize()
+        w.token_slot, w.T_live = token_slot, n_live
+        out = dict(hidden=W.bits(h_static), scores=scores.cpu().numpy(), topk_idx=tk_idx.cpu().numpy(),
+                   topk_val=tk_val.cpu().numpy(), n_active=n_act.cpu().numpy(), status=m.get_status())
+        check_parity(W.host(w), out)
+    m.destroy()
