@@ -396,10 +396,17 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
       // this warp's columns of the bias (and feature scale) go to shared memory now, while the accumulator is
       // still being computed: read from global memory inside the loop below, 32 columns at a time between
       // tensor-memory loads, they were four exposed round trips per tile
+      // (Not where both operands are 8-bit and the epilogue selects TopK candidates: there the epilogue, not the
+      // main loop, sets the pace -- the accumulator is ready when the warp asks for it -- so a load to wait for in
+      // front of every tile costs more than the loads spread over the loop: config 2 with 8-bit operands 240 us
+      // against 210 us.  Asking one tile ahead, the vectors held in registers meanwhile, was slower still: 256 us.)
       constexpr bool kScaled = kEnc != 0;      // the accumulator is in units of the codes
+      constexpr bool kStageVec = !(kEnc == 2 && kEpi == 8);
       float* wb = epi_vec + (warp - 2) * kEpiCols;
       float* ws = wb + kEpiWarps * kEpiCols;
-      {
+      const float* bias_t = groups[t.group].b_eff + (size_t)t.n_tile * kTileN + c_lo;
+      const float* wsc_t = kScaled ? groups[t.group].w_scale + (size_t)t.n_tile * kTileN + c_lo : nullptr;
+      if (kStageVec) {
         const float* bias_g = groups[t.group].b_eff + (size_t)t.n_tile * kTileN + c_lo;
         const float* wsc_g = kScaled ? groups[t.group].w_scale + (size_t)t.n_tile * kTileN + c_lo : nullptr;
         for (int j = lane * 4; j < kEpiCols; j += 128) {
@@ -430,9 +437,11 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
           tmem_ld32(taddr + c, v);
 #pragma unroll
           for (int i = 0; i < 32; i += 4) {
-            const float4 b4 = *reinterpret_cast<const float4*>(wb + (c - c_lo) + i);
+            const float4 b4 = kStageVec ? *reinterpret_cast<const float4*>(wb + (c - c_lo) + i)
+                                        : __ldg(reinterpret_cast<const float4*>(bias_t + (c - c_lo) + i));
             float4 s4 = make_float4(1.f, 1.f, 1.f, 1.f);
-            if (kScaled) s4 = *reinterpret_cast<const float4*>(ws + (c - c_lo) + i);
+            if (kScaled) s4 = kStageVec ? *reinterpret_cast<const float4*>(ws + (c - c_lo) + i)
+                                        : __ldg(reinterpret_cast<const float4*>(wsc_t + (c - c_lo) + i));
             if (kE4) { s4.x *= ars; s4.y *= ars; s4.z *= ars; s4.w *= ars; }
             v[i] = kScaled ? fmaf(v[i], s4.x, b4.x) : v[i] + b4.x;
             v[i + 1] = kScaled ? fmaf(v[i + 1], s4.y, b4.y) : v[i + 1] + b4.y;
@@ -519,9 +528,11 @@ encode_tc_kernel(const __grid_constant__ CUtensorMap tmap_panel, const CUtensorM
           if (valid) {
 #pragma unroll
             for (int i = 0; i < 32; i += 4) {
-              const float4 b4 = *reinterpret_cast<const float4*>(wb + (c - c_lo) + i);
+              const float4 b4 = kStageVec ? *reinterpret_cast<const float4*>(wb + (c - c_lo) + i)
+                                          : __ldg(reinterpret_cast<const float4*>(bias_t + (c - c_lo) + i));
               float4 s4 = make_float4(1.f, 1.f, 1.f, 1.f);
-              if (kScaled) s4 = *reinterpret_cast<const float4*>(ws + (c - c_lo) + i);
+              if (kScaled) s4 = kStageVec ? *reinterpret_cast<const float4*>(ws + (c - c_lo) + i)
+                                          : __ldg(reinterpret_cast<const float4*>(wsc_t + (c - c_lo) + i));
               if (kE4) { s4.x *= ars; s4.y *= ars; s4.z *= ars; s4.w *= ars; }
               float4 o;
               o.x = kScaled ? fmaf(v[i], s4.x, b4.x) : v[i] + b4.x;
