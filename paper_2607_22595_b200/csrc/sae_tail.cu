@@ -465,11 +465,21 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh, int n_groups) {
   }
   __syncthreads();
   const int n_work = sh.cum[n_groups];
-  for (int w = blockIdx.x; w < n_work; w += gridDim.x) {
+  // A call with few rows leaves most of the grid without work while each row's gather runs with one CTA's worth
+  // of loads in flight (32 KiB, i.e. about 30 GB/s at DRAM latency).  Where the grid has room, 2 or 4 CTAs take a
+  // TopK row together: each repeats the selection for itself -- a few KB of candidates out of L2 -- and gathers
+  // every 2nd or 4th pass of 2048 columns; the first of them writes what exists once per row (read-out, flags).
+  int n_split = 1;
+  if (n_work > 0 && a.mode != kTailFallback) {
+    const int room = (int)gridDim.x / n_work, passes = (nvec + kTailThreads - 1) / kTailThreads;
+    while (n_split < 4 && 2 * n_split <= room && 2 * n_split <= passes) n_split *= 2;
+  }
+  for (int item = blockIdx.x; item < n_work * n_split; item += gridDim.x) {
+    const int w = item / n_split, part = item - w * n_split;
     int g_w = 0;
     while (g_w + 1 < n_groups && w >= sh.cum[g_w + 1]) ++g_w;
     const int p = sh.row0[g_w] + (w - sh.cum[g_w]);
-    const bool stamp = w == 0 && tid == 0 && a.mode != kTailFallback;
+    const bool stamp = item == 0 && tid == 0 && a.mode != kTailFallback;
     phase_stamp(a.clk, 9, stamp);
     const RowRec rec = a.row_rec[p];
     const int t = rec.t;
@@ -479,6 +489,7 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh, int n_groups) {
     const int act = (rec.group_flags >> kRecActShift) & 3;
     const bool add_error = (rec.group_flags & kRecAddError) != 0;
     const bool topk = act == MIX_SAE_TOPK;
+    if (part > 0 && !topk) continue;                   // rows of the other activations are one CTA's
     if (a.mode == kTailFallback && !(topk && a.row_flag[p])) continue;
     if (!topk && add_error && a.out_n_active == nullptr) continue;     // the delta role's row, and nobody wants its active count
     const int slot = rec.slot, n_edit = rec.n_edit;
@@ -546,7 +557,7 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh, int n_groups) {
           flag = __syncthreads_or(ninth_max >= kth) != 0;
         }
         if (flag) {
-          if (tid == 0) {
+          if (tid == 0 && part == 0) {
             a.row_flag[p] = 1;
             a.mtile_flag[p / kTileM] = 1;
             atomicAdd(a.n_flagged, 1);
@@ -562,7 +573,7 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh, int n_groups) {
       } else {
         ZRow src{z, S};
         const int how = radix_collect<true, 11>(src, k, sh.sel);
-        if (how == 2 && tid == 0) atomicOr(a.status, MIX_STATUS_TOPK_GENERAL);
+        if (how == 2 && tid == 0 && part == 0) atomicOr(a.status, MIX_STATUS_TOPK_GENERAL);
         sorted = sort_desc(sh.sel);
         for (int i = tid; i < k; i += kTailThreads) {
           win_id[i] = comp_id(sorted[i]);
@@ -571,7 +582,7 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh, int n_groups) {
       }
       __syncthreads();
       phase_stamp(a.clk, 12, stamp);
-      emit_topk(win_id, win_val, k, a.k_max, t, a.out_idx, a.out_val, a.out_n_active, &sh.sel.count);
+      if (part == 0) emit_topk(win_id, win_val, k, a.k_max, t, a.out_idx, a.out_val, a.out_n_active, &sh.sel.count);
     } else {
       if (a.out_n_active != nullptr) {
         int cnt = 0;
@@ -612,7 +623,7 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh, int n_groups) {
       }
       phase_stamp(a.clk, 13, stamp);
       if (__syncthreads_or(delta != 0.f)) {            // no effective edit: the row stays as it is, bit for bit
-        for (int v = tid; v < nvec; v += kTailThreads) {
+        for (int v = part * kTailThreads + tid; v < nvec; v += n_split * kTailThreads) {
           float acc[8];
           load8(acc, hrow[v]);
           gather_list(acc, sh.coef, sh.feat, n_edit, W_dec, d, v, true);
@@ -640,7 +651,7 @@ __device__ void tail_rows(const TailArgs& a, RowShared& sh, int n_groups) {
         win_id[i] = in_range ? j : 0;
       }
       __syncthreads();
-      for (int v = tid; v < nvec; v += kTailThreads) {
+      for (int v = part * kTailThreads + tid; v < nvec; v += n_split * kTailThreads) {
         float acc[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) acc[i] = b_dec ? b_dec[v * 8 + i] : 0.f;
